@@ -1,0 +1,180 @@
+/*
+ * libsentinel -- the verifier-node check of Sentinel (arXiv 2603.03592) for NVIDIA B200.
+ *
+ * A verifier sits between two pipeline stages and screens every tensor that crosses the
+ * boundary: activations h on the way forward, activation-gradients g on the way back
+ * (Sec. 2.1, Def. 2.1).  For each submitted tensor x it measures the distance to an
+ * exponential moving average m of past clean submissions (Eq. 1, Eq. 2), compares each
+ * distance with adaptive median/IQR bounds (Eq. 3, Alg. 5), reports flags, and moves the
+ * average only when nothing was flagged.  One handle holds the state of one boundary for one
+ * stream of submissions (the per-trainer form of the SWARM appendix: one tensor per update).
+ *
+ * Units.  Every quantity is computed for 1+B "units": row 0 is the whole tensor (the paper's
+ * per-worker test), rows 1..B are the B samples, each tested on its own [T,d] slice against
+ * the same slice of m with a history pooled over samples.
+ *
+ * Metrics (Sec. 3.1), index i:   0  L1    mean over elements of |x - m|
+ *                                1  L2z   mean squared difference of the z-scored x and m
+ *                                         (scalar mean / population std over the unit; a
+ *                                         constant vector z-scores to zero)
+ *                                2  SFR   fraction of elements with sign(x) != sign(m),
+ *                                         sign in {-1,0,+1}
+ *
+ * Conventions.  All tensors are dense, row-major [B,T,d] with d fastest.  x is bf16; the
+ * reference m is fp32 and owned by the library.  Pointers named dev_* are device pointers on
+ * the handle's device, host_* are host pointers.  `cuda_stream` is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  Calls only enqueue work unless stated otherwise;
+ * outputs are valid once the stream reaches that point.  A handle is not thread-safe and its
+ * calls must be stream-ordered; different handles are independent.
+ *
+ * Errors.  Every call returns 0 or a negative sentinel_status; nothing throws or aborts.
+ * Arguments are checked before anything is launched, so an invalid call leaves the state
+ * untouched.  sentinel_last_error() gives a message for the last failure.
+ */
+#ifndef SENTINEL_H
+#define SENTINEL_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SENTINEL_NUM_METRICS 3
+#define SENTINEL_NUM_STATS 8      /* mean_x var_x |x|_2 mean_m var_m cov_xm |m|_2 rho */
+#define SENTINEL_NUM_THRESHOLDS 6 /* q1 q2 q3 k tau_lower tau_upper                   */
+#define SENTINEL_MAX_B 64         /* samples per tensor                               */
+#define SENTINEL_MAX_WINDOW 4096  /* window_steps * B must not exceed this            */
+
+typedef enum sentinel_status {
+  SENTINEL_OK = 0,
+  SENTINEL_ERR_INVALID_ARG = -1,    /* NULL pointer, bad kind, value out of range           */
+  SENTINEL_ERR_SHAPE_MISMATCH = -2, /* B,T,d differ from the handle's                       */
+  SENTINEL_ERR_UNALIGNED = -3,      /* pointer not 16-byte aligned, or d not a multiple of 8 */
+  SENTINEL_ERR_CUDA = -4,           /* a CUDA runtime call failed (see sentinel_last_error)  */
+  SENTINEL_ERR_STATE_SIZE = -5,     /* state buffer too small or of another shape/version    */
+  SENTINEL_ERR_TIMEOUT = -6,        /* reserved: a bounded device-side wait gave up          */
+  SENTINEL_ERR_UNSUPPORTED = -7     /* shape or window beyond the compiled limits            */
+} sentinel_status;
+
+typedef enum sentinel_kind { SENTINEL_ACT = 0, SENTINEL_GRAD = 1 } sentinel_kind;
+
+/* Bits of a flags word.  Rows 0..B carry the per-unit bits; row 0 also carries the status. */
+#define SENTINEL_FLAG_L1 (1u << 0)            /* metric i outside [tau_lower, tau_upper]     */
+#define SENTINEL_FLAG_L2Z (1u << 1)
+#define SENTINEL_FLAG_SFR (1u << 2)
+#define SENTINEL_FLAG_NONFINITE (1u << 7)     /* the unit holds a NaN or an infinity         */
+#define SENTINEL_FLAG_COMMITTED (1u << 16)    /* row 0: the reference was updated            */
+#define SENTINEL_FLAG_SEVERE (1u << 17)       /* row 0: deviation >= severe_mult * allowed   */
+#define SENTINEL_FLAG_BANNED (1u << 18)       /* row 0: sticky until sentinel_reset_worker   */
+#define SENTINEL_FLAG_NO_THRESHOLDS (1u << 19) /* row 0: some history was still empty         */
+
+/* Hyper-parameters.  Arrays are indexed by kind.  Defaults: table "verification_config",
+ * column "8x16 Mesh, 0.6B"; c and T_forgiveness from Sec. 3.1; the window from Sec. 5. */
+typedef struct sentinel_config {
+  double beta[2];          /* EMA decay (Eq. 1), in [0,1)                      0.90  0.80  */
+  double k0[2];            /* initial IQR multiplier (Alg. 5)                  1.5   3.0   */
+  double alpha[2];         /* target false-positive rate                       1e-4  1e-3  */
+  int    n_max[2];         /* max widen / narrow iterations                    10    10    */
+  double gamma_grow[2];    /* widen factor  (> 1)                              1.1   1.01  */
+  double gamma_shrink[2];  /* narrow factor (< 1)                              0.9   0.99  */
+  double lambda_min[2];    /* bounds at least lambda*|median| from the median  0.15  0.05  */
+  double iqr_eps[2];       /* floor of the IQR                                 1e-3  5e-5  */
+  double shrink_ratio;     /* narrow while FP-rate < shrink_ratio*alpha        0.5         */
+  double severe_mult;      /* immediate ban multiple (Sec. 3.1)                100         */
+  int    window_steps;     /* history length l, in steps                       100         */
+  int    ban_violations;   /* c                                                5           */
+  int    forgiveness_steps;/* T_forgiveness                                    100         */
+  unsigned metric_mask;    /* bit i set: metric i may raise a flag             7           */
+  int    B, T, d;          /* shape of every submission; d % 8 == 0, B <= SENTINEL_MAX_B   */
+  int    device;           /* CUDA device ordinal                                           */
+} sentinel_config;
+
+typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundary */
+
+/* Fills *cfg with the defaults above; B = T = d = 0 and device = 0 are left for the caller. */
+int sentinel_default_config(sentinel_config *cfg);
+
+/* Allocates the state of one boundary on cfg->device: two fp32 [B,T,d] buffers per kind (the
+ * reference and its candidate; m_0 = 0 as in Alg. 1), the history windows, thresholds and
+ * counters.  Synchronous.  The library owns this memory until sentinel_destroy. */
+int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out);
+
+/* Verified step: the body of Alg. 2 (kind = ACT) / Alg. 3 (kind = GRAD) for one submission.
+ *   Gamma_i = Omega_i(x, m_{t-1}) for every unit (Eq. 2); a unit is flagged when an enabled
+ *   metric lies outside the bounds left by the previous step (Eq. 3, Alg. 5); any flag is one
+ *   violation (counter, forgiveness, ban: Sec. 3.1); unflagged units join the history and the
+ *   bounds are refreshed; m_t = beta m_{t-1} + (1-beta) x only if nothing was flagged.
+ * dev_x          bf16 [B,T,d], 16-byte aligned, read once.
+ * dev_scores_out fp32 [(1+B)*3], scores_out[row*3+i] = Gamma_i of that unit (NaN for a
+ *                non-finite unit).
+ * dev_flags_out  u32 [1+B], bits as defined above.
+ * x is read exactly once; the library keeps no reference to caller memory afterwards. */
+int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T,
+                    int d, void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out);
+
+/* Warm-up step (the warm-up loop of Alg. 1, honest workers only): scores as above, every unit
+ * joins the history, the bounds are refreshed and the reference is updated unconditionally.
+ * No flags, no counters.  A non-finite x changes nothing.  dev_scores_out may be NULL. */
+int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B,
+                              int T, int d, void *cuda_stream, float *dev_scores_out);
+
+/* sentinel_verify for callers whose tensor and results live in host memory: copies x to a
+ * staging buffer owned by the handle (allocated on first use), runs the check, copies scores
+ * and flags back and waits for the stream.  host_x: bf16 [B,T,d] (pinned memory copies
+ * fastest); host_scores_out: fp32 [(1+B)*3]; host_flags_out: u32 [1+B]. */
+int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind kind, int B,
+                         int T, int d, void *cuda_stream, float *host_scores_out,
+                         unsigned *host_flags_out);
+
+/* Stateless form of Eq. 2 / Sec. 3.1: the three distances and the statistics of x against a
+ * reference supplied by the caller.  dev_m: fp32 [B,T,d], 16-byte aligned.  dev_scores_out
+ * fp32 [(1+B)*3]; dev_stats_out fp32 [(1+B)*8] or NULL.  Needs a few KiB of scratch, which it
+ * takes from and returns to the stream's memory pool (cudaMallocAsync). */
+int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d, int device,
+                      void *cuda_stream, float *dev_scores_out, float *dev_stats_out);
+
+/* Statistics of the last call of this kind, fp32 [(1+B)*8] per unit:
+ * mean_x, var_x, ||x||_2, mean_m, var_m, cov(x,m), ||m||_2, Pearson rho.  Enqueues a copy. */
+int sentinel_get_stats(sentinel_verifier *h, sentinel_kind kind, float *dev_stats_out,
+                       void *cuda_stream);
+
+/* Current bounds, host_out double [2 levels][3 metrics][6] = q1 q2 q3 k tau_lower tau_upper
+ * (level 0 = whole tensor, 1 = samples); host_valid int [2][3] (0 while that history is
+ * empty), may be NULL.  Waits for the stream. */
+int sentinel_get_thresholds(sentinel_verifier *h, sentinel_kind kind, double *host_out,
+                            int *host_valid, void *cuda_stream);
+
+/* host_out int64 [6]: violations v, clean streak, banned, steps(ACT), steps(GRAD), the error
+ * word written by device code (0 = none).  Waits for the stream. */
+int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_stream);
+
+/* Per-token partial sums of the pass, written by every later call while registered:
+ * dev_buf fp32 [B,T,4] = sum_c x, sum_c x^2, sum_c |x-m|, count of sign mismatches over the
+ * token's d channels.  NULL unregisters.  The buffer stays the caller's. */
+int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf);
+
+/* A new worker now feeds this boundary: clears the violation counter, the clean streak and
+ * the ban (the paper keeps these per worker).  Enqueued on cuda_stream. */
+int sentinel_reset_worker(sentinel_verifier *h, void *cuda_stream);
+
+/* Checkpointing.  The state is one self-describing blob: a 64-byte header
+ * {u64 magic, u32 version, i32 B, T, d, window_steps, violations, clean_streak, banned},
+ * then per kind {i64 steps; i32 count[2]; i32 valid[2][3]; f64 thr[2][3][6];
+ * f64 history[level 0: 3][window_steps], [level 1: 3][window_steps*B] (oldest first,
+ * zero-padded); f32 m[B*T*d]}.  Export and import wait for the stream. */
+size_t sentinel_state_bytes(const sentinel_verifier *h);
+int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *cuda_stream);
+int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, void *cuda_stream);
+
+/* Message of the last failure on this handle (h == NULL: of the calling thread's last failed
+ * call that had no handle).  The string is owned by the library. */
+const char *sentinel_last_error(const sentinel_verifier *h);
+
+/* Frees everything the handle owns.  Waits for the device to finish the handle's work. */
+int sentinel_destroy(sentinel_verifier *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SENTINEL_H */

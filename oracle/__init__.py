@@ -1,0 +1,283 @@
+"""Reference oracle for the Sentinel verifier check -- TEST INFRASTRUCTURE ONLY.
+
+A thin ctypes wrapper around ``sentinel_oracle.c`` (plain C, float64), which restates the
+paper's definitions: the distance measures of Sec. 3.1, the EMA of Eq. (1), the per-submission
+body of Alg. 2 / Alg. 3, the warm-up loop of Alg. 1 and the adaptive IQR thresholds of Alg. 5.
+
+Only the test-suite, the smoke check and the benchmark's CPU-baseline leg may import this
+package.  It shares no code with the CUDA library and does not import it.
+
+Parity unpinned (conventions the paper leaves open, each a parameter): the reading of
+"FP-rate << alpha" (``shrink_ratio``), the severe-deviation multiple (``severe_mult``), the
+forgiveness bookkeeping, and the percentile interpolation rule.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sentinel_oracle.c")
+_HDR = os.path.join(_HERE, "sentinel_oracle.h")
+_LIB = os.path.join(_HERE, "libsentinel_oracle.so")
+
+ACT, GRAD = 0, 1
+L1, L2Z, SFR = 0, 1, 2
+NMETRIC, NSTAT, NTHR = 3, 8, 6
+
+FLAG_L1, FLAG_L2Z, FLAG_SFR = 1 << 0, 1 << 1, 1 << 2
+FLAG_NONFINITE = 1 << 7
+FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
+METRIC_BITS = FLAG_L1 | FLAG_L2Z | FLAG_SFR
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no CUDA involved); returns the library path."""
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-Wall", "-Wextra",
+             "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Params(C.Structure):
+    _fields_ = [
+        ("beta", C.c_double * 2), ("k0", C.c_double * 2), ("alpha", C.c_double * 2),
+        ("n_max", C.c_int * 2), ("gamma_g", C.c_double * 2), ("gamma_s", C.c_double * 2),
+        ("lam", C.c_double * 2), ("eps", C.c_double * 2),
+        ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
+        ("l", C.c_int), ("c", C.c_int), ("t_forgiveness", C.c_int),
+        ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
+    ]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        dp, u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint16)
+        L.so_default_params.argtypes = [C.POINTER(_Params)]
+        L.so_default_params.restype = None
+        L.so_bf16.argtypes = [C.c_uint16]
+        L.so_bf16.restype = C.c_double
+        L.so_distance.argtypes = [u16p, dp, C.c_size_t, dp, dp]
+        L.so_distance.restype = C.c_int
+        L.so_percentile.argtypes = [dp, C.c_size_t, C.c_double]
+        L.so_percentile.restype = C.c_double
+        L.so_adaptive_iqr.argtypes = [dp, C.c_size_t, C.c_double, C.c_int, C.c_double,
+                                      C.c_double, C.c_double, C.c_double, C.c_double, dp,
+                                      C.POINTER(C.c_int)]
+        L.so_adaptive_iqr.restype = C.c_int
+        L.so_create.argtypes = [C.POINTER(_Params)]
+        L.so_create.restype = C.c_void_p
+        L.so_destroy.argtypes = [C.c_void_p]
+        L.so_destroy.restype = None
+        L.so_update_reference.argtypes = [C.c_void_p, u16p, C.c_int, dp]
+        L.so_update_reference.restype = C.c_int
+        L.so_verify.argtypes = [C.c_void_p, u16p, C.c_int, dp, C.POINTER(C.c_uint32)]
+        L.so_verify.restype = C.c_int
+        L.so_reset_worker.argtypes = [C.c_void_p]
+        L.so_reset_worker.restype = None
+        L.so_ema.argtypes = [C.c_void_p, C.c_int]
+        L.so_ema.restype = dp
+        L.so_set_ema.argtypes = [C.c_void_p, C.c_int, dp]
+        L.so_set_ema.restype = None
+        L.so_history.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, dp, C.c_size_t]
+        L.so_history.restype = C.c_size_t
+        L.so_thresholds.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, dp]
+        L.so_thresholds.restype = C.c_int
+        L.so_last_stats.argtypes = [C.c_void_p, C.c_int, dp]
+        L.so_last_stats.restype = None
+        L.so_counters.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
+        L.so_counters.restype = None
+        L.so_steps.argtypes = [C.c_void_p, C.c_int]
+        L.so_steps.restype = C.c_long
+        _lib = L
+    return _lib
+
+
+def _dptr(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_double))
+
+
+def _bits(x) -> np.ndarray:
+    """bf16 bit patterns as a contiguous uint16 array (accepts uint16/int16 arrays)."""
+    a = np.ascontiguousarray(x)
+    if a.dtype == np.int16:
+        a = a.view(np.uint16)
+    if a.dtype != np.uint16:
+        raise TypeError("bf16 input must be given as uint16 bit patterns")
+    return a
+
+
+def _u16ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_uint16))
+
+
+def bf16_to_f64(bits) -> np.ndarray:
+    """bf16 bit patterns -> float64 values (exact)."""
+    b = _bits(bits)
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+@dataclass
+class Params:
+    """Hyper-parameters (index 0 = activations, 1 = gradients); defaults from the paper."""
+    B: int = 1
+    T: int = 1
+    d: int = 8
+    beta: tuple = (0.90, 0.80)
+    k0: tuple = (1.5, 3.0)
+    alpha: tuple = (1e-4, 1e-3)
+    n_max: tuple = (10, 10)
+    gamma_g: tuple = (1.1, 1.01)
+    gamma_s: tuple = (0.9, 0.99)
+    lam: tuple = (0.15, 0.05)
+    eps: tuple = (1e-3, 5e-5)
+    shrink_ratio: float = 0.5
+    severe_mult: float = 100.0
+    l: int = 100
+    c: int = 5
+    t_forgiveness: int = 100
+    metric_mask: int = 7
+
+    def to_c(self) -> _Params:
+        p = _Params()
+        for name in ("beta", "k0", "alpha", "gamma_g", "gamma_s", "lam", "eps"):
+            arr = getattr(p, name)
+            arr[0], arr[1] = getattr(self, name)
+        p.n_max[0], p.n_max[1] = self.n_max
+        p.shrink_ratio, p.severe_mult = self.shrink_ratio, self.severe_mult
+        p.l, p.c, p.t_forgiveness = self.l, self.c, self.t_forgiveness
+        p.metric_mask = self.metric_mask
+        p.B, p.T, p.d = self.B, self.T, self.d
+        return p
+
+
+def default_params_from_c() -> dict:
+    p = _Params()
+    lib().so_default_params(C.byref(p))
+    out = {}
+    for name, _ in _Params._fields_:
+        v = getattr(p, name)
+        out[name] = tuple(v) if hasattr(v, "__len__") else v
+    return out
+
+
+def distance(x_bits, m) -> tuple[np.ndarray, np.ndarray, bool]:
+    """Omega_i(x, m) of one unit: (gamma[3], stat[8], nonfinite)."""
+    xb = _bits(x_bits).reshape(-1)
+    mm = np.ascontiguousarray(m, dtype=np.float64).reshape(-1)
+    assert xb.size == mm.size and xb.size > 0
+    g = np.empty(NMETRIC)
+    s = np.empty(NSTAT)
+    nf = lib().so_distance(_u16ptr(xb), _dptr(mm), xb.size, _dptr(g), _dptr(s))
+    return g, s, bool(nf)
+
+
+def percentile(sorted_vals, p: float) -> float:
+    a = np.ascontiguousarray(sorted_vals, dtype=np.float64)
+    return float(lib().so_percentile(_dptr(a), a.size, p))
+
+
+def adaptive_iqr(window, k_prev, alpha, n_max, gamma_g, gamma_s, lam, eps, shrink_ratio=0.5):
+    """Alg. 5 on one window.  Returns (thr[6] or None, (grow_iters, shrink_iters))."""
+    w = np.ascontiguousarray(window, dtype=np.float64)
+    thr = np.zeros(NTHR)
+    thr[3] = k_prev
+    it = (C.c_int * 2)()
+    ok = lib().so_adaptive_iqr(_dptr(w), w.size, alpha, n_max, gamma_g, gamma_s, lam, eps,
+                               shrink_ratio, _dptr(thr), it)
+    return (thr if ok else None), (it[0], it[1])
+
+
+class Verifier:
+    """State of one stage boundary: EMAs, histories, thresholds, counters."""
+
+    def __init__(self, params: Params):
+        self.params = params
+        self._h = lib().so_create(C.byref(params.to_c()))
+        if not self._h:
+            raise ValueError("invalid oracle parameters")
+        self.B, self.T, self.d = params.B, params.T, params.d
+        self.rows = 1 + params.B
+        self.N = params.B * params.T * params.d
+
+    def close(self):
+        if self._h:
+            lib().so_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def update_reference(self, x_bits, kind: int):
+        xb = _bits(x_bits).reshape(-1)
+        assert xb.size == self.N
+        scores = np.empty((self.rows, NMETRIC))
+        bad = lib().so_update_reference(self._h, _u16ptr(xb), kind, _dptr(scores))
+        return scores, bool(bad)
+
+    def verify(self, x_bits, kind: int):
+        xb = _bits(x_bits).reshape(-1)
+        assert xb.size == self.N
+        scores = np.empty((self.rows, NMETRIC))
+        flags = np.zeros(self.rows, dtype=np.uint32)
+        commit = lib().so_verify(self._h, _u16ptr(xb), kind, _dptr(scores),
+                                 flags.ctypes.data_as(C.POINTER(C.c_uint32)))
+        return scores, flags, bool(commit)
+
+    def reset_worker(self):
+        lib().so_reset_worker(self._h)
+
+    def ema(self, kind: int) -> np.ndarray:
+        p = lib().so_ema(self._h, kind)
+        return np.ctypeslib.as_array(p, shape=(self.N,)).copy().reshape(self.B, self.T, self.d)
+
+    def set_ema(self, kind: int, m):
+        mm = np.ascontiguousarray(m, dtype=np.float64).reshape(-1)
+        assert mm.size == self.N
+        lib().so_set_ema(self._h, kind, _dptr(mm))
+
+    def history(self, kind: int, level: int, metric: int) -> np.ndarray:
+        cap = self.params.l * (self.B if level else 1)
+        out = np.empty(cap)
+        n = lib().so_history(self._h, kind, level, metric, _dptr(out), cap)
+        return out[:n].copy()
+
+    def thresholds(self, kind: int):
+        """(thr[2][3][6], valid[2][3]) -- q1 q2 q3 k tau_lower tau_upper."""
+        thr = np.zeros((2, NMETRIC, NTHR))
+        valid = np.zeros((2, NMETRIC), dtype=bool)
+        for L in range(2):
+            for i in range(NMETRIC):
+                t = np.zeros(NTHR)
+                valid[L, i] = bool(lib().so_thresholds(self._h, kind, L, i, _dptr(t)))
+                thr[L, i] = t
+        return thr, valid
+
+    def last_stats(self, kind: int) -> np.ndarray:
+        s = np.empty((self.rows, NSTAT))
+        lib().so_last_stats(self._h, kind, _dptr(s))
+        return s
+
+    def counters(self) -> tuple[int, int, int]:
+        out = (C.c_int * 3)()
+        lib().so_counters(self._h, out)
+        return out[0], out[1], out[2]
+
+    def steps(self, kind: int) -> int:
+        return int(lib().so_steps(self._h, kind))

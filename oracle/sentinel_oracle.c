@@ -1,0 +1,399 @@
+/*
+ * Reference oracle for the Sentinel verifier check (arXiv 2603.03592) -- TEST INFRASTRUCTURE.
+ * See sentinel_oracle.h.  Plain C, float64, one explicit loop per definition.
+ */
+#include "sentinel_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------------------ */
+/* element helpers                                                                       */
+
+double so_bf16(uint16_t bits) {
+  uint32_t u = (uint32_t)bits << 16; /* bf16 is the upper half of an IEEE binary32 */
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/* three-valued sign: -1, 0, +1 (both zeros give 0) */
+static int sign3(double v) { return (v > 0.0) - (v < 0.0); }
+
+void so_default_params(so_params *p) {
+  memset(p, 0, sizeof *p);
+  /* Tab. "verification_config", column "8x16 Mesh, 0.6B": activation | gradient */
+  p->beta[0] = 0.90;     p->beta[1] = 0.80;
+  p->k0[0] = 1.5;        p->k0[1] = 3.0;
+  p->alpha[0] = 1e-4;    p->alpha[1] = 1e-3;
+  p->n_max[0] = 10;      p->n_max[1] = 10;
+  p->gamma_g[0] = 1.1;   p->gamma_g[1] = 1.01;
+  p->gamma_s[0] = 0.9;   p->gamma_s[1] = 0.99;
+  p->lambda[0] = 0.15;   p->lambda[1] = 0.05;
+  p->eps[0] = 1e-3;      p->eps[1] = 5e-5;
+  p->shrink_ratio = 0.5;
+  p->severe_mult = 100.0;        /* Sec. 3.1, "Violation Counter with Forgiveness" */
+  p->l = 100;                    /* Sec. 5: window of the past 100 steps            */
+  p->c = 5;                      /* Sec. 3.1                                        */
+  p->t_forgiveness = 100;        /* Sec. 3.1                                        */
+  p->metric_mask = 7u;
+  p->B = 1; p->T = 1; p->d = 8;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Sec. 3.1: the distance measures Omega_i(x, m) of one unit                             */
+
+int so_distance(const uint16_t *x, const double *m, size_t n, double gamma[3], double stat[8]) {
+  size_t e;
+  const double dn = (double)n;
+
+  for (e = 0; e < n; ++e) {
+    if (!isfinite(so_bf16(x[e]))) {
+      int i;
+      for (i = 0; i < SO_NMETRIC; ++i) gamma[i] = NAN;
+      for (i = 0; i < SO_NSTAT; ++i) stat[i] = NAN;
+      return 1;
+    }
+  }
+
+  /* Mean absolute difference: the average over all features of |x_e - m_e|. */
+  double abs_sum = 0.0;
+  for (e = 0; e < n; ++e) abs_sum += fabs(so_bf16(x[e]) - m[e]);
+  gamma[SO_L1] = abs_sum / dn;
+
+  /* Normalised Euclidean distance: z-score x and m (scalar mean and population standard
+   * deviation over all elements of the unit), then average the squared difference.  A vector
+   * whose elements are all equal has standard deviation 0 and z-scores to the zero vector. */
+  double sum_x = 0.0, sum_m = 0.0;
+  double min_x = so_bf16(x[0]), max_x = min_x, min_m = m[0], max_m = min_m;
+  for (e = 0; e < n; ++e) {
+    const double xe = so_bf16(x[e]), me = m[e];
+    sum_x += xe; sum_m += me;
+    if (xe < min_x) min_x = xe;
+    if (xe > max_x) max_x = xe;
+    if (me < min_m) min_m = me;
+    if (me > max_m) max_m = me;
+  }
+  const double mu_x = sum_x / dn, mu_m = sum_m / dn;
+  double ss_x = 0.0, ss_m = 0.0, ss_xm = 0.0, sq_x = 0.0, sq_m = 0.0;
+  for (e = 0; e < n; ++e) {
+    const double xe = so_bf16(x[e]), me = m[e];
+    ss_x += (xe - mu_x) * (xe - mu_x);
+    ss_m += (me - mu_m) * (me - mu_m);
+    ss_xm += (xe - mu_x) * (me - mu_m);
+    sq_x += xe * xe;
+    sq_m += me * me;
+  }
+  const double var_x = (min_x == max_x) ? 0.0 : ss_x / dn;
+  const double var_m = (min_m == max_m) ? 0.0 : ss_m / dn;
+  const double sd_x = sqrt(var_x), sd_m = sqrt(var_m);
+  double z_sum = 0.0;
+  for (e = 0; e < n; ++e) {
+    const double zx = (sd_x > 0.0) ? (so_bf16(x[e]) - mu_x) / sd_x : 0.0;
+    const double zm = (sd_m > 0.0) ? (m[e] - mu_m) / sd_m : 0.0;
+    z_sum += (zx - zm) * (zx - zm);
+  }
+  gamma[SO_L2Z] = z_sum / dn;
+
+  /* Sign flip ratio: the fraction of coordinates whose signs differ. */
+  size_t flips = 0;
+  for (e = 0; e < n; ++e) flips += (sign3(so_bf16(x[e])) != sign3(m[e]));
+  gamma[SO_SFR] = (double)flips / dn;
+
+  stat[0] = mu_x; stat[1] = var_x; stat[2] = sqrt(sq_x);
+  stat[3] = mu_m; stat[4] = var_m; stat[5] = ss_xm / dn; stat[6] = sqrt(sq_m);
+  stat[7] = (sd_x > 0.0 && sd_m > 0.0) ? (ss_xm / dn) / (sd_x * sd_m) : 0.0;
+  return 0;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Alg. 5: adaptive IQR thresholds                                                       */
+
+double so_percentile(const double *sorted, size_t n, double p) {
+  const double pos = p * (double)(n - 1);
+  const size_t lo = (size_t)floor(pos);
+  const size_t hi = (lo + 1 < n) ? lo + 1 : lo;
+  const double frac = pos - (double)lo;
+  return sorted[lo] + frac * (sorted[hi] - sorted[lo]);
+}
+
+static int cmp_double(const void *a, const void *b) {
+  const double x = *(const double *)a, y = *(const double *)b;
+  return (x > y) - (x < y);
+}
+
+/* fraction of the window strictly outside the closed interval [lo, hi] */
+static double fp_rate(const double *w, size_t n, double lo, double hi) {
+  size_t out = 0, j;
+  for (j = 0; j < n; ++j) out += (w[j] < lo || w[j] > hi);
+  return (double)out / (double)n;
+}
+
+int so_adaptive_iqr(const double *window, size_t n, double alpha, int n_max, double gamma_g,
+                    double gamma_s, double lambda, double eps, double shrink_ratio,
+                    double thr[6], int iters[2]) {
+  if (iters) { iters[0] = 0; iters[1] = 0; }
+  if (n == 0) return 0;
+
+  double *sorted = (double *)malloc(n * sizeof(double));
+  memcpy(sorted, window, n * sizeof(double));
+  qsort(sorted, n, sizeof(double), cmp_double);
+  const double q1 = so_percentile(sorted, n, 0.25);
+  const double q2 = so_percentile(sorted, n, 0.50);
+  const double q3 = so_percentile(sorted, n, 0.75);
+  free(sorted);
+
+  const double iqr = fmax(q3 - q1, eps);
+  double k = thr[3]; /* the multiplier persists from call to call */
+  double tau_lower = q2 - k * iqr;
+  double tau_upper = q2 + k * iqr;
+  double fp = fp_rate(window, n, tau_lower, tau_upper);
+
+  int it = 0;
+  while (fp > alpha && it < n_max) { /* widen */
+    k = k * gamma_g;
+    tau_lower = q2 - k * iqr;
+    tau_upper = q2 + k * iqr;
+    fp = fp_rate(window, n, tau_lower, tau_upper);
+    ++it;
+  }
+  if (iters) iters[0] = it;
+
+  it = 0;
+  while (fp < shrink_ratio * alpha && it < n_max) { /* narrow */
+    k = k * gamma_s;
+    tau_lower = q2 - k * iqr;
+    tau_upper = q2 + k * iqr;
+    fp = fp_rate(window, n, tau_lower, tau_upper);
+    ++it;
+  }
+  if (iters) iters[1] = it;
+
+  const double d_min = fabs(q2) * lambda; /* minimum distance from the median */
+  tau_lower = fmin(tau_lower, q2 - d_min);
+  tau_upper = fmax(tau_upper, q2 + d_min);
+
+  thr[0] = q1; thr[1] = q2; thr[2] = q3; thr[3] = k; thr[4] = tau_lower; thr[5] = tau_upper;
+  return 1;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* verifier state                                                                        */
+
+typedef struct so_window {      /* one history list, oldest first */
+  double *v;
+  size_t n, cap;
+} so_window;
+
+typedef struct so_kind_state {
+  double *m;                                  /* EMA reference, B*T*d, starts at zero */
+  so_window hist[2][SO_NMETRIC];              /* [level][metric]                      */
+  double thr[2][SO_NMETRIC][SO_NTHR];
+  int has_thr[2][SO_NMETRIC];
+  double *stats;                              /* (1+B)*8 of the last call             */
+  long steps;
+} so_kind_state;
+
+struct so_verifier {
+  so_params p;
+  size_t N, Ns;
+  so_kind_state ks[2];
+  int violations, clean_streak, banned;
+};
+
+static void window_push(so_window *w, double val) {
+  if (w->n == w->cap) { /* truncate to the last `cap` entries: the oldest leaves */
+    memmove(w->v, w->v + 1, (w->cap - 1) * sizeof(double));
+    w->n = w->cap - 1;
+  }
+  w->v[w->n++] = val;
+}
+
+so_verifier *so_create(const so_params *p) {
+  if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1) return NULL;
+  so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
+  v->p = *p;
+  v->Ns = (size_t)p->T * (size_t)p->d;
+  v->N = v->Ns * (size_t)p->B;
+  for (int kind = 0; kind < 2; ++kind) {
+    so_kind_state *ks = &v->ks[kind];
+    ks->m = (double *)calloc(v->N, sizeof(double));
+    ks->stats = (double *)calloc((size_t)(1 + p->B) * SO_NSTAT, sizeof(double));
+    for (int L = 0; L < 2; ++L)
+      for (int i = 0; i < SO_NMETRIC; ++i) {
+        so_window *w = &ks->hist[L][i];
+        w->cap = (L == 0) ? (size_t)p->l : (size_t)p->l * (size_t)p->B;
+        w->v = (double *)calloc(w->cap, sizeof(double));
+        w->n = 0;
+        ks->thr[L][i][3] = p->k0[kind];
+        ks->has_thr[L][i] = 0;
+      }
+  }
+  return v;
+}
+
+void so_destroy(so_verifier *v) {
+  if (!v) return;
+  for (int kind = 0; kind < 2; ++kind) {
+    free(v->ks[kind].m);
+    free(v->ks[kind].stats);
+    for (int L = 0; L < 2; ++L)
+      for (int i = 0; i < SO_NMETRIC; ++i) free(v->ks[kind].hist[L][i].v);
+  }
+  free(v);
+}
+
+/* scores and statistics of every unit against the current EMA: row 0 = the whole tensor,
+ * row 1+b = sample b.  Returns a bit per row set when that row holds non-finite input. */
+static void all_units(so_verifier *v, const uint16_t *x, int kind, double *gam, int *nonfinite) {
+  so_kind_state *ks = &v->ks[kind];
+  nonfinite[0] = so_distance(x, ks->m, v->N, gam, ks->stats);
+  for (int b = 0; b < v->p.B; ++b)
+    nonfinite[1 + b] = so_distance(x + (size_t)b * v->Ns, ks->m + (size_t)b * v->Ns, v->Ns,
+                                   gam + (size_t)(1 + b) * SO_NMETRIC,
+                                   ks->stats + (size_t)(1 + b) * SO_NSTAT);
+}
+
+static void refresh_thresholds(so_verifier *v, int kind) {
+  so_kind_state *ks = &v->ks[kind];
+  const so_params *p = &v->p;
+  for (int L = 0; L < 2; ++L)
+    for (int i = 0; i < SO_NMETRIC; ++i) {
+      so_window *w = &ks->hist[L][i];
+      if (so_adaptive_iqr(w->v, w->n, p->alpha[kind], p->n_max[kind], p->gamma_g[kind],
+                          p->gamma_s[kind], p->lambda[kind], p->eps[kind], p->shrink_ratio,
+                          ks->thr[L][i], NULL))
+        ks->has_thr[L][i] = 1;
+    }
+}
+
+/* Eq. (1) with one submission per update (the per-trainer form of the SWARM appendix). */
+static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
+  double *m = v->ks[kind].m;
+  const double beta = v->p.beta[kind];
+  for (size_t e = 0; e < v->N; ++e) m[e] = beta * m[e] + (1.0 - beta) * so_bf16(x[e]);
+}
+
+int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *scores) {
+  const int rows = 1 + v->p.B;
+  so_kind_state *ks = &v->ks[kind];
+  double *gam = (double *)malloc((size_t)rows * SO_NMETRIC * sizeof(double));
+  int *nf = (int *)malloc((size_t)rows * sizeof(int));
+  all_units(v, x, kind, gam, nf);
+  if (scores) memcpy(scores, gam, (size_t)rows * SO_NMETRIC * sizeof(double));
+  ks->steps += 1;
+  const int bad = nf[0];
+  if (!bad) {
+    /* warm-up: every deviation joins the history, then thresholds, then the EMA */
+    for (int i = 0; i < SO_NMETRIC; ++i) window_push(&ks->hist[0][i], gam[i]);
+    for (int b = 0; b < v->p.B; ++b)
+      for (int i = 0; i < SO_NMETRIC; ++i)
+        window_push(&ks->hist[1][i], gam[(size_t)(1 + b) * SO_NMETRIC + i]);
+    refresh_thresholds(v, kind);
+    ema_update(v, x, kind);
+  }
+  free(gam); free(nf);
+  return bad;
+}
+
+int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint32_t *flags) {
+  const so_params *p = &v->p;
+  const int rows = 1 + p->B;
+  so_kind_state *ks = &v->ks[kind];
+  double *gam = (double *)malloc((size_t)rows * SO_NMETRIC * sizeof(double));
+  int *nf = (int *)malloc((size_t)rows * sizeof(int));
+
+  /* 1. Gamma_i = Omega_i(x_t, m_{t-1}) for every unit */
+  all_units(v, x, kind, gam, nf);
+  memcpy(scores, gam, (size_t)rows * SO_NMETRIC * sizeof(double));
+  ks->steps += 1;
+
+  /* 2. Tukey test against the thresholds left by the previous step */
+  int any_flag = 0, severe = 0, no_thr = 0;
+  for (int r = 0; r < rows; ++r) {
+    const int L = (r == 0) ? 0 : 1;
+    uint32_t f = 0;
+    if (nf[r]) {
+      f |= SO_FLAG_NONFINITE;
+    } else {
+      for (int i = 0; i < SO_NMETRIC; ++i) {
+        if (!ks->has_thr[L][i]) { no_thr = 1; continue; }
+        if (!((p->metric_mask >> i) & 1u)) continue;
+        const double *t = ks->thr[L][i];
+        const double g = gam[(size_t)r * SO_NMETRIC + i];
+        if (g < t[4] || g > t[5]) f |= (1u << i);
+        /* 3. severe deviation, tested on the whole-tensor unit */
+        if (r == 0 && fabs(g - t[1]) >= p->severe_mult * (t[5] - t[1])) severe = 1;
+      }
+    }
+    flags[r] = f;
+    if (f) any_flag = 1;
+  }
+
+  /* 4. violation counter with forgiveness */
+  if (any_flag) {
+    v->violations += 1;
+    v->clean_streak = 0;
+    if (v->violations >= p->c || severe) v->banned = 1;
+  } else {
+    v->clean_streak += 1;
+    if (v->clean_streak >= p->t_forgiveness) {
+      v->violations = (v->violations > 0) ? v->violations - 1 : 0;
+      v->clean_streak = 0;
+    }
+  }
+
+  /* 5. clean units join the history; thresholds are refreshed for the next step */
+  for (int r = 0; r < rows; ++r) {
+    if (flags[r]) continue;
+    const int L = (r == 0) ? 0 : 1;
+    for (int i = 0; i < SO_NMETRIC; ++i)
+      window_push(&ks->hist[L][i], gam[(size_t)r * SO_NMETRIC + i]);
+  }
+  refresh_thresholds(v, kind);
+
+  /* 6. the EMA moves only when nothing was flagged */
+  const int commit = !any_flag;
+  if (commit) ema_update(v, x, kind);
+
+  if (commit) flags[0] |= SO_FLAG_COMMITTED;
+  if (severe) flags[0] |= SO_FLAG_SEVERE;
+  if (v->banned) flags[0] |= SO_FLAG_BANNED;
+  if (no_thr) flags[0] |= SO_FLAG_NO_THRESHOLDS;
+  free(gam); free(nf);
+  return commit;
+}
+
+void so_reset_worker(so_verifier *v) { v->violations = 0; v->clean_streak = 0; v->banned = 0; }
+
+/* ------------------------------------------------------------------------------------ */
+/* accessors                                                                             */
+
+const double *so_ema(const so_verifier *v, int kind) { return v->ks[kind].m; }
+
+void so_set_ema(so_verifier *v, int kind, const double *m) {
+  memcpy(v->ks[kind].m, m, v->N * sizeof(double));
+}
+
+size_t so_history(const so_verifier *v, int kind, int level, int metric, double *out, size_t cap) {
+  const so_window *w = &v->ks[kind].hist[level][metric];
+  const size_t n = (w->n < cap) ? w->n : cap;
+  if (out) memcpy(out, w->v, n * sizeof(double));
+  return w->n;
+}
+
+int so_thresholds(const so_verifier *v, int kind, int level, int metric, double thr[6]) {
+  memcpy(thr, v->ks[kind].thr[level][metric], SO_NTHR * sizeof(double));
+  return v->ks[kind].has_thr[level][metric];
+}
+
+void so_last_stats(const so_verifier *v, int kind, double *stats) {
+  memcpy(stats, v->ks[kind].stats, (size_t)(1 + v->p.B) * SO_NSTAT * sizeof(double));
+}
+
+void so_counters(const so_verifier *v, int out[3]) {
+  out[0] = v->violations; out[1] = v->clean_streak; out[2] = v->banned;
+}
+
+long so_steps(const so_verifier *v, int kind) { return v->ks[kind].steps; }

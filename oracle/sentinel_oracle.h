@@ -1,0 +1,117 @@
+/*
+ * Reference oracle for the Sentinel verifier check (arXiv 2603.03592).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, float64 CPU restatement of what the
+ * paper defines: the distance measures of Sec. 3.1, the EMA reference of Eq. (1) in its
+ * one-submission-per-update (SWARM trainer) form, the per-submission body of Alg. 2 / Alg. 3,
+ * the warm-up body of Alg. 1 and the adaptive IQR thresholds of Alg. 5.  It exists so that
+ * tests can check the CUDA library against it and so that the benchmark can time it as a
+ * reported CPU baseline.  It shares no code with the CUDA library and must never be linked,
+ * imported or called from the product path.
+ *
+ * Every metric is written from its definition (two passes for the z-scores, an explicit
+ * loop per element); nothing is blocked, fused or reordered.
+ *
+ * Parity unpinned (the paper gives no value to pin these conventions to; each is a
+ * parameter so that a later correction is one constant):
+ *   - the meaning of "FP-rate << alpha" in Alg. 5 (read as FP-rate < shrink_ratio * alpha),
+ *   - the "x100 above the threshold" severe-deviation rule of Sec. 3.1,
+ *   - the forgiveness bookkeeping ("decrements after T_forgiveness consecutive clean steps"),
+ *   - the percentile convention (linear interpolation at p*(n-1)).
+ */
+#ifndef SENTINEL_ORACLE_H
+#define SENTINEL_ORACLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { SO_ACT = 0, SO_GRAD = 1 };                 /* h (forward) or g (backward)           */
+enum { SO_L1 = 0, SO_L2Z = 1, SO_SFR = 2, SO_NMETRIC = 3 };
+enum { SO_NSTAT = 8 };                            /* mean_x var_x |x|_2 mean_m var_m cov |m|_2 rho */
+enum { SO_NTHR = 6 };                             /* q1 q2 q3 k tau_lower tau_upper        */
+
+/* report bits, one word per unit (row 0 = whole tensor, rows 1..B = samples) */
+enum {
+  SO_FLAG_L1 = 1u << 0, SO_FLAG_L2Z = 1u << 1, SO_FLAG_SFR = 1u << 2,
+  SO_FLAG_NONFINITE = 1u << 7,
+  SO_FLAG_COMMITTED = 1u << 16, SO_FLAG_SEVERE = 1u << 17,
+  SO_FLAG_BANNED = 1u << 18, SO_FLAG_NO_THRESHOLDS = 1u << 19
+};
+
+/* Hyper-parameters; index 0 = activations, 1 = gradients (Tab. "verification_config"). */
+typedef struct so_params {
+  double beta[2];          /* EMA decay, Eq. (1)                                   */
+  double k0[2];            /* initial IQR multiplier, Alg. 5                        */
+  double alpha[2];         /* target false-positive rate, Alg. 5                    */
+  int    n_max[2];         /* max grow / shrink iterations, Alg. 5                  */
+  double gamma_g[2];       /* grow factor  > 1                                      */
+  double gamma_s[2];       /* shrink factor < 1                                     */
+  double lambda[2];        /* minimum-distance multiplier                           */
+  double eps[2];           /* IQR floor                                             */
+  double shrink_ratio;     /* "FP-rate << alpha"  :=  FP-rate < shrink_ratio*alpha  */
+  double severe_mult;      /* immediate ban when deviation >= severe_mult * allowed */
+  int    l;                /* history window, in steps                              */
+  int    c;                /* violations before a ban                               */
+  int    t_forgiveness;    /* clean steps before the counter decrements             */
+  unsigned metric_mask;    /* which metrics may raise a flag (bit i = metric i)     */
+  int    B, T, d;          /* submission shape                                      */
+} so_params;
+
+typedef struct so_verifier so_verifier;
+
+/* Defaults: the "8x16 mesh, 0.6B" column of the hyper-parameter table; c, T_forgiveness
+ * from Sec. 3.1; l from Sec. 5. */
+void so_default_params(so_params *p);
+
+/* bf16 bit pattern -> double, exactly. */
+double so_bf16(uint16_t bits);
+
+/* Sec. 3.1 distance measures of one unit: n elements of x (bf16 bits) against n reference
+ * values m.  gamma[3] = {L1, normalised L2, SFR}; stat[8] as listed above.  Returns 1 when x
+ * holds a NaN or an infinity (then every output is NaN), else 0. */
+int so_distance(const uint16_t *x, const double *m, size_t n, double gamma[3], double stat[8]);
+
+/* Percentile of an ascending array by linear interpolation at position p*(n-1), p in [0,1]. */
+double so_percentile(const double *sorted, size_t n, double p);
+
+/* Alg. 5 for one (kind, level, metric) window.  thr[SO_NTHR] holds q1 q2 q3 k tau_lower
+ * tau_upper; on entry thr[3] is the multiplier carried over from the previous call (k0 the
+ * first time).  An empty window leaves thr untouched and returns 0; otherwise returns 1.
+ * iters[2], if not NULL, receives the number of grow and shrink iterations taken. */
+int so_adaptive_iqr(const double *window, size_t n, double alpha, int n_max, double gamma_g,
+                    double gamma_s, double lambda, double eps, double shrink_ratio,
+                    double thr[6], int iters[2]);
+
+so_verifier *so_create(const so_params *p);
+void so_destroy(so_verifier *v);
+
+/* Warm-up step (Alg. 1, warm-up loop): scores against the current EMA, every unit appended
+ * to the history, thresholds refreshed, EMA updated.  scores: (1+B)*3 doubles or NULL.
+ * Returns 0, or 1 if the input was non-finite (then nothing changes). */
+int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *scores);
+
+/* Verified step (body of Alg. 2 / Alg. 3 for one submission).  scores: (1+B)*3 doubles,
+ * flags: (1+B) words.  Returns 1 if the EMA was updated (no unit flagged), else 0. */
+int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint32_t *flags);
+
+/* A new worker now feeds this boundary: clear its violation counter, streak and ban. */
+void so_reset_worker(so_verifier *v);
+
+/* State access for tests. */
+const double *so_ema(const so_verifier *v, int kind);                 /* B*T*d values      */
+void   so_set_ema(so_verifier *v, int kind, const double *m);
+size_t so_history(const so_verifier *v, int kind, int level, int metric,
+                  double *out, size_t cap);                            /* oldest first      */
+int    so_thresholds(const so_verifier *v, int kind, int level, int metric, double thr[6]);
+void   so_last_stats(const so_verifier *v, int kind, double *stats);  /* (1+B)*8           */
+void   so_counters(const so_verifier *v, int out[3]);                 /* v, streak, banned */
+long   so_steps(const so_verifier *v, int kind);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,252 @@
+"""Pins for the oracle's stateful part: Eq. (1), the warm-up loop of Alg. 1, the per-submission
+body of Alg. 2 / Alg. 3 and the violation counter of Sec. 3.1.  Expected values are closed
+forms, hand-scripted sequences, or library routines applied to the recorded history."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_03592_b200 import synth
+from test_oracle_pins import from_bits, to_bits
+
+ACT, GRAD = 0, 1
+
+
+def make(oracle_mod, B=2, T=4, d=8, **kw):
+    return oracle_mod.Verifier(oracle_mod.Params(B=B, T=T, d=d, **kw))
+
+
+def test_ema_closed_form_for_identical_inputs(oracle_mod):
+    """m_0 = 0 and t identical submissions x give m_t = (1 - beta^t) x (Eq. 1)."""
+    rs = np.random.default_rng(1)
+    v = make(oracle_mod)
+    xb = to_bits(rs.normal(0, 1, (2, 4, 8)))
+    x = from_bits(xb)
+    assert np.all(v.ema(ACT) == 0.0)
+    for t in range(1, 8):
+        v.update_reference(xb, ACT)
+        v.update_reference(xb, GRAD)
+        assert v.ema(ACT) == pytest.approx((1 - 0.9 ** t) * x, rel=1e-13)
+        assert v.ema(GRAD) == pytest.approx((1 - 0.8 ** t) * x, rel=1e-13)
+
+
+def test_ema_is_the_weighted_sum_of_past_inputs(oracle_mod):
+    rs = np.random.default_rng(2)
+    v = make(oracle_mod, beta=(0.5, 0.25))
+    xs = [to_bits(rs.normal(0, 1, (2, 4, 8))) for _ in range(5)]
+    for xb in xs:
+        v.update_reference(xb, GRAD)
+    want = sum(0.75 * 0.25 ** (4 - i) * from_bits(xb) for i, xb in enumerate(xs))
+    assert v.ema(GRAD) == pytest.approx(want, rel=1e-13, abs=1e-16)
+    assert np.all(v.ema(ACT) == 0.0)                  # the two kinds have separate references
+
+
+def test_beta_zero_keeps_the_last_submission(oracle_mod):
+    rs = np.random.default_rng(3)
+    v = make(oracle_mod, beta=(0.0, 0.0))
+    for _ in range(3):
+        xb = to_bits(rs.normal(0, 1, (2, 4, 8)))
+        v.update_reference(xb, ACT)
+        assert np.array_equal(v.ema(ACT), from_bits(xb))
+
+
+def test_first_warmup_step_scores_against_the_zero_reference(oracle_mod):
+    """m_0 = 0: L1 = mean|x|, L2 = 1 (z-score of a constant is zero), SFR = fraction non-zero."""
+    rs = np.random.default_rng(4)
+    v = make(oracle_mod)
+    x = from_bits(to_bits(rs.normal(0, 1, (2, 4, 8))))
+    x[0, 0, :3] = 0.0
+    scores, bad = v.update_reference(to_bits(x), ACT)
+    assert not bad
+    units = [x] + [x[b] for b in range(2)]
+    for r, u in enumerate(units):
+        assert scores[r, 0] == pytest.approx(np.mean(np.abs(u)), rel=1e-13)
+        assert scores[r, 1] == pytest.approx(1.0, rel=1e-12)
+        assert scores[r, 2] == np.count_nonzero(u) / u.size
+    # scores of a step are measured against the reference *before* that step's update
+    scores2, _ = v.update_reference(to_bits(x), ACT)
+    assert scores2[0, 0] == pytest.approx(np.mean(np.abs(x - 0.1 * x)), rel=1e-12)
+    assert scores2[0, 2] == 0.0
+
+
+def test_tensor_level_is_the_mean_of_equal_sized_samples(oracle_mod):
+    rs = np.random.default_rng(5)
+    v = make(oracle_mod, B=4, T=8, d=16)
+    v.update_reference(to_bits(rs.normal(0, 1, (4, 8, 16))), ACT)
+    scores, _ = v.update_reference(to_bits(rs.normal(0, 1, (4, 8, 16))), ACT)
+    assert scores[0, 0] == pytest.approx(scores[1:, 0].mean(), rel=1e-13)
+    assert scores[0, 2] == pytest.approx(scores[1:, 2].mean(), rel=1e-13)
+    s = v.last_stats(ACT)
+    assert s[0, 0] == pytest.approx(s[1:, 0].mean(), rel=1e-12, abs=1e-16)
+    assert s[0, 2] ** 2 == pytest.approx(np.sum(s[1:, 2] ** 2), rel=1e-13)
+
+
+def test_warmup_history_and_thresholds(oracle_mod):
+    """Every warm-up deviation joins the window (oldest leaves after l entries per unit) and the
+    stored thresholds are Alg. 5 applied to that window with the multiplier carried over."""
+    rs = np.random.default_rng(6)
+    B, l = 3, 5
+    v = make(oracle_mod, B=B, T=4, d=8, l=l)
+    rec = [[], []]
+    k = [[1.5] * 3, [1.5] * 3]
+    for t in range(9):
+        scores, _ = v.update_reference(to_bits(rs.normal(0, 1, (B, 4, 8))), ACT)
+        rec[0].append(scores[0])
+        rec[1].extend(scores[1:])
+        thr, valid = v.thresholds(ACT)
+        assert valid.all()
+        for L, cap in ((0, l), (1, l * B)):
+            for i in range(3):
+                want_hist = np.array(rec[L])[-cap:, i]
+                assert np.array_equal(v.history(ACT, L, i), want_hist)
+                want, _ = oracle_mod.adaptive_iqr(want_hist, k[L][i], 1e-4, 10, 1.1, 0.9, 0.15, 1e-3)
+                assert np.array_equal(thr[L, i], want)
+                q = np.percentile(want_hist, [25, 50, 75])
+                assert thr[L, i, :3] == pytest.approx(q, rel=1e-13)
+                k[L][i] = want[3]
+    tg, vg = v.thresholds(GRAD)
+    assert not vg.any() and np.all(tg[:, :, 3] == 3.0)     # untouched kind keeps k0
+
+
+def _warm(oracle_mod, w, n, **kw):
+    v = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, **kw))
+    for t in range(n):
+        for kind in (ACT, GRAD):
+            v.update_reference(synth.bits(synth.clean(w, 0, kind, t)), kind)
+    return v
+
+
+@pytest.fixture(scope="module")
+def small():
+    return synth.scaled(synth.WORKLOADS["cfg1"], "cfg1_small", 8, 32, 128)
+
+
+def test_clean_stream_raises_no_flags(oracle_mod, small):
+    v = _warm(oracle_mod, small, 16)
+    for t in range(16, 56):
+        for kind in (ACT, GRAD):
+            scores, flags, commit = v.verify(synth.bits(synth.clean(small, 0, kind, t)), kind)
+            assert commit
+            assert np.all((flags & 0xFFFF) == 0)
+            assert flags[0] == oracle_mod.FLAG_COMMITTED
+    assert v.counters() == (0, 40 * 2, 0)
+
+
+def test_scaled_sample_is_flagged_and_reference_is_kept(oracle_mod, small):
+    """Config-1 scenario: sample 3 multiplied by 10 after 16 clean warm-up microbatches."""
+    v = _warm(oracle_mod, small, 16)
+    clean = synth.clean(small, 0, ACT, 16)
+    bad = synth.corrupt(small, clean, "scale_sample3", 0, ACT, 16)
+    m_before = v.ema(ACT)
+    hist_before = [v.history(ACT, L, 0).size for L in (0, 1)]
+    clean_scores, _ = oracle_mod.distance(synth.bits(clean)[3], m_before[3])[:2]
+    scores, flags, commit = v.verify(synth.bits(bad), ACT)
+    assert not commit and not (flags[0] & oracle_mod.FLAG_COMMITTED)
+    assert flags[4] & oracle_mod.FLAG_L1                      # row 1+3
+    assert scores[4, 0] > 5 * clean_scores[0]                 # L1 grows about tenfold
+    others = [r for r in range(1, 9) if r != 4]
+    assert np.all(flags[others] == 0)
+    assert np.array_equal(v.ema(ACT), m_before)               # flagged => EMA not updated
+    # flagged units stay out of the history, clean samples still join it
+    n_flagged = int(np.count_nonzero(flags[1:] & 0xFFFF))
+    assert v.history(ACT, 1, 0).size == min(hist_before[1] + 8 - n_flagged, 100 * 8)
+    level0_flagged = bool(flags[0] & 0xFFFF)
+    assert v.history(ACT, 0, 0).size == hist_before[0] + (0 if level0_flagged else 1)
+    assert v.counters()[0] == 1
+
+
+def test_gradient_sign_flip_is_statistically_invisible(oracle_mod, small):
+    """The paper's tables show a 0% detection of gradients multiplied by -1: against an EMA of
+    independent zero-mean gradients, -g has the same three scores up to sampling noise."""
+    v = _warm(oracle_mod, small, 16)
+    g = synth.clean(small, 0, GRAD, 16)
+    m = v.ema(GRAD)
+    a, _, _ = oracle_mod.distance(synth.bits(g), m)
+    b, _, _ = oracle_mod.distance(synth.bits(-g), m)
+    assert b == pytest.approx(a, rel=0.02)
+    _, flags, commit = v.verify(synth.bits(-g), GRAD)
+    assert commit and np.all((flags & 0xFFFF) == 0)
+
+
+def test_violation_counter_ban_and_forgiveness(oracle_mod, small):
+    v = _warm(oracle_mod, small, 16, c=3, t_forgiveness=4)
+    step = [16]
+
+    def send(corrupt):
+        x = synth.clean(small, 0, ACT, step[0])
+        if corrupt:
+            x = (x.float() * 3.0).to(torch.bfloat16)         # mild: caught, far from severe
+        step[0] += 1
+        return v.verify(synth.bits(x), ACT)
+
+    _, f, c = send(True)
+    assert not c and v.counters() == (1, 0, 0) and not (f[0] & oracle_mod.FLAG_SEVERE)
+    for i in range(3):
+        _, f, c = send(False)
+        assert c and v.counters() == (1, i + 1, 0)
+    send(False)                                               # 4th clean step: forgiven
+    assert v.counters() == (0, 0, 0)
+    for i in range(4):
+        send(False)
+    assert v.counters() == (0, 0, 0)                          # never below zero
+    send(True); send(False); send(True)
+    assert v.counters() == (2, 0, 0)                          # a clean step does not reset v
+    _, f, _ = send(True)
+    assert v.counters() == (3, 0, 1) and (f[0] & oracle_mod.FLAG_BANNED)
+    _, f, c = send(False)
+    assert c and (f[0] & oracle_mod.FLAG_BANNED)              # the ban is sticky ...
+    v.reset_worker()
+    _, f, _ = send(False)
+    assert not (f[0] & oracle_mod.FLAG_BANNED) and v.counters() == (0, 1, 0)   # ... until reset
+
+
+def test_severe_deviation_bans_at_once(oracle_mod, small):
+    v = _warm(oracle_mod, small, 16)
+    x = (synth.clean(small, 0, ACT, 16).float() * 4096.0).to(torch.bfloat16)
+    thr, _ = v.thresholds(ACT)
+    scores, flags, commit = v.verify(synth.bits(x), ACT)
+    assert abs(scores[0, 0] - thr[0, 0, 1]) >= 100 * (thr[0, 0, 5] - thr[0, 0, 1])
+    assert (flags[0] & oracle_mod.FLAG_SEVERE) and (flags[0] & oracle_mod.FLAG_BANNED)
+    assert v.counters() == (1, 0, 1)
+
+
+def test_verify_without_warmup_flags_nothing(oracle_mod):
+    rs = np.random.default_rng(8)
+    v = make(oracle_mod)
+    xb = to_bits(rs.normal(0, 1, (2, 4, 8)))
+    scores, flags, commit = v.verify(xb, ACT)
+    assert commit
+    assert flags[0] == (oracle_mod.FLAG_COMMITTED | oracle_mod.FLAG_NO_THRESHOLDS)
+    assert np.all(flags[1:] == 0)
+    assert v.history(ACT, 0, 0).size == 1 and v.history(ACT, 1, 0).size == 2
+    assert v.ema(ACT) == pytest.approx(0.1 * from_bits(xb), rel=1e-13)
+    _, flags, _ = v.verify(xb, ACT)
+    assert not (flags[0] & oracle_mod.FLAG_NO_THRESHOLDS)
+
+
+def test_non_finite_submission_is_a_violation_and_changes_nothing(oracle_mod, small):
+    v = _warm(oracle_mod, small, 4)
+    x = synth.clean(small, 0, ACT, 4).float()
+    x[2, 1, 5] = float("nan")
+    m0, h0 = v.ema(ACT), v.history(ACT, 1, 0).size
+    scores, flags, commit = v.verify(synth.bits(x.to(torch.bfloat16)), ACT)
+    assert not commit
+    assert flags[0] & oracle_mod.FLAG_NONFINITE and flags[3] & oracle_mod.FLAG_NONFINITE
+    assert np.all(np.isnan(scores[0])) and np.all(np.isnan(scores[3]))
+    assert np.all(np.isfinite(scores[[1, 2, 4, 5, 6, 7, 8]]))
+    assert np.array_equal(v.ema(ACT), m0)
+    assert v.history(ACT, 1, 0).size == h0 + 7 and v.counters()[0] == 1
+    # warm-up refuses it outright
+    s, bad = v.update_reference(synth.bits(x.to(torch.bfloat16)), ACT)
+    assert bad and np.array_equal(v.ema(ACT), m0) and v.history(ACT, 1, 0).size == h0 + 7
+
+
+def test_metric_mask_limits_which_metrics_may_flag(oracle_mod, small):
+    x = (synth.clean(small, 0, ACT, 16).float() * 3.0).to(torch.bfloat16)
+    v = _warm(oracle_mod, small, 16)
+    _, f_all, _ = v.verify(synth.bits(x), ACT)
+    assert f_all[0] & oracle_mod.FLAG_L1
+    v = _warm(oracle_mod, small, 16, metric_mask=0b110)       # L1 switched off
+    scores, f, commit = v.verify(synth.bits(x), ACT)
+    assert not np.any(f & oracle_mod.FLAG_L1)
+    # scaling by 3 leaves the z-scored distance and the signs alone, so nothing else fires
+    assert commit and np.all((f & 0xFFFF) == 0)
