@@ -1,0 +1,314 @@
+#!/usr/bin/env python
+"""Benchmark of the Sentinel verifier check on B200.
+
+One *step* is one microbatch crossing a stage boundary: ``sentinel_verify`` on the activation
+tensor h (forward) and on the activation-gradient tensor g (backward), i.e. two launches of
+the streaming kernel, each of which reads x (bf16) and the reference m (fp32) once and writes
+the EMA candidate once: 10 bytes per element.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+Prints ONE JSON line.  ``value`` is verified GB/s (10 B/element moved, all ranks) with inputs
+resident in HBM; ``e2e`` is the same metric through ``sentinel_verify_host`` with pinned host
+buffers (H2D of x and D2H of scores/flags inside the timed region).  With N > 1 (torchrun)
+every rank runs an independent replica of the workload on its own GPU: the check has no
+cross-GPU data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_03592_b200 import replicas, synth  # noqa: E402
+
+ACT, GRAD = 0, 1
+BYTES_PER_ELEMENT = 10          # 2 (x, bf16 read) + 4 (m read) + 4 (EMA candidate write)
+MAX_DISTINCT = 24               # distinct input tensors per kind kept resident
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *exc):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()          # the exact process started above
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self) -> dict:
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            tok = [t.strip() for t in line.split(",")]
+            if len(tok) < 6:
+                continue
+            try:
+                sm.append(float(tok[0]))
+                smax.append(float(tok[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, tok[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_stream(w, device, count):
+    """`count` microbatches per kind after the warm-up, following the workload's recipe."""
+    xs = {ACT: [], GRAD: []}
+    n = min(count, MAX_DISTINCT)
+    for kind in (ACT, GRAD):
+        for i in range(n):
+            x, _ = synth.microbatch(w, 0, kind, w.warmup + i, device)
+            xs[kind].append(x)
+    return xs
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2603_03592_b200 import binding
+    binding.lib()                                   # no library, no benchmark: there is no fallback
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    w = synth.WORKLOADS[args.workload]
+    N = w.B * w.T * w.d
+    v = binding.Verifier(w.B, w.T, w.d, device=local_rank)
+    stream = torch.cuda.current_stream()
+
+    # reference warm-up on clean traffic (untimed set-up, as the method prescribes)
+    for t in range(w.warmup):
+        for kind in (ACT, GRAD):
+            v.sentinel_update_reference(synth.clean(w, 0, kind, t, device), kind)
+    torch.cuda.synchronize()
+
+    total = args.warmup + args.steps
+    xs = build_stream(w, device, total)
+    nd = len(xs[ACT])
+    scores = torch.empty(2, 1 + w.B, 3, dtype=torch.float32, device=device)
+    flags = torch.empty(2, 1 + w.B, dtype=torch.int32, device=device)
+
+    def step(i):
+        v.sentinel_verify(xs[ACT][i % nd], ACT, scores[0], flags[0], stream)
+        v.sentinel_verify(xs[GRAD][i % nd], GRAD, scores[1], flags[1], stream)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    torch.cuda.synchronize()
+
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    with ClockSampler(local_rank) as clocks:
+        marks[0].record(stream)
+        for i in range(args.steps):
+            step(args.warmup + i)
+            marks[i + 1].record(stream)
+        torch.cuda.synchronize()
+    replicas.barrier()
+    torch.cuda.synchronize()
+    local_ms = elapsed_ms = marks[0].elapsed_time(marks[-1])
+    step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms)
+    launches = 2 * args.steps
+    counters = v.sentinel_get_counters()
+
+    # end to end through the host-buffer entry point
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    hx = {k: [xs[k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 4))] for k in (ACT, GRAD)}
+    hs = torch.empty(2, 1 + w.B, 3, dtype=torch.float32).pin_memory()
+    hf = torch.empty(2, 1 + w.B, dtype=torch.int32).pin_memory()
+    v.sentinel_verify_host(hx[ACT][0], ACT, hs[0], hf[0], stream)        # allocates the staging
+    torch.cuda.synchronize()
+    replicas.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        v.sentinel_verify_host(hx[ACT][i % len(hx[ACT])], ACT, hs[0], hf[0], stream)
+        v.sentinel_verify_host(hx[GRAD][i % len(hx[GRAD])], GRAD, hs[1], hf[1], stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1))
+    v.sentinel_destroy()
+
+    bytes_step = 2 * N * BYTES_PER_ELEMENT                  # two tensors per step
+    gbs = world * args.steps * bytes_step / (elapsed_ms * 1e-3) / 1e9
+    e2e_gbs = world * e2e_steps * bytes_step / (e2e_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak_gbs()
+    kernel_ms = local_ms / launches              # the timed region holds these launches only
+    achieved = N * BYTES_PER_ELEMENT / (kernel_ms * 1e-3) / 1e9
+    out = {
+        "metric": "verified GB/s (x bf16 read + reference fp32 read + EMA fp32 write = 10 B/element)",
+        "value": round(gbs, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(elapsed_ms / args.steps, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "impl": "sentinel_b200",
+        "config": {"workload": "%s: B=%d x T=%d x d=%d bf16, activations %s, gradients N(0,%g), "
+                               "%g%% corrupted" % (w.name, w.B, w.T, w.d, w.act, w.grad_std, 100 * w.corrupt_rate),
+                   "step": "sentinel_verify(h, ACT) + sentinel_verify(g, GRAD)",
+                   "l2": "inputs larger than L2: %d MiB read+written per launch, %d distinct tensors per kind"
+                         % (N * BYTES_PER_ELEMENT >> 20, nd),
+                   "replicas": world},
+        "microbatches_per_s": round(world * args.steps / (elapsed_ms * 1e-3), 1),
+        "tensor_gbs": round(world * args.steps * 2 * N * 2 / (elapsed_ms * 1e-3) / 1e9, 1),
+        "ms_per_step_median": round(step_ms[len(step_ms) // 2], 4),
+        "frac_of_8000_nominal": round(gbs / world / 8000.0, 4),
+        "gpu_launches": launches,
+        "violations_seen": int(counters["violations"]),
+        "clocks": clocks.summary(),
+        "e2e": {"value": round(e2e_gbs, 2), "unit": "GB/s", "steps": e2e_steps,
+                "h2d_bytes_per_step": 2 * N * 2,
+                "d2h_bytes_per_step": 2 * (1 + w.B) * (3 * 4 + 4),
+                "api": "sentinel_verify_host"},
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "peak_source": "%s copy bandwidth" % peak_kind,
+                     "kernel": "stream_kernel", "avg_launch_ms": round(kernel_ms, 4),
+                     "traffic": args.traffic},
+    }
+    if rank == 0 and args.cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
+    return out
+
+
+def oracle_sample_shape(w, rows):
+    """A bounded slice of the workload for the CPU oracle: one sample, `rows` token rows."""
+    return synth.scaled(w, w.name + "_cpu_sample", 1, min(rows, w.T), w.d)
+
+
+def cpu_baseline(w, budget_s):
+    """The float64 oracle, as it stands, timed on this host on a bounded sample."""
+    import oracle
+    ws = oracle_sample_shape(w, 8192)
+    n = ws.B * ws.T * ws.d
+    v = oracle.Verifier(oracle.Params(B=ws.B, T=ws.T, d=ws.d))
+    for kind in (ACT, GRAD):
+        v.update_reference(synth.bits(synth.clean(ws, 0, kind, 0)), kind)
+    done, t_total = 0, 0.0
+    while t_total < budget_s and done < 8:
+        xa = synth.bits(synth.clean(ws, 0, ACT, 1 + done))
+        xg = synth.bits(synth.clean(ws, 0, GRAD, 1 + done))
+        t0 = time.perf_counter()
+        v.verify(xa, ACT)
+        v.verify(xg, GRAD)
+        t_total += time.perf_counter() - t0
+        done += 1
+    v.close()
+    return {"value": round(done * 2 * n * BYTES_PER_ELEMENT / t_total / 1e9, 4), "unit": "GB/s",
+            "cores": 1, "kind": "oracle",
+            "host_cores_available": len(os.sched_getaffinity(0)),
+            "sample": "%d steps (h and g) of one sample [1,%d,%d] of the workload, float64, single thread"
+                      % (done, ws.T, ws.d),
+            "ms_per_step": round(1e3 * t_total / done, 1)}
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the CPU oracle on the same workload's shape, each step a bounded sample."""
+    if rank != 0:
+        return None
+    import oracle
+    w = synth.WORKLOADS[args.workload]
+    ws = oracle_sample_shape(w, 1024)
+    n = ws.B * ws.T * ws.d
+    v = oracle.Verifier(oracle.Params(B=ws.B, T=ws.T, d=ws.d))
+    for t in range(2):
+        for kind in (ACT, GRAD):
+            v.update_reference(synth.bits(synth.clean(ws, 0, kind, t)), kind)
+    xs = [(synth.bits(synth.clean(ws, 0, ACT, 2 + i)), synth.bits(synth.clean(ws, 0, GRAD, 2 + i)))
+          for i in range(min(args.warmup + args.steps, 8))]
+    for i in range(args.warmup):
+        v.verify(xs[i % len(xs)][0], ACT)
+        v.verify(xs[i % len(xs)][1], GRAD)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        xa, xg = xs[(args.warmup + i) % len(xs)]
+        v.verify(xa, ACT)
+        v.verify(xg, GRAD)
+    dt = time.perf_counter() - t0
+    v.close()
+    gbs = args.steps * 2 * n * BYTES_PER_ELEMENT / dt / 1e9
+    sample = "each step: h and g of one sample slice [1,%d,%d] of %s, float64, single thread" % (ws.T, ws.d, w.name)
+    return {
+        "metric": "verified GB/s (x bf16 read + reference fp32 read + EMA fp32 write = 10 B/element)",
+        "value": round(gbs, 4), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(1e3 * dt / args.steps, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "impl": "reference",
+        "config": {"workload": "%s: B=%d x T=%d x d=%d bf16" % (w.name, w.B, w.T, w.d), "sample": sample},
+        "cpu_baseline": {"value": round(gbs, 4), "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(gbs, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="ncu DRAM bytes per launch of the current kernel, if known")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":        # rank 0 alone works; no process group is needed
+        rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+        out = run_reference(args, rank, world)
+    else:
+        rank, world, local_rank = replicas.init_from_env(backend="nccl")
+        out = run_ours(args, rank, world, local_rank)
+        replicas.shutdown()
+    if rank == 0 and out is not None:
+        print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,232 @@
+"""ctypes binding of ``libsentinel.so`` -- the same names as ``include/sentinel.h``.
+
+Argument marshalling only: every step of the check runs in the library's CUDA kernels.  Torch
+is used for device memory and streams; tensors are passed as raw pointers.  There is no CPU
+fallback: if the library is missing or cannot be loaded, importing ``lib()`` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import _build
+
+ACT, GRAD = 0, 1
+NUM_METRICS, NUM_STATS, NUM_THRESHOLDS = 3, 8, 6
+MAX_B, MAX_WINDOW = 64, 4096
+
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE_MISMATCH, ERR_UNALIGNED, ERR_CUDA = -1, -2, -3, -4
+ERR_STATE_SIZE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -7
+
+FLAG_L1, FLAG_L2Z, FLAG_SFR = 1 << 0, 1 << 1, 1 << 2
+FLAG_NONFINITE = 1 << 7
+FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
+
+EXPORTS = (
+    "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
+    "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
+    "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
+    "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
+    "sentinel_export_state", "sentinel_import_state", "sentinel_last_error", "sentinel_destroy",
+)
+
+
+class sentinel_config(C.Structure):
+    _fields_ = [
+        ("beta", C.c_double * 2), ("k0", C.c_double * 2), ("alpha", C.c_double * 2),
+        ("n_max", C.c_int * 2), ("gamma_grow", C.c_double * 2), ("gamma_shrink", C.c_double * 2),
+        ("lambda_min", C.c_double * 2), ("iqr_eps", C.c_double * 2),
+        ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
+        ("window_steps", C.c_int), ("ban_violations", C.c_int), ("forgiveness_steps", C.c_int),
+        ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
+        ("device", C.c_int),
+    ]
+
+
+class SentinelError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__("sentinel error %d: %s" % (code, message))
+        self.code = code
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise ImportError(
+                "libsentinel.so is missing at %s: build it with "
+                "`python -m paper_2603_03592_b200._build` (needs nvcc)" % path)
+        L = C.CDLL(path)
+        vp, ip = C.c_void_p, C.c_int
+        L.sentinel_default_config.argtypes = [C.POINTER(sentinel_config)]
+        L.sentinel_verifier_create.argtypes = [C.POINTER(sentinel_config), C.POINTER(vp)]
+        L.sentinel_verify.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_update_reference.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp]
+        L.sentinel_verify_host.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_distance.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_get_stats.argtypes = [vp, ip, vp, vp]
+        L.sentinel_get_thresholds.argtypes = [vp, ip, vp, vp, vp]
+        L.sentinel_get_counters.argtypes = [vp, vp, vp]
+        L.sentinel_set_token_stats_buffer.argtypes = [vp, vp]
+        L.sentinel_reset_worker.argtypes = [vp, vp]
+        L.sentinel_state_bytes.argtypes = [vp]
+        L.sentinel_state_bytes.restype = C.c_size_t
+        L.sentinel_export_state.argtypes = [vp, vp, C.c_size_t, vp]
+        L.sentinel_import_state.argtypes = [vp, vp, C.c_size_t, vp]
+        L.sentinel_last_error.argtypes = [vp]
+        L.sentinel_last_error.restype = C.c_char_p
+        L.sentinel_destroy.argtypes = [vp]
+        for name in EXPORTS:
+            if name not in ("sentinel_state_bytes", "sentinel_last_error"):
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, handle=None):
+    if code != OK:
+        msg = lib().sentinel_last_error(handle)
+        raise SentinelError(code, msg.decode() if msg else "")
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def sentinel_default_config(**overrides) -> sentinel_config:
+    cfg = sentinel_config()
+    _check(lib().sentinel_default_config(C.byref(cfg)))
+    for k, v in overrides.items():
+        cur = getattr(cfg, k)
+        if hasattr(cur, "__len__"):
+            cur[0], cur[1] = v
+        else:
+            setattr(cfg, k, v)
+    return cfg
+
+
+def sentinel_distance(x: torch.Tensor, m: torch.Tensor, scores_out: torch.Tensor,
+                      stats_out: torch.Tensor | None = None, stream=None) -> None:
+    """Stateless Omega_i(x, m) for every unit; outputs are device tensors."""
+    B, T, d = x.shape
+    _check(lib().sentinel_distance(_ptr(x), _ptr(m), B, T, d, x.device.index or 0,
+                                   _stream_ptr(stream), _ptr(scores_out), _ptr(stats_out)))
+
+
+class Verifier:
+    """One stage boundary (a ``sentinel_verifier`` handle).  Methods mirror the C entry points."""
+
+    def __init__(self, B: int, T: int, d: int, device: int = 0, **overrides):
+        self.cfg = sentinel_default_config(B=B, T=T, d=d, device=device, **overrides)
+        self.B, self.T, self.d = B, T, d
+        self.rows = 1 + B
+        self.device = torch.device("cuda", device)
+        h = C.c_void_p()
+        _check(lib().sentinel_verifier_create(C.byref(self.cfg), C.byref(h)))
+        self._h = h
+
+    # -- hot path ---------------------------------------------------------------------------
+    def sentinel_verify(self, x: torch.Tensor, kind: int, scores_out: torch.Tensor,
+                        flags_out: torch.Tensor, stream=None) -> None:
+        B, T, d = x.shape
+        _check(lib().sentinel_verify(self._h, _ptr(x), kind, B, T, d, _stream_ptr(stream),
+                                     _ptr(scores_out), _ptr(flags_out)), self._h)
+
+    def sentinel_update_reference(self, x: torch.Tensor, kind: int,
+                                  scores_out: torch.Tensor | None = None, stream=None) -> None:
+        B, T, d = x.shape
+        _check(lib().sentinel_update_reference(self._h, _ptr(x), kind, B, T, d,
+                                               _stream_ptr(stream), _ptr(scores_out)), self._h)
+
+    def sentinel_verify_host(self, x_host: torch.Tensor, kind: int, scores_host: torch.Tensor,
+                             flags_host: torch.Tensor, stream=None) -> None:
+        B, T, d = x_host.shape
+        _check(lib().sentinel_verify_host(self._h, _ptr(x_host), kind, B, T, d,
+                                          _stream_ptr(stream), _ptr(scores_host),
+                                          _ptr(flags_host)), self._h)
+
+    # convenience wrappers that allocate the outputs (tests, examples)
+    def verify(self, x: torch.Tensor, kind: int, stream=None):
+        scores = torch.empty(self.rows, NUM_METRICS, dtype=torch.float32, device=x.device)
+        flags = torch.empty(self.rows, dtype=torch.int32, device=x.device)
+        self.sentinel_verify(x, kind, scores, flags, stream)
+        return scores, flags
+
+    def update_reference(self, x: torch.Tensor, kind: int, stream=None):
+        scores = torch.empty(self.rows, NUM_METRICS, dtype=torch.float32, device=x.device)
+        self.sentinel_update_reference(x, kind, scores, stream)
+        return scores
+
+    # -- queries ----------------------------------------------------------------------------
+    def sentinel_get_stats(self, kind: int, stream=None) -> torch.Tensor:
+        out = torch.empty(self.rows, NUM_STATS, dtype=torch.float32, device=self.device)
+        _check(lib().sentinel_get_stats(self._h, kind, _ptr(out), _stream_ptr(stream)), self._h)
+        return out
+
+    def sentinel_get_thresholds(self, kind: int, stream=None):
+        thr = (C.c_double * (2 * NUM_METRICS * NUM_THRESHOLDS))()
+        valid = (C.c_int * (2 * NUM_METRICS))()
+        _check(lib().sentinel_get_thresholds(self._h, kind, thr, valid, _stream_ptr(stream)), self._h)
+        t = torch.tensor(list(thr), dtype=torch.float64).reshape(2, NUM_METRICS, NUM_THRESHOLDS)
+        v = torch.tensor(list(valid), dtype=torch.bool).reshape(2, NUM_METRICS)
+        return t.numpy(), v.numpy()
+
+    def sentinel_get_counters(self, stream=None) -> dict:
+        out = (C.c_longlong * 6)()
+        _check(lib().sentinel_get_counters(self._h, out, _stream_ptr(stream)), self._h)
+        return {"violations": out[0], "clean_streak": out[1], "banned": out[2],
+                "steps_act": out[3], "steps_grad": out[4], "error": out[5]}
+
+    def sentinel_set_token_stats_buffer(self, buf: torch.Tensor | None) -> None:
+        self._token_buf = buf          # keep the tensor alive while registered
+        _check(lib().sentinel_set_token_stats_buffer(self._h, _ptr(buf)), self._h)
+
+    def sentinel_reset_worker(self, stream=None) -> None:
+        _check(lib().sentinel_reset_worker(self._h, _stream_ptr(stream)), self._h)
+
+    # -- checkpointing ------------------------------------------------------------------------
+    def sentinel_state_bytes(self) -> int:
+        return int(lib().sentinel_state_bytes(self._h))
+
+    def sentinel_export_state(self, stream=None) -> bytearray:
+        n = self.sentinel_state_bytes()
+        buf = bytearray(n)
+        cbuf = (C.c_char * n).from_buffer(buf)
+        _check(lib().sentinel_export_state(self._h, cbuf, n, _stream_ptr(stream)), self._h)
+        return buf
+
+    def sentinel_import_state(self, blob, stream=None) -> None:
+        data = bytes(blob)
+        _check(lib().sentinel_import_state(self._h, data, len(data), _stream_ptr(stream)), self._h)
+
+    # -- lifetime -----------------------------------------------------------------------------
+    def sentinel_destroy(self) -> None:
+        if getattr(self, "_h", None):
+            h, self._h = self._h, None
+            _check(lib().sentinel_destroy(h))
+
+    close = sentinel_destroy
+
+    def __del__(self):
+        try:
+            self.sentinel_destroy()
+        except Exception:
+            pass

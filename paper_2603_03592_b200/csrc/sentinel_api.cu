@@ -1,0 +1,556 @@
+// Host side of libsentinel: argument checks, state ownership, launches.  See include/sentinel.h.
+#include "sentinel.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "sentinel_kernels.cuh"
+
+using namespace sentinel;
+
+namespace {
+
+thread_local std::string g_error;   // failures of calls that have no handle
+
+constexpr unsigned long long kMagic = 0x4c454e49544e4553ull;  // "SENTINEL", little endian
+constexpr unsigned kVersion = 1;
+constexpr size_t kHeaderBytes = 64;
+
+struct BlobHeader {
+  unsigned long long magic;
+  unsigned version;
+  int B, T, d, window_steps, violations, clean_streak, banned;
+};
+static_assert(sizeof(BlobHeader) <= kHeaderBytes, "header must fit its slot");
+
+struct BlobKindHead {
+  long long steps;
+  int count[2];
+  int valid[2][kNumMetrics];
+  double thr[2][kNumMetrics][kNumThr];
+};
+static_assert(sizeof(BlobKindHead) == 8 + 8 + 24 + 288, "packed layout expected");
+
+}  // namespace
+
+struct sentinel_verifier {
+  sentinel_config cfg;
+  size_t N = 0, Ns = 0;
+  int cap0 = 0, cap1 = 0;
+  int P = 1, grid = 2;
+  float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
+  HandleState *hs = nullptr;
+  double *hist[2] = {nullptr, nullptr};
+  unsigned long long *partials = nullptr;
+  float *stats[2] = {nullptr, nullptr};
+  float *token_buf = nullptr;
+  void *stage_x = nullptr;          // staging for sentinel_verify_host, allocated on first use
+  float *stage_scores = nullptr;
+  unsigned *stage_flags = nullptr;
+  std::string err;
+};
+
+namespace {
+
+int fail(sentinel_verifier *h, int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (h) h->err = buf; else g_error = buf;
+  return code;
+}
+
+#define SENTINEL_CUDA(h, call)                                                              \
+  do {                                                                                      \
+    cudaError_t e_ = (call);                                                                \
+    if (e_ != cudaSuccess)                                                                  \
+      return fail((h), SENTINEL_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));  \
+  } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t hist_doubles(const sentinel_verifier *h) {
+  return (size_t)kNumMetrics * ((size_t)h->cap0 + (size_t)h->cap1);
+}
+
+size_t kind_blob_bytes(const sentinel_verifier *h) {
+  return sizeof(BlobKindHead) + hist_doubles(h) * sizeof(double) + h->N * sizeof(float);
+}
+
+Alg5Params alg5_of(const sentinel_config &c, int kind) {
+  Alg5Params p;
+  p.alpha = c.alpha[kind];
+  p.gamma_g = c.gamma_grow[kind];
+  p.gamma_s = c.gamma_shrink[kind];
+  p.lambda = c.lambda_min[kind];
+  p.eps = c.iqr_eps[kind];
+  p.shrink_ratio = c.shrink_ratio;
+  p.n_max = c.n_max[kind];
+  p.pad = 0;
+  return p;
+}
+
+// how many pieces each sample is cut into, and the grid that follows
+int pieces_per_sample(int device, int B, int T, int *grid_out, std::string *err) {
+  int sms = 0, occ = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, stream_kernel, kThreads, 0);
+  if (e != cudaSuccess || sms < 1 || occ < 1) {
+    if (err) *err = std::string("occupancy query failed: ") + cudaGetErrorString(e);
+    return -1;
+  }
+  const int resident = sms * occ;                   // one slot is CTA 0's
+  int P = (resident - 1) / B;
+  if (P < 1) P = 1;
+  if (P > T) P = T;
+  *grid_out = 1 + B * P;
+  return P;
+}
+
+int check_shape(sentinel_verifier *h, int B, int T, int d) {
+  if (B < 1 || T < 1 || d < 1) return fail(h, SENTINEL_ERR_INVALID_ARG, "B, T, d must be positive (got %d, %d, %d)", B, T, d);
+  if (d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", d);
+  if (B > SENTINEL_MAX_B) return fail(h, SENTINEL_ERR_UNSUPPORTED, "B = %d exceeds SENTINEL_MAX_B = %d", B, SENTINEL_MAX_B);
+  return SENTINEL_OK;
+}
+
+int check_call(sentinel_verifier *h, const void *x, int kind, int B, int T, int d) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!x) return fail(h, SENTINEL_ERR_INVALID_ARG, "x is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", kind);
+  if (B != h->cfg.B || T != h->cfg.T || d != h->cfg.d)
+    return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
+  if (!aligned16(x)) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 16-byte aligned");
+  return SENTINEL_OK;
+}
+
+StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, float *scores, unsigned *flags) {
+  StreamArgs a;
+  memset(&a, 0, sizeof a);
+  a.x = static_cast<const uint16_t *>(x);
+  a.ema[0] = h->ema[kind][0];
+  a.ema[1] = h->ema[kind][1];
+  a.hs = h->hs;
+  a.hist = h->hist[kind];
+  a.partials = h->partials;
+  a.ticket = &h->hs->ticket;
+  a.scores_out = scores;
+  a.flags_out = flags;
+  a.stats_out = h->stats[kind];
+  a.token_out = h->token_buf;
+  a.B = h->cfg.B; a.T = h->cfg.T; a.d = h->cfg.d;
+  a.P = h->P;
+  a.mode = mode;
+  a.kind = kind;
+  a.beta = (float)h->cfg.beta[kind];
+  a.one_minus_beta = (float)(1.0 - h->cfg.beta[kind]);
+  a.cap0 = h->cap0; a.cap1 = h->cap1;
+  a.a5 = alg5_of(h->cfg, kind);
+  a.severe_mult = h->cfg.severe_mult;
+  a.ban_violations = h->cfg.ban_violations;
+  a.forgiveness_steps = h->cfg.forgiveness_steps;
+  a.metric_mask = h->cfg.metric_mask;
+  return a;
+}
+
+int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) {
+  stream_kernel<<<grid, kThreads, 0, s>>>(a);
+  SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
+}
+
+int run_refresh(sentinel_verifier *h, cudaStream_t s) {
+  refresh_kernel<<<1, kThreads, 0, s>>>(h->hs, h->hist[0], h->hist[1], h->cap0, h->cap1,
+                                        alg5_of(h->cfg, 0), alg5_of(h->cfg, 1));
+  SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
+}
+
+struct DeviceGuard {   // restores the caller's current device
+  int prev = -1;
+  cudaError_t status;
+  explicit DeviceGuard(int dev) {
+    status = cudaGetDevice(&prev);
+    if (status == cudaSuccess && prev != dev) status = cudaSetDevice(dev);
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+void free_all(sentinel_verifier *h) {
+  for (int k = 0; k < 2; ++k) {
+    for (int j = 0; j < 2; ++j) cudaFree(h->ema[k][j]);
+    cudaFree(h->hist[k]);
+    cudaFree(h->stats[k]);
+  }
+  cudaFree(h->hs);
+  cudaFree(h->partials);
+  cudaFree(h->stage_x);
+  cudaFree(h->stage_scores);
+  cudaFree(h->stage_flags);
+}
+
+}  // namespace
+
+extern "C" {
+
+int sentinel_default_config(sentinel_config *cfg) {
+  if (!cfg) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "cfg is NULL");
+  memset(cfg, 0, sizeof *cfg);
+  cfg->beta[0] = 0.90;         cfg->beta[1] = 0.80;
+  cfg->k0[0] = 1.5;            cfg->k0[1] = 3.0;
+  cfg->alpha[0] = 1e-4;        cfg->alpha[1] = 1e-3;
+  cfg->n_max[0] = 10;          cfg->n_max[1] = 10;
+  cfg->gamma_grow[0] = 1.1;    cfg->gamma_grow[1] = 1.01;
+  cfg->gamma_shrink[0] = 0.9;  cfg->gamma_shrink[1] = 0.99;
+  cfg->lambda_min[0] = 0.15;   cfg->lambda_min[1] = 0.05;
+  cfg->iqr_eps[0] = 1e-3;      cfg->iqr_eps[1] = 5e-5;
+  cfg->shrink_ratio = 0.5;
+  cfg->severe_mult = 100.0;
+  cfg->window_steps = 100;
+  cfg->ban_violations = 5;
+  cfg->forgiveness_steps = 100;
+  cfg->metric_mask = 7u;
+  return SENTINEL_OK;
+}
+
+int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out) {
+  if (!cfg || !out) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "cfg or out is NULL");
+  *out = nullptr;
+  int rc = check_shape(nullptr, cfg->B, cfg->T, cfg->d);
+  if (rc) return rc;
+  for (int k = 0; k < 2; ++k) {
+    if (!(cfg->beta[k] >= 0.0 && cfg->beta[k] < 1.0)) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "beta[%d] = %g is outside [0,1)", k, cfg->beta[k]);
+    if (!(cfg->k0[k] > 0.0) || !(cfg->gamma_grow[k] > 1.0) || !(cfg->gamma_shrink[k] > 0.0 && cfg->gamma_shrink[k] < 1.0) ||
+        !(cfg->alpha[k] >= 0.0) || cfg->n_max[k] < 0 || !(cfg->lambda_min[k] >= 0.0) || !(cfg->iqr_eps[k] >= 0.0))
+      return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "threshold parameters of kind %d are out of range", k);
+  }
+  if (cfg->window_steps < 1 || cfg->ban_violations < 1 || cfg->forgiveness_steps < 1 || !(cfg->severe_mult > 0.0) || !(cfg->shrink_ratio >= 0.0))
+    return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "window_steps, ban_violations, forgiveness_steps, severe_mult must be positive");
+  if ((long long)cfg->window_steps * cfg->B > SENTINEL_MAX_WINDOW)
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*B = %lld exceeds SENTINEL_MAX_WINDOW = %d", (long long)cfg->window_steps * cfg->B, SENTINEL_MAX_WINDOW);
+  int ndev = 0;
+  SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
+  if (cfg->device < 0 || cfg->device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist (%d devices)", cfg->device, ndev);
+
+  DeviceGuard guard(cfg->device);
+  SENTINEL_CUDA(nullptr, guard.status);
+
+  sentinel_verifier *h = new (std::nothrow) sentinel_verifier();
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "out of host memory");
+  h->cfg = *cfg;
+  h->Ns = (size_t)cfg->T * cfg->d;
+  h->N = h->Ns * cfg->B;
+  h->cap0 = cfg->window_steps;
+  h->cap1 = cfg->window_steps * cfg->B;
+  std::string oerr;
+  h->P = pieces_per_sample(cfg->device, cfg->B, cfg->T, &h->grid, &oerr);
+  if (h->P < 1) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "%s", oerr.c_str()); }
+
+  cudaError_t e = cudaSuccess;
+  auto alloc = [&](void **p, size_t bytes) {
+    if (e == cudaSuccess) e = cudaMalloc(p, bytes);
+    if (e == cudaSuccess) e = cudaMemset(*p, 0, bytes);
+  };
+  for (int k = 0; k < 2; ++k) {
+    for (int j = 0; j < 2; ++j) alloc((void **)&h->ema[k][j], h->N * sizeof(float));   // m_0 = 0
+    alloc((void **)&h->hist[k], hist_doubles(h) * sizeof(double));
+    alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
+  }
+  alloc((void **)&h->partials, (size_t)cfg->B * h->P * kSlotWords * sizeof(unsigned long long));
+  alloc((void **)&h->hs, sizeof(HandleState));
+  if (e == cudaSuccess) {
+    HandleState init;
+    memset(&init, 0, sizeof init);
+    for (int k = 0; k < 2; ++k)
+      for (int L = 0; L < 2; ++L)
+        for (int i = 0; i < kNumMetrics; ++i) init.kind[k].thr[L][i][3] = cfg->k0[k];
+    e = cudaMemcpy(h->hs, &init, sizeof init, cudaMemcpyHostToDevice);
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    free_all(h);
+    delete h;
+    return fail(nullptr, SENTINEL_ERR_CUDA, "allocating verifier state failed: %s", cudaGetErrorString(e));
+  }
+  *out = h;
+  return SENTINEL_OK;
+}
+
+int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T, int d,
+                    void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out) {
+  int rc = check_call(h, dev_x, kind, B, T, d);
+  if (rc) return rc;
+  if (!dev_scores_out || !dev_flags_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  return launch(h, make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out), h->grid,
+                static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T,
+                              int d, void *cuda_stream, float *dev_scores_out) {
+  int rc = check_call(h, dev_x, kind, B, T, d);
+  if (rc) return rc;
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  return launch(h, make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr), h->grid,
+                static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind kind, int B, int T,
+                         int d, void *cuda_stream, float *host_scores_out, unsigned *host_flags_out) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_x || !host_scores_out || !host_flags_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "a host pointer is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", (int)kind);
+  if (B != h->cfg.B || T != h->cfg.T || d != h->cfg.d)
+    return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t rows = 1 + (size_t)B;
+  if (!h->stage_x) {
+    SENTINEL_CUDA(h, cudaMalloc(&h->stage_x, h->N * sizeof(uint16_t)));
+    SENTINEL_CUDA(h, cudaMalloc((void **)&h->stage_scores, rows * kNumMetrics * sizeof(float)));
+    SENTINEL_CUDA(h, cudaMalloc((void **)&h->stage_flags, rows * sizeof(unsigned)));
+  }
+  SENTINEL_CUDA(h, cudaMemcpyAsync(h->stage_x, host_x, h->N * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
+  int rc = launch(h, make_args(h, h->stage_x, kind, kModeVerify, h->stage_scores, h->stage_flags), h->grid, s);
+  if (rc) return rc;
+  SENTINEL_CUDA(h, cudaMemcpyAsync(host_scores_out, h->stage_scores, rows * kNumMetrics * sizeof(float), cudaMemcpyDeviceToHost, s));
+  SENTINEL_CUDA(h, cudaMemcpyAsync(host_flags_out, h->stage_flags, rows * sizeof(unsigned), cudaMemcpyDeviceToHost, s));
+  SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+  return SENTINEL_OK;
+}
+
+int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d, int device,
+                      void *cuda_stream, float *dev_scores_out, float *dev_stats_out) {
+  if (!dev_x || !dev_m || !dev_scores_out) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "x, m or scores_out is NULL");
+  int rc = check_shape(nullptr, B, T, d);
+  if (rc) return rc;
+  if (!aligned16(dev_x) || !aligned16(dev_m)) return fail(nullptr, SENTINEL_ERR_UNALIGNED, "x or m is not 16-byte aligned");
+  int ndev = 0;
+  SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
+  if (device < 0 || device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist", device);
+  DeviceGuard guard(device);
+  SENTINEL_CUDA(nullptr, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+  int grid = 0;
+  std::string oerr;
+  const int P = pieces_per_sample(device, B, T, &grid, &oerr);
+  if (P < 1) return fail(nullptr, SENTINEL_ERR_CUDA, "%s", oerr.c_str());
+  // scratch: one slot per piece, then the ticket word
+  const size_t slot_bytes = (size_t)B * P * kSlotWords * sizeof(unsigned long long);
+  unsigned char *scratch = nullptr;
+  SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, slot_bytes + 256, s));
+  SENTINEL_CUDA(nullptr, cudaMemsetAsync(scratch + slot_bytes, 0, 256, s));
+
+  StreamArgs a;
+  memset(&a, 0, sizeof a);
+  a.x = static_cast<const uint16_t *>(dev_x);
+  a.m_ext = dev_m;
+  a.partials = reinterpret_cast<unsigned long long *>(scratch);
+  a.ticket = reinterpret_cast<unsigned *>(scratch + slot_bytes);
+  a.scores_out = dev_scores_out;
+  a.stats_out = dev_stats_out;
+  a.B = B; a.T = T; a.d = d; a.P = P;
+  a.mode = kModeDistance;
+  stream_kernel<<<grid, kThreads, 0, s>>>(a);
+  cudaError_t le = cudaGetLastError();
+  cudaError_t fe = cudaFreeAsync(scratch, s);
+  SENTINEL_CUDA(nullptr, le);
+  SENTINEL_CUDA(nullptr, fe);
+  return SENTINEL_OK;
+}
+
+int sentinel_get_stats(sentinel_verifier *h, sentinel_kind kind, float *dev_stats_out, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!dev_stats_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "stats_out is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "bad kind %d", (int)kind);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  SENTINEL_CUDA(h, cudaMemcpyAsync(dev_stats_out, h->stats[kind], (size_t)(1 + h->cfg.B) * kNumStats * sizeof(float),
+                                   cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
+  return SENTINEL_OK;
+}
+
+int sentinel_get_thresholds(sentinel_verifier *h, sentinel_kind kind, double *host_out, int *host_valid, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "host_out is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "bad kind %d", (int)kind);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int rc = run_refresh(h, s);
+  if (rc) return rc;
+  HandleState snap;
+  SENTINEL_CUDA(h, cudaMemcpyAsync(&snap, h->hs, sizeof snap, cudaMemcpyDeviceToHost, s));
+  SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+  memcpy(host_out, snap.kind[kind].thr, sizeof snap.kind[kind].thr);
+  if (host_valid) memcpy(host_valid, snap.kind[kind].has_thr, sizeof snap.kind[kind].has_thr);
+  return SENTINEL_OK;
+}
+
+int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "host_out is NULL");
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  HandleState snap;
+  SENTINEL_CUDA(h, cudaMemcpyAsync(&snap, h->hs, sizeof snap, cudaMemcpyDeviceToHost, s));
+  SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+  host_out[0] = snap.violations;
+  host_out[1] = snap.clean_streak;
+  host_out[2] = snap.banned;
+  host_out[3] = snap.kind[0].steps;
+  host_out[4] = snap.kind[1].steps;
+  host_out[5] = snap.error;
+  return SENTINEL_OK;
+}
+
+int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (dev_buf && !aligned16(dev_buf)) return fail(h, SENTINEL_ERR_UNALIGNED, "token buffer is not 16-byte aligned");
+  h->token_buf = dev_buf;
+  return SENTINEL_OK;
+}
+
+int sentinel_reset_worker(sentinel_verifier *h, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  reset_worker_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>(h->hs);
+  SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
+}
+
+size_t sentinel_state_bytes(const sentinel_verifier *h) {
+  if (!h) return 0;
+  return kHeaderBytes + 2 * kind_blob_bytes(h);
+}
+
+int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_buf) return fail(h, SENTINEL_ERR_INVALID_ARG, "host_buf is NULL");
+  if (n < sentinel_state_bytes(h)) return fail(h, SENTINEL_ERR_STATE_SIZE, "buffer of %zu bytes, %zu needed", n, sentinel_state_bytes(h));
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int rc = run_refresh(h, s);
+  if (rc) return rc;
+  HandleState snap;
+  SENTINEL_CUDA(h, cudaMemcpyAsync(&snap, h->hs, sizeof snap, cudaMemcpyDeviceToHost, s));
+  SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+
+  unsigned char *out = static_cast<unsigned char *>(host_buf);
+  memset(out, 0, kHeaderBytes);
+  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps,
+                   snap.violations, snap.clean_streak, snap.banned};
+  memcpy(out, &hd, sizeof hd);
+  out += kHeaderBytes;
+  std::vector<double> ring(hist_doubles(h));
+  for (int k = 0; k < 2; ++k) {
+    const KindState &ks = snap.kind[k];
+    BlobKindHead kh;
+    memset(&kh, 0, sizeof kh);
+    kh.steps = ks.steps;
+    memcpy(kh.count, ks.hist_count, sizeof kh.count);
+    memcpy(kh.valid, ks.has_thr, sizeof kh.valid);
+    memcpy(kh.thr, ks.thr, sizeof kh.thr);
+    memcpy(out, &kh, sizeof kh);
+    out += sizeof kh;
+    SENTINEL_CUDA(h, cudaMemcpyAsync(ring.data(), h->hist[k], ring.size() * sizeof(double), cudaMemcpyDeviceToHost, s));
+    SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+    double *dst = reinterpret_cast<double *>(out);
+    size_t src_off = 0;
+    for (int L = 0; L < 2; ++L) {                   // unroll each ring, oldest entry first
+      const int cap = L ? h->cap1 : h->cap0;
+      for (int i = 0; i < kNumMetrics; ++i) {
+        for (int j = 0; j < cap; ++j)
+          dst[j] = (j < ks.hist_count[L]) ? ring[src_off + (size_t)((ks.hist_head[L] + j) % cap)] : 0.0;
+        dst += cap;
+        src_off += cap;
+      }
+    }
+    out = reinterpret_cast<unsigned char *>(dst);
+    SENTINEL_CUDA(h, cudaMemcpyAsync(out, h->ema[k][ks.active], h->N * sizeof(float), cudaMemcpyDeviceToHost, s));
+    SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+    out += h->N * sizeof(float);
+  }
+  return SENTINEL_OK;
+}
+
+int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_buf) return fail(h, SENTINEL_ERR_INVALID_ARG, "host_buf is NULL");
+  if (n < sentinel_state_bytes(h)) return fail(h, SENTINEL_ERR_STATE_SIZE, "blob of %zu bytes, %zu needed", n, sentinel_state_bytes(h));
+  const unsigned char *in = static_cast<const unsigned char *>(host_buf);
+  BlobHeader hd;
+  memcpy(&hd, in, sizeof hd);
+  if (hd.magic != kMagic || hd.version != kVersion)
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "not a sentinel state blob of version %u", kVersion);
+  if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps)
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d", hd.B, hd.T, hd.d, hd.window_steps);
+  // validate both kinds before touching the device
+  const unsigned char *p = in + kHeaderBytes;
+  for (int k = 0; k < 2; ++k) {
+    BlobKindHead kh;
+    memcpy(&kh, p, sizeof kh);
+    if (kh.count[0] < 0 || kh.count[0] > h->cap0 || kh.count[1] < 0 || kh.count[1] > h->cap1)
+      return fail(h, SENTINEL_ERR_STATE_SIZE, "history counts in the blob are out of range");
+    p += kind_blob_bytes(h);
+  }
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+  HandleState st;
+  memset(&st, 0, sizeof st);
+  st.violations = hd.violations;
+  st.clean_streak = hd.clean_streak;
+  st.banned = hd.banned;
+  p = in + kHeaderBytes;
+  for (int k = 0; k < 2; ++k) {
+    BlobKindHead kh;
+    memcpy(&kh, p, sizeof kh);
+    p += sizeof kh;
+    KindState &ks = st.kind[k];
+    ks.steps = kh.steps;
+    ks.active = 0;
+    ks.refresh_pending = 0;
+    memcpy(ks.hist_count, kh.count, sizeof kh.count);
+    ks.hist_head[0] = ks.hist_head[1] = 0;
+    memcpy(ks.has_thr, kh.valid, sizeof kh.valid);
+    memcpy(ks.thr, kh.thr, sizeof kh.thr);
+    SENTINEL_CUDA(h, cudaMemcpyAsync(h->hist[k], p, hist_doubles(h) * sizeof(double), cudaMemcpyHostToDevice, s));
+    p += hist_doubles(h) * sizeof(double);
+    SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], p, h->N * sizeof(float), cudaMemcpyHostToDevice, s));
+    p += h->N * sizeof(float);
+  }
+  SENTINEL_CUDA(h, cudaMemcpyAsync(h->hs, &st, sizeof st, cudaMemcpyHostToDevice, s));
+  SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+  return SENTINEL_OK;
+}
+
+const char *sentinel_last_error(const sentinel_verifier *h) { return h ? h->err.c_str() : g_error.c_str(); }
+
+int sentinel_destroy(sentinel_verifier *h) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  DeviceGuard guard(h->cfg.device);
+  cudaError_t e = guard.status;
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  free_all(h);
+  delete h;
+  if (e != cudaSuccess) return fail(nullptr, SENTINEL_ERR_CUDA, "destroy: %s", cudaGetErrorString(e));
+  return SENTINEL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,624 @@
+// Device code of libsentinel: one streaming pass over a [B,T,d] bf16 tensor x and the fp32
+// reference m that (1) accumulates, per sample, the sufficient statistics of the paper's
+// distance measures (Sec. 3.1), (2) writes the EMA candidate beta*m + (1-beta)*x (Eq. 1) into
+// the spare reference buffer, and (3) in the last CTA to finish, turns the sums into scores,
+// applies the Tukey test (Eq. 3), keeps the violation counter, appends to the history and
+// commits the candidate by flipping the active-buffer index.  Thresholds (Alg. 5) for the next
+// step are recomputed by CTA 0 of the *next* launch while the other CTAs stream.
+//
+// sm_100a only: 256-bit global loads/stores (ld/st.global.v8.f32).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace sentinel {
+
+constexpr int kNumMetrics = 3;
+constexpr int kNumStats = 8;
+constexpr int kNumThr = 6;
+constexpr int kMaxB = 64;
+constexpr int kMaxWindow = 4096;
+constexpr int kThreads = 512;             // threads per CTA
+constexpr int kWarps = kThreads / 32;
+constexpr int kSlotWords = 8;             // 64-bit words per partial slot
+constexpr int kUnroll = 4;                // 8-element chunks per lane per loop trip
+
+enum Mode : int { kModeVerify = 0, kModeWarmup = 1, kModeDistance = 2 };
+
+// flag bits (mirrors the public header)
+constexpr unsigned kFlagNonfinite = 1u << 7;
+constexpr unsigned kFlagCommitted = 1u << 16;
+constexpr unsigned kFlagSevere = 1u << 17;
+constexpr unsigned kFlagBanned = 1u << 18;
+constexpr unsigned kFlagNoThresholds = 1u << 19;
+
+// bits of word 7 of a partial slot
+constexpr unsigned long long kBitNonfinite = 1ull, kBitXVaries = 2ull, kBitMVaries = 4ull;
+
+struct Alg5Params {
+  double alpha, gamma_g, gamma_s, lambda, eps, shrink_ratio;
+  int n_max;
+  int pad;
+};
+
+// Device-resident state of one kind (activations or gradients) of one boundary.
+struct KindState {
+  long long steps;
+  int active;             // which of the two EMA buffers holds m_{t-1}
+  int refresh_pending;    // Alg. 5 is owed for the history as it stands
+  int hist_count[2];      // entries in the window, per level
+  int hist_head[2];       // ring position of the oldest entry
+  int has_thr[2][kNumMetrics];
+  double thr[2][kNumMetrics][kNumThr];   // q1 q2 q3 k tau_lower tau_upper
+};
+
+struct HandleState {
+  int violations, clean_streak, banned, error;
+  unsigned ticket;
+  int pad[3];
+  KindState kind[2];
+};
+
+struct StreamArgs {
+  const uint16_t *x;               // bf16 [B,T,d]
+  const float *m_ext;              // distance mode: caller's reference; else unused
+  float *ema[2];                   // the two reference buffers of this kind
+  HandleState *hs;                 // nullptr in distance mode
+  double *hist;                    // this kind's rings: level 0 [3][cap0], level 1 [3][cap1]
+  unsigned long long *partials;    // [pieces][kSlotWords]
+  unsigned *ticket;
+  float *scores_out;               // [(1+B)*3] or nullptr
+  unsigned *flags_out;             // [1+B] or nullptr
+  float *stats_out;                // [(1+B)*8] or nullptr
+  float *token_out;                // [B,T,4] or nullptr
+  int B, T, d;
+  int P;                           // pieces per sample
+  int mode, kind;
+  float beta, one_minus_beta;
+  int cap0, cap1;
+  Alg5Params a5;
+  double severe_mult;
+  int ban_violations, forgiveness_steps;
+  unsigned metric_mask;
+  int pad;
+};
+
+// ---------------------------------------------------------------------------------------------
+// memory access helpers
+
+struct __align__(32) F8 { float v[8]; };
+
+__device__ __forceinline__ uint4 ld_x128(const uint16_t *p) {
+  uint4 r;
+  asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+      : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
+}
+__device__ __forceinline__ F8 ld_m256(const float *p) {
+  F8 r;
+  asm("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+      : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]),
+        "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7]) : "l"(p));
+  return r;
+}
+__device__ __forceinline__ void st_m256(float *p, const F8 &r) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]),
+                  "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7]) : "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-element work
+
+struct GroupAcc {            // fp32 partial sums over one loop trip (<= 8*kUnroll elements)
+  float sx, sxx, sm, smm, sxm, ab;
+  unsigned flips;
+};
+
+// First and second moments are accumulated on x - x0 and m - m0, where x0 / m0 is the first
+// element of the sample: variance and covariance do not depend on the shift, and the shifted
+// values are of the size of the spread, so a mean far from zero costs no digits.
+__device__ __forceinline__ void element(float xf, float mf, float x0, float m0, GroupAcc &g) {
+  const float xs = xf - x0, ms = mf - m0;
+  g.sx += xs;
+  g.sxx = fmaf(xs, xs, g.sxx);
+  g.sm += ms;
+  g.smm = fmaf(ms, ms, g.smm);
+  g.sxm = fmaf(xs, ms, g.sxm);
+  g.ab += fabsf(xf - mf);
+  const int sgx = (xf > 0.f) - (xf < 0.f);
+  const int sgm = (mf > 0.f) - (mf < 0.f);
+  g.flips += (sgx != sgm);
+}
+
+struct ThreadAcc {           // carried over the whole piece
+  double sx, sxx, sm, smm, sxm, ab;
+  unsigned flips;
+  unsigned nf_bits;          // non-zero: a bf16 exponent of all ones was seen
+  unsigned x_diff, m_diff;   // non-zero: some element differs bitwise from the sample's first
+};
+
+// one 8-element chunk: x as 4 packed bf16 pairs, m as 8 floats; returns the EMA candidate in m
+__device__ __forceinline__ void chunk(const uint4 &xv, F8 &mv, GroupAcc &g, ThreadAcc &t,
+                                      unsigned x0pair, unsigned m0bits, float beta, float omb,
+                                      bool write_ema) {
+  const float x0 = __uint_as_float(x0pair << 16), m0 = __uint_as_float(m0bits);
+  const unsigned w[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    // exponent field 0xFF in either half <=> NaN or infinity
+    t.nf_bits |= ((w[j] & 0x7F807F80u) + 0x00800080u) & 0x80008000u;
+    t.x_diff |= w[j] ^ x0pair;
+    const float x_lo = __uint_as_float(w[j] << 16);
+    const float x_hi = __uint_as_float(w[j] & 0xFFFF0000u);
+    const float m_lo = mv.v[2 * j], m_hi = mv.v[2 * j + 1];
+    t.m_diff |= (__float_as_uint(m_lo) ^ m0bits) | (__float_as_uint(m_hi) ^ m0bits);
+    element(x_lo, m_lo, x0, m0, g);
+    element(x_hi, m_hi, x0, m0, g);
+    if (write_ema) {
+      mv.v[2 * j] = fmaf(beta, m_lo, omb * x_lo);
+      mv.v[2 * j + 1] = fmaf(beta, m_hi, omb * x_hi);
+    }
+  }
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// streaming phase: CTA `piece` covers rows [r0, r1) of one sample; a warp owns whole rows
+
+__device__ void stream_piece(const StreamArgs &a, int piece, const float *m_in, float *m_out,
+                             unsigned long long (*s_part)[kSlotWords]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = piece / a.P, p = piece - b * a.P;
+  const long long row_base = (long long)b * a.T;
+  const int r0 = (int)(((long long)p * a.T) / a.P);
+  const int r1 = (int)(((long long)(p + 1) * a.T) / a.P);
+  const int chunks = a.d >> 3;
+  const size_t sample_off = (size_t)row_base * a.d;
+  const bool write_ema = (m_out != nullptr);
+  const bool tokens = (a.token_out != nullptr);
+  const float beta = a.beta, omb = a.one_minus_beta;
+
+  const unsigned x0 = a.x[sample_off];
+  const unsigned x0pair = x0 | (x0 << 16);
+  const unsigned m0bits = __float_as_uint(m_in[sample_off]);
+
+  ThreadAcc t = {0., 0., 0., 0., 0., 0., 0u, 0u, 0u, 0u};
+
+  for (int r = r0 + warp; r < r1; r += kWarps) {
+    const size_t off = (size_t)(row_base + r) * a.d;
+    const uint16_t *xrow = a.x + off;
+    const float *mrow = m_in + off;
+    float *orow = write_ema ? m_out + off : nullptr;
+    float tk_sx = 0.f, tk_sxx = 0.f, tk_ab = 0.f;
+    unsigned tk_flips = 0u;
+
+    for (int base = 0; base < chunks; base += 32 * kUnroll) {
+      uint4 xv[kUnroll];
+      F8 mv[kUnroll];
+      bool ok[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int c = base + u * 32 + lane;
+        ok[u] = c < chunks;
+        if (ok[u]) {
+          xv[u] = ld_x128(xrow + (size_t)c * 8);
+          mv[u] = ld_m256(mrow + (size_t)c * 8);
+        }
+      }
+      GroupAcc g = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0u};
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (ok[u]) {
+          chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
+          if (write_ema) st_m256(orow + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+        }
+      }
+      // fold the short fp32 run into the fp64 accumulators
+      t.sx += (double)g.sx;   t.sxx += (double)g.sxx;
+      t.sm += (double)g.sm;   t.smm += (double)g.smm;
+      t.sxm += (double)g.sxm; t.ab += (double)g.ab;
+      t.flips += g.flips;
+      if (tokens) { tk_sx += g.sx; tk_sxx += g.sxx; tk_ab += g.ab; tk_flips += g.flips; }
+    }
+    if (tokens) {
+      tk_sx = warp_sum(tk_sx);
+      tk_sxx = warp_sum(tk_sxx);
+      tk_ab = warp_sum(tk_ab);
+      const float fl = warp_sum((float)tk_flips);
+      if (lane == 0) {                       // back from shifted to raw sums over the d channels
+        const float x0f = __uint_as_float(x0 << 16), dd = (float)a.d;
+        const float raw_sx = fmaf(dd, x0f, tk_sx);
+        const float raw_sxx = fmaf(dd * x0f, x0f, fmaf(2.f * x0f, tk_sx, tk_sxx));
+        reinterpret_cast<float4 *>(a.token_out)[row_base + r] = make_float4(raw_sx, raw_sxx, tk_ab, fl);
+      }
+    }
+  }
+
+  // warp -> CTA, in a fixed order so that two runs give bit-identical sums
+  const double ws[6] = {warp_sum(t.sx), warp_sum(t.sxx), warp_sum(t.sm),
+                        warp_sum(t.smm), warp_sum(t.sxm), warp_sum(t.ab)};
+  const unsigned long long wf = warp_sum((unsigned long long)t.flips);
+  unsigned long long bits = (t.nf_bits ? kBitNonfinite : 0ull) | (t.x_diff ? kBitXVaries : 0ull) |
+                            (t.m_diff ? kBitMVaries : 0ull);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < 6; ++j) s_part[warp][j] = (unsigned long long)__double_as_longlong(ws[j]);
+    s_part[warp][6] = wf;
+    s_part[warp][7] = bits;
+  }
+  __syncthreads();
+  if (threadIdx.x < kSlotWords) {
+    const int j = threadIdx.x;
+    unsigned long long out;
+    if (j < 6) {
+      double s = 0.;
+      for (int w = 0; w < kWarps; ++w) s += __longlong_as_double((long long)s_part[w][j]);
+      out = (unsigned long long)__double_as_longlong(s);
+    } else if (j == 6) {
+      out = 0ull;
+      for (int w = 0; w < kWarps; ++w) out += s_part[w][6];
+    } else {
+      out = 0ull;
+      for (int w = 0; w < kWarps; ++w) out |= s_part[w][7];
+    }
+    a.partials[(size_t)piece * kSlotWords + j] = out;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Alg. 5 on the device (one CTA)
+
+__device__ __forceinline__ double percentile_sorted(const double *s, int n, double p) {
+  const double pos = __dmul_rn(p, (double)(n - 1));
+  const int lo = (int)floor(pos);
+  const int hi = (lo + 1 < n) ? lo + 1 : lo;
+  const double frac = __dsub_rn(pos, (double)lo);
+  return __dadd_rn(s[lo], __dmul_rn(frac, __dsub_rn(s[hi], s[lo])));
+}
+
+// entries strictly outside [lo, hi], counted by one warp
+__device__ __forceinline__ int warp_count_outside(const double *s, int n, double lo, double hi, int lane) {
+  int c = 0;
+  for (int j = lane; j < n; j += 32) c += (s[j] < lo || s[j] > hi);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  return c;
+}
+
+// Refreshes q1,q2,q3,k,tau of every (level, metric) window of one kind.  Whole CTA.
+__device__ void refresh_thresholds(KindState *ks, const double *hist, int cap0, int cap1,
+                                   const Alg5Params &a5, double *s_sort) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  for (int L = 0; L < 2; ++L) {
+    const int n = ks->hist_count[L];
+    if (n == 0) continue;                          // empty window: nothing to compute
+    const int cap = L ? cap1 : cap0;
+    int npad = 1;
+    while (npad < n) npad <<= 1;
+    for (int i = 0; i < kNumMetrics; ++i) {
+      const double *ring = hist + (L ? (size_t)kNumMetrics * cap0 : 0) + (size_t)i * cap;
+      __syncthreads();
+      // the order of the window is immaterial to Alg. 5, so the ring is read as it lies
+      for (int j = tid; j < npad; j += kThreads) s_sort[j] = (j < n) ? ring[j] : CUDART_INF;
+      __syncthreads();
+      for (int k2 = 2; k2 <= npad; k2 <<= 1) {     // bitonic sort, ascending
+        for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
+          for (int t = tid; t < npad; t += kThreads) {
+            const int partner = t ^ j2;
+            if (partner > t) {
+              const double va = s_sort[t], vb = s_sort[partner];
+              const bool up = ((t & k2) == 0);
+              if ((va > vb) == up) { s_sort[t] = vb; s_sort[partner] = va; }
+            }
+          }
+          __syncthreads();
+        }
+      }
+      if (tid < 32) {                              // warp 0 walks the algorithm's steps
+        const double q1 = percentile_sorted(s_sort, n, 0.25);
+        const double q2 = percentile_sorted(s_sort, n, 0.50);
+        const double q3 = percentile_sorted(s_sort, n, 0.75);
+        const double iqr = fmax(__dsub_rn(q3, q1), a5.eps);
+        double k = ks->thr[L][i][3];
+        double lo = __dsub_rn(q2, __dmul_rn(k, iqr));
+        double hi = __dadd_rn(q2, __dmul_rn(k, iqr));
+        const double dn = (double)n;
+        double fp = (double)warp_count_outside(s_sort, n, lo, hi, lane) / dn;
+        int it = 0;
+        while (fp > a5.alpha && it < a5.n_max) {   // widen
+          k = __dmul_rn(k, a5.gamma_g);
+          lo = __dsub_rn(q2, __dmul_rn(k, iqr));
+          hi = __dadd_rn(q2, __dmul_rn(k, iqr));
+          fp = (double)warp_count_outside(s_sort, n, lo, hi, lane) / dn;
+          ++it;
+        }
+        it = 0;
+        const double low_mark = __dmul_rn(a5.shrink_ratio, a5.alpha);
+        while (fp < low_mark && it < a5.n_max) {   // narrow
+          k = __dmul_rn(k, a5.gamma_s);
+          lo = __dsub_rn(q2, __dmul_rn(k, iqr));
+          hi = __dadd_rn(q2, __dmul_rn(k, iqr));
+          fp = (double)warp_count_outside(s_sort, n, lo, hi, lane) / dn;
+          ++it;
+        }
+        const double d_min = __dmul_rn(fabs(q2), a5.lambda);
+        lo = fmin(lo, __dsub_rn(q2, d_min));
+        hi = fmax(hi, __dadd_rn(q2, d_min));
+        if (lane == 0) {
+          double *t = ks->thr[L][i];
+          t[0] = q1; t[1] = q2; t[2] = q3; t[3] = k; t[4] = lo; t[5] = hi;
+          ks->has_thr[L][i] = 1;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (tid == 0) ks->refresh_pending = 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// finalize: last CTA only
+
+struct UnitSums {
+  double s[6];               // sums of (x-x0) (x-x0)^2 (m-m0) (m-m0)^2 (x-x0)(m-m0) |x-m|
+  unsigned long long flips;
+  unsigned long long bits;
+  double x0, m0;             // the shift the sums were taken about
+};
+
+__device__ __forceinline__ void push_history(KindState *ks, double *hist, int L, int cap, int cap0,
+                                             const double g[kNumMetrics]) {
+  int idx;
+  if (ks->hist_count[L] < cap) {
+    idx = (ks->hist_head[L] + ks->hist_count[L]) % cap;
+    ks->hist_count[L] += 1;
+  } else {                                         // window full: the oldest entry leaves
+    idx = ks->hist_head[L];
+    ks->hist_head[L] = (idx + 1) % cap;
+  }
+  double *base = hist + (L ? (size_t)kNumMetrics * cap0 : 0);
+  for (int i = 0; i < kNumMetrics; ++i) base[(size_t)i * cap + idx] = g[i];
+}
+
+__device__ void finalize(const StreamArgs &a, const float *m_in) {
+  __shared__ UnitSums s_unit[kMaxB + 1];
+  __shared__ double s_gamma[kMaxB + 1][kNumMetrics];
+  __shared__ unsigned s_flag[kMaxB + 1];
+  __shared__ int s_severe, s_no_thr;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int B = a.B, rows = B + 1;
+  const size_t Ns = (size_t)a.T * a.d;
+
+  if (tid == 0) { s_severe = 0; s_no_thr = 0; }
+
+  // per-sample sums over that sample's pieces, in a fixed order
+  for (int b = warp; b < B; b += kWarps) {
+    double v[6] = {0., 0., 0., 0., 0., 0.};
+    unsigned long long fl = 0ull, bits = 0ull;
+    for (int p = lane; p < a.P; p += 32) {
+      const unsigned long long *slot = a.partials + ((size_t)b * a.P + p) * kSlotWords;
+#pragma unroll
+      for (int j = 0; j < 6; ++j) v[j] += __longlong_as_double((long long)__ldcg(slot + j));
+      fl += __ldcg(slot + 6);
+      bits |= __ldcg(slot + 7);
+    }
+#pragma unroll
+    for (int j = 0; j < 6; ++j) v[j] = warp_sum(v[j]);
+    fl = warp_sum(fl);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+    if (lane == 0) {
+#pragma unroll
+      for (int j = 0; j < 6; ++j) s_unit[1 + b].s[j] = v[j];
+      s_unit[1 + b].flips = fl;
+      s_unit[1 + b].bits = bits;
+      s_unit[1 + b].x0 = (double)__uint_as_float((unsigned)a.x[b * Ns] << 16);
+      s_unit[1 + b].m0 = (double)m_in[b * Ns];
+    }
+  }
+  __syncthreads();
+
+  // whole-tensor unit = the samples added up in order, re-centred on sample 0's shift:
+  // sum (x-K) = sum (x-x0) + n dx,  sum (x-K)^2 = sum (x-x0)^2 + 2 dx sum (x-x0) + n dx^2, ...
+  if (tid == 0) {
+    UnitSums u = {{0., 0., 0., 0., 0., 0.}, 0ull, 0ull, s_unit[1].x0, s_unit[1].m0};
+    const unsigned x_first = a.x[0];
+    const unsigned m_first = __float_as_uint(m_in[0]);
+    const double n = (double)Ns;
+    for (int b = 0; b < B; ++b) {
+      const UnitSums &v = s_unit[1 + b];
+      const double dx = v.x0 - u.x0, dm = v.m0 - u.m0;
+      u.s[0] += v.s[0] + n * dx;
+      u.s[1] += v.s[1] + 2. * dx * v.s[0] + n * dx * dx;
+      u.s[2] += v.s[2] + n * dm;
+      u.s[3] += v.s[3] + 2. * dm * v.s[2] + n * dm * dm;
+      u.s[4] += v.s[4] + dx * v.s[2] + dm * v.s[0] + n * dx * dm;
+      u.s[5] += v.s[5];
+      u.flips += v.flips;
+      u.bits |= v.bits;
+      if ((unsigned)a.x[b * Ns] != x_first) u.bits |= kBitXVaries;
+      if (__float_as_uint(m_in[b * Ns]) != m_first) u.bits |= kBitMVaries;
+    }
+    s_unit[0] = u;
+  }
+  __syncthreads();
+
+  KindState *ks = a.hs ? &a.hs->kind[a.kind] : nullptr;
+
+  // scores, statistics and the Tukey test: one thread per unit
+  unsigned my_flag = 0u;
+  if (tid < rows) {
+    const UnitSums u = s_unit[tid];
+    const double n = (tid == 0) ? (double)B * (double)Ns : (double)Ns;
+    const bool nonfinite = (u.bits & kBitNonfinite) != 0ull;
+    // a vector whose elements all equal its first one (bitwise, or +0 against -0) has
+    // variance exactly 0
+    const bool x_const = !(u.bits & kBitXVaries) || u.s[1] == 0.;
+    const bool m_const = !(u.bits & kBitMVaries) || u.s[3] == 0.;
+    const double dmean_x = u.s[0] / n, dmean_m = u.s[2] / n;      // means of the shifted values
+    const double mean_x = u.x0 + dmean_x, mean_m = u.m0 + dmean_m;
+    const double var_x = x_const ? 0. : fmax(u.s[1] / n - dmean_x * dmean_x, 0.);
+    const double var_m = m_const ? 0. : fmax(u.s[3] / n - dmean_m * dmean_m, 0.);
+    const double cov = u.s[4] / n - dmean_x * dmean_m;
+    const double sq_x = fmax(u.s[1] + 2. * u.x0 * u.s[0] + n * u.x0 * u.x0, 0.);   // sum x^2
+    const double sq_m = fmax(u.s[3] + 2. * u.m0 * u.s[2] + n * u.m0 * u.m0, 0.);
+    const double sd_x = sqrt(var_x), sd_m = sqrt(var_m);
+    double rho = 0., l2z;
+    if (sd_x > 0. && sd_m > 0.) {
+      rho = fmin(fmax(cov / (sd_x * sd_m), -1.), 1.);
+      l2z = 2. - 2. * rho;                    // mean (zx - zm)^2 = 2 - 2 rho
+    } else {
+      l2z = (sd_x > 0. || sd_m > 0.) ? 1. : 0.;   // a constant vector z-scores to zero
+    }
+    double g[kNumMetrics] = {u.s[5] / n, l2z, (double)u.flips / n};
+    double st[kNumStats] = {mean_x, var_x, sqrt(sq_x), mean_m, var_m, cov, sqrt(sq_m), rho};
+    if (nonfinite) {
+      for (int i = 0; i < kNumMetrics; ++i) g[i] = CUDART_NAN;
+      for (int i = 0; i < kNumStats; ++i) st[i] = CUDART_NAN;
+    }
+    for (int i = 0; i < kNumMetrics; ++i) s_gamma[tid][i] = g[i];
+    if (a.scores_out)
+      for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = (float)g[i];
+    if (a.stats_out)
+      for (int i = 0; i < kNumStats; ++i) a.stats_out[tid * kNumStats + i] = (float)st[i];
+
+    if (nonfinite) {
+      my_flag = kFlagNonfinite;
+    } else if (a.mode == kModeVerify) {
+      const int L = (tid == 0) ? 0 : 1;
+      for (int i = 0; i < kNumMetrics; ++i) {
+        // CTA 0 of this launch may have rewritten the thresholds: read them from L2
+        if (!__ldcg(&ks->has_thr[L][i])) { s_no_thr = 1; continue; }
+        if (!((a.metric_mask >> i) & 1u)) continue;
+        const double q2 = __ldcg(&ks->thr[L][i][1]);
+        const double tau_lower = __ldcg(&ks->thr[L][i][4]), tau_upper = __ldcg(&ks->thr[L][i][5]);
+        if (g[i] < tau_lower || g[i] > tau_upper) my_flag |= (1u << i);
+        if (tid == 0 && fabs(g[i] - q2) >= a.severe_mult * (tau_upper - q2)) s_severe = 1;
+      }
+    }
+    s_flag[tid] = my_flag;
+  }
+  const int any_flag = __syncthreads_or(my_flag != 0u);
+
+  if (tid == 0 && a.mode != kModeDistance) {
+    HandleState *hs = a.hs;
+    unsigned status = 0u;
+    if (a.mode == kModeVerify) {
+      ks->steps += 1;
+      if (any_flag) {                            // violation counter with forgiveness
+        hs->violations += 1;
+        hs->clean_streak = 0;
+        if (hs->violations >= a.ban_violations || s_severe) hs->banned = 1;
+      } else {
+        hs->clean_streak += 1;
+        if (hs->clean_streak >= a.forgiveness_steps) {
+          hs->violations = hs->violations > 0 ? hs->violations - 1 : 0;
+          hs->clean_streak = 0;
+        }
+      }
+      for (int r = 0; r < rows; ++r)             // only clean units join the history
+        if (!s_flag[r]) push_history(ks, a.hist, r ? 1 : 0, r ? a.cap1 : a.cap0, a.cap0, s_gamma[r]);
+      ks->refresh_pending = 1;
+      if (!any_flag) { ks->active ^= 1; status |= kFlagCommitted; }   // m_t := candidate
+      if (s_severe) status |= kFlagSevere;
+      if (hs->banned) status |= kFlagBanned;
+      if (s_no_thr) status |= kFlagNoThresholds;
+    } else {                                     // warm-up: everything joins, always commit
+      ks->steps += 1;
+      if (!any_flag) {                           // (any_flag here means non-finite input)
+        for (int r = 0; r < rows; ++r)
+          push_history(ks, a.hist, r ? 1 : 0, r ? a.cap1 : a.cap0, a.cap0, s_gamma[r]);
+        ks->refresh_pending = 1;
+        ks->active ^= 1;
+      }
+    }
+    s_flag[0] |= status;
+  }
+  __syncthreads();
+  if (a.flags_out && tid < rows) a.flags_out[tid] = s_flag[tid];
+  if (tid == 0) *a.ticket = 0u;                  // ready for the next launch
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernels
+
+// grid = 1 + B*P CTAs.  CTA 0 owes no rows: it brings the thresholds up to date (if the last
+// step left that pending) while the others stream.  Every CTA then takes a ticket; whoever
+// draws the last one has, by the fence/atomic order, everybody's partial sums and the fresh
+// thresholds in view, and finalizes.  No CTA ever waits for another.
+__global__ void __launch_bounds__(kThreads)
+stream_kernel(const StreamArgs a) {
+  __shared__ unsigned long long s_part[kWarps][kSlotWords];
+  __shared__ double s_sort[kMaxWindow];
+  __shared__ int s_last;
+
+  const float *m_in;
+  float *m_out;
+  if (a.mode == kModeDistance) {
+    m_in = a.m_ext;
+    m_out = nullptr;
+  } else {
+    const int act = __ldcg(&a.hs->kind[a.kind].active);   // written by an earlier launch only
+    m_in = a.ema[act];
+    m_out = a.ema[act ^ 1];
+  }
+
+  if (blockIdx.x == 0) {
+    if (a.hs) {
+      KindState *ks = &a.hs->kind[a.kind];
+      if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.cap0, a.cap1, a.a5, s_sort);
+    }
+  } else {
+    stream_piece(a, blockIdx.x - 1, m_in, m_out, s_part);
+  }
+
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(a.ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  finalize(a, m_in);
+}
+
+// Brings both kinds' thresholds up to date outside a streaming launch (queries, export).
+__global__ void __launch_bounds__(kThreads)
+refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, int cap0, int cap1,
+               Alg5Params a5_act, Alg5Params a5_grad) {
+  __shared__ double s_sort[kMaxWindow];
+  if (hs->kind[0].refresh_pending) refresh_thresholds(&hs->kind[0], hist_act, cap0, cap1, a5_act, s_sort);
+  __syncthreads();
+  if (hs->kind[1].refresh_pending) refresh_thresholds(&hs->kind[1], hist_grad, cap0, cap1, a5_grad, s_sort);
+}
+
+__global__ void reset_worker_kernel(HandleState *hs) {
+  hs->violations = 0;
+  hs->clean_streak = 0;
+  hs->banned = 0;
+}
+
+}  // namespace sentinel

@@ -1,0 +1,103 @@
+"""Shared helpers of the GPU parity tests: tolerances, oracle <-> library state blobs."""
+from __future__ import annotations
+
+import struct
+
+import numpy as np
+
+REL = 1e-3            # statistics and scores: relative error allowed against the float64 oracle
+MAGIC = 0x4C454E49544E4553
+METRIC_MASK = 0x7
+UNIT_BITS = 0xFFFF
+
+
+def assert_scores_close(gpu, ref, x_scale, what=""):
+    """|gpu - ref| <= 1e-3 * max(|ref|, floor).  Floors: 1e-3 for the bounded scores (L2z in
+    [0,4], SFR in [0,1]: an absolute 1e-6, the resolution fp32 products leave on a
+    correlation), 1e-3 * mean|x| for L1."""
+    gpu = np.asarray(gpu, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
+    floors = np.array([1e-3 * x_scale, 1e-3, 1e-3])
+    both_nan = np.isnan(gpu) & np.isnan(ref)
+    tol = REL * np.maximum(np.abs(ref), floors)
+    bad = ~both_nan & ~(np.abs(gpu - ref) <= tol)
+    assert not bad.any(), "%s scores differ: gpu=%s ref=%s" % (what, gpu[bad][:6], ref[bad][:6])
+
+
+def assert_stats_close(gpu, ref, x_scale, m_scale, what=""):
+    """Same rule for mean_x var_x |x| mean_m var_m cov |m| rho; floors follow each
+    quantity's natural scale (a mean is compared on the scale of the standard deviation)."""
+    gpu = np.asarray(gpu, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    sx, sm = max(x_scale, 1e-30), max(m_scale, 1e-30)
+    floors = np.array([sx, sx * sx, sx, sm, sm * sm, sx * sm, sm, 1.0]) * 1e-3
+    both_nan = np.isnan(gpu) & np.isnan(ref)
+    tol = REL * np.maximum(np.abs(ref), floors)
+    bad = ~both_nan & ~(np.abs(gpu - ref) <= tol)
+    assert not bad.any(), "%s stats differ: gpu=%s ref=%s" % (what, gpu[bad][:6], ref[bad][:6])
+
+
+def near_threshold(scores, thr, valid, B, rel=REL):
+    """Rows whose score lies within `rel` of a bound it is tested against (oracle values)."""
+    near = np.zeros(1 + B, dtype=bool)
+    for r in range(1 + B):
+        L = 0 if r == 0 else 1
+        for i in range(3):
+            if not valid[L, i] or np.isnan(scores[r, i]):
+                continue
+            for bound in (thr[L, i, 4], thr[L, i, 5]):
+                if abs(scores[r, i] - bound) <= rel * max(abs(bound), 1e-30):
+                    near[r] = True
+    return near
+
+
+# ---------------------------------------------------------------------------------------------
+# state blobs (layout documented in include/sentinel.h)
+
+def oracle_to_blob(v, params) -> bytes:
+    """Serialise an oracle verifier into the library's checkpoint format."""
+    B, T, d, l = params.B, params.T, params.d, params.l
+    viol, streak, banned = v.counters()
+    out = bytearray(struct.pack("<QI7i", MAGIC, 1, B, T, d, l, viol, streak, banned))
+    out += b"\0" * (64 - len(out))
+    for kind in (0, 1):
+        thr, valid = v.thresholds(kind)
+        counts = [v.history(kind, L, 0).size for L in (0, 1)]
+        out += struct.pack("<q2i6i", v.steps(kind), *counts, *valid.astype(int).reshape(-1))
+        out += thr.astype("<f8").tobytes()
+        for L, cap in ((0, l), (1, l * B)):
+            for i in range(3):
+                h = np.zeros(cap)
+                hv = v.history(kind, L, i)
+                h[:hv.size] = hv
+                out += h.astype("<f8").tobytes()
+        out += v.ema(kind).astype("<f4").tobytes()
+    return bytes(out)
+
+
+def parse_blob(blob, B, T, d, l) -> dict:
+    """Decode a checkpoint blob into plain numpy pieces."""
+    buf = memoryview(bytes(blob))
+    magic, version, b, t, dd, ll, viol, streak, banned = struct.unpack_from("<QI7i", buf, 0)
+    assert magic == MAGIC and version == 1 and (b, t, dd, ll) == (B, T, d, l)
+    off = 64
+    out = {"violations": viol, "clean_streak": streak, "banned": banned, "kinds": []}
+    N = B * T * d
+    for _ in range(2):
+        steps, c0, c1 = struct.unpack_from("<q2i", buf, off)
+        valid = np.array(struct.unpack_from("<6i", buf, off + 16)).reshape(2, 3).astype(bool)
+        off += 40
+        thr = np.frombuffer(buf, dtype="<f8", count=36, offset=off).reshape(2, 3, 6).copy()
+        off += 288
+        hist = [[None] * 3, [None] * 3]
+        for L, cap, cnt in ((0, l, c0), (1, l * B, c1)):
+            for i in range(3):
+                hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
+                off += 8 * cap
+        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape(B, T, d).copy()
+        off += 4 * N
+        out["kinds"].append({"steps": steps, "count": (c0, c1), "valid": valid, "thr": thr,
+                             "hist": hist, "m": m})
+    assert off == len(buf)
+    return out

@@ -1,0 +1,495 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle on
+the same seeded inputs.  Scores/statistics within 1e-3 relative, decisions bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import (UNIT_BITS, assert_scores_close, assert_stats_close, near_threshold,
+                     oracle_to_blob, parse_blob)
+from paper_2603_03592_b200 import synth
+
+pytestmark = pytest.mark.gpu
+ACT, GRAD = 0, 1
+
+
+@pytest.fixture(scope="module")
+def sb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_03592_b200 import binding
+    binding.lib()                      # a missing library is an error, never a fallback
+    return binding
+
+
+def dev(a, dtype):
+    return torch.as_tensor(np.ascontiguousarray(a)).to(dtype).cuda()
+
+
+def run_distance(sb, x_bf16, m_f32):
+    B = x_bf16.shape[0]
+    scores = torch.empty(1 + B, 3, dtype=torch.float32, device="cuda")
+    stats = torch.empty(1 + B, 8, dtype=torch.float32, device="cuda")
+    sb.sentinel_distance(x_bf16, m_f32, scores, stats)
+    torch.cuda.synchronize()
+    return scores.cpu().numpy(), stats.cpu().numpy()
+
+
+def oracle_distance_all(oracle_mod, xb, m64):
+    B = xb.shape[0]
+    g = np.empty((1 + B, 3))
+    s = np.empty((1 + B, 8))
+    g[0], s[0], _ = oracle_mod.distance(xb, m64)
+    for b in range(B):
+        g[1 + b], s[1 + b], _ = oracle_mod.distance(xb[b], m64[b])
+    return g, s
+
+
+SHAPES = [(1, 1, 8), (2, 3, 8), (1, 7, 16), (3, 5, 520), (4, 33, 1024), (8, 128, 512),
+          (2, 19, 4104), (5, 64, 2048), (64, 2, 64), (3, 1, 8192), (2, 300, 136)]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_distance_matches_oracle_over_shapes(sb, oracle_mod, shape):
+    """Stateless Omega_i(x, m): tiny, ragged (d not a multiple of the warp tile), multi-tile."""
+    B, T, d = shape
+    g = torch.Generator(device="cuda").manual_seed(1000 + B * 7 + T * 13 + d)
+    x = (torch.randn(B, T, d, generator=g, device="cuda") * 1.7 + 0.3).to(torch.bfloat16)
+    m = (0.6 * x.float() + 0.8 * torch.randn(B, T, d, generator=g, device="cuda")).contiguous()
+    scores, stats = run_distance(sb, x, m)
+    ref_g, ref_s = oracle_distance_all(oracle_mod, synth.bits(x), m.double().cpu().numpy())
+    scale = float(x.float().abs().mean())
+    assert_scores_close(scores, ref_g, scale, str(shape))
+    assert_stats_close(stats, ref_s, float(x.float().std()) if x.numel() > 1 else scale,
+                       float(m.std()) if m.numel() > 1 else scale, str(shape))
+
+
+def test_distance_degenerate_inputs(sb, oracle_mod):
+    B, T, d = 3, 9, 264
+    g = torch.Generator(device="cuda").manual_seed(5)
+    rnd = torch.randn(B, T, d, generator=g, device="cuda")
+    cases = {
+        "zero_reference": (rnd.to(torch.bfloat16), torch.zeros(B, T, d, device="cuda")),
+        "constant_x": (torch.full((B, T, d), -1.0, device="cuda").to(torch.bfloat16), rnd.clone()),
+        "constant_both": (torch.full((B, T, d), 2.0, device="cuda").to(torch.bfloat16),
+                          torch.full((B, T, d), 0.03, device="cuda")),
+        "all_zero": (torch.zeros(B, T, d, device="cuda").to(torch.bfloat16), torch.zeros(B, T, d, device="cuda")),
+        "identical": (rnd.to(torch.bfloat16), rnd.to(torch.bfloat16).float()),
+        "large_mean": ((rnd * 0.5 + 40.0).to(torch.bfloat16), rnd * 0.5 + 40.0),
+    }
+    xz = rnd.clone()
+    xz[:, ::3] = 0.0
+    xz[:, 1::5] = -0.0
+    cases["signed_zeros"] = (xz.to(torch.bfloat16), torch.zeros(B, T, d, device="cuda"))
+    one_const = rnd.clone()
+    one_const[1] = 0.75                              # one sample constant, the tensor is not
+    cases["one_constant_sample"] = (one_const.to(torch.bfloat16), rnd * 0.1)
+    for name, (x, m) in cases.items():
+        scores, stats = run_distance(sb, x, m.contiguous())
+        ref_g, ref_s = oracle_distance_all(oracle_mod, synth.bits(x), m.double().cpu().numpy())
+        scale = max(float(x.float().abs().mean()), 1e-3)
+        assert_scores_close(scores, ref_g, scale, name)
+        assert_stats_close(stats, ref_s, max(float(x.float().std()), 1e-3), max(float(m.std()), 1e-3), name)
+        if name in ("constant_x", "constant_both", "all_zero"):
+            assert np.all(stats[:, 1] == 0.0), name          # variance of a constant: exactly 0
+        if name == "one_constant_sample":
+            assert stats[2, 1] == 0.0 and scores[2, 1] == pytest.approx(1.0, rel=1e-6)
+        if name == "signed_zeros":
+            assert scores[0, 2] == pytest.approx(np.count_nonzero(x.float().cpu().numpy()) / x.numel(), rel=1e-6)
+
+
+def test_distance_non_finite_units(sb, oracle_mod):
+    B, T, d = 4, 6, 128
+    g = torch.Generator(device="cuda").manual_seed(6)
+    x = torch.randn(B, T, d, generator=g, device="cuda")
+    x[1, 2, 77] = float("inf")
+    x[3, 5, 127] = float("nan")
+    x = x.to(torch.bfloat16)
+    m = torch.randn(B, T, d, generator=g, device="cuda")
+    scores, stats = run_distance(sb, x, m)
+    ref_g, _ = oracle_distance_all(oracle_mod, synth.bits(x), m.double().cpu().numpy())
+    assert np.all(np.isnan(scores[[0, 2, 4]])) and np.all(np.isnan(stats[[0, 2, 4]]))
+    assert_scores_close(scores, ref_g, 0.8, "nonfinite")
+
+
+def test_scaling_and_permutation_invariants_on_gpu(sb):
+    B, T, d = 2, 64, 256
+    g = torch.Generator(device="cuda").manual_seed(7)
+    x = torch.randn(B, T, d, generator=g, device="cuda").to(torch.bfloat16)
+    m = torch.randn(B, T, d, generator=g, device="cuda")
+    s1, t1 = run_distance(sb, x, m)
+    s8, t8 = run_distance(sb, (x.float() * -8).to(torch.bfloat16), m)
+    assert t8[:, 2] == pytest.approx(8 * t1[:, 2], rel=1e-6)         # norm scales by |c|
+    assert t8[:, 1] == pytest.approx(64 * t1[:, 1], rel=1e-5)        # variance by c^2
+    perm = torch.randperm(T, generator=g, device="cuda")
+    sp, tp = run_distance(sb, x[:, perm].contiguous(), m[:, perm].contiguous())
+    assert sp == pytest.approx(s1, rel=1e-5)
+    assert tp[:, :3] == pytest.approx(t1[:, :3], rel=1e-5, abs=1e-7)
+
+
+# ---------------------------------------------------------------------------------------------
+# stateful path
+
+def make_pair(sb, oracle_mod, w, **kw):
+    okw = dict(kw)
+    gkw = {}
+    names = {"l": "window_steps", "c": "ban_violations", "t_forgiveness": "forgiveness_steps",
+             "gamma_g": "gamma_grow", "gamma_s": "gamma_shrink", "lam": "lambda_min", "eps": "iqr_eps"}
+    for k, v in kw.items():
+        gkw[names.get(k, k)] = v
+    gv = sb.Verifier(w.B, w.T, w.d, **gkw)
+    params = oracle_mod.Params(B=w.B, T=w.T, d=w.d, **okw)
+    return gv, oracle_mod.Verifier(params), params
+
+
+def compare_thresholds(gv, ov, kind, rel=1e-3):
+    """The multiplier k moves by whole factors, so it must agree to rounding; quartiles and
+    bounds are functions of scores that agree to 1e-3, and tau = q2 -+ k*IQR can cancel, so
+    they are compared on the scale of the median."""
+    gt, gvalid = gv.sentinel_get_thresholds(kind)
+    ot, ovalid = ov.thresholds(kind)
+    assert np.array_equal(gvalid, ovalid)
+    for L in range(2):
+        for i in range(3):
+            if ovalid[L, i]:
+                assert gt[L, i, 3] == pytest.approx(ot[L, i, 3], rel=1e-12), "multiplier k"
+                tol = rel * np.maximum(np.abs(ot[L, i]), abs(ot[L, i, 1]))
+                assert np.all(np.abs(gt[L, i] - ot[L, i]) <= tol), (L, i, gt[L, i], ot[L, i])
+
+
+def multiplier_events(gv, ov, params, kind):
+    """Alg. 5 compares every window entry with a fence; an entry that lies on a fence to within
+    the score tolerance may fall on either side, which moves k by one whole widen/narrow step.
+    Returns the number of (level, metric) windows where that happened; anything else fails."""
+    gt, gvalid = gv.sentinel_get_thresholds(kind)
+    ot, ovalid = ov.thresholds(kind)
+    assert np.array_equal(gvalid, ovalid)
+    events = 0
+    lg, ls = np.log(params.gamma_g[kind]), np.log(params.gamma_s[kind])
+    for L in range(2):
+        for i in range(3):
+            if not ovalid[L, i] or gt[L, i, 3] == pytest.approx(ot[L, i, 3], rel=1e-12):
+                continue
+            r = np.log(gt[L, i, 3] / ot[L, i, 3])
+            n = params.n_max[kind]
+            whole = any(abs(r - (a * lg + b * ls)) < 1e-9 for a in range(-n, n + 1) for b in range(-n, n + 1))
+            assert whole, "k differs by no whole number of steps: %r vs %r" % (gt[L, i, 3], ot[L, i, 3])
+            events += 1
+    return events
+
+
+def lockstep(sb, oracle_mod, w, gv, ov, params, steps, boundary=0, kinds=(ACT, GRAD), resync=True):
+    """Runs the stream of workload `w` through both sides.  Returns per-step records."""
+    near_events, flagged_steps, corrupted, k_events = 0, 0, 0, 0
+    for t in range(steps):
+        for kind in kinds:
+            x, name = synth.microbatch(w, boundary, kind, t, "cuda")
+            xb = synth.bits(x)
+            scale = max(float(x.float().abs().mean()), 1e-12)
+            if t < w.warmup:
+                gs = gv.update_reference(x, kind)
+                os_, _ = ov.update_reference(xb, kind)
+                torch.cuda.synchronize()
+                assert_scores_close(gs.cpu().numpy(), os_, scale, "warm-up step %d kind %d" % (t, kind))
+                ev = multiplier_events(gv, ov, params, kind)
+                if ev:
+                    k_events += ev
+                    gv.sentinel_import_state(oracle_to_blob(ov, params))
+                continue
+            corrupted += name is not None
+            thr, valid = ov.thresholds(kind)
+            gs, gf = gv.verify(x, kind)
+            os_, of, _ = ov.verify(xb, kind)
+            torch.cuda.synchronize()
+            gs, gf = gs.cpu().numpy(), gf.cpu().numpy().view(np.uint32)
+            assert_scores_close(gs, os_, scale, "step %d kind %d (%s)" % (t, kind, name))
+            flagged_steps += bool(np.any(of & UNIT_BITS))
+            if not np.array_equal(gf, of):
+                near = near_threshold(os_, thr, valid, w.B)
+                differ = (gf ^ of) & UNIT_BITS
+                assert np.all(near[differ != 0]), "flags differ away from a bound at step %d: %s vs %s" % (t, gf, of)
+                near_events += 1
+                assert resync, "near-threshold disagreement"
+                gv.sentinel_import_state(oracle_to_blob(ov, params))   # oracle -> library
+            ev = multiplier_events(gv, ov, params, kind)
+            if ev:
+                k_events += ev
+                gv.sentinel_import_state(oracle_to_blob(ov, params))
+    return {"near": near_events, "flagged": flagged_steps, "corrupted": corrupted, "k_events": k_events}
+
+
+def compare_state(gv, ov, params, m_scale_rel=1e-5):
+    st = parse_blob(gv.sentinel_export_state(), params.B, params.T, params.d, params.l)
+    assert (st["violations"], st["clean_streak"], st["banned"]) == ov.counters()
+    for kind in (ACT, GRAD):
+        ks = st["kinds"][kind]
+        assert ks["steps"] == ov.steps(kind)
+        m_ref = ov.ema(kind)
+        tol = m_scale_rel * max(float(np.abs(m_ref).max()), 1e-30)
+        assert np.max(np.abs(ks["m"].astype(np.float64) - m_ref)) <= tol
+        for L in range(2):
+            for i in range(3):
+                href = ov.history(kind, L, i)
+                assert ks["hist"][L][i].size == href.size
+                floor = 1e-3 * (np.abs(href).mean() if i == 0 and href.size else 1.0)
+                assert np.all(np.abs(ks["hist"][L][i] - href) <= 1e-3 * np.maximum(np.abs(href), floor))
+
+
+def test_config1_scenario(sb, oracle_mod):
+    """B=8 x T=128 x d=512, N(0,1): 16 clean warm-up microbatches, then sample 3 times 10."""
+    w = synth.WORKLOADS["cfg1"]
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, w.warmup, kinds=(ACT,))
+    compare_thresholds(gv, ov, ACT)
+    x, name = synth.microbatch(w, 0, ACT, w.warmup, "cuda")
+    assert name == "scale_sample3"
+    gs, gf = gv.verify(x, ACT)
+    os_, of, commit = ov.verify(synth.bits(x), ACT)
+    gf = gf.cpu().numpy().view(np.uint32)
+    assert np.array_equal(gf, of)
+    assert not commit and (gf[4] & sb.FLAG_L1) and not (gf[0] & sb.FLAG_COMMITTED)
+    assert_scores_close(gs.cpu().numpy(), os_, 0.8, "verify")
+    assert gs[4, 0] > 5 * gs[1, 0]
+    compare_state(gv, ov, params)
+    compare_thresholds(gv, ov, ACT)
+    assert rec["near"] == 0 and rec["k_events"] == 0
+    gv.close()
+
+
+STREAMS = [
+    ("cfg2", (6, 40, 1024), 60),       # lognormal channel scales; additive noise, gradient sign flips
+    ("cfg3", (4, 96, 520), 90),        # zeroed token rows, stale replays (needs > 50 steps)
+    ("cfg4", (4, 24, 2056), 50),       # Student-t activations; uniform noise on one sample
+]
+
+
+@pytest.mark.parametrize("name,shape,steps", STREAMS, ids=[s[0] for s in STREAMS])
+def test_streams_in_lockstep(sb, oracle_mod, name, shape, steps):
+    """The recipe of each benchmark configuration at a size the oracle finishes in seconds
+    (several row tiles, ragged d), with a corruption rate raised so that every kind occurs."""
+    w = synth.scaled(synth.WORKLOADS[name], name + "_small", *shape, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, steps)
+    assert rec["corrupted"] >= 5
+    compare_state(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+    assert rec["near"] <= 1 and rec["k_events"] <= 3, rec
+    print(name, rec)
+    gv.close()
+
+
+def test_many_boundaries_on_separate_streams(sb, oracle_mod):
+    """Config-5 pattern: independent handles, one CUDA stream each, interleaved act/grad."""
+    w = synth.scaled(synth.WORKLOADS["cfg5"], "cfg5_small", 4, 32, 512, corrupt_rate=0.2, boundaries=4)
+    pairs = [make_pair(sb, oracle_mod, w) for _ in range(w.boundaries)]
+    streams = [torch.cuda.Stream() for _ in range(w.boundaries)]
+    steps = w.warmup + 24
+    outs = []
+    for t in range(steps):
+        for b, ((gv, ov, params), s) in enumerate(zip(pairs, streams)):
+            for kind in (ACT, GRAD):
+                x, _ = synth.microbatch(w, b, kind, t, "cuda")
+                torch.cuda.current_stream().synchronize()
+                x.record_stream(s)
+                with torch.cuda.stream(s):
+                    if t < w.warmup:
+                        gv.update_reference(x, kind, stream=s)
+                        ov.update_reference(synth.bits(x), kind)
+                    else:
+                        gs, gf = gv.verify(x, kind, stream=s)
+                        os_, of, _ = ov.verify(synth.bits(x), kind)
+                        outs.append((gs, gf, os_, of, float(x.float().abs().mean())))
+    torch.cuda.synchronize()
+    for gs, gf, os_, of, scale in outs:
+        assert_scores_close(gs.cpu().numpy(), os_, scale, "multi-stream")
+        assert np.array_equal(gf.cpu().numpy().view(np.uint32), of)
+    for gv, ov, params in pairs:
+        compare_state(gv, ov, params)
+        gv.close()
+
+
+def test_import_oracle_state_then_verify(sb, oracle_mod):
+    """Load the oracle's state into the library and compare one verified step: isolates the
+    finalize logic from differences accumulated in the history."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_tiny", 3, 16, 264)
+    gv, ov, params = make_pair(sb, oracle_mod, w, l=7)
+    for t in range(12):                                  # more steps than the window holds
+        for kind in (ACT, GRAD):
+            ov.update_reference(synth.bits(synth.clean(w, 0, kind, t, "cuda")), kind)
+    gv.sentinel_import_state(oracle_to_blob(ov, params))
+    for kind in (ACT, GRAD):
+        gt, gvalid = gv.sentinel_get_thresholds(kind)
+        ot, ovalid = ov.thresholds(kind)
+        assert np.array_equal(gt, ot) and np.array_equal(gvalid, ovalid)     # exact round trip
+    for t in range(12, 20):
+        for kind in (ACT, GRAD):
+            x = synth.clean(w, 0, kind, t, "cuda")
+            if t == 15:
+                x = (x.float() * 2.5).to(torch.bfloat16)
+            gs, gf = gv.verify(x, kind)
+            os_, of, _ = ov.verify(synth.bits(x), kind)
+            assert np.array_equal(gf.cpu().numpy().view(np.uint32), of)
+            assert_scores_close(gs.cpu().numpy(), os_, float(x.float().abs().mean()), "after import")
+            compare_thresholds(gv, ov, kind)
+    compare_state(gv, ov, params)
+    # export -> import into a fresh handle -> identical behaviour
+    blob = gv.sentinel_export_state()
+    gv2 = sb.Verifier(w.B, w.T, w.d, window_steps=7)
+    gv2.sentinel_import_state(blob)
+    x = synth.clean(w, 0, ACT, 20, "cuda")
+    a = gv.verify(x, ACT)
+    b = gv2.verify(x, ACT)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    assert bytes(gv.sentinel_export_state()) == bytes(gv2.sentinel_export_state())
+    gv.close(); gv2.close()
+
+
+def test_counters_ban_forgiveness_and_reset(sb, oracle_mod):
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "cfg1_small", 4, 16, 128)
+    gv, ov, params = make_pair(sb, oracle_mod, w, c=3, t_forgiveness=4)
+    for t in range(16):
+        x = synth.clean(w, 0, ACT, t, "cuda")
+        gv.update_reference(x, ACT)
+        ov.update_reference(synth.bits(x), ACT)
+    script = [3.0, 1, 1, 1, 1, 1, 3.0, 1, 3.0, 3.0, 1, "reset", 1, 4096.0, 1]
+    t = 16
+    for item in script:
+        if item == "reset":
+            gv.sentinel_reset_worker()
+            ov.reset_worker()
+            continue
+        x = (synth.clean(w, 0, ACT, t, "cuda").float() * float(item)).to(torch.bfloat16)
+        t += 1
+        gs, gf = gv.verify(x, ACT)
+        os_, of, _ = ov.verify(synth.bits(x), ACT)
+        assert np.array_equal(gf.cpu().numpy().view(np.uint32), of), item
+        c = gv.sentinel_get_counters()
+        assert (c["violations"], c["clean_streak"], c["banned"]) == ov.counters()
+        assert c["steps_act"] == ov.steps(ACT) and c["error"] == 0
+    assert of[0] & sb.FLAG_BANNED                       # the 4096x step was severe
+    gv.close()
+
+
+def test_non_finite_and_no_warmup_paths(sb, oracle_mod):
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "cfg1_small", 3, 8, 64)
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    x = synth.clean(w, 0, ACT, 0, "cuda")
+    gs, gf = gv.verify(x, ACT)                           # no warm-up at all
+    os_, of, _ = ov.verify(synth.bits(x), ACT)
+    assert np.array_equal(gf.cpu().numpy().view(np.uint32), of)
+    assert of[0] == (sb.FLAG_COMMITTED | sb.FLAG_NO_THRESHOLDS)
+    bad = synth.clean(w, 0, ACT, 1, "cuda").float()
+    bad[1, 3, 5] = float("nan")
+    bad = bad.to(torch.bfloat16)
+    gs, gf = gv.verify(bad, ACT)
+    os_, of, _ = ov.verify(synth.bits(bad), ACT)
+    assert np.array_equal(gf.cpu().numpy().view(np.uint32), of)
+    assert_scores_close(gs.cpu().numpy(), os_, 0.8, "nan step")
+    gv.update_reference(bad, ACT)                        # refused: nothing changes
+    ov.update_reference(synth.bits(bad), ACT)
+    compare_state(gv, ov, params)
+    gv.close()
+
+
+def test_token_statistics_buffer(sb, oracle_mod):
+    """Per-token partial sums: sum_c x, sum_c x^2, sum_c |x-m|, sign mismatches, against their
+    definitions in float64 with the oracle's reference."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_tok", 3, 21, 392)
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    buf = torch.full((w.B, w.T, 4), -1.0, dtype=torch.float32, device="cuda")
+    gv.sentinel_set_token_stats_buffer(buf)
+    for t in range(3):
+        x = synth.clean(w, 0, ACT, t, "cuda")
+        m = ov.ema(ACT)
+        gv.update_reference(x, ACT)
+        ov.update_reference(synth.bits(x), ACT)
+        xv = oracle_mod.bf16_to_f64(synth.bits(x))
+        want = np.stack([xv.sum(-1), (xv * xv).sum(-1), np.abs(xv - m).sum(-1),
+                         (np.sign(xv) != np.sign(m)).sum(-1)], axis=-1)
+        got = buf.cpu().numpy().astype(np.float64)
+        scale = np.array([np.sqrt(w.d) * xv.std(), 1.0, 1.0, 1.0])
+        assert np.all(np.abs(got - want) <= 1e-3 * np.maximum(np.abs(want), scale))
+    gv.sentinel_set_token_stats_buffer(None)
+    buf.fill_(-1.0)
+    gv.update_reference(synth.clean(w, 0, ACT, 3, "cuda"), ACT)
+    torch.cuda.synchronize()
+    assert torch.all(buf == -1.0)
+    gv.close()
+
+
+def test_runs_are_bit_reproducible(sb):
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_rep", 4, 50, 1024)
+    blobs, outs = [], []
+    for _ in range(2):
+        gv = sb.Verifier(w.B, w.T, w.d)
+        o = []
+        for t in range(6):
+            for kind in (ACT, GRAD):
+                x, _ = synth.microbatch(w, 0, kind, t, "cuda")
+                o.append(gv.update_reference(x, kind) if t < 3 else gv.verify(x, kind)[0])
+        outs.append(torch.stack(o).cpu())
+        blobs.append(bytes(gv.sentinel_export_state()))
+        gv.close()
+    assert torch.equal(outs[0], outs[1])
+    assert blobs[0] == blobs[1]
+
+
+def test_verify_host_matches_device_call(sb):
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "cfg1_host", 4, 32, 256)
+    a, b = sb.Verifier(w.B, w.T, w.d), sb.Verifier(w.B, w.T, w.d)
+    for t in range(5):
+        x = synth.clean(w, 0, ACT, t, "cuda")
+        a.update_reference(x, ACT)
+        b.update_reference(x, ACT)
+    x = (synth.clean(w, 0, ACT, 5, "cuda").float() * 4).to(torch.bfloat16)
+    ds, df = a.verify(x, ACT)
+    hx = x.cpu().pin_memory()
+    hs = torch.empty(1 + w.B, 3, dtype=torch.float32).pin_memory()
+    hf = torch.empty(1 + w.B, dtype=torch.int32).pin_memory()
+    b.sentinel_verify_host(hx, ACT, hs, hf)
+    assert torch.equal(ds.cpu(), hs) and torch.equal(df.cpu(), hf)
+    a.close(); b.close()
+
+
+def test_argument_errors_never_reach_the_gpu(sb):
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(2, 4, 12)
+    assert e.value.code == sb.ERR_UNALIGNED
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(65, 4, 8)
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(64, 4, 8, window_steps=100)
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    for bad in (dict(beta=(1.0, 0.5)), dict(gamma_grow=(0.9, 1.1)), dict(window_steps=0), dict(device=99)):
+        with pytest.raises(sb.SentinelError) as e:
+            sb.Verifier(2, 4, 8, **bad)
+        assert e.value.code == sb.ERR_INVALID_ARG
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(0, 4, 8)
+    assert e.value.code == sb.ERR_INVALID_ARG
+
+    v = sb.Verifier(2, 4, 16)
+    x = torch.zeros(2, 4, 16, dtype=torch.bfloat16, device="cuda")
+    scores = torch.zeros(3, 3, device="cuda")
+    flags = torch.zeros(3, dtype=torch.int32, device="cuda")
+    before = bytes(v.sentinel_export_state())
+    L, h = sb.lib(), v._h
+    s = torch.cuda.current_stream().cuda_stream
+    assert L.sentinel_verify(h, x.data_ptr(), 0, 2, 4, 8, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_SHAPE_MISMATCH
+    assert b"differs" in L.sentinel_last_error(h)
+    assert L.sentinel_verify(h, x.data_ptr() + 2, 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_UNALIGNED
+    assert L.sentinel_verify(h, x.data_ptr(), 2, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_INVALID_ARG
+    assert L.sentinel_verify(h, None, 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_INVALID_ARG
+    assert L.sentinel_verify(h, x.data_ptr(), 0, 2, 4, 16, s, None, flags.data_ptr()) == sb.ERR_INVALID_ARG
+    assert L.sentinel_verify(None, x.data_ptr(), 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_INVALID_ARG
+    assert L.sentinel_update_reference(h, x.data_ptr(), 0, 3, 4, 16, s, None) == sb.ERR_SHAPE_MISMATCH
+    assert L.sentinel_export_state(h, bytes(8), 8, s) == sb.ERR_STATE_SIZE
+    junk = bytearray(before)
+    junk[0] ^= 0xFF
+    assert L.sentinel_import_state(h, bytes(junk), len(junk), s) == sb.ERR_STATE_SIZE
+    assert L.sentinel_distance(x.data_ptr(), None, 2, 4, 16, 0, s, scores.data_ptr(), None) == sb.ERR_INVALID_ARG
+    assert L.sentinel_distance(x.data_ptr(), scores.data_ptr(), 2, 4, 12, 0, s, scores.data_ptr(), None) == sb.ERR_UNALIGNED
+    torch.cuda.synchronize()
+    assert bytes(v.sentinel_export_state()) == before      # none of the above touched the state
+    v.close()

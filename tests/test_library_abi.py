@@ -1,0 +1,88 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU and exports every entry point that
+include/sentinel.h declares (no compute calls here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def built():
+    from paper_2603_03592_b200 import _build
+    return _build.build()
+
+
+def declared_entry_points():
+    text = open(os.path.join(ROOT, "include", "sentinel.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sentinel_[a-z_]+)\s*\(", text)))
+
+
+def test_header_declares_the_named_calls():
+    names = declared_entry_points()
+    for must in ("sentinel_verifier_create", "sentinel_verify", "sentinel_update_reference", "sentinel_destroy"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(built):
+    lib = ctypes.CDLL(built)
+    for name in declared_entry_points():
+        assert hasattr(lib, name), name
+
+
+def test_binding_mirrors_the_header(built):
+    from paper_2603_03592_b200 import binding
+    assert sorted(binding.EXPORTS) == declared_entry_points()
+    binding.lib()
+    for name in binding.EXPORTS:
+        if name in ("sentinel_default_config", "sentinel_distance"):
+            assert hasattr(binding, name)
+        elif name not in ("sentinel_verifier_create", "sentinel_last_error"):
+            assert hasattr(binding.Verifier, name), name
+
+
+def test_default_config_matches_the_paper_table(built):
+    """Host-only call: the library's defaults against the golden copy of the paper's table."""
+    from paper_2603_03592_b200 import binding
+    cfg = binding.sentinel_default_config()
+    want = {}
+    with open(os.path.join(ROOT, "tests", "golden", "hyperparams_table.txt")) as fh:
+        for line in fh:
+            if line.startswith("#") or not line.strip():
+                continue
+            tok = line.split()
+            want[tok[0]] = tuple(float(v) for v in tok[1:])
+    for key, field in [("beta", "beta"), ("k0", "k0"), ("alpha", "alpha"), ("n_max", "n_max"),
+                       ("gamma_g", "gamma_grow"), ("gamma_s", "gamma_shrink"),
+                       ("lambda", "lambda_min"), ("eps", "iqr_eps")]:
+        assert tuple(getattr(cfg, field)) == want[key]
+    assert cfg.ban_violations == want["c"][0] and cfg.forgiveness_steps == want["t_forgiveness"][0]
+    assert cfg.window_steps == want["l"][0] and cfg.severe_mult == want["severe_mult"][0]
+    assert cfg.metric_mask == 7 and cfg.shrink_ratio == 0.5
+
+
+def test_host_side_argument_checks_need_no_gpu(built):
+    from paper_2603_03592_b200 import binding
+    L = binding.lib()
+    assert L.sentinel_default_config(None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_verifier_create(None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_destroy(None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_state_bytes(None) == 0
+    assert b"NULL" in L.sentinel_last_error(None)
+    cfg = binding.sentinel_default_config(B=2, T=4, d=12)
+    h = ctypes.c_void_p()
+    assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_UNALIGNED
+    assert not h.value
+
+
+def test_product_path_does_not_touch_the_oracle():
+    """Nothing under the package imports, reads or links the oracle."""
+    pkg = os.path.join(ROOT, "paper_2603_03592_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), os.path.join(dirpath, f)
