@@ -99,10 +99,10 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_stream(w, device, count):
+def build_stream(w, device, count, distinct):
     """`count` microbatches per kind after the warm-up, following the workload's recipe."""
     xs = {ACT: [], GRAD: []}
-    n = min(count, MAX_DISTINCT)
+    n = min(count, distinct)
     for kind in (ACT, GRAD):
         for i in range(n):
             x, _ = synth.microbatch(w, 0, kind, w.warmup + i, device)
@@ -127,7 +127,7 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.synchronize()
 
     total = args.warmup + args.steps
-    xs = build_stream(w, device, total)
+    xs = build_stream(w, device, total, args.distinct)
     nd = len(xs[ACT])
     scores = torch.empty(2, 1 + w.B, 3, dtype=torch.float32, device=device)
     flags = torch.empty(2, 1 + w.B, dtype=torch.int32, device=device)
@@ -292,6 +292,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--distinct", type=int, default=MAX_DISTINCT,
+                    help="distinct input tensors per kind kept resident (they rotate beyond that)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--traffic", type=float, default=None,

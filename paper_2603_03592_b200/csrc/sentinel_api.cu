@@ -41,13 +41,14 @@ struct sentinel_verifier {
   sentinel_config cfg;
   size_t N = 0, Ns = 0;
   int cap0 = 0, cap1 = 0;
-  int P = 1, grid = 2;
+  int G = 1;                        // streaming CTAs; launches use G + 1
   float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
   HandleState *hs = nullptr;
   double *hist[2] = {nullptr, nullptr};
   unsigned long long *partials = nullptr;
   float *stats[2] = {nullptr, nullptr};
   float *token_buf = nullptr;
+  float *token_part = nullptr;      // per-tile token sums, allocated when a row spans several tiles
   void *stage_x = nullptr;          // staging for sentinel_verify_host, allocated on first use
   float *stage_scores = nullptr;
   unsigned *stage_flags = nullptr;
@@ -96,8 +97,9 @@ Alg5Params alg5_of(const sentinel_config &c, int kind) {
   return p;
 }
 
-// how many pieces each sample is cut into, and the grid that follows
-int pieces_per_sample(int device, int B, int T, int *grid_out, std::string *err) {
+// How many CTAs stream: every resident slot but the one of CTA 0, never more than there are
+// rows.  A CTA's rows may straddle one sample boundary at most, which needs G >= B.
+int streaming_ctas(int device, int B, int T, std::string *err) {
   int sms = 0, occ = 0;
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess)
@@ -106,13 +108,17 @@ int pieces_per_sample(int device, int B, int T, int *grid_out, std::string *err)
     if (err) *err = std::string("occupancy query failed: ") + cudaGetErrorString(e);
     return -1;
   }
-  const int resident = sms * occ;                   // one slot is CTA 0's
-  int P = (resident - 1) / B;
-  if (P < 1) P = 1;
-  if (P > T) P = T;
-  *grid_out = 1 + B * P;
-  return P;
+  long long G = (long long)sms * occ - 1;
+  const long long rows = (long long)B * T;
+  if (G > rows) G = rows;
+  if (G < B) {
+    if (err) *err = "this device keeps fewer CTAs resident than the tensor has samples";
+    return -1;
+  }
+  return (int)G;
 }
+
+int tiles_per_row(int d) { return ((d >> 3) + 32 * kUnroll - 1) / (32 * kUnroll); }
 
 int check_shape(sentinel_verifier *h, int B, int T, int d) {
   if (B < 1 || T < 1 || d < 1) return fail(h, SENTINEL_ERR_INVALID_ARG, "B, T, d must be positive (got %d, %d, %d)", B, T, d);
@@ -145,8 +151,9 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.flags_out = flags;
   a.stats_out = h->stats[kind];
   a.token_out = h->token_buf;
+  a.token_part = h->token_part;
   a.B = h->cfg.B; a.T = h->cfg.T; a.d = h->cfg.d;
-  a.P = h->P;
+  a.G = h->G;
   a.mode = mode;
   a.kind = kind;
   a.beta = (float)h->cfg.beta[kind];
@@ -191,6 +198,7 @@ void free_all(sentinel_verifier *h) {
   }
   cudaFree(h->hs);
   cudaFree(h->partials);
+  cudaFree(h->token_part);
   cudaFree(h->stage_x);
   cudaFree(h->stage_scores);
   cudaFree(h->stage_flags);
@@ -250,8 +258,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->cap0 = cfg->window_steps;
   h->cap1 = cfg->window_steps * cfg->B;
   std::string oerr;
-  h->P = pieces_per_sample(cfg->device, cfg->B, cfg->T, &h->grid, &oerr);
-  if (h->P < 1) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "%s", oerr.c_str()); }
+  h->G = streaming_ctas(cfg->device, cfg->B, cfg->T, &oerr);
+  if (h->G < 1) { delete h; return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str()); }
 
   cudaError_t e = cudaSuccess;
   auto alloc = [&](void **p, size_t bytes) {
@@ -263,7 +271,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     alloc((void **)&h->hist[k], hist_doubles(h) * sizeof(double));
     alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
   }
-  alloc((void **)&h->partials, (size_t)cfg->B * h->P * kSlotWords * sizeof(unsigned long long));
+  alloc((void **)&h->partials, (size_t)h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));
   alloc((void **)&h->hs, sizeof(HandleState));
   if (e == cudaSuccess) {
     HandleState init;
@@ -290,7 +298,7 @@ int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
   if (!dev_scores_out || !dev_flags_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
-  return launch(h, make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out), h->grid,
+  return launch(h, make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out), h->G + 1,
                 static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -300,7 +308,7 @@ int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_
   if (rc) return rc;
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
-  return launch(h, make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr), h->grid,
+  return launch(h, make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr), h->G + 1,
                 static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -321,7 +329,7 @@ int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind
     SENTINEL_CUDA(h, cudaMalloc((void **)&h->stage_flags, rows * sizeof(unsigned)));
   }
   SENTINEL_CUDA(h, cudaMemcpyAsync(h->stage_x, host_x, h->N * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
-  int rc = launch(h, make_args(h, h->stage_x, kind, kModeVerify, h->stage_scores, h->stage_flags), h->grid, s);
+  int rc = launch(h, make_args(h, h->stage_x, kind, kModeVerify, h->stage_scores, h->stage_flags), h->G + 1, s);
   if (rc) return rc;
   SENTINEL_CUDA(h, cudaMemcpyAsync(host_scores_out, h->stage_scores, rows * kNumMetrics * sizeof(float), cudaMemcpyDeviceToHost, s));
   SENTINEL_CUDA(h, cudaMemcpyAsync(host_flags_out, h->stage_flags, rows * sizeof(unsigned), cudaMemcpyDeviceToHost, s));
@@ -342,12 +350,11 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   SENTINEL_CUDA(nullptr, guard.status);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
 
-  int grid = 0;
   std::string oerr;
-  const int P = pieces_per_sample(device, B, T, &grid, &oerr);
-  if (P < 1) return fail(nullptr, SENTINEL_ERR_CUDA, "%s", oerr.c_str());
-  // scratch: one slot per piece, then the ticket word
-  const size_t slot_bytes = (size_t)B * P * kSlotWords * sizeof(unsigned long long);
+  const int G = streaming_ctas(device, B, T, &oerr);
+  if (G < 1) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str());
+  // scratch: two partial slots per streaming CTA, then the ticket word
+  const size_t slot_bytes = (size_t)G * kSegsPerCta * kSlotWords * sizeof(unsigned long long);
   unsigned char *scratch = nullptr;
   SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, slot_bytes + 256, s));
   SENTINEL_CUDA(nullptr, cudaMemsetAsync(scratch + slot_bytes, 0, 256, s));
@@ -360,9 +367,9 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   a.ticket = reinterpret_cast<unsigned *>(scratch + slot_bytes);
   a.scores_out = dev_scores_out;
   a.stats_out = dev_stats_out;
-  a.B = B; a.T = T; a.d = d; a.P = P;
+  a.B = B; a.T = T; a.d = d; a.G = G;
   a.mode = kModeDistance;
-  stream_kernel<<<grid, kThreads, 0, s>>>(a);
+  stream_kernel<<<G + 1, kThreads, 0, s>>>(a);
   cudaError_t le = cudaGetLastError();
   cudaError_t fe = cudaFreeAsync(scratch, s);
   SENTINEL_CUDA(nullptr, le);
@@ -419,6 +426,12 @@ int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_
 int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (dev_buf && !aligned16(dev_buf)) return fail(h, SENTINEL_ERR_UNALIGNED, "token buffer is not 16-byte aligned");
+  const int tpr = tiles_per_row(h->cfg.d);
+  if (dev_buf && tpr > 1 && !h->token_part) {      // rows of several tiles need a place for the shares
+    DeviceGuard guard(h->cfg.device);
+    SENTINEL_CUDA(h, guard.status);
+    SENTINEL_CUDA(h, cudaMalloc((void **)&h->token_part, (size_t)h->cfg.B * h->cfg.T * tpr * 4 * sizeof(float)));
+  }
   h->token_buf = dev_buf;
   return SENTINEL_OK;
 }

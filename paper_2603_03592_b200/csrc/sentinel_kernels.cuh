@@ -20,10 +20,11 @@ constexpr int kNumStats = 8;
 constexpr int kNumThr = 6;
 constexpr int kMaxB = 64;
 constexpr int kMaxWindow = 4096;
-constexpr int kThreads = 512;             // threads per CTA
+constexpr int kThreads = 640;             // threads per CTA: with kUnroll = 2 about 60 KB of loads
+                                          // in flight per SM, where the read/write mix peaked in sweeps
 constexpr int kWarps = kThreads / 32;
 constexpr int kSlotWords = 8;             // 64-bit words per partial slot
-constexpr int kUnroll = 4;                // 8-element chunks per lane per loop trip
+constexpr int kUnroll = 2;                // 8-element chunks per lane per loop trip
 
 enum Mode : int { kModeVerify = 0, kModeWarmup = 1, kModeDistance = 2 };
 
@@ -34,8 +35,10 @@ constexpr unsigned kFlagSevere = 1u << 17;
 constexpr unsigned kFlagBanned = 1u << 18;
 constexpr unsigned kFlagNoThresholds = 1u << 19;
 
-// bits of word 7 of a partial slot
+// word 7 of a partial slot: bits 0-2 flags, bits 8-15 tag (1 + sample index, 0 = slot unused),
+// bits 16-31 the sample's first x (bf16 bits), bits 32-63 the sample's first m (fp32 bits)
 constexpr unsigned long long kBitNonfinite = 1ull, kBitXVaries = 2ull, kBitMVaries = 4ull;
+constexpr int kTagShift = 8, kX0Shift = 16, kM0Shift = 32;
 
 struct Alg5Params {
   double alpha, gamma_g, gamma_s, lambda, eps, shrink_ratio;
@@ -67,14 +70,15 @@ struct StreamArgs {
   float *ema[2];                   // the two reference buffers of this kind
   HandleState *hs;                 // nullptr in distance mode
   double *hist;                    // this kind's rings: level 0 [3][cap0], level 1 [3][cap1]
-  unsigned long long *partials;    // [pieces][kSlotWords]
+  unsigned long long *partials;    // [G][2][kSlotWords]
   unsigned *ticket;
   float *scores_out;               // [(1+B)*3] or nullptr
   unsigned *flags_out;             // [1+B] or nullptr
   float *stats_out;                // [(1+B)*8] or nullptr
   float *token_out;                // [B,T,4] or nullptr
+  float *token_part;               // [B*T][tiles per row][4]: per-tile shares when a row has several tiles
   int B, T, d;
-  int P;                           // pieces per sample
+  int G;                           // streaming CTAs (the grid has one more)
   int mode, kind;
   float beta, one_minus_beta;
   int cap0, cap1;
@@ -128,12 +132,13 @@ __device__ __forceinline__ void element(float xf, float mf, float x0, float m0, 
   g.smm = fmaf(ms, ms, g.smm);
   g.sxm = fmaf(xs, ms, g.sxm);
   g.ab += fabsf(xf - mf);
-  const int sgx = (xf > 0.f) - (xf < 0.f);
-  const int sgm = (mf > 0.f) - (mf < 0.f);
-  g.flips += (sgx != sgm);
+  // sign(x) != sign(m) with sign in {-1,0,+1}: either exactly one of them is zero, or both are
+  // non-zero and x carrying the extra sign of m is negative
+  const float xt = __uint_as_float(__float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u));
+  g.flips += (((xf == 0.f) != (mf == 0.f)) || (xt < 0.f)) ? 1u : 0u;
 }
 
-struct ThreadAcc {           // carried over the whole piece
+struct ThreadAcc {           // carried over the CTA's rows of one sample
   double sx, sxx, sm, smm, sxm, ab;
   unsigned flips;
   unsigned nf_bits;          // non-zero: a bf16 exponent of all ones was seen
@@ -181,17 +186,26 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// streaming phase: CTA `piece` covers rows [r0, r1) of one sample; a warp owns whole rows
+// streaming phase
+//
+// Streaming CTA c owns the rows [c*R/G, (c+1)*R/G) of the flat [B*T, d] view (R = B*T rows, G
+// streaming CTAs), so every CTA moves the same number of bytes to within one row.  Inside the
+// CTA the rows are cut into warp tiles of 32*kUnroll chunks (512 elements) that never cross a
+// row, dealt round-robin to the warps, so the warps finish within one tile of each other.  A
+// CTA's rows can straddle one sample boundary (the host guarantees at most one), hence two
+// partial slots per CTA, each tagged with its sample.
 
-__device__ void stream_piece(const StreamArgs &a, int piece, const float *m_in, float *m_out,
-                             unsigned long long (*s_part)[kSlotWords]) {
+constexpr int kSegsPerCta = 2;
+
+__device__ void stream_segment(const StreamArgs &a, int b, long long ra, long long rb,
+                               const float *m_in, float *m_out,
+                               unsigned long long (*s_part)[kSlotWords],
+                               unsigned long long *slot) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int b = piece / a.P, p = piece - b * a.P;
-  const long long row_base = (long long)b * a.T;
-  const int r0 = (int)(((long long)p * a.T) / a.P);
-  const int r1 = (int)(((long long)(p + 1) * a.T) / a.P);
   const int chunks = a.d >> 3;
-  const size_t sample_off = (size_t)row_base * a.d;
+  const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
+  const int n_tiles = (int)(rb - ra) * tiles_per_row;       // < 2^31: rows/G * d/1024
+  const size_t sample_off = (size_t)b * a.T * a.d;
   const bool write_ema = (m_out != nullptr);
   const bool tokens = (a.token_out != nullptr);
   const float beta = a.beta, omb = a.one_minus_beta;
@@ -202,53 +216,73 @@ __device__ void stream_piece(const StreamArgs &a, int piece, const float *m_in, 
 
   ThreadAcc t = {0., 0., 0., 0., 0., 0., 0u, 0u, 0u, 0u};
 
-  for (int r = r0 + warp; r < r1; r += kWarps) {
-    const size_t off = (size_t)(row_base + r) * a.d;
-    const uint16_t *xrow = a.x + off;
-    const float *mrow = m_in + off;
-    float *orow = write_ema ? m_out + off : nullptr;
-    float tk_sx = 0.f, tk_sxx = 0.f, tk_ab = 0.f;
-    unsigned tk_flips = 0u;
+  // tile j = (row rr, segment seg); j advances by kWarps, so (rr, seg) advance by a fixed step
+  const int step_rr = kWarps / tiles_per_row, step_seg = kWarps % tiles_per_row;
+  int rr = warp / tiles_per_row, seg = warp % tiles_per_row;
+  for (int j = warp; j < n_tiles; j += kWarps) {
+    const long long row = ra + rr;
+    const size_t off = (size_t)row * a.d;
+    const int base = seg * 32 * kUnroll;
 
-    for (int base = 0; base < chunks; base += 32 * kUnroll) {
-      uint4 xv[kUnroll];
-      F8 mv[kUnroll];
-      bool ok[kUnroll];
+    uint4 xv[kUnroll];
+    F8 mv[kUnroll];
+    bool ok[kUnroll];
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int c = base + u * 32 + lane;
-        ok[u] = c < chunks;
-        if (ok[u]) {
-          xv[u] = ld_x128(xrow + (size_t)c * 8);
-          mv[u] = ld_m256(mrow + (size_t)c * 8);
-        }
+    for (int u = 0; u < kUnroll; ++u) {
+      const int c = base + u * 32 + lane;
+      ok[u] = c < chunks;
+      if (ok[u]) {
+        xv[u] = ld_x128(a.x + off + (size_t)c * 8);
+        mv[u] = ld_m256(m_in + off + (size_t)c * 8);
       }
-      GroupAcc g = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0u};
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        if (ok[u]) {
-          chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
-          if (write_ema) st_m256(orow + (size_t)(base + u * 32 + lane) * 8, mv[u]);
-        }
-      }
-      // fold the short fp32 run into the fp64 accumulators
-      t.sx += (double)g.sx;   t.sxx += (double)g.sxx;
-      t.sm += (double)g.sm;   t.smm += (double)g.smm;
-      t.sxm += (double)g.sxm; t.ab += (double)g.ab;
-      t.flips += g.flips;
-      if (tokens) { tk_sx += g.sx; tk_sxx += g.sxx; tk_ab += g.ab; tk_flips += g.flips; }
     }
-    if (tokens) {
-      tk_sx = warp_sum(tk_sx);
-      tk_sxx = warp_sum(tk_sxx);
-      tk_ab = warp_sum(tk_ab);
-      const float fl = warp_sum((float)tk_flips);
-      if (lane == 0) {                       // back from shifted to raw sums over the d channels
-        const float x0f = __uint_as_float(x0 << 16), dd = (float)a.d;
-        const float raw_sx = fmaf(dd, x0f, tk_sx);
-        const float raw_sxx = fmaf(dd * x0f, x0f, fmaf(2.f * x0f, tk_sx, tk_sxx));
-        reinterpret_cast<float4 *>(a.token_out)[row_base + r] = make_float4(raw_sx, raw_sxx, tk_ab, fl);
+    GroupAcc g = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0u};
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (ok[u]) {
+        chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
+        if (write_ema) st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
       }
+    }
+    // fold the short fp32 run into the fp64 accumulators
+    t.sx += (double)g.sx;   t.sxx += (double)g.sxx;
+    t.sm += (double)g.sm;   t.smm += (double)g.smm;
+    t.sxm += (double)g.sxm; t.ab += (double)g.ab;
+    t.flips += g.flips;
+
+    if (tokens) {                       // this tile's share of the token's sums
+      const float sx = warp_sum(g.sx), sxx = warp_sum(g.sxx), ab = warp_sum(g.ab);
+      const float fl = warp_sum((float)g.flips);
+      if (lane == 0) {
+        float4 *dst = (tiles_per_row == 1) ? reinterpret_cast<float4 *>(a.token_out) + row
+                                           : reinterpret_cast<float4 *>(a.token_part) + row * tiles_per_row + seg;
+        float4 v = make_float4(sx, sxx, ab, fl);
+        if (tiles_per_row == 1) {       // back from shifted to raw sums over the d channels
+          const float x0f = __uint_as_float(x0 << 16), dd = (float)a.d;
+          v.y = fmaf(dd * x0f, x0f, fmaf(2.f * x0f, sx, sxx));
+          v.x = fmaf(dd, x0f, sx);
+        }
+        *dst = v;
+      }
+    }
+    rr += step_rr;
+    seg += step_seg;
+    if (seg >= tiles_per_row) { seg -= tiles_per_row; ++rr; }
+  }
+
+  if (tokens && tiles_per_row > 1) {    // a row's tiles went to several warps: add them in order
+    __syncthreads();
+    const float x0f = __uint_as_float(x0 << 16), dd = (float)a.d;
+    for (long long row = ra + threadIdx.x; row < rb; row += kThreads) {
+      const float4 *src = reinterpret_cast<const float4 *>(a.token_part) + row * tiles_per_row;
+      float4 acc = __ldcg(src);
+      for (int sgm = 1; sgm < tiles_per_row; ++sgm) {
+        const float4 v = __ldcg(src + sgm);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      const float raw_sx = fmaf(dd, x0f, acc.x);
+      const float raw_sxx = fmaf(dd * x0f, x0f, fmaf(2.f * x0f, acc.x, acc.y));
+      reinterpret_cast<float4 *>(a.token_out)[row] = make_float4(raw_sx, raw_sxx, acc.z, acc.w);
     }
   }
 
@@ -260,6 +294,7 @@ __device__ void stream_piece(const StreamArgs &a, int piece, const float *m_in, 
                             (t.m_diff ? kBitMVaries : 0ull);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+  __syncthreads();                      // s_part may still be read from the previous segment
   if (lane == 0) {
 #pragma unroll
     for (int j = 0; j < 6; ++j) s_part[warp][j] = (unsigned long long)__double_as_longlong(ws[j]);
@@ -271,17 +306,37 @@ __device__ void stream_piece(const StreamArgs &a, int piece, const float *m_in, 
     const int j = threadIdx.x;
     unsigned long long out;
     if (j < 6) {
-      double s = 0.;
-      for (int w = 0; w < kWarps; ++w) s += __longlong_as_double((long long)s_part[w][j]);
-      out = (unsigned long long)__double_as_longlong(s);
+      double sum = 0.;
+      for (int w = 0; w < kWarps; ++w) sum += __longlong_as_double((long long)s_part[w][j]);
+      out = (unsigned long long)__double_as_longlong(sum);
     } else if (j == 6) {
       out = 0ull;
       for (int w = 0; w < kWarps; ++w) out += s_part[w][6];
     } else {
-      out = 0ull;
+      out = ((unsigned long long)(b + 1) << kTagShift) | ((unsigned long long)x0 << kX0Shift) |
+            ((unsigned long long)m0bits << kM0Shift);       // sample tag and the shift of the sums
       for (int w = 0; w < kWarps; ++w) out |= s_part[w][7];
     }
-    a.partials[(size_t)piece * kSlotWords + j] = out;
+    slot[j] = out;
+  }
+}
+
+__device__ void stream_cta(const StreamArgs &a, int c, const float *m_in, float *m_out,
+                           unsigned long long (*s_part)[kSlotWords]) {
+  const long long R = (long long)a.B * a.T;
+  const long long R0 = (R * c) / a.G, R1 = (R * (c + 1)) / a.G;
+  long long ra = R0;
+  for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
+    unsigned long long *slot = a.partials + ((size_t)c * kSegsPerCta + sgm) * kSlotWords;
+    if (ra < R1) {
+      const int b = (int)(ra / a.T);
+      const long long sample_end = (long long)(b + 1) * a.T;
+      const long long rb = sample_end < R1 ? sample_end : R1;
+      stream_segment(a, b, ra, rb, m_in, m_out, s_part, slot);
+      ra = rb;
+    } else if (threadIdx.x == 0) {
+      slot[7] = 0ull;                   // tag 0: unused
+    }
   }
 }
 
@@ -383,6 +438,7 @@ struct UnitSums {
   double s[6];               // sums of (x-x0) (x-x0)^2 (m-m0) (m-m0)^2 (x-x0)(m-m0) |x-m|
   unsigned long long flips;
   unsigned long long bits;
+  unsigned long long first;  // bits 0-15 first x (bf16), bits 16-47 first m (fp32)
   double x0, m0;             // the shift the sums were taken about
 };
 
@@ -400,7 +456,7 @@ __device__ __forceinline__ void push_history(KindState *ks, double *hist, int L,
   for (int i = 0; i < kNumMetrics; ++i) base[(size_t)i * cap + idx] = g[i];
 }
 
-__device__ void finalize(const StreamArgs &a, const float *m_in) {
+__device__ void finalize(const StreamArgs &a) {
   __shared__ UnitSums s_unit[kMaxB + 1];
   __shared__ double s_gamma[kMaxB + 1][kNumMetrics];
   __shared__ unsigned s_flag[kMaxB + 1];
@@ -412,29 +468,42 @@ __device__ void finalize(const StreamArgs &a, const float *m_in) {
 
   if (tid == 0) { s_severe = 0; s_no_thr = 0; }
 
-  // per-sample sums over that sample's pieces, in a fixed order
+  // per-sample sums over the slots tagged with that sample, in CTA order
   for (int b = warp; b < B; b += kWarps) {
     double v[6] = {0., 0., 0., 0., 0., 0.};
-    unsigned long long fl = 0ull, bits = 0ull;
-    for (int p = lane; p < a.P; p += 32) {
-      const unsigned long long *slot = a.partials + ((size_t)b * a.P + p) * kSlotWords;
+    unsigned long long fl = 0ull, bits = 0ull, first = 0ull;
+    // streaming CTAs whose rows can touch sample b (a superset; the tag decides)
+    const long long R = (long long)B * a.T;
+    long long c_lo = ((long long)b * a.T * a.G) / R - 1, c_hi = ((long long)(b + 1) * a.T * a.G + R - 1) / R;
+    if (c_lo < 0) c_lo = 0;
+    if (c_hi > a.G - 1) c_hi = a.G - 1;
+    const long long n_slots = (c_hi - c_lo + 1) * kSegsPerCta;
+    for (long long q = lane; q < n_slots; q += 32) {
+      const unsigned long long *slot = a.partials + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
+      const unsigned long long w7 = __ldcg(slot + 7);
+      if (((w7 >> kTagShift) & 0xFFull) != (unsigned long long)(b + 1)) continue;
 #pragma unroll
       for (int j = 0; j < 6; ++j) v[j] += __longlong_as_double((long long)__ldcg(slot + j));
       fl += __ldcg(slot + 6);
-      bits |= __ldcg(slot + 7);
+      bits |= w7 & 0x7ull;
+      first = w7 >> kX0Shift;            // the same in every slot of this sample
     }
 #pragma unroll
     for (int j = 0; j < 6; ++j) v[j] = warp_sum(v[j]);
     fl = warp_sum(fl);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+    for (int o = 16; o > 0; o >>= 1) {
+      bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+      first |= __shfl_xor_sync(0xffffffffu, first, o);
+    }
     if (lane == 0) {
 #pragma unroll
       for (int j = 0; j < 6; ++j) s_unit[1 + b].s[j] = v[j];
       s_unit[1 + b].flips = fl;
       s_unit[1 + b].bits = bits;
-      s_unit[1 + b].x0 = (double)__uint_as_float((unsigned)a.x[b * Ns] << 16);
-      s_unit[1 + b].m0 = (double)m_in[b * Ns];
+      s_unit[1 + b].first = first;
+      s_unit[1 + b].x0 = (double)__uint_as_float(((unsigned)first & 0xFFFFu) << 16);
+      s_unit[1 + b].m0 = (double)__uint_as_float((unsigned)(first >> 16));
     }
   }
   __syncthreads();
@@ -442,9 +511,7 @@ __device__ void finalize(const StreamArgs &a, const float *m_in) {
   // whole-tensor unit = the samples added up in order, re-centred on sample 0's shift:
   // sum (x-K) = sum (x-x0) + n dx,  sum (x-K)^2 = sum (x-x0)^2 + 2 dx sum (x-x0) + n dx^2, ...
   if (tid == 0) {
-    UnitSums u = {{0., 0., 0., 0., 0., 0.}, 0ull, 0ull, s_unit[1].x0, s_unit[1].m0};
-    const unsigned x_first = a.x[0];
-    const unsigned m_first = __float_as_uint(m_in[0]);
+    UnitSums u = {{0., 0., 0., 0., 0., 0.}, 0ull, 0ull, s_unit[1].first, s_unit[1].x0, s_unit[1].m0};
     const double n = (double)Ns;
     for (int b = 0; b < B; ++b) {
       const UnitSums &v = s_unit[1 + b];
@@ -457,8 +524,8 @@ __device__ void finalize(const StreamArgs &a, const float *m_in) {
       u.s[5] += v.s[5];
       u.flips += v.flips;
       u.bits |= v.bits;
-      if ((unsigned)a.x[b * Ns] != x_first) u.bits |= kBitXVaries;
-      if (__float_as_uint(m_in[b * Ns]) != m_first) u.bits |= kBitMVaries;
+      if ((v.first & 0xFFFFull) != (u.first & 0xFFFFull)) u.bits |= kBitXVaries;
+      if ((v.first >> 16) != (u.first >> 16)) u.bits |= kBitMVaries;
     }
     s_unit[0] = u;
   }
@@ -563,7 +630,7 @@ __device__ void finalize(const StreamArgs &a, const float *m_in) {
 // ---------------------------------------------------------------------------------------------
 // kernels
 
-// grid = 1 + B*P CTAs.  CTA 0 owes no rows: it brings the thresholds up to date (if the last
+// grid = 1 + G CTAs.  CTA 0 owes no rows: it brings the thresholds up to date (if the last
 // step left that pending) while the others stream.  Every CTA then takes a ticket; whoever
 // draws the last one has, by the fence/atomic order, everybody's partial sums and the fresh
 // thresholds in view, and finalizes.  No CTA ever waits for another.
@@ -590,7 +657,7 @@ stream_kernel(const StreamArgs a) {
       if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.cap0, a.cap1, a.a5, s_sort);
     }
   } else {
-    stream_piece(a, blockIdx.x - 1, m_in, m_out, s_part);
+    stream_cta(a, blockIdx.x - 1, m_in, m_out, s_part);
   }
 
   __threadfence();
@@ -602,7 +669,7 @@ stream_kernel(const StreamArgs a) {
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  finalize(a, m_in);
+  finalize(a);
 }
 
 // Brings both kinds' thresholds up to date outside a streaming launch (queries, export).

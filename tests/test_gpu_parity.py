@@ -391,10 +391,11 @@ def test_non_finite_and_no_warmup_paths(sb, oracle_mod):
     gv.close()
 
 
-def test_token_statistics_buffer(sb, oracle_mod):
+@pytest.mark.parametrize("d", [392, 1024, 2568])
+def test_token_statistics_buffer(sb, oracle_mod, d):
     """Per-token partial sums: sum_c x, sum_c x^2, sum_c |x-m|, sign mismatches, against their
-    definitions in float64 with the oracle's reference."""
-    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_tok", 3, 21, 392)
+    definitions in float64 with the oracle's reference; rows of one and of several tiles."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_tok", 3, 21, d)
     gv, ov, params = make_pair(sb, oracle_mod, w)
     buf = torch.full((w.B, w.T, 4), -1.0, dtype=torch.float32, device="cuda")
     gv.sentinel_set_token_stats_buffer(buf)
@@ -408,7 +409,11 @@ def test_token_statistics_buffer(sb, oracle_mod):
                          (np.sign(xv) != np.sign(m)).sum(-1)], axis=-1)
         got = buf.cpu().numpy().astype(np.float64)
         scale = np.array([np.sqrt(w.d) * xv.std(), 1.0, 1.0, 1.0])
-        assert np.all(np.abs(got - want) <= 1e-3 * np.maximum(np.abs(want), scale))
+        tol = 1e-3 * np.maximum(np.abs(want), scale)
+        # where the EMA cancels to zero up to rounding (bf16 inputs in the ratio -beta/(1-beta))
+        # its sign, hence one mismatch count, is decided by rounding noise on either side
+        tol[..., 3] += (np.abs(m) <= 1e-9 * np.abs(m).mean()).sum(-1)
+        assert np.all(np.abs(got - want) <= tol)
     gv.sentinel_set_token_stats_buffer(None)
     buf.fill_(-1.0)
     gv.update_reference(synth.clean(w, 0, ACT, 3, "cuda"), ACT)
