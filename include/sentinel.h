@@ -134,6 +134,28 @@ int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind
 int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d, int device,
                       void *cuda_stream, float *dev_scores_out, float *dev_stats_out);
 
+/* The same computation as sentinel_distance for callers that must not allocate device memory
+ * while they run: code whose memory pool has been frozen after start-up, real-time loops
+ * that cannot afford an allocator call of unbounded duration, and processes whose
+ * device-memory budget was handed out up front and may not grow.  (The paper
+ * has no counterpart; this is a property of the library, not of the method.)
+ * The kernel's scratch (two 64-byte partial slots per streaming CTA plus a ticket word) lives
+ * in a fixed array of SENTINEL_NOALLOC_SCRATCH_BYTES that is part of the library image, so
+ * every GPU that loads the library holds those bytes until the process exits.  The call
+ * performs no cudaMalloc / cudaFree / pool allocation of any kind; inputs and outputs are
+ * still the caller's.  If this device's launch needs more scratch than the array holds the
+ * call fails with SENTINEL_ERR_UNSUPPORTED and a message naming both sizes; nothing is
+ * launched.
+ * The first call on each device looks up the array's device address (once per device, under a
+ * lock); make that first call outside any stream capture.  All calls on a device share the
+ * one array: it keeps whatever the last call left, so each call re-zeroes its ticket word on
+ * the stream before launching, and two calls whose kernels could overlap on the GPU (two
+ * streams, two threads) race on it -- order them on one stream or with events. */
+#define SENTINEL_NOALLOC_SCRATCH_BYTES 65536
+int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int T, int d,
+                              int device, void *cuda_stream, float *dev_scores_out,
+                              float *dev_stats_out);
+
 /* Statistics of the last call of this kind, fp32 [(1+B)*8] per unit:
  * mean_x, var_x, ||x||_2, mean_m, var_m, cov(x,m), ||m||_2, Pearson rho.  Enqueues a copy. */
 int sentinel_get_stats(sentinel_verifier *h, sentinel_kind kind, float *dev_stats_out,

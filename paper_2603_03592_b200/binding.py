@@ -28,6 +28,7 @@ FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17,
 EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
+    "sentinel_distance_noalloc",
     "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
     "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
     "sentinel_export_state", "sentinel_import_state", "sentinel_last_error", "sentinel_destroy",
@@ -76,6 +77,7 @@ def lib():
         L.sentinel_update_reference.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp]
         L.sentinel_verify_host.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_distance.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_distance_noalloc.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_get_stats.argtypes = [vp, ip, vp, vp]
         L.sentinel_get_thresholds.argtypes = [vp, ip, vp, vp, vp]
         L.sentinel_get_counters.argtypes = [vp, vp, vp]
@@ -129,6 +131,20 @@ def sentinel_distance(x: torch.Tensor, m: torch.Tensor, scores_out: torch.Tensor
     B, T, d = x.shape
     _check(lib().sentinel_distance(_ptr(x), _ptr(m), B, T, d, x.device.index or 0,
                                    _stream_ptr(stream), _ptr(scores_out), _ptr(stats_out)))
+
+
+NOALLOC_SCRATCH_BYTES = 65536
+
+
+def sentinel_distance_noalloc(x: torch.Tensor, m: torch.Tensor, scores_out: torch.Tensor,
+                              stats_out: torch.Tensor | None = None, stream=None) -> None:
+    """``sentinel_distance`` for callers that may not allocate device memory during the call
+    (frozen pools, fixed budgets, latency-critical loops): its scratch is a fixed array inside
+    the library.  Calls on one device share that array, so keep them ordered on one stream;
+    make the first call on a device outside any stream capture."""
+    B, T, d = x.shape
+    _check(lib().sentinel_distance_noalloc(_ptr(x), _ptr(m), B, T, d, x.device.index or 0,
+                                           _stream_ptr(stream), _ptr(scores_out), _ptr(stats_out)))
 
 
 class Verifier:

@@ -4,6 +4,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -550,6 +551,83 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
   }
   SENTINEL_CUDA(h, cudaMemcpyAsync(h->hs, &st, sizeof st, cudaMemcpyHostToDevice, s));
   SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+  return SENTINEL_OK;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// sentinel_distance_noalloc: the stateless distance with its scratch in the library image
+
+namespace {
+
+// Scratch of the no-allocation entry point.  In host code this name is only a stand-in for the
+// symbol: the address a kernel may use is looked up per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SENTINEL_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kNoAllocMaxDevices = 64;
+constexpr size_t kNoAllocTicketBytes = 256;          // the ticket word, kept on its own 256 bytes
+std::mutex g_noalloc_mutex;
+unsigned char *g_noalloc_addr[kNoAllocMaxDevices];  // device address of the array, per device
+
+// Resolves the array's address on `device` (which must be current).  Once per device.
+cudaError_t noalloc_scratch_address(int device, unsigned char **out) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_addr[device]) {
+    void *p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_addr[device] = static_cast<unsigned char *>(p);
+  }
+  *out = g_noalloc_addr[device];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int T, int d, int device,
+                              void *cuda_stream, float *dev_scores_out, float *dev_stats_out) {
+  if (!dev_x || !dev_m || !dev_scores_out) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "x, m or scores_out is NULL");
+  int rc = check_shape(nullptr, B, T, d);
+  if (rc) return rc;
+  if (!aligned16(dev_x) || !aligned16(dev_m)) return fail(nullptr, SENTINEL_ERR_UNALIGNED, "x or m is not 16-byte aligned");
+  int ndev = 0;
+  SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
+  if (device < 0 || device >= ndev || device >= kNoAllocMaxDevices)
+    return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist or is beyond the %d this entry point tracks", device, kNoAllocMaxDevices);
+  DeviceGuard guard(device);
+  SENTINEL_CUDA(nullptr, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+  std::string oerr;
+  const int G = streaming_ctas(device, B, T, &oerr);
+  if (G < 1) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str());
+  const size_t slot_bytes = (size_t)G * kSegsPerCta * kSlotWords * sizeof(unsigned long long);
+  if (slot_bytes + kNoAllocTicketBytes > (size_t)SENTINEL_NOALLOC_SCRATCH_BYTES)
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED,
+                "this launch needs %zu bytes of scratch (%d streaming CTAs), the built-in array holds %d",
+                slot_bytes + kNoAllocTicketBytes, G, SENTINEL_NOALLOC_SCRATCH_BYTES);
+
+  unsigned char *scratch = nullptr;
+  SENTINEL_CUDA(nullptr, noalloc_scratch_address(device, &scratch));
+  // layout: [ticket: 256 bytes][slots]; the slots are rewritten by every launch, the ticket
+  // must start at zero whatever an earlier call left there
+  SENTINEL_CUDA(nullptr, cudaMemsetAsync(scratch, 0, kNoAllocTicketBytes, s));
+
+  StreamArgs a;
+  memset(&a, 0, sizeof a);
+  a.x = static_cast<const uint16_t *>(dev_x);
+  a.m_ext = dev_m;
+  a.partials = reinterpret_cast<unsigned long long *>(scratch + kNoAllocTicketBytes);
+  a.ticket = reinterpret_cast<unsigned *>(scratch);
+  a.scores_out = dev_scores_out;
+  a.stats_out = dev_stats_out;
+  a.B = B; a.T = T; a.d = d; a.G = G;
+  a.mode = kModeDistance;
+  stream_kernel<<<G + 1, kThreads, 0, s>>>(a);
+  SENTINEL_CUDA(nullptr, cudaGetLastError());
   return SENTINEL_OK;
 }
 
