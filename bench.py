@@ -34,6 +34,11 @@ from paper_2603_03592_b200 import replicas, synth  # noqa: E402
 ACT, GRAD = 0, 1
 BYTES_PER_ELEMENT = 10          # 2 (x, bf16 read) + 4 (m read) + 4 (EMA candidate write)
 MAX_DISTINCT = 24               # distinct input tensors per kind kept resident
+# dram__bytes_read.sum + dram__bytes_write.sum per element of the current stream_kernel, from the
+# ncu capture summarised in profiles/stream_kernel_cfg3_ncu_full.md (B=8 x 4096 x 4096; traffic
+# grows in proportion to the element count, so a launch of N elements moves this times N).
+# Set to None whenever the kernel changes until the capture is retaken.
+NCU_DRAM_BYTES_PER_ELEMENT = 9.673
 
 
 def measured_peak_gbs():
@@ -207,7 +212,9 @@ def run_ours(args, rank, world, local_rank):
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "peak_source": "%s copy bandwidth" % peak_kind,
                      "kernel": "stream_kernel", "avg_launch_ms": round(kernel_ms, 4),
-                     "traffic": args.traffic},
+                     "traffic": (args.traffic if args.traffic is not None else
+                                 (round(NCU_DRAM_BYTES_PER_ELEMENT * N) if NCU_DRAM_BYTES_PER_ELEMENT else None)),
+                     "traffic_source": "ncu on B=8x4096x4096, scaled by element count"},
     }
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)

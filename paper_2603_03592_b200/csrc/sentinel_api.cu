@@ -43,6 +43,7 @@ struct sentinel_verifier {
   size_t N = 0, Ns = 0;
   int cap0 = 0, cap1 = 0;
   int G = 1;                        // streaming CTAs; launches use G + 1
+  size_t refresh_smem = 0;          // dynamic shared memory of a launch that may refresh thresholds
   float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
   HandleState *hs = nullptr;
   double *hist[2] = {nullptr, nullptr};
@@ -169,13 +170,13 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
 }
 
 int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) {
-  stream_kernel<<<grid, kThreads, 0, s>>>(a);
+  stream_kernel<<<grid, kThreads, h->refresh_smem, s>>>(a);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
 }
 
 int run_refresh(sentinel_verifier *h, cudaStream_t s) {
-  refresh_kernel<<<1, kThreads, 0, s>>>(h->hs, h->hist[0], h->hist[1], h->cap0, h->cap1,
+  refresh_kernel<<<1, kThreads, h->refresh_smem, s>>>(h->hs, h->hist[0], h->hist[1], h->cap0, h->cap1,
                                         alg5_of(h->cfg, 0), alg5_of(h->cfg, 1));
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
@@ -258,6 +259,13 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->N = h->Ns * cfg->B;
   h->cap0 = cfg->window_steps;
   h->cap1 = cfg->window_steps * cfg->B;
+  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1) * sizeof(double);
+  {   // the six padded windows may exceed the 48 KiB a kernel gets without asking
+    const int most = (int)(refresh_smem_doubles(SENTINEL_MAX_WINDOW, SENTINEL_MAX_WINDOW) * sizeof(double));
+    cudaError_t ae = cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
+  }
   std::string oerr;
   h->G = streaming_ctas(cfg->device, cfg->B, cfg->T, &oerr);
   if (h->G < 1) { delete h; return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str()); }

@@ -360,25 +360,46 @@ __device__ __forceinline__ int warp_count_outside(const double *s, int n, double
   return c;
 }
 
-// Refreshes q1,q2,q3,k,tau of every (level, metric) window of one kind.  Whole CTA.
+constexpr int kGroupThreads = 96;        // three warps work on one (level, metric) window
+constexpr int kRefreshGroups = 2 * kNumMetrics;
+static_assert(kRefreshGroups * kGroupThreads <= kThreads, "one thread group per window");
+
+__device__ __forceinline__ void group_barrier(int group) {   // named barrier 1 + group
+  asm volatile("bar.sync %0, %1;" :: "r"(group + 1), "r"(kGroupThreads) : "memory");
+}
+
+__host__ __device__ inline int pow2_at_least(int n) {
+  int p = 1;
+  while (p < n) p <<= 1;
+  return p;
+}
+
+// doubles of shared memory the refresh needs: a padded copy of each of the six windows
+__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1) {
+  return (size_t)kNumMetrics * ((size_t)pow2_at_least(cap0) + (size_t)pow2_at_least(cap1));
+}
+
+// Refreshes q1,q2,q3,k,tau of every (level, metric) window of one kind (Alg. 5).  Whole CTA:
+// the six windows are handled side by side, each by three warps with their own named barrier.
 __device__ void refresh_thresholds(KindState *ks, const double *hist, int cap0, int cap1,
-                                   const Alg5Params &a5, double *s_sort) {
-  const int tid = threadIdx.x, lane = tid & 31;
-  for (int L = 0; L < 2; ++L) {
+                                   const Alg5Params &a5, double *s_dyn) {
+  const int group = threadIdx.x / kGroupThreads;
+  const int gt = threadIdx.x - group * kGroupThreads;
+  if (group < kRefreshGroups) {
+    const int L = group / kNumMetrics, i = group - L * kNumMetrics;
     const int n = ks->hist_count[L];
-    if (n == 0) continue;                          // empty window: nothing to compute
-    const int cap = L ? cap1 : cap0;
-    int npad = 1;
-    while (npad < n) npad <<= 1;
-    for (int i = 0; i < kNumMetrics; ++i) {
+    if (n > 0) {                                   // an empty window leaves everything as it is
+      const int cap = L ? cap1 : cap0;
+      const int pad0 = pow2_at_least(cap0), pad1 = pow2_at_least(cap1);
+      double *s_sort = s_dyn + (L ? (size_t)kNumMetrics * pad0 + (size_t)i * pad1 : (size_t)i * pad0);
       const double *ring = hist + (L ? (size_t)kNumMetrics * cap0 : 0) + (size_t)i * cap;
-      __syncthreads();
+      const int npad = pow2_at_least(n);
       // the order of the window is immaterial to Alg. 5, so the ring is read as it lies
-      for (int j = tid; j < npad; j += kThreads) s_sort[j] = (j < n) ? ring[j] : CUDART_INF;
-      __syncthreads();
+      for (int j = gt; j < npad; j += kGroupThreads) s_sort[j] = (j < n) ? ring[j] : CUDART_INF;
+      group_barrier(group);
       for (int k2 = 2; k2 <= npad; k2 <<= 1) {     // bitonic sort, ascending
         for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
-          for (int t = tid; t < npad; t += kThreads) {
+          for (int t = gt; t < npad; t += kGroupThreads) {
             const int partner = t ^ j2;
             if (partner > t) {
               const double va = s_sort[t], vb = s_sort[partner];
@@ -386,34 +407,45 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, int cap0, 
               if ((va > vb) == up) { s_sort[t] = vb; s_sort[partner] = va; }
             }
           }
-          __syncthreads();
+          group_barrier(group);
         }
       }
-      if (tid < 32) {                              // warp 0 walks the algorithm's steps
+      if (gt < 32) {                               // the group's first warp walks the steps
+        const int lane = gt;
         const double q1 = percentile_sorted(s_sort, n, 0.25);
         const double q2 = percentile_sorted(s_sort, n, 0.50);
         const double q3 = percentile_sorted(s_sort, n, 0.75);
         const double iqr = fmax(__dsub_rn(q3, q1), a5.eps);
+        const double dn = (double)n;
+        // FP-rate = count/n is monotone in the count, so "FP-rate > alpha" and
+        // "FP-rate < shrink_ratio*alpha" are thresholds on the count, found once with the
+        // very division the comparison is defined by
+        const double low_mark = __dmul_rn(a5.shrink_ratio, a5.alpha);
+        int widen_from = (int)floor(a5.alpha * dn) - 1;       // smallest count with count/n > alpha
+        if (widen_from < 0) widen_from = 0;
+        while (widen_from <= n && !((double)widen_from / dn > a5.alpha)) ++widen_from;
+        int narrow_to = (int)ceil(low_mark * dn) + 1;         // largest count with count/n < low_mark
+        if (narrow_to > n) narrow_to = n;
+        while (narrow_to >= 0 && !((double)narrow_to / dn < low_mark)) --narrow_to;
+
         double k = ks->thr[L][i][3];
         double lo = __dsub_rn(q2, __dmul_rn(k, iqr));
         double hi = __dadd_rn(q2, __dmul_rn(k, iqr));
-        const double dn = (double)n;
-        double fp = (double)warp_count_outside(s_sort, n, lo, hi, lane) / dn;
+        int outside = warp_count_outside(s_sort, n, lo, hi, lane);
         int it = 0;
-        while (fp > a5.alpha && it < a5.n_max) {   // widen
+        while (outside >= widen_from && it < a5.n_max) {      // widen
           k = __dmul_rn(k, a5.gamma_g);
           lo = __dsub_rn(q2, __dmul_rn(k, iqr));
           hi = __dadd_rn(q2, __dmul_rn(k, iqr));
-          fp = (double)warp_count_outside(s_sort, n, lo, hi, lane) / dn;
+          outside = warp_count_outside(s_sort, n, lo, hi, lane);
           ++it;
         }
         it = 0;
-        const double low_mark = __dmul_rn(a5.shrink_ratio, a5.alpha);
-        while (fp < low_mark && it < a5.n_max) {   // narrow
+        while (outside <= narrow_to && it < a5.n_max) {       // narrow
           k = __dmul_rn(k, a5.gamma_s);
           lo = __dsub_rn(q2, __dmul_rn(k, iqr));
           hi = __dadd_rn(q2, __dmul_rn(k, iqr));
-          fp = (double)warp_count_outside(s_sort, n, lo, hi, lane) / dn;
+          outside = warp_count_outside(s_sort, n, lo, hi, lane);
           ++it;
         }
         const double d_min = __dmul_rn(fabs(q2), a5.lambda);
@@ -428,7 +460,7 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, int cap0, 
     }
   }
   __syncthreads();
-  if (tid == 0) ks->refresh_pending = 0;
+  if (threadIdx.x == 0) ks->refresh_pending = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -461,12 +493,22 @@ __device__ void finalize(const StreamArgs &a) {
   __shared__ double s_gamma[kMaxB + 1][kNumMetrics];
   __shared__ unsigned s_flag[kMaxB + 1];
   __shared__ int s_severe, s_no_thr;
+  // The handle's small state is fetched once, in one batch, and written back once: by now it
+  // has long left the L2, and touching it field by field would cost a DRAM round trip each.
+  __shared__ __align__(8) HandleState s_hs;
+  static_assert(sizeof(HandleState) % 8 == 0, "copied as 64-bit words");
+  constexpr int kStateWords = (int)(sizeof(HandleState) / 8);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = a.B, rows = B + 1;
   const size_t Ns = (size_t)a.T * a.d;
 
   if (tid == 0) { s_severe = 0; s_no_thr = 0; }
+  if (a.hs && tid >= kThreads - kStateWords) {      // the last warps: the first ones gather sums
+    const int w = tid - (kThreads - kStateWords);
+    reinterpret_cast<unsigned long long *>(&s_hs)[w] =
+        __ldcg(reinterpret_cast<const unsigned long long *>(a.hs) + w);
+  }
 
   // per-sample sums over the slots tagged with that sample, in CTA order
   for (int b = warp; b < B; b += kWarps) {
@@ -531,7 +573,7 @@ __device__ void finalize(const StreamArgs &a) {
   }
   __syncthreads();
 
-  KindState *ks = a.hs ? &a.hs->kind[a.kind] : nullptr;
+  KindState *ks = a.hs ? &s_hs.kind[a.kind] : nullptr;     // the shared copy
 
   // scores, statistics and the Tukey test: one thread per unit
   unsigned my_flag = 0u;
@@ -575,11 +617,12 @@ __device__ void finalize(const StreamArgs &a) {
     } else if (a.mode == kModeVerify) {
       const int L = (tid == 0) ? 0 : 1;
       for (int i = 0; i < kNumMetrics; ++i) {
-        // CTA 0 of this launch may have rewritten the thresholds: read them from L2
-        if (!__ldcg(&ks->has_thr[L][i])) { s_no_thr = 1; continue; }
+        // (the copy was read from L2 after the ticket, so it holds what CTA 0 of this launch
+        // may have just rewritten)
+        if (!ks->has_thr[L][i]) { s_no_thr = 1; continue; }
         if (!((a.metric_mask >> i) & 1u)) continue;
-        const double q2 = __ldcg(&ks->thr[L][i][1]);
-        const double tau_lower = __ldcg(&ks->thr[L][i][4]), tau_upper = __ldcg(&ks->thr[L][i][5]);
+        const double q2 = ks->thr[L][i][1];
+        const double tau_lower = ks->thr[L][i][4], tau_upper = ks->thr[L][i][5];
         if (g[i] < tau_lower || g[i] > tau_upper) my_flag |= (1u << i);
         if (tid == 0 && fabs(g[i] - q2) >= a.severe_mult * (tau_upper - q2)) s_severe = 1;
       }
@@ -589,7 +632,7 @@ __device__ void finalize(const StreamArgs &a) {
   const int any_flag = __syncthreads_or(my_flag != 0u);
 
   if (tid == 0 && a.mode != kModeDistance) {
-    HandleState *hs = a.hs;
+    HandleState *hs = &s_hs;
     unsigned status = 0u;
     if (a.mode == kModeVerify) {
       ks->steps += 1;
@@ -624,7 +667,14 @@ __device__ void finalize(const StreamArgs &a) {
   }
   __syncthreads();
   if (a.flags_out && tid < rows) a.flags_out[tid] = s_flag[tid];
-  if (tid == 0) *a.ticket = 0u;                  // ready for the next launch
+  if (a.hs) {                                    // write the state back, ticket cleared
+    if (tid == 0) s_hs.ticket = 0u;
+    __syncthreads();
+    if (tid < kStateWords)
+      reinterpret_cast<unsigned long long *>(a.hs)[tid] = reinterpret_cast<unsigned long long *>(&s_hs)[tid];
+  } else if (tid == 0) {
+    *a.ticket = 0u;                              // ready for the next launch
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -637,8 +687,8 @@ __device__ void finalize(const StreamArgs &a) {
 __global__ void __launch_bounds__(kThreads)
 stream_kernel(const StreamArgs a) {
   __shared__ unsigned long long s_part[kWarps][kSlotWords];
-  __shared__ double s_sort[kMaxWindow];
   __shared__ int s_last;
+  extern __shared__ double s_dyn[];            // refresh_smem_doubles(cap0, cap1) when a handle is given
 
   const float *m_in;
   float *m_out;
@@ -654,7 +704,7 @@ stream_kernel(const StreamArgs a) {
   if (blockIdx.x == 0) {
     if (a.hs) {
       KindState *ks = &a.hs->kind[a.kind];
-      if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.cap0, a.cap1, a.a5, s_sort);
+      if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.cap0, a.cap1, a.a5, s_dyn);
     }
   } else {
     stream_cta(a, blockIdx.x - 1, m_in, m_out, s_part);
@@ -676,10 +726,10 @@ stream_kernel(const StreamArgs a) {
 __global__ void __launch_bounds__(kThreads)
 refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, int cap0, int cap1,
                Alg5Params a5_act, Alg5Params a5_grad) {
-  __shared__ double s_sort[kMaxWindow];
-  if (hs->kind[0].refresh_pending) refresh_thresholds(&hs->kind[0], hist_act, cap0, cap1, a5_act, s_sort);
+  extern __shared__ double s_dyn[];
+  if (hs->kind[0].refresh_pending) refresh_thresholds(&hs->kind[0], hist_act, cap0, cap1, a5_act, s_dyn);
   __syncthreads();
-  if (hs->kind[1].refresh_pending) refresh_thresholds(&hs->kind[1], hist_grad, cap0, cap1, a5_grad, s_sort);
+  if (hs->kind[1].refresh_pending) refresh_thresholds(&hs->kind[1], hist_grad, cap0, cap1, a5_grad, s_dyn);
 }
 
 __global__ void reset_worker_kernel(HandleState *hs) {

@@ -1,0 +1,99 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration ``bench.py`` times
+(same entry points, same shapes): every score of every unit and every flag against the float64
+oracle run on the same tensors.  A few steps per shape keep the oracle within about a minute."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import UNIT_BITS, assert_scores_close, assert_stats_close, near_threshold
+from paper_2603_03592_b200 import synth
+
+pytestmark = pytest.mark.gpu
+ACT, GRAD = 0, 1
+
+
+@pytest.fixture(scope="module")
+def sb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_03592_b200 import binding
+    binding.lib()
+    return binding
+
+
+def run_steps(sb, oracle_mod, w, kind, n_warm, corruption):
+    gv = sb.Verifier(w.B, w.T, w.d)
+    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d))
+    for t in range(n_warm):
+        x = synth.clean(w, 0, kind, t, "cuda")
+        gs = gv.update_reference(x, kind)
+        os_, _ = ov.update_reference(synth.bits(x), kind)
+        assert_scores_close(gs.cpu().numpy(), os_, float(x.float().abs().mean()), "%s warm-up %d" % (w.name, t))
+        st = gv.sentinel_get_stats(kind).cpu().numpy()
+        assert_stats_close(st, ov.last_stats(kind), float(x.float().std()),
+                           max(float(np.abs(ov.last_stats(kind)[0, 4])) ** 0.5, 1e-30), "%s stats %d" % (w.name, t))
+    # a clean verified step, then a corrupted one
+    for t, name in ((n_warm, None), (n_warm + 1, corruption)):
+        x = synth.clean(w, 0, kind, t, "cuda")
+        if name:
+            x = synth.corrupt(w, x, name, 0, kind, t)
+        thr, valid = ov.thresholds(kind)
+        gs, gf = gv.verify(x, kind)
+        os_, of, commit = ov.verify(synth.bits(x), kind)
+        gs, gf = gs.cpu().numpy(), gf.cpu().numpy().view(np.uint32)
+        assert_scores_close(gs, os_, float(x.float().abs().mean()), "%s verify (%s)" % (w.name, name))
+        if not np.array_equal(gf, of):
+            near = near_threshold(os_, thr, valid, w.B)
+            assert np.all(near[((gf ^ of) & UNIT_BITS) != 0]), (gf, of)
+        assert bool(gf[0] & sb.FLAG_COMMITTED) == commit
+    c = gv.sentinel_get_counters()
+    assert (c["violations"], c["clean_streak"], c["banned"]) == ov.counters()
+    gv.close()
+
+
+def test_cfg4_wide_model_activations(sb, oracle_mod):
+    """B=4 x T=8192 x d=8192 (512 MiB per tensor), Student-t activations, uniform noise on one sample."""
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], ACT, 2, "add_uniform_sample")
+
+
+def test_cfg4_wide_model_gradients(sb, oracle_mod):
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], GRAD, 1, "add_uniform_sample")
+
+
+def test_cfg3_1b_class_zeroed_tokens(sb, oracle_mod):
+    """B=8 x T=4096 x d=4096, lognormal channel scales; 10% of the token rows zeroed."""
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg3"], ACT, 2, "zero_tokens")
+
+
+def test_cfg5_boundary_shape_gradients(sb, oracle_mod):
+    """B=16 x T=2048 x d=4096 (the many-boundary sweep's shape), additive Gaussian noise."""
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg5"], GRAD, 2, "add_gauss")
+
+
+def test_cfg2_small_lm_stream_prefix(sb, oracle_mod):
+    """B=16 x T=1024 x d=2048: the full 16-step warm-up and the first verified steps of the
+    stream, corruptions as the recipe draws them."""
+    w = synth.WORKLOADS["cfg2"]
+    gv = sb.Verifier(w.B, w.T, w.d)
+    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d))
+    for t in range(w.warmup + 6):
+        x, name = synth.microbatch(w, 0, ACT, t, "cuda")
+        if t == w.warmup + 3 and name is None:
+            x, name = synth.corrupt(w, x, "add_gauss", 0, ACT, t), "add_gauss"
+        scale = float(x.float().abs().mean())
+        if t < w.warmup:
+            gs = gv.update_reference(x, ACT)
+            os_, _ = ov.update_reference(synth.bits(x), ACT)
+            assert_scores_close(gs.cpu().numpy(), os_, scale, "cfg2 warm-up %d" % t)
+        else:
+            thr, valid = ov.thresholds(ACT)
+            gs, gf = gv.verify(x, ACT)
+            os_, of, _ = ov.verify(synth.bits(x), ACT)
+            gf = gf.cpu().numpy().view(np.uint32)
+            assert_scores_close(gs.cpu().numpy(), os_, scale, "cfg2 verify %d" % t)
+            if not np.array_equal(gf, of):
+                near = near_threshold(os_, thr, valid, w.B)
+                assert np.all(near[((gf ^ of) & UNIT_BITS) != 0]), (t, gf, of)
+            if name is not None:
+                assert np.any(of & UNIT_BITS), "additive noise of the tensor's own std is caught"
+    gv.close()
