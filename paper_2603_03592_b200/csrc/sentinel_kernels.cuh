@@ -474,36 +474,23 @@ struct UnitSums {
   double x0, m0;             // the shift the sums were taken about
 };
 
-__device__ __forceinline__ void push_history(KindState *ks, double *hist, int L, int cap, int cap0,
-                                             const double g[kNumMetrics]) {
-  int idx;
-  if (ks->hist_count[L] < cap) {
-    idx = (ks->hist_head[L] + ks->hist_count[L]) % cap;
-    ks->hist_count[L] += 1;
-  } else {                                         // window full: the oldest entry leaves
-    idx = ks->hist_head[L];
-    ks->hist_head[L] = (idx + 1) % cap;
-  }
-  double *base = hist + (L ? (size_t)kNumMetrics * cap0 : 0);
-  for (int i = 0; i < kNumMetrics; ++i) base[(size_t)i * cap + idx] = g[i];
-}
-
 __device__ void finalize(const StreamArgs &a) {
   __shared__ UnitSums s_unit[kMaxB + 1];
-  __shared__ double s_gamma[kMaxB + 1][kNumMetrics];
   __shared__ unsigned s_flag[kMaxB + 1];
   __shared__ int s_severe, s_no_thr;
+  __shared__ unsigned s_status;                  // status bits of row 0
   // The handle's small state is fetched once, in one batch, and written back once: by now it
   // has long left the L2, and touching it field by field would cost a DRAM round trip each.
   __shared__ __align__(8) HandleState s_hs;
   static_assert(sizeof(HandleState) % 8 == 0, "copied as 64-bit words");
   constexpr int kStateWords = (int)(sizeof(HandleState) / 8);
+  constexpr int kDecider = kThreads - 1;         // the thread that keeps the counters
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = a.B, rows = B + 1;
   const size_t Ns = (size_t)a.T * a.d;
 
-  if (tid == 0) { s_severe = 0; s_no_thr = 0; }
+  if (tid == 0) { s_severe = 0; s_no_thr = 0; s_status = 0u; }
   if (a.hs && tid >= kThreads - kStateWords) {      // the last warps: the first ones gather sums
     const int w = tid - (kThreads - kStateWords);
     reinterpret_cast<unsigned long long *>(&s_hs)[w] =
@@ -522,13 +509,15 @@ __device__ void finalize(const StreamArgs &a) {
     const long long n_slots = (c_hi - c_lo + 1) * kSegsPerCta;
     for (long long q = lane; q < n_slots; q += 32) {
       const unsigned long long *slot = a.partials + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
-      const unsigned long long w7 = __ldcg(slot + 7);
-      if (((w7 >> kTagShift) & 0xFFull) != (unsigned long long)(b + 1)) continue;
+      unsigned long long w[kSlotWords];
 #pragma unroll
-      for (int j = 0; j < 6; ++j) v[j] += __longlong_as_double((long long)__ldcg(slot + j));
-      fl += __ldcg(slot + 6);
-      bits |= w7 & 0x7ull;
-      first = w7 >> kX0Shift;            // the same in every slot of this sample
+      for (int j = 0; j < kSlotWords; ++j) w[j] = __ldcg(slot + j);   // one round trip, then the tag
+      if (((w[7] >> kTagShift) & 0xFFull) != (unsigned long long)(b + 1)) continue;
+#pragma unroll
+      for (int j = 0; j < 6; ++j) v[j] += __longlong_as_double((long long)w[j]);
+      fl += w[6];
+      bits |= w[7] & 0x7ull;
+      first = w[7] >> kX0Shift;          // the same in every slot of this sample
     }
 #pragma unroll
     for (int j = 0; j < 6; ++j) v[j] = warp_sum(v[j]);
@@ -550,69 +539,78 @@ __device__ void finalize(const StreamArgs &a) {
   }
   __syncthreads();
 
-  // whole-tensor unit = the samples added up in order, re-centred on sample 0's shift:
-  // sum (x-K) = sum (x-x0) + n dx,  sum (x-K)^2 = sum (x-x0)^2 + 2 dx sum (x-x0) + n dx^2, ...
-  if (tid == 0) {
-    UnitSums u = {{0., 0., 0., 0., 0., 0.}, 0ull, 0ull, s_unit[1].first, s_unit[1].x0, s_unit[1].m0};
+  // whole-tensor unit = the samples added up (warp 0, fixed tree), re-centred on sample 0's
+  // shift K: sum (x-K) = sum (x-x0) + n dx,  sum (x-K)^2 = sum (x-x0)^2 + 2 dx sum (x-x0) + n dx^2,
+  // sum (x-Kx)(m-Km) = sum (x-x0)(m-m0) + dx sum (m-m0) + dm sum (x-x0) + n dx dm
+  if (warp == 0) {
+    const UnitSums &ref = s_unit[1];
     const double n = (double)Ns;
-    for (int b = 0; b < B; ++b) {
+    double t[6] = {0., 0., 0., 0., 0., 0.};
+    unsigned long long fl = 0ull, bits = 0ull;
+    for (int b = lane; b < B; b += 32) {
       const UnitSums &v = s_unit[1 + b];
-      const double dx = v.x0 - u.x0, dm = v.m0 - u.m0;
-      u.s[0] += v.s[0] + n * dx;
-      u.s[1] += v.s[1] + 2. * dx * v.s[0] + n * dx * dx;
-      u.s[2] += v.s[2] + n * dm;
-      u.s[3] += v.s[3] + 2. * dm * v.s[2] + n * dm * dm;
-      u.s[4] += v.s[4] + dx * v.s[2] + dm * v.s[0] + n * dx * dm;
-      u.s[5] += v.s[5];
-      u.flips += v.flips;
-      u.bits |= v.bits;
-      if ((v.first & 0xFFFFull) != (u.first & 0xFFFFull)) u.bits |= kBitXVaries;
-      if ((v.first >> 16) != (u.first >> 16)) u.bits |= kBitMVaries;
+      const double dx = v.x0 - ref.x0, dm = v.m0 - ref.m0;
+      t[0] += v.s[0] + n * dx;
+      t[1] += v.s[1] + 2. * dx * v.s[0] + n * dx * dx;
+      t[2] += v.s[2] + n * dm;
+      t[3] += v.s[3] + 2. * dm * v.s[2] + n * dm * dm;
+      t[4] += v.s[4] + dx * v.s[2] + dm * v.s[0] + n * dx * dm;
+      t[5] += v.s[5];
+      fl += v.flips;
+      bits |= v.bits;
+      if ((v.first & 0xFFFFull) != (ref.first & 0xFFFFull)) bits |= kBitXVaries;
+      if ((v.first >> 16) != (ref.first >> 16)) bits |= kBitMVaries;
     }
-    s_unit[0] = u;
+#pragma unroll
+    for (int j = 0; j < 6; ++j) t[j] = warp_sum(t[j]);
+    fl = warp_sum(fl);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+    if (lane == 0) {
+#pragma unroll
+      for (int j = 0; j < 6; ++j) s_unit[0].s[j] = t[j];
+      s_unit[0].flips = fl;
+      s_unit[0].bits = bits;
+      s_unit[0].first = ref.first;
+      s_unit[0].x0 = ref.x0;
+      s_unit[0].m0 = ref.m0;
+    }
   }
   __syncthreads();
 
   KindState *ks = a.hs ? &s_hs.kind[a.kind] : nullptr;     // the shared copy
 
-  // scores, statistics and the Tukey test: one thread per unit
+  // scores and the Tukey test: one thread per unit
   unsigned my_flag = 0u;
+  double g[kNumMetrics] = {0., 0., 0.};
+  double st_var_x = 0., st_var_m = 0., st_cov = 0., st_rho = 0., inv_n = 0.;
+  bool nonfinite = false;
+  int ring_head = 0, ring_count = 0;              // this unit's level, before this step
   if (tid < rows) {
-    const UnitSums u = s_unit[tid];
+    const UnitSums &u = s_unit[tid];
     const double n = (tid == 0) ? (double)B * (double)Ns : (double)Ns;
-    const bool nonfinite = (u.bits & kBitNonfinite) != 0ull;
+    inv_n = 1. / n;
+    nonfinite = (u.bits & kBitNonfinite) != 0ull;
     // a vector whose elements all equal its first one (bitwise, or +0 against -0) has
     // variance exactly 0
     const bool x_const = !(u.bits & kBitXVaries) || u.s[1] == 0.;
     const bool m_const = !(u.bits & kBitMVaries) || u.s[3] == 0.;
-    const double dmean_x = u.s[0] / n, dmean_m = u.s[2] / n;      // means of the shifted values
-    const double mean_x = u.x0 + dmean_x, mean_m = u.m0 + dmean_m;
-    const double var_x = x_const ? 0. : fmax(u.s[1] / n - dmean_x * dmean_x, 0.);
-    const double var_m = m_const ? 0. : fmax(u.s[3] / n - dmean_m * dmean_m, 0.);
-    const double cov = u.s[4] / n - dmean_x * dmean_m;
-    const double sq_x = fmax(u.s[1] + 2. * u.x0 * u.s[0] + n * u.x0 * u.x0, 0.);   // sum x^2
-    const double sq_m = fmax(u.s[3] + 2. * u.m0 * u.s[2] + n * u.m0 * u.m0, 0.);
-    const double sd_x = sqrt(var_x), sd_m = sqrt(var_m);
-    double rho = 0., l2z;
-    if (sd_x > 0. && sd_m > 0.) {
-      rho = fmin(fmax(cov / (sd_x * sd_m), -1.), 1.);
-      l2z = 2. - 2. * rho;                    // mean (zx - zm)^2 = 2 - 2 rho
+    const double dmean_x = u.s[0] * inv_n, dmean_m = u.s[2] * inv_n;   // means of the shifted values
+    st_var_x = x_const ? 0. : fmax(u.s[1] * inv_n - dmean_x * dmean_x, 0.);
+    st_var_m = m_const ? 0. : fmax(u.s[3] * inv_n - dmean_m * dmean_m, 0.);
+    st_cov = u.s[4] * inv_n - dmean_x * dmean_m;
+    double l2z;
+    if (st_var_x > 0. && st_var_m > 0.) {
+      st_rho = fmin(fmax(st_cov * rsqrt(st_var_x) * rsqrt(st_var_m), -1.), 1.);
+      l2z = 2. - 2. * st_rho;                 // mean (zx - zm)^2 = 2 - 2 rho
     } else {
-      l2z = (sd_x > 0. || sd_m > 0.) ? 1. : 0.;   // a constant vector z-scores to zero
+      l2z = (st_var_x > 0. || st_var_m > 0.) ? 1. : 0.;   // a constant vector z-scores to zero
     }
-    double g[kNumMetrics] = {u.s[5] / n, l2z, (double)u.flips / n};
-    double st[kNumStats] = {mean_x, var_x, sqrt(sq_x), mean_m, var_m, cov, sqrt(sq_m), rho};
+    g[0] = u.s[5] * inv_n;
+    g[1] = l2z;
+    g[2] = (double)u.flips * inv_n;
     if (nonfinite) {
       for (int i = 0; i < kNumMetrics; ++i) g[i] = CUDART_NAN;
-      for (int i = 0; i < kNumStats; ++i) st[i] = CUDART_NAN;
-    }
-    for (int i = 0; i < kNumMetrics; ++i) s_gamma[tid][i] = g[i];
-    if (a.scores_out)
-      for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = (float)g[i];
-    if (a.stats_out)
-      for (int i = 0; i < kNumStats; ++i) a.stats_out[tid * kNumStats + i] = (float)st[i];
-
-    if (nonfinite) {
       my_flag = kFlagNonfinite;
     } else if (a.mode == kModeVerify) {
       const int L = (tid == 0) ? 0 : 1;
@@ -628,14 +626,48 @@ __device__ void finalize(const StreamArgs &a) {
       }
     }
     s_flag[tid] = my_flag;
+    if (ks) { ring_head = ks->hist_head[tid ? 1 : 0]; ring_count = ks->hist_count[tid ? 1 : 0]; }
   }
   const int any_flag = __syncthreads_or(my_flag != 0u);
 
-  if (tid == 0 && a.mode != kModeDistance) {
+  // Who joins the history: verified step, the units that raised nothing; warm-up, every unit
+  // unless the input was non-finite (then nothing changes).
+  const bool warmup_ok = (a.mode == kModeWarmup) && !any_flag;
+  if (tid < rows) {
+    const bool joins = (a.mode == kModeVerify) ? (my_flag == 0u) : warmup_ok;
+    if (joins) {
+      // the k-th unit of a level to join goes to ring slot (head + count + k) mod cap, which
+      // is the oldest entry's slot once the window is full
+      const int L = tid ? 1 : 0, cap = L ? a.cap1 : a.cap0;
+      int k = 0;
+      if (L && a.mode == kModeVerify)
+        for (int r = 1; r < tid; ++r) k += (s_flag[r] == 0u);
+      else if (L)
+        k = tid - 1;
+      const int idx = (int)(((long long)ring_head + ring_count + k) % cap);
+      double *base = a.hist + (L ? (size_t)kNumMetrics * a.cap0 : 0);
+      for (int i = 0; i < kNumMetrics; ++i) base[(size_t)i * cap + idx] = g[i];
+    }
+    if (a.scores_out)
+      for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = (float)g[i];
+    if (a.stats_out) {                           // off the decision path
+      const UnitSums &u = s_unit[tid];
+      const double n = (tid == 0) ? (double)B * (double)Ns : (double)Ns;
+      const double sq_x = fmax(u.s[1] + 2. * u.x0 * u.s[0] + n * u.x0 * u.x0, 0.);   // sum x^2
+      const double sq_m = fmax(u.s[3] + 2. * u.m0 * u.s[2] + n * u.m0 * u.m0, 0.);
+      double st[kNumStats] = {u.x0 + u.s[0] * inv_n, st_var_x, sqrt(sq_x), u.m0 + u.s[2] * inv_n,
+                              st_var_m, st_cov, sqrt(sq_m), st_rho};
+      for (int i = 0; i < kNumStats; ++i)
+        a.stats_out[tid * kNumStats + i] = nonfinite ? CUDART_NAN_F : (float)st[i];
+    }
+  }
+
+  if (tid == kDecider && a.mode != kModeDistance) {
     HandleState *hs = &s_hs;
     unsigned status = 0u;
+    ks->steps += 1;
+    int joined[2] = {0, 0};
     if (a.mode == kModeVerify) {
-      ks->steps += 1;
       if (any_flag) {                            // violation counter with forgiveness
         hs->violations += 1;
         hs->clean_streak = 0;
@@ -647,33 +679,37 @@ __device__ void finalize(const StreamArgs &a) {
           hs->clean_streak = 0;
         }
       }
-      for (int r = 0; r < rows; ++r)             // only clean units join the history
-        if (!s_flag[r]) push_history(ks, a.hist, r ? 1 : 0, r ? a.cap1 : a.cap0, a.cap0, s_gamma[r]);
+      joined[0] = (s_flag[0] == 0u);
+      for (int r = 1; r < rows; ++r) joined[1] += (s_flag[r] == 0u);
       ks->refresh_pending = 1;
       if (!any_flag) { ks->active ^= 1; status |= kFlagCommitted; }   // m_t := candidate
       if (s_severe) status |= kFlagSevere;
       if (hs->banned) status |= kFlagBanned;
       if (s_no_thr) status |= kFlagNoThresholds;
-    } else {                                     // warm-up: everything joins, always commit
-      ks->steps += 1;
-      if (!any_flag) {                           // (any_flag here means non-finite input)
-        for (int r = 0; r < rows; ++r)
-          push_history(ks, a.hist, r ? 1 : 0, r ? a.cap1 : a.cap0, a.cap0, s_gamma[r]);
-        ks->refresh_pending = 1;
-        ks->active ^= 1;
-      }
+    } else if (warmup_ok) {                      // warm-up: everything joins, always commit
+      joined[0] = 1;
+      joined[1] = B;
+      ks->refresh_pending = 1;
+      ks->active ^= 1;
     }
-    s_flag[0] |= status;
+    for (int L = 0; L < 2; ++L) {                // window bookkeeping after `joined` appends
+      const int cap = L ? a.cap1 : a.cap0;
+      const int total = ks->hist_count[L] + joined[L];
+      const int evicted = total > cap ? total - cap : 0;
+      ks->hist_count[L] = total - evicted;
+      ks->hist_head[L] = (int)(((long long)ks->hist_head[L] + evicted) % cap);
+    }
+    s_hs.ticket = 0u;                            // ready for the next launch
+    s_status = status;
   }
   __syncthreads();
-  if (a.flags_out && tid < rows) a.flags_out[tid] = s_flag[tid];
-  if (a.hs) {                                    // write the state back, ticket cleared
-    if (tid == 0) s_hs.ticket = 0u;
-    __syncthreads();
+  if (a.flags_out && tid < rows)
+    a.flags_out[tid] = s_flag[tid] | (tid == 0 ? s_status : 0u);
+  if (a.hs) {                                    // write the state back
     if (tid < kStateWords)
       reinterpret_cast<unsigned long long *>(a.hs)[tid] = reinterpret_cast<unsigned long long *>(&s_hs)[tid];
   } else if (tid == 0) {
-    *a.ticket = 0u;                              // ready for the next launch
+    *a.ticket = 0u;
   }
 }
 
