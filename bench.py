@@ -104,13 +104,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_stream(w, device, count, distinct):
+def build_stream(w, boundary, device, count, distinct):
     """`count` microbatches per kind after the warm-up, following the workload's recipe."""
     xs = {ACT: [], GRAD: []}
     n = min(count, distinct)
     for kind in (ACT, GRAD):
         for i in range(n):
-            x, _ = synth.microbatch(w, 0, kind, w.warmup + i, device)
+            x, _ = synth.microbatch(w, boundary, kind, w.warmup + i, device)
             xs[kind].append(x)
     return xs
 
@@ -122,65 +122,99 @@ def run_ours(args, rank, world, local_rank):
     device = torch.device("cuda", local_rank)
     w = synth.WORKLOADS[args.workload]
     N = w.B * w.T * w.d
-    v = binding.Verifier(w.B, w.T, w.d, device=local_rank)
-    stream = torch.cuda.current_stream()
+    nb = w.boundaries                               # independent stage boundaries, one stream each
+    main = torch.cuda.current_stream()
+    streams = [main] if nb == 1 else [torch.cuda.Stream(device=device) for _ in range(nb)]
+    vs = [binding.Verifier(w.B, w.T, w.d, device=local_rank) for _ in range(nb)]
 
     # reference warm-up on clean traffic (untimed set-up, as the method prescribes)
-    for t in range(w.warmup):
-        for kind in (ACT, GRAD):
-            v.sentinel_update_reference(synth.clean(w, 0, kind, t, device), kind)
+    for b, v in enumerate(vs):
+        for t in range(w.warmup):
+            for kind in (ACT, GRAD):
+                v.sentinel_update_reference(synth.clean(w, b, kind, t, device), kind)
     torch.cuda.synchronize()
 
     total = args.warmup + args.steps
-    xs = build_stream(w, device, total, args.distinct)
-    nd = len(xs[ACT])
-    scores = torch.empty(2, 1 + w.B, 3, dtype=torch.float32, device=device)
-    flags = torch.empty(2, 1 + w.B, dtype=torch.int32, device=device)
+    distinct = args.distinct if nb == 1 else min(args.distinct, 12)   # 8 boundaries: bound the footprint
+    xs = [build_stream(w, b, device, total, distinct) for b in range(nb)]
+    nd = len(xs[0][ACT])
+    scores = torch.empty(nb, 2, 1 + w.B, 3, dtype=torch.float32, device=device)
+    flags = torch.empty(nb, 2, 1 + w.B, dtype=torch.int32, device=device)
+    torch.cuda.synchronize()
 
     def step(i):
-        v.sentinel_verify(xs[ACT][i % nd], ACT, scores[0], flags[0], stream)
-        v.sentinel_verify(xs[GRAD][i % nd], GRAD, scores[1], flags[1], stream)
+        for b, (v, s) in enumerate(zip(vs, streams)):
+            v.sentinel_verify(xs[b][ACT][i % nd], ACT, scores[b, 0], flags[b, 0], s)
+            v.sentinel_verify(xs[b][GRAD][i % nd], GRAD, scores[b, 1], flags[b, 1], s)
 
+    def fork():                                      # side streams start after `main` gets here
+        if nb > 1:
+            ev = torch.cuda.Event()
+            ev.record(main)
+            for s in streams:
+                s.wait_event(ev)
+
+    def join():                                      # `main` continues after every side stream
+        if nb > 1:
+            for s in streams:
+                ev = torch.cuda.Event()
+                ev.record(s)
+                main.wait_event(ev)
+
+    fork()
     for i in range(args.warmup):
         step(i)
+    join()
     torch.cuda.synchronize()
     replicas.barrier()
     torch.cuda.synchronize()
 
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     with ClockSampler(local_rank) as clocks:
-        marks[0].record(stream)
+        marks[0].record(main)
+        fork()
         for i in range(args.steps):
             step(args.warmup + i)
-            marks[i + 1].record(stream)
+            if nb == 1:
+                marks[i + 1].record(main)
+        join()
+        if nb > 1:
+            marks[-1].record(main)
         torch.cuda.synchronize()
     replicas.barrier()
     torch.cuda.synchronize()
     local_ms = elapsed_ms = marks[0].elapsed_time(marks[-1])
-    step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    if nb == 1:
+        step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    else:
+        step_ms = [local_ms / args.steps]
     elapsed_ms = replicas.max_over_ranks(elapsed_ms)
-    launches = 2 * args.steps
-    counters = v.sentinel_get_counters()
+    launches = 2 * args.steps * nb
+    violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
 
     # end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    hx = {k: [xs[k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 4))] for k in (ACT, GRAD)}
+    hx = [{k: [xs[b][k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 2 if nb > 1 else 4))]
+           for k in (ACT, GRAD)} for b in range(nb)]
     hs = torch.empty(2, 1 + w.B, 3, dtype=torch.float32).pin_memory()
     hf = torch.empty(2, 1 + w.B, dtype=torch.int32).pin_memory()
-    v.sentinel_verify_host(hx[ACT][0], ACT, hs[0], hf[0], stream)        # allocates the staging
+    for b, v in enumerate(vs):                       # allocates the staging buffers
+        v.sentinel_verify_host(hx[b][ACT][0], ACT, hs[0], hf[0], main)
     torch.cuda.synchronize()
     replicas.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
+    e0.record(main)
     for i in range(e2e_steps):
-        v.sentinel_verify_host(hx[ACT][i % len(hx[ACT])], ACT, hs[0], hf[0], stream)
-        v.sentinel_verify_host(hx[GRAD][i % len(hx[GRAD])], GRAD, hs[1], hf[1], stream)
-    e1.record(stream)
+        for b, v in enumerate(vs):
+            v.sentinel_verify_host(hx[b][ACT][i % len(hx[b][ACT])], ACT, hs[0], hf[0], main)
+            v.sentinel_verify_host(hx[b][GRAD][i % len(hx[b][GRAD])], GRAD, hs[1], hf[1], main)
+    e1.record(main)
     torch.cuda.synchronize()
     e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1))
-    v.sentinel_destroy()
+    for v in vs:
+        v.sentinel_destroy()
 
-    bytes_step = 2 * N * BYTES_PER_ELEMENT                  # two tensors per step
+    bytes_step = 2 * N * BYTES_PER_ELEMENT * nb             # two tensors per boundary per step
     gbs = world * args.steps * bytes_step / (elapsed_ms * 1e-3) / 1e9
     e2e_gbs = world * e2e_steps * bytes_step / (e2e_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak_gbs()
@@ -193,25 +227,30 @@ def run_ours(args, rank, world, local_rank):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "impl": "sentinel_b200",
         "config": {"workload": "%s: B=%d x T=%d x d=%d bf16, activations %s, gradients N(0,%g), "
-                               "%g%% corrupted" % (w.name, w.B, w.T, w.d, w.act, w.grad_std, 100 * w.corrupt_rate),
-                   "step": "sentinel_verify(h, ACT) + sentinel_verify(g, GRAD)",
+                               "%g%% corrupted%s" % (w.name, w.B, w.T, w.d, w.act, w.grad_std, 100 * w.corrupt_rate,
+                                                     ", %d boundaries on %d CUDA streams" % (nb, nb) if nb > 1 else ""),
+                   "step": "sentinel_verify(h, ACT) + sentinel_verify(g, GRAD)" + (" on each boundary" if nb > 1 else ""),
                    "l2": "inputs larger than L2: %d MiB read+written per launch, %d distinct tensors per kind"
                          % (N * BYTES_PER_ELEMENT >> 20, nd),
                    "replicas": world},
-        "microbatches_per_s": round(world * args.steps / (elapsed_ms * 1e-3), 1),
-        "tensor_gbs": round(world * args.steps * 2 * N * 2 / (elapsed_ms * 1e-3) / 1e9, 1),
+        "microbatches_per_s": round(world * args.steps * nb / (elapsed_ms * 1e-3), 1),
+        "tensor_gbs": round(world * args.steps * nb * 2 * N * 2 / (elapsed_ms * 1e-3) / 1e9, 1),
         "ms_per_step_median": round(step_ms[len(step_ms) // 2], 4),
         "frac_of_8000_nominal": round(gbs / world / 8000.0, 4),
         "gpu_launches": launches,
-        "violations_seen": int(counters["violations"]),
+        "violations_seen": violations,
         "clocks": clocks.summary(),
         "e2e": {"value": round(e2e_gbs, 2), "unit": "GB/s", "steps": e2e_steps,
-                "h2d_bytes_per_step": 2 * N * 2,
-                "d2h_bytes_per_step": 2 * (1 + w.B) * (3 * 4 + 4),
+                "h2d_bytes_per_step": 2 * N * 2 * nb,
+                "d2h_bytes_per_step": 2 * (1 + w.B) * (3 * 4 + 4) * nb,
                 "api": "sentinel_verify_host"},
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "peak_source": "%s copy bandwidth" % peak_kind,
-                     "kernel": "stream_kernel", "avg_launch_ms": round(kernel_ms, 4),
+                     "kernel": "stream_kernel",
+                     "avg_launch_ms": round(kernel_ms, 4),
+                     "note": ("launches of different boundaries overlap: time per launch is the "
+                              "timed region divided by the launches" if nb > 1 else
+                              "timed region / launches; the region holds these launches only"),
                      "traffic": (args.traffic if args.traffic is not None else
                                  (round(NCU_DRAM_BYTES_PER_ELEMENT * N) if NCU_DRAM_BYTES_PER_ELEMENT else None)),
                      "traffic_source": "ncu on B=8x4096x4096, scaled by element count"},
