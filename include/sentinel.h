@@ -44,7 +44,7 @@ extern "C" {
 #define SENTINEL_NUM_STATS 8      /* mean_x var_x |x|_2 mean_m var_m cov_xm |m|_2 rho */
 #define SENTINEL_NUM_THRESHOLDS 6 /* q1 q2 q3 k tau_lower tau_upper                   */
 #define SENTINEL_MAX_B 64         /* samples per tensor                               */
-#define SENTINEL_MAX_WINDOW 4096  /* window_steps * B must not exceed this            */
+#define SENTINEL_MAX_WINDOW 4096  /* window_steps * (B + 1) must not exceed this      */
 
 typedef enum sentinel_status {
   SENTINEL_OK = 0,

@@ -1,6 +1,7 @@
 // Host side of libsentinel: argument checks, state ownership, launches.  See include/sentinel.h.
 #include "sentinel.h"
 
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -46,7 +47,8 @@ struct sentinel_verifier {
   size_t refresh_smem = 0;          // dynamic shared memory of a launch that may refresh thresholds
   float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
   HandleState *hs = nullptr;
-  double *hist[2] = {nullptr, nullptr};
+  double *hist[2] = {nullptr, nullptr};      // rings, device layout (ring_offset)
+  double *sorted[2] = {nullptr, nullptr};    // ascending copies of the windows (sorted_offset)
   unsigned long long *partials = nullptr;
   float *stats[2] = {nullptr, nullptr};
   float *token_buf = nullptr;
@@ -78,8 +80,14 @@ int fail(sentinel_verifier *h, int code, const char *fmt, ...) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// doubles of history in a checkpoint blob (and of the ascending copies on the device)
 size_t hist_doubles(const sentinel_verifier *h) {
   return (size_t)kNumMetrics * ((size_t)h->cap0 + (size_t)h->cap1);
+}
+
+// doubles of the rings on the device: each ring has one step's worth of slots more than its window
+size_t ring_doubles(const sentinel_verifier *h) {
+  return (size_t)kNumMetrics * ((size_t)ring_size(h->cap0, 1) + (size_t)ring_size(h->cap1, h->cfg.B));
 }
 
 size_t kind_blob_bytes(const sentinel_verifier *h) {
@@ -147,6 +155,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.ema[1] = h->ema[kind][1];
   a.hs = h->hs;
   a.hist = h->hist[kind];
+  a.sorted = h->sorted[kind];
   a.partials = h->partials;
   a.ticket = &h->hs->ticket;
   a.scores_out = scores;
@@ -176,8 +185,8 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) 
 }
 
 int run_refresh(sentinel_verifier *h, cudaStream_t s) {
-  refresh_kernel<<<1, kThreads, h->refresh_smem, s>>>(h->hs, h->hist[0], h->hist[1], h->cap0, h->cap1,
-                                        alg5_of(h->cfg, 0), alg5_of(h->cfg, 1));
+  refresh_kernel<<<1, kThreads, h->refresh_smem, s>>>(h->hs, h->hist[0], h->hist[1], h->sorted[0], h->sorted[1],
+                                                      h->cap0, h->cap1, h->cfg.B, alg5_of(h->cfg, 0), alg5_of(h->cfg, 1));
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
 }
@@ -196,6 +205,7 @@ void free_all(sentinel_verifier *h) {
   for (int k = 0; k < 2; ++k) {
     for (int j = 0; j < 2; ++j) cudaFree(h->ema[k][j]);
     cudaFree(h->hist[k]);
+    cudaFree(h->sorted[k]);
     cudaFree(h->stats[k]);
   }
   cudaFree(h->hs);
@@ -243,8 +253,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   }
   if (cfg->window_steps < 1 || cfg->ban_violations < 1 || cfg->forgiveness_steps < 1 || !(cfg->severe_mult > 0.0) || !(cfg->shrink_ratio >= 0.0))
     return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "window_steps, ban_violations, forgiveness_steps, severe_mult must be positive");
-  if ((long long)cfg->window_steps * cfg->B > SENTINEL_MAX_WINDOW)
-    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*B = %lld exceeds SENTINEL_MAX_WINDOW = %d", (long long)cfg->window_steps * cfg->B, SENTINEL_MAX_WINDOW);
+  if ((long long)cfg->window_steps * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d", (long long)cfg->window_steps * (cfg->B + 1), SENTINEL_MAX_WINDOW);
   int ndev = 0;
   SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
   if (cfg->device < 0 || cfg->device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist (%d devices)", cfg->device, ndev);
@@ -259,9 +269,10 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->N = h->Ns * cfg->B;
   h->cap0 = cfg->window_steps;
   h->cap1 = cfg->window_steps * cfg->B;
-  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1) * sizeof(double);
-  {   // the six padded windows may exceed the 48 KiB a kernel gets without asking
-    const int most = (int)(refresh_smem_doubles(SENTINEL_MAX_WINDOW, SENTINEL_MAX_WINDOW) * sizeof(double));
+  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1, cfg->B) * sizeof(double);
+  {   // the windows' working copies may exceed the 48 KiB a kernel gets without asking;
+      // window_steps*(B+1) <= SENTINEL_MAX_WINDOW bounds them
+    const int most = (int)((size_t)kNumMetrics * (2 * (size_t)SENTINEL_MAX_WINDOW + 4 * (SENTINEL_MAX_B + 1)) * sizeof(double));
     cudaError_t ae = cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
@@ -277,7 +288,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   };
   for (int k = 0; k < 2; ++k) {
     for (int j = 0; j < 2; ++j) alloc((void **)&h->ema[k][j], h->N * sizeof(float));   // m_0 = 0
-    alloc((void **)&h->hist[k], hist_doubles(h) * sizeof(double));
+    alloc((void **)&h->hist[k], ring_doubles(h) * sizeof(double));
+    alloc((void **)&h->sorted[k], hist_doubles(h) * sizeof(double));
     alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
   }
   alloc((void **)&h->partials, (size_t)h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));
@@ -478,7 +490,7 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
                    snap.violations, snap.clean_streak, snap.banned};
   memcpy(out, &hd, sizeof hd);
   out += kHeaderBytes;
-  std::vector<double> ring(hist_doubles(h));
+  std::vector<double> ring(ring_doubles(h));
   for (int k = 0; k < 2; ++k) {
     const KindState &ks = snap.kind[k];
     BlobKindHead kh;
@@ -492,14 +504,13 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
     SENTINEL_CUDA(h, cudaMemcpyAsync(ring.data(), h->hist[k], ring.size() * sizeof(double), cudaMemcpyDeviceToHost, s));
     SENTINEL_CUDA(h, cudaStreamSynchronize(s));
     double *dst = reinterpret_cast<double *>(out);
-    size_t src_off = 0;
     for (int L = 0; L < 2; ++L) {                   // unroll each ring, oldest entry first
-      const int cap = L ? h->cap1 : h->cap0;
+      const int cap = L ? h->cap1 : h->cap0, size = ring_size(cap, L ? h->cfg.B : 1);
       for (int i = 0; i < kNumMetrics; ++i) {
+        const size_t src_off = ring_offset(L, i, h->cap0, h->cap1, h->cfg.B);
         for (int j = 0; j < cap; ++j)
-          dst[j] = (j < ks.hist_count[L]) ? ring[src_off + (size_t)((ks.hist_head[L] + j) % cap)] : 0.0;
+          dst[j] = (j < ks.hist_count[L]) ? ring[src_off + (size_t)((ks.hist_head[L] + j) % size)] : 0.0;
         dst += cap;
-        src_off += cap;
       }
     }
     out = reinterpret_cast<unsigned char *>(dst);
@@ -552,7 +563,26 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
     ks.hist_head[0] = ks.hist_head[1] = 0;
     memcpy(ks.has_thr, kh.valid, sizeof kh.valid);
     memcpy(ks.thr, kh.thr, sizeof kh.thr);
-    SENTINEL_CUDA(h, cudaMemcpyAsync(h->hist[k], p, hist_doubles(h) * sizeof(double), cudaMemcpyHostToDevice, s));
+    ks.last_joined[0] = ks.last_joined[1] = 0;
+    ks.last_evicted[0] = ks.last_evicted[1] = 0;
+    {   // windows start at ring slot 0; the ascending copies are sorted here, on the host
+      std::vector<double> rings(ring_doubles(h), 0.0), asc(hist_doubles(h), 0.0);
+      const double *src = reinterpret_cast<const double *>(p);
+      for (int L = 0; L < 2; ++L) {
+        const int cap = L ? h->cap1 : h->cap0;
+        for (int i = 0; i < kNumMetrics; ++i) {
+          double *r = rings.data() + ring_offset(L, i, h->cap0, h->cap1, h->cfg.B);
+          double *a = asc.data() + sorted_offset(L, i, h->cap0, h->cap1);
+          std::copy(src, src + kh.count[L], r);
+          std::copy(src, src + kh.count[L], a);
+          std::sort(a, a + kh.count[L]);
+          src += cap;
+        }
+      }
+      SENTINEL_CUDA(h, cudaMemcpyAsync(h->hist[k], rings.data(), rings.size() * sizeof(double), cudaMemcpyHostToDevice, s));
+      SENTINEL_CUDA(h, cudaMemcpyAsync(h->sorted[k], asc.data(), asc.size() * sizeof(double), cudaMemcpyHostToDevice, s));
+      SENTINEL_CUDA(h, cudaStreamSynchronize(s));     // the staging vectors go out of scope
+    }
     p += hist_doubles(h) * sizeof(double);
     SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], p, h->N * sizeof(float), cudaMemcpyHostToDevice, s));
     p += h->N * sizeof(float);

@@ -53,6 +53,8 @@ struct KindState {
   int refresh_pending;    // Alg. 5 is owed for the history as it stands
   int hist_count[2];      // entries in the window, per level
   int hist_head[2];       // ring position of the oldest entry
+  int last_joined[2];     // entries the last step appended / pushed out, per level: what the
+  int last_evicted[2];    //   pending refresh has to merge into the sorted copy
   int has_thr[2][kNumMetrics];
   double thr[2][kNumMetrics][kNumThr];   // q1 q2 q3 k tau_lower tau_upper
 };
@@ -69,7 +71,8 @@ struct StreamArgs {
   const float *m_ext;              // distance mode: caller's reference; else unused
   float *ema[2];                   // the two reference buffers of this kind
   HandleState *hs;                 // nullptr in distance mode
-  double *hist;                    // this kind's rings: level 0 [3][cap0], level 1 [3][cap1]
+  double *hist;                    // this kind's rings: level 0 [3][cap0+1], level 1 [3][cap1+B]
+  double *sorted;                  // the same windows kept ascending: [3][cap0], [3][cap1]
   unsigned long long *partials;    // [G][2][kSlotWords]
   unsigned *ticket;
   float *scores_out;               // [(1+B)*3] or nullptr
@@ -351,13 +354,18 @@ __device__ __forceinline__ double percentile_sorted(const double *s, int n, doub
   return __dadd_rn(s[lo], __dmul_rn(frac, __dsub_rn(s[hi], s[lo])));
 }
 
-// entries strictly outside [lo, hi], counted by one warp
-__device__ __forceinline__ int warp_count_outside(const double *s, int n, double lo, double hi, int lane) {
-  int c = 0;
-  for (int j = lane; j < n; j += 32) c += (s[j] < lo || s[j] > hi);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-  return c;
+// History layout.  A window of at most `cap` entries lives in a ring of cap + units slots
+// (units = entries one step can append: 1 at level 0, B at level 1), so the entries a step
+// pushes out stay readable until the next step appends: the refresh that follows a step finds
+// both what joined and what left.  Next to each ring the same window is kept in ascending
+// order; a refresh merges the few changes into it instead of sorting the window again.
+__host__ __device__ inline int ring_size(int cap, int units) { return cap + units; }
+__host__ __device__ inline size_t ring_offset(int L, int i, int cap0, int cap1, int B) {
+  return L ? (size_t)kNumMetrics * ring_size(cap0, 1) + (size_t)i * ring_size(cap1, B)
+           : (size_t)i * ring_size(cap0, 1);
+}
+__host__ __device__ inline size_t sorted_offset(int L, int i, int cap0, int cap1) {
+  return L ? (size_t)kNumMetrics * cap0 + (size_t)i * cap1 : (size_t)i * cap0;
 }
 
 constexpr int kGroupThreads = 96;        // three warps work on one (level, metric) window
@@ -368,50 +376,113 @@ __device__ __forceinline__ void group_barrier(int group) {   // named barrier 1 
   asm volatile("bar.sync %0, %1;" :: "r"(group + 1), "r"(kGroupThreads) : "memory");
 }
 
-__host__ __device__ inline int pow2_at_least(int n) {
-  int p = 1;
-  while (p < n) p <<= 1;
-  return p;
+// doubles of shared memory the refresh needs: per window the old and the new ascending copy
+// (cap each), a staging area for what left and what joined (2*units) and their sorted lists
+// (units each)
+__host__ __device__ inline size_t window_smem_doubles(int cap, int units) {
+  return 2 * (size_t)cap + 4 * (size_t)units;
+}
+__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1, int B) {
+  return (size_t)kNumMetrics * (window_smem_doubles(cap0, 1) + window_smem_doubles(cap1, B));
 }
 
-// doubles of shared memory the refresh needs: a padded copy of each of the six windows
-__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1) {
-  return (size_t)kNumMetrics * ((size_t)pow2_at_least(cap0) + (size_t)pow2_at_least(cap1));
+__device__ __forceinline__ int lower_bound(const double *a, int n, double v) {   // # entries < v
+  int lo = 0, hi = n;
+  while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] < v) lo = mid + 1; else hi = mid; }
+  return lo;
+}
+__device__ __forceinline__ int upper_bound(const double *a, int n, double v) {   // # entries <= v
+  int lo = 0, hi = n;
+  while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] <= v) lo = mid + 1; else hi = mid; }
+  return lo;
+}
+
+// # entries of the ascending array s that are < x (strict) or <= x, found by one warp in two
+// rounds: 32 evenly spaced probes pick a block, then the block is scanned
+template <bool kOrEqual>
+__device__ __forceinline__ int warp_rank(const double *s, int n, double x, int lane) {
+  const int stride = (n + 31) >> 5;
+  const int i0 = lane * stride;
+  const bool below0 = (i0 < n) && (kOrEqual ? (s[i0] <= x) : (s[i0] < x));
+  const int c = __popc(__ballot_sync(0xffffffffu, below0));   // block starts below x: a prefix
+  if (c == 0) return 0;
+  const int base = (c - 1) * stride;
+  int count = base;
+  for (int t = 0; t < stride; t += 32) {
+    const int idx = base + t + lane;
+    const bool below = (t + lane < stride) && (idx < n) && (kOrEqual ? (s[idx] <= x) : (s[idx] < x));
+    count += __popc(__ballot_sync(0xffffffffu, below));
+  }
+  return count;
+}
+
+// entries strictly outside [lo, hi] of an ascending window
+__device__ __forceinline__ int warp_count_outside(const double *s, int n, double lo, double hi, int lane) {
+  return warp_rank<false>(s, n, lo, lane) + (n - warp_rank<true>(s, n, hi, lane));
 }
 
 // Refreshes q1,q2,q3,k,tau of every (level, metric) window of one kind (Alg. 5).  Whole CTA:
 // the six windows are handled side by side, each by three warps with their own named barrier.
-__device__ void refresh_thresholds(KindState *ks, const double *hist, int cap0, int cap1,
-                                   const Alg5Params &a5, double *s_dyn) {
+__device__ void refresh_thresholds(KindState *ks, const double *hist, double *sorted, int cap0, int cap1,
+                                   int B, const Alg5Params &a5, double *s_dyn) {
   const int group = threadIdx.x / kGroupThreads;
   const int gt = threadIdx.x - group * kGroupThreads;
   if (group < kRefreshGroups) {
     const int L = group / kNumMetrics, i = group - L * kNumMetrics;
     const int n = ks->hist_count[L];
     if (n > 0) {                                   // an empty window leaves everything as it is
-      const int cap = L ? cap1 : cap0;
-      const int pad0 = pow2_at_least(cap0), pad1 = pow2_at_least(cap1);
-      double *s_sort = s_dyn + (L ? (size_t)kNumMetrics * pad0 + (size_t)i * pad1 : (size_t)i * pad0);
-      const double *ring = hist + (L ? (size_t)kNumMetrics * cap0 : 0) + (size_t)i * cap;
-      const int npad = pow2_at_least(n);
-      // the order of the window is immaterial to Alg. 5, so the ring is read as it lies
-      for (int j = gt; j < npad; j += kGroupThreads) s_sort[j] = (j < n) ? ring[j] : CUDART_INF;
+      const int cap = L ? cap1 : cap0, units = L ? B : 1, size = ring_size(cap, units);
+      const int joined = ks->last_joined[L], evicted = ks->last_evicted[L], head = ks->hist_head[L];
+      const int n_old = n - joined + evicted;
+      const double *ring = hist + ring_offset(L, i, cap0, cap1, B);
+      double *srt = sorted + sorted_offset(L, i, cap0, cap1);
+      // this window's shared memory: old copy, new copy, staging, what left, what joined
+      double *s_old = s_dyn + (L ? (size_t)kNumMetrics * window_smem_doubles(cap0, 1) +
+                                       (size_t)i * window_smem_doubles(cap1, B)
+                                 : (size_t)i * window_smem_doubles(cap0, 1));
+      double *s_new = s_old + cap, *s_stage = s_new + cap, *s_out = s_stage + 2 * units, *s_in = s_out + units;
+
+      for (int p = gt; p < n_old; p += kGroupThreads) s_old[p] = srt[p];
+      // the entries pushed out sit just before the head, the ones that joined at the tail;
+      // stage them, then rank-sort them (they are few) into s_out / s_in
+      for (int j = gt; j < evicted; j += kGroupThreads) s_stage[j] = ring[(head - evicted + j + size) % size];
+      for (int j = gt; j < joined; j += kGroupThreads) s_stage[evicted + j] = ring[(head + n - joined + j) % size];
       group_barrier(group);
-      for (int k2 = 2; k2 <= npad; k2 <<= 1) {     // bitonic sort, ascending
-        for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
-          for (int t = gt; t < npad; t += kGroupThreads) {
-            const int partner = t ^ j2;
-            if (partner > t) {
-              const double va = s_sort[t], vb = s_sort[partner];
-              const bool up = ((t & k2) == 0);
-              if ((va > vb) == up) { s_sort[t] = vb; s_sort[partner] = va; }
-            }
-          }
-          group_barrier(group);
-        }
+      for (int j = gt; j < evicted + joined; j += kGroupThreads) {
+        const bool is_out = j < evicted;
+        const double *src = is_out ? s_stage : s_stage + evicted;
+        const int m = is_out ? evicted : joined, jj = is_out ? j : j - evicted;
+        const double v = src[jj];
+        int rank = 0;
+        for (int q = 0; q < m; ++q) rank += (src[q] < v) || (src[q] == v && q < jj);
+        (is_out ? s_out : s_in)[rank] = v;
       }
+      group_barrier(group);
+      // merge: old entries keep their order, lose the first copies of what left, and make
+      // room for what joined (a joining value goes after equal old ones)
+      for (int p = gt; p < n_old; p += kGroupThreads) {
+        const double v = s_old[p];
+        const int out_lt = lower_bound(s_out, evicted, v);
+        const int out_eq = upper_bound(s_out, evicted, v) - out_lt;
+        int gone_before = out_lt;
+        bool gone = false;
+        if (out_eq > 0) {                          // v is a value that left: its first copies go
+          const int copy = p - lower_bound(s_old, n_old, v);
+          gone = copy < out_eq;
+          gone_before += gone ? copy : out_eq;
+        }
+        if (!gone) s_new[p - gone_before + lower_bound(s_in, joined, v)] = v;
+      }
+      for (int j = gt; j < joined; j += kGroupThreads) {
+        const double v = s_in[j];
+        s_new[j + upper_bound(s_old, n_old, v) - upper_bound(s_out, evicted, v)] = v;
+      }
+      group_barrier(group);
+      for (int p = gt; p < n; p += kGroupThreads) srt[p] = s_new[p];
+
       if (gt < 32) {                               // the group's first warp walks the steps
         const int lane = gt;
+        const double *s_sort = s_new;
         const double q1 = percentile_sorted(s_sort, n, 0.25);
         const double q2 = percentile_sorted(s_sort, n, 0.50);
         const double q3 = percentile_sorted(s_sort, n, 0.75);
@@ -460,7 +531,11 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, int cap0, 
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0) ks->refresh_pending = 0;
+  if (threadIdx.x == 0) {
+    ks->refresh_pending = 0;
+    ks->last_joined[0] = ks->last_joined[1] = 0;   // the sorted copies are up to date
+    ks->last_evicted[0] = ks->last_evicted[1] = 0;
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -636,17 +711,16 @@ __device__ void finalize(const StreamArgs &a) {
   if (tid < rows) {
     const bool joins = (a.mode == kModeVerify) ? (my_flag == 0u) : warmup_ok;
     if (joins) {
-      // the k-th unit of a level to join goes to ring slot (head + count + k) mod cap, which
-      // is the oldest entry's slot once the window is full
-      const int L = tid ? 1 : 0, cap = L ? a.cap1 : a.cap0;
+      // the k-th unit of a level to join goes to ring slot (head + count + k) mod size; the
+      // ring has `units` slots more than the window, so what is pushed out is not overwritten
+      const int L = tid ? 1 : 0, size = ring_size(L ? a.cap1 : a.cap0, L ? B : 1);
       int k = 0;
       if (L && a.mode == kModeVerify)
         for (int r = 1; r < tid; ++r) k += (s_flag[r] == 0u);
       else if (L)
         k = tid - 1;
-      const int idx = (int)(((long long)ring_head + ring_count + k) % cap);
-      double *base = a.hist + (L ? (size_t)kNumMetrics * a.cap0 : 0);
-      for (int i = 0; i < kNumMetrics; ++i) base[(size_t)i * cap + idx] = g[i];
+      const int idx = (int)(((long long)ring_head + ring_count + k) % size);
+      for (int i = 0; i < kNumMetrics; ++i) a.hist[ring_offset(L, i, a.cap0, a.cap1, B) + idx] = g[i];
     }
     if (a.scores_out)
       for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = (float)g[i];
@@ -693,11 +767,12 @@ __device__ void finalize(const StreamArgs &a) {
       ks->active ^= 1;
     }
     for (int L = 0; L < 2; ++L) {                // window bookkeeping after `joined` appends
-      const int cap = L ? a.cap1 : a.cap0;
+      const int cap = L ? a.cap1 : a.cap0, size = ring_size(cap, L ? B : 1);
       const int total = ks->hist_count[L] + joined[L];
       const int evicted = total > cap ? total - cap : 0;
       ks->hist_count[L] = total - evicted;
-      ks->hist_head[L] = (int)(((long long)ks->hist_head[L] + evicted) % cap);
+      ks->hist_head[L] = (int)(((long long)ks->hist_head[L] + evicted) % size);
+      if (ks->refresh_pending) { ks->last_joined[L] = joined[L]; ks->last_evicted[L] = evicted; }
     }
     s_hs.ticket = 0u;                            // ready for the next launch
     s_status = status;
@@ -740,7 +815,7 @@ stream_kernel(const StreamArgs a) {
   if (blockIdx.x == 0) {
     if (a.hs) {
       KindState *ks = &a.hs->kind[a.kind];
-      if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.cap0, a.cap1, a.a5, s_dyn);
+      if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.B, a.a5, s_dyn);
     }
   } else {
     stream_cta(a, blockIdx.x - 1, m_in, m_out, s_part);
@@ -760,12 +835,14 @@ stream_kernel(const StreamArgs a) {
 
 // Brings both kinds' thresholds up to date outside a streaming launch (queries, export).
 __global__ void __launch_bounds__(kThreads)
-refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, int cap0, int cap1,
-               Alg5Params a5_act, Alg5Params a5_grad) {
+refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, double *sorted_act,
+               double *sorted_grad, int cap0, int cap1, int B, Alg5Params a5_act, Alg5Params a5_grad) {
   extern __shared__ double s_dyn[];
-  if (hs->kind[0].refresh_pending) refresh_thresholds(&hs->kind[0], hist_act, cap0, cap1, a5_act, s_dyn);
+  if (hs->kind[0].refresh_pending)
+    refresh_thresholds(&hs->kind[0], hist_act, sorted_act, cap0, cap1, B, a5_act, s_dyn);
   __syncthreads();
-  if (hs->kind[1].refresh_pending) refresh_thresholds(&hs->kind[1], hist_grad, cap0, cap1, a5_grad, s_dyn);
+  if (hs->kind[1].refresh_pending)
+    refresh_thresholds(&hs->kind[1], hist_grad, sorted_grad, cap0, cap1, B, a5_grad, s_dyn);
 }
 
 __global__ void reset_worker_kernel(HandleState *hs) {

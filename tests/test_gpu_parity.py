@@ -278,6 +278,22 @@ def test_streams_in_lockstep(sb, oracle_mod, name, shape, steps):
     gv.close()
 
 
+@pytest.mark.parametrize("shape,l", [((5, 2, 8), 4), ((3, 4, 16), 9), ((16, 8, 64), 6)],
+                         ids=["5x2x8_l4", "3x4x16_l9", "16x8x64_l6"])
+def test_long_streams_with_small_windows(sb, oracle_mod, shape, l):
+    """Many more steps than the window holds, on tensors so small that the sign-flip ratio takes
+    few distinct values: the windows wrap again and again and are full of equal entries, which
+    is what the incrementally maintained ascending copies have to get right."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "tiny_stream", *shape, corrupt_rate=0.3, warmup=6)
+    gv, ov, params = make_pair(sb, oracle_mod, w, l=l)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, 70)
+    compare_state(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+    assert rec["near"] + rec["k_events"] <= 6, rec
+    gv.close()
+
+
 def test_many_boundaries_on_separate_streams(sb, oracle_mod):
     """Config-5 pattern: independent handles, one CUDA stream each, interleaved act/grad."""
     w = synth.scaled(synth.WORKLOADS["cfg5"], "cfg5_small", 4, 32, 512, corrupt_rate=0.2, boundaries=4)
@@ -466,6 +482,10 @@ def test_argument_errors_never_reach_the_gpu(sb):
     with pytest.raises(sb.SentinelError) as e:
         sb.Verifier(64, 4, 8, window_steps=100)
     assert e.value.code == sb.ERR_UNSUPPORTED
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(40, 4, 8, window_steps=100)           # 100 * 41 > 4096
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    sb.Verifier(39, 4, 8, window_steps=100).close()      # 100 * 40 fits
     for bad in (dict(beta=(1.0, 0.5)), dict(gamma_grow=(0.9, 1.1)), dict(window_steps=0), dict(device=99)):
         with pytest.raises(sb.SentinelError) as e:
             sb.Verifier(2, 4, 8, **bad)
