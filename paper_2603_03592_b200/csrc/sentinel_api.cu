@@ -179,8 +179,20 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
 }
 
 int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) {
-  stream_kernel<<<grid, kThreads, h->refresh_smem, s>>>(a);
-  SENTINEL_CUDA(h, cudaGetLastError());
+  // launched with programmatic stream serialization: the grid may be set up while the previous
+  // kernel on the stream drains; every CTA waits for that kernel before it reads anything
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = dim3((unsigned)grid);
+  lc.blockDim = dim3(kThreads);
+  lc.dynamicSmemBytes = h->refresh_smem;
+  lc.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &attr;
+  lc.numAttrs = 1;
+  SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel, a));
   return SENTINEL_OK;
 }
 

@@ -801,6 +801,12 @@ stream_kernel(const StreamArgs a) {
   __shared__ int s_last;
   extern __shared__ double s_dyn[];            // refresh_smem_doubles(cap0, cap1) when a handle is given
 
+  // Programmatic dependent launch: let the next launch on the stream be set up while this one
+  // runs, and do not touch memory before the previous launch has completed and flushed.  With
+  // a plain launch both instructions do nothing.
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   const float *m_in;
   float *m_out;
   if (a.mode == kModeDistance) {
