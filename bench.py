@@ -192,6 +192,27 @@ def run_ours(args, rank, world, local_rank):
     launches = 2 * args.steps * nb
     violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
 
+    # extra figure, outside the timed region: gradient replacement (Alg. 4) after a flagged step
+    replace = None
+    if nb == 1:
+        v0 = vs[0]
+        loud = (xs[0][GRAD][0].float() * 64.0).to(torch.bfloat16)
+        v0.sentinel_verify(loud, GRAD, scores[0, 1], flags[0, 1], main)       # flagged: no commit
+        outs = [torch.empty_like(loud) for _ in range(4)]
+        for o in outs:
+            v0.sentinel_replace_if_flagged(o, GRAD, 0, None, main)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        r0.record(main)
+        for i in range(12):
+            v0.sentinel_replace_if_flagged(outs[i % 4], GRAD, 0, None, main)
+        r1.record(main)
+        torch.cuda.synchronize()
+        rms = r0.elapsed_time(r1) / 12
+        replace = {"kernel": "replace_kernel", "bytes_per_element": 6, "ms_per_launch": round(rms, 4),
+                   "achieved_gbs": round(6 * N / (rms * 1e-3) / 1e9, 1),
+                   "flagged": bool(int(flags[0, 1, 0]) & 0xFFFF)}
+
     # end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     hx = [{k: [xs[b][k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 2 if nb > 1 else 4))]
@@ -255,6 +276,8 @@ def run_ours(args, rank, world, local_rank):
                                  (round(NCU_DRAM_BYTES_PER_ELEMENT * N) if NCU_DRAM_BYTES_PER_ELEMENT else None)),
                      "traffic_source": "ncu on B=8x4096x4096, scaled by element count"},
     }
+    if replace is not None:
+        out["gradient_replacement"] = replace
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
     return out

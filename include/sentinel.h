@@ -176,6 +176,17 @@ int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_
  * token's d channels.  NULL unregisters.  The buffer stays the caller's. */
 int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf);
 
+/* Gradient replacement (Alg. 4) for the submission this handle sees.  If the last
+ * sentinel_verify of `kind` raised a flag (the step was not committed), dev_x_inout -- the
+ * tensor about to be forwarded, bf16 [B,T,d], 16-byte aligned -- is overwritten with the stored
+ * reference m_{t-1} rounded to bf16 (fill = 0), or with zeros (fill = 1, the variant the SWARM
+ * appendix prefers); if it was clean, the tensor is left as it is.  The decision is taken on
+ * the device: the call only enqueues work and never waits for the verify call before it.
+ * dev_replaced_out (u32, may be NULL) receives 1 if the tensor was overwritten, else 0. */
+int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentinel_kind kind, int B,
+                                int T, int d, int fill, void *cuda_stream,
+                                unsigned *dev_replaced_out);
+
 /* A new worker now feeds this boundary: clears the violation counter, the clean streak and
  * the ban (the paper keeps these per worker).  Enqueued on cuda_stream. */
 int sentinel_reset_worker(sentinel_verifier *h, void *cuda_stream);

@@ -86,6 +86,10 @@ def lib():
         L.so_update_reference.restype = C.c_int
         L.so_verify.argtypes = [C.c_void_p, u16p, C.c_int, dp, C.POINTER(C.c_uint32)]
         L.so_verify.restype = C.c_int
+        L.so_bf16_round.argtypes = [C.c_double]
+        L.so_bf16_round.restype = C.c_uint16
+        L.so_replace_if_flagged.argtypes = [C.c_void_p, u16p, C.c_int, C.c_int]
+        L.so_replace_if_flagged.restype = C.c_int
         L.so_reset_worker.argtypes = [C.c_void_p]
         L.so_reset_worker.restype = None
         L.so_ema.argtypes = [C.c_void_p, C.c_int]
@@ -185,6 +189,11 @@ def distance(x_bits, m) -> tuple[np.ndarray, np.ndarray, bool]:
     return g, s, bool(nf)
 
 
+def bf16_round(v: float) -> int:
+    """double -> bf16 bit pattern, round to nearest even in one step."""
+    return int(lib().so_bf16_round(float(v)))
+
+
 def percentile(sorted_vals, p: float) -> float:
     a = np.ascontiguousarray(sorted_vals, dtype=np.float64)
     return float(lib().so_percentile(_dptr(a), a.size, p))
@@ -239,6 +248,13 @@ class Verifier:
         commit = lib().so_verify(self._h, _u16ptr(xb), kind, _dptr(scores),
                                  flags.ctypes.data_as(C.POINTER(C.c_uint32)))
         return scores, flags, bool(commit)
+
+    def replace_if_flagged(self, x_bits, kind: int, fill: int = 0):
+        """Alg. 4 on a copy of x: (new bit patterns, replaced?)."""
+        xb = _bits(x_bits).reshape(-1).copy()
+        assert xb.size == self.N
+        did = lib().so_replace_if_flagged(self._h, _u16ptr(xb), kind, fill)
+        return xb.reshape(self.B, self.T, self.d), bool(did)
 
     def reset_worker(self):
         lib().so_reset_worker(self._h)

@@ -18,6 +18,28 @@ double so_bf16(uint16_t bits) {
   return (double)f;
 }
 
+uint16_t so_bf16_round(double v) {
+  if (isnan(v)) return 0x7FC0;
+  const uint16_t sign = signbit(v) ? 0x8000 : 0x0000;
+  const double a = fabs(v);
+  if (isinf(a)) return (uint16_t)(sign | 0x7F80);
+  /* lo = the largest bf16 magnitude <= a, hi = the next one; pick the nearer, ties to even */
+  float f = (float)a;
+  uint32_t u;
+  memcpy(&u, &f, sizeof u);
+  u &= 0xFFFF0000u;
+  if (so_bf16((uint16_t)(u >> 16)) > a) u -= 0x10000u;   /* the float rounding went above a */
+  const uint16_t lo = (uint16_t)(u >> 16), hi = (uint16_t)(lo + 1);
+  const double dlo = a - so_bf16(lo);
+  /* past the largest finite bf16 the next grid point is 2^128, which rounds to infinity */
+  const double dhi = (isinf(so_bf16(hi)) ? ldexp(1.0, 128) : so_bf16(hi)) - a;
+  uint16_t pick;
+  if (dlo < dhi) pick = lo;
+  else if (dlo > dhi) pick = hi;
+  else pick = (lo & 1) ? hi : lo;
+  return (uint16_t)(sign | pick);
+}
+
 /* three-valued sign: -1, 0, +1 (both zeros give 0) */
 static int sign3(double v) { return (v > 0.0) - (v < 0.0); }
 
@@ -193,6 +215,7 @@ typedef struct so_kind_state {
   int has_thr[2][SO_NMETRIC];
   double *stats;                              /* (1+B)*8 of the last call             */
   long steps;
+  int last_flagged;                           /* the last verified step raised a flag */
 } so_kind_state;
 
 struct so_verifier {
@@ -355,6 +378,7 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
 
   /* 6. the EMA moves only when nothing was flagged */
   const int commit = !any_flag;
+  ks->last_flagged = any_flag;
   if (commit) ema_update(v, x, kind);
 
   if (commit) flags[0] |= SO_FLAG_COMMITTED;
@@ -363,6 +387,13 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
   if (no_thr) flags[0] |= SO_FLAG_NO_THRESHOLDS;
   free(gam); free(nf);
   return commit;
+}
+
+int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill) {
+  if (!v->ks[kind].last_flagged) return 0;
+  const double *m = v->ks[kind].m;                 /* a flagged step left m at m_{t-1} */
+  for (size_t e = 0; e < v->N; ++e) x[e] = fill ? 0 : so_bf16_round(m[e]);
+  return 1;
 }
 
 void so_reset_worker(so_verifier *v) { v->violations = 0; v->clean_streak = 0; v->banned = 0; }

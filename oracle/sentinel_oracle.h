@@ -98,6 +98,15 @@ int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *sco
  * flags: (1+B) words.  Returns 1 if the EMA was updated (no unit flagged), else 0. */
 int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint32_t *flags);
 
+/* double -> bf16 bit pattern, round to nearest, ties to even (one rounding, straight from
+ * the double). */
+uint16_t so_bf16_round(double v);
+
+/* Alg. 4 (GradientReplacement) for one submission: if the last verified step of `kind` was
+ * flagged, x (n = B*T*d bf16 bit patterns) becomes the reference m_{t-1} rounded to bf16
+ * (fill = 0) or zeros (fill = 1); otherwise x is left alone.  Returns 1 if it replaced. */
+int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill);
+
 /* A new worker now feeds this boundary: clear its violation counter, streak and ban. */
 void so_reset_worker(so_verifier *v);
 

@@ -28,7 +28,7 @@ FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17,
 EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
-    "sentinel_distance_noalloc",
+    "sentinel_distance_noalloc", "sentinel_replace_if_flagged",
     "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
     "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
     "sentinel_export_state", "sentinel_import_state", "sentinel_last_error", "sentinel_destroy",
@@ -78,6 +78,7 @@ def lib():
         L.sentinel_verify_host.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_distance.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_distance_noalloc.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_replace_if_flagged.argtypes = [vp, vp, ip, ip, ip, ip, ip, vp, vp]
         L.sentinel_get_stats.argtypes = [vp, ip, vp, vp]
         L.sentinel_get_thresholds.argtypes = [vp, ip, vp, vp, vp]
         L.sentinel_get_counters.argtypes = [vp, vp, vp]
@@ -178,6 +179,14 @@ class Verifier:
         _check(lib().sentinel_verify_host(self._h, _ptr(x_host), kind, B, T, d,
                                           _stream_ptr(stream), _ptr(scores_host),
                                           _ptr(flags_host)), self._h)
+
+    def sentinel_replace_if_flagged(self, x_inout: torch.Tensor, kind: int, fill: int = 0,
+                                    replaced_out: torch.Tensor | None = None, stream=None) -> None:
+        """Alg. 4: overwrite x with the reference (fill=0) or zeros (fill=1) iff the last
+        verified step of this kind was flagged; decided on the device."""
+        B, T, d = x_inout.shape
+        _check(lib().sentinel_replace_if_flagged(self._h, _ptr(x_inout), kind, B, T, d, fill,
+                                                 _stream_ptr(stream), _ptr(replaced_out)), self._h)
 
     # convenience wrappers that allocate the outputs (tests, examples)
     def verify(self, x: torch.Tensor, kind: int, stream=None):

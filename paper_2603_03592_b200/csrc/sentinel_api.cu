@@ -410,6 +410,26 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   return SENTINEL_OK;
 }
 
+int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentinel_kind kind, int B, int T,
+                                int d, int fill, void *cuda_stream, unsigned *dev_replaced_out) {
+  int rc = check_call(h, dev_x_inout, kind, B, T, d);
+  if (rc) return rc;
+  if (fill != 0 && fill != 1) return fail(h, SENTINEL_ERR_INVALID_ARG, "fill must be 0 (reference) or 1 (zeros), got %d", fill);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  int sms = 0;
+  SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
+  const long long n_chunks = (long long)(h->N / 8);
+  long long grid = (long long)sms * 8;                       // 2048 threads per SM, grid-stride
+  const long long need = (n_chunks + kReplaceThreads - 1) / kReplaceThreads;
+  if (grid > need) grid = need;
+  replace_kernel<<<(unsigned)grid, kReplaceThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], static_cast<uint16_t *>(dev_x_inout), n_chunks, fill,
+      dev_replaced_out);
+  SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
+}
+
 int sentinel_get_stats(sentinel_verifier *h, sentinel_kind kind, float *dev_stats_out, void *cuda_stream) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (!dev_stats_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "stats_out is NULL");

@@ -55,6 +55,8 @@ struct KindState {
   int hist_head[2];       // ring position of the oldest entry
   int last_joined[2];     // entries the last step appended / pushed out, per level: what the
   int last_evicted[2];    //   pending refresh has to merge into the sorted copy
+  int last_flagged;       // the last verified step of this kind raised a flag (no commit)
+  int pad;
   int has_thr[2][kNumMetrics];
   double thr[2][kNumMetrics][kNumThr];   // q1 q2 q3 k tau_lower tau_upper
 };
@@ -756,6 +758,7 @@ __device__ void finalize(const StreamArgs &a) {
       joined[0] = (s_flag[0] == 0u);
       for (int r = 1; r < rows; ++r) joined[1] += (s_flag[r] == 0u);
       ks->refresh_pending = 1;
+      ks->last_flagged = any_flag ? 1 : 0;
       if (!any_flag) { ks->active ^= 1; status |= kFlagCommitted; }   // m_t := candidate
       if (s_severe) status |= kFlagSevere;
       if (hs->banned) status |= kFlagBanned;
@@ -849,6 +852,47 @@ refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, double *sor
   __syncthreads();
   if (hs->kind[1].refresh_pending)
     refresh_thresholds(&hs->kind[1], hist_grad, sorted_grad, cap0, cap1, B, a5_grad, s_dyn);
+}
+
+// Alg. 4 (GradientReplacement) for the one submission a handle sees: if the last verified step
+// of this kind was flagged, the outgoing tensor is overwritten with the reference m_{t-1}
+// rounded to bf16 (or with zeros, the variant of the SWARM appendix); otherwise nothing is
+// touched.  The decision is read on the device, so the call needs no host round trip.  A
+// flagged step did not commit, so the active buffer still holds m_{t-1}.
+// Traffic when it replaces: 4 B read + 2 B written per element (2 B written when zero-filling).
+constexpr int kReplaceThreads = 256;
+
+__device__ __forceinline__ void st_x128(uint16_t *p, const uint4 &v) {
+  asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__device__ __forceinline__ unsigned pack_bf16x2_rn(float lo, float hi) {
+  unsigned r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // upper half <- first operand
+  return r;
+}
+
+__global__ void __launch_bounds__(kReplaceThreads)
+replace_kernel(const HandleState *hs, int kind, const float *ema0, const float *ema1, uint16_t *x,
+               long long n_chunks, int zero_fill, unsigned *replaced_out) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const KindState *ks = &hs->kind[kind];
+  const int flagged = ks->last_flagged;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && replaced_out) *replaced_out = flagged ? 1u : 0u;
+  if (!flagged) return;
+  const float *m = ks->active ? ema1 : ema0;
+  const long long stride = (long long)gridDim.x * kReplaceThreads;
+  for (long long c = (long long)blockIdx.x * kReplaceThreads + threadIdx.x; c < n_chunks; c += stride) {
+    uint4 out = make_uint4(0u, 0u, 0u, 0u);
+    if (!zero_fill) {
+      const F8 v = ld_m256(m + c * 8);
+      out.x = pack_bf16x2_rn(v.v[0], v.v[1]);
+      out.y = pack_bf16x2_rn(v.v[2], v.v[3]);
+      out.z = pack_bf16x2_rn(v.v[4], v.v[5]);
+      out.w = pack_bf16x2_rn(v.v[6], v.v[7]);
+    }
+    st_x128(x + c * 8, out);
+  }
 }
 
 __global__ void reset_worker_kernel(HandleState *hs) {

@@ -438,6 +438,52 @@ def test_token_statistics_buffer(sb, oracle_mod, d):
     gv.close()
 
 
+@pytest.mark.parametrize("shape", [(3, 7, 264), (4, 64, 2048)], ids=["3x7x264", "4x64x2048"])
+def test_gradient_replacement(sb, oracle_mod, shape):
+    """Alg. 4 on the device: untouched after a clean step, the reference (bf16) or zeros after
+    a flagged one.  The library rounds its fp32 reference, the oracle its float64 one, so the
+    bf16 results may differ by one unit in the last place where the two references straddle a
+    rounding boundary (or by the EMA's own absolute accuracy where it nearly cancels): at most
+    1 element in 1000."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_repl", *shape)
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    for t in range(10):
+        g = synth.clean(w, 0, GRAD, t, "cuda")
+        gv.update_reference(g, GRAD)
+        ov.update_reference(synth.bits(g), GRAD)
+    did = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    g = synth.clean(w, 0, GRAD, 10, "cuda")
+    gv.verify(g, GRAD)
+    ov.verify(synth.bits(g), GRAD)
+    out = g.clone()
+    gv.sentinel_replace_if_flagged(out, GRAD, 0, did)
+    ref, ref_did = ov.replace_if_flagged(synth.bits(g), GRAD)
+    assert int(did) == 0 and not ref_did and torch.equal(out, g)
+
+    bad = (synth.clean(w, 0, GRAD, 11, "cuda").float() * 40.0).to(torch.bfloat16)
+    _, gf = gv.verify(bad, GRAD)
+    _, of, _ = ov.verify(synth.bits(bad), GRAD)
+    assert np.array_equal(gf.cpu().numpy().view(np.uint32), of) and (of[0] & 0xFFFF)
+    for fill in (0, 1):
+        out = bad.clone()
+        gv.sentinel_replace_if_flagged(out, GRAD, fill, did)   # enqueued right behind the verify
+        ref, ref_did = ov.replace_if_flagged(synth.bits(bad), GRAD, fill)
+        assert int(did) == 1 and ref_did
+        got = synth.bits(out)
+        gv_, rv_ = oracle_mod.bf16_to_f64(got), oracle_mod.bf16_to_f64(ref)
+        # one bf16 ulp of the value, plus the absolute accuracy of an fp32 EMA (elements where
+        # the EMA nearly cancels are tiny, and there the two references differ relatively a lot)
+        tol = 2.0 ** -7 * np.abs(rv_) + 1e-6 * rv_.std()
+        assert np.all(np.abs(gv_ - rv_) <= tol)
+        assert np.count_nonzero(got != ref) <= 1e-3 * got.size, np.count_nonzero(got != ref)
+        if fill:
+            assert not got.any()
+    out = torch.ones_like(bad)                                 # the other kind was never flagged
+    gv.sentinel_replace_if_flagged(out, ACT, 0, did)
+    assert int(did) == 0 and torch.all(out == 1)
+    gv.close()
+
+
 def test_runs_are_bit_reproducible(sb):
     w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_rep", 4, 50, 1024)
     blobs, outs = [], []
@@ -509,6 +555,9 @@ def test_argument_errors_never_reach_the_gpu(sb):
     assert L.sentinel_verify(h, x.data_ptr(), 0, 2, 4, 16, s, None, flags.data_ptr()) == sb.ERR_INVALID_ARG
     assert L.sentinel_verify(None, x.data_ptr(), 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_INVALID_ARG
     assert L.sentinel_update_reference(h, x.data_ptr(), 0, 3, 4, 16, s, None) == sb.ERR_SHAPE_MISMATCH
+    assert L.sentinel_replace_if_flagged(h, x.data_ptr(), 0, 2, 4, 16, 2, s, None) == sb.ERR_INVALID_ARG
+    assert L.sentinel_replace_if_flagged(h, x.data_ptr() + 2, 0, 2, 4, 16, 0, s, None) == sb.ERR_UNALIGNED
+    assert L.sentinel_replace_if_flagged(h, x.data_ptr(), 0, 2, 4, 8, 0, s, None) == sb.ERR_SHAPE_MISMATCH
     assert L.sentinel_export_state(h, bytes(8), 8, s) == sb.ERR_STATE_SIZE
     junk = bytearray(before)
     junk[0] ^= 0xFF

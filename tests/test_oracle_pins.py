@@ -277,3 +277,25 @@ def test_default_hyperparameters_match_the_paper_table(oracle_mod):
     for key, cname in [("c", "c"), ("t_forgiveness", "t_forgiveness"), ("l", "l"), ("severe_mult", "severe_mult")]:
         assert float(got[cname]) == want[key][0]
         assert float(getattr(py, cname)) == want[key][0]
+
+
+# ---------------------------------------------------------------- bf16 rounding (Alg. 4 output)
+
+def test_bf16_rounding_matches_the_library_on_floats_and_rounds_once(oracle_mod, rng):
+    """For values a float holds exactly, round-to-nearest-even to bf16 is torch's conversion; a
+    double just above a tie must go up although its float image sits on the tie."""
+    vals = np.concatenate([rng.normal(0, 1, 4000), rng.normal(0, 1e-4, 2000), rng.normal(0, 1e4, 2000),
+                           [0.0, -0.0, 1.0, -1.0, 65504.0, 3.3e38, 1e-40, -1e-40]]).astype(np.float32)
+    want = torch.from_numpy(vals).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([oracle_mod.bf16_round(float(v)) for v in vals], dtype=np.uint16)
+    assert np.array_equal(got, want)
+    # ties to even, by hand: 1 + 2^-8 is halfway between 1 (even) and 1 + 2^-7
+    assert oracle_mod.bf16_round(1 + 2.0 ** -8) == 0x3F80
+    assert oracle_mod.bf16_round(1 + 3 * 2.0 ** -8) == 0x3F82
+    assert oracle_mod.bf16_round(1 + 2.0 ** -8 + 2.0 ** -40) == 0x3F81      # one rounding, not two
+    assert oracle_mod.bf16_round(1 + 2.0 ** -8 - 2.0 ** -40) == 0x3F80
+    assert oracle_mod.bf16_round(float("inf")) == 0x7F80 and oracle_mod.bf16_round(-1e39) == 0xFF80
+    assert oracle_mod.bf16_round(float("nan")) & 0x7FC0 == 0x7FC0
+    # rounding is the identity on bf16 values
+    b = np.arange(0, 0x7F80, 37, dtype=np.uint16)
+    assert all(oracle_mod.bf16_round(float(v)) == int(u) for u, v in zip(b, from_bits(b)))

@@ -250,3 +250,28 @@ def test_metric_mask_limits_which_metrics_may_flag(oracle_mod, small):
     assert not np.any(f & oracle_mod.FLAG_L1)
     # scaling by 3 leaves the z-scored distance and the signs alone, so nothing else fires
     assert commit and np.all((f & 0xFFFF) == 0)
+
+
+def test_gradient_replacement_follows_the_last_verdict(oracle_mod, small):
+    """Alg. 4: a flagged submission is replaced by the reference m_{t-1} (or zeros); a clean one
+    is forwarded untouched."""
+    v = _warm(oracle_mod, small, 16)
+    g = synth.clean(small, 0, GRAD, 16)
+    _, flags, commit = v.verify(synth.bits(g), GRAD)
+    assert commit
+    out, did = v.replace_if_flagged(synth.bits(g), GRAD)
+    assert not did and np.array_equal(out, synth.bits(g))
+    bad = (synth.clean(small, 0, GRAD, 17).float() * 50.0).to(torch.bfloat16)
+    m_before = v.ema(GRAD)
+    _, flags, commit = v.verify(synth.bits(bad), GRAD)
+    assert not commit
+    out, did = v.replace_if_flagged(synth.bits(bad), GRAD)
+    assert did
+    got = from_bits(out)
+    assert np.all(np.abs(got - m_before) <= 2.0 ** -8 * np.abs(m_before) + 1e-45)   # half an ulp of bf16
+    zeros, did = v.replace_if_flagged(synth.bits(bad), GRAD, fill=1)
+    assert did and not zeros.any()
+    # the verdict is per kind: the activation side was never flagged
+    a = synth.clean(small, 0, ACT, 16)
+    out, did = v.replace_if_flagged(synth.bits(a), ACT)
+    assert not did
