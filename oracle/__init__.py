@@ -86,6 +86,8 @@ def lib():
         L.so_update_reference.restype = C.c_int
         L.so_verify.argtypes = [C.c_void_p, u16p, C.c_int, dp, C.POINTER(C.c_uint32)]
         L.so_verify.restype = C.c_int
+        L.so_sliced_wasserstein.argtypes = [u16p, dp, C.c_size_t, C.c_size_t, u16p, C.c_size_t, dp]
+        L.so_sliced_wasserstein.restype = C.c_double
         L.so_bf16_round.argtypes = [C.c_double]
         L.so_bf16_round.restype = C.c_uint16
         L.so_replace_if_flagged.argtypes = [C.c_void_p, u16p, C.c_int, C.c_int]
@@ -187,6 +189,21 @@ def distance(x_bits, m) -> tuple[np.ndarray, np.ndarray, bool]:
     s = np.empty(NSTAT)
     nf = lib().so_distance(_u16ptr(xb), _dptr(mm), xb.size, _dptr(g), _dptr(s))
     return g, s, bool(nf)
+
+
+def sliced_wasserstein(x_bits, m, u_bits):
+    """Sliced Wasserstein distance of one unit: x bits [tokens, d], m [tokens, d], directions
+    u bits [L, d].  Returns (mean over directions, per-direction W1)."""
+    xb = _bits(x_bits)
+    ub = _bits(u_bits)
+    tokens, d = xb.shape[-2] if xb.ndim == 2 else int(np.prod(xb.shape[:-1])), xb.shape[-1]
+    xb = xb.reshape(tokens, d)
+    mm = np.ascontiguousarray(m, dtype=np.float64).reshape(tokens, d)
+    Ld = ub.shape[0]
+    assert ub.shape == (Ld, d)
+    w1 = np.empty(Ld)
+    val = lib().so_sliced_wasserstein(_u16ptr(xb), _dptr(mm), tokens, d, _u16ptr(np.ascontiguousarray(ub)), Ld, _dptr(w1))
+    return float(val), w1
 
 
 def bf16_round(v: float) -> int:

@@ -130,6 +130,44 @@ int so_distance(const uint16_t *x, const double *m, size_t n, double gamma[3], d
 }
 
 /* ------------------------------------------------------------------------------------ */
+/* Sec. 3.1: sliced Wasserstein distance                                                  */
+
+static int cmp_double(const void *a, const void *b);
+
+double so_sliced_wasserstein(const uint16_t *x, const double *m, size_t tokens, size_t d,
+                             const uint16_t *u, size_t L, double *w1_per_direction) {
+  size_t t, c, l;
+  for (t = 0; t < tokens * d; ++t)
+    if (!isfinite(so_bf16(x[t]))) return NAN;
+  double *px = (double *)malloc(tokens * sizeof(double));
+  double *pm = (double *)malloc(tokens * sizeof(double));
+  double total = 0.0;
+  for (l = 0; l < L; ++l) {
+    /* push both clouds forward along direction u_l: one number per token */
+    for (t = 0; t < tokens; ++t) {
+      double ax = 0.0, am = 0.0;
+      for (c = 0; c < d; ++c) {
+        const double ul = so_bf16(u[l * d + c]);
+        ax += so_bf16(x[t * d + c]) * ul;
+        am += m[t * d + c] * ul;
+      }
+      px[t] = ax;
+      pm[t] = am;
+    }
+    /* W1 of two empirical measures with equally many atoms: match the order statistics */
+    qsort(px, tokens, sizeof(double), cmp_double);
+    qsort(pm, tokens, sizeof(double), cmp_double);
+    double w1 = 0.0;
+    for (t = 0; t < tokens; ++t) w1 += fabs(px[t] - pm[t]);
+    w1 /= (double)tokens;
+    if (w1_per_direction) w1_per_direction[l] = w1;
+    total += w1;
+  }
+  free(px); free(pm);
+  return total / (double)L;
+}
+
+/* ------------------------------------------------------------------------------------ */
 /* Alg. 5: adaptive IQR thresholds                                                       */
 
 double so_percentile(const double *sorted, size_t n, double p) {

@@ -98,6 +98,17 @@ int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *sco
  * flags: (1+B) words.  Returns 1 if the EMA was updated (no unit flagged), else 0. */
 int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint32_t *flags);
 
+/* Sec. 3.1, sliced Wasserstein distance of one unit.  x (bf16 bits) and m are clouds of
+ * `tokens` points in R^d (row-major [tokens][d]); u holds L directions as bf16 bit patterns,
+ * [L][d], which the caller has normalised.  For every direction both clouds are projected, the
+ * two sets of `tokens` projections are sorted, and W1 between the two empirical distributions
+ * is the mean absolute difference of the order statistics; the result is the mean over the
+ * L directions (a Monte-Carlo estimate of the expectation over the sphere with the caller's
+ * draws).  w1_per_direction, if not NULL, receives the L terms.  Returns NaN if x holds a
+ * non-finite value. */
+double so_sliced_wasserstein(const uint16_t *x, const double *m, size_t tokens, size_t d,
+                             const uint16_t *u, size_t L, double *w1_per_direction);
+
 /* double -> bf16 bit pattern, round to nearest, ties to even (one rounding, straight from
  * the double). */
 uint16_t so_bf16_round(double v);

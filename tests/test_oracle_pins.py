@@ -299,3 +299,43 @@ def test_bf16_rounding_matches_the_library_on_floats_and_rounds_once(oracle_mod,
     # rounding is the identity on bf16 values
     b = np.arange(0, 0x7F80, 37, dtype=np.uint16)
     assert all(oracle_mod.bf16_round(float(v)) == int(u) for u, v in zip(b, from_bits(b)))
+
+
+# ---------------------------------------------------------------- sliced Wasserstein (Sec. 3.1)
+
+def _directions(rng, L, d):
+    u = rng.normal(0, 1, (L, d))
+    u /= np.linalg.norm(u, axis=1, keepdims=True)
+    ub = to_bits(u)
+    return ub, from_bits(ub)
+
+
+def test_sliced_wasserstein_against_scipy_and_closed_forms(oracle_mod, rng):
+    tokens, d, L = 96, 40, 5
+    ub, u = _directions(rng, L, d)
+    xb = to_bits(rng.normal(0.2, 1.0, (tokens, d)))
+    x = from_bits(xb)
+    m = rng.normal(-0.1, 1.5, (tokens, d))
+    val, w1 = oracle_mod.sliced_wasserstein(xb, m, ub)
+    for l in range(L):                     # 1-D W1 of equal-size samples is scipy's routine
+        want = scipy.stats.wasserstein_distance(x @ u[l], m @ u[l])
+        assert w1[l] == pytest.approx(want, rel=1e-11)
+    assert val == pytest.approx(w1.mean(), rel=1e-14)
+    # identical clouds: zero; a cloud shifted by one vector v: every projection moves by u.v
+    assert oracle_mod.sliced_wasserstein(xb, x, ub)[0] == 0.0
+    v = rng.normal(0, 1, d)
+    val_s, w1_s = oracle_mod.sliced_wasserstein(xb, x + v, ub)
+    assert w1_s == pytest.approx(np.abs(u @ v), rel=1e-11)
+    # the order of the tokens is immaterial, separately for the two clouds
+    p1, p2 = rng.permutation(tokens), rng.permutation(tokens)
+    assert oracle_mod.sliced_wasserstein(xb[p1], m[p2], ub)[0] == pytest.approx(val, rel=1e-12)
+    # absolutely homogeneous: scaling both clouds by -4 (exact in bf16) scales the distance by 4
+    assert oracle_mod.sliced_wasserstein(to_bits(-4 * x), -4 * m, ub)[0] == pytest.approx(4 * val, rel=1e-12)
+    # two point masses per cloud, by hand: x projects to {0, 2}, m to {1, 5} along e1 -> (1 + 3)/2
+    e1 = to_bits(np.array([[1.0, 0.0]]))
+    val2, _ = oracle_mod.sliced_wasserstein(to_bits(np.array([[2.0, 7.0], [0.0, -3.0]])),
+                                            np.array([[5.0, 0.0], [1.0, 9.0]]), e1)
+    assert val2 == 2.0
+    bad = x.copy()
+    bad[3, 4] = np.inf
+    assert np.isnan(oracle_mod.sliced_wasserstein(to_bits(bad), m, ub)[0])
