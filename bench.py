@@ -213,6 +213,29 @@ def run_ours(args, rank, world, local_rank):
                    "achieved_gbs": round(6 * N / (rms * 1e-3) / 1e9, 1),
                    "flagged": bool(int(flags[0, 1, 0]) & 0xFFFF)}
 
+    # extra figure, outside the timed region: sliced Wasserstein distance along 8 directions
+    swd = None
+    if nb == 1 and 8 * w.d * 2 <= 200 * 1024 and w.T <= 16384:
+        g = torch.Generator(device=device).manual_seed(11)
+        u = torch.randn(8, w.d, generator=g, device=device)
+        u = (u / u.norm(dim=1, keepdim=True)).to(torch.bfloat16).contiguous()
+        ref = xs[0][ACT][1 % nd].float().mul_(0.1).contiguous()
+        sw = torch.empty(1 + w.B, dtype=torch.float32, device=device)
+        for _ in range(2):
+            binding.sentinel_sliced_wasserstein(xs[0][ACT][0], ref, u, sw, main)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        s0.record(main)
+        for i in range(8):
+            binding.sentinel_sliced_wasserstein(xs[0][ACT][i % nd], ref, u, sw, main)
+        s1.record(main)
+        torch.cuda.synchronize()
+        sms = s0.elapsed_time(s1) / 8
+        swd = {"directions": 8, "bytes_per_element": 6, "ms_per_call": round(sms, 4),
+               "achieved_gbs": round(6 * N / (sms * 1e-3) / 1e9, 1),
+               "kernels": "swd_project_kernel + sort, merge, finish", "value_row0": float(sw[0])}
+        del ref
+
     # end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     hx = [{k: [xs[b][k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 2 if nb > 1 else 4))]
@@ -278,6 +301,8 @@ def run_ours(args, rank, world, local_rank):
     }
     if replace is not None:
         out["gradient_replacement"] = replace
+    if swd is not None:
+        out["sliced_wasserstein"] = swd
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
     return out

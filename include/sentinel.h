@@ -130,9 +130,25 @@ int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind
 /* Stateless form of Eq. 2 / Sec. 3.1: the three distances and the statistics of x against a
  * reference supplied by the caller.  dev_m: fp32 [B,T,d], 16-byte aligned.  dev_scores_out
  * fp32 [(1+B)*3]; dev_stats_out fp32 [(1+B)*8] or NULL.  Needs a few KiB of scratch, which it
- * takes from and returns to the stream's memory pool (cudaMallocAsync). */
+ * takes from and returns to the stream's memory pool (cudaMallocAsync).  On first use the
+ * library raises the release threshold of the device's default pool to 64 MiB (never lowers
+ * it), so that the scratch is not handed back to the driver at every synchronisation. */
 int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d, int device,
                       void *cuda_stream, float *dev_scores_out, float *dev_stats_out);
+
+/* Sliced Wasserstein distance (Sec. 3.1), stateless: x and the reference m are read as clouds
+ * of tokens in R^d (B*T points for the whole tensor, T points for a sample); along each of L
+ * directions both clouds are projected, W1 of the two sets of projections is the mean
+ * absolute difference of their order statistics, and the L values are averaged.
+ * dev_u_bf16: the directions, bf16 [L, d], unit vectors chosen by the caller (the paper fixes
+ * neither their number nor their draw), 16-byte aligned.  L must be 4, 8 or 16; L*d*2 bytes
+ * must fit in 200 KiB of shared memory; T <= 16384.  dev_m: fp32 [B,T,d].
+ * dev_sw_out: fp32 [1+B], row 0 the whole tensor, row 1+b sample b; NaN propagates from a
+ * non-finite x.  Scratch (the projections, about 24*L*B*T bytes) comes from and returns to
+ * the stream's memory pool. */
+int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const void *dev_u_bf16, int L,
+                                int B, int T, int d, int device, void *cuda_stream,
+                                float *dev_sw_out);
 
 /* The same computation as sentinel_distance for callers that must not allocate device memory
  * while they run: code whose memory pool has been frozen after start-up, real-time loops

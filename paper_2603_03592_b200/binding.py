@@ -28,7 +28,7 @@ FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17,
 EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
-    "sentinel_distance_noalloc", "sentinel_replace_if_flagged",
+    "sentinel_distance_noalloc", "sentinel_replace_if_flagged", "sentinel_sliced_wasserstein",
     "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
     "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
     "sentinel_export_state", "sentinel_import_state", "sentinel_last_error", "sentinel_destroy",
@@ -78,6 +78,7 @@ def lib():
         L.sentinel_verify_host.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_distance.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_distance_noalloc.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_sliced_wasserstein.argtypes = [vp, vp, vp, ip, ip, ip, ip, ip, vp, vp]
         L.sentinel_replace_if_flagged.argtypes = [vp, vp, ip, ip, ip, ip, ip, vp, vp]
         L.sentinel_get_stats.argtypes = [vp, ip, vp, vp]
         L.sentinel_get_thresholds.argtypes = [vp, ip, vp, vp, vp]
@@ -132,6 +133,14 @@ def sentinel_distance(x: torch.Tensor, m: torch.Tensor, scores_out: torch.Tensor
     B, T, d = x.shape
     _check(lib().sentinel_distance(_ptr(x), _ptr(m), B, T, d, x.device.index or 0,
                                    _stream_ptr(stream), _ptr(scores_out), _ptr(stats_out)))
+
+
+def sentinel_sliced_wasserstein(x: torch.Tensor, m: torch.Tensor, u_bf16: torch.Tensor,
+                                sw_out: torch.Tensor, stream=None) -> None:
+    """Sliced Wasserstein distance of every unit along the caller's directions u (bf16 [L, d])."""
+    B, T, d = x.shape
+    _check(lib().sentinel_sliced_wasserstein(_ptr(x), _ptr(m), _ptr(u_bf16), u_bf16.shape[0], B, T, d,
+                                             x.device.index or 0, _stream_ptr(stream), _ptr(sw_out)))
 
 
 NOALLOC_SCRATCH_BYTES = 65536

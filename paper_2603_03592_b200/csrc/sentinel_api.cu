@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "sentinel_kernels.cuh"
+#include "sentinel_swd.cuh"
 
 using namespace sentinel;
 
@@ -126,6 +127,24 @@ int streaming_ctas(int device, int B, int T, std::string *err) {
     return -1;
   }
   return (int)G;
+}
+
+// The stateless entry points take their scratch from the device's default memory pool.  By
+// default that pool hands everything back to the driver whenever the stream is synchronised, so
+// the next call pays for a fresh driver allocation; keeping a little memory cached avoids that.
+// Only ever raises the threshold, once per device.
+void keep_pool_warm(int device) {
+  static std::mutex mu;
+  static bool done[64] = {false};
+  std::lock_guard<std::mutex> lock(mu);
+  if (device < 0 || device >= 64 || done[device]) return;
+  done[device] = true;
+  cudaMemPool_t pool;
+  if (cudaDeviceGetDefaultMemPool(&pool, device) != cudaSuccess) { cudaGetLastError(); return; }
+  unsigned long long cur = 0, want = 64ull << 20;
+  if (cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &cur) == cudaSuccess && cur < want)
+    cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &want);
+  cudaGetLastError();
 }
 
 int tiles_per_row(int d) { return ((d >> 3) + 32 * kUnroll - 1) / (32 * kUnroll); }
@@ -389,6 +408,7 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   // scratch: two partial slots per streaming CTA, then the ticket word
   const size_t slot_bytes = (size_t)G * kSegsPerCta * kSlotWords * sizeof(unsigned long long);
   unsigned char *scratch = nullptr;
+  keep_pool_warm(device);
   SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, slot_bytes + 256, s));
   SENTINEL_CUDA(nullptr, cudaMemsetAsync(scratch + slot_bytes, 0, 256, s));
 
@@ -427,6 +447,91 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
       h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], static_cast<uint16_t *>(dev_x_inout), n_chunks, fill,
       dev_replaced_out);
   SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+template <int L>
+cudaError_t launch_projection(const uint16_t *x, const float *m, const uint16_t *u, float *proj, long long rows,
+                              int d, int sms, cudaStream_t s) {
+  const size_t smem = (size_t)L * d * sizeof(uint16_t);
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, swd_project_kernel<L>, kSwdThreads, smem);
+  if (e != cudaSuccess) return e;
+  if (occ < 1) return cudaErrorInvalidConfiguration;
+  long long grid = (long long)sms * occ;
+  const long long need = (rows + kSwdThreads / 32 - 1) / (kSwdThreads / 32);
+  if (grid > need) grid = need;
+  swd_project_kernel<L><<<(unsigned)grid, kSwdThreads, smem, s>>>(x, m, u, proj, rows, d);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" {
+
+int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const void *dev_u_bf16, int L, int B,
+                                int T, int d, int device, void *cuda_stream, float *dev_sw_out) {
+  if (!dev_x || !dev_m || !dev_u_bf16 || !dev_sw_out) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "x, m, u or sw_out is NULL");
+  int rc = check_shape(nullptr, B, T, d);
+  if (rc) return rc;
+  if (!aligned16(dev_x) || !aligned16(dev_m) || !aligned16(dev_u_bf16)) return fail(nullptr, SENTINEL_ERR_UNALIGNED, "x, m or u is not 16-byte aligned");
+  if (L != 4 && L != 8 && L != 16) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "L = %d: the number of directions must be 4, 8 or 16", L);
+  if ((size_t)L * d * sizeof(uint16_t) > 200u * 1024u) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "L*d = %d*%d directions do not fit in 200 KiB of shared memory", L, d);
+  if (T > kSwdMaxTokensPerSample) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "T = %d exceeds the %d tokens sorted per sample", T, kSwdMaxTokensPerSample);
+  int ndev = 0;
+  SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
+  if (device < 0 || device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist", device);
+  DeviceGuard guard(device);
+  SENTINEL_CUDA(nullptr, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int sms = 0;
+  SENTINEL_CUDA(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+
+  const long long rows = (long long)B * T;
+  const size_t list_floats = (size_t)2 * L * rows;        // L lists for x, L for m
+  float *scratch = nullptr;
+  keep_pool_warm(device);
+  SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, (3 * list_floats + (size_t)(B + 1) * L) * sizeof(float), s));
+  float *proj = scratch, *buf_a = proj + list_floats, *buf_b = buf_a + list_floats, *w1_sample = buf_b + list_floats;
+  float *w1_tensor = w1_sample + (size_t)B * L;
+
+  const uint16_t *x = static_cast<const uint16_t *>(dev_x), *u = static_cast<const uint16_t *>(dev_u_bf16);
+  cudaError_t e;
+  if (L == 4) e = launch_projection<4>(x, dev_m, u, proj, rows, d, sms, s);
+  else if (L == 8) e = launch_projection<8>(x, dev_m, u, proj, rows, d, sms, s);
+  else e = launch_projection<16>(x, dev_m, u, proj, rows, d, sms, s);
+  if (e == cudaSuccess) {
+    int npad = 1;
+    while (npad < T) npad <<= 1;
+    const size_t smem = (size_t)2 * npad * sizeof(float);
+    e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             2 * kSwdMaxTokensPerSample * (int)sizeof(float));
+    if (e == cudaSuccess) {
+      swd_sort_samples_kernel<<<B * L, kSwdSortThreads, smem, s>>>(proj, buf_a, w1_sample, B, T, L, rows);
+      e = cudaGetLastError();
+    }
+  }
+  float *cur = buf_a, *nxt = buf_b;
+  for (int run = 1; run < B && e == cudaSuccess; run *= 2) {     // merge the samples' sorted lists
+    const long long total = rows * 2 * L;
+    swd_merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(cur, nxt, rows, T, run, 2 * L);
+    e = cudaGetLastError();
+    float *t = cur; cur = nxt; nxt = t;
+  }
+  if (e == cudaSuccess) {
+    swd_tensor_w1_kernel<<<L, kSwdSortThreads, 0, s>>>(cur, w1_tensor, rows, L);
+    swd_finish_kernel<<<1, 128, 0, s>>>(w1_tensor, w1_sample, dev_sw_out, B, L);
+    e = cudaGetLastError();
+  }
+  cudaError_t fe = cudaFreeAsync(scratch, s);
+  SENTINEL_CUDA(nullptr, e);
+  SENTINEL_CUDA(nullptr, fe);
   return SENTINEL_OK;
 }
 

@@ -1,0 +1,179 @@
+// Sliced Wasserstein distance (Sec. 3.1) on the device.  x and m are clouds of tokens in R^d;
+// for each of L caller-supplied directions both clouds are projected (a skinny contraction,
+// [B*T, d] x [d, L], done while x and m stream through once), the projections of each sample
+// are sorted and matched (W1 of two empirical measures = mean |a_(i) - b_(i)|), the samples'
+// sorted lists are merged for the whole-tensor unit, and the L terms are averaged.
+#pragma once
+
+#include "sentinel_kernels.cuh"
+
+namespace sentinel {
+
+constexpr int kSwdThreads = 512;
+constexpr int kSwdSortThreads = 1024;
+constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are sorted in shared memory
+
+// ---------------------------------------------------------------------------------------------
+// projections: proj[(t*L + l)*rows + row] = sum_c v[row][c] * u[l][c], t = 0 for x, 1 for m.
+// A warp owns whole rows; the directions sit in shared memory as bf16 (they are given as bf16).
+// Traffic: x and m are read once, 6 B/element; per element L multiply-adds for each of x and m.
+template <int L>
+__global__ void __launch_bounds__(kSwdThreads)
+swd_project_kernel(const uint16_t *x, const float *m, const uint16_t *u, float *proj, long long rows, int d) {
+  extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
+  const int chunks = d >> 3;
+  for (int i = threadIdx.x; i < L * chunks; i += kSwdThreads)
+    s_u[i] = reinterpret_cast<const uint4 *>(u)[i];
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (kSwdThreads / 32) + (threadIdx.x >> 5);
+  const long long n_warps = (long long)gridDim.x * (kSwdThreads / 32);
+  for (long long row = warp; row < rows; row += n_warps) {
+    float ax[L], am[L];
+#pragma unroll
+    for (int l = 0; l < L; ++l) { ax[l] = 0.f; am[l] = 0.f; }
+    const size_t off = (size_t)row * d;
+    for (int c = lane; c < chunks; c += 32) {
+      const uint4 xv = ld_x128(x + off + (size_t)c * 8);
+      const F8 mv = ld_m256(m + off + (size_t)c * 8);
+      const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
+      float xf[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        xf[2 * j] = __uint_as_float(xw[j] << 16);
+        xf[2 * j + 1] = __uint_as_float(xw[j] & 0xFFFF0000u);
+      }
+#pragma unroll
+      for (int l = 0; l < L; ++l) {
+        const uint4 uv = s_u[l * chunks + c];
+        const unsigned uw[4] = {uv.x, uv.y, uv.z, uv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float u_lo = __uint_as_float(uw[j] << 16), u_hi = __uint_as_float(uw[j] & 0xFFFF0000u);
+          ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
+          ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
+          am[l] = fmaf(mv.v[2 * j], u_lo, am[l]);
+          am[l] = fmaf(mv.v[2 * j + 1], u_hi, am[l]);
+        }
+      }
+    }
+#pragma unroll
+    for (int l = 0; l < L; ++l) {
+      const float sx = warp_sum(ax[l]), sm = warp_sum(am[l]);
+      if (lane == l) {
+        proj[(size_t)l * rows + row] = sx;
+        proj[((size_t)L + l) * rows + row] = sm;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// per sample and direction: sort the T projections of x and of m, W1 = mean |a_(i) - b_(i)|
+__device__ __forceinline__ double block_sum_ordered(double v, double *s_red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) s_red[warp] = v;
+  __syncthreads();
+  double total = 0.;
+  if (threadIdx.x == 0)
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) total += s_red[w];
+  return total;                                   // valid in thread 0
+}
+
+__global__ void __launch_bounds__(kSwdSortThreads)
+swd_sort_samples_kernel(const float *proj, float *sorted, float *w1_sample, int B, int T, int L, long long rows) {
+  extern __shared__ float s_val[];                // [2][npad]
+  __shared__ double s_red[kSwdSortThreads / 32];
+  const int b = blockIdx.x / L, l = blockIdx.x - b * L;
+  int npad = 1;
+  while (npad < T) npad <<= 1;
+  float *sa = s_val, *sb = s_val + npad;
+  const float *px = proj + (size_t)l * rows + (size_t)b * T;
+  const float *pm = proj + ((size_t)L + l) * rows + (size_t)b * T;
+  for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) {
+    sa[i] = i < T ? px[i] : CUDART_INF_F;
+    sb[i] = i < T ? pm[i] : CUDART_INF_F;
+  }
+  __syncthreads();
+  for (int k2 = 2; k2 <= npad; k2 <<= 1) {        // bitonic sort of both lists, ascending
+    for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
+      for (int t = threadIdx.x; t < npad; t += kSwdSortThreads) {
+        const int partner = t ^ j2;
+        if (partner > t) {
+          const bool up = ((t & k2) == 0);
+          const float a0 = sa[t], a1 = sa[partner];
+          if ((a0 > a1) == up) { sa[t] = a1; sa[partner] = a0; }
+          const float b0 = sb[t], b1 = sb[partner];
+          if ((b0 > b1) == up) { sb[t] = b1; sb[partner] = b0; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  double acc = 0.;
+  float *ox = sorted + (size_t)l * rows + (size_t)b * T;
+  float *om = sorted + ((size_t)L + l) * rows + (size_t)b * T;
+  for (int i = threadIdx.x; i < T; i += kSwdSortThreads) {
+    acc += (double)fabsf(sa[i] - sb[i]);
+    ox[i] = sa[i];
+    om[i] = sb[i];
+  }
+  const double total = block_sum_ordered(acc, s_red);
+  if (threadIdx.x == 0) w1_sample[b * L + l] = (float)(total / (double)T);
+}
+
+// ---------------------------------------------------------------------------------------------
+// one round of merging: in every list (2L of them, each B sorted runs of T) neighbouring pairs
+// of runs of `run` samples become one sorted run; an element's place is its index in its own
+// run plus its rank in the partner run (left run first on ties)
+__global__ void swd_merge_kernel(const float *in, float *out, long long rows, int T, int run, int lists) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * lists) return;
+  const long long list = e / rows, i = e - list * rows;
+  const float *src = in + list * rows;
+  const long long run_len = (long long)run * T;
+  const long long r = i / run_len, pair_start = (r & ~1ll) * run_len;
+  const long long own_start = r * run_len;
+  const long long other_start = (r & 1) ? own_start - run_len : own_start + run_len;
+  const float v = src[i];
+  long long pos = i - own_start;
+  if (other_start < rows) {
+    long long lo = 0, hi = run_len;
+    if (other_start + hi > rows) hi = rows - other_start;
+    const float *other = src + other_start;
+    if (r & 1) {                                  // right run: after the left entries <= v
+      while (lo < hi) { const long long mid = (lo + hi) >> 1; if (other[mid] <= v) lo = mid + 1; else hi = mid; }
+    } else {                                      // left run: after the right entries < v
+      while (lo < hi) { const long long mid = (lo + hi) >> 1; if (other[mid] < v) lo = mid + 1; else hi = mid; }
+    }
+    pos += lo;
+  }
+  out[list * rows + pair_start + pos] = v;
+}
+
+// whole-tensor unit: W1 per direction from the fully merged lists, one CTA per direction
+__global__ void __launch_bounds__(kSwdSortThreads)
+swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int L) {
+  __shared__ double s_red[kSwdSortThreads / 32];
+  const int l = blockIdx.x;
+  const float *a = merged + (size_t)l * rows, *b = merged + ((size_t)L + l) * rows;
+  double acc = 0.;
+  for (long long i = threadIdx.x; i < rows; i += kSwdSortThreads) acc += (double)fabsf(a[i] - b[i]);
+  const double total = block_sum_ordered(acc, s_red);
+  if (threadIdx.x == 0) w1_tensor[l] = (float)(total / (double)rows);
+}
+
+// the means over the directions for every unit: out[0] = tensor, out[1+b] = sample b
+__global__ void swd_finish_kernel(const float *w1_tensor, const float *w1_sample, float *out, int B, int L) {
+  for (int r = threadIdx.x; r <= B; r += blockDim.x) {
+    const float *w = r ? w1_sample + (size_t)(r - 1) * L : w1_tensor;
+    double s = 0.;
+    for (int l = 0; l < L; ++l) s += (double)w[l];
+    out[r] = (float)(s / L);
+  }
+}
+
+}  // namespace sentinel

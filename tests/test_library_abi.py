@@ -38,7 +38,8 @@ def test_binding_mirrors_the_header(built):
     assert sorted(binding.EXPORTS) == declared_entry_points()
     binding.lib()
     for name in binding.EXPORTS:
-        if name in ("sentinel_default_config", "sentinel_distance", "sentinel_distance_noalloc"):
+        if name in ("sentinel_default_config", "sentinel_distance", "sentinel_distance_noalloc",
+                    "sentinel_sliced_wasserstein"):
             assert hasattr(binding, name)
         elif name not in ("sentinel_verifier_create", "sentinel_last_error"):
             assert hasattr(binding.Verifier, name), name
