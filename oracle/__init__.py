@@ -32,6 +32,7 @@ NMETRIC, NSTAT, NTHR = 3, 8, 6
 FLAG_L1, FLAG_L2Z, FLAG_SFR = 1 << 0, 1 << 1, 1 << 2
 FLAG_NONFINITE = 1 << 7
 FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
+FLAG_NATURAL_SHIFT = 1 << 20
 METRIC_BITS = FLAG_L1 | FLAG_L2Z | FLAG_SFR
 
 
@@ -55,6 +56,7 @@ class _Params(C.Structure):
         ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
         ("l", C.c_int), ("c", C.c_int), ("t_forgiveness", C.c_int),
         ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
+        ("R", C.c_int),
     ]
 
 
@@ -92,6 +94,10 @@ def lib():
         L.so_bf16_round.restype = C.c_uint16
         L.so_replace_if_flagged.argtypes = [C.c_void_p, u16p, C.c_int, C.c_int]
         L.so_replace_if_flagged.restype = C.c_int
+        L.so_step_replicas.argtypes = [C.c_void_p, C.POINTER(u16p), C.c_int, C.c_int, dp, C.POINTER(C.c_uint32)]
+        L.so_step_replicas.restype = C.c_int
+        L.so_worker_counters.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int)]
+        L.so_worker_counters.restype = None
         L.so_reset_worker.argtypes = [C.c_void_p]
         L.so_reset_worker.restype = None
         L.so_ema.argtypes = [C.c_void_p, C.c_int]
@@ -156,6 +162,7 @@ class Params:
     c: int = 5
     t_forgiveness: int = 100
     metric_mask: int = 7
+    R: int = 1
 
     def to_c(self) -> _Params:
         p = _Params()
@@ -167,6 +174,7 @@ class Params:
         p.l, p.c, p.t_forgiveness = self.l, self.c, self.t_forgiveness
         p.metric_mask = self.metric_mask
         p.B, p.T, p.d = self.B, self.T, self.d
+        p.R = self.R
         return p
 
 
@@ -237,6 +245,7 @@ class Verifier:
             raise ValueError("invalid oracle parameters")
         self.B, self.T, self.d = params.B, params.T, params.d
         self.rows = 1 + params.B
+        self.R = params.R
         self.N = params.B * params.T * params.d
 
     def close(self):
@@ -273,6 +282,24 @@ class Verifier:
         did = lib().so_replace_if_flagged(self._h, _u16ptr(xb), kind, fill)
         return xb.reshape(self.B, self.T, self.d), bool(did)
 
+    def step_replicas(self, xs_bits, kind: int, warmup: bool = False):
+        """One iteration with all R workers' tensors: (scores [R,1+B,3], flags [R,1+B], number of
+        submissions that entered the EMA)."""
+        assert len(xs_bits) == self.R
+        keep = [_bits(x).reshape(-1) for x in xs_bits]
+        assert all(k.size == self.N for k in keep)
+        ptrs = (C.POINTER(C.c_uint16) * self.R)(*[_u16ptr(k) for k in keep])
+        scores = np.empty((self.R, self.rows, NMETRIC))
+        flags = np.zeros((self.R, self.rows), dtype=np.uint32)
+        n = lib().so_step_replicas(self._h, ptrs, kind, int(warmup), _dptr(scores),
+                                   flags.ctypes.data_as(C.POINTER(C.c_uint32)))
+        return scores, flags, int(n)
+
+    def worker_counters(self, r: int) -> tuple[int, int, int]:
+        out = (C.c_int * 3)()
+        lib().so_worker_counters(self._h, r, out)
+        return out[0], out[1], out[2]
+
     def reset_worker(self):
         lib().so_reset_worker(self._h)
 
@@ -286,7 +313,7 @@ class Verifier:
         lib().so_set_ema(self._h, kind, _dptr(mm))
 
     def history(self, kind: int, level: int, metric: int) -> np.ndarray:
-        cap = self.params.l * (self.B if level else 1)
+        cap = self.params.l * self.R * (self.B if level else 1)
         out = np.empty(cap)
         n = lib().so_history(self._h, kind, level, metric, _dptr(out), cap)
         return out[:n].copy()

@@ -61,6 +61,7 @@ void so_default_params(so_params *p) {
   p->t_forgiveness = 100;        /* Sec. 3.1                                        */
   p->metric_mask = 7u;
   p->B = 1; p->T = 1; p->d = 8;
+  p->R = 1;
 }
 
 /* ------------------------------------------------------------------------------------ */
@@ -260,7 +261,7 @@ struct so_verifier {
   so_params p;
   size_t N, Ns;
   so_kind_state ks[2];
-  int violations, clean_streak, banned;
+  int violations[SO_MAX_WORKERS], clean_streak[SO_MAX_WORKERS], banned[SO_MAX_WORKERS];
 };
 
 static void window_push(so_window *w, double val) {
@@ -272,7 +273,7 @@ static void window_push(so_window *w, double val) {
 }
 
 so_verifier *so_create(const so_params *p) {
-  if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1) return NULL;
+  if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1 || p->R < 1 || p->R > SO_MAX_WORKERS) return NULL;
   so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
   v->p = *p;
   v->Ns = (size_t)p->T * (size_t)p->d;
@@ -284,7 +285,8 @@ so_verifier *so_create(const so_params *p) {
     for (int L = 0; L < 2; ++L)
       for (int i = 0; i < SO_NMETRIC; ++i) {
         so_window *w = &ks->hist[L][i];
-        w->cap = (L == 0) ? (size_t)p->l : (size_t)p->l * (size_t)p->B;
+        /* the window spans l iterations of all R workers (and of their B samples) */
+        w->cap = (size_t)p->l * (size_t)p->R * ((L == 0) ? 1u : (size_t)p->B);
         w->v = (double *)calloc(w->cap, sizeof(double));
         w->n = 0;
         ks->thr[L][i][3] = p->k0[kind];
@@ -334,6 +336,22 @@ static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
   double *m = v->ks[kind].m;
   const double beta = v->p.beta[kind];
   for (size_t e = 0; e < v->N; ++e) m[e] = beta * m[e] + (1.0 - beta) * so_bf16(x[e]);
+}
+
+/* Sec. 3.1, violation counter with forgiveness, kept per worker */
+static void count_violation(so_verifier *v, int r, int flagged, int severe) {
+  const so_params *p = &v->p;
+  if (flagged) {
+    v->violations[r] += 1;
+    v->clean_streak[r] = 0;
+    if (v->violations[r] >= p->c || severe) v->banned[r] = 1;
+  } else {
+    v->clean_streak[r] += 1;
+    if (v->clean_streak[r] >= p->t_forgiveness) {
+      v->violations[r] = (v->violations[r] > 0) ? v->violations[r] - 1 : 0;
+      v->clean_streak[r] = 0;
+    }
+  }
 }
 
 int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *scores) {
@@ -393,17 +411,7 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
   }
 
   /* 4. violation counter with forgiveness */
-  if (any_flag) {
-    v->violations += 1;
-    v->clean_streak = 0;
-    if (v->violations >= p->c || severe) v->banned = 1;
-  } else {
-    v->clean_streak += 1;
-    if (v->clean_streak >= p->t_forgiveness) {
-      v->violations = (v->violations > 0) ? v->violations - 1 : 0;
-      v->clean_streak = 0;
-    }
-  }
+  count_violation(v, 0, any_flag, severe);
 
   /* 5. clean units join the history; thresholds are refreshed for the next step */
   for (int r = 0; r < rows; ++r) {
@@ -421,10 +429,105 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
 
   if (commit) flags[0] |= SO_FLAG_COMMITTED;
   if (severe) flags[0] |= SO_FLAG_SEVERE;
-  if (v->banned) flags[0] |= SO_FLAG_BANNED;
+  if (v->banned[0]) flags[0] |= SO_FLAG_BANNED;
   if (no_thr) flags[0] |= SO_FLAG_NO_THRESHOLDS;
   free(gam); free(nf);
   return commit;
+}
+
+void so_worker_counters(const so_verifier *v, int r, int out[3]) {
+  out[0] = v->violations[r]; out[1] = v->clean_streak[r]; out[2] = v->banned[r];
+}
+
+int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int warmup,
+                     double *scores, uint32_t *flags) {
+  const so_params *p = &v->p;
+  const int R = p->R, rows = 1 + p->B;
+  so_kind_state *ks = &v->ks[kind];
+  double *gam = (double *)malloc((size_t)rows * SO_NMETRIC * sizeof(double));
+  int *nf = (int *)malloc((size_t)rows * sizeof(int));
+  int collected[SO_MAX_WORKERS], tainted[SO_MAX_WORKERS], severe_w[SO_MAX_WORKERS];
+  int no_thr = 0;
+  ks->steps += 1;
+
+  for (int r = 0; r < R; ++r) {
+    double *sc = scores + (size_t)r * rows * SO_NMETRIC;
+    uint32_t *fl = flags + (size_t)r * rows;
+    collected[r] = 0; tainted[r] = 0; severe_w[r] = 0;
+    for (int u = 0; u < rows; ++u) fl[u] = 0;
+    if (!warmup && v->banned[r]) {          /* banned workers are not collected any more */
+      for (int j = 0; j < rows * SO_NMETRIC; ++j) sc[j] = NAN;
+      continue;
+    }
+    collected[r] = 1;
+    all_units(v, xs[r], kind, gam, nf);     /* Gamma = Omega(x_t^(r), m_{t-1}) */
+    memcpy(sc, gam, (size_t)rows * SO_NMETRIC * sizeof(double));
+    int any_flag = 0;
+    for (int u = 0; u < rows; ++u) {
+      const int L = (u == 0) ? 0 : 1;
+      uint32_t f = 0;
+      if (nf[u]) {
+        f |= SO_FLAG_NONFINITE;
+      } else if (!warmup) {
+        for (int i = 0; i < SO_NMETRIC; ++i) {
+          if (!ks->has_thr[L][i]) { no_thr = 1; continue; }
+          if (!((p->metric_mask >> i) & 1u)) continue;
+          const double *t = ks->thr[L][i];
+          const double g = gam[(size_t)u * SO_NMETRIC + i];
+          if (g < t[4] || g > t[5]) f |= (1u << i);
+          if (u == 0 && fabs(g - t[1]) >= p->severe_mult * (t[5] - t[1])) severe_w[r] = 1;
+        }
+      }
+      fl[u] = f;
+      if (f) any_flag = 1;
+    }
+    tainted[r] = any_flag;
+    if (!warmup) count_violation(v, r, any_flag, severe_w[r]);
+    /* deviations of unflagged units join the pooled history (warm-up: of every unit, unless
+     * the submission is non-finite) */
+    if (!(warmup && any_flag))
+      for (int u = 0; u < rows; ++u) {
+        if (fl[u]) continue;
+        const int L = (u == 0) ? 0 : 1;
+        for (int i = 0; i < SO_NMETRIC; ++i)
+          window_push(&ks->hist[L][i], gam[(size_t)u * SO_NMETRIC + i]);
+      }
+  }
+  refresh_thresholds(v, kind);              /* once, after the worker loop */
+
+  /* more than half of the workers still in the pool flagged: a natural shift, not an attack */
+  int n_tainted = 0, n_banned = 0, natural = 0;
+  for (int r = 0; r < R; ++r) { n_tainted += tainted[r]; n_banned += v->banned[r]; }
+  if (!warmup && 2 * n_tainted > R - n_banned) {
+    natural = 1;
+    for (int r = 0; r < R; ++r)
+      if (!(flags[(size_t)r * rows] & SO_FLAG_NONFINITE)) tainted[r] = 0;
+  }
+
+  /* Eq. 1 with the mean over the clean submissions */
+  int n_clean = 0;
+  for (int r = 0; r < R; ++r) n_clean += (collected[r] && !tainted[r]);
+  if (n_clean > 0) {
+    double *m = ks->m;
+    const double beta = p->beta[kind];
+    for (size_t e = 0; e < v->N; ++e) {
+      double sum = 0.0;
+      for (int r = 0; r < R; ++r)
+        if (collected[r] && !tainted[r]) sum += so_bf16(xs[r][e]);
+      m[e] = beta * m[e] + (1.0 - beta) * (sum / (double)n_clean);
+    }
+  }
+  ks->last_flagged = (n_tainted > 0) && !natural;
+  for (int r = 0; r < R; ++r) {
+    uint32_t *fl = flags + (size_t)r * rows;
+    if (collected[r] && !tainted[r]) fl[0] |= SO_FLAG_COMMITTED;
+    if (severe_w[r]) fl[0] |= SO_FLAG_SEVERE;
+    if (!warmup && v->banned[r]) fl[0] |= SO_FLAG_BANNED;
+    if (no_thr && collected[r]) fl[0] |= SO_FLAG_NO_THRESHOLDS;
+    if (natural) fl[0] |= SO_FLAG_NATURAL_SHIFT;
+  }
+  free(gam); free(nf);
+  return n_clean;
 }
 
 int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill) {
@@ -434,7 +537,9 @@ int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill)
   return 1;
 }
 
-void so_reset_worker(so_verifier *v) { v->violations = 0; v->clean_streak = 0; v->banned = 0; }
+void so_reset_worker(so_verifier *v) {
+  for (int r = 0; r < SO_MAX_WORKERS; ++r) { v->violations[r] = 0; v->clean_streak[r] = 0; v->banned[r] = 0; }
+}
 
 /* ------------------------------------------------------------------------------------ */
 /* accessors                                                                             */
@@ -462,7 +567,7 @@ void so_last_stats(const so_verifier *v, int kind, double *stats) {
 }
 
 void so_counters(const so_verifier *v, int out[3]) {
-  out[0] = v->violations; out[1] = v->clean_streak; out[2] = v->banned;
+  out[0] = v->violations[0]; out[1] = v->clean_streak[0]; out[2] = v->banned[0];
 }
 
 long so_steps(const so_verifier *v, int kind) { return v->ks[kind].steps; }

@@ -32,6 +32,7 @@ extern "C" {
 enum { SO_ACT = 0, SO_GRAD = 1 };                 /* h (forward) or g (backward)           */
 enum { SO_L1 = 0, SO_L2Z = 1, SO_SFR = 2, SO_NMETRIC = 3 };
 enum { SO_NSTAT = 8 };                            /* mean_x var_x |x|_2 mean_m var_m cov |m|_2 rho */
+enum { SO_MAX_WORKERS = 16 };
 enum { SO_NTHR = 6 };                             /* q1 q2 q3 k tau_lower tau_upper        */
 
 /* report bits, one word per unit (row 0 = whole tensor, rows 1..B = samples) */
@@ -39,7 +40,8 @@ enum {
   SO_FLAG_L1 = 1u << 0, SO_FLAG_L2Z = 1u << 1, SO_FLAG_SFR = 1u << 2,
   SO_FLAG_NONFINITE = 1u << 7,
   SO_FLAG_COMMITTED = 1u << 16, SO_FLAG_SEVERE = 1u << 17,
-  SO_FLAG_BANNED = 1u << 18, SO_FLAG_NO_THRESHOLDS = 1u << 19
+  SO_FLAG_BANNED = 1u << 18, SO_FLAG_NO_THRESHOLDS = 1u << 19,
+  SO_FLAG_NATURAL_SHIFT = 1u << 20   /* more than half of the workers flagged: taint cleared */
 };
 
 /* Hyper-parameters; index 0 = activations, 1 = gradients (Tab. "verification_config"). */
@@ -59,6 +61,7 @@ typedef struct so_params {
   int    t_forgiveness;    /* clean steps before the counter decrements             */
   unsigned metric_mask;    /* which metrics may raise a flag (bit i = metric i)     */
   int    B, T, d;          /* submission shape                                      */
+  int    R;                /* workers (replicas) feeding this boundary, d_s >= 1    */
 } so_params;
 
 typedef struct so_verifier so_verifier;
@@ -117,6 +120,21 @@ uint16_t so_bf16_round(double v);
  * flagged, x (n = B*T*d bf16 bit patterns) becomes the reference m_{t-1} rounded to bf16
  * (fill = 0) or zeros (fill = 1); otherwise x is left alone.  Returns 1 if it replaced. */
 int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill);
+
+/* One iteration at this boundary with all R workers' submissions (Alg. 1 main loop, Alg. 2 /
+ * Alg. 3 with their worker loop; the EMA is Eq. 1 with the mean over the clean workers).
+ * xs[r] = worker r's tensor.  Every non-banned worker is scored against the same m_{t-1} and
+ * tested against the same bounds; its violation counter, forgiveness and ban are its own;
+ * clean units join the history pooled over workers (l*R entries at the tensor level, l*R*B at
+ * the sample level); Alg. 5 runs once after the loop; if more than half of the non-banned
+ * workers were flagged the taint set is cleared (natural distribution shift); the EMA moves
+ * with the mean of the submissions that are not tainted.  warmup != 0: the warm-up loop of
+ * Alg. 1 instead (no test, no counters, everything joins, mean over all workers).
+ * scores: [R][1+B][3]; flags: [R][1+B] (row 0 of each worker carries its status bits).
+ * Returns the number of submissions that entered the EMA. */
+int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int warmup,
+                     double *scores, uint32_t *flags);
+void so_worker_counters(const so_verifier *v, int r, int out[3]);   /* v_r, streak, banned */
 
 /* A new worker now feeds this boundary: clear its violation counter, streak and ban. */
 void so_reset_worker(so_verifier *v);

@@ -275,3 +275,120 @@ def test_gradient_replacement_follows_the_last_verdict(oracle_mod, small):
     a = synth.clean(small, 0, ACT, 16)
     out, did = v.replace_if_flagged(synth.bits(a), ACT)
     assert not did
+
+
+# ---------------------------------------------------------------- several workers per stage
+
+def _replica_inputs(w, R, step, kind=ACT):
+    return [synth.clean(w, r, kind, step) for r in range(R)]      # boundary index = worker index
+
+
+def test_replica_warmup_is_the_mean_over_workers(oracle_mod, small):
+    """Eq. 1: m_t = beta m_{t-1} + (1-beta) * (1/d_s) sum_r x^(r); the pooled window holds the
+    deviations of all workers (l*R entries per level-0 metric)."""
+    R = 3
+    v = oracle_mod.Verifier(oracle_mod.Params(B=small.B, T=small.T, d=small.d, R=R, l=4))
+    xs = _replica_inputs(small, R, 0)
+    scores, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT, warmup=True)
+    assert n == R and np.all(flags == oracle_mod.FLAG_COMMITTED * (np.arange(1 + small.B) == 0))
+    mean = sum(from_bits(synth.bits(x)) for x in xs) / R
+    assert v.ema(ACT) == pytest.approx(0.1 * mean, rel=1e-13, abs=1e-15)
+    for r in range(R):                       # every worker is scored against the same m_{t-1} = 0
+        assert scores[r, 0, 0] == pytest.approx(np.mean(np.abs(from_bits(synth.bits(xs[r])))), rel=1e-13)
+    assert v.history(ACT, 0, 0).size == R and v.history(ACT, 1, 0).size == R * small.B
+    for t in range(1, 7):
+        v.step_replicas([synth.bits(x) for x in _replica_inputs(small, R, t)], ACT, warmup=True)
+    assert v.history(ACT, 0, 0).size == 4 * R and v.history(ACT, 1, 0).size == 4 * R * small.B
+
+
+def test_one_worker_is_the_single_submission_path(oracle_mod, small):
+    """On clean traffic the worker loop with one worker is the single-submission call.  (On a
+    flagged step it is not: one flagged worker out of one is a majority, so the >50% rule of
+    Alg. 2 clears the taint, whereas the per-trainer form has no such rule.)"""
+    a = oracle_mod.Verifier(oracle_mod.Params(B=small.B, T=small.T, d=small.d))
+    b = oracle_mod.Verifier(oracle_mod.Params(B=small.B, T=small.T, d=small.d, R=1))
+    for t in range(12):
+        xb = synth.bits(synth.clean(small, 0, GRAD, t))
+        if t < 6:
+            sa, _ = a.update_reference(xb, GRAD)
+            sb_, fb, _ = b.step_replicas([xb], GRAD, warmup=True)
+        else:
+            sa, fa, _ = a.verify(xb, GRAD)
+            sb_, fb, _ = b.step_replicas([xb], GRAD)
+            assert np.array_equal(fa, fb[0])
+        assert np.array_equal(sa, sb_[0])
+        assert np.array_equal(a.ema(GRAD), b.ema(GRAD))
+        assert a.counters() == b.worker_counters(0)
+        ta, tb = a.thresholds(GRAD), b.thresholds(GRAD)
+        assert np.array_equal(ta[0], tb[0])
+
+
+def _warm_replicas(oracle_mod, w, R, n, **kw):
+    v = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, R=R, **kw))
+    for t in range(n):
+        v.step_replicas([synth.bits(x) for x in _replica_inputs(w, R, t)], ACT, warmup=True)
+    return v
+
+
+def test_tainted_worker_is_left_out_of_the_mean(oracle_mod, small):
+    R = 4
+    v = _warm_replicas(oracle_mod, small, R, 12)
+    xs = _replica_inputs(small, R, 12)
+    xs[2] = (xs[2].float() * 6).to(torch.bfloat16)
+    m0 = v.ema(ACT)
+    scores, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
+    assert n == 3
+    assert flags[2, 0] & 0xFFFF and not (flags[2, 0] & oracle_mod.FLAG_COMMITTED)
+    for r in (0, 1, 3):
+        assert flags[r, 0] == oracle_mod.FLAG_COMMITTED and not np.any(flags[r, 1:])
+    mean = sum(from_bits(synth.bits(xs[r])) for r in (0, 1, 3)) / 3
+    assert v.ema(ACT) == pytest.approx(0.9 * m0 + 0.1 * mean, rel=1e-12, abs=1e-15)
+    assert [v.worker_counters(r)[0] for r in range(R)] == [0, 0, 1, 0]
+
+
+def test_majority_flagged_is_a_natural_shift(oracle_mod, small):
+    """More than half of the workers flagged: the taint set is cleared, every submission enters
+    the EMA, but the violation counters have already moved (Alg. 2)."""
+    R = 4
+    v = _warm_replicas(oracle_mod, small, R, 12)
+    xs = _replica_inputs(small, R, 12)
+    for r in (0, 1, 3):
+        xs[r] = (xs[r].float() * 3).to(torch.bfloat16)
+    m0 = v.ema(ACT)
+    h0 = v.history(ACT, 0, 0).size
+    scores, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
+    assert n == 4 and np.all(flags[:, 0] & oracle_mod.FLAG_NATURAL_SHIFT)
+    assert np.all(flags[:, 0] & oracle_mod.FLAG_COMMITTED)
+    mean = sum(from_bits(synth.bits(x)) for x in xs) / 4
+    assert v.ema(ACT) == pytest.approx(0.9 * m0 + 0.1 * mean, rel=1e-12, abs=1e-15)
+    assert [v.worker_counters(r)[0] for r in range(R)] == [1, 1, 0, 1]
+    assert v.history(ACT, 0, 0).size == h0 + 1          # only the unflagged worker's deviation joined
+    # exactly half flagged is not a majority
+    v = _warm_replicas(oracle_mod, small, R, 12)
+    xs = _replica_inputs(small, R, 12)
+    for r in (0, 1):
+        xs[r] = (xs[r].float() * 3).to(torch.bfloat16)
+    _, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
+    assert n == 2 and not np.any(flags[:, 0] & oracle_mod.FLAG_NATURAL_SHIFT)
+
+
+def test_banned_worker_is_no_longer_collected(oracle_mod, small):
+    R = 3
+    v = _warm_replicas(oracle_mod, small, R, 12, c=2)
+    for t in range(12, 14):
+        xs = _replica_inputs(small, R, t)
+        xs[1] = (xs[1].float() * 6).to(torch.bfloat16)
+        _, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
+        assert n == 2
+    assert v.worker_counters(1) == (2, 0, 1) and flags[1, 0] & oracle_mod.FLAG_BANNED
+    xs = _replica_inputs(small, R, 14)
+    m0 = v.ema(ACT)
+    scores, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
+    assert n == 2 and np.all(np.isnan(scores[1])) and flags[1, 0] == oracle_mod.FLAG_BANNED
+    mean = sum(from_bits(synth.bits(xs[r])) for r in (0, 2)) / 2
+    assert v.ema(ACT) == pytest.approx(0.9 * m0 + 0.1 * mean, rel=1e-12, abs=1e-15)
+    # with one of three banned, one flagged worker of the remaining two is exactly half: no shift
+    xs = _replica_inputs(small, R, 15)
+    xs[0] = (xs[0].float() * 6).to(torch.bfloat16)
+    _, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
+    assert n == 1 and not (flags[0, 0] & oracle_mod.FLAG_NATURAL_SHIFT)
