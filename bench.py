@@ -236,6 +236,33 @@ def run_ours(args, rank, world, local_rank):
                "kernels": "swd_project_kernel + sort, merge, finish", "value_row0": float(sw[0])}
         del ref
 
+    # extra figure, outside the timed region: one iteration with R workers of the stage
+    # (R scoring launches at 6 B/element + the mean over the clean workers at 8 + 2R B/element)
+    replicas_fig = None
+    if nb == 1:
+        R = 4 if 100 * 4 * (w.B + 1) <= 4096 else 2
+        vr = binding.Verifier(w.B, w.T, w.d, device=local_rank, n_workers=R)
+        rs = torch.empty(R, 1 + w.B, 3, dtype=torch.float32, device=device)
+        rf = torch.zeros(R, 1 + w.B, dtype=torch.int32, device=device)
+        pick = lambda i: [xs[0][ACT][(i * R + r) % nd] for r in range(R)]
+        for i in range(4):
+            vr.sentinel_update_reference_replicas(pick(i), ACT, rs, rf, main)
+        vr.sentinel_verify_replicas(pick(4), ACT, rs, rf, main)
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        q0.record(main)
+        for i in range(6):
+            vr.sentinel_verify_replicas(pick(5 + i), ACT, rs, rf, main)
+        q1.record(main)
+        torch.cuda.synchronize()
+        qms = q0.elapsed_time(q1) / 6
+        per_el = 6 * R + 8 + 2 * R
+        replicas_fig = {"workers": R, "bytes_per_element": per_el, "ms_per_iteration": round(qms, 4),
+                        "achieved_gbs": round(per_el * N / (qms * 1e-3) / 1e9, 1),
+                        "submissions_per_s": round(R / (qms * 1e-3), 1),
+                        "kernels": "%d x stream_kernel (scores only) + ema_mean_kernel" % R}
+        vr.sentinel_destroy()
+
     # end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     hx = [{k: [xs[b][k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 2 if nb > 1 else 4))]
@@ -303,6 +330,8 @@ def run_ours(args, rank, world, local_rank):
         out["gradient_replacement"] = replace
     if swd is not None:
         out["sliced_wasserstein"] = swd
+    if replicas_fig is not None:
+        out["multi_worker_iteration"] = replicas_fig
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
     return out

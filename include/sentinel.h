@@ -44,7 +44,8 @@ extern "C" {
 #define SENTINEL_NUM_STATS 8      /* mean_x var_x |x|_2 mean_m var_m cov_xm |m|_2 rho */
 #define SENTINEL_NUM_THRESHOLDS 6 /* q1 q2 q3 k tau_lower tau_upper                   */
 #define SENTINEL_MAX_B 64         /* samples per tensor                               */
-#define SENTINEL_MAX_WINDOW 4096  /* window_steps * (B + 1) must not exceed this      */
+#define SENTINEL_MAX_WORKERS 16   /* workers (replicas of the stage) per handle       */
+#define SENTINEL_MAX_WINDOW 4096  /* window_steps * n_workers * (B + 1) must not exceed this */
 
 typedef enum sentinel_status {
   SENTINEL_OK = 0,
@@ -68,6 +69,7 @@ typedef enum sentinel_kind { SENTINEL_ACT = 0, SENTINEL_GRAD = 1 } sentinel_kind
 #define SENTINEL_FLAG_SEVERE (1u << 17)       /* row 0: deviation >= severe_mult * allowed   */
 #define SENTINEL_FLAG_BANNED (1u << 18)       /* row 0: sticky until sentinel_reset_worker   */
 #define SENTINEL_FLAG_NO_THRESHOLDS (1u << 19) /* row 0: some history was still empty         */
+#define SENTINEL_FLAG_NATURAL_SHIFT (1u << 20) /* row 0: more than half of the workers flagged */
 
 /* Hyper-parameters.  Arrays are indexed by kind.  Defaults: table "verification_config",
  * column "8x16 Mesh, 0.6B"; c and T_forgiveness from Sec. 3.1; the window from Sec. 5. */
@@ -88,6 +90,7 @@ typedef struct sentinel_config {
   unsigned metric_mask;    /* bit i set: metric i may raise a flag             7           */
   int    B, T, d;          /* shape of every submission; d % 8 == 0, B <= SENTINEL_MAX_B   */
   int    device;           /* CUDA device ordinal                                           */
+  int    n_workers;        /* workers d_s feeding this boundary (multi-worker calls)   1    */
 } sentinel_config;
 
 typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundary */
@@ -183,14 +186,42 @@ int sentinel_get_stats(sentinel_verifier *h, sentinel_kind kind, float *dev_stat
 int sentinel_get_thresholds(sentinel_verifier *h, sentinel_kind kind, double *host_out,
                             int *host_valid, void *cuda_stream);
 
-/* host_out int64 [6]: violations v, clean streak, banned, steps(ACT), steps(GRAD), the error
- * word written by device code (0 = none).  Waits for the stream. */
+/* host_out int64 [6]: violations v, clean streak, banned (of worker 0), steps(ACT),
+ * steps(GRAD), the error word written by device code (0 = none).  Waits for the stream. */
 int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_stream);
+
+/* host_out int64 [3]: violations, clean streak, banned of worker `worker`.  Waits. */
+int sentinel_get_worker_counters(sentinel_verifier *h, int worker, long long *host_out, void *cuda_stream);
 
 /* Per-token partial sums of the pass, written by every later call while registered:
  * dev_buf fp32 [B,T,4] = sum_c x, sum_c x^2, sum_c |x-m|, count of sign mismatches over the
  * token's d channels.  NULL unregisters.  The buffer stays the caller's. */
 int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf);
+
+/* One iteration with the submissions of all n_workers workers of the stage (the worker loop
+ * of Alg. 2 / Alg. 3 and the reference update of Alg. 1 / Eq. 1).  host_dev_xs: a HOST array of
+ * n_workers device pointers, each bf16 [B,T,d], 16-byte aligned (read by the call itself; the
+ * tensors are read on the stream).  Every worker that is not banned is scored against the same
+ * m_{t-1} and tested against the same bounds; violation counter, forgiveness and ban are kept
+ * per worker; unflagged units join histories pooled over the workers (window_steps*n_workers
+ * entries for the whole-tensor unit, times B for samples); the bounds are refreshed once per
+ * iteration; if more than half of the workers still in the pool were flagged, the taint set
+ * is cleared (natural distribution shift, SENTINEL_FLAG_NATURAL_SHIFT) and the counters stay
+ * as they moved; the reference then moves with the mean of the untainted submissions (each
+ * tensor is read once for its scores and once more for the mean).  A banned worker is not
+ * read: its scores are NaN and its row 0 reports SENTINEL_FLAG_BANNED.
+ * dev_scores_out fp32 [n_workers][1+B][3]; dev_flags_out u32 [n_workers][1+B]; row 0 of worker
+ * r carries COMMITTED iff its tensor entered the mean. */
+int sentinel_verify_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind,
+                             int B, int T, int d, void *cuda_stream, float *dev_scores_out,
+                             unsigned *dev_flags_out);
+
+/* The warm-up loop of Alg. 1 with all workers: no test, no counters, every unit of every worker
+ * joins the history, the reference moves with the mean over all workers.  Outputs as above
+ * (dev_flags_out may be NULL). */
+int sentinel_update_reference_replicas(sentinel_verifier *h, const void *const *host_dev_xs,
+                                       sentinel_kind kind, int B, int T, int d, void *cuda_stream,
+                                       float *dev_scores_out, unsigned *dev_flags_out);
 
 /* Gradient replacement (Alg. 4) for the submission this handle sees.  If the last
  * sentinel_verify of `kind` raised a flag (the step was not committed), dev_x_inout -- the
@@ -203,15 +234,16 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
                                 int T, int d, int fill, void *cuda_stream,
                                 unsigned *dev_replaced_out);
 
-/* A new worker now feeds this boundary: clears the violation counter, the clean streak and
- * the ban (the paper keeps these per worker).  Enqueued on cuda_stream. */
-int sentinel_reset_worker(sentinel_verifier *h, void *cuda_stream);
+/* Worker slot `worker` (0 for single-submission use) is now fed by a new worker: clears its
+ * violation counter, clean streak and ban.  Enqueued on cuda_stream. */
+int sentinel_reset_worker(sentinel_verifier *h, int worker, void *cuda_stream);
 
 /* Checkpointing.  The state is one self-describing blob: a 64-byte header
- * {u64 magic, u32 version, i32 B, T, d, window_steps, violations, clean_streak, banned},
- * then per kind {i64 steps; i32 count[2]; i32 valid[2][3]; f64 thr[2][3][6];
- * f64 history[level 0: 3][window_steps], [level 1: 3][window_steps*B] (oldest first,
- * zero-padded); f32 m[B*T*d]}.  Export and import wait for the stream. */
+ * {u64 magic, u32 version = 2, i32 B, T, d, window_steps, n_workers}, then
+ * i32 violations[16], clean_streak[16], banned[16], then per kind {i64 steps; i32 count[2];
+ * i32 valid[2][3]; f64 thr[2][3][6]; f64 history[level 0: 3][window_steps*n_workers],
+ * [level 1: 3][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d]}.
+ * Export and import wait for the stream. */
 size_t sentinel_state_bytes(const sentinel_verifier *h);
 int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *cuda_stream);
 int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, void *cuda_stream);

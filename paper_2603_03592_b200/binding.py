@@ -24,10 +24,13 @@ ERR_STATE_SIZE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -7
 FLAG_L1, FLAG_L2Z, FLAG_SFR = 1 << 0, 1 << 1, 1 << 2
 FLAG_NONFINITE = 1 << 7
 FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
+FLAG_NATURAL_SHIFT = 1 << 20
+MAX_WORKERS = 16
 
 EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
+    "sentinel_verify_replicas", "sentinel_update_reference_replicas", "sentinel_get_worker_counters",
     "sentinel_distance_noalloc", "sentinel_replace_if_flagged", "sentinel_sliced_wasserstein",
     "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
     "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
@@ -43,7 +46,7 @@ class sentinel_config(C.Structure):
         ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
         ("window_steps", C.c_int), ("ban_violations", C.c_int), ("forgiveness_steps", C.c_int),
         ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
-        ("device", C.c_int),
+        ("device", C.c_int), ("n_workers", C.c_int),
     ]
 
 
@@ -84,7 +87,10 @@ def lib():
         L.sentinel_get_thresholds.argtypes = [vp, ip, vp, vp, vp]
         L.sentinel_get_counters.argtypes = [vp, vp, vp]
         L.sentinel_set_token_stats_buffer.argtypes = [vp, vp]
-        L.sentinel_reset_worker.argtypes = [vp, vp]
+        L.sentinel_reset_worker.argtypes = [vp, ip, vp]
+        L.sentinel_verify_replicas.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_update_reference_replicas.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_get_worker_counters.argtypes = [vp, ip, vp, vp]
         L.sentinel_state_bytes.argtypes = [vp]
         L.sentinel_state_bytes.restype = C.c_size_t
         L.sentinel_export_state.argtypes = [vp, vp, C.c_size_t, vp]
@@ -163,6 +169,7 @@ class Verifier:
     def __init__(self, B: int, T: int, d: int, device: int = 0, **overrides):
         self.cfg = sentinel_default_config(B=B, T=T, d=d, device=device, **overrides)
         self.B, self.T, self.d = B, T, d
+        self.R = self.cfg.n_workers
         self.rows = 1 + B
         self.device = torch.device("cuda", device)
         h = C.c_void_p()
@@ -188,6 +195,38 @@ class Verifier:
         _check(lib().sentinel_verify_host(self._h, _ptr(x_host), kind, B, T, d,
                                           _stream_ptr(stream), _ptr(scores_host),
                                           _ptr(flags_host)), self._h)
+
+    def _worker_pointers(self, xs):
+        assert len(xs) == self.R, "one tensor per worker"
+        return (C.c_void_p * self.R)(*[x.data_ptr() for x in xs])
+
+    def sentinel_verify_replicas(self, xs, kind: int, scores_out: torch.Tensor,
+                                 flags_out: torch.Tensor, stream=None) -> None:
+        """One iteration with all workers' tensors (worker loop of Alg. 2/3, mean over the clean)."""
+        B, T, d = xs[0].shape
+        _check(lib().sentinel_verify_replicas(self._h, self._worker_pointers(xs), kind, B, T, d,
+                                              _stream_ptr(stream), _ptr(scores_out), _ptr(flags_out)), self._h)
+
+    def sentinel_update_reference_replicas(self, xs, kind: int, scores_out: torch.Tensor,
+                                           flags_out: torch.Tensor | None = None, stream=None) -> None:
+        B, T, d = xs[0].shape
+        _check(lib().sentinel_update_reference_replicas(self._h, self._worker_pointers(xs), kind, B, T, d,
+                                                        _stream_ptr(stream), _ptr(scores_out),
+                                                        _ptr(flags_out)), self._h)
+
+    def step_replicas(self, xs, kind: int, warmup: bool = False, stream=None):
+        scores = torch.empty(self.R, self.rows, NUM_METRICS, dtype=torch.float32, device=xs[0].device)
+        flags = torch.zeros(self.R, self.rows, dtype=torch.int32, device=xs[0].device)
+        if warmup:
+            self.sentinel_update_reference_replicas(xs, kind, scores, flags, stream)
+        else:
+            self.sentinel_verify_replicas(xs, kind, scores, flags, stream)
+        return scores, flags
+
+    def sentinel_get_worker_counters(self, worker: int, stream=None) -> tuple:
+        out = (C.c_longlong * 3)()
+        _check(lib().sentinel_get_worker_counters(self._h, worker, out, _stream_ptr(stream)), self._h)
+        return out[0], out[1], out[2]
 
     def sentinel_replace_if_flagged(self, x_inout: torch.Tensor, kind: int, fill: int = 0,
                                     replaced_out: torch.Tensor | None = None, stream=None) -> None:
@@ -233,8 +272,8 @@ class Verifier:
         self._token_buf = buf          # keep the tensor alive while registered
         _check(lib().sentinel_set_token_stats_buffer(self._h, _ptr(buf)), self._h)
 
-    def sentinel_reset_worker(self, stream=None) -> None:
-        _check(lib().sentinel_reset_worker(self._h, _stream_ptr(stream)), self._h)
+    def sentinel_reset_worker(self, worker: int = 0, stream=None) -> None:
+        _check(lib().sentinel_reset_worker(self._h, worker, _stream_ptr(stream)), self._h)
 
     # -- checkpointing ------------------------------------------------------------------------
     def sentinel_state_bytes(self) -> int:

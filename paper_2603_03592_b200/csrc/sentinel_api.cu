@@ -20,13 +20,17 @@ namespace {
 thread_local std::string g_error;   // failures of calls that have no handle
 
 constexpr unsigned long long kMagic = 0x4c454e49544e4553ull;  // "SENTINEL", little endian
-constexpr unsigned kVersion = 1;
+constexpr unsigned kVersion = 2;
 constexpr size_t kHeaderBytes = 64;
 
 struct BlobHeader {
   unsigned long long magic;
   unsigned version;
-  int B, T, d, window_steps, violations, clean_streak, banned;
+  int B, T, d, window_steps, n_workers;
+};
+
+struct BlobWorkers {      // follows the header
+  int violations[kMaxWorkers], clean_streak[kMaxWorkers], banned[kMaxWorkers];
 };
 static_assert(sizeof(BlobHeader) <= kHeaderBytes, "header must fit its slot");
 
@@ -44,6 +48,7 @@ struct sentinel_verifier {
   sentinel_config cfg;
   size_t N = 0, Ns = 0;
   int cap0 = 0, cap1 = 0;
+  int R = 1, units0 = 1, units1 = 1; // workers; entries one iteration can append per level
   int G = 1;                        // streaming CTAs; launches use G + 1
   size_t refresh_smem = 0;          // dynamic shared memory of a launch that may refresh thresholds
   float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
@@ -88,7 +93,7 @@ size_t hist_doubles(const sentinel_verifier *h) {
 
 // doubles of the rings on the device: each ring has one step's worth of slots more than its window
 size_t ring_doubles(const sentinel_verifier *h) {
-  return (size_t)kNumMetrics * ((size_t)ring_size(h->cap0, 1) + (size_t)ring_size(h->cap1, h->cfg.B));
+  return (size_t)kNumMetrics * ((size_t)ring_size(h->cap0, h->units0) + (size_t)ring_size(h->cap1, h->units1));
 }
 
 size_t kind_blob_bytes(const sentinel_verifier *h) {
@@ -189,6 +194,8 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.beta = (float)h->cfg.beta[kind];
   a.one_minus_beta = (float)(1.0 - h->cfg.beta[kind]);
   a.cap0 = h->cap0; a.cap1 = h->cap1;
+  a.units0 = h->units0; a.units1 = h->units1;
+  a.R = h->R; a.worker = 0;
   a.a5 = alg5_of(h->cfg, kind);
   a.severe_mult = h->cfg.severe_mult;
   a.ban_violations = h->cfg.ban_violations;
@@ -217,7 +224,8 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) 
 
 int run_refresh(sentinel_verifier *h, cudaStream_t s) {
   refresh_kernel<<<1, kThreads, h->refresh_smem, s>>>(h->hs, h->hist[0], h->hist[1], h->sorted[0], h->sorted[1],
-                                                      h->cap0, h->cap1, h->cfg.B, alg5_of(h->cfg, 0), alg5_of(h->cfg, 1));
+                                                      h->cap0, h->cap1, h->units0, h->units1, alg5_of(h->cfg, 0),
+                                                      alg5_of(h->cfg, 1));
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
 }
@@ -268,6 +276,7 @@ int sentinel_default_config(sentinel_config *cfg) {
   cfg->ban_violations = 5;
   cfg->forgiveness_steps = 100;
   cfg->metric_mask = 7u;
+  cfg->n_workers = 1;
   return SENTINEL_OK;
 }
 
@@ -284,8 +293,11 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   }
   if (cfg->window_steps < 1 || cfg->ban_violations < 1 || cfg->forgiveness_steps < 1 || !(cfg->severe_mult > 0.0) || !(cfg->shrink_ratio >= 0.0))
     return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "window_steps, ban_violations, forgiveness_steps, severe_mult must be positive");
-  if ((long long)cfg->window_steps * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
-    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d", (long long)cfg->window_steps * (cfg->B + 1), SENTINEL_MAX_WINDOW);
+  if (cfg->n_workers < 1 || cfg->n_workers > SENTINEL_MAX_WORKERS)
+    return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "n_workers = %d is outside 1..%d", cfg->n_workers, SENTINEL_MAX_WORKERS);
+  if ((long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*n_workers*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d",
+                (long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1), SENTINEL_MAX_WINDOW);
   int ndev = 0;
   SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
   if (cfg->device < 0 || cfg->device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist (%d devices)", cfg->device, ndev);
@@ -298,12 +310,19 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->cfg = *cfg;
   h->Ns = (size_t)cfg->T * cfg->d;
   h->N = h->Ns * cfg->B;
-  h->cap0 = cfg->window_steps;
-  h->cap1 = cfg->window_steps * cfg->B;
-  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1, cfg->B) * sizeof(double);
-  {   // the windows' working copies may exceed the 48 KiB a kernel gets without asking;
-      // window_steps*(B+1) <= SENTINEL_MAX_WINDOW bounds them
-    const int most = (int)((size_t)kNumMetrics * (2 * (size_t)SENTINEL_MAX_WINDOW + 4 * (SENTINEL_MAX_B + 1)) * sizeof(double));
+  h->R = cfg->n_workers;
+  h->units0 = h->R;                       // the window spans window_steps iterations of all workers
+  h->units1 = h->R * cfg->B;
+  h->cap0 = cfg->window_steps * h->units0;
+  h->cap1 = cfg->window_steps * h->units1;
+  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1, h->units0, h->units1) * sizeof(double);
+  if (h->refresh_smem > 200u * 1024u) {
+    const size_t need = h->refresh_smem;
+    delete h;
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "the windows' working copies need %zu bytes of shared memory, 204800 are available", need);
+  }
+  {   // the windows' working copies may exceed the 48 KiB a kernel gets without asking
+    const int most = 200 * 1024;
     cudaError_t ae = cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
@@ -428,6 +447,62 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   SENTINEL_CUDA(nullptr, le);
   SENTINEL_CUDA(nullptr, fe);
   return SENTINEL_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, int B, int T, int d, void *cuda_stream,
+                  float *scores, unsigned *flags, bool warmup) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!xs) return fail(h, SENTINEL_ERR_INVALID_ARG, "the array of tensors is NULL");
+  for (int r = 0; r < h->R; ++r) {
+    int rc = check_call(h, xs[r], kind, B, T, d);
+    if (rc) return rc;
+  }
+  if (!scores || (!warmup && !flags)) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t rows = 1 + (size_t)B;
+  if (warmup && flags) SENTINEL_CUDA(h, cudaMemsetAsync(flags, 0, h->R * rows * sizeof(unsigned), s));
+  WorkerPointers wp;
+  memset(&wp, 0, sizeof wp);
+  for (int r = 0; r < h->R; ++r) {                 // every worker against the same m_{t-1}
+    StreamArgs a = make_args(h, xs[r], kind, warmup ? kModeReplicaWarmup : kModeReplicaVerify,
+                             scores + r * rows * kNumMetrics, warmup ? nullptr : flags + r * rows);
+    a.worker = r;
+    int rc = launch(h, a, h->G + 1, s);
+    if (rc) return rc;
+    wp.x[r] = static_cast<const uint16_t *>(xs[r]);
+  }
+  int sms = 0;
+  SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
+  const long long n_chunks = (long long)(h->N / 8);
+  long long grid = (long long)sms * 8;
+  const long long need = (n_chunks + kReplaceThreads - 1) / kReplaceThreads;
+  if (grid > need) grid = need;
+  ema_mean_kernel<<<(unsigned)grid, kReplaceThreads, 0, s>>>(
+      h->hs, kind, wp, h->ema[kind][0], h->ema[kind][1], n_chunks, h->R, (int)rows, (float)h->cfg.beta[kind],
+      (float)(1.0 - h->cfg.beta[kind]), warmup ? 1 : 0, flags);
+  SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sentinel_verify_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind, int B,
+                             int T, int d, void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out) {
+  return step_replicas(h, host_dev_xs, kind, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, false);
+}
+
+int sentinel_update_reference_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind,
+                                       int B, int T, int d, void *cuda_stream, float *dev_scores_out,
+                                       unsigned *dev_flags_out) {
+  return step_replicas(h, host_dev_xs, kind, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, true);
 }
 
 int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentinel_kind kind, int B, int T,
@@ -572,9 +647,9 @@ int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_
   HandleState snap;
   SENTINEL_CUDA(h, cudaMemcpyAsync(&snap, h->hs, sizeof snap, cudaMemcpyDeviceToHost, s));
   SENTINEL_CUDA(h, cudaStreamSynchronize(s));
-  host_out[0] = snap.violations;
-  host_out[1] = snap.clean_streak;
-  host_out[2] = snap.banned;
+  host_out[0] = snap.violations[0];
+  host_out[1] = snap.clean_streak[0];
+  host_out[2] = snap.banned[0];
   host_out[3] = snap.kind[0].steps;
   host_out[4] = snap.kind[1].steps;
   host_out[5] = snap.error;
@@ -594,18 +669,35 @@ int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf) {
   return SENTINEL_OK;
 }
 
-int sentinel_reset_worker(sentinel_verifier *h, void *cuda_stream) {
+int sentinel_get_worker_counters(sentinel_verifier *h, int worker, long long *host_out, void *cuda_stream) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "host_out is NULL");
+  if (worker < 0 || worker >= h->R) return fail(h, SENTINEL_ERR_INVALID_ARG, "worker %d is outside 0..%d", worker, h->R - 1);
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
-  reset_worker_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>(h->hs);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  HandleState snap;
+  SENTINEL_CUDA(h, cudaMemcpyAsync(&snap, h->hs, sizeof snap, cudaMemcpyDeviceToHost, s));
+  SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+  host_out[0] = snap.violations[worker];
+  host_out[1] = snap.clean_streak[worker];
+  host_out[2] = snap.banned[worker];
+  return SENTINEL_OK;
+}
+
+int sentinel_reset_worker(sentinel_verifier *h, int worker, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (worker < 0 || worker >= h->R) return fail(h, SENTINEL_ERR_INVALID_ARG, "worker %d is outside 0..%d", worker, h->R - 1);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  reset_worker_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>(h->hs, worker);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
 }
 
 size_t sentinel_state_bytes(const sentinel_verifier *h) {
   if (!h) return 0;
-  return kHeaderBytes + 2 * kind_blob_bytes(h);
+  return kHeaderBytes + sizeof(BlobWorkers) + 2 * kind_blob_bytes(h);
 }
 
 int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *cuda_stream) {
@@ -623,10 +715,15 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
 
   unsigned char *out = static_cast<unsigned char *>(host_buf);
   memset(out, 0, kHeaderBytes);
-  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps,
-                   snap.violations, snap.clean_streak, snap.banned};
+  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R};
   memcpy(out, &hd, sizeof hd);
   out += kHeaderBytes;
+  BlobWorkers bw;
+  memcpy(bw.violations, snap.violations, sizeof bw.violations);
+  memcpy(bw.clean_streak, snap.clean_streak, sizeof bw.clean_streak);
+  memcpy(bw.banned, snap.banned, sizeof bw.banned);
+  memcpy(out, &bw, sizeof bw);
+  out += sizeof bw;
   std::vector<double> ring(ring_doubles(h));
   for (int k = 0; k < 2; ++k) {
     const KindState &ks = snap.kind[k];
@@ -642,9 +739,9 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
     SENTINEL_CUDA(h, cudaStreamSynchronize(s));
     double *dst = reinterpret_cast<double *>(out);
     for (int L = 0; L < 2; ++L) {                   // unroll each ring, oldest entry first
-      const int cap = L ? h->cap1 : h->cap0, size = ring_size(cap, L ? h->cfg.B : 1);
+      const int cap = L ? h->cap1 : h->cap0, size = ring_size(cap, L ? h->units1 : h->units0);
       for (int i = 0; i < kNumMetrics; ++i) {
-        const size_t src_off = ring_offset(L, i, h->cap0, h->cap1, h->cfg.B);
+        const size_t src_off = ring_offset(L, i, h->cap0, h->cap1, h->units0, h->units1);
         for (int j = 0; j < cap; ++j)
           dst[j] = (j < ks.hist_count[L]) ? ring[src_off + (size_t)((ks.hist_head[L] + j) % size)] : 0.0;
         dst += cap;
@@ -667,10 +764,10 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
   memcpy(&hd, in, sizeof hd);
   if (hd.magic != kMagic || hd.version != kVersion)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "not a sentinel state blob of version %u", kVersion);
-  if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps)
-    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d", hd.B, hd.T, hd.d, hd.window_steps);
+  if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps || hd.n_workers != h->R)
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d, %d workers", hd.B, hd.T, hd.d, hd.window_steps, hd.n_workers);
   // validate both kinds before touching the device
-  const unsigned char *p = in + kHeaderBytes;
+  const unsigned char *p = in + kHeaderBytes + sizeof(BlobWorkers);
   for (int k = 0; k < 2; ++k) {
     BlobKindHead kh;
     memcpy(&kh, p, sizeof kh);
@@ -684,10 +781,12 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
 
   HandleState st;
   memset(&st, 0, sizeof st);
-  st.violations = hd.violations;
-  st.clean_streak = hd.clean_streak;
-  st.banned = hd.banned;
-  p = in + kHeaderBytes;
+  BlobWorkers bw;
+  memcpy(&bw, in + kHeaderBytes, sizeof bw);
+  memcpy(st.violations, bw.violations, sizeof bw.violations);
+  memcpy(st.clean_streak, bw.clean_streak, sizeof bw.clean_streak);
+  memcpy(st.banned, bw.banned, sizeof bw.banned);
+  p = in + kHeaderBytes + sizeof(BlobWorkers);
   for (int k = 0; k < 2; ++k) {
     BlobKindHead kh;
     memcpy(&kh, p, sizeof kh);
@@ -708,7 +807,7 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
       for (int L = 0; L < 2; ++L) {
         const int cap = L ? h->cap1 : h->cap0;
         for (int i = 0; i < kNumMetrics; ++i) {
-          double *r = rings.data() + ring_offset(L, i, h->cap0, h->cap1, h->cfg.B);
+          double *r = rings.data() + ring_offset(L, i, h->cap0, h->cap1, h->units0, h->units1);
           double *a = asc.data() + sorted_offset(L, i, h->cap0, h->cap1);
           std::copy(src, src + kh.count[L], r);
           std::copy(src, src + kh.count[L], a);

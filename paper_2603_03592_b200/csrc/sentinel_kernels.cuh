@@ -26,7 +26,12 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kSlotWords = 8;             // 64-bit words per partial slot
 constexpr int kUnroll = 2;                // 8-element chunks per lane per loop trip
 
-enum Mode : int { kModeVerify = 0, kModeWarmup = 1, kModeDistance = 2 };
+constexpr int kMaxWorkers = 16;           // workers (replicas of a stage) one handle can follow
+
+// single submission: verify / warm-up / stateless distance; one worker of a multi-worker
+// iteration: verify / warm-up (no EMA write: the mean over the clean workers follows)
+enum Mode : int { kModeVerify = 0, kModeWarmup = 1, kModeDistance = 2,
+                  kModeReplicaVerify = 3, kModeReplicaWarmup = 4 };
 
 // flag bits (mirrors the public header)
 constexpr unsigned kFlagNonfinite = 1u << 7;
@@ -34,6 +39,7 @@ constexpr unsigned kFlagCommitted = 1u << 16;
 constexpr unsigned kFlagSevere = 1u << 17;
 constexpr unsigned kFlagBanned = 1u << 18;
 constexpr unsigned kFlagNoThresholds = 1u << 19;
+constexpr unsigned kFlagNaturalShift = 1u << 20;
 
 // word 7 of a partial slot: bits 0-2 flags, bits 8-15 tag (1 + sample index, 0 = slot unused),
 // bits 16-31 the sample's first x (bf16 bits), bits 32-63 the sample's first m (fp32 bits)
@@ -56,15 +62,18 @@ struct KindState {
   int last_joined[2];     // entries the last step appended / pushed out, per level: what the
   int last_evicted[2];    //   pending refresh has to merge into the sorted copy
   int last_flagged;       // the last verified step of this kind raised a flag (no commit)
-  int pad;
+  unsigned step_collected;  // multi-worker iteration in progress: workers scored so far,
+  unsigned step_tainted;    //   workers that raised a flag,
+  unsigned step_nonfinite;  //   workers whose tensor held a NaN or an infinity
   int has_thr[2][kNumMetrics];
   double thr[2][kNumMetrics][kNumThr];   // q1 q2 q3 k tau_lower tau_upper
 };
 
 struct HandleState {
-  int violations, clean_streak, banned, error;
+  int error;
   unsigned ticket;
-  int pad[3];
+  int pad[2];
+  int violations[kMaxWorkers], clean_streak[kMaxWorkers], banned[kMaxWorkers];   // per worker
   KindState kind[2];
 };
 
@@ -87,6 +96,8 @@ struct StreamArgs {
   int mode, kind;
   float beta, one_minus_beta;
   int cap0, cap1;
+  int units0, units1;              // entries one iteration can append per level: R and R*B
+  int R, worker;                   // workers of the stage; which one this launch scores
   Alg5Params a5;
   double severe_mult;
   int ban_violations, forgiveness_steps;
@@ -362,9 +373,9 @@ __device__ __forceinline__ double percentile_sorted(const double *s, int n, doub
 // both what joined and what left.  Next to each ring the same window is kept in ascending
 // order; a refresh merges the few changes into it instead of sorting the window again.
 __host__ __device__ inline int ring_size(int cap, int units) { return cap + units; }
-__host__ __device__ inline size_t ring_offset(int L, int i, int cap0, int cap1, int B) {
-  return L ? (size_t)kNumMetrics * ring_size(cap0, 1) + (size_t)i * ring_size(cap1, B)
-           : (size_t)i * ring_size(cap0, 1);
+__host__ __device__ inline size_t ring_offset(int L, int i, int cap0, int cap1, int units0, int units1) {
+  return L ? (size_t)kNumMetrics * ring_size(cap0, units0) + (size_t)i * ring_size(cap1, units1)
+           : (size_t)i * ring_size(cap0, units0);
 }
 __host__ __device__ inline size_t sorted_offset(int L, int i, int cap0, int cap1) {
   return L ? (size_t)kNumMetrics * cap0 + (size_t)i * cap1 : (size_t)i * cap0;
@@ -384,8 +395,8 @@ __device__ __forceinline__ void group_barrier(int group) {   // named barrier 1 
 __host__ __device__ inline size_t window_smem_doubles(int cap, int units) {
   return 2 * (size_t)cap + 4 * (size_t)units;
 }
-__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1, int B) {
-  return (size_t)kNumMetrics * (window_smem_doubles(cap0, 1) + window_smem_doubles(cap1, B));
+__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1, int units0, int units1) {
+  return (size_t)kNumMetrics * (window_smem_doubles(cap0, units0) + window_smem_doubles(cap1, units1));
 }
 
 __device__ __forceinline__ int lower_bound(const double *a, int n, double v) {   // # entries < v
@@ -426,22 +437,22 @@ __device__ __forceinline__ int warp_count_outside(const double *s, int n, double
 // Refreshes q1,q2,q3,k,tau of every (level, metric) window of one kind (Alg. 5).  Whole CTA:
 // the six windows are handled side by side, each by three warps with their own named barrier.
 __device__ void refresh_thresholds(KindState *ks, const double *hist, double *sorted, int cap0, int cap1,
-                                   int B, const Alg5Params &a5, double *s_dyn) {
+                                   int units0, int units1, const Alg5Params &a5, double *s_dyn) {
   const int group = threadIdx.x / kGroupThreads;
   const int gt = threadIdx.x - group * kGroupThreads;
   if (group < kRefreshGroups) {
     const int L = group / kNumMetrics, i = group - L * kNumMetrics;
     const int n = ks->hist_count[L];
     if (n > 0) {                                   // an empty window leaves everything as it is
-      const int cap = L ? cap1 : cap0, units = L ? B : 1, size = ring_size(cap, units);
+      const int cap = L ? cap1 : cap0, units = L ? units1 : units0, size = ring_size(cap, units);
       const int joined = ks->last_joined[L], evicted = ks->last_evicted[L], head = ks->hist_head[L];
       const int n_old = n - joined + evicted;
-      const double *ring = hist + ring_offset(L, i, cap0, cap1, B);
+      const double *ring = hist + ring_offset(L, i, cap0, cap1, units0, units1);
       double *srt = sorted + sorted_offset(L, i, cap0, cap1);
       // this window's shared memory: old copy, new copy, staging, what left, what joined
-      double *s_old = s_dyn + (L ? (size_t)kNumMetrics * window_smem_doubles(cap0, 1) +
-                                       (size_t)i * window_smem_doubles(cap1, B)
-                                 : (size_t)i * window_smem_doubles(cap0, 1));
+      double *s_old = s_dyn + (L ? (size_t)kNumMetrics * window_smem_doubles(cap0, units0) +
+                                       (size_t)i * window_smem_doubles(cap1, units1)
+                                 : (size_t)i * window_smem_doubles(cap0, units0));
       double *s_new = s_old + cap, *s_stage = s_new + cap, *s_out = s_stage + 2 * units, *s_in = s_out + units;
 
       for (int p = gt; p < n_old; p += kGroupThreads) s_old[p] = srt[p];
@@ -656,6 +667,29 @@ __device__ void finalize(const StreamArgs &a) {
   __syncthreads();
 
   KindState *ks = a.hs ? &s_hs.kind[a.kind] : nullptr;     // the shared copy
+  const bool replica = (a.mode == kModeReplicaVerify || a.mode == kModeReplicaWarmup);
+  const bool testing = (a.mode == kModeVerify || a.mode == kModeReplicaVerify);
+  const int w = replica ? a.worker : 0;                      // whose counters this launch moves
+
+  if (a.mode == kModeReplicaVerify && s_hs.banned[w]) {      // banned: not collected, only reported
+    if (tid < rows) {
+      if (a.scores_out)
+        for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = CUDART_NAN_F;
+      if (a.flags_out) a.flags_out[tid] = tid == 0 ? kFlagBanned : 0u;
+    }
+    if (tid == kDecider) {
+      if (w == 0) {                                          // the iteration still starts here
+        ks->steps += 1;
+        ks->step_collected = ks->step_tainted = ks->step_nonfinite = 0u;
+      }
+      ks->refresh_pending = 1;                               // Alg. 5 still runs once per iteration
+      s_hs.ticket = 0u;
+    }
+    __syncthreads();
+    if (tid < kStateWords)
+      reinterpret_cast<unsigned long long *>(a.hs)[tid] = reinterpret_cast<unsigned long long *>(&s_hs)[tid];
+    return;
+  }
 
   // scores and the Tukey test: one thread per unit
   unsigned my_flag = 0u;
@@ -689,7 +723,7 @@ __device__ void finalize(const StreamArgs &a) {
     if (nonfinite) {
       for (int i = 0; i < kNumMetrics; ++i) g[i] = CUDART_NAN;
       my_flag = kFlagNonfinite;
-    } else if (a.mode == kModeVerify) {
+    } else if (testing) {
       const int L = (tid == 0) ? 0 : 1;
       for (int i = 0; i < kNumMetrics; ++i) {
         // (the copy was read from L2 after the ticket, so it holds what CTA 0 of this launch
@@ -709,20 +743,21 @@ __device__ void finalize(const StreamArgs &a) {
 
   // Who joins the history: verified step, the units that raised nothing; warm-up, every unit
   // unless the input was non-finite (then nothing changes).
-  const bool warmup_ok = (a.mode == kModeWarmup) && !any_flag;
+  const bool warmup_ok = (a.mode == kModeWarmup || a.mode == kModeReplicaWarmup) && !any_flag;
   if (tid < rows) {
-    const bool joins = (a.mode == kModeVerify) ? (my_flag == 0u) : warmup_ok;
+    const bool joins = testing ? (my_flag == 0u) : warmup_ok;
     if (joins) {
       // the k-th unit of a level to join goes to ring slot (head + count + k) mod size; the
       // ring has `units` slots more than the window, so what is pushed out is not overwritten
-      const int L = tid ? 1 : 0, size = ring_size(L ? a.cap1 : a.cap0, L ? B : 1);
+      const int L = tid ? 1 : 0, size = ring_size(L ? a.cap1 : a.cap0, L ? a.units1 : a.units0);
       int k = 0;
-      if (L && a.mode == kModeVerify)
+      if (L && testing)
         for (int r = 1; r < tid; ++r) k += (s_flag[r] == 0u);
       else if (L)
         k = tid - 1;
       const int idx = (int)(((long long)ring_head + ring_count + k) % size);
-      for (int i = 0; i < kNumMetrics; ++i) a.hist[ring_offset(L, i, a.cap0, a.cap1, B) + idx] = g[i];
+      for (int i = 0; i < kNumMetrics; ++i)
+        a.hist[ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx] = g[i];
     }
     if (a.scores_out)
       for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = (float)g[i];
@@ -741,41 +776,52 @@ __device__ void finalize(const StreamArgs &a) {
   if (tid == kDecider && a.mode != kModeDistance) {
     HandleState *hs = &s_hs;
     unsigned status = 0u;
-    ks->steps += 1;
+    if (!replica || w == 0) {                    // an iteration starts with its first worker
+      ks->steps += 1;
+      ks->step_collected = ks->step_tainted = ks->step_nonfinite = 0u;
+    }
     int joined[2] = {0, 0};
-    if (a.mode == kModeVerify) {
-      if (any_flag) {                            // violation counter with forgiveness
-        hs->violations += 1;
-        hs->clean_streak = 0;
-        if (hs->violations >= a.ban_violations || s_severe) hs->banned = 1;
+    if (testing) {
+      if (any_flag) {                            // violation counter with forgiveness, per worker
+        hs->violations[w] += 1;
+        hs->clean_streak[w] = 0;
+        if (hs->violations[w] >= a.ban_violations || s_severe) hs->banned[w] = 1;
       } else {
-        hs->clean_streak += 1;
-        if (hs->clean_streak >= a.forgiveness_steps) {
-          hs->violations = hs->violations > 0 ? hs->violations - 1 : 0;
-          hs->clean_streak = 0;
+        hs->clean_streak[w] += 1;
+        if (hs->clean_streak[w] >= a.forgiveness_steps) {
+          hs->violations[w] = hs->violations[w] > 0 ? hs->violations[w] - 1 : 0;
+          hs->clean_streak[w] = 0;
         }
       }
       joined[0] = (s_flag[0] == 0u);
       for (int r = 1; r < rows; ++r) joined[1] += (s_flag[r] == 0u);
       ks->refresh_pending = 1;
-      ks->last_flagged = any_flag ? 1 : 0;
-      if (!any_flag) { ks->active ^= 1; status |= kFlagCommitted; }   // m_t := candidate
+      if (!replica) {
+        ks->last_flagged = any_flag ? 1 : 0;
+        if (!any_flag) { ks->active ^= 1; status |= kFlagCommitted; }   // m_t := candidate
+      }
       if (s_severe) status |= kFlagSevere;
-      if (hs->banned) status |= kFlagBanned;
+      if (hs->banned[w]) status |= kFlagBanned;
       if (s_no_thr) status |= kFlagNoThresholds;
     } else if (warmup_ok) {                      // warm-up: everything joins, always commit
       joined[0] = 1;
       joined[1] = B;
       ks->refresh_pending = 1;
-      ks->active ^= 1;
+      if (!replica) ks->active ^= 1;
+    }
+    if (replica) {                               // what the mean over the clean workers needs
+      ks->step_collected |= 1u << w;
+      if (any_flag) ks->step_tainted |= 1u << w;
+      if (s_flag[0] & kFlagNonfinite) ks->step_nonfinite |= 1u << w;
     }
     for (int L = 0; L < 2; ++L) {                // window bookkeeping after `joined` appends
-      const int cap = L ? a.cap1 : a.cap0, size = ring_size(cap, L ? B : 1);
+      const int cap = L ? a.cap1 : a.cap0, size = ring_size(cap, L ? a.units1 : a.units0);
       const int total = ks->hist_count[L] + joined[L];
       const int evicted = total > cap ? total - cap : 0;
       ks->hist_count[L] = total - evicted;
       ks->hist_head[L] = (int)(((long long)ks->hist_head[L] + evicted) % size);
-      if (ks->refresh_pending) { ks->last_joined[L] = joined[L]; ks->last_evicted[L] = evicted; }
+      // (several workers append between two refreshes: what the refresh merges accumulates)
+      if (ks->refresh_pending) { ks->last_joined[L] += joined[L]; ks->last_evicted[L] += evicted; }
     }
     s_hs.ticket = 0u;                            // ready for the next launch
     s_status = status;
@@ -812,6 +858,7 @@ stream_kernel(const StreamArgs a) {
 
   const float *m_in;
   float *m_out;
+  bool skip_stream = false;
   if (a.mode == kModeDistance) {
     m_in = a.m_ext;
     m_out = nullptr;
@@ -819,14 +866,23 @@ stream_kernel(const StreamArgs a) {
     const int act = __ldcg(&a.hs->kind[a.kind].active);   // written by an earlier launch only
     m_in = a.ema[act];
     m_out = a.ema[act ^ 1];
+    if (a.mode == kModeReplicaVerify || a.mode == kModeReplicaWarmup) {
+      m_out = nullptr;                     // the reference moves once, after all workers
+      // a banned worker is no longer collected: nothing of its tensor is read
+      skip_stream = (a.mode == kModeReplicaVerify) && __ldcg(&a.hs->banned[a.worker]) != 0;
+    }
   }
 
   if (blockIdx.x == 0) {
     if (a.hs) {
       KindState *ks = &a.hs->kind[a.kind];
-      if (ks->refresh_pending) refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.B, a.a5, s_dyn);
+      // within a multi-worker iteration only the first worker's launch refreshes: Alg. 5 runs
+      // once per iteration, after the worker loop
+      const bool may_refresh = (a.mode != kModeReplicaVerify && a.mode != kModeReplicaWarmup) || a.worker == 0;
+      if (ks->refresh_pending && may_refresh)
+        refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.a5, s_dyn);
     }
-  } else {
+  } else if (!skip_stream) {
     stream_cta(a, blockIdx.x - 1, m_in, m_out, s_part);
   }
 
@@ -845,13 +901,14 @@ stream_kernel(const StreamArgs a) {
 // Brings both kinds' thresholds up to date outside a streaming launch (queries, export).
 __global__ void __launch_bounds__(kThreads)
 refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, double *sorted_act,
-               double *sorted_grad, int cap0, int cap1, int B, Alg5Params a5_act, Alg5Params a5_grad) {
+               double *sorted_grad, int cap0, int cap1, int units0, int units1, Alg5Params a5_act,
+               Alg5Params a5_grad) {
   extern __shared__ double s_dyn[];
   if (hs->kind[0].refresh_pending)
-    refresh_thresholds(&hs->kind[0], hist_act, sorted_act, cap0, cap1, B, a5_act, s_dyn);
+    refresh_thresholds(&hs->kind[0], hist_act, sorted_act, cap0, cap1, units0, units1, a5_act, s_dyn);
   __syncthreads();
   if (hs->kind[1].refresh_pending)
-    refresh_thresholds(&hs->kind[1], hist_grad, sorted_grad, cap0, cap1, B, a5_grad, s_dyn);
+    refresh_thresholds(&hs->kind[1], hist_grad, sorted_grad, cap0, cap1, units0, units1, a5_grad, s_dyn);
 }
 
 // Alg. 4 (GradientReplacement) for the one submission a handle sees: if the last verified step
@@ -895,10 +952,60 @@ replace_kernel(const HandleState *hs, int kind, const float *ema0, const float *
   }
 }
 
-__global__ void reset_worker_kernel(HandleState *hs) {
-  hs->violations = 0;
-  hs->clean_streak = 0;
-  hs->banned = 0;
+// Second half of a multi-worker iteration (Alg. 1 main loop, Eq. 1): after every worker has
+// been scored, decide who is tainted -- the flagged workers, unless more than half of the
+// workers still in the pool were flagged, which Alg. 2 reads as a natural distribution shift
+// and clears -- and move the reference with the mean over the others, in place:
+//   m <- beta m + (1 - beta) / |clean| * sum_{r clean} x^(r).
+// Every CTA derives the same clean set from the masks the scoring launches left in the state.
+// Traffic: 4 B read + 4 B written of m and 2 B per clean worker, per element.
+struct WorkerPointers { const uint16_t *x[kMaxWorkers]; };
+
+__global__ void __launch_bounds__(kReplaceThreads)
+ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, float *ema0, float *ema1, long long n_chunks,
+                int R, int rows, float beta, float one_minus_beta, int warmup, unsigned *flags_out) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  KindState *ks = &hs->kind[kind];
+  const unsigned collected = ks->step_collected, tainted = ks->step_tainted, nonfinite = ks->step_nonfinite;
+  int n_banned = 0;
+  for (int r = 0; r < R; ++r) n_banned += hs->banned[r] != 0;
+  const bool natural = !warmup && 2 * __popc(tainted) > R - n_banned;
+  const unsigned clean = collected & ~(natural ? nonfinite : tainted);
+  const int n_clean = __popc(clean);
+
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    ks->last_flagged = (tainted != 0u && !natural) ? 1 : 0;
+    if (flags_out)
+      for (int r = 0; r < R; ++r)
+        flags_out[(size_t)r * rows] |= ((clean >> r) & 1u ? kFlagCommitted : 0u) | (natural ? kFlagNaturalShift : 0u);
+  }
+  if (n_clean == 0) return;
+  float *m = ks->active ? ema1 : ema0;
+  const float wgt = one_minus_beta / (float)n_clean;
+  const long long stride = (long long)gridDim.x * kReplaceThreads;
+  for (long long c = (long long)blockIdx.x * kReplaceThreads + threadIdx.x; c < n_chunks; c += stride) {
+    F8 mv = ld_m256(m + c * 8);
+    float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int r = 0; r < R; ++r) {
+      if (!((clean >> r) & 1u)) continue;
+      const uint4 xv = ld_x128(xs.x[r] + c * 8);
+      const unsigned wv[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        sum[2 * j] += __uint_as_float(wv[j] << 16);
+        sum[2 * j + 1] += __uint_as_float(wv[j] & 0xFFFF0000u);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mv.v[j] = fmaf(beta, mv.v[j], wgt * sum[j]);
+    st_m256(m + c * 8, mv);
+  }
+}
+
+__global__ void reset_worker_kernel(HandleState *hs, int worker) {
+  hs->violations[worker] = 0;
+  hs->clean_streak[worker] = 0;
+  hs->banned[worker] = 0;
 }
 
 }  // namespace sentinel

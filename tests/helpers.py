@@ -57,16 +57,19 @@ def near_threshold(scores, thr, valid, B, rel=REL):
 
 def oracle_to_blob(v, params) -> bytes:
     """Serialise an oracle verifier into the library's checkpoint format."""
-    B, T, d, l = params.B, params.T, params.d, params.l
-    viol, streak, banned = v.counters()
-    out = bytearray(struct.pack("<QI7i", MAGIC, 1, B, T, d, l, viol, streak, banned))
+    B, T, d, l, R = params.B, params.T, params.d, params.l, params.R
+    out = bytearray(struct.pack("<QI5i", MAGIC, 2, B, T, d, l, R))
     out += b"\0" * (64 - len(out))
+    workers = np.zeros((3, 16), dtype="<i4")
+    for r in range(R):
+        workers[:, r] = v.worker_counters(r)
+    out += workers.tobytes()
     for kind in (0, 1):
         thr, valid = v.thresholds(kind)
         counts = [v.history(kind, L, 0).size for L in (0, 1)]
         out += struct.pack("<q2i6i", v.steps(kind), *counts, *valid.astype(int).reshape(-1))
         out += thr.astype("<f8").tobytes()
-        for L, cap in ((0, l), (1, l * B)):
+        for L, cap in ((0, l * R), (1, l * R * B)):
             for i in range(3):
                 h = np.zeros(cap)
                 hv = v.history(kind, L, i)
@@ -76,13 +79,15 @@ def oracle_to_blob(v, params) -> bytes:
     return bytes(out)
 
 
-def parse_blob(blob, B, T, d, l) -> dict:
+def parse_blob(blob, B, T, d, l, R=1) -> dict:
     """Decode a checkpoint blob into plain numpy pieces."""
     buf = memoryview(bytes(blob))
-    magic, version, b, t, dd, ll, viol, streak, banned = struct.unpack_from("<QI7i", buf, 0)
-    assert magic == MAGIC and version == 1 and (b, t, dd, ll) == (B, T, d, l)
-    off = 64
-    out = {"violations": viol, "clean_streak": streak, "banned": banned, "kinds": []}
+    magic, version, b, t, dd, ll, rr = struct.unpack_from("<QI5i", buf, 0)
+    assert magic == MAGIC and version == 2 and (b, t, dd, ll, rr) == (B, T, d, l, R)
+    workers = np.frombuffer(buf, dtype="<i4", count=48, offset=64).reshape(3, 16)
+    off = 64 + 192
+    out = {"violations": int(workers[0, 0]), "clean_streak": int(workers[1, 0]), "banned": int(workers[2, 0]),
+           "workers": workers.copy(), "kinds": []}
     N = B * T * d
     for _ in range(2):
         steps, c0, c1 = struct.unpack_from("<q2i", buf, off)
@@ -91,7 +96,7 @@ def parse_blob(blob, B, T, d, l) -> dict:
         thr = np.frombuffer(buf, dtype="<f8", count=36, offset=off).reshape(2, 3, 6).copy()
         off += 288
         hist = [[None] * 3, [None] * 3]
-        for L, cap, cnt in ((0, l, c0), (1, l * B, c1)):
+        for L, cap, cnt in ((0, l * R, c0), (1, l * R * B, c1)):
             for i in range(3):
                 hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
                 off += 8 * cap
@@ -101,3 +106,23 @@ def parse_blob(blob, B, T, d, l) -> dict:
                              "hist": hist, "m": m})
     assert off == len(buf)
     return out
+
+
+def whole_step_k_events(gt, gvalid, ot, ovalid, params, kind) -> int:
+    """Alg. 5 compares every window entry with a fence; an entry that lies on a fence to within the
+    score tolerance may fall on either side, which moves k by whole widen/narrow steps.  Returns
+    the number of (level, metric) windows where the two multipliers differ that way; any other
+    difference fails."""
+    assert np.array_equal(gvalid, ovalid)
+    events = 0
+    lg, ls = np.log(params.gamma_g[kind]), np.log(params.gamma_s[kind])
+    n = params.n_max[kind]
+    for L in range(2):
+        for i in range(3):
+            if not ovalid[L, i] or abs(gt[L, i, 3] / ot[L, i, 3] - 1.0) <= 1e-12:
+                continue
+            r = np.log(gt[L, i, 3] / ot[L, i, 3])
+            whole = any(abs(r - (a * lg + b * ls)) < 1e-9 for a in range(-n, n + 1) for b in range(-n, n + 1))
+            assert whole, "k differs by no whole number of steps: %r vs %r" % (gt[L, i, 3], ot[L, i, 3])
+            events += 1
+    return events

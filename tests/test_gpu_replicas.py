@@ -1,0 +1,146 @@
+"""GPU parity of the multi-worker iteration (worker loop of Alg. 2 / Alg. 3, pooled history,
+>50% rule, Eq. 1 with the mean over the clean workers) against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import (UNIT_BITS, assert_scores_close, near_threshold, oracle_to_blob, parse_blob,
+                     whole_step_k_events)
+from paper_2603_03592_b200 import synth
+
+pytestmark = pytest.mark.gpu
+ACT, GRAD = 0, 1
+
+
+@pytest.fixture(scope="module")
+def sb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_03592_b200 import binding
+    binding.lib()
+    return binding
+
+
+def pair(sb, oracle_mod, w, R, **kw):
+    names = {"l": "window_steps", "c": "ban_violations", "t_forgiveness": "forgiveness_steps"}
+    gv = sb.Verifier(w.B, w.T, w.d, n_workers=R, **{names.get(k, k): v for k, v in kw.items()})
+    params = oracle_mod.Params(B=w.B, T=w.T, d=w.d, R=R, **kw)
+    return gv, oracle_mod.Verifier(params), params
+
+
+def inputs(w, R, kind, t, scale=None):
+    xs = [synth.clean(w, r, kind, t, "cuda") for r in range(R)]
+    for r, c in (scale or {}).items():
+        xs[r] = (xs[r].float() * c).to(torch.bfloat16)
+    return xs
+
+
+def step_both(gv, ov, xs, kind, warmup=False):
+    gs, gf = gv.step_replicas(xs, kind, warmup)
+    os_, of, n = ov.step_replicas([synth.bits(x) for x in xs], kind, warmup)
+    torch.cuda.synchronize()
+    return gs.cpu().numpy(), gf.cpu().numpy().view(np.uint32), os_, of, n
+
+
+def check_state(gv, ov, params, kinds=(ACT, GRAD)):
+    st = parse_blob(gv.sentinel_export_state(), params.B, params.T, params.d, params.l, params.R)
+    for r in range(params.R):
+        assert tuple(int(v) for v in st["workers"][:, r]) == ov.worker_counters(r), r
+        assert gv.sentinel_get_worker_counters(r) == ov.worker_counters(r)
+    for kind in kinds:
+        ks = st["kinds"][kind]
+        m_ref = ov.ema(kind)
+        assert np.max(np.abs(ks["m"].astype(np.float64) - m_ref)) <= 1e-5 * max(float(np.abs(m_ref).max()), 1e-30)
+        assert ks["steps"] == ov.steps(kind)
+        for L in range(2):
+            for i in range(3):
+                href = ov.history(kind, L, i)
+                assert ks["hist"][L][i].size == href.size
+                floor = 1e-3 * (np.abs(href).mean() if i == 0 and href.size else 1.0)
+                assert np.all(np.abs(ks["hist"][L][i] - href) <= 1e-3 * np.maximum(np.abs(href), floor))
+        gt, gvalid = gv.sentinel_get_thresholds(kind)
+        ot, ovalid = ov.thresholds(kind)
+        assert np.array_equal(gvalid, ovalid)
+        for L in range(2):
+            for i in range(3):
+                if ovalid[L, i]:
+                    assert gt[L, i, 3] == pytest.approx(ot[L, i, 3], rel=1e-12)
+
+
+@pytest.mark.parametrize("shape,R", [((3, 12, 264), 4), ((2, 40, 1024), 5), ((4, 6, 64), 16)],
+                         ids=["3x12x264_R4", "2x40x1024_R5", "4x6x64_R16"])
+def test_iterations_in_lockstep(sb, oracle_mod, shape, R):
+    """Warm-up, clean iterations, one tainted worker, a majority of flagged workers, a worker
+    that gets banned and is then skipped -- scores, flags, counters, histories, multipliers and
+    the reference after every phase."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "replicas", *shape)
+    gv, ov, params = pair(sb, oracle_mod, w, R, l=5, c=2)
+    script = [("warm", {})] * 8 + [("verify", {})] * 3 + [("verify", {1: 6.0})] + [("verify", {})] + \
+             [("verify", {r: 3.0 for r in range(R // 2 + 1)})] + [("verify", {1: 6.0})] + [("verify", {})] * 2
+    k_events = 0
+    for kind in (ACT, GRAD):
+        for t, (what, scale) in enumerate(script):
+            xs = inputs(w, R, kind, t, scale)
+            thr, valid = ov.thresholds(kind)
+            gs, gf, os_, of, n = step_both(gv, ov, xs, kind, warmup=(what == "warm"))
+            for r in range(R):
+                x_scale = float(xs[r].float().abs().mean())
+                assert_scores_close(gs[r], os_[r], x_scale, "kind %d step %d worker %d" % (kind, t, r))
+            if what == "warm":
+                assert np.array_equal(gf & ~np.uint32(UNIT_BITS), of & ~np.uint32(UNIT_BITS))
+                continue
+            if not np.array_equal(gf, of):
+                for r in range(R):
+                    near = near_threshold(os_[r], thr, valid, w.B)
+                    assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+                gv.sentinel_import_state(oracle_to_blob(ov, params))
+            if scale and len(scale) > 1:
+                assert np.all(of[:, 0] & sb.FLAG_NATURAL_SHIFT)
+            ev = whole_step_k_events(*gv.sentinel_get_thresholds(kind), *ov.thresholds(kind), params, kind)
+            if ev:                                          # an entry sat on a fence: re-align
+                k_events += ev
+                gv.sentinel_import_state(oracle_to_blob(ov, params))
+        check_state(gv, ov, params, kinds=(kind,))
+    assert ov.worker_counters(1)[2] == 1                    # worker 1 ended up banned
+    assert k_events <= 4, k_events
+    gv.close()
+
+
+def test_full_width_rows(sb, oracle_mod):
+    """Two workers at a stage-traffic width (d = 4096, several tiles per row)."""
+    w = synth.scaled(synth.WORKLOADS["cfg3"], "replicas_wide", 2, 96, 4096)
+    gv, ov, params = pair(sb, oracle_mod, w, 2)
+    for t in range(6):
+        xs = inputs(w, 2, ACT, t, {0: 5.0} if t == 5 else None)
+        gs, gf, os_, of, n = step_both(gv, ov, xs, ACT, warmup=t < 4)
+        for r in range(2):
+            assert_scores_close(gs[r], os_[r], float(xs[r].float().abs().mean()), "wide %d %d" % (t, r))
+        if t >= 4:
+            assert np.array_equal(gf, of)
+    check_state(gv, ov, params, kinds=(ACT,))
+    gv.close()
+
+
+def test_argument_checks(sb):
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(2, 4, 16, n_workers=17)
+    assert e.value.code == sb.ERR_INVALID_ARG
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(8, 4, 16, n_workers=8)                  # 100 * 8 * 9 > 4096
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    v = sb.Verifier(2, 4, 16, n_workers=2)
+    x = torch.zeros(2, 4, 16, dtype=torch.bfloat16, device="cuda")
+    scores = torch.zeros(2, 3, 3, device="cuda")
+    flags = torch.zeros(2, 3, dtype=torch.int32, device="cuda")
+    L, s = sb.lib(), torch.cuda.current_stream().cuda_stream
+    import ctypes as C
+    good = (C.c_void_p * 2)(x.data_ptr(), x.data_ptr())
+    bad = (C.c_void_p * 2)(x.data_ptr(), None)
+    assert L.sentinel_verify_replicas(v._h, bad, 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_INVALID_ARG
+    assert L.sentinel_verify_replicas(v._h, None, 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_INVALID_ARG
+    assert L.sentinel_verify_replicas(v._h, good, 0, 2, 4, 8, s, scores.data_ptr(), flags.data_ptr()) == sb.ERR_SHAPE_MISMATCH
+    assert L.sentinel_verify_replicas(v._h, good, 0, 2, 4, 16, s, scores.data_ptr(), None) == sb.ERR_INVALID_ARG
+    assert L.sentinel_reset_worker(v._h, 2, s) == sb.ERR_INVALID_ARG
+    assert L.sentinel_verify_replicas(v._h, good, 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.OK
+    torch.cuda.synchronize()
+    v.close()
