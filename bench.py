@@ -263,6 +263,24 @@ def run_ours(args, rank, world, local_rank):
                         "kernels": "%d x stream_kernel (scores only) + ema_mean_kernel" % R}
         vr.sentinel_destroy()
 
+    # extra figure, outside the timed region: the strided (compressed-signal) layout, rows d+1 apart
+    strided = None
+    if nb == 1:
+        wide = [torch.nn.functional.pad(xs[0][ACT][i % nd], (0, 1)).contiguous() for i in range(3)]
+        for i in range(2):
+            vs[0].sentinel_update_reference_strided(wide[i], ACT, scores[0, 0], main)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        c0.record(main)
+        for i in range(9):
+            vs[0].sentinel_update_reference_strided(wide[i % 3], ACT, scores[0, 0], main)
+        c1.record(main)
+        torch.cuda.synchronize()
+        cms = c0.elapsed_time(c1) / 9
+        strided = {"row_stride": w.d + 1, "bytes_per_element": 10, "ms_per_launch": round(cms, 4),
+                   "achieved_gbs": round(10 * N / (cms * 1e-3) / 1e9, 1), "kernel": "stream_kernel_t<true>"}
+        del wide
+
     # end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     hx = [{k: [xs[b][k][i % nd].cpu().pin_memory() for i in range(min(e2e_steps, 2 if nb > 1 else 4))]
@@ -332,6 +350,8 @@ def run_ours(args, rank, world, local_rank):
         out["sliced_wasserstein"] = swd
     if replicas_fig is not None:
         out["multi_worker_iteration"] = replicas_fig
+    if strided is not None:
+        out["compressed_layout"] = strided
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
     return out

@@ -88,7 +88,8 @@ typedef struct sentinel_config {
   int    ban_violations;   /* c                                                5           */
   int    forgiveness_steps;/* T_forgiveness                                    100         */
   unsigned metric_mask;    /* bit i set: metric i may raise a flag             7           */
-  int    B, T, d;          /* shape of every submission; d % 8 == 0, B <= SENTINEL_MAX_B   */
+  int    B, T, d;          /* shape of every submission; B <= SENTINEL_MAX_B; d % 8 == 0
+                              unless only the _strided entry points are used              */
   int    device;           /* CUDA device ordinal                                           */
   int    n_workers;        /* workers d_s feeding this boundary (multi-worker calls)   1    */
 } sentinel_config;
@@ -121,6 +122,21 @@ int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
  * No flags, no counters.  A non-finite x changes nothing.  dev_scores_out may be NULL. */
 int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B,
                               int T, int d, void *cuda_stream, float *dev_scores_out);
+
+/* sentinel_verify / sentinel_update_reference for a tensor whose rows are not packed: row
+ * (b,t) starts row_stride elements after the previous one (row_stride >= d) and dev_x needs
+ * 2-byte alignment only; d may be any positive number.  This is the layout of a
+ * subspace-compressed signal, of which the verifier checks x[:, :, :-1] (SWARM appendix,
+ * "compatibility with subspace compression"): pass the [B,T,k+1] tensor with d = k and
+ * row_stride = k+1.  The reference stays dense [B,T,d].  Same arithmetic, scalar instead of
+ * 128/256-bit memory accesses.  A handle created with d % 8 != 0 can only be used through
+ * these two calls (and the queries / checkpointing). */
+int sentinel_verify_strided(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T,
+                            int d, long long row_stride, void *cuda_stream, float *dev_scores_out,
+                            unsigned *dev_flags_out);
+int sentinel_update_reference_strided(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
+                                      int B, int T, int d, long long row_stride, void *cuda_stream,
+                                      float *dev_scores_out);
 
 /* sentinel_verify for callers whose tensor and results live in host memory: copies x to a
  * staging buffer owned by the handle (allocated on first use), runs the check, copies scores

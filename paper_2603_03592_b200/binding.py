@@ -31,6 +31,7 @@ EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
     "sentinel_verify_replicas", "sentinel_update_reference_replicas", "sentinel_get_worker_counters",
+    "sentinel_verify_strided", "sentinel_update_reference_strided",
     "sentinel_distance_noalloc", "sentinel_replace_if_flagged", "sentinel_sliced_wasserstein",
     "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
     "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
@@ -88,6 +89,8 @@ def lib():
         L.sentinel_get_counters.argtypes = [vp, vp, vp]
         L.sentinel_set_token_stats_buffer.argtypes = [vp, vp]
         L.sentinel_reset_worker.argtypes = [vp, ip, vp]
+        L.sentinel_verify_strided.argtypes = [vp, vp, ip, ip, ip, ip, C.c_longlong, vp, vp, vp]
+        L.sentinel_update_reference_strided.argtypes = [vp, vp, ip, ip, ip, ip, C.c_longlong, vp, vp]
         L.sentinel_verify_replicas.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_update_reference_replicas.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_get_worker_counters.argtypes = [vp, ip, vp, vp]
@@ -195,6 +198,19 @@ class Verifier:
         _check(lib().sentinel_verify_host(self._h, _ptr(x_host), kind, B, T, d,
                                           _stream_ptr(stream), _ptr(scores_host),
                                           _ptr(flags_host)), self._h)
+
+    def sentinel_verify_strided(self, x_wide: torch.Tensor, kind: int, scores_out: torch.Tensor,
+                                flags_out: torch.Tensor, stream=None) -> None:
+        """x_wide: [B, T, row_stride] bf16 of which the first d channels of every row are verified."""
+        _check(lib().sentinel_verify_strided(self._h, _ptr(x_wide), kind, self.B, self.T, self.d,
+                                             x_wide.shape[2], _stream_ptr(stream), _ptr(scores_out),
+                                             _ptr(flags_out)), self._h)
+
+    def sentinel_update_reference_strided(self, x_wide: torch.Tensor, kind: int,
+                                          scores_out: torch.Tensor | None = None, stream=None) -> None:
+        _check(lib().sentinel_update_reference_strided(self._h, _ptr(x_wide), kind, self.B, self.T, self.d,
+                                                       x_wide.shape[2], _stream_ptr(stream),
+                                                       _ptr(scores_out)), self._h)
 
     def _worker_pointers(self, xs):
         assert len(xs) == self.R, "one tensor per worker"

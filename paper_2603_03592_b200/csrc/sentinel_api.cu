@@ -119,7 +119,7 @@ int streaming_ctas(int device, int B, int T, std::string *err) {
   int sms = 0, occ = 0;
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess)
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, stream_kernel, kThreads, 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, stream_kernel_t<false>, kThreads, 0);
   if (e != cudaSuccess || sms < 1 || occ < 1) {
     if (err) *err = std::string("occupancy query failed: ") + cudaGetErrorString(e);
     return -1;
@@ -152,11 +152,11 @@ void keep_pool_warm(int device) {
   cudaGetLastError();
 }
 
-int tiles_per_row(int d) { return ((d >> 3) + 32 * kUnroll - 1) / (32 * kUnroll); }
+int tiles_per_row(int d) { return (((d + 7) >> 3) + 32 * kUnroll - 1) / (32 * kUnroll); }
 
-int check_shape(sentinel_verifier *h, int B, int T, int d) {
+int check_shape(sentinel_verifier *h, int B, int T, int d, bool vector_path = true) {
   if (B < 1 || T < 1 || d < 1) return fail(h, SENTINEL_ERR_INVALID_ARG, "B, T, d must be positive (got %d, %d, %d)", B, T, d);
-  if (d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", d);
+  if (vector_path && d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", d);
   if (B > SENTINEL_MAX_B) return fail(h, SENTINEL_ERR_UNSUPPORTED, "B = %d exceeds SENTINEL_MAX_B = %d", B, SENTINEL_MAX_B);
   return SENTINEL_OK;
 }
@@ -167,7 +167,20 @@ int check_call(sentinel_verifier *h, const void *x, int kind, int B, int T, int 
   if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", kind);
   if (B != h->cfg.B || T != h->cfg.T || d != h->cfg.d)
     return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
+  if (d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8: use the _strided entry points", d);
   if (!aligned16(x)) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 16-byte aligned");
+  return SENTINEL_OK;
+}
+
+// the strided entry points: any d, rows row_stride elements apart, 2-byte alignment
+int check_call_strided(sentinel_verifier *h, const void *x, int kind, int B, int T, int d, long long row_stride) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!x) return fail(h, SENTINEL_ERR_INVALID_ARG, "x is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", kind);
+  if (B != h->cfg.B || T != h->cfg.T || d != h->cfg.d)
+    return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
+  if (row_stride < d) return fail(h, SENTINEL_ERR_INVALID_ARG, "row_stride = %lld is smaller than d = %d", row_stride, d);
+  if (reinterpret_cast<uintptr_t>(x) & 1u) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 2-byte aligned");
   return SENTINEL_OK;
 }
 
@@ -196,6 +209,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.cap0 = h->cap0; a.cap1 = h->cap1;
   a.units0 = h->units0; a.units1 = h->units1;
   a.R = h->R; a.worker = 0;
+  a.x_row_stride = h->cfg.d;
   a.a5 = alg5_of(h->cfg, kind);
   a.severe_mult = h->cfg.severe_mult;
   a.ban_violations = h->cfg.ban_violations;
@@ -204,7 +218,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   return a;
 }
 
-int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) {
+int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, bool scalar = false) {
   // launched with programmatic stream serialization: the grid may be set up while the previous
   // kernel on the stream drains; every CTA waits for that kernel before it reads anything
   cudaLaunchConfig_t lc;
@@ -218,7 +232,8 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s) 
   attr.val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = &attr;
   lc.numAttrs = 1;
-  SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel, a));
+  if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true>, a));
+  else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false>, a));
   return SENTINEL_OK;
 }
 
@@ -283,7 +298,7 @@ int sentinel_default_config(sentinel_config *cfg) {
 int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out) {
   if (!cfg || !out) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "cfg or out is NULL");
   *out = nullptr;
-  int rc = check_shape(nullptr, cfg->B, cfg->T, cfg->d);
+  int rc = check_shape(nullptr, cfg->B, cfg->T, cfg->d, false);   // d % 8 != 0: strided entry points only
   if (rc) return rc;
   for (int k = 0; k < 2; ++k) {
     if (!(cfg->beta[k] >= 0.0 && cfg->beta[k] < 1.0)) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "beta[%d] = %g is outside [0,1)", k, cfg->beta[k]);
@@ -323,7 +338,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   }
   {   // the windows' working copies may exceed the 48 KiB a kernel gets without asking
     const int most = 200 * 1024;
-    cudaError_t ae = cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaError_t ae = cudaFuncSetAttribute(stream_kernel_t<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
   }
@@ -383,6 +399,29 @@ int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_
                 static_cast<cudaStream_t>(cuda_stream));
 }
 
+int sentinel_verify_strided(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T, int d,
+                            long long row_stride, void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out) {
+  int rc = check_call_strided(h, dev_x, kind, B, T, d, row_stride);
+  if (rc) return rc;
+  if (!dev_scores_out || !dev_flags_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  StreamArgs a = make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out);
+  a.x_row_stride = row_stride;
+  return launch(h, a, h->G + 1, static_cast<cudaStream_t>(cuda_stream), true);
+}
+
+int sentinel_update_reference_strided(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T,
+                                      int d, long long row_stride, void *cuda_stream, float *dev_scores_out) {
+  int rc = check_call_strided(h, dev_x, kind, B, T, d, row_stride);
+  if (rc) return rc;
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  StreamArgs a = make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr);
+  a.x_row_stride = row_stride;
+  return launch(h, a, h->G + 1, static_cast<cudaStream_t>(cuda_stream), true);
+}
+
 int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind kind, int B, int T,
                          int d, void *cuda_stream, float *host_scores_out, unsigned *host_flags_out) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
@@ -390,6 +429,7 @@ int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind
   if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", (int)kind);
   if (B != h->cfg.B || T != h->cfg.T || d != h->cfg.d)
     return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
+  if (d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8: use the _strided entry points", d);
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
@@ -440,8 +480,9 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   a.scores_out = dev_scores_out;
   a.stats_out = dev_stats_out;
   a.B = B; a.T = T; a.d = d; a.G = G;
+  a.x_row_stride = d;
   a.mode = kModeDistance;
-  stream_kernel<<<G + 1, kThreads, 0, s>>>(a);
+  stream_kernel_t<false><<<G + 1, kThreads, 0, s>>>(a);
   cudaError_t le = cudaGetLastError();
   cudaError_t fe = cudaFreeAsync(scratch, s);
   SENTINEL_CUDA(nullptr, le);
@@ -899,8 +940,9 @@ int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int 
   a.scores_out = dev_scores_out;
   a.stats_out = dev_stats_out;
   a.B = B; a.T = T; a.d = d; a.G = G;
+  a.x_row_stride = d;
   a.mode = kModeDistance;
-  stream_kernel<<<G + 1, kThreads, 0, s>>>(a);
+  stream_kernel_t<false><<<G + 1, kThreads, 0, s>>>(a);
   SENTINEL_CUDA(nullptr, cudaGetLastError());
   return SENTINEL_OK;
 }

@@ -98,6 +98,8 @@ struct StreamArgs {
   int cap0, cap1;
   int units0, units1;              // entries one iteration can append per level: R and R*B
   int R, worker;                   // workers of the stage; which one this launch scores
+  long long x_row_stride;          // elements from one row of x to the next (d when dense)
+  int pad2[2];
   Alg5Params a5;
   double severe_mult;
   int ban_violations, forgiveness_steps;
@@ -213,12 +215,17 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
 
 constexpr int kSegsPerCta = 2;
 
+// kScalar: the layout of a subspace-compressed signal, x[:, :, :-1] of a [B,T,k+1] tensor (SWARM
+// appendix): rows of x are row_stride elements apart and start on any 2-byte boundary, and d
+// need not be a multiple of 8.  Lanes then own interleaved columns (col = tile + q*32 + lane),
+// so that every 2-byte / 4-byte access of a warp is contiguous; the arithmetic is the same.
+template <bool kScalar>
 __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long long rb,
                                const float *m_in, float *m_out,
                                unsigned long long (*s_part)[kSlotWords],
                                unsigned long long *slot) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int chunks = a.d >> 3;
+  const int chunks = (a.d + 7) >> 3;
   const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
   const int n_tiles = (int)(rb - ra) * tiles_per_row;       // < 2^31: rows/G * d/1024
   const size_t sample_off = (size_t)b * a.T * a.d;
@@ -226,7 +233,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
   const bool tokens = (a.token_out != nullptr);
   const float beta = a.beta, omb = a.one_minus_beta;
 
-  const unsigned x0 = a.x[sample_off];
+  const unsigned x0 = a.x[(size_t)b * a.T * (size_t)a.x_row_stride];
   const unsigned x0pair = x0 | (x0 << 16);
   const unsigned m0bits = __float_as_uint(m_in[sample_off]);
 
@@ -239,25 +246,52 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
     const long long row = ra + rr;
     const size_t off = (size_t)row * a.d;
     const int base = seg * 32 * kUnroll;
-
-    uint4 xv[kUnroll];
-    F8 mv[kUnroll];
-    bool ok[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int c = base + u * 32 + lane;
-      ok[u] = c < chunks;
-      if (ok[u]) {
-        xv[u] = ld_x128(a.x + off + (size_t)c * 8);
-        mv[u] = ld_m256(m_in + off + (size_t)c * 8);
-      }
-    }
     GroupAcc g = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0u};
+
+    if (kScalar) {
+      constexpr int kPerLane = 8 * kUnroll;
+      const size_t off_x = (size_t)row * (size_t)a.x_row_stride;
+      const int col0 = base * 8 + lane;
+      const float x0f = __uint_as_float(x0 << 16), m0f = __uint_as_float(m0bits);
+      unsigned short xs[kPerLane];
+      float ms[kPerLane];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      if (ok[u]) {
-        chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
-        if (write_ema) st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+      for (int q = 0; q < kPerLane; ++q) {
+        const int col = col0 + q * 32;
+        if (col < a.d) { xs[q] = a.x[off_x + col]; ms[q] = m_in[off + col]; }
+      }
+#pragma unroll
+      for (int q = 0; q < kPerLane; ++q) {
+        const int col = col0 + q * 32;
+        if (col < a.d) {
+          const unsigned xb = xs[q];
+          t.nf_bits |= ((xb & 0x7F80u) == 0x7F80u) ? 1u : 0u;
+          t.x_diff |= xb ^ x0;
+          t.m_diff |= __float_as_uint(ms[q]) ^ m0bits;
+          const float xf = __uint_as_float(xb << 16);
+          element(xf, ms[q], x0f, m0f, g);
+          if (write_ema) m_out[off + col] = fmaf(beta, ms[q], omb * xf);
+        }
+      }
+    } else {
+      uint4 xv[kUnroll];
+      F8 mv[kUnroll];
+      bool ok[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int c = base + u * 32 + lane;
+        ok[u] = c < chunks;
+        if (ok[u]) {
+          xv[u] = ld_x128(a.x + off + (size_t)c * 8);
+          mv[u] = ld_m256(m_in + off + (size_t)c * 8);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (ok[u]) {
+          chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
+          if (write_ema) st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+        }
       }
     }
     // fold the short fp32 run into the fp64 accumulators
@@ -337,6 +371,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
   }
 }
 
+template <bool kScalar>
 __device__ void stream_cta(const StreamArgs &a, int c, const float *m_in, float *m_out,
                            unsigned long long (*s_part)[kSlotWords]) {
   const long long R = (long long)a.B * a.T;
@@ -348,7 +383,7 @@ __device__ void stream_cta(const StreamArgs &a, int c, const float *m_in, float 
       const int b = (int)(ra / a.T);
       const long long sample_end = (long long)(b + 1) * a.T;
       const long long rb = sample_end < R1 ? sample_end : R1;
-      stream_segment(a, b, ra, rb, m_in, m_out, s_part, slot);
+      stream_segment<kScalar>(a, b, ra, rb, m_in, m_out, s_part, slot);
       ra = rb;
     } else if (threadIdx.x == 0) {
       slot[7] = 0ull;                   // tag 0: unused
@@ -844,8 +879,11 @@ __device__ void finalize(const StreamArgs &a) {
 // step left that pending) while the others stream.  Every CTA then takes a ticket; whoever
 // draws the last one has, by the fence/atomic order, everybody's partial sums and the fresh
 // thresholds in view, and finalizes.  No CTA ever waits for another.
+// (kScalar = true is the variant for rows of x that are strided or not 16-byte aligned; it is a
+// kernel of its own so that the vector path keeps its registers)
+template <bool kScalar>
 __global__ void __launch_bounds__(kThreads)
-stream_kernel(const StreamArgs a) {
+stream_kernel_t(const StreamArgs a) {
   __shared__ unsigned long long s_part[kWarps][kSlotWords];
   __shared__ int s_last;
   extern __shared__ double s_dyn[];            // refresh_smem_doubles(cap0, cap1) when a handle is given
@@ -883,7 +921,7 @@ stream_kernel(const StreamArgs a) {
         refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.a5, s_dyn);
     }
   } else if (!skip_stream) {
-    stream_cta(a, blockIdx.x - 1, m_in, m_out, s_part);
+    stream_cta<kScalar>(a, blockIdx.x - 1, m_in, m_out, s_part);
   }
 
   __threadfence();

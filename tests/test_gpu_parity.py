@@ -484,6 +484,43 @@ def test_gradient_replacement(sb, oracle_mod, shape):
     gv.close()
 
 
+@pytest.mark.parametrize("k,stride", [(40, 41), (41, 42), (1024, 1025), (264, 264), (523, 530)],
+                         ids=["k40_s41", "k41_s42", "k1024_s1025", "k264_dense", "k523_s530"])
+def test_compressed_signal_layout(sb, oracle_mod, k, stride):
+    """x[:, :, :k] of a [B, T, stride] tensor (the subspace-compressed signal of the SWARM
+    appendix, whose last channel is not verified): rows start on odd 2-byte boundaries and k
+    need not be a multiple of 8.  The oracle sees the packed slice."""
+    B, T = 3, 29
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "compressed", B, T, stride)
+    gv = sb.Verifier(B, T, k)
+    params = oracle_mod.Params(B=B, T=T, d=k)
+    ov = oracle_mod.Verifier(params)
+    buf = torch.full((B, T, 4), -1.0, dtype=torch.float32, device="cuda")
+    gv.sentinel_set_token_stats_buffer(buf)
+    for t in range(14):
+        wide = synth.clean(w, 0, ACT, t, "cuda")
+        if t == 12:
+            wide = (wide.float() * 5).to(torch.bfloat16)
+        wide[:, :, k:] = 1000.0                                # never looked at
+        packed = wide[:, :, :k].contiguous()
+        scale = float(packed.float().abs().mean())
+        if t < 8:
+            gs = torch.empty(1 + B, 3, device="cuda")
+            gv.sentinel_update_reference_strided(wide, ACT, gs)
+            os_, _ = ov.update_reference(synth.bits(packed), ACT)
+        else:
+            gs = torch.empty(1 + B, 3, device="cuda")
+            gf = torch.empty(1 + B, dtype=torch.int32, device="cuda")
+            gv.sentinel_verify_strided(wide, ACT, gs, gf)
+            os_, of, _ = ov.verify(synth.bits(packed), ACT)
+            assert np.array_equal(gf.cpu().numpy().view(np.uint32), of), t
+        assert_scores_close(gs.cpu().numpy(), os_, scale, "compressed step %d" % t)
+        xv = oracle_mod.bf16_to_f64(synth.bits(packed))
+        assert np.allclose(buf.cpu().numpy()[..., 0], xv.sum(-1), rtol=1e-3, atol=1e-3 * np.sqrt(k))
+    compare_state(gv, ov, params)
+    gv.close()
+
+
 def test_runs_are_bit_reproducible(sb):
     w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_rep", 4, 50, 1024)
     blobs, outs = [], []
@@ -519,9 +556,19 @@ def test_verify_host_matches_device_call(sb):
 
 
 def test_argument_errors_never_reach_the_gpu(sb):
+    odd = sb.Verifier(2, 4, 12)                           # d % 8 != 0: strided entry points only
+    xo = torch.zeros(2, 4, 12, dtype=torch.bfloat16, device="cuda")
+    so, fo = torch.zeros(3, 3, device="cuda"), torch.zeros(3, dtype=torch.int32, device="cuda")
     with pytest.raises(sb.SentinelError) as e:
-        sb.Verifier(2, 4, 12)
+        odd.sentinel_verify(xo, 0, so, fo)
     assert e.value.code == sb.ERR_UNALIGNED
+    odd.sentinel_verify_strided(xo, 0, so, fo)
+    Lo, st_ = sb.lib(), torch.cuda.current_stream().cuda_stream
+    assert Lo.sentinel_verify_strided(odd._h, xo.data_ptr(), 0, 2, 4, 12, 11, st_, so.data_ptr(), fo.data_ptr()) == sb.ERR_INVALID_ARG
+    assert Lo.sentinel_verify_strided(odd._h, xo.data_ptr() + 1, 0, 2, 4, 12, 12, st_, so.data_ptr(), fo.data_ptr()) == sb.ERR_UNALIGNED
+    assert Lo.sentinel_verify_strided(odd._h, xo.data_ptr(), 0, 2, 4, 16, 16, st_, so.data_ptr(), fo.data_ptr()) == sb.ERR_SHAPE_MISMATCH
+    torch.cuda.synchronize()
+    odd.close()
     with pytest.raises(sb.SentinelError) as e:
         sb.Verifier(65, 4, 8)
     assert e.value.code == sb.ERR_UNSUPPORTED

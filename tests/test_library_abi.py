@@ -73,10 +73,12 @@ def test_host_side_argument_checks_need_no_gpu(built):
     assert L.sentinel_destroy(None) == binding.ERR_INVALID_ARG
     assert L.sentinel_state_bytes(None) == 0
     assert b"NULL" in L.sentinel_last_error(None)
-    cfg = binding.sentinel_default_config(B=2, T=4, d=12)
+    cfg = binding.sentinel_default_config(B=65, T=4, d=16)
     h = ctypes.c_void_p()
-    assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_UNALIGNED
+    assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_UNSUPPORTED
     assert not h.value
+    cfg = binding.sentinel_default_config(B=2, T=0, d=16)
+    assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_INVALID_ARG
 
 
 def test_product_path_does_not_touch_the_oracle():
