@@ -27,13 +27,13 @@ _LIB = os.path.join(_HERE, "libsentinel_oracle.so")
 
 ACT, GRAD = 0, 1
 L1, L2Z, SFR = 0, 1, 2
-NMETRIC, NSTAT, NTHR = 3, 8, 6
+NMETRIC, NSTAT, NTHR = 4, 8, 6   # room for four metrics; a verifier uses three until directions are set
 
-FLAG_L1, FLAG_L2Z, FLAG_SFR = 1 << 0, 1 << 1, 1 << 2
+FLAG_L1, FLAG_L2Z, FLAG_SFR, FLAG_SW = 1 << 0, 1 << 1, 1 << 2, 1 << 3
 FLAG_NONFINITE = 1 << 7
 FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
 FLAG_NATURAL_SHIFT = 1 << 20
-METRIC_BITS = FLAG_L1 | FLAG_L2Z | FLAG_SFR
+METRIC_BITS = FLAG_L1 | FLAG_L2Z | FLAG_SFR | FLAG_SW
 
 
 def build(force: bool = False) -> str:
@@ -83,6 +83,8 @@ def lib():
         L.so_create.argtypes = [C.POINTER(_Params)]
         L.so_create.restype = C.c_void_p
         L.so_destroy.argtypes = [C.c_void_p]
+        L.so_set_directions.argtypes = [C.c_void_p, u16p, C.c_int]
+        L.so_set_directions.restype = C.c_int
         L.so_destroy.restype = None
         L.so_update_reference.argtypes = [C.c_void_p, u16p, C.c_int, dp]
         L.so_update_reference.restype = C.c_int
@@ -161,7 +163,7 @@ class Params:
     l: int = 100
     c: int = 5
     t_forgiveness: int = 100
-    metric_mask: int = 7
+    metric_mask: int = 15
     R: int = 1
 
     def to_c(self) -> _Params:
@@ -193,7 +195,7 @@ def distance(x_bits, m) -> tuple[np.ndarray, np.ndarray, bool]:
     xb = _bits(x_bits).reshape(-1)
     mm = np.ascontiguousarray(m, dtype=np.float64).reshape(-1)
     assert xb.size == mm.size and xb.size > 0
-    g = np.empty(NMETRIC)
+    g = np.empty(3)
     s = np.empty(NSTAT)
     nf = lib().so_distance(_u16ptr(xb), _dptr(mm), xb.size, _dptr(g), _dptr(s))
     return g, s, bool(nf)
@@ -247,6 +249,7 @@ class Verifier:
         self.rows = 1 + params.B
         self.R = params.R
         self.N = params.B * params.T * params.d
+        self.nm = 3   # metrics in use: the columns of every score array returned below
 
     def close(self):
         if self._h:
@@ -259,12 +262,21 @@ class Verifier:
         except Exception:
             pass
 
+    def set_directions(self, u_bits) -> None:
+        """Sec. 3.1: switch the sliced Wasserstein metric on with the caller's directions
+        (bf16 bit patterns, [L, d]); only before the first step."""
+        ub = _bits(u_bits)
+        assert ub.ndim == 2 and ub.shape[1] == self.d
+        if lib().so_set_directions(self._h, _u16ptr(ub.reshape(-1)), ub.shape[0]) != 0:
+            raise RuntimeError("so_set_directions refused (steps already taken?)")
+        self.nm = NMETRIC
+
     def update_reference(self, x_bits, kind: int):
         xb = _bits(x_bits).reshape(-1)
         assert xb.size == self.N
         scores = np.empty((self.rows, NMETRIC))
         bad = lib().so_update_reference(self._h, _u16ptr(xb), kind, _dptr(scores))
-        return scores, bool(bad)
+        return scores[:, :self.nm].copy(), bool(bad)
 
     def verify(self, x_bits, kind: int):
         xb = _bits(x_bits).reshape(-1)
@@ -273,7 +285,7 @@ class Verifier:
         flags = np.zeros(self.rows, dtype=np.uint32)
         commit = lib().so_verify(self._h, _u16ptr(xb), kind, _dptr(scores),
                                  flags.ctypes.data_as(C.POINTER(C.c_uint32)))
-        return scores, flags, bool(commit)
+        return scores[:, :self.nm].copy(), flags, bool(commit)
 
     def replace_if_flagged(self, x_bits, kind: int, fill: int = 0):
         """Alg. 4 on a copy of x: (new bit patterns, replaced?)."""
@@ -283,7 +295,7 @@ class Verifier:
         return xb.reshape(self.B, self.T, self.d), bool(did)
 
     def step_replicas(self, xs_bits, kind: int, warmup: bool = False):
-        """One iteration with all R workers' tensors: (scores [R,1+B,3], flags [R,1+B], number of
+        """One iteration with all R workers' tensors: (scores [R,1+B,M], flags [R,1+B], number of
         submissions that entered the EMA)."""
         assert len(xs_bits) == self.R
         keep = [_bits(x).reshape(-1) for x in xs_bits]
@@ -293,7 +305,7 @@ class Verifier:
         flags = np.zeros((self.R, self.rows), dtype=np.uint32)
         n = lib().so_step_replicas(self._h, ptrs, kind, int(warmup), _dptr(scores),
                                    flags.ctypes.data_as(C.POINTER(C.c_uint32)))
-        return scores, flags, int(n)
+        return scores[:, :, :self.nm].copy(), flags, int(n)
 
     def worker_counters(self, r: int) -> tuple[int, int, int]:
         out = (C.c_int * 3)()
@@ -319,11 +331,11 @@ class Verifier:
         return out[:n].copy()
 
     def thresholds(self, kind: int):
-        """(thr[2][3][6], valid[2][3]) -- q1 q2 q3 k tau_lower tau_upper."""
-        thr = np.zeros((2, NMETRIC, NTHR))
-        valid = np.zeros((2, NMETRIC), dtype=bool)
+        """(thr[2][M][6], valid[2][M]) -- q1 q2 q3 k tau_lower tau_upper; M metrics in use."""
+        thr = np.zeros((2, self.nm, NTHR))
+        valid = np.zeros((2, self.nm), dtype=bool)
         for L in range(2):
-            for i in range(NMETRIC):
+            for i in range(self.nm):
                 t = np.zeros(NTHR)
                 valid[L, i] = bool(lib().so_thresholds(self._h, kind, L, i, _dptr(t)))
                 thr[L, i] = t

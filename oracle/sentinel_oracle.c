@@ -59,7 +59,7 @@ void so_default_params(so_params *p) {
   p->l = 100;                    /* Sec. 5: window of the past 100 steps            */
   p->c = 5;                      /* Sec. 3.1                                        */
   p->t_forgiveness = 100;        /* Sec. 3.1                                        */
-  p->metric_mask = 7u;
+  p->metric_mask = 15u;
   p->B = 1; p->T = 1; p->d = 8;
   p->R = 1;
 }
@@ -74,7 +74,7 @@ int so_distance(const uint16_t *x, const double *m, size_t n, double gamma[3], d
   for (e = 0; e < n; ++e) {
     if (!isfinite(so_bf16(x[e]))) {
       int i;
-      for (i = 0; i < SO_NMETRIC; ++i) gamma[i] = NAN;
+      for (i = 0; i < 3; ++i) gamma[i] = NAN;
       for (i = 0; i < SO_NSTAT; ++i) stat[i] = NAN;
       return 1;
     }
@@ -262,6 +262,9 @@ struct so_verifier {
   size_t N, Ns;
   so_kind_state ks[2];
   int violations[SO_MAX_WORKERS], clean_streak[SO_MAX_WORKERS], banned[SO_MAX_WORKERS];
+  uint16_t *u;   /* directions of the sliced Wasserstein metric, bf16 [n_dir][d]; NULL = metric off */
+  int n_dir;
+  int nm;        /* metrics in use: 3, or 4 once directions are set */
 };
 
 static void window_push(so_window *w, double val) {
@@ -278,6 +281,7 @@ so_verifier *so_create(const so_params *p) {
   v->p = *p;
   v->Ns = (size_t)p->T * (size_t)p->d;
   v->N = v->Ns * (size_t)p->B;
+  v->u = NULL; v->n_dir = 0; v->nm = 3;
   for (int kind = 0; kind < 2; ++kind) {
     so_kind_state *ks = &v->ks[kind];
     ks->m = (double *)calloc(v->N, sizeof(double));
@@ -296,6 +300,17 @@ so_verifier *so_create(const so_params *p) {
   return v;
 }
 
+int so_set_directions(so_verifier *v, const uint16_t *u, int n_dir) {
+  if (n_dir < 1 || !u) return -1;
+  if (v->ks[0].steps || v->ks[1].steps) return -1;   /* the metric set is fixed before the first step */
+  free(v->u);
+  v->u = (uint16_t *)malloc((size_t)n_dir * (size_t)v->p.d * sizeof(uint16_t));
+  memcpy(v->u, u, (size_t)n_dir * (size_t)v->p.d * sizeof(uint16_t));
+  v->n_dir = n_dir;
+  v->nm = SO_NMETRIC;
+  return 0;
+}
+
 void so_destroy(so_verifier *v) {
   if (!v) return;
   for (int kind = 0; kind < 2; ++kind) {
@@ -304,6 +319,7 @@ void so_destroy(so_verifier *v) {
     for (int L = 0; L < 2; ++L)
       for (int i = 0; i < SO_NMETRIC; ++i) free(v->ks[kind].hist[L][i].v);
   }
+  free(v->u);
   free(v);
 }
 
@@ -311,18 +327,23 @@ void so_destroy(so_verifier *v) {
  * row 1+b = sample b.  Returns a bit per row set when that row holds non-finite input. */
 static void all_units(so_verifier *v, const uint16_t *x, int kind, double *gam, int *nonfinite) {
   so_kind_state *ks = &v->ks[kind];
-  nonfinite[0] = so_distance(x, ks->m, v->N, gam, ks->stats);
-  for (int b = 0; b < v->p.B; ++b)
-    nonfinite[1 + b] = so_distance(x + (size_t)b * v->Ns, ks->m + (size_t)b * v->Ns, v->Ns,
-                                   gam + (size_t)(1 + b) * SO_NMETRIC,
-                                   ks->stats + (size_t)(1 + b) * SO_NSTAT);
+  const size_t d = (size_t)v->p.d;
+  for (int r = 0; r <= v->p.B; ++r) {
+    /* unit r: the whole tensor (B*T tokens) or sample r-1 (T tokens) */
+    const size_t off = (r == 0) ? 0 : (size_t)(r - 1) * v->Ns;
+    const size_t n = (r == 0) ? v->N : v->Ns;
+    double *g = gam + (size_t)r * SO_NMETRIC;
+    nonfinite[r] = so_distance(x + off, ks->m + off, n, g, ks->stats + (size_t)r * SO_NSTAT);
+    g[SO_SW] = v->u ? so_sliced_wasserstein(x + off, ks->m + off, n / d, d, v->u, (size_t)v->n_dir, NULL)
+                    : NAN;
+  }
 }
 
 static void refresh_thresholds(so_verifier *v, int kind) {
   so_kind_state *ks = &v->ks[kind];
   const so_params *p = &v->p;
   for (int L = 0; L < 2; ++L)
-    for (int i = 0; i < SO_NMETRIC; ++i) {
+    for (int i = 0; i < v->nm; ++i) {
       so_window *w = &ks->hist[L][i];
       if (so_adaptive_iqr(w->v, w->n, p->alpha[kind], p->n_max[kind], p->gamma_g[kind],
                           p->gamma_s[kind], p->lambda[kind], p->eps[kind], p->shrink_ratio,
@@ -365,9 +386,9 @@ int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *sco
   const int bad = nf[0];
   if (!bad) {
     /* warm-up: every deviation joins the history, then thresholds, then the EMA */
-    for (int i = 0; i < SO_NMETRIC; ++i) window_push(&ks->hist[0][i], gam[i]);
+    for (int i = 0; i < v->nm; ++i) window_push(&ks->hist[0][i], gam[i]);
     for (int b = 0; b < v->p.B; ++b)
-      for (int i = 0; i < SO_NMETRIC; ++i)
+      for (int i = 0; i < v->nm; ++i)
         window_push(&ks->hist[1][i], gam[(size_t)(1 + b) * SO_NMETRIC + i]);
     refresh_thresholds(v, kind);
     ema_update(v, x, kind);
@@ -396,7 +417,7 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
     if (nf[r]) {
       f |= SO_FLAG_NONFINITE;
     } else {
-      for (int i = 0; i < SO_NMETRIC; ++i) {
+      for (int i = 0; i < v->nm; ++i) {
         if (!ks->has_thr[L][i]) { no_thr = 1; continue; }
         if (!((p->metric_mask >> i) & 1u)) continue;
         const double *t = ks->thr[L][i];
@@ -417,7 +438,7 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
   for (int r = 0; r < rows; ++r) {
     if (flags[r]) continue;
     const int L = (r == 0) ? 0 : 1;
-    for (int i = 0; i < SO_NMETRIC; ++i)
+    for (int i = 0; i < v->nm; ++i)
       window_push(&ks->hist[L][i], gam[(size_t)r * SO_NMETRIC + i]);
   }
   refresh_thresholds(v, kind);
@@ -469,7 +490,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
       if (nf[u]) {
         f |= SO_FLAG_NONFINITE;
       } else if (!warmup) {
-        for (int i = 0; i < SO_NMETRIC; ++i) {
+        for (int i = 0; i < v->nm; ++i) {
           if (!ks->has_thr[L][i]) { no_thr = 1; continue; }
           if (!((p->metric_mask >> i) & 1u)) continue;
           const double *t = ks->thr[L][i];
@@ -489,7 +510,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
       for (int u = 0; u < rows; ++u) {
         if (fl[u]) continue;
         const int L = (u == 0) ? 0 : 1;
-        for (int i = 0; i < SO_NMETRIC; ++i)
+        for (int i = 0; i < v->nm; ++i)
           window_push(&ks->hist[L][i], gam[(size_t)u * SO_NMETRIC + i]);
       }
   }

@@ -30,14 +30,14 @@ extern "C" {
 #endif
 
 enum { SO_ACT = 0, SO_GRAD = 1 };                 /* h (forward) or g (backward)           */
-enum { SO_L1 = 0, SO_L2Z = 1, SO_SFR = 2, SO_NMETRIC = 3 };
+enum { SO_L1 = 0, SO_L2Z = 1, SO_SFR = 2, SO_SW = 3, SO_NMETRIC = 4 };
 enum { SO_NSTAT = 8 };                            /* mean_x var_x |x|_2 mean_m var_m cov |m|_2 rho */
 enum { SO_MAX_WORKERS = 16 };
 enum { SO_NTHR = 6 };                             /* q1 q2 q3 k tau_lower tau_upper        */
 
 /* report bits, one word per unit (row 0 = whole tensor, rows 1..B = samples) */
 enum {
-  SO_FLAG_L1 = 1u << 0, SO_FLAG_L2Z = 1u << 1, SO_FLAG_SFR = 1u << 2,
+  SO_FLAG_L1 = 1u << 0, SO_FLAG_L2Z = 1u << 1, SO_FLAG_SFR = 1u << 2, SO_FLAG_SW = 1u << 3,
   SO_FLAG_NONFINITE = 1u << 7,
   SO_FLAG_COMMITTED = 1u << 16, SO_FLAG_SEVERE = 1u << 17,
   SO_FLAG_BANNED = 1u << 18, SO_FLAG_NO_THRESHOLDS = 1u << 19,
@@ -90,14 +90,22 @@ int so_adaptive_iqr(const double *window, size_t n, double alpha, int n_max, dou
                     double thr[6], int iters[2]);
 
 so_verifier *so_create(const so_params *p);
+
+/* Sec. 3.1: adds the sliced Wasserstein distance to the metric set M of this verifier.  u: the
+ * caller's n_dir unit directions as bf16 bit patterns, [n_dir][d] (copied).  From then on every
+ * unit's fourth score is so_sliced_wasserstein of the unit (B*T tokens for the whole tensor,
+ * T tokens for a sample) against the EMA, with its own history and thresholds like the other
+ * metrics; without directions the fourth score is NaN and takes no part.  Only before the
+ * first step; returns 0, or -1 if refused. */
+int so_set_directions(so_verifier *v, const uint16_t *u, int n_dir);
 void so_destroy(so_verifier *v);
 
 /* Warm-up step (Alg. 1, warm-up loop): scores against the current EMA, every unit appended
- * to the history, thresholds refreshed, EMA updated.  scores: (1+B)*3 doubles or NULL.
+ * to the history, thresholds refreshed, EMA updated.  scores: (1+B)*4 doubles or NULL.
  * Returns 0, or 1 if the input was non-finite (then nothing changes). */
 int so_update_reference(so_verifier *v, const uint16_t *x, int kind, double *scores);
 
-/* Verified step (body of Alg. 2 / Alg. 3 for one submission).  scores: (1+B)*3 doubles,
+/* Verified step (body of Alg. 2 / Alg. 3 for one submission).  scores: (1+B)*4 doubles,
  * flags: (1+B) words.  Returns 1 if the EMA was updated (no unit flagged), else 0. */
 int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint32_t *flags);
 
@@ -130,7 +138,7 @@ int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill)
  * workers were flagged the taint set is cleared (natural distribution shift); the EMA moves
  * with the mean of the submissions that are not tainted.  warmup != 0: the warm-up loop of
  * Alg. 1 instead (no test, no counters, everything joins, mean over all workers).
- * scores: [R][1+B][3]; flags: [R][1+B] (row 0 of each worker carries its status bits).
+ * scores: [R][1+B][4]; flags: [R][1+B] (row 0 of each worker carries its status bits).
  * Returns the number of submissions that entered the EMA. */
 int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int warmup,
                      double *scores, uint32_t *flags);

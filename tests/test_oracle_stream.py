@@ -392,3 +392,94 @@ def test_banned_worker_is_no_longer_collected(oracle_mod, small):
     xs[0] = (xs[0].float() * 6).to(torch.bfloat16)
     _, flags, n = v.step_replicas([synth.bits(x) for x in xs], ACT)
     assert n == 1 and not (flags[0, 0] & oracle_mod.FLAG_NATURAL_SHIFT)
+
+
+# ---------------------------------------------------------------------------------------------
+# the sliced Wasserstein distance as a fourth member of the metric set M (Sec. 3.1)
+
+def _directions(rs, L, d):
+    u = rs.normal(0, 1, (L, d))
+    return to_bits(u / np.linalg.norm(u, axis=1, keepdims=True))
+
+
+def _sw_numpy(x, m, u):
+    """mean over directions of W1 between the projected token clouds, from scipy's 1-D W1."""
+    import scipy.stats
+    return float(np.mean([scipy.stats.wasserstein_distance(x @ ul, m @ ul) for ul in u]))
+
+
+def test_fourth_metric_is_the_sliced_wasserstein_distance_of_every_unit(oracle_mod):
+    """With directions set, column 3 of the scores is SW(unit, m_{t-1}): B*T tokens for the whole
+    tensor, T tokens for a sample; the other three columns are what they were without it."""
+    rs = np.random.default_rng(21)
+    B, T, d, L = 3, 6, 8, 4
+    ub = _directions(rs, L, d)
+    u = from_bits(ub)
+    v, v3 = make(oracle_mod, B=B, T=T, d=d), make(oracle_mod, B=B, T=T, d=d)
+    v.set_directions(ub)
+    for t in range(6):
+        xb = to_bits(rs.normal(0.3, 1, (B, T, d)))
+        m = v.ema(ACT).copy()
+        if t < 4:
+            scores, _ = v.update_reference(xb, ACT)
+            scores3, _ = v3.update_reference(xb, ACT)
+        else:
+            scores, _, _ = v.verify(xb, ACT)
+            scores3, _, _ = v3.verify(xb, ACT)
+        assert scores.shape == (1 + B, 4) and scores3.shape == (1 + B, 3)
+        assert np.array_equal(scores[:, :3], scores3)
+        x = from_bits(xb)
+        assert scores[0, 3] == pytest.approx(_sw_numpy(x.reshape(-1, d), m.reshape(-1, d), u), rel=1e-12)
+        for b in range(B):
+            assert scores[1 + b, 3] == pytest.approx(_sw_numpy(x[b], m[b], u), rel=1e-12)
+
+
+def test_fourth_metric_has_its_own_history_and_thresholds(oracle_mod):
+    rs = np.random.default_rng(22)
+    B, l = 2, 4
+    v = make(oracle_mod, B=B, T=5, d=8, l=l)
+    v.set_directions(_directions(rs, 4, 8))
+    rec = [[], []]
+    k = [1.5, 1.5]
+    for t in range(7):
+        scores, _ = v.update_reference(to_bits(rs.normal(0, 1, (B, 5, 8))), ACT)
+        rec[0].append(scores[0, 3])
+        rec[1].extend(scores[1:, 3])
+        thr, valid = v.thresholds(ACT)
+        assert thr.shape == (2, 4, 6) and valid.all()
+        for L, cap in ((0, l), (1, l * B)):
+            want_hist = np.array(rec[L])[-cap:]
+            assert np.array_equal(v.history(ACT, L, 3), want_hist)
+            want, _ = oracle_mod.adaptive_iqr(want_hist, k[L], 1e-4, 10, 1.1, 0.9, 0.15, 1e-3)
+            assert np.array_equal(thr[L, 3], want)
+            k[L] = want[3]
+
+
+def test_a_shift_seen_only_by_the_sliced_wasserstein_distance_is_flagged(oracle_mod):
+    """A verifier that may flag on SW alone (metric_mask = 8): a submission whose tokens are
+    spread three times as wide along every direction moves SW far outside its window and raises bit 3,
+    nothing else; the EMA stays.  The same verifier without directions sees no metric at all."""
+    rs = np.random.default_rng(23)
+    B, T, d = 2, 32, 16
+    v = make(oracle_mod, B=B, T=T, d=d, metric_mask=8)
+    v.set_directions(_directions(rs, 8, d))
+    base = rs.normal(0, 1, (B, T, d))
+    for t in range(12):
+        v.update_reference(to_bits(base + 0.05 * rs.normal(0, 1, (B, T, d))), ACT)
+    ok, f_ok, commit = v.verify(to_bits(base + 0.05 * rs.normal(0, 1, (B, T, d))), ACT)
+    assert commit and not (f_ok & oracle_mod.METRIC_BITS).any()
+    m0 = v.ema(ACT).copy()
+    scores, flags, commit = v.verify(to_bits(3.0 * base), ACT)
+    assert not commit and np.array_equal(v.ema(ACT), m0)
+    assert np.all(flags & oracle_mod.METRIC_BITS == oracle_mod.FLAG_SW)
+    assert np.all(scores[:, 3] > 5 * ok[:, 3])
+    thr, _ = v.thresholds(ACT)
+    assert np.all(scores[0, 3] > thr[0, 3, 5]) and np.all(scores[1:, 3] > thr[1, 3, 5])
+
+
+def test_directions_are_refused_after_the_first_step(oracle_mod):
+    rs = np.random.default_rng(24)
+    v = make(oracle_mod)
+    v.update_reference(to_bits(rs.normal(0, 1, (2, 4, 8))), GRAD)
+    with pytest.raises(RuntimeError):
+        v.set_directions(_directions(rs, 4, 8))
