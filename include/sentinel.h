@@ -40,7 +40,8 @@
 extern "C" {
 #endif
 
-#define SENTINEL_NUM_METRICS 3
+#define SENTINEL_NUM_METRICS 3     /* L1, z-scored L2, sign-flip ratio: the metrics every verifier uses */
+#define SENTINEL_MAX_METRICS 4     /* ... plus the sliced Wasserstein distance once directions are set  */
 #define SENTINEL_NUM_STATS 8      /* mean_x var_x |x|_2 mean_m var_m cov_xm |m|_2 rho */
 #define SENTINEL_NUM_THRESHOLDS 6 /* q1 q2 q3 k tau_lower tau_upper                   */
 #define SENTINEL_MAX_B 64         /* samples per tensor                               */
@@ -64,6 +65,7 @@ typedef enum sentinel_kind { SENTINEL_ACT = 0, SENTINEL_GRAD = 1 } sentinel_kind
 #define SENTINEL_FLAG_L1 (1u << 0)            /* metric i outside [tau_lower, tau_upper]     */
 #define SENTINEL_FLAG_L2Z (1u << 1)
 #define SENTINEL_FLAG_SFR (1u << 2)
+#define SENTINEL_FLAG_SWD (1u << 3)           /* sliced Wasserstein distance (needs directions) */
 #define SENTINEL_FLAG_NONFINITE (1u << 7)     /* the unit holds a NaN or an infinity         */
 #define SENTINEL_FLAG_COMMITTED (1u << 16)    /* row 0: the reference was updated            */
 #define SENTINEL_FLAG_SEVERE (1u << 17)       /* row 0: deviation >= severe_mult * allowed   */
@@ -87,7 +89,7 @@ typedef struct sentinel_config {
   int    window_steps;     /* history length l, in steps                       100         */
   int    ban_violations;   /* c                                                5           */
   int    forgiveness_steps;/* T_forgiveness                                    100         */
-  unsigned metric_mask;    /* bit i set: metric i may raise a flag             7           */
+  unsigned metric_mask;    /* bit i set: metric i may raise a flag             15          */
   int    B, T, d;          /* shape of every submission; B <= SENTINEL_MAX_B; d % 8 == 0
                               unless only the _strided entry points are used              */
   int    device;           /* CUDA device ordinal                                           */
@@ -110,12 +112,34 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
  *   violation (counter, forgiveness, ban: Sec. 3.1); unflagged units join the history and the
  *   bounds are refreshed; m_t = beta m_{t-1} + (1-beta) x only if nothing was flagged.
  * dev_x          bf16 [B,T,d], 16-byte aligned, read once.
- * dev_scores_out fp32 [(1+B)*3], scores_out[row*3+i] = Gamma_i of that unit (NaN for a
- *                non-finite unit).
+ * dev_scores_out fp32 [(1+B)*M], scores_out[row*M+i] = Gamma_i of that unit (NaN for a
+ *                non-finite unit); M = sentinel_num_metrics(h): 3, or 4 once directions are set.
  * dev_flags_out  u32 [1+B], bits as defined above.
  * x is read exactly once; the library keeps no reference to caller memory afterwards. */
 int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T,
                     int d, void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out);
+
+/* Sec. 3.1: adds the sliced Wasserstein distance to this verifier's metric set.  From the next
+ * step on every unit has a fourth score, SW(unit, m_{t-1}) as sentinel_sliced_wasserstein
+ * defines it (B*T tokens for the whole tensor, T for a sample), with its own history window,
+ * bounds and flag bit (SENTINEL_FLAG_SWD, metric_mask bit 3) like the other three; score
+ * rows, sentinel_get_thresholds and the replica calls then carry M = 4 columns.
+ * dev_u_bf16: bf16 [L, d] unit directions chosen by the caller (the paper fixes neither
+ * their number nor their draw), 16-byte aligned; copied on cuda_stream, and the call waits
+ * for it.  L must be 4, 8 or 16; L*d*2 bytes <= 200 KiB; T <= 16384; d a multiple of 8.
+ * Every later step first runs the projection / sort launches on the caller's stream (they
+ * read x and the reference once more: 6 B/element on top of the streaming pass), then the
+ * streaming launch, which picks the distances up.  The projections are fp32: inputs whose
+ * projections leave the fp32 range give a score that is not a number, which counts as a
+ * flag.  Allowed only before the first step and before sentinel_import_state
+ * (SENTINEL_ERR_INVALID_ARG afterwards); the four windows' working copies must fit the
+ * 200 KiB of shared memory (about window_steps*n_workers*(B+1) <= 3000), else
+ * SENTINEL_ERR_UNSUPPORTED.  The strided entry points refuse a verifier with directions.
+ * The scratch (about 24*L*B*T bytes) belongs to the handle. */
+int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L, void *cuda_stream);
+
+/* Metrics this verifier uses (M above): 3, or 4 after sentinel_set_directions; 0 if h is NULL. */
+int sentinel_num_metrics(const sentinel_verifier *h);
 
 /* Warm-up step (the warm-up loop of Alg. 1, honest workers only): scores as above, every unit
  * joins the history, the bounds are refreshed and the reference is updated unconditionally.
@@ -141,7 +165,7 @@ int sentinel_update_reference_strided(sentinel_verifier *h, const void *dev_x, s
 /* sentinel_verify for callers whose tensor and results live in host memory: copies x to a
  * staging buffer owned by the handle (allocated on first use), runs the check, copies scores
  * and flags back and waits for the stream.  host_x: bf16 [B,T,d] (pinned memory copies
- * fastest); host_scores_out: fp32 [(1+B)*3]; host_flags_out: u32 [1+B]. */
+ * fastest); host_scores_out: fp32 [(1+B)*M]; host_flags_out: u32 [1+B]. */
 int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind kind, int B,
                          int T, int d, void *cuda_stream, float *host_scores_out,
                          unsigned *host_flags_out);
@@ -196,9 +220,9 @@ int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int 
 int sentinel_get_stats(sentinel_verifier *h, sentinel_kind kind, float *dev_stats_out,
                        void *cuda_stream);
 
-/* Current bounds, host_out double [2 levels][3 metrics][6] = q1 q2 q3 k tau_lower tau_upper
- * (level 0 = whole tensor, 1 = samples); host_valid int [2][3] (0 while that history is
- * empty), may be NULL.  Waits for the stream. */
+/* Current bounds, host_out double [2 levels][M metrics][6] = q1 q2 q3 k tau_lower tau_upper
+ * (level 0 = whole tensor, 1 = samples; M = sentinel_num_metrics(h)); host_valid int [2][M]
+ * (0 while that history is empty), may be NULL.  Waits for the stream. */
 int sentinel_get_thresholds(sentinel_verifier *h, sentinel_kind kind, double *host_out,
                             int *host_valid, void *cuda_stream);
 
@@ -226,7 +250,7 @@ int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf);
  * as they moved; the reference then moves with the mean of the untainted submissions (each
  * tensor is read once for its scores and once more for the mean).  A banned worker is not
  * read: its scores are NaN and its row 0 reports SENTINEL_FLAG_BANNED.
- * dev_scores_out fp32 [n_workers][1+B][3]; dev_flags_out u32 [n_workers][1+B]; row 0 of worker
+ * dev_scores_out fp32 [n_workers][1+B][M]; dev_flags_out u32 [n_workers][1+B]; row 0 of worker
  * r carries COMMITTED iff its tensor entered the mean. */
 int sentinel_verify_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind,
                              int B, int T, int d, void *cuda_stream, float *dev_scores_out,
@@ -255,11 +279,14 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
 int sentinel_reset_worker(sentinel_verifier *h, int worker, void *cuda_stream);
 
 /* Checkpointing.  The state is one self-describing blob: a 64-byte header
- * {u64 magic, u32 version = 2, i32 B, T, d, window_steps, n_workers}, then
+ * {u64 magic, u32 version = 3, i32 B, T, d, window_steps, n_workers, n_metrics}, then
  * i32 violations[16], clean_streak[16], banned[16], then per kind {i64 steps; i32 count[2];
- * i32 valid[2][3]; f64 thr[2][3][6]; f64 history[level 0: 3][window_steps*n_workers],
- * [level 1: 3][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d]}.
- * Export and import wait for the stream. */
+ * i32 valid[2][4]; f64 thr[2][4][6]; f64 history[level 0: 4][window_steps*n_workers],
+ * [level 1: 4][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d]}.  The
+ * layout always has room for four metrics; with n_metrics = 3 the fourth slots are unused.
+ * A blob goes back only into a verifier with the same n_metrics (the directions themselves
+ * are not part of the state: set them before importing).  Export and import wait for the
+ * stream. */
 size_t sentinel_state_bytes(const sentinel_verifier *h);
 int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *cuda_stream);
 int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, void *cuda_stream);

@@ -15,13 +15,14 @@ from . import _build
 
 ACT, GRAD = 0, 1
 NUM_METRICS, NUM_STATS, NUM_THRESHOLDS = 3, 8, 6
+MAX_METRICS = 4        # with the sliced Wasserstein distance (Verifier.sentinel_set_directions)
 MAX_B, MAX_WINDOW = 64, 4096
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE_MISMATCH, ERR_UNALIGNED, ERR_CUDA = -1, -2, -3, -4
 ERR_STATE_SIZE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -7
 
-FLAG_L1, FLAG_L2Z, FLAG_SFR = 1 << 0, 1 << 1, 1 << 2
+FLAG_L1, FLAG_L2Z, FLAG_SFR, FLAG_SWD = 1 << 0, 1 << 1, 1 << 2, 1 << 3
 FLAG_NONFINITE = 1 << 7
 FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
 FLAG_NATURAL_SHIFT = 1 << 20
@@ -29,6 +30,7 @@ MAX_WORKERS = 16
 
 EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
+    "sentinel_set_directions", "sentinel_num_metrics",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
     "sentinel_verify_replicas", "sentinel_update_reference_replicas", "sentinel_get_worker_counters",
     "sentinel_verify_strided", "sentinel_update_reference_strided",
@@ -78,6 +80,8 @@ def lib():
         L.sentinel_default_config.argtypes = [C.POINTER(sentinel_config)]
         L.sentinel_verifier_create.argtypes = [C.POINTER(sentinel_config), C.POINTER(vp)]
         L.sentinel_verify.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
+        L.sentinel_set_directions.argtypes = [vp, vp, ip, vp]
+        L.sentinel_num_metrics.argtypes = [vp]
         L.sentinel_update_reference.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp]
         L.sentinel_verify_host.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_distance.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
@@ -178,6 +182,17 @@ class Verifier:
         h = C.c_void_p()
         _check(lib().sentinel_verifier_create(C.byref(self.cfg), C.byref(h)))
         self._h = h
+        self.M = NUM_METRICS          # columns of every score array
+
+    def sentinel_set_directions(self, u_bf16: torch.Tensor, stream=None) -> None:
+        """Sec. 3.1: adds the sliced Wasserstein distance along the caller's directions
+        (bf16 [L, d], L in 4/8/16) as a fourth metric; only before the first step."""
+        assert u_bf16.dtype == torch.bfloat16 and u_bf16.is_contiguous() and u_bf16.shape[1] == self.d
+        _check(lib().sentinel_set_directions(self._h, _ptr(u_bf16), u_bf16.shape[0], _stream_ptr(stream)), self._h)
+        self.M = self.sentinel_num_metrics()
+
+    def sentinel_num_metrics(self) -> int:
+        return int(lib().sentinel_num_metrics(self._h))
 
     # -- hot path ---------------------------------------------------------------------------
     def sentinel_verify(self, x: torch.Tensor, kind: int, scores_out: torch.Tensor,
@@ -231,7 +246,7 @@ class Verifier:
                                                         _ptr(flags_out)), self._h)
 
     def step_replicas(self, xs, kind: int, warmup: bool = False, stream=None):
-        scores = torch.empty(self.R, self.rows, NUM_METRICS, dtype=torch.float32, device=xs[0].device)
+        scores = torch.empty(self.R, self.rows, self.M, dtype=torch.float32, device=xs[0].device)
         flags = torch.zeros(self.R, self.rows, dtype=torch.int32, device=xs[0].device)
         if warmup:
             self.sentinel_update_reference_replicas(xs, kind, scores, flags, stream)
@@ -254,13 +269,13 @@ class Verifier:
 
     # convenience wrappers that allocate the outputs (tests, examples)
     def verify(self, x: torch.Tensor, kind: int, stream=None):
-        scores = torch.empty(self.rows, NUM_METRICS, dtype=torch.float32, device=x.device)
+        scores = torch.empty(self.rows, self.M, dtype=torch.float32, device=x.device)
         flags = torch.empty(self.rows, dtype=torch.int32, device=x.device)
         self.sentinel_verify(x, kind, scores, flags, stream)
         return scores, flags
 
     def update_reference(self, x: torch.Tensor, kind: int, stream=None):
-        scores = torch.empty(self.rows, NUM_METRICS, dtype=torch.float32, device=x.device)
+        scores = torch.empty(self.rows, self.M, dtype=torch.float32, device=x.device)
         self.sentinel_update_reference(x, kind, scores, stream)
         return scores
 
@@ -271,11 +286,11 @@ class Verifier:
         return out
 
     def sentinel_get_thresholds(self, kind: int, stream=None):
-        thr = (C.c_double * (2 * NUM_METRICS * NUM_THRESHOLDS))()
-        valid = (C.c_int * (2 * NUM_METRICS))()
+        thr = (C.c_double * (2 * self.M * NUM_THRESHOLDS))()
+        valid = (C.c_int * (2 * self.M))()
         _check(lib().sentinel_get_thresholds(self._h, kind, thr, valid, _stream_ptr(stream)), self._h)
-        t = torch.tensor(list(thr), dtype=torch.float64).reshape(2, NUM_METRICS, NUM_THRESHOLDS)
-        v = torch.tensor(list(valid), dtype=torch.bool).reshape(2, NUM_METRICS)
+        t = torch.tensor(list(thr), dtype=torch.float64).reshape(2, self.M, NUM_THRESHOLDS)
+        v = torch.tensor(list(valid), dtype=torch.bool).reshape(2, self.M)
         return t.numpy(), v.numpy()
 
     def sentinel_get_counters(self, stream=None) -> dict:

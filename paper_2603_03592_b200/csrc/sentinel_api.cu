@@ -20,13 +20,13 @@ namespace {
 thread_local std::string g_error;   // failures of calls that have no handle
 
 constexpr unsigned long long kMagic = 0x4c454e49544e4553ull;  // "SENTINEL", little endian
-constexpr unsigned kVersion = 2;
+constexpr unsigned kVersion = 3;
 constexpr size_t kHeaderBytes = 64;
 
 struct BlobHeader {
   unsigned long long magic;
   unsigned version;
-  int B, T, d, window_steps, n_workers;
+  int B, T, d, window_steps, n_workers, n_metrics;
 };
 
 struct BlobWorkers {      // follows the header
@@ -40,7 +40,7 @@ struct BlobKindHead {
   int valid[2][kNumMetrics];
   double thr[2][kNumMetrics][kNumThr];
 };
-static_assert(sizeof(BlobKindHead) == 8 + 8 + 24 + 288, "packed layout expected");
+static_assert(sizeof(BlobKindHead) == 8 + 8 + 32 + 384, "packed layout expected");
 
 }  // namespace
 
@@ -51,6 +51,12 @@ struct sentinel_verifier {
   int R = 1, units0 = 1, units1 = 1; // workers; entries one iteration can append per level
   int G = 1;                        // streaming CTAs; launches use G + 1
   size_t refresh_smem = 0;          // dynamic shared memory of a launch that may refresh thresholds
+  int n_metrics = 3;                // metrics in use; 4 once directions are set
+  bool started = false;             // a step was taken or a state imported: the metric set is fixed
+  int sw_L = 0;                     // number of directions
+  uint16_t *sw_u = nullptr;         // directions, bf16 [sw_L][d]
+  float *sw_scratch = nullptr;      // projections and sorted lists
+  float *sw_out = nullptr;          // [1+B] distances of the submission being checked
   float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
   HandleState *hs = nullptr;
   double *hist[2] = {nullptr, nullptr};      // rings, device layout (ring_offset)
@@ -181,6 +187,8 @@ int check_call_strided(sentinel_verifier *h, const void *x, int kind, int B, int
     return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
   if (row_stride < d) return fail(h, SENTINEL_ERR_INVALID_ARG, "row_stride = %lld is smaller than d = %d", row_stride, d);
   if (reinterpret_cast<uintptr_t>(x) & 1u) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 2-byte aligned");
+  if (h->sw_u) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein metric reads dense rows: a verifier with directions takes no strided tensor");
+  h->started = true;
   return SENTINEL_OK;
 }
 
@@ -215,6 +223,8 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.ban_violations = h->cfg.ban_violations;
   a.forgiveness_steps = h->cfg.forgiveness_steps;
   a.metric_mask = h->cfg.metric_mask;
+  a.n_metrics = h->n_metrics;
+  a.sw = h->sw_out;                 // nullptr until directions are set
   return a;
 }
 
@@ -239,8 +249,8 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
 
 int run_refresh(sentinel_verifier *h, cudaStream_t s) {
   refresh_kernel<<<1, kThreads, h->refresh_smem, s>>>(h->hs, h->hist[0], h->hist[1], h->sorted[0], h->sorted[1],
-                                                      h->cap0, h->cap1, h->units0, h->units1, alg5_of(h->cfg, 0),
-                                                      alg5_of(h->cfg, 1));
+                                                      h->cap0, h->cap1, h->units0, h->units1, h->n_metrics,
+                                                      alg5_of(h->cfg, 0), alg5_of(h->cfg, 1));
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
 }
@@ -255,6 +265,88 @@ struct DeviceGuard {   // restores the caller's current device
   ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
+// ---------------------------------------------------------------------------------------------
+// sliced Wasserstein distance: the chain of launches, shared by the stateless entry point and
+// by verifiers that carry it as their fourth metric
+
+template <int L>
+cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
+                              const uint16_t *u, float *proj, long long rows, int d, int sms, cudaStream_t s) {
+  const size_t smem = (size_t)L * d * sizeof(uint16_t);
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, swd_project_kernel<L>, kSwdThreads, smem);
+  if (e != cudaSuccess) return e;
+  if (occ < 1) return cudaErrorInvalidConfiguration;
+  long long grid = (long long)sms * occ;
+  const long long need = (rows + kSwdThreads / 32 - 1) / (kSwdThreads / 32);
+  if (grid > need) grid = need;
+  swd_project_kernel<L><<<(unsigned)grid, kSwdThreads, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d);
+  return cudaGetLastError();
+}
+
+// floats of scratch: the projections and two buffers of sorted lists (2L lists of B*T each),
+// then W1 per (sample, direction) and per direction
+size_t swd_scratch_floats(int L, int B, int T) {
+  return (size_t)3 * 2 * L * ((size_t)B * T) + (size_t)(B + 1) * L;
+}
+
+int check_swd_shape(sentinel_verifier *h, int L, int T, int d) {
+  if (L != 4 && L != 8 && L != 16) return fail(h, SENTINEL_ERR_UNSUPPORTED, "L = %d: the number of directions must be 4, 8 or 16", L);
+  if ((size_t)L * d * sizeof(uint16_t) > 200u * 1024u) return fail(h, SENTINEL_ERR_UNSUPPORTED, "L*d = %d*%d directions do not fit in 200 KiB of shared memory", L, d);
+  if (T > kSwdMaxTokensPerSample) return fail(h, SENTINEL_ERR_UNSUPPORTED, "T = %d exceeds the %d tokens sorted per sample", T, kSwdMaxTokensPerSample);
+  return SENTINEL_OK;
+}
+
+// out[0] = the whole tensor, out[1+b] = sample b.  The reference is m1 if *active != 0, else m0;
+// nothing runs if *skip != 0 (both read on the device; either may be nullptr).
+cudaError_t run_swd(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
+                    const uint16_t *u, int L, int B, int T, int d, int sms, float *scratch, float *out,
+                    cudaStream_t s) {
+  const long long rows = (long long)B * T;
+  const size_t list_floats = (size_t)2 * L * rows;        // L lists for x, L for m
+  float *proj = scratch, *buf_a = proj + list_floats, *buf_b = buf_a + list_floats, *w1_sample = buf_b + list_floats;
+  float *w1_tensor = w1_sample + (size_t)B * L;
+  cudaError_t e;
+  if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, s);
+  else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, s);
+  else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, s);
+  if (e != cudaSuccess) return e;
+  int npad = 1;
+  while (npad < T) npad <<= 1;
+  const size_t smem = (size_t)2 * npad * sizeof(float);
+  e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           2 * kSwdMaxTokensPerSample * (int)sizeof(float));
+  if (e != cudaSuccess) return e;
+  swd_sort_samples_kernel<<<B * L, kSwdSortThreads, smem, s>>>(proj, buf_a, w1_sample, B, T, L, rows, skip);
+  e = cudaGetLastError();
+  float *cur = buf_a, *nxt = buf_b;
+  for (int run = 1; run < B && e == cudaSuccess; run *= 2) {     // merge the samples' sorted lists
+    const long long total = rows * 2 * L;
+    swd_merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(cur, nxt, rows, T, run, 2 * L, skip);
+    e = cudaGetLastError();
+    float *t = cur; cur = nxt; nxt = t;
+  }
+  if (e != cudaSuccess) return e;
+  swd_tensor_w1_kernel<<<L, kSwdSortThreads, 0, s>>>(cur, w1_tensor, rows, L, skip);
+  swd_finish_kernel<<<1, 128, 0, s>>>(w1_tensor, w1_sample, out, B, L, skip);
+  return cudaGetLastError();
+}
+
+// A verifier with directions: the distances of this submission against the reference in force,
+// left in h->sw_out for the streaming launch that follows on the same stream.
+int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bool may_skip, cudaStream_t s) {
+  if (!h->sw_u) return SENTINEL_OK;
+  int sms = 0;
+  SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
+  SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), h->ema[kind][0], h->ema[kind][1], &h->hs->kind[kind].active,
+                           may_skip ? &h->hs->banned[worker] : nullptr, h->sw_u, h->sw_L, h->cfg.B, h->cfg.T,
+                           h->cfg.d, sms, h->sw_scratch, h->sw_out, s));
+  return SENTINEL_OK;
+}
+
+
 void free_all(sentinel_verifier *h) {
   for (int k = 0; k < 2; ++k) {
     for (int j = 0; j < 2; ++j) cudaFree(h->ema[k][j]);
@@ -268,6 +360,9 @@ void free_all(sentinel_verifier *h) {
   cudaFree(h->stage_x);
   cudaFree(h->stage_scores);
   cudaFree(h->stage_flags);
+  cudaFree(h->sw_u);
+  cudaFree(h->sw_scratch);
+  cudaFree(h->sw_out);
 }
 
 }  // namespace
@@ -290,7 +385,7 @@ int sentinel_default_config(sentinel_config *cfg) {
   cfg->window_steps = 100;
   cfg->ban_violations = 5;
   cfg->forgiveness_steps = 100;
-  cfg->metric_mask = 7u;
+  cfg->metric_mask = 15u;
   cfg->n_workers = 1;
   return SENTINEL_OK;
 }
@@ -330,7 +425,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->units1 = h->R * cfg->B;
   h->cap0 = cfg->window_steps * h->units0;
   h->cap1 = cfg->window_steps * h->units1;
-  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1, h->units0, h->units1) * sizeof(double);
+  h->refresh_smem = refresh_smem_doubles(h->cap0, h->cap1, h->units0, h->units1, h->n_metrics) * sizeof(double);
   if (h->refresh_smem > 200u * 1024u) {
     const size_t need = h->refresh_smem;
     delete h;
@@ -385,6 +480,9 @@ int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
   if (!dev_scores_out || !dev_flags_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
+  h->started = true;
+  rc = run_handle_swd(h, dev_x, kind, 0, false, static_cast<cudaStream_t>(cuda_stream));
+  if (rc) return rc;
   return launch(h, make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out), h->G + 1,
                 static_cast<cudaStream_t>(cuda_stream));
 }
@@ -395,6 +493,9 @@ int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_
   if (rc) return rc;
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
+  h->started = true;
+  rc = run_handle_swd(h, dev_x, kind, 0, false, static_cast<cudaStream_t>(cuda_stream));
+  if (rc) return rc;
   return launch(h, make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr), h->G + 1,
                 static_cast<cudaStream_t>(cuda_stream));
 }
@@ -440,9 +541,12 @@ int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind
     SENTINEL_CUDA(h, cudaMalloc((void **)&h->stage_flags, rows * sizeof(unsigned)));
   }
   SENTINEL_CUDA(h, cudaMemcpyAsync(h->stage_x, host_x, h->N * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
-  int rc = launch(h, make_args(h, h->stage_x, kind, kModeVerify, h->stage_scores, h->stage_flags), h->G + 1, s);
+  h->started = true;
+  int rc = run_handle_swd(h, h->stage_x, kind, 0, false, s);
   if (rc) return rc;
-  SENTINEL_CUDA(h, cudaMemcpyAsync(host_scores_out, h->stage_scores, rows * kNumMetrics * sizeof(float), cudaMemcpyDeviceToHost, s));
+  rc = launch(h, make_args(h, h->stage_x, kind, kModeVerify, h->stage_scores, h->stage_flags), h->G + 1, s);
+  if (rc) return rc;
+  SENTINEL_CUDA(h, cudaMemcpyAsync(host_scores_out, h->stage_scores, rows * h->n_metrics * sizeof(float), cudaMemcpyDeviceToHost, s));
   SENTINEL_CUDA(h, cudaMemcpyAsync(host_flags_out, h->stage_flags, rows * sizeof(unsigned), cudaMemcpyDeviceToHost, s));
   SENTINEL_CUDA(h, cudaStreamSynchronize(s));
   return SENTINEL_OK;
@@ -481,6 +585,7 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   a.stats_out = dev_stats_out;
   a.B = B; a.T = T; a.d = d; a.G = G;
   a.x_row_stride = d;
+  a.n_metrics = 3;
   a.mode = kModeDistance;
   stream_kernel_t<false><<<G + 1, kThreads, 0, s>>>(a);
   cudaError_t le = cudaGetLastError();
@@ -507,14 +612,17 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, int B, 
   SENTINEL_CUDA(h, guard.status);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const size_t rows = 1 + (size_t)B;
+  h->started = true;
   if (warmup && flags) SENTINEL_CUDA(h, cudaMemsetAsync(flags, 0, h->R * rows * sizeof(unsigned), s));
   WorkerPointers wp;
   memset(&wp, 0, sizeof wp);
   for (int r = 0; r < h->R; ++r) {                 // every worker against the same m_{t-1}
     StreamArgs a = make_args(h, xs[r], kind, warmup ? kModeReplicaWarmup : kModeReplicaVerify,
-                             scores + r * rows * kNumMetrics, warmup ? nullptr : flags + r * rows);
+                             scores + r * rows * h->n_metrics, warmup ? nullptr : flags + r * rows);
     a.worker = r;
-    int rc = launch(h, a, h->G + 1, s);
+    int rc = run_handle_swd(h, xs[r], kind, r, !warmup, s);
+    if (rc) return rc;
+    rc = launch(h, a, h->G + 1, s);
     if (rc) return rc;
     wp.x[r] = static_cast<const uint16_t *>(xs[r]);
   }
@@ -566,30 +674,41 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
   return SENTINEL_OK;
 }
 
-}  // extern "C"
-
-namespace {
-
-template <int L>
-cudaError_t launch_projection(const uint16_t *x, const float *m, const uint16_t *u, float *proj, long long rows,
-                              int d, int sms, cudaStream_t s) {
-  const size_t smem = (size_t)L * d * sizeof(uint16_t);
-  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  if (e != cudaSuccess) return e;
-  int occ = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, swd_project_kernel<L>, kSwdThreads, smem);
-  if (e != cudaSuccess) return e;
-  if (occ < 1) return cudaErrorInvalidConfiguration;
-  long long grid = (long long)sms * occ;
-  const long long need = (rows + kSwdThreads / 32 - 1) / (kSwdThreads / 32);
-  if (grid > need) grid = need;
-  swd_project_kernel<L><<<(unsigned)grid, kSwdThreads, smem, s>>>(x, m, u, proj, rows, d);
-  return cudaGetLastError();
+int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (!dev_u_bf16) return fail(h, SENTINEL_ERR_INVALID_ARG, "u is NULL");
+  if (h->started) return fail(h, SENTINEL_ERR_INVALID_ARG, "the metric set is fixed once a step was taken or a state imported");
+  if (h->cfg.d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", h->cfg.d);
+  int rc = check_swd_shape(h, L, h->cfg.T, h->cfg.d);
+  if (rc) return rc;
+  const size_t smem = refresh_smem_doubles(h->cap0, h->cap1, h->units0, h->units1, kNumMetrics) * sizeof(double);
+  if (smem > 200u * 1024u)
+    return fail(h, SENTINEL_ERR_UNSUPPORTED, "with four metrics the windows' working copies need %zu bytes of shared memory, 204800 are available", smem);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t u_bytes = (size_t)L * h->cfg.d * sizeof(uint16_t);
+  uint16_t *u = nullptr;
+  float *scratch = nullptr, *out = nullptr;
+  cudaError_t e = cudaMalloc((void **)&u, u_bytes);
+  if (e == cudaSuccess) e = cudaMalloc((void **)&scratch, swd_scratch_floats(L, h->cfg.B, h->cfg.T) * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc((void **)&out, (size_t)(1 + h->cfg.B) * sizeof(float));
+  if (e == cudaSuccess) e = cudaMemcpyAsync(u, dev_u_bf16, u_bytes, cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(out, 0, (size_t)(1 + h->cfg.B) * sizeof(float), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) {
+    cudaFree(u); cudaFree(scratch); cudaFree(out);
+    return fail(h, SENTINEL_ERR_CUDA, "setting the directions failed: %s", cudaGetErrorString(e));
+  }
+  cudaFree(h->sw_u); cudaFree(h->sw_scratch); cudaFree(h->sw_out);   // directions set twice before the first step
+  h->sw_u = u; h->sw_scratch = scratch; h->sw_out = out;
+  h->sw_L = L;
+  h->n_metrics = kNumMetrics;
+  h->refresh_smem = smem;
+  return SENTINEL_OK;
 }
 
-}  // namespace
-
-extern "C" {
+int sentinel_num_metrics(const sentinel_verifier *h) { return h ? h->n_metrics : 0; }
 
 int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const void *dev_u_bf16, int L, int B,
                                 int T, int d, int device, void *cuda_stream, float *dev_sw_out) {
@@ -597,9 +716,8 @@ int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const voi
   int rc = check_shape(nullptr, B, T, d);
   if (rc) return rc;
   if (!aligned16(dev_x) || !aligned16(dev_m) || !aligned16(dev_u_bf16)) return fail(nullptr, SENTINEL_ERR_UNALIGNED, "x, m or u is not 16-byte aligned");
-  if (L != 4 && L != 8 && L != 16) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "L = %d: the number of directions must be 4, 8 or 16", L);
-  if ((size_t)L * d * sizeof(uint16_t) > 200u * 1024u) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "L*d = %d*%d directions do not fit in 200 KiB of shared memory", L, d);
-  if (T > kSwdMaxTokensPerSample) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "T = %d exceeds the %d tokens sorted per sample", T, kSwdMaxTokensPerSample);
+  rc = check_swd_shape(nullptr, L, T, d);
+  if (rc) return rc;
   int ndev = 0;
   SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
   if (device < 0 || device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist", device);
@@ -609,42 +727,11 @@ int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const voi
   int sms = 0;
   SENTINEL_CUDA(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
 
-  const long long rows = (long long)B * T;
-  const size_t list_floats = (size_t)2 * L * rows;        // L lists for x, L for m
   float *scratch = nullptr;
   keep_pool_warm(device);
-  SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, (3 * list_floats + (size_t)(B + 1) * L) * sizeof(float), s));
-  float *proj = scratch, *buf_a = proj + list_floats, *buf_b = buf_a + list_floats, *w1_sample = buf_b + list_floats;
-  float *w1_tensor = w1_sample + (size_t)B * L;
-
-  const uint16_t *x = static_cast<const uint16_t *>(dev_x), *u = static_cast<const uint16_t *>(dev_u_bf16);
-  cudaError_t e;
-  if (L == 4) e = launch_projection<4>(x, dev_m, u, proj, rows, d, sms, s);
-  else if (L == 8) e = launch_projection<8>(x, dev_m, u, proj, rows, d, sms, s);
-  else e = launch_projection<16>(x, dev_m, u, proj, rows, d, sms, s);
-  if (e == cudaSuccess) {
-    int npad = 1;
-    while (npad < T) npad <<= 1;
-    const size_t smem = (size_t)2 * npad * sizeof(float);
-    e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             2 * kSwdMaxTokensPerSample * (int)sizeof(float));
-    if (e == cudaSuccess) {
-      swd_sort_samples_kernel<<<B * L, kSwdSortThreads, smem, s>>>(proj, buf_a, w1_sample, B, T, L, rows);
-      e = cudaGetLastError();
-    }
-  }
-  float *cur = buf_a, *nxt = buf_b;
-  for (int run = 1; run < B && e == cudaSuccess; run *= 2) {     // merge the samples' sorted lists
-    const long long total = rows * 2 * L;
-    swd_merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(cur, nxt, rows, T, run, 2 * L);
-    e = cudaGetLastError();
-    float *t = cur; cur = nxt; nxt = t;
-  }
-  if (e == cudaSuccess) {
-    swd_tensor_w1_kernel<<<L, kSwdSortThreads, 0, s>>>(cur, w1_tensor, rows, L);
-    swd_finish_kernel<<<1, 128, 0, s>>>(w1_tensor, w1_sample, dev_sw_out, B, L);
-    e = cudaGetLastError();
-  }
+  SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, swd_scratch_floats(L, B, T) * sizeof(float), s));
+  cudaError_t e = run_swd(static_cast<const uint16_t *>(dev_x), dev_m, nullptr, nullptr, nullptr,
+                          static_cast<const uint16_t *>(dev_u_bf16), L, B, T, d, sms, scratch, dev_sw_out, s);
   cudaError_t fe = cudaFreeAsync(scratch, s);
   SENTINEL_CUDA(nullptr, e);
   SENTINEL_CUDA(nullptr, fe);
@@ -674,8 +761,11 @@ int sentinel_get_thresholds(sentinel_verifier *h, sentinel_kind kind, double *ho
   HandleState snap;
   SENTINEL_CUDA(h, cudaMemcpyAsync(&snap, h->hs, sizeof snap, cudaMemcpyDeviceToHost, s));
   SENTINEL_CUDA(h, cudaStreamSynchronize(s));
-  memcpy(host_out, snap.kind[kind].thr, sizeof snap.kind[kind].thr);
-  if (host_valid) memcpy(host_valid, snap.kind[kind].has_thr, sizeof snap.kind[kind].has_thr);
+  for (int L = 0; L < 2; ++L)                     // packed to the metrics in use
+    for (int i = 0; i < h->n_metrics; ++i) {
+      memcpy(host_out + ((size_t)L * h->n_metrics + i) * kNumThr, snap.kind[kind].thr[L][i], kNumThr * sizeof(double));
+      if (host_valid) host_valid[L * h->n_metrics + i] = snap.kind[kind].has_thr[L][i];
+    }
   return SENTINEL_OK;
 }
 
@@ -756,7 +846,7 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
 
   unsigned char *out = static_cast<unsigned char *>(host_buf);
   memset(out, 0, kHeaderBytes);
-  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R};
+  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics};
   memcpy(out, &hd, sizeof hd);
   out += kHeaderBytes;
   BlobWorkers bw;
@@ -807,6 +897,8 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
     return fail(h, SENTINEL_ERR_STATE_SIZE, "not a sentinel state blob of version %u", kVersion);
   if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps || hd.n_workers != h->R)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d, %d workers", hd.B, hd.T, hd.d, hd.window_steps, hd.n_workers);
+  if (hd.n_metrics != h->n_metrics)
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob holds %d metrics, this verifier uses %d (set the directions before importing)", hd.n_metrics, h->n_metrics);
   // validate both kinds before touching the device
   const unsigned char *p = in + kHeaderBytes + sizeof(BlobWorkers);
   for (int k = 0; k < 2; ++k) {
@@ -820,6 +912,7 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
   SENTINEL_CUDA(h, guard.status);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
 
+  h->started = true;
   HandleState st;
   memset(&st, 0, sizeof st);
   BlobWorkers bw;
@@ -941,6 +1034,7 @@ int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int 
   a.stats_out = dev_stats_out;
   a.B = B; a.T = T; a.d = d; a.G = G;
   a.x_row_stride = d;
+  a.n_metrics = 3;
   a.mode = kModeDistance;
   stream_kernel_t<false><<<G + 1, kThreads, 0, s>>>(a);
   SENTINEL_CUDA(nullptr, cudaGetLastError());

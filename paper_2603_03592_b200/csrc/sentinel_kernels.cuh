@@ -15,7 +15,8 @@
 
 namespace sentinel {
 
-constexpr int kNumMetrics = 3;
+constexpr int kNumMetrics = 4;          // room for L1, z-scored L2, sign flips and the sliced Wasserstein
+                                        // distance; a launch uses the first n_metrics (3 or 4) of them
 constexpr int kNumStats = 8;
 constexpr int kNumThr = 6;
 constexpr int kMaxB = 64;
@@ -82,11 +83,11 @@ struct StreamArgs {
   const float *m_ext;              // distance mode: caller's reference; else unused
   float *ema[2];                   // the two reference buffers of this kind
   HandleState *hs;                 // nullptr in distance mode
-  double *hist;                    // this kind's rings: level 0 [3][cap0+1], level 1 [3][cap1+B]
-  double *sorted;                  // the same windows kept ascending: [3][cap0], [3][cap1]
+  double *hist;                    // this kind's rings: level 0 [4][cap0+units0], level 1 [4][cap1+units1]
+  double *sorted;                  // the same windows kept ascending: [4][cap0], [4][cap1]
   unsigned long long *partials;    // [G][2][kSlotWords]
   unsigned *ticket;
-  float *scores_out;               // [(1+B)*3] or nullptr
+  float *scores_out;               // [(1+B)*n_metrics] or nullptr
   unsigned *flags_out;             // [1+B] or nullptr
   float *stats_out;                // [(1+B)*8] or nullptr
   float *token_out;                // [B,T,4] or nullptr
@@ -99,7 +100,10 @@ struct StreamArgs {
   int units0, units1;              // entries one iteration can append per level: R and R*B
   int R, worker;                   // workers of the stage; which one this launch scores
   long long x_row_stride;          // elements from one row of x to the next (d when dense)
-  int pad2[2];
+  const float *sw;                 // [1+B] sliced Wasserstein distance of every unit, computed by the
+                                   // launches before this one; nullptr when n_metrics = 3
+  int n_metrics;                   // metrics in use: 3, or 4 with the sliced Wasserstein distance
+  int pad2;
   Alg5Params a5;
   double severe_mult;
   int ban_violations, forgiveness_steps;
@@ -416,12 +420,13 @@ __host__ __device__ inline size_t sorted_offset(int L, int i, int cap0, int cap1
   return L ? (size_t)kNumMetrics * cap0 + (size_t)i * cap1 : (size_t)i * cap0;
 }
 
-constexpr int kGroupThreads = 96;        // three warps work on one (level, metric) window
-constexpr int kRefreshGroups = 2 * kNumMetrics;
-static_assert(kRefreshGroups * kGroupThreads <= kThreads, "one thread group per window");
+// One thread group per (level, metric) window: three warps each with three metrics in use, two
+// with four.
+__host__ __device__ inline int refresh_group_threads(int n_metrics) { return (kThreads / (2 * n_metrics)) & ~31; }
+static_assert(2 * kNumMetrics * 64 <= kThreads, "one thread group per window");
 
-__device__ __forceinline__ void group_barrier(int group) {   // named barrier 1 + group
-  asm volatile("bar.sync %0, %1;" :: "r"(group + 1), "r"(kGroupThreads) : "memory");
+__device__ __forceinline__ void group_barrier(int group, int group_threads) {   // named barrier 1 + group
+  asm volatile("bar.sync %0, %1;" :: "r"(group + 1), "r"(group_threads) : "memory");
 }
 
 // doubles of shared memory the refresh needs: per window the old and the new ascending copy
@@ -430,8 +435,8 @@ __device__ __forceinline__ void group_barrier(int group) {   // named barrier 1 
 __host__ __device__ inline size_t window_smem_doubles(int cap, int units) {
   return 2 * (size_t)cap + 4 * (size_t)units;
 }
-__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1, int units0, int units1) {
-  return (size_t)kNumMetrics * (window_smem_doubles(cap0, units0) + window_smem_doubles(cap1, units1));
+__host__ __device__ inline size_t refresh_smem_doubles(int cap0, int cap1, int units0, int units1, int n_metrics) {
+  return (size_t)n_metrics * (window_smem_doubles(cap0, units0) + window_smem_doubles(cap1, units1));
 }
 
 __device__ __forceinline__ int lower_bound(const double *a, int n, double v) {   // # entries < v
@@ -470,13 +475,14 @@ __device__ __forceinline__ int warp_count_outside(const double *s, int n, double
 }
 
 // Refreshes q1,q2,q3,k,tau of every (level, metric) window of one kind (Alg. 5).  Whole CTA:
-// the six windows are handled side by side, each by three warps with their own named barrier.
+// the windows are handled side by side, each by a group of warps with its own named barrier.
 __device__ void refresh_thresholds(KindState *ks, const double *hist, double *sorted, int cap0, int cap1,
-                                   int units0, int units1, const Alg5Params &a5, double *s_dyn) {
-  const int group = threadIdx.x / kGroupThreads;
-  const int gt = threadIdx.x - group * kGroupThreads;
-  if (group < kRefreshGroups) {
-    const int L = group / kNumMetrics, i = group - L * kNumMetrics;
+                                   int units0, int units1, int n_metrics, const Alg5Params &a5, double *s_dyn) {
+  const int group_threads = refresh_group_threads(n_metrics);
+  const int group = threadIdx.x / group_threads;
+  const int gt = threadIdx.x - group * group_threads;
+  if (group < 2 * n_metrics) {
+    const int L = group / n_metrics, i = group - L * n_metrics;
     const int n = ks->hist_count[L];
     if (n > 0) {                                   // an empty window leaves everything as it is
       const int cap = L ? cap1 : cap0, units = L ? units1 : units0, size = ring_size(cap, units);
@@ -485,18 +491,18 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, double *so
       const double *ring = hist + ring_offset(L, i, cap0, cap1, units0, units1);
       double *srt = sorted + sorted_offset(L, i, cap0, cap1);
       // this window's shared memory: old copy, new copy, staging, what left, what joined
-      double *s_old = s_dyn + (L ? (size_t)kNumMetrics * window_smem_doubles(cap0, units0) +
+      double *s_old = s_dyn + (L ? (size_t)n_metrics * window_smem_doubles(cap0, units0) +
                                        (size_t)i * window_smem_doubles(cap1, units1)
                                  : (size_t)i * window_smem_doubles(cap0, units0));
       double *s_new = s_old + cap, *s_stage = s_new + cap, *s_out = s_stage + 2 * units, *s_in = s_out + units;
 
-      for (int p = gt; p < n_old; p += kGroupThreads) s_old[p] = srt[p];
+      for (int p = gt; p < n_old; p += group_threads) s_old[p] = srt[p];
       // the entries pushed out sit just before the head, the ones that joined at the tail;
       // stage them, then rank-sort them (they are few) into s_out / s_in
-      for (int j = gt; j < evicted; j += kGroupThreads) s_stage[j] = ring[(head - evicted + j + size) % size];
-      for (int j = gt; j < joined; j += kGroupThreads) s_stage[evicted + j] = ring[(head + n - joined + j) % size];
-      group_barrier(group);
-      for (int j = gt; j < evicted + joined; j += kGroupThreads) {
+      for (int j = gt; j < evicted; j += group_threads) s_stage[j] = ring[(head - evicted + j + size) % size];
+      for (int j = gt; j < joined; j += group_threads) s_stage[evicted + j] = ring[(head + n - joined + j) % size];
+      group_barrier(group, group_threads);
+      for (int j = gt; j < evicted + joined; j += group_threads) {
         const bool is_out = j < evicted;
         const double *src = is_out ? s_stage : s_stage + evicted;
         const int m = is_out ? evicted : joined, jj = is_out ? j : j - evicted;
@@ -505,10 +511,10 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, double *so
         for (int q = 0; q < m; ++q) rank += (src[q] < v) || (src[q] == v && q < jj);
         (is_out ? s_out : s_in)[rank] = v;
       }
-      group_barrier(group);
+      group_barrier(group, group_threads);
       // merge: old entries keep their order, lose the first copies of what left, and make
       // room for what joined (a joining value goes after equal old ones)
-      for (int p = gt; p < n_old; p += kGroupThreads) {
+      for (int p = gt; p < n_old; p += group_threads) {
         const double v = s_old[p];
         const int out_lt = lower_bound(s_out, evicted, v);
         const int out_eq = upper_bound(s_out, evicted, v) - out_lt;
@@ -521,12 +527,12 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, double *so
         }
         if (!gone) s_new[p - gone_before + lower_bound(s_in, joined, v)] = v;
       }
-      for (int j = gt; j < joined; j += kGroupThreads) {
+      for (int j = gt; j < joined; j += group_threads) {
         const double v = s_in[j];
         s_new[j + upper_bound(s_old, n_old, v) - upper_bound(s_out, evicted, v)] = v;
       }
-      group_barrier(group);
-      for (int p = gt; p < n; p += kGroupThreads) srt[p] = s_new[p];
+      group_barrier(group, group_threads);
+      for (int p = gt; p < n; p += group_threads) srt[p] = s_new[p];
 
       if (gt < 32) {                               // the group's first warp walks the steps
         const int lane = gt;
@@ -709,7 +715,7 @@ __device__ void finalize(const StreamArgs &a) {
   if (a.mode == kModeReplicaVerify && s_hs.banned[w]) {      // banned: not collected, only reported
     if (tid < rows) {
       if (a.scores_out)
-        for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = CUDART_NAN_F;
+        for (int i = 0; i < a.n_metrics; ++i) a.scores_out[tid * a.n_metrics + i] = CUDART_NAN_F;
       if (a.flags_out) a.flags_out[tid] = tid == 0 ? kFlagBanned : 0u;
     }
     if (tid == kDecider) {
@@ -728,7 +734,7 @@ __device__ void finalize(const StreamArgs &a) {
 
   // scores and the Tukey test: one thread per unit
   unsigned my_flag = 0u;
-  double g[kNumMetrics] = {0., 0., 0.};
+  double g[kNumMetrics] = {0., 0., 0., 0.};
   double st_var_x = 0., st_var_m = 0., st_cov = 0., st_rho = 0., inv_n = 0.;
   bool nonfinite = false;
   int ring_head = 0, ring_count = 0;              // this unit's level, before this step
@@ -755,19 +761,24 @@ __device__ void finalize(const StreamArgs &a) {
     g[0] = u.s[5] * inv_n;
     g[1] = l2z;
     g[2] = (double)u.flips * inv_n;
+    if (a.sw) g[3] = (double)__ldcg(a.sw + tid);   // left by the launches that precede this one
     if (nonfinite) {
       for (int i = 0; i < kNumMetrics; ++i) g[i] = CUDART_NAN;
       my_flag = kFlagNonfinite;
     } else if (testing) {
       const int L = (tid == 0) ? 0 : 1;
+#pragma unroll
       for (int i = 0; i < kNumMetrics; ++i) {
+        if (i >= a.n_metrics) break;
         // (the copy was read from L2 after the ticket, so it holds what CTA 0 of this launch
         // may have just rewritten)
         if (!ks->has_thr[L][i]) { s_no_thr = 1; continue; }
         if (!((a.metric_mask >> i) & 1u)) continue;
         const double q2 = ks->thr[L][i][1];
         const double tau_lower = ks->thr[L][i][4], tau_upper = ks->thr[L][i][5];
-        if (g[i] < tau_lower || g[i] > tau_upper) my_flag |= (1u << i);
+        // (written so that a score that is not a number -- projections beyond the fp32 range --
+        // counts as outside and never joins the history)
+        if (!(g[i] >= tau_lower && g[i] <= tau_upper)) my_flag |= (1u << i);
         if (tid == 0 && fabs(g[i] - q2) >= a.severe_mult * (tau_upper - q2)) s_severe = 1;
       }
     }
@@ -791,11 +802,15 @@ __device__ void finalize(const StreamArgs &a) {
       else if (L)
         k = tid - 1;
       const int idx = (int)(((long long)ring_head + ring_count + k) % size);
+#pragma unroll
       for (int i = 0; i < kNumMetrics; ++i)
-        a.hist[ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx] = g[i];
+        if (i < a.n_metrics) a.hist[ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx] = g[i];
     }
-    if (a.scores_out)
-      for (int i = 0; i < kNumMetrics; ++i) a.scores_out[tid * kNumMetrics + i] = (float)g[i];
+    if (a.scores_out) {
+#pragma unroll
+      for (int i = 0; i < kNumMetrics; ++i)
+        if (i < a.n_metrics) a.scores_out[tid * a.n_metrics + i] = (float)g[i];
+    }
     if (a.stats_out) {                           // off the decision path
       const UnitSums &u = s_unit[tid];
       const double n = (tid == 0) ? (double)B * (double)Ns : (double)Ns;
@@ -918,7 +933,7 @@ stream_kernel_t(const StreamArgs a) {
       // once per iteration, after the worker loop
       const bool may_refresh = (a.mode != kModeReplicaVerify && a.mode != kModeReplicaWarmup) || a.worker == 0;
       if (ks->refresh_pending && may_refresh)
-        refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.a5, s_dyn);
+        refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
     }
   } else if (!skip_stream) {
     stream_cta<kScalar>(a, blockIdx.x - 1, m_in, m_out, s_part);
@@ -939,14 +954,14 @@ stream_kernel_t(const StreamArgs a) {
 // Brings both kinds' thresholds up to date outside a streaming launch (queries, export).
 __global__ void __launch_bounds__(kThreads)
 refresh_kernel(HandleState *hs, double *hist_act, double *hist_grad, double *sorted_act,
-               double *sorted_grad, int cap0, int cap1, int units0, int units1, Alg5Params a5_act,
-               Alg5Params a5_grad) {
+               double *sorted_grad, int cap0, int cap1, int units0, int units1, int n_metrics,
+               Alg5Params a5_act, Alg5Params a5_grad) {
   extern __shared__ double s_dyn[];
   if (hs->kind[0].refresh_pending)
-    refresh_thresholds(&hs->kind[0], hist_act, sorted_act, cap0, cap1, units0, units1, a5_act, s_dyn);
+    refresh_thresholds(&hs->kind[0], hist_act, sorted_act, cap0, cap1, units0, units1, n_metrics, a5_act, s_dyn);
   __syncthreads();
   if (hs->kind[1].refresh_pending)
-    refresh_thresholds(&hs->kind[1], hist_grad, sorted_grad, cap0, cap1, units0, units1, a5_grad, s_dyn);
+    refresh_thresholds(&hs->kind[1], hist_grad, sorted_grad, cap0, cap1, units0, units1, n_metrics, a5_grad, s_dyn);
 }
 
 // Alg. 4 (GradientReplacement) for the one submission a handle sees: if the last verified step

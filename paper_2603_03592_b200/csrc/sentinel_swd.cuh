@@ -17,10 +17,16 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 // projections: proj[(t*L + l)*rows + row] = sum_c v[row][c] * u[l][c], t = 0 for x, 1 for m.
 // A warp owns whole rows; the directions sit in shared memory as bf16 (they are given as bf16).
 // Traffic: x and m are read once, 6 B/element; per element L multiply-adds for each of x and m.
+// The reference is m1 if *active is non-zero, else m0 (a verifier keeps two buffers and flips
+// between them on the device); every kernel of the chain returns at once if *skip is non-zero
+// (a banned worker's tensor is not read).  Both pointers may be nullptr.
 template <int L>
 __global__ void __launch_bounds__(kSwdThreads)
-swd_project_kernel(const uint16_t *x, const float *m, const uint16_t *u, float *proj, long long rows, int d) {
+swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
+                   const uint16_t *u, float *proj, long long rows, int d) {
   extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
+  if (skip && __ldcg(skip)) return;
+  const float *m = (active && __ldcg(active)) ? m1 : m0;
   const int chunks = d >> 3;
   for (int i = threadIdx.x; i < L * chunks; i += kSwdThreads)
     s_u[i] = reinterpret_cast<const uint4 *>(u)[i];
@@ -84,9 +90,11 @@ __device__ __forceinline__ double block_sum_ordered(double v, double *s_red) {
 }
 
 __global__ void __launch_bounds__(kSwdSortThreads)
-swd_sort_samples_kernel(const float *proj, float *sorted, float *w1_sample, int B, int T, int L, long long rows) {
+swd_sort_samples_kernel(const float *proj, float *sorted, float *w1_sample, int B, int T, int L, long long rows,
+                        const int *skip) {
   extern __shared__ float s_val[];                // [2][npad]
   __shared__ double s_red[kSwdSortThreads / 32];
+  if (skip && __ldcg(skip)) return;
   const int b = blockIdx.x / L, l = blockIdx.x - b * L;
   int npad = 1;
   while (npad < T) npad <<= 1;
@@ -129,9 +137,10 @@ swd_sort_samples_kernel(const float *proj, float *sorted, float *w1_sample, int 
 // one round of merging: in every list (2L of them, each B sorted runs of T) neighbouring pairs
 // of runs of `run` samples become one sorted run; an element's place is its index in its own
 // run plus its rank in the partner run (left run first on ties)
-__global__ void swd_merge_kernel(const float *in, float *out, long long rows, int T, int run, int lists) {
+__global__ void swd_merge_kernel(const float *in, float *out, long long rows, int T, int run, int lists,
+                                 const int *skip) {
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= rows * lists) return;
+  if (e >= rows * lists || (skip && __ldcg(skip))) return;
   const long long list = e / rows, i = e - list * rows;
   const float *src = in + list * rows;
   const long long run_len = (long long)run * T;
@@ -156,8 +165,9 @@ __global__ void swd_merge_kernel(const float *in, float *out, long long rows, in
 
 // whole-tensor unit: W1 per direction from the fully merged lists, one CTA per direction
 __global__ void __launch_bounds__(kSwdSortThreads)
-swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int L) {
+swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int L, const int *skip) {
   __shared__ double s_red[kSwdSortThreads / 32];
+  if (skip && __ldcg(skip)) return;
   const int l = blockIdx.x;
   const float *a = merged + (size_t)l * rows, *b = merged + ((size_t)L + l) * rows;
   double acc = 0.;
@@ -167,7 +177,9 @@ swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int 
 }
 
 // the means over the directions for every unit: out[0] = tensor, out[1+b] = sample b
-__global__ void swd_finish_kernel(const float *w1_tensor, const float *w1_sample, float *out, int B, int L) {
+__global__ void swd_finish_kernel(const float *w1_tensor, const float *w1_sample, float *out, int B, int L,
+                                  const int *skip) {
+  if (skip && __ldcg(skip)) return;
   for (int r = threadIdx.x; r <= B; r += blockDim.x) {
     const float *w = r ? w1_sample + (size_t)(r - 1) * L : w1_tensor;
     double s = 0.;

@@ -147,3 +147,11 @@ def microbatch(w: Workload, boundary: int, kind: int, step: int, device="cpu"):
 def bits(x: torch.Tensor):
     """bf16 tensor -> numpy uint16 bit patterns on the host."""
     return x.detach().contiguous().view(torch.int16).cpu().numpy().view("uint16")
+
+
+def directions(L: int, d: int, seed: int, device="cpu") -> torch.Tensor:
+    """L random unit vectors of R^d as bf16 [L, d]: the directions a caller hands to the sliced
+    Wasserstein metric (the paper fixes neither their number nor their draw)."""
+    g = torch.Generator(device="cpu").manual_seed(0x5EED0000 + seed)
+    u = torch.randn(L, d, generator=g, dtype=torch.float64)
+    return (u / u.norm(dim=1, keepdim=True)).to(torch.bfloat16).contiguous().to(device)

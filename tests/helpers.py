@@ -7,18 +7,19 @@ import numpy as np
 
 REL = 1e-3            # statistics and scores: relative error allowed against the float64 oracle
 MAGIC = 0x4C454E49544E4553
-METRIC_MASK = 0x7
+METRIC_MASK = 0xF
 UNIT_BITS = 0xFFFF
 
 
 def assert_scores_close(gpu, ref, x_scale, what=""):
     """|gpu - ref| <= 1e-3 * max(|ref|, floor).  Floors: 1e-3 for the bounded scores (L2z in
     [0,4], SFR in [0,1]: an absolute 1e-6, the resolution fp32 products leave on a
-    correlation), 1e-3 * mean|x| for L1."""
+    correlation), 1e-3 * mean|x| for L1 and for the sliced Wasserstein distance (a fourth
+    column, present when the verifier has directions)."""
     gpu = np.asarray(gpu, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
-    floors = np.array([1e-3 * x_scale, 1e-3, 1e-3])
+    floors = np.array([1e-3 * x_scale, 1e-3, 1e-3, 1e-3 * x_scale])[:gpu.shape[-1]]
     both_nan = np.isnan(gpu) & np.isnan(ref)
     tol = REL * np.maximum(np.abs(ref), floors)
     bad = ~both_nan & ~(np.abs(gpu - ref) <= tol)
@@ -43,7 +44,7 @@ def near_threshold(scores, thr, valid, B, rel=REL):
     near = np.zeros(1 + B, dtype=bool)
     for r in range(1 + B):
         L = 0 if r == 0 else 1
-        for i in range(3):
+        for i in range(scores.shape[1]):
             if not valid[L, i] or np.isnan(scores[r, i]):
                 continue
             for bound in (thr[L, i, 4], thr[L, i, 5]):
@@ -58,7 +59,8 @@ def near_threshold(scores, thr, valid, B, rel=REL):
 def oracle_to_blob(v, params) -> bytes:
     """Serialise an oracle verifier into the library's checkpoint format."""
     B, T, d, l, R = params.B, params.T, params.d, params.l, params.R
-    out = bytearray(struct.pack("<QI5i", MAGIC, 2, B, T, d, l, R))
+    M = v.nm                                   # metrics in use; the layout has room for four
+    out = bytearray(struct.pack("<QI6i", MAGIC, 3, B, T, d, l, R, M))
     out += b"\0" * (64 - len(out))
     workers = np.zeros((3, 16), dtype="<i4")
     for r in range(R):
@@ -67,13 +69,18 @@ def oracle_to_blob(v, params) -> bytes:
     for kind in (0, 1):
         thr, valid = v.thresholds(kind)
         counts = [v.history(kind, L, 0).size for L in (0, 1)]
-        out += struct.pack("<q2i6i", v.steps(kind), *counts, *valid.astype(int).reshape(-1))
-        out += thr.astype("<f8").tobytes()
+        valid4 = np.zeros((2, 4), dtype=int)
+        valid4[:, :M] = valid
+        thr4 = np.zeros((2, 4, 6))
+        thr4[:, :M] = thr
+        out += struct.pack("<q2i8i", v.steps(kind), *counts, *valid4.reshape(-1))
+        out += thr4.astype("<f8").tobytes()
         for L, cap in ((0, l * R), (1, l * R * B)):
-            for i in range(3):
+            for i in range(4):
                 h = np.zeros(cap)
-                hv = v.history(kind, L, i)
-                h[:hv.size] = hv
+                if i < M:
+                    hv = v.history(kind, L, i)
+                    h[:hv.size] = hv
                 out += h.astype("<f8").tobytes()
         out += v.ema(kind).astype("<f4").tobytes()
     return bytes(out)
@@ -82,23 +89,24 @@ def oracle_to_blob(v, params) -> bytes:
 def parse_blob(blob, B, T, d, l, R=1) -> dict:
     """Decode a checkpoint blob into plain numpy pieces."""
     buf = memoryview(bytes(blob))
-    magic, version, b, t, dd, ll, rr = struct.unpack_from("<QI5i", buf, 0)
-    assert magic == MAGIC and version == 2 and (b, t, dd, ll, rr) == (B, T, d, l, R)
+    magic, version, b, t, dd, ll, rr, M = struct.unpack_from("<QI6i", buf, 0)
+    assert magic == MAGIC and version == 3 and (b, t, dd, ll, rr) == (B, T, d, l, R) and M in (3, 4)
     workers = np.frombuffer(buf, dtype="<i4", count=48, offset=64).reshape(3, 16)
     off = 64 + 192
     out = {"violations": int(workers[0, 0]), "clean_streak": int(workers[1, 0]), "banned": int(workers[2, 0]),
-           "workers": workers.copy(), "kinds": []}
+           "workers": workers.copy(), "n_metrics": M, "kinds": []}
     N = B * T * d
     for _ in range(2):
         steps, c0, c1 = struct.unpack_from("<q2i", buf, off)
-        valid = np.array(struct.unpack_from("<6i", buf, off + 16)).reshape(2, 3).astype(bool)
-        off += 40
-        thr = np.frombuffer(buf, dtype="<f8", count=36, offset=off).reshape(2, 3, 6).copy()
-        off += 288
-        hist = [[None] * 3, [None] * 3]
+        valid = np.array(struct.unpack_from("<8i", buf, off + 16)).reshape(2, 4).astype(bool)[:, :M]
+        off += 48
+        thr = np.frombuffer(buf, dtype="<f8", count=48, offset=off).reshape(2, 4, 6)[:, :M].copy()
+        off += 384
+        hist = [[None] * M, [None] * M]
         for L, cap, cnt in ((0, l * R, c0), (1, l * R * B, c1)):
-            for i in range(3):
-                hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
+            for i in range(4):
+                if i < M:
+                    hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
                 off += 8 * cap
         m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape(B, T, d).copy()
         off += 4 * N
@@ -118,7 +126,7 @@ def whole_step_k_events(gt, gvalid, ot, ovalid, params, kind) -> int:
     lg, ls = np.log(params.gamma_g[kind]), np.log(params.gamma_s[kind])
     n = params.n_max[kind]
     for L in range(2):
-        for i in range(3):
+        for i in range(ovalid.shape[1]):
             if not ovalid[L, i] or abs(gt[L, i, 3] / ot[L, i, 3] - 1.0) <= 1e-12:
                 continue
             r = np.log(gt[L, i, 3] / ot[L, i, 3])

@@ -149,7 +149,7 @@ def compare_thresholds(gv, ov, kind, rel=1e-3):
     ot, ovalid = ov.thresholds(kind)
     assert np.array_equal(gvalid, ovalid)
     for L in range(2):
-        for i in range(3):
+        for i in range(ovalid.shape[1]):
             if ovalid[L, i]:
                 assert gt[L, i, 3] == pytest.approx(ot[L, i, 3], rel=1e-12), "multiplier k"
                 tol = rel * np.maximum(np.abs(ot[L, i]), abs(ot[L, i, 1]))
@@ -166,7 +166,7 @@ def multiplier_events(gv, ov, params, kind):
     events = 0
     lg, ls = np.log(params.gamma_g[kind]), np.log(params.gamma_s[kind])
     for L in range(2):
-        for i in range(3):
+        for i in range(ovalid.shape[1]):
             if not ovalid[L, i] or gt[L, i, 3] == pytest.approx(ot[L, i, 3], rel=1e-12):
                 continue
             r = np.log(gt[L, i, 3] / ot[L, i, 3])
@@ -226,11 +226,12 @@ def compare_state(gv, ov, params, m_scale_rel=1e-5):
         m_ref = ov.ema(kind)
         tol = m_scale_rel * max(float(np.abs(m_ref).max()), 1e-30)
         assert np.max(np.abs(ks["m"].astype(np.float64) - m_ref)) <= tol
+        assert st["n_metrics"] == ov.nm
         for L in range(2):
-            for i in range(3):
+            for i in range(ov.nm):
                 href = ov.history(kind, L, i)
                 assert ks["hist"][L][i].size == href.size
-                floor = 1e-3 * (np.abs(href).mean() if i == 0 and href.size else 1.0)
+                floor = 1e-3 * (np.abs(href).mean() if i in (0, 3) and href.size else 1.0)
                 assert np.all(np.abs(ks["hist"][L][i] - href) <= 1e-3 * np.maximum(np.abs(href), floor))
 
 

@@ -53,16 +53,16 @@ def check_state(gv, ov, params, kinds=(ACT, GRAD)):
         assert np.max(np.abs(ks["m"].astype(np.float64) - m_ref)) <= 1e-5 * max(float(np.abs(m_ref).max()), 1e-30)
         assert ks["steps"] == ov.steps(kind)
         for L in range(2):
-            for i in range(3):
+            for i in range(ov.nm):
                 href = ov.history(kind, L, i)
                 assert ks["hist"][L][i].size == href.size
-                floor = 1e-3 * (np.abs(href).mean() if i == 0 and href.size else 1.0)
+                floor = 1e-3 * (np.abs(href).mean() if i in (0, 3) and href.size else 1.0)
                 assert np.all(np.abs(ks["hist"][L][i] - href) <= 1e-3 * np.maximum(np.abs(href), floor))
         gt, gvalid = gv.sentinel_get_thresholds(kind)
         ot, ovalid = ov.thresholds(kind)
         assert np.array_equal(gvalid, ovalid)
         for L in range(2):
-            for i in range(3):
+            for i in range(ov.nm):
                 if ovalid[L, i]:
                     assert gt[L, i, 3] == pytest.approx(ot[L, i, 3], rel=1e-12)
 

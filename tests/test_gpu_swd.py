@@ -113,3 +113,137 @@ def test_argument_checks(sb):
     assert f(x.data_ptr(), m.data_ptr(), u.data_ptr(), 8, 2, 20000, 16, 0, s, o.data_ptr()) == sb.ERR_UNSUPPORTED
     assert f(x.data_ptr(), m.data_ptr(), u.data_ptr(), 16, 2, 4, 8192, 0, s, o.data_ptr()) == sb.ERR_UNSUPPORTED
     assert f(x.data_ptr(), m.data_ptr(), u.data_ptr(), 8, 2, 4, 12, 0, s, o.data_ptr()) == sb.ERR_UNALIGNED
+
+
+# ---------------------------------------------------------------------------------------------
+# the distance as the fourth metric of a verifier (sentinel_set_directions)
+
+from helpers import UNIT_BITS, assert_scores_close, near_threshold, oracle_to_blob, parse_blob  # noqa: E402
+from test_gpu_parity import compare_state, compare_thresholds, lockstep, make_pair  # noqa: E402
+import test_gpu_replicas as rep  # noqa: E402
+
+ACT, GRAD = 0, 1
+
+
+def with_directions(gv, ov, L, d, seed=3):
+    u = synth.directions(L, d, seed, "cuda")
+    gv.sentinel_set_directions(u)
+    ov.set_directions(synth.bits(u))
+    assert gv.sentinel_num_metrics() == 4 and gv.M == 4
+    return u
+
+
+@pytest.mark.parametrize("name,shape,L,steps", [("cfg2", (4, 40, 264), 8, 50), ("cfg4", (3, 24, 1024), 4, 40),
+                                                ("cfg3", (5, 33, 520), 16, 60)],
+                         ids=["cfg2_L8", "cfg4_L4", "cfg3_L16"])
+def test_streams_in_lockstep_with_four_metrics(sb, oracle_mod, name, shape, L, steps):
+    """The benchmark recipes at oracle size with the sliced Wasserstein distance switched on:
+    four score columns, four flag bits, four histories and sets of bounds, step by step."""
+    w = synth.scaled(synth.WORKLOADS[name], name + "_sw", *shape, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    with_directions(gv, ov, L, w.d)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, steps)
+    assert rec["corrupted"] >= 4
+    compare_state(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+        gt, gvalid = gv.sentinel_get_thresholds(kind)
+        assert gt.shape == (2, 4, 6) and gvalid.all()
+    assert rec["near"] <= 2 and rec["k_events"] <= 4, rec
+    gv.close()
+
+
+def test_fourth_column_equals_the_stateless_distance(sb, oracle_mod):
+    """Column 3 of a verified step is sentinel_sliced_wasserstein of the same tensor against the
+    reference the step was tested with (exported just before), bit for bit."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "sw_col", 3, 50, 512)
+    gv, ov, params = make_pair(sb, oracle_mod, w)
+    u = with_directions(gv, ov, 8, w.d)
+    for t in range(5):
+        gv.update_reference(synth.clean(w, 0, ACT, t, "cuda"), ACT)
+    m = torch.from_numpy(parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, params.l)["kinds"][ACT]["m"]).cuda()
+    x = synth.clean(w, 0, ACT, 5, "cuda")
+    gs, gf = gv.verify(x, ACT)
+    torch.cuda.synchronize()
+    want = torch.empty(1 + w.B, device="cuda")
+    sb.sentinel_sliced_wasserstein(x, m, u, want)
+    torch.cuda.synchronize()
+    assert torch.equal(gs[:, 3], want)
+    gv.close()
+
+
+def test_only_the_sliced_wasserstein_bit_with_mask_8(sb, oracle_mod):
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "sw_mask", 2, 32, 64)
+    gv, ov, params = make_pair(sb, oracle_mod, w, metric_mask=8)
+    with_directions(gv, ov, 4, w.d)
+    for t in range(12):
+        x = synth.clean(w, 0, ACT, t, "cuda")
+        gv.update_reference(x, ACT)
+        ov.update_reference(synth.bits(x), ACT)
+    x = (synth.clean(w, 0, ACT, 12, "cuda").float() * 4.0).to(torch.bfloat16)
+    gs, gf = gv.verify(x, ACT)
+    os_, of, commit = ov.verify(synth.bits(x), ACT)
+    gf = gf.cpu().numpy().view(np.uint32)
+    assert np.array_equal(gf, of) and not commit
+    assert np.all(gf & UNIT_BITS == sb.FLAG_SWD)
+    assert_scores_close(gs.cpu().numpy(), os_, float(x.float().abs().mean()), "mask 8")
+    gv.close()
+
+
+def test_worker_iterations_with_four_metrics(sb, oracle_mod):
+    """The multi-worker iteration with directions: every worker's launch is preceded by its own
+    projection / sort chain; a banned worker's chain is skipped on the device."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "replicas_sw", 3, 20, 264)
+    R = 4
+    gv, ov, params = rep.pair(sb, oracle_mod, w, R, l=5, c=2)
+    with_directions(gv, ov, 8, w.d)
+    script = [("warm", {})] * 8 + [("verify", {})] * 2 + [("verify", {1: 6.0})] + [("verify", {})] + \
+             [("verify", {1: 6.0})] + [("verify", {})] * 2
+    for t, (what, scale) in enumerate(script):
+        xs = rep.inputs(w, R, ACT, t, scale)
+        thr, valid = ov.thresholds(ACT)
+        gs, gf, os_, of, n = rep.step_both(gv, ov, xs, ACT, warmup=(what == "warm"))
+        assert gs.shape == (R, 1 + w.B, 4)
+        for r in range(R):
+            assert_scores_close(gs[r], os_[r], float(xs[r].float().abs().mean()), "step %d worker %d" % (t, r))
+        if what != "warm" and not np.array_equal(gf, of):
+            for r in range(R):
+                near = near_threshold(os_[r], thr, valid, w.B)
+                assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            gv.sentinel_import_state(oracle_to_blob(ov, params))
+        ev = rep.whole_step_k_events(*gv.sentinel_get_thresholds(ACT), *ov.thresholds(ACT), params, ACT)
+        if ev:
+            gv.sentinel_import_state(oracle_to_blob(ov, params))
+    assert ov.worker_counters(1)[2] == 1                    # banned, then skipped
+    rep.check_state(gv, ov, params, kinds=(ACT,))
+    gv.close()
+
+
+def test_directions_argument_checks(sb):
+    gv = sb.Verifier(2, 8, 64)
+    u = synth.directions(8, 64, 1, "cuda")
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_set_directions(synth.directions(5, 64, 1, "cuda"))      # L not 4, 8 or 16
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    gv.sentinel_set_directions(u)
+    gv.sentinel_set_directions(u)                                           # again, before any step: fine
+    blob3 = sb.Verifier(2, 8, 64).sentinel_export_state()
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_import_state(blob3)                                     # a three-metric state
+    assert e.value.code == sb.ERR_STATE_SIZE
+    x = torch.zeros(2, 8, 64, dtype=torch.bfloat16, device="cuda")
+    gv.update_reference(x, ACT)
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_set_directions(u)                                       # after the first step
+    assert e.value.code == sb.ERR_INVALID_ARG
+    wide = torch.zeros(2, 8, 65, dtype=torch.bfloat16, device="cuda")
+    s, f = torch.zeros(3, 4, device="cuda"), torch.zeros(3, dtype=torch.int32, device="cuda")
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_verify_strided(wide, ACT, s, f)                         # dense rows only
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    gv.close()
+    big = sb.Verifier(31, 8, 64)                                            # 100 * 32 = 3200 entries
+    with pytest.raises(sb.SentinelError) as e:
+        big.sentinel_set_directions(u)                                      # four windows' copies do not fit
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    big.close()

@@ -62,7 +62,7 @@ def test_default_config_matches_the_paper_table(built):
         assert tuple(getattr(cfg, field)) == want[key]
     assert cfg.ban_violations == want["c"][0] and cfg.forgiveness_steps == want["t_forgiveness"][0]
     assert cfg.window_steps == want["l"][0] and cfg.severe_mult == want["severe_mult"][0]
-    assert cfg.metric_mask == 7 and cfg.shrink_ratio == 0.5 and cfg.n_workers == 1
+    assert cfg.metric_mask == 15 and cfg.shrink_ratio == 0.5 and cfg.n_workers == 1   # every metric of M may flag
 
 
 def test_host_side_argument_checks_need_no_gpu(built):
