@@ -193,8 +193,9 @@ def run_ours(args, rank, world, local_rank):
     violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
 
     # extra figure, outside the timed region: gradient replacement (Alg. 4) after a flagged step
+    extras = nb == 1 and args.extras
     replace = None
-    if nb == 1:
+    if extras:
         v0 = vs[0]
         loud = (xs[0][GRAD][0].float() * 64.0).to(torch.bfloat16)
         v0.sentinel_verify(loud, GRAD, scores[0, 1], flags[0, 1], main)       # flagged: no commit
@@ -215,7 +216,7 @@ def run_ours(args, rank, world, local_rank):
 
     # extra figure, outside the timed region: sliced Wasserstein distance along 8 directions
     swd = None
-    if nb == 1 and 8 * w.d * 2 <= 200 * 1024 and w.T <= 16384:
+    if extras and 8 * w.d * 2 <= 200 * 1024 and w.T <= 16384:
         g = torch.Generator(device=device).manual_seed(11)
         u = torch.randn(8, w.d, generator=g, device=device)
         u = (u / u.norm(dim=1, keepdim=True)).to(torch.bfloat16).contiguous()
@@ -235,11 +236,30 @@ def run_ours(args, rank, world, local_rank):
                "achieved_gbs": round(6 * N / (sms * 1e-3) / 1e9, 1),
                "kernels": "swd_project_kernel + sort, merge, finish", "value_row0": float(sw[0])}
         del ref
+        # the same distance as the verifier's fourth metric: one verified tensor per call, the
+        # projection / sort chain followed by the streaming launch (6 + 6 B/element read, 4 written)
+        v4 = binding.Verifier(w.B, w.T, w.d, device=local_rank)
+        v4.sentinel_set_directions(u, main)
+        s4 = torch.empty(1 + w.B, 4, dtype=torch.float32, device=device)
+        f4 = torch.zeros(1 + w.B, dtype=torch.int32, device=device)
+        for i in range(4):
+            v4.sentinel_update_reference(xs[0][ACT][i % nd], ACT, s4, main)
+        v4.sentinel_verify(xs[0][ACT][4 % nd], ACT, s4, f4, main)
+        torch.cuda.synchronize()
+        s0.record(main)
+        for i in range(8):
+            v4.sentinel_verify(xs[0][ACT][(5 + i) % nd], ACT, s4, f4, main)
+        s1.record(main)
+        torch.cuda.synchronize()
+        vms = s0.elapsed_time(s1) / 8
+        swd["verify_with_four_metrics"] = {"ms_per_tensor": round(vms, 4), "bytes_per_element": 16,
+                                           "achieved_gbs": round(16 * N / (vms * 1e-3) / 1e9, 1)}
+        v4.close()
 
     # extra figure, outside the timed region: one iteration with R workers of the stage
     # (R scoring launches at 6 B/element + the mean over the clean workers at 8 + 2R B/element)
     replicas_fig = None
-    if nb == 1:
+    if extras:
         R = 4 if 100 * 4 * (w.B + 1) <= 4096 else 2
         vr = binding.Verifier(w.B, w.T, w.d, device=local_rank, n_workers=R)
         rs = torch.empty(R, 1 + w.B, 3, dtype=torch.float32, device=device)
@@ -265,7 +285,7 @@ def run_ours(args, rank, world, local_rank):
 
     # extra figure, outside the timed region: the strided (compressed-signal) layout, rows d+1 apart
     strided = None
-    if nb == 1:
+    if extras:
         wide = [torch.nn.functional.pad(xs[0][ACT][i % nd], (0, 1)).contiguous() for i in range(3)]
         for i in range(2):
             vs[0].sentinel_update_reference_strided(wide[i], ACT, scores[0, 0], main)
@@ -439,6 +459,8 @@ def main():
                     help="distinct input tensors per kind kept resident (they rotate beyond that)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--no-extras", dest="extras", action="store_false",
+                    help="skip the extra figures measured after the timed region")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the current kernel, if known")
     args = ap.parse_args()
