@@ -33,6 +33,7 @@ FLAG_L1, FLAG_L2Z, FLAG_SFR, FLAG_SW = 1 << 0, 1 << 1, 1 << 2, 1 << 3
 FLAG_NONFINITE = 1 << 7
 FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
 FLAG_NATURAL_SHIFT = 1 << 20
+FLAG_TAINTED_ELSEWHERE = 1 << 21
 METRIC_BITS = FLAG_L1 | FLAG_L2Z | FLAG_SFR | FLAG_SW
 
 
@@ -96,7 +97,9 @@ def lib():
         L.so_bf16_round.restype = C.c_uint16
         L.so_replace_if_flagged.argtypes = [C.c_void_p, u16p, C.c_int, C.c_int]
         L.so_replace_if_flagged.restype = C.c_int
-        L.so_step_replicas.argtypes = [C.c_void_p, C.POINTER(u16p), C.c_int, C.c_int, dp, C.POINTER(C.c_uint32)]
+        L.so_step_replicas.argtypes = [C.c_void_p, C.POINTER(u16p), C.c_int, C.c_int, C.c_uint, dp, C.POINTER(C.c_uint32)]
+        L.so_skip_tainted.argtypes = [C.c_void_p, C.c_int]
+        L.so_skip_tainted.restype = None
         L.so_step_replicas.restype = C.c_int
         L.so_worker_counters.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int)]
         L.so_worker_counters.restype = None
@@ -294,18 +297,25 @@ class Verifier:
         did = lib().so_replace_if_flagged(self._h, _u16ptr(xb), kind, fill)
         return xb.reshape(self.B, self.T, self.d), bool(did)
 
-    def step_replicas(self, xs_bits, kind: int, warmup: bool = False):
+    def step_replicas(self, xs_bits, kind: int, warmup: bool = False, tainted_in: int = 0):
         """One iteration with all R workers' tensors: (scores [R,1+B,M], flags [R,1+B], number of
-        submissions that entered the EMA)."""
+        submissions that entered the EMA).  tainted_in: bit r = worker r was tainted at another
+        stage (its entry of xs_bits may be None)."""
         assert len(xs_bits) == self.R
-        keep = [_bits(x).reshape(-1) for x in xs_bits]
-        assert all(k.size == self.N for k in keep)
-        ptrs = (C.POINTER(C.c_uint16) * self.R)(*[_u16ptr(k) for k in keep])
+        keep = [None if x is None else _bits(x).reshape(-1) for x in xs_bits]
+        assert all(k is None or k.size == self.N for k in keep)
+        assert all(k is not None or (tainted_in >> r) & 1 for r, k in enumerate(keep))
+        ptrs = (C.POINTER(C.c_uint16) * self.R)(*[C.POINTER(C.c_uint16)() if k is None else _u16ptr(k)
+                                                  for k in keep])
         scores = np.empty((self.R, self.rows, NMETRIC))
         flags = np.zeros((self.R, self.rows), dtype=np.uint32)
-        n = lib().so_step_replicas(self._h, ptrs, kind, int(warmup), _dptr(scores),
+        n = lib().so_step_replicas(self._h, ptrs, kind, int(warmup), int(tainted_in), _dptr(scores),
                                    flags.ctypes.data_as(C.POINTER(C.c_uint32)))
         return scores[:, :, :self.nm].copy(), flags, int(n)
+
+    def skip_tainted(self, kind: int) -> None:
+        """The worker this verifier follows was tainted at another stage in this step."""
+        lib().so_skip_tainted(self._h, kind)
 
     def worker_counters(self, r: int) -> tuple[int, int, int]:
         out = (C.c_int * 3)()

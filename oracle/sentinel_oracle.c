@@ -461,23 +461,32 @@ void so_worker_counters(const so_verifier *v, int r, int out[3]) {
 }
 
 int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int warmup,
-                     double *scores, uint32_t *flags) {
+                     unsigned tainted_in, double *scores, uint32_t *flags) {
   const so_params *p = &v->p;
   const int R = p->R, rows = 1 + p->B;
   so_kind_state *ks = &v->ks[kind];
   double *gam = (double *)malloc((size_t)rows * SO_NMETRIC * sizeof(double));
   int *nf = (int *)malloc((size_t)rows * sizeof(int));
   int collected[SO_MAX_WORKERS], tainted[SO_MAX_WORKERS], severe_w[SO_MAX_WORKERS];
+  int elsewhere[SO_MAX_WORKERS];            /* tainted at another stage: not collected here */
   int no_thr = 0;
   ks->steps += 1;
+  if (warmup) tainted_in = 0;               /* the warm-up phase has honest workers only */
 
   for (int r = 0; r < R; ++r) {
     double *sc = scores + (size_t)r * rows * SO_NMETRIC;
     uint32_t *fl = flags + (size_t)r * rows;
-    collected[r] = 0; tainted[r] = 0; severe_w[r] = 0;
+    collected[r] = 0; tainted[r] = 0; severe_w[r] = 0; elsewhere[r] = 0;
     for (int u = 0; u < rows; ++u) fl[u] = 0;
     if (!warmup && v->banned[r]) {          /* banned workers are not collected any more */
       for (int j = 0; j < rows * SO_NMETRIC; ++j) sc[j] = NAN;
+      continue;
+    }
+    if ((tainted_in >> r) & 1u) {
+      /* Alg. 3: a worker tainted at another stage is marked and not collected; Alg. 2 leaves
+       * such a worker out of its loop.  Either way: no metrics, no counter, no history. */
+      for (int j = 0; j < rows * SO_NMETRIC; ++j) sc[j] = NAN;
+      elsewhere[r] = 1;
       continue;
     }
     collected[r] = 1;
@@ -517,9 +526,12 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
   refresh_thresholds(v, kind);              /* once, after the worker loop */
 
   /* more than half of the workers still in the pool flagged: a natural shift, not an attack */
-  int n_tainted = 0, n_banned = 0, natural = 0;
-  for (int r = 0; r < R; ++r) { n_tainted += tainted[r]; n_banned += v->banned[r]; }
-  if (!warmup && 2 * n_tainted > R - n_banned) {
+  int n_tainted = 0, n_banned = 0, n_elsewhere = 0, natural = 0;
+  for (int r = 0; r < R; ++r) { n_tainted += tainted[r]; n_banned += v->banned[r]; n_elsewhere += elsewhere[r]; }
+  /* the stage's tainted set: the workers flagged here and, for gradients (Alg. 3), the ones
+   * marked as tainted at another stage */
+  const int n_stage = n_tainted + (kind == SO_GRAD ? n_elsewhere : 0);
+  if (!warmup && 2 * n_stage > R - n_banned) {
     natural = 1;
     for (int r = 0; r < R; ++r)
       if (!(flags[(size_t)r * rows] & SO_FLAG_NONFINITE)) tainted[r] = 0;
@@ -538,7 +550,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
       m[e] = beta * m[e] + (1.0 - beta) * (sum / (double)n_clean);
     }
   }
-  ks->last_flagged = (n_tainted > 0) && !natural;
+  ks->last_flagged = (n_stage > 0) && !natural;
   for (int r = 0; r < R; ++r) {
     uint32_t *fl = flags + (size_t)r * rows;
     if (collected[r] && !tainted[r]) fl[0] |= SO_FLAG_COMMITTED;
@@ -546,6 +558,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
     if (!warmup && v->banned[r]) fl[0] |= SO_FLAG_BANNED;
     if (no_thr && collected[r]) fl[0] |= SO_FLAG_NO_THRESHOLDS;
     if (natural) fl[0] |= SO_FLAG_NATURAL_SHIFT;
+    if (elsewhere[r]) fl[0] |= SO_FLAG_TAINTED_ELSEWHERE;
   }
   free(gam); free(nf);
   return n_clean;
@@ -556,6 +569,11 @@ int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill)
   const double *m = v->ks[kind].m;                 /* a flagged step left m at m_{t-1} */
   for (size_t e = 0; e < v->N; ++e) x[e] = fill ? 0 : so_bf16_round(m[e]);
   return 1;
+}
+
+void so_skip_tainted(so_verifier *v, int kind) {
+  v->ks[kind].steps += 1;
+  v->ks[kind].last_flagged = 1;
 }
 
 void so_reset_worker(so_verifier *v) {

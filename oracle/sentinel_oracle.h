@@ -41,7 +41,8 @@ enum {
   SO_FLAG_NONFINITE = 1u << 7,
   SO_FLAG_COMMITTED = 1u << 16, SO_FLAG_SEVERE = 1u << 17,
   SO_FLAG_BANNED = 1u << 18, SO_FLAG_NO_THRESHOLDS = 1u << 19,
-  SO_FLAG_NATURAL_SHIFT = 1u << 20   /* more than half of the workers flagged: taint cleared */
+  SO_FLAG_NATURAL_SHIFT = 1u << 20,  /* more than half of the workers flagged: taint cleared */
+  SO_FLAG_TAINTED_ELSEWHERE = 1u << 21 /* the worker was tainted at another stage: not collected */
 };
 
 /* Hyper-parameters; index 0 = activations, 1 = gradients (Tab. "verification_config"). */
@@ -138,10 +139,22 @@ int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill)
  * workers were flagged the taint set is cleared (natural distribution shift); the EMA moves
  * with the mean of the submissions that are not tainted.  warmup != 0: the warm-up loop of
  * Alg. 1 instead (no test, no counters, everything joins, mean over all workers).
+ * tainted_in: bit r set = worker r was tainted at another stage in this iteration (Sec. 3.1,
+ * cascading effects; the set "tainted downstream" of Alg. 3, the workers "in T_t" that the loop
+ * of Alg. 2 leaves out).  Such a worker is not collected (xs[r] may be NULL): no metrics (NaN
+ * scores), no counter change, no history entry, never part of the mean; its row 0 reports
+ * SO_FLAG_TAINTED_ELSEWHERE.  For gradients it belongs to the stage's tainted set (Alg. 3) and
+ * so counts towards the >50% rule and marks the step as flagged for Alg. 4; for activations it
+ * does not (Alg. 2).  Ignored during warm-up; a banned worker is skipped as banned.
  * scores: [R][1+B][4]; flags: [R][1+B] (row 0 of each worker carries its status bits).
  * Returns the number of submissions that entered the EMA. */
 int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int warmup,
-                     double *scores, uint32_t *flags);
+                     unsigned tainted_in, double *scores, uint32_t *flags);
+
+/* The single-submission form of the same event: the one worker this verifier follows was
+ * tainted at another stage in this step.  Nothing is collected or recorded; the step counts,
+ * and it is marked flagged so that so_replace_if_flagged replaces the outgoing tensor. */
+void so_skip_tainted(so_verifier *v, int kind);
 void so_worker_counters(const so_verifier *v, int r, int out[3]);   /* v_r, streak, banned */
 
 /* A new worker now feeds this boundary: clear its violation counter, streak and ban. */

@@ -394,6 +394,92 @@ def test_banned_worker_is_no_longer_collected(oracle_mod, small):
     assert n == 1 and not (flags[0, 0] & oracle_mod.FLAG_NATURAL_SHIFT)
 
 
+def _warm_replicas_kind(oracle_mod, w, R, n, kind, **kw):
+    v = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, R=R, **kw))
+    for t in range(n):
+        v.step_replicas([synth.bits(x) for x in _replica_inputs(w, R, t, kind)], kind, warmup=True)
+    return v
+
+
+@pytest.mark.parametrize("kind", [ACT, GRAD])
+def test_worker_tainted_at_another_stage_is_not_collected(oracle_mod, small, kind):
+    """Sec. 3.1 (cascading effects), Alg. 2 / Alg. 3: no metrics, no counter, no history entry for
+    such a worker, and the mean of Eq. 1 runs over the others; its tensor is never touched."""
+    R = 4
+    v = _warm_replicas_kind(oracle_mod, small, R, 12, kind)
+    xs = _replica_inputs(small, R, 12, kind)
+    m0 = v.ema(kind)
+    h0 = [v.history(kind, L, 0).size for L in (0, 1)]
+    bits = [synth.bits(x) for x in xs]
+    bits[1] = None                                          # not even supplied
+    scores, flags, n = v.step_replicas(bits, kind, tainted_in=0b0010)
+    assert n == 3 and np.all(np.isnan(scores[1]))
+    assert flags[1, 0] == oracle_mod.FLAG_TAINTED_ELSEWHERE and not np.any(flags[1, 1:])
+    for r in (0, 2, 3):
+        assert flags[r, 0] == oracle_mod.FLAG_COMMITTED
+    mean = sum(from_bits(synth.bits(xs[r])) for r in (0, 2, 3)) / 3
+    assert v.ema(kind) == pytest.approx((0.9 if kind == ACT else 0.8) * m0 + (0.1 if kind == ACT else 0.2) * mean,
+                                        rel=1e-12, abs=1e-15 if kind == ACT else 1e-18)
+    assert v.worker_counters(1) == (0, 0, 0)                # neither a violation nor a clean step
+    assert v.worker_counters(0) == (0, 1, 0)
+    assert [v.history(kind, L, 0).size for L in (0, 1)] == [min(h0[0] + 3, 100 * R), min(h0[1] + 3 * small.B, 100 * R * small.B)]
+    # Alg. 4 needs the verdict: for gradients the stage's tainted set holds the worker (Alg. 3)
+    out, did = v.replace_if_flagged(synth.bits(xs[1]), kind)
+    assert did == (kind == GRAD)
+
+
+def test_workers_tainted_elsewhere_count_towards_the_majority_for_gradients_only(oracle_mod, small):
+    """Alg. 3 adds a worker tainted downstream to the stage's tainted set, Alg. 2 leaves a worker
+    tainted upstream out of its loop: with 2 of 4 workers tainted elsewhere and a third flagged
+    here, the gradient side sees 3 of 4 (a natural shift: the flagged submission enters the EMA
+    after all), the activation side 1 of 4."""
+    R = 4
+    for kind, beta in ((GRAD, 0.8), (ACT, 0.9)):
+        v = _warm_replicas_kind(oracle_mod, small, R, 12, kind)
+        xs = _replica_inputs(small, R, 12, kind)
+        xs[0] = (xs[0].float() * 6).to(torch.bfloat16)
+        m0 = v.ema(kind)
+        scores, flags, n = v.step_replicas([synth.bits(x) for x in xs], kind, tainted_in=0b1100)
+        assert flags[0, 0] & 0xFFFF and v.worker_counters(0)[0] == 1
+        natural = bool(flags[0, 0] & oracle_mod.FLAG_NATURAL_SHIFT)
+        assert natural == (kind == GRAD)
+        clean = (0, 1) if natural else (1,)
+        assert n == len(clean)
+        mean = sum(from_bits(synth.bits(xs[r])) for r in clean) / len(clean)
+        assert v.ema(kind) == pytest.approx(beta * m0 + (1 - beta) * mean, rel=1e-12, abs=1e-15 if kind == ACT else 1e-18)
+        for r in (2, 3):                                    # never part of the mean, shift or not
+            assert flags[r, 0] & oracle_mod.FLAG_TAINTED_ELSEWHERE and not (flags[r, 0] & oracle_mod.FLAG_COMMITTED)
+
+
+def test_tainted_elsewhere_is_ignored_for_banned_workers_and_in_warmup(oracle_mod, small):
+    R = 3
+    v = _warm_replicas(oracle_mod, small, R, 12, c=1)
+    xs = _replica_inputs(small, R, 12)
+    xs[1] = (xs[1].float() * 6).to(torch.bfloat16)
+    v.step_replicas([synth.bits(x) for x in xs], ACT)
+    assert v.worker_counters(1)[2] == 1
+    _, flags, n = v.step_replicas([synth.bits(x) for x in _replica_inputs(small, R, 13)], ACT, tainted_in=0b010)
+    assert flags[1, 0] == oracle_mod.FLAG_BANNED and n == 2
+    _, flags, n = v.step_replicas([synth.bits(x) for x in _replica_inputs(small, R, 14)], ACT, warmup=True,
+                                  tainted_in=0b001)
+    assert n == 3 and not np.any(flags & oracle_mod.FLAG_TAINTED_ELSEWHERE)
+
+
+def test_skip_tainted_counts_the_step_and_asks_for_replacement(oracle_mod, small):
+    v = _warm(oracle_mod, small, 2)
+    for t in range(14):
+        v.update_reference(synth.bits(synth.clean(small, 0, GRAD, t)), GRAD)
+    m0, h0, c0, s0 = v.ema(GRAD), v.history(GRAD, 0, 0).copy(), v.counters(), v.steps(GRAD)
+    v.skip_tainted(GRAD)
+    assert v.steps(GRAD) == s0 + 1 and v.counters() == c0
+    assert np.array_equal(v.ema(GRAD), m0) and np.array_equal(v.history(GRAD, 0, 0), h0)
+    g = synth.clean(small, 0, GRAD, 15)
+    out, did = v.replace_if_flagged(synth.bits(g), GRAD)
+    assert did and np.all(np.abs(from_bits(out) - m0) <= 2.0 ** -8 * np.abs(m0) + 1e-45)
+    assert v.verify(synth.bits(g), GRAD)[2]                 # a clean step clears the verdict
+    assert not v.replace_if_flagged(synth.bits(g), GRAD)[1]
+
+
 # ---------------------------------------------------------------------------------------------
 # the sliced Wasserstein distance as a fourth member of the metric set M (Sec. 3.1)
 
