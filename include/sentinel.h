@@ -71,6 +71,7 @@ typedef enum sentinel_kind { SENTINEL_ACT = 0, SENTINEL_GRAD = 1 } sentinel_kind
 #define SENTINEL_FLAG_SEVERE (1u << 17)       /* row 0: deviation >= severe_mult * allowed   */
 #define SENTINEL_FLAG_BANNED (1u << 18)       /* row 0: sticky until sentinel_reset_worker   */
 #define SENTINEL_FLAG_NO_THRESHOLDS (1u << 19) /* row 0: some history was still empty         */
+#define SENTINEL_FLAG_TAINTED_ELSEWHERE (1u << 21) /* row 0: tainted at another stage, not collected */
 #define SENTINEL_FLAG_NATURAL_SHIFT (1u << 20) /* row 0: more than half of the workers flagged */
 
 /* Hyper-parameters.  Arrays are indexed by kind.  Defaults: table "verification_config",
@@ -247,14 +248,37 @@ int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf);
  * entries for the whole-tensor unit, times B for samples); the bounds are refreshed once per
  * iteration; if more than half of the workers still in the pool were flagged, the taint set
  * is cleared (natural distribution shift, SENTINEL_FLAG_NATURAL_SHIFT) and the counters stay
- * as they moved; the reference then moves with the mean of the untainted submissions (each
- * tensor is read once for its scores and once more for the mean).  A banned worker is not
- * read: its scores are NaN and its row 0 reports SENTINEL_FLAG_BANNED.
+ * as they moved; the reference then moves with the mean of the untainted submissions.  All
+ * workers are scored by ONE launch that reads every tensor and the reference once and writes
+ * the mean over all collected workers into the spare reference buffer (2*R + 8 bytes per
+ * element); if nobody was flagged that buffer becomes the reference, else a second launch takes
+ * the mean over the clean workers from the untouched m_{t-1} (reading those tensors again).  A
+ * banned worker is not read: its scores are NaN and its row 0 reports SENTINEL_FLAG_BANNED.
+ * The per-token buffer of sentinel_set_token_stats_buffer is not written by these calls.
  * dev_scores_out fp32 [n_workers][1+B][M]; dev_flags_out u32 [n_workers][1+B]; row 0 of worker
  * r carries COMMITTED iff its tensor entered the mean. */
 int sentinel_verify_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind,
                              int B, int T, int d, void *cuda_stream, float *dev_scores_out,
                              unsigned *dev_flags_out);
+
+/* sentinel_verify_replicas with the cascading-effect input of Sec. 3.1: bit r of tainted_in
+ * says that worker r was tainted at another stage in this iteration (the set "tainted
+ * downstream" of Alg. 3; the workers already in T_t that the loop of Alg. 2 leaves out).  Such
+ * a worker is not collected: host_dev_xs[r] is ignored (may be NULL), its scores are NaN, its
+ * counter, the histories and the mean are untouched, and its row 0 reports
+ * SENTINEL_FLAG_TAINTED_ELSEWHERE.  For kind = GRAD it belongs to the stage's tainted set
+ * (Alg. 3): it counts towards the >50% rule and leaves the step marked as flagged for
+ * sentinel_replace_if_flagged; for kind = ACT it does not (Alg. 2).  A banned worker is
+ * reported as banned whatever its bit says.  Bits at or above n_workers are an error. */
+int sentinel_verify_replicas_tainted(sentinel_verifier *h, const void *const *host_dev_xs,
+                                     sentinel_kind kind, unsigned tainted_in, int B, int T, int d,
+                                     void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out);
+
+/* The single-submission form of the same event: the worker this verifier follows was tainted
+ * at another stage in this step.  Nothing is read or recorded (statistics paused, Sec. 3.1);
+ * the step counts, and it is left marked as flagged so that sentinel_replace_if_flagged
+ * overwrites the outgoing tensor (Alg. 4).  Enqueued on cuda_stream. */
+int sentinel_skip_tainted(sentinel_verifier *h, sentinel_kind kind, void *cuda_stream);
 
 /* The warm-up loop of Alg. 1 with all workers: no test, no counters, every unit of every worker
  * joins the history, the reference moves with the mean over all workers.  Outputs as above

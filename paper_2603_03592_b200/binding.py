@@ -26,11 +26,12 @@ FLAG_L1, FLAG_L2Z, FLAG_SFR, FLAG_SWD = 1 << 0, 1 << 1, 1 << 2, 1 << 3
 FLAG_NONFINITE = 1 << 7
 FLAG_COMMITTED, FLAG_SEVERE, FLAG_BANNED, FLAG_NO_THRESHOLDS = 1 << 16, 1 << 17, 1 << 18, 1 << 19
 FLAG_NATURAL_SHIFT = 1 << 20
+FLAG_TAINTED_ELSEWHERE = 1 << 21
 MAX_WORKERS = 16
 
 EXPORTS = (
     "sentinel_default_config", "sentinel_verifier_create", "sentinel_verify",
-    "sentinel_set_directions", "sentinel_num_metrics",
+    "sentinel_set_directions", "sentinel_num_metrics", "sentinel_verify_replicas_tainted", "sentinel_skip_tainted",
     "sentinel_update_reference", "sentinel_verify_host", "sentinel_distance",
     "sentinel_verify_replicas", "sentinel_update_reference_replicas", "sentinel_get_worker_counters",
     "sentinel_verify_strided", "sentinel_update_reference_strided",
@@ -98,6 +99,8 @@ def lib():
         L.sentinel_verify_replicas.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_update_reference_replicas.argtypes = [vp, vp, ip, ip, ip, ip, vp, vp, vp]
         L.sentinel_get_worker_counters.argtypes = [vp, ip, vp, vp]
+        L.sentinel_verify_replicas_tainted.argtypes = [vp, vp, ip, C.c_uint, ip, ip, ip, vp, vp, vp]
+        L.sentinel_skip_tainted.argtypes = [vp, ip, vp]
         L.sentinel_state_bytes.argtypes = [vp]
         L.sentinel_state_bytes.restype = C.c_size_t
         L.sentinel_export_state.argtypes = [vp, vp, C.c_size_t, vp]
@@ -229,7 +232,7 @@ class Verifier:
 
     def _worker_pointers(self, xs):
         assert len(xs) == self.R, "one tensor per worker"
-        return (C.c_void_p * self.R)(*[x.data_ptr() for x in xs])
+        return (C.c_void_p * self.R)(*[None if x is None else x.data_ptr() for x in xs])
 
     def sentinel_verify_replicas(self, xs, kind: int, scores_out: torch.Tensor,
                                  flags_out: torch.Tensor, stream=None) -> None:
@@ -245,11 +248,24 @@ class Verifier:
                                                         _stream_ptr(stream), _ptr(scores_out),
                                                         _ptr(flags_out)), self._h)
 
-    def step_replicas(self, xs, kind: int, warmup: bool = False, stream=None):
-        scores = torch.empty(self.R, self.rows, self.M, dtype=torch.float32, device=xs[0].device)
-        flags = torch.zeros(self.R, self.rows, dtype=torch.int32, device=xs[0].device)
+    def sentinel_verify_replicas_tainted(self, xs, kind: int, tainted_in: int, scores_out: torch.Tensor,
+                                         flags_out: torch.Tensor, stream=None) -> None:
+        """As sentinel_verify_replicas; bit r of tainted_in: worker r was tainted at another stage and
+        is not collected (xs[r] may be None)."""
+        _check(lib().sentinel_verify_replicas_tainted(self._h, self._worker_pointers(xs), kind, tainted_in,
+                                                      self.B, self.T, self.d, _stream_ptr(stream),
+                                                      _ptr(scores_out), _ptr(flags_out)), self._h)
+
+    def sentinel_skip_tainted(self, kind: int, stream=None) -> None:
+        _check(lib().sentinel_skip_tainted(self._h, kind, _stream_ptr(stream)), self._h)
+
+    def step_replicas(self, xs, kind: int, warmup: bool = False, stream=None, tainted_in: int = 0):
+        scores = torch.empty(self.R, self.rows, self.M, dtype=torch.float32, device=self.device)
+        flags = torch.zeros(self.R, self.rows, dtype=torch.int32, device=self.device)
         if warmup:
             self.sentinel_update_reference_replicas(xs, kind, scores, flags, stream)
+        elif tainted_in:
+            self.sentinel_verify_replicas_tainted(xs, kind, tainted_in, scores, flags, stream)
         else:
             self.sentinel_verify_replicas(xs, kind, scores, flags, stream)
         return scores, flags

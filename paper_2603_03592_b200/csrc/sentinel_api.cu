@@ -216,7 +216,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.one_minus_beta = (float)(1.0 - h->cfg.beta[kind]);
   a.cap0 = h->cap0; a.cap1 = h->cap1;
   a.units0 = h->units0; a.units1 = h->units1;
-  a.R = h->R; a.worker = 0;
+  a.R = h->R;
   a.x_row_stride = h->cfg.d;
   a.a5 = alg5_of(h->cfg, kind);
   a.severe_mult = h->cfg.severe_mult;
@@ -342,7 +342,7 @@ int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bo
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
   SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), h->ema[kind][0], h->ema[kind][1], &h->hs->kind[kind].active,
                            may_skip ? &h->hs->banned[worker] : nullptr, h->sw_u, h->sw_L, h->cfg.B, h->cfg.T,
-                           h->cfg.d, sms, h->sw_scratch, h->sw_out, s));
+                           h->cfg.d, sms, h->sw_scratch, h->sw_out + (size_t)worker * (1 + h->cfg.B), s));
   return SENTINEL_OK;
 }
 
@@ -436,6 +436,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     cudaError_t ae = cudaFuncSetAttribute(stream_kernel_t<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
   }
   std::string oerr;
@@ -453,7 +454,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     alloc((void **)&h->sorted[k], hist_doubles(h) * sizeof(double));
     alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
   }
-  alloc((void **)&h->partials, (size_t)h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));
+  alloc((void **)&h->partials, (size_t)h->R * h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));   // per worker
   alloc((void **)&h->hs, sizeof(HandleState));
   if (e == cudaSuccess) {
     HandleState init;
@@ -599,32 +600,59 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
 
 namespace {
 
-int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, int B, int T, int d, void *cuda_stream,
-                  float *scores, unsigned *flags, bool warmup) {
+int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigned tainted_in, int B, int T, int d,
+                  void *cuda_stream, float *scores, unsigned *flags, bool warmup) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (!xs) return fail(h, SENTINEL_ERR_INVALID_ARG, "the array of tensors is NULL");
+  if (warmup) tainted_in = 0;                        // the warm-up phase has honest workers only
+  if (h->R < 32 && (tainted_in >> h->R) != 0) return fail(h, SENTINEL_ERR_INVALID_ARG, "tainted_in names workers beyond n_workers = %d", h->R);
   for (int r = 0; r < h->R; ++r) {
+    if ((tainted_in >> r) & 1u) continue;            // not collected: its pointer is not looked at
     int rc = check_call(h, xs[r], kind, B, T, d);
     if (rc) return rc;
   }
   if (!scores || (!warmup && !flags)) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", kind);
+  if (B != h->cfg.B || T != h->cfg.T || d != h->cfg.d)
+    return fail(h, SENTINEL_ERR_SHAPE_MISMATCH, "shape [%d,%d,%d] differs from the handle's [%d,%d,%d]", B, T, d, h->cfg.B, h->cfg.T, h->cfg.d);
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const size_t rows = 1 + (size_t)B;
   h->started = true;
   if (warmup && flags) SENTINEL_CUDA(h, cudaMemsetAsync(flags, 0, h->R * rows * sizeof(unsigned), s));
+
+  ReplicaArgs ra;
+  memset(&ra, 0, sizeof ra);
+  ra.s = make_args(h, nullptr, kind, warmup ? kModeReplicaWarmup : kModeReplicaVerify, nullptr, nullptr);
+  ra.s.sw = nullptr;
+  ra.partials = h->partials;
+  ra.scores_all = scores;
+  ra.flags_all = warmup ? nullptr : flags;
+  ra.sw_all = h->sw_out;
+  ra.tainted_in = tainted_in;
   WorkerPointers wp;
   memset(&wp, 0, sizeof wp);
-  for (int r = 0; r < h->R; ++r) {                 // every worker against the same m_{t-1}
-    StreamArgs a = make_args(h, xs[r], kind, warmup ? kModeReplicaWarmup : kModeReplicaVerify,
-                             scores + r * rows * h->n_metrics, warmup ? nullptr : flags + r * rows);
-    a.worker = r;
+  for (int r = 0; r < h->R; ++r) {
+    if ((tainted_in >> r) & 1u) continue;
+    ra.xs[r] = wp.x[r] = static_cast<const uint16_t *>(xs[r]);
+    // with directions: every collected worker's distances first, each into its own row block
     int rc = run_handle_swd(h, xs[r], kind, r, !warmup, s);
     if (rc) return rc;
-    rc = launch(h, a, h->G + 1, s);
-    if (rc) return rc;
-    wp.x[r] = static_cast<const uint16_t *>(xs[r]);
+  }
+  {   // every worker against the same m_{t-1}, in one launch
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3((unsigned)(h->G + 1));
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = h->refresh_smem;
+    lc.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &attr;
+    lc.numAttrs = 1;
+    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel, ra));
   }
   int sms = 0;
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
@@ -645,13 +673,30 @@ extern "C" {
 
 int sentinel_verify_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind, int B,
                              int T, int d, void *cuda_stream, float *dev_scores_out, unsigned *dev_flags_out) {
-  return step_replicas(h, host_dev_xs, kind, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, false);
+  return step_replicas(h, host_dev_xs, kind, 0u, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, false);
+}
+
+int sentinel_verify_replicas_tainted(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind,
+                                     unsigned tainted_in, int B, int T, int d, void *cuda_stream,
+                                     float *dev_scores_out, unsigned *dev_flags_out) {
+  return step_replicas(h, host_dev_xs, kind, tainted_in, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, false);
+}
+
+int sentinel_skip_tainted(sentinel_verifier *h, sentinel_kind kind, void *cuda_stream) {
+  if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
+  if (kind != SENTINEL_ACT && kind != SENTINEL_GRAD) return fail(h, SENTINEL_ERR_INVALID_ARG, "kind %d is neither ACT nor GRAD", (int)kind);
+  DeviceGuard guard(h->cfg.device);
+  SENTINEL_CUDA(h, guard.status);
+  h->started = true;
+  skip_tainted_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>(h->hs, (int)kind);
+  SENTINEL_CUDA(h, cudaGetLastError());
+  return SENTINEL_OK;
 }
 
 int sentinel_update_reference_replicas(sentinel_verifier *h, const void *const *host_dev_xs, sentinel_kind kind,
                                        int B, int T, int d, void *cuda_stream, float *dev_scores_out,
                                        unsigned *dev_flags_out) {
-  return step_replicas(h, host_dev_xs, kind, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, true);
+  return step_replicas(h, host_dev_xs, kind, 0u, B, T, d, cuda_stream, dev_scores_out, dev_flags_out, true);
 }
 
 int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentinel_kind kind, int B, int T,
@@ -692,9 +737,10 @@ int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L,
   float *scratch = nullptr, *out = nullptr;
   cudaError_t e = cudaMalloc((void **)&u, u_bytes);
   if (e == cudaSuccess) e = cudaMalloc((void **)&scratch, swd_scratch_floats(L, h->cfg.B, h->cfg.T) * sizeof(float));
-  if (e == cudaSuccess) e = cudaMalloc((void **)&out, (size_t)(1 + h->cfg.B) * sizeof(float));
+  const size_t out_floats = (size_t)h->R * (1 + h->cfg.B);      // a block of 1+B per worker
+  if (e == cudaSuccess) e = cudaMalloc((void **)&out, out_floats * sizeof(float));
   if (e == cudaSuccess) e = cudaMemcpyAsync(u, dev_u_bf16, u_bytes, cudaMemcpyDeviceToDevice, s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(out, 0, (size_t)(1 + h->cfg.B) * sizeof(float), s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(out, 0, out_floats * sizeof(float), s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
     cudaFree(u); cudaFree(scratch); cudaFree(out);

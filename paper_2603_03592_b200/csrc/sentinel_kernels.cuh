@@ -41,6 +41,7 @@ constexpr unsigned kFlagSevere = 1u << 17;
 constexpr unsigned kFlagBanned = 1u << 18;
 constexpr unsigned kFlagNoThresholds = 1u << 19;
 constexpr unsigned kFlagNaturalShift = 1u << 20;
+constexpr unsigned kFlagTaintedElsewhere = 1u << 21;
 
 // word 7 of a partial slot: bits 0-2 flags, bits 8-15 tag (1 + sample index, 0 = slot unused),
 // bits 16-31 the sample's first x (bf16 bits), bits 32-63 the sample's first m (fp32 bits)
@@ -65,7 +66,10 @@ struct KindState {
   int last_flagged;       // the last verified step of this kind raised a flag (no commit)
   unsigned step_collected;  // multi-worker iteration in progress: workers scored so far,
   unsigned step_tainted;    //   workers that raised a flag,
-  unsigned step_nonfinite;  //   workers whose tensor held a NaN or an infinity
+  unsigned step_nonfinite;  //   workers whose tensor held a NaN or an infinity,
+  unsigned step_elsewhere;  //   workers tainted at another stage (not collected)
+  int pad;
+  long long mean_done_step; // the iteration whose mean over the workers is already in place
   int has_thr[2][kNumMetrics];
   double thr[2][kNumMetrics][kNumThr];   // q1 q2 q3 k tau_lower tau_upper
 };
@@ -98,7 +102,7 @@ struct StreamArgs {
   float beta, one_minus_beta;
   int cap0, cap1;
   int units0, units1;              // entries one iteration can append per level: R and R*B
-  int R, worker;                   // workers of the stage; which one this launch scores
+  int R, pad3;                     // workers of the stage
   long long x_row_stride;          // elements from one row of x to the next (d when dense)
   const float *sw;                 // [1+B] sliced Wasserstein distance of every unit, computed by the
                                    // launches before this one; nullptr when n_metrics = 3
@@ -603,7 +607,18 @@ struct UnitSums {
   double x0, m0;             // the shift the sums were taken about
 };
 
-__device__ void finalize(const StreamArgs &a) {
+// What one pass of finalize reports on: a single submission, or one worker of an iteration.
+struct FinalizeTarget {
+  int worker;                            // whose counters move (0 for a single submission)
+  const unsigned long long *partials;    // that tensor's partial slots
+  float *scores_out;                     // [(1+B)*n_metrics] or nullptr
+  unsigned *flags_out;                   // [1+B] or nullptr
+  const float *sw;                       // [1+B] sliced Wasserstein distances, or nullptr
+  int elsewhere;                         // the worker was tainted at another stage: not collected
+  int last;                              // the launch ends with this pass: the ticket is re-armed
+};
+
+__device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
   __shared__ UnitSums s_unit[kMaxB + 1];
   __shared__ unsigned s_flag[kMaxB + 1];
   __shared__ int s_severe, s_no_thr;
@@ -637,7 +652,7 @@ __device__ void finalize(const StreamArgs &a) {
     if (c_hi > a.G - 1) c_hi = a.G - 1;
     const long long n_slots = (c_hi - c_lo + 1) * kSegsPerCta;
     for (long long q = lane; q < n_slots; q += 32) {
-      const unsigned long long *slot = a.partials + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
+      const unsigned long long *slot = ft.partials + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
       unsigned long long w[kSlotWords];
 #pragma unroll
       for (int j = 0; j < kSlotWords; ++j) w[j] = __ldcg(slot + j);   // one round trip, then the tag
@@ -710,21 +725,25 @@ __device__ void finalize(const StreamArgs &a) {
   KindState *ks = a.hs ? &s_hs.kind[a.kind] : nullptr;     // the shared copy
   const bool replica = (a.mode == kModeReplicaVerify || a.mode == kModeReplicaWarmup);
   const bool testing = (a.mode == kModeVerify || a.mode == kModeReplicaVerify);
-  const int w = replica ? a.worker : 0;                      // whose counters this launch moves
+  const int w = replica ? ft.worker : 0;                     // whose counters this pass moves
 
-  if (a.mode == kModeReplicaVerify && s_hs.banned[w]) {      // banned: not collected, only reported
+  // banned, or tainted at another stage (Alg. 3; left out of the loop of Alg. 2): not
+  // collected, only reported
+  if (a.mode == kModeReplicaVerify && (s_hs.banned[w] || ft.elsewhere)) {
+    const bool banned = s_hs.banned[w] != 0;
     if (tid < rows) {
-      if (a.scores_out)
-        for (int i = 0; i < a.n_metrics; ++i) a.scores_out[tid * a.n_metrics + i] = CUDART_NAN_F;
-      if (a.flags_out) a.flags_out[tid] = tid == 0 ? kFlagBanned : 0u;
+      if (ft.scores_out)
+        for (int i = 0; i < a.n_metrics; ++i) ft.scores_out[tid * a.n_metrics + i] = CUDART_NAN_F;
+      if (ft.flags_out) ft.flags_out[tid] = tid == 0 ? (banned ? kFlagBanned : kFlagTaintedElsewhere) : 0u;
     }
     if (tid == kDecider) {
       if (w == 0) {                                          // the iteration still starts here
         ks->steps += 1;
-        ks->step_collected = ks->step_tainted = ks->step_nonfinite = 0u;
+        ks->step_collected = ks->step_tainted = ks->step_nonfinite = ks->step_elsewhere = 0u;
       }
+      if (!banned) ks->step_elsewhere |= 1u << w;
       ks->refresh_pending = 1;                               // Alg. 5 still runs once per iteration
-      s_hs.ticket = 0u;
+      if (ft.last) s_hs.ticket = 0u;
     }
     __syncthreads();
     if (tid < kStateWords)
@@ -761,7 +780,7 @@ __device__ void finalize(const StreamArgs &a) {
     g[0] = u.s[5] * inv_n;
     g[1] = l2z;
     g[2] = (double)u.flips * inv_n;
-    if (a.sw) g[3] = (double)__ldcg(a.sw + tid);   // left by the launches that precede this one
+    if (ft.sw) g[3] = (double)__ldcg(ft.sw + tid);   // left by the launches that precede this one
     if (nonfinite) {
       for (int i = 0; i < kNumMetrics; ++i) g[i] = CUDART_NAN;
       my_flag = kFlagNonfinite;
@@ -806,10 +825,10 @@ __device__ void finalize(const StreamArgs &a) {
       for (int i = 0; i < kNumMetrics; ++i)
         if (i < a.n_metrics) a.hist[ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx] = g[i];
     }
-    if (a.scores_out) {
+    if (ft.scores_out) {
 #pragma unroll
       for (int i = 0; i < kNumMetrics; ++i)
-        if (i < a.n_metrics) a.scores_out[tid * a.n_metrics + i] = (float)g[i];
+        if (i < a.n_metrics) ft.scores_out[tid * a.n_metrics + i] = (float)g[i];
     }
     if (a.stats_out) {                           // off the decision path
       const UnitSums &u = s_unit[tid];
@@ -828,7 +847,7 @@ __device__ void finalize(const StreamArgs &a) {
     unsigned status = 0u;
     if (!replica || w == 0) {                    // an iteration starts with its first worker
       ks->steps += 1;
-      ks->step_collected = ks->step_tainted = ks->step_nonfinite = 0u;
+      ks->step_collected = ks->step_tainted = ks->step_nonfinite = ks->step_elsewhere = 0u;
     }
     int joined[2] = {0, 0};
     if (testing) {
@@ -873,12 +892,12 @@ __device__ void finalize(const StreamArgs &a) {
       // (several workers append between two refreshes: what the refresh merges accumulates)
       if (ks->refresh_pending) { ks->last_joined[L] += joined[L]; ks->last_evicted[L] += evicted; }
     }
-    s_hs.ticket = 0u;                            // ready for the next launch
+    if (ft.last) s_hs.ticket = 0u;               // ready for the next launch
     s_status = status;
   }
   __syncthreads();
-  if (a.flags_out && tid < rows)
-    a.flags_out[tid] = s_flag[tid] | (tid == 0 ? s_status : 0u);
+  if (ft.flags_out && tid < rows)
+    ft.flags_out[tid] = s_flag[tid] | (tid == 0 ? s_status : 0u);
   if (a.hs) {                                    // write the state back
     if (tid < kStateWords)
       reinterpret_cast<unsigned long long *>(a.hs)[tid] = reinterpret_cast<unsigned long long *>(&s_hs)[tid];
@@ -911,7 +930,6 @@ stream_kernel_t(const StreamArgs a) {
 
   const float *m_in;
   float *m_out;
-  bool skip_stream = false;
   if (a.mode == kModeDistance) {
     m_in = a.m_ext;
     m_out = nullptr;
@@ -919,23 +937,15 @@ stream_kernel_t(const StreamArgs a) {
     const int act = __ldcg(&a.hs->kind[a.kind].active);   // written by an earlier launch only
     m_in = a.ema[act];
     m_out = a.ema[act ^ 1];
-    if (a.mode == kModeReplicaVerify || a.mode == kModeReplicaWarmup) {
-      m_out = nullptr;                     // the reference moves once, after all workers
-      // a banned worker is no longer collected: nothing of its tensor is read
-      skip_stream = (a.mode == kModeReplicaVerify) && __ldcg(&a.hs->banned[a.worker]) != 0;
-    }
   }
 
   if (blockIdx.x == 0) {
     if (a.hs) {
       KindState *ks = &a.hs->kind[a.kind];
-      // within a multi-worker iteration only the first worker's launch refreshes: Alg. 5 runs
-      // once per iteration, after the worker loop
-      const bool may_refresh = (a.mode != kModeReplicaVerify && a.mode != kModeReplicaWarmup) || a.worker == 0;
-      if (ks->refresh_pending && may_refresh)
+      if (ks->refresh_pending)
         refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
     }
-  } else if (!skip_stream) {
+  } else {
     stream_cta<kScalar>(a, blockIdx.x - 1, m_in, m_out, s_part);
   }
 
@@ -948,7 +958,274 @@ stream_kernel_t(const StreamArgs a) {
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  finalize(a);
+  const FinalizeTarget ft = {0, a.partials, a.scores_out, a.flags_out, a.sw, 0, 1};
+  finalize(a, ft);
+}
+
+// ---------------------------------------------------------------------------------------------
+// All workers of a stage in one launch (worker loop of Alg. 2 / Alg. 3, Alg. 1 main loop).
+//
+// Every worker's tensor is tested against the same m_{t-1}, so a tile of m is loaded once and
+// each worker's tile of x is streamed past it: 2 B per worker and element plus 4 B of m read and
+// 4 B written, instead of a pass over m per worker and another over every x for the mean.  The
+// write is the mean over all collected workers, m' = beta m + (1-beta)/n sum_r x^(r), put into
+// the spare buffer on the assumption that nobody will be flagged; the last CTA scores the workers
+// one after the other (pooled history, per-worker counters) and, if indeed nobody was flagged,
+// makes that buffer the reference.  Otherwise the mean over the clean workers is taken afterwards
+// by ema_mean_kernel from the untouched m_{t-1}.
+//
+// A thread cannot carry fp64 sums for 16 workers, so after every warp tile (512 elements) the
+// tile's fp32 sums are added up across the warp and one lane folds them into the warp's fp64
+// accumulators in shared memory.
+struct ReplicaArgs {
+  StreamArgs s;                       // x, scores_out, flags_out, sw unused
+  const uint16_t *xs[kMaxWorkers];    // worker r's tensor; not read for a worker in tainted_in
+  unsigned long long *partials;       // [R][G][2][kSlotWords]
+  float *scores_all;                  // [R][(1+B)*n_metrics]
+  unsigned *flags_all;                // [R][1+B] or nullptr (warm-up)
+  const float *sw_all;                // [R][1+B] sliced Wasserstein distances, or nullptr
+  unsigned tainted_in;                // bit r: worker r was tainted at another stage
+  int pad;
+};
+
+struct ReplicaShared {
+  double acc[kWarps][kMaxWorkers][4];             // sums of (x-x0), (x-x0)^2, (x-x0)(m-m0), |x-m|
+  unsigned long long flips[kWarps][kMaxWorkers];
+  unsigned bits[kWarps][kMaxWorkers];             // kBitNonfinite | kBitXVaries
+  double m_acc[kWarps][2];                        // sums of (m-m0), (m-m0)^2
+  unsigned m_varies[kWarps];
+  unsigned x0[kMaxWorkers];                       // the sample's first element, per worker
+};
+
+__device__ void replica_segment(const ReplicaArgs &ra, int b, long long row_a, long long row_b, const float *m_in,
+                                float *m_out, unsigned streamed, int c, int sgm, ReplicaShared &sh) {
+  const StreamArgs &a = ra.s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunks = a.d >> 3;                               // d is a multiple of 8 here
+  const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
+  const int n_tiles = (int)(row_b - row_a) * tiles_per_row;
+  const size_t sample_off = (size_t)b * a.T * a.d;
+  const float beta = a.beta, wgt = a.one_minus_beta / (float)__popc(streamed);
+
+  __syncthreads();                                           // the previous segment is done with sh
+  for (int i = threadIdx.x; i < kWarps * kMaxWorkers; i += kThreads) {
+    const int w = i / kMaxWorkers, r = i - w * kMaxWorkers;
+    sh.acc[w][r][0] = sh.acc[w][r][1] = sh.acc[w][r][2] = sh.acc[w][r][3] = 0.;
+    sh.flips[w][r] = 0ull;
+    sh.bits[w][r] = 0u;
+  }
+  if (threadIdx.x < kWarps) { sh.m_acc[threadIdx.x][0] = sh.m_acc[threadIdx.x][1] = 0.; sh.m_varies[threadIdx.x] = 0u; }
+  if (threadIdx.x < a.R && ((streamed >> threadIdx.x) & 1u)) sh.x0[threadIdx.x] = ra.xs[threadIdx.x][sample_off];
+  const unsigned m0bits = __float_as_uint(m_in[sample_off]);
+  const float m0 = __uint_as_float(m0bits);
+  __syncthreads();
+
+  const int first = __ffs(streamed) - 1;
+  const int step_rr = kWarps / tiles_per_row, step_seg = kWarps % tiles_per_row;
+  int rr = warp / tiles_per_row, seg = warp % tiles_per_row;
+  for (int j = warp; j < n_tiles; j += kWarps) {
+    const size_t off = (size_t)(row_a + rr) * a.d;
+    const int base = seg * 32 * kUnroll;
+    F8 mv[kUnroll];
+    uint4 xv[kUnroll];
+    bool ok[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int ch = base + u * 32 + lane;
+      ok[u] = ch < chunks;
+      if (ok[u]) {
+        mv[u] = ld_m256(m_in + off + (size_t)ch * 8);
+        xv[u] = ld_x128(ra.xs[first] + off + (size_t)ch * 8);
+      }
+    }
+    // the reference's own sums, once per tile
+    float g_sm = 0.f, g_smm = 0.f;
+    unsigned m_diff = 0u;
+    float sum[kUnroll][8];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        sum[u][e] = 0.f;
+        if (ok[u]) {
+          const float ms = mv[u].v[e] - m0;
+          g_sm += ms;
+          g_smm = fmaf(ms, ms, g_smm);
+          m_diff |= __float_as_uint(mv[u].v[e]) ^ m0bits;
+        }
+      }
+    }
+
+    for (unsigned rem = streamed; rem != 0u;) {              // the workers, in order
+      const int r = __ffs(rem) - 1;
+      rem &= rem - 1u;
+      uint4 cur[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) cur[u] = xv[u];
+      if (rem != 0u) {                                       // the next worker's tile, ahead of the arithmetic
+        const uint16_t *xn = ra.xs[__ffs(rem) - 1] + off;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          if (ok[u]) xv[u] = ld_x128(xn + (size_t)(base + u * 32 + lane) * 8);
+      }
+      const unsigned x0 = sh.x0[r], x0pair = x0 | (x0 << 16);
+      const float x0f = __uint_as_float(x0 << 16);
+      float sx = 0.f, sxx = 0.f, sxm = 0.f, ab = 0.f;
+      unsigned flips = 0u, nf = 0u, x_diff = 0u;
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (!ok[u]) continue;
+        const unsigned w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          nf |= ((w4[q] & 0x7F807F80u) + 0x00800080u) & 0x80008000u;
+          x_diff |= w4[q] ^ x0pair;
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
+            const float mf = mv[u].v[2 * q + hlf];
+            const float xs = xf - x0f, ms = mf - m0;
+            sx += xs;
+            sxx = fmaf(xs, xs, sxx);
+            sxm = fmaf(xs, ms, sxm);
+            ab += fabsf(xf - mf);
+            const float xt = __uint_as_float(__float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u));
+            flips += (((xf == 0.f) != (mf == 0.f)) || (xt < 0.f)) ? 1u : 0u;
+            sum[u][2 * q + hlf] += xf;
+          }
+        }
+      }
+      sx = warp_sum(sx); sxx = warp_sum(sxx); sxm = warp_sum(sxm); ab = warp_sum(ab);
+      flips = __reduce_add_sync(0xffffffffu, flips);
+      nf = __reduce_or_sync(0xffffffffu, nf);
+      x_diff = __reduce_or_sync(0xffffffffu, x_diff);
+      if (lane == 0) {
+        sh.acc[warp][r][0] += (double)sx;
+        sh.acc[warp][r][1] += (double)sxx;
+        sh.acc[warp][r][2] += (double)sxm;
+        sh.acc[warp][r][3] += (double)ab;
+        sh.flips[warp][r] += flips;
+        sh.bits[warp][r] |= (nf ? (unsigned)kBitNonfinite : 0u) | (x_diff ? (unsigned)kBitXVaries : 0u);
+      }
+    }
+    g_sm = warp_sum(g_sm);
+    g_smm = warp_sum(g_smm);
+    m_diff = __reduce_or_sync(0xffffffffu, m_diff);
+    if (lane == 0) {
+      sh.m_acc[warp][0] += (double)g_sm;
+      sh.m_acc[warp][1] += (double)g_smm;
+      sh.m_varies[warp] |= m_diff;
+    }
+    // Eq. 1 with the mean over the collected workers, written where ema_mean_kernel would put it
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (!ok[u]) continue;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mv[u].v[e] = fmaf(beta, mv[u].v[e], wgt * sum[u][e]);
+      st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+    }
+    rr += step_rr;
+    seg += step_seg;
+    if (seg >= tiles_per_row) { seg -= tiles_per_row; ++rr; }
+  }
+
+  __syncthreads();
+  // warps -> CTA in a fixed order, one thread per (worker, slot word)
+  if (threadIdx.x < a.R * kSlotWords) {
+    const int r = threadIdx.x / kSlotWords, w8 = threadIdx.x - r * kSlotWords;
+    if ((streamed >> r) & 1u) {
+      unsigned long long out;
+      if (w8 < 6) {
+        double t = 0.;
+        for (int w = 0; w < kWarps; ++w)
+          t += (w8 == 0) ? sh.acc[w][r][0] : (w8 == 1) ? sh.acc[w][r][1] : (w8 == 2) ? sh.m_acc[w][0]
+             : (w8 == 3) ? sh.m_acc[w][1] : (w8 == 4) ? sh.acc[w][r][2] : sh.acc[w][r][3];
+        out = (unsigned long long)__double_as_longlong(t);
+      } else if (w8 == 6) {
+        out = 0ull;
+        for (int w = 0; w < kWarps; ++w) out += sh.flips[w][r];
+      } else {
+        out = ((unsigned long long)(b + 1) << kTagShift) | ((unsigned long long)sh.x0[r] << kX0Shift) |
+              ((unsigned long long)m0bits << kM0Shift);
+        for (int w = 0; w < kWarps; ++w) out |= sh.bits[w][r] | (sh.m_varies[w] ? kBitMVaries : 0ull);
+      }
+      ra.partials[(((size_t)r * a.G + c) * kSegsPerCta + sgm) * kSlotWords + w8] = out;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+replica_kernel(const ReplicaArgs ra) {
+  __shared__ ReplicaShared sh;
+  __shared__ int s_last;
+  extern __shared__ double s_dyn[];            // the refresh's working copies (CTA 0)
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  const StreamArgs &a = ra.s;
+  const bool warmup = (a.mode == kModeReplicaWarmup);
+  const int act = __ldcg(&a.hs->kind[a.kind].active);
+  // collected: everybody in the warm-up; afterwards whoever is neither banned nor tainted at
+  // another stage (both known before the launch: bans only change in the last CTA)
+  unsigned streamed = 0u;
+  for (int r = 0; r < a.R; ++r) {
+    const bool skip = !warmup && (__ldcg(&a.hs->banned[r]) != 0 || ((ra.tainted_in >> r) & 1u));
+    if (!skip) streamed |= 1u << r;
+  }
+
+  if (blockIdx.x == 0) {
+    KindState *ks = &a.hs->kind[a.kind];
+    if (ks->refresh_pending)
+      refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
+  } else if (streamed != 0u) {
+    const int c = blockIdx.x - 1;
+    const long long rows = (long long)a.B * a.T;
+    const long long r0 = (rows * c) / a.G, r1 = (rows * (c + 1)) / a.G;
+    long long row = r0;
+    for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
+      if (row < r1) {
+        const int b = (int)(row / a.T);
+        const long long sample_end = (long long)(b + 1) * a.T;
+        const long long row_b = sample_end < r1 ? sample_end : r1;
+        replica_segment(ra, b, row, row_b, a.ema[act], a.ema[act ^ 1], streamed, c, sgm, sh);
+        row = row_b;
+      } else if (threadIdx.x < a.R) {
+        ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + sgm) * kSlotWords + 7] = 0ull;   // unused
+      }
+    }
+  }
+
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(a.ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // the worker loop: scores, test, counters, history, one worker after the other
+  const int rows = a.B + 1;
+  for (int r = 0; r < a.R; ++r) {
+    const FinalizeTarget ft = {r, ra.partials + (size_t)r * a.G * kSegsPerCta * kSlotWords,
+                               ra.scores_all + (size_t)r * rows * a.n_metrics,
+                               ra.flags_all ? ra.flags_all + (size_t)r * rows : nullptr,
+                               ra.sw_all ? ra.sw_all + (size_t)r * rows : nullptr,
+                               (!warmup && ((ra.tainted_in >> r) & 1u)) ? 1 : 0, r == a.R - 1};
+    finalize(a, ft);
+    __threadfence();                           // the next pass reads the state this one wrote
+    __syncthreads();
+  }
+  // nobody flagged: the mean over all collected workers is already in the spare buffer
+  if (threadIdx.x == 0) {
+    KindState *ks = &a.hs->kind[a.kind];
+    const unsigned collected = __ldcg(&ks->step_collected), tainted = __ldcg(&ks->step_tainted);
+    if (collected != 0u && tainted == 0u) {
+      ks->active = act ^ 1;
+      ks->mean_done_step = __ldcg(&ks->steps);
+    }
+  }
 }
 
 // Brings both kinds' thresholds up to date outside a streaming launch (queries, export).
@@ -1006,12 +1283,15 @@ replace_kernel(const HandleState *hs, int kind, const float *ema0, const float *
 }
 
 // Second half of a multi-worker iteration (Alg. 1 main loop, Eq. 1): after every worker has
-// been scored, decide who is tainted -- the flagged workers, unless more than half of the
-// workers still in the pool were flagged, which Alg. 2 reads as a natural distribution shift
-// and clears -- and move the reference with the mean over the others, in place:
+// been scored, decide who is tainted -- the flagged workers and, for gradients (Alg. 3), the
+// ones tainted at another stage, unless more than half of the workers still in the pool are in
+// that set, which Alg. 2 / Alg. 3 read as a natural distribution shift and clear -- and move the
+// reference with the mean over the clean collected workers, in place:
 //   m <- beta m + (1 - beta) / |clean| * sum_{r clean} x^(r).
-// Every CTA derives the same clean set from the masks the scoring launches left in the state.
-// Traffic: 4 B read + 4 B written of m and 2 B per clean worker, per element.
+// When nobody was flagged the scoring launch has already put that mean in place (it marks the
+// iteration in mean_done_step) and only the report bits are left to do here.
+// Every CTA derives the same clean set from the masks the scoring launch left in the state.
+// Traffic when it runs: 4 B read + 4 B written of m and 2 B per clean worker, per element.
 struct WorkerPointers { const uint16_t *x[kMaxWorkers]; };
 
 __global__ void __launch_bounds__(kReplaceThreads)
@@ -1022,17 +1302,19 @@ ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, float *ema0, float
   const unsigned collected = ks->step_collected, tainted = ks->step_tainted, nonfinite = ks->step_nonfinite;
   int n_banned = 0;
   for (int r = 0; r < R; ++r) n_banned += hs->banned[r] != 0;
-  const bool natural = !warmup && 2 * __popc(tainted) > R - n_banned;
+  const int n_stage = __popc(tainted) + (kind == 1 ? __popc(ks->step_elsewhere) : 0);   // the stage's tainted set
+  const bool natural = !warmup && 2 * n_stage > R - n_banned;
   const unsigned clean = collected & ~(natural ? nonfinite : tainted);
   const int n_clean = __popc(clean);
+  const bool done = ks->mean_done_step == ks->steps;
 
   if (blockIdx.x == 0 && threadIdx.x == 0) {
-    ks->last_flagged = (tainted != 0u && !natural) ? 1 : 0;
+    ks->last_flagged = (n_stage != 0 && !natural) ? 1 : 0;
     if (flags_out)
       for (int r = 0; r < R; ++r)
         flags_out[(size_t)r * rows] |= ((clean >> r) & 1u ? kFlagCommitted : 0u) | (natural ? kFlagNaturalShift : 0u);
   }
-  if (n_clean == 0) return;
+  if (n_clean == 0 || done) return;
   float *m = ks->active ? ema1 : ema0;
   const float wgt = one_minus_beta / (float)n_clean;
   const long long stride = (long long)gridDim.x * kReplaceThreads;
@@ -1053,6 +1335,13 @@ ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, float *ema0, float
     for (int j = 0; j < 8; ++j) mv.v[j] = fmaf(beta, mv.v[j], wgt * sum[j]);
     st_m256(m + c * 8, mv);
   }
+}
+
+// The one worker this verifier follows was tainted at another stage in this step: nothing is
+// collected or recorded; the step counts and asks for gradient replacement (Alg. 4).
+__global__ void skip_tainted_kernel(HandleState *hs, int kind) {
+  hs->kind[kind].steps += 1;
+  hs->kind[kind].last_flagged = 1;
 }
 
 __global__ void reset_worker_kernel(HandleState *hs, int worker) {

@@ -144,3 +144,100 @@ def test_argument_checks(sb):
     assert L.sentinel_verify_replicas(v._h, good, 0, 2, 4, 16, s, scores.data_ptr(), flags.data_ptr()) == sb.OK
     torch.cuda.synchronize()
     v.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# workers tainted at another stage (Sec. 3.1, cascading effects; Alg. 2 / Alg. 3)
+
+def step_both_tainted(gv, ov, xs, kind, mask):
+    gx = [None if (mask >> r) & 1 else x for r, x in enumerate(xs)]
+    gs, gf = gv.step_replicas(gx, kind, False, tainted_in=mask)
+    os_, of, n = ov.step_replicas([None if x is None else synth.bits(x) for x in gx], kind, False, tainted_in=mask)
+    torch.cuda.synchronize()
+    return gs.cpu().numpy(), gf.cpu().numpy().view(np.uint32), os_, of, n
+
+
+@pytest.mark.parametrize("kind", [ACT, GRAD], ids=["act", "grad"])
+def test_workers_tainted_elsewhere(sb, oracle_mod, kind):
+    """Not collected, reported, out of the mean; for gradients part of the stage's tainted set
+    (majority rule, verdict for Alg. 4), for activations not."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "tainted_in", 3, 24, 264)
+    R = 4
+    gv, ov, params = pair(sb, oracle_mod, w, R, l=6, c=2)
+    for t in range(10):
+        step_both(gv, ov, inputs(w, R, kind, t), kind, warmup=True)
+    plan = [(0b0000, {}), (0b0010, {}), (0b1100, {0: 6.0}), (0b0001, {}), (0b0000, {3: 6.0}), (0b0000, {3: 6.0}),
+            (0b1000, {}), (0b1111, {}), (0b0000, {})]
+    for t, (mask, scale) in enumerate(plan, start=10):
+        xs = inputs(w, R, kind, t, scale)
+        thr, valid = ov.thresholds(kind)
+        gs, gf, os_, of, n = step_both_tainted(gv, ov, xs, kind, mask)
+        for r in range(R):
+            assert_scores_close(gs[r], os_[r], float(xs[r].float().abs().mean()), "step %d worker %d" % (t, r))
+        if not np.array_equal(gf, of):
+            for r in range(R):
+                near = near_threshold(os_[r], thr, valid, w.B)
+                assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            gv.sentinel_import_state(oracle_to_blob(ov, params))
+        ev = whole_step_k_events(*gv.sentinel_get_thresholds(kind), *ov.thresholds(kind), params, kind)
+        if ev:
+            gv.sentinel_import_state(oracle_to_blob(ov, params))
+        # the verdict Alg. 4 acts on
+        probe = xs[0].clone()
+        replaced = torch.zeros(1, dtype=torch.int32, device="cuda")
+        gv.sentinel_replace_if_flagged(probe, kind, 0, replaced)
+        torch.cuda.synchronize()
+        assert bool(replaced.item()) == ov.replace_if_flagged(synth.bits(xs[0]), kind)[1], (t, mask)
+        check_state(gv, ov, params, kinds=(kind,))
+    assert ov.worker_counters(3)[2] == 1                    # banned on the way; its bit then changes nothing
+    gv.close()
+
+
+def test_tainted_in_argument_checks(sb):
+    gv = sb.Verifier(2, 8, 64, n_workers=3)
+    x = torch.zeros(2, 8, 64, dtype=torch.bfloat16, device="cuda")
+    s, f = torch.zeros(3, 3, 3, device="cuda"), torch.zeros(3, 3, dtype=torch.int32, device="cuda")
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_verify_replicas_tainted([x, x, x], ACT, 0b1000, s, f)     # worker 3 does not exist
+    assert e.value.code == sb.ERR_INVALID_ARG
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_verify_replicas_tainted([x, None, x], ACT, 0b0000, s, f)  # collected, but no tensor
+    assert e.value.code == sb.ERR_INVALID_ARG
+    gv.sentinel_verify_replicas_tainted([x, None, x], ACT, 0b0010, s, f)
+    torch.cuda.synchronize()
+    assert int(f[1, 0].item()) & sb.FLAG_TAINTED_ELSEWHERE
+    gv.close()
+
+
+def test_skip_tainted_single_submission(sb, oracle_mod):
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "skip", 2, 16, 128)
+    gv = sb.Verifier(w.B, w.T, w.d)
+    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d))
+    for t in range(14):
+        x = synth.clean(w, 0, GRAD, t, "cuda")
+        gv.update_reference(x, GRAD)
+        ov.update_reference(synth.bits(x), GRAD)
+    before = bytes(gv.sentinel_export_state())
+    gv.sentinel_skip_tainted(GRAD)
+    ov.skip_tainted(GRAD)
+    st0 = parse_blob(before, w.B, w.T, w.d, 100)
+    st1 = parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, 100)
+    assert st1["kinds"][GRAD]["steps"] == st0["kinds"][GRAD]["steps"] + 1 == ov.steps(GRAD)
+    assert np.array_equal(st1["kinds"][GRAD]["m"], st0["kinds"][GRAD]["m"])
+    assert all(np.array_equal(a, b) for a, b in zip(st1["kinds"][GRAD]["hist"][0], st0["kinds"][GRAD]["hist"][0]))
+    assert (st1["violations"], st1["clean_streak"], st1["banned"]) == ov.counters()
+    g = synth.clean(w, 0, GRAD, 15, "cuda")
+    out = g.clone()
+    replaced = torch.zeros(1, dtype=torch.int32, device="cuda")
+    gv.sentinel_replace_if_flagged(out, GRAD, 0, replaced)
+    torch.cuda.synchronize()
+    want, did = ov.replace_if_flagged(synth.bits(g), GRAD)
+    assert did and replaced.item() == 1
+    got = synth.bits(out)
+    assert np.mean(got != want) <= 1e-3                     # fp32 reference vs float64, then one rounding
+    gs, gf = gv.verify(g, GRAD)
+    assert int(gf[0].item()) & sb.FLAG_COMMITTED
+    gv.sentinel_replace_if_flagged(out, GRAD, 0, replaced)
+    torch.cuda.synchronize()
+    assert replaced.item() == 0
+    gv.close()
