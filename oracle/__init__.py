@@ -57,7 +57,7 @@ class _Params(C.Structure):
         ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
         ("l", C.c_int), ("c", C.c_int), ("t_forgiveness", C.c_int),
         ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
-        ("R", C.c_int),
+        ("R", C.c_int), ("ema_bf16", C.c_int),
     ]
 
 
@@ -168,6 +168,7 @@ class Params:
     t_forgiveness: int = 100
     metric_mask: int = 15
     R: int = 1
+    ema_bf16: int = 0
 
     def to_c(self) -> _Params:
         p = _Params()
@@ -180,6 +181,7 @@ class Params:
         p.metric_mask = self.metric_mask
         p.B, p.T, p.d = self.B, self.T, self.d
         p.R = self.R
+        p.ema_bf16 = self.ema_bf16
         return p
 
 

@@ -62,6 +62,7 @@ void so_default_params(so_params *p) {
   p->metric_mask = 15u;
   p->B = 1; p->T = 1; p->d = 8;
   p->R = 1;
+  p->ema_bf16 = 0;
 }
 
 /* ------------------------------------------------------------------------------------ */
@@ -277,6 +278,7 @@ static void window_push(so_window *w, double val) {
 
 so_verifier *so_create(const so_params *p) {
   if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1 || p->R < 1 || p->R > SO_MAX_WORKERS) return NULL;
+  if (p->ema_bf16 && p->R != 1) return NULL;   /* the bf16 reference exists for one submission per update */
   so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
   v->p = *p;
   v->Ns = (size_t)p->T * (size_t)p->d;
@@ -301,7 +303,7 @@ so_verifier *so_create(const so_params *p) {
 }
 
 int so_set_directions(so_verifier *v, const uint16_t *u, int n_dir) {
-  if (n_dir < 1 || !u) return -1;
+  if (n_dir < 1 || !u || v->p.ema_bf16) return -1;
   if (v->ks[0].steps || v->ks[1].steps) return -1;   /* the metric set is fixed before the first step */
   free(v->u);
   v->u = (uint16_t *)malloc((size_t)n_dir * (size_t)v->p.d * sizeof(uint16_t));
@@ -356,6 +358,15 @@ static void refresh_thresholds(so_verifier *v, int kind) {
 static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
   double *m = v->ks[kind].m;
   const double beta = v->p.beta[kind];
+  if (v->p.ema_bf16) {
+    /* The reference is stored as bf16.  Which of two neighbouring bf16 values an element takes
+     * is a decision of the arithmetic, so it is taken in the arithmetic of the stored format's
+     * producer: single precision, one fused multiply-add, then one rounding to nearest even. */
+    const float bf = (float)beta, of = (float)(1.0 - beta);
+    for (size_t e = 0; e < v->N; ++e)
+      m[e] = so_bf16(so_bf16_round((double)fmaf(bf, (float)m[e], of * (float)so_bf16(x[e]))));
+    return;
+  }
   for (size_t e = 0; e < v->N; ++e) m[e] = beta * m[e] + (1.0 - beta) * so_bf16(x[e]);
 }
 
@@ -587,6 +598,8 @@ const double *so_ema(const so_verifier *v, int kind) { return v->ks[kind].m; }
 
 void so_set_ema(so_verifier *v, int kind, const double *m) {
   memcpy(v->ks[kind].m, m, v->N * sizeof(double));
+  if (v->p.ema_bf16)
+    for (size_t e = 0; e < v->N; ++e) v->ks[kind].m[e] = so_bf16(so_bf16_round(m[e]));
 }
 
 size_t so_history(const so_verifier *v, int kind, int level, int metric, double *out, size_t cap) {

@@ -63,6 +63,7 @@ typedef struct so_params {
   unsigned metric_mask;    /* which metrics may raise a flag (bit i = metric i)     */
   int    B, T, d;          /* submission shape                                      */
   int    R;                /* workers (replicas) feeding this boundary, d_s >= 1    */
+  int    ema_bf16;         /* != 0: the reference is stored as bf16 (R = 1 only)    */
 } so_params;
 
 typedef struct so_verifier so_verifier;

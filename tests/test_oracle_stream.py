@@ -569,3 +569,72 @@ def test_directions_are_refused_after_the_first_step(oracle_mod):
     v.update_reference(to_bits(rs.normal(0, 1, (2, 4, 8))), GRAD)
     with pytest.raises(RuntimeError):
         v.set_directions(_directions(rs, 4, 8))
+
+
+# ---------------------------------------------------------------------------------------------
+# the reference stored as bf16
+
+def _as_bf16_f32(a32):
+    """float32 -> nearest bf16 (ties to even) -> float32, by torch's conversion."""
+    return torch.from_numpy(np.ascontiguousarray(a32, dtype=np.float32)).to(torch.bfloat16).float().numpy()
+
+
+def test_bf16_reference_is_the_single_precision_update_rounded_once(oracle_mod):
+    """m_t = bf16(fma(beta, m_{t-1}, (1-beta)*x)) in float32.  Expected values: the product and
+    the fused sum formed exactly in float64 (24-bit times 8-bit and 24-bit operands) and rounded
+    to float32, then torch's float32 -> bfloat16 conversion."""
+    rs = np.random.default_rng(31)
+    v = make(oracle_mod, B=2, T=6, d=16, ema_bf16=1)
+    beta32, omb32 = np.float32(0.9), np.float32(1.0 - 0.9)
+    m = np.zeros((2, 6, 16), dtype=np.float32)
+    for t in range(12):
+        xb = to_bits(rs.normal(0.2, 1.5, (2, 6, 16)))
+        x32 = from_bits(xb).astype(np.float32)
+        v.update_reference(xb, ACT)
+        prod = (omb32.astype(np.float64) * x32.astype(np.float64)).astype(np.float32)
+        fused = (np.float64(beta32) * m.astype(np.float64) + prod.astype(np.float64)).astype(np.float32)
+        m = _as_bf16_f32(fused)
+        got = v.ema(ACT)
+        assert np.array_equal(got, m.astype(np.float64)), t
+    assert np.all(v.ema(GRAD) == 0.0)
+
+
+def test_bf16_reference_scores_use_the_rounded_reference(oracle_mod):
+    rs = np.random.default_rng(32)
+    v = make(oracle_mod, B=2, T=4, d=8, ema_bf16=1)
+    for t in range(5):
+        v.update_reference(to_bits(rs.normal(0, 1, (2, 4, 8))), GRAD)
+    m = v.ema(GRAD).copy()
+    assert np.array_equal(from_bits(to_bits(m)), m)          # every entry is a bf16 value
+    xb = to_bits(rs.normal(0, 1, (2, 4, 8)))
+    scores, _, _ = v.verify(xb, GRAD)
+    want, _, _ = oracle_mod.distance(xb, m)
+    assert np.array_equal(scores[0], want)
+
+
+def test_bf16_reference_settles_within_a_few_ulps_of_a_constant_input(oracle_mod):
+    """With x fixed the update stalls once (1-beta)|x - m| drops below half a bf16 ulp of m:
+    the reference ends within 1/(2(1-beta)) = 5 ulps (each at most 2^-7 relative) of x."""
+    rs = np.random.default_rng(33)
+    v = make(oracle_mod, B=1, T=8, d=16, ema_bf16=1)
+    xb = to_bits(rs.normal(0, 1, (1, 8, 16)) + 3.0)
+    x = from_bits(xb)
+    for t in range(200):
+        v.update_reference(xb, ACT)
+    m1 = v.ema(ACT).copy()
+    v.update_reference(xb, ACT)
+    assert np.array_equal(v.ema(ACT), m1)                    # a fixed point
+    assert np.all(np.abs(m1 - x) <= 5.5 * 2.0 ** -7 * np.abs(x))
+    assert np.any(m1 != x)                                   # and it is not x itself everywhere
+
+
+def test_bf16_reference_is_for_single_submissions_without_directions(oracle_mod):
+    with pytest.raises(ValueError):
+        make(oracle_mod, ema_bf16=1, R=2)
+    v = make(oracle_mod, ema_bf16=1)
+    with pytest.raises(RuntimeError):
+        v.set_directions(_directions(np.random.default_rng(1), 4, 8))
+    rs = np.random.default_rng(34)
+    m = rs.normal(0, 1, (2, 4, 8))
+    v.set_ema(ACT, m)
+    assert np.array_equal(v.ema(ACT), from_bits(to_bits(m)))  # stored rounded
