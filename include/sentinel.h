@@ -95,11 +95,21 @@ typedef struct sentinel_config {
                               unless only the _strided entry points are used              */
   int    device;           /* CUDA device ordinal                                           */
   int    n_workers;        /* workers d_s feeding this boundary (multi-worker calls)   1    */
+  int    ema_bf16;         /* 1: the reference is stored as bf16 (see below)           0    */
 } sentinel_config;
 
 typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundary */
 
 /* Fills *cfg with the defaults above; B = T = d = 0 and device = 0 are left for the caller. */
+/* ema_bf16 = 1 keeps the reference as bf16 instead of fp32: a verified tensor then moves
+ * 2 B (x) + 2 B (reference read) + 2 B (candidate written) = 6 B per element instead of 10, and
+ * the state takes half the memory.  The paper does not fix the reference's precision; with bf16
+ * the update is m_t = bf16(fma(beta, m_{t-1}, (1-beta) x)) in single precision with one
+ * rounding to nearest even, so a reference stops moving once (1-beta)|x - m| falls below half
+ * a bf16 ulp of m (it settles within 1/(2(1-beta)) ulps of a steady input).  Scores, bounds and
+ * flags are computed exactly as with fp32, against the rounded reference.  Restrictions:
+ * n_workers = 1, no sentinel_set_directions.  State blobs carry the reference as fp32 either
+ * way (widened exactly on export, rounded to nearest even on import). */
 int sentinel_default_config(sentinel_config *cfg);
 
 /* Allocates the state of one boundary on cfg->device: two fp32 [B,T,d] buffers per kind (the

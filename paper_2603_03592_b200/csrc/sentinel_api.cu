@@ -57,7 +57,9 @@ struct sentinel_verifier {
   uint16_t *sw_u = nullptr;         // directions, bf16 [sw_L][d]
   float *sw_scratch = nullptr;      // projections and sorted lists
   float *sw_out = nullptr;          // [1+B] distances of the submission being checked
-  float *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
+  void *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // fp32, or bf16 if bf16
+  bool bf16 = false;                // the reference is stored as bf16
+  size_t ema_bytes = 0;             // bytes of one reference buffer
   HandleState *hs = nullptr;
   double *hist[2] = {nullptr, nullptr};      // rings, device layout (ring_offset)
   double *sorted[2] = {nullptr, nullptr};    // ascending copies of the windows (sorted_offset)
@@ -125,7 +127,7 @@ int streaming_ctas(int device, int B, int T, std::string *err) {
   int sms = 0, occ = 0;
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess)
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, stream_kernel_t<false>, kThreads, 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, stream_kernel_t<false, false>, kThreads, 0);
   if (e != cudaSuccess || sms < 1 || occ < 1) {
     if (err) *err = std::string("occupancy query failed: ") + cudaGetErrorString(e);
     return -1;
@@ -223,6 +225,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.ban_violations = h->cfg.ban_violations;
   a.forgiveness_steps = h->cfg.forgiveness_steps;
   a.metric_mask = h->cfg.metric_mask;
+  a.ema_bf16 = h->bf16 ? 1 : 0;
   a.n_metrics = h->n_metrics;
   a.sw = h->sw_out;                 // nullptr until directions are set
   return a;
@@ -242,8 +245,13 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
   attr.val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = &attr;
   lc.numAttrs = 1;
-  if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true>, a));
-  else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false>, a));
+  if (h->bf16) {
+    if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, true>, a));
+    else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, true>, a));
+  } else {
+    if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, false>, a));
+    else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, false>, a));
+  }
   return SENTINEL_OK;
 }
 
@@ -340,7 +348,8 @@ int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bo
   if (!h->sw_u) return SENTINEL_OK;
   int sms = 0;
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
-  SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), h->ema[kind][0], h->ema[kind][1], &h->hs->kind[kind].active,
+  SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), static_cast<const float *>(h->ema[kind][0]),
+                           static_cast<const float *>(h->ema[kind][1]), &h->hs->kind[kind].active,
                            may_skip ? &h->hs->banned[worker] : nullptr, h->sw_u, h->sw_L, h->cfg.B, h->cfg.T,
                            h->cfg.d, sms, h->sw_scratch, h->sw_out + (size_t)worker * (1 + h->cfg.B), s));
   return SENTINEL_OK;
@@ -405,6 +414,9 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "window_steps, ban_violations, forgiveness_steps, severe_mult must be positive");
   if (cfg->n_workers < 1 || cfg->n_workers > SENTINEL_MAX_WORKERS)
     return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "n_workers = %d is outside 1..%d", cfg->n_workers, SENTINEL_MAX_WORKERS);
+  if (cfg->ema_bf16 != 0 && cfg->ema_bf16 != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ema_bf16 must be 0 or 1, got %d", cfg->ema_bf16);
+  if (cfg->ema_bf16 && cfg->n_workers != 1)
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "the bf16 reference is kept for single submissions only (n_workers = 1)");
   if ((long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*n_workers*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d",
                 (long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1), SENTINEL_MAX_WINDOW);
@@ -421,6 +433,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->Ns = (size_t)cfg->T * cfg->d;
   h->N = h->Ns * cfg->B;
   h->R = cfg->n_workers;
+  h->bf16 = cfg->ema_bf16 != 0;
+  h->ema_bytes = h->N * (h->bf16 ? sizeof(uint16_t) : sizeof(float));
   h->units0 = h->R;                       // the window spans window_steps iterations of all workers
   h->units1 = h->R * cfg->B;
   h->cap0 = cfg->window_steps * h->units0;
@@ -433,8 +447,10 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   }
   {   // the windows' working copies may exceed the 48 KiB a kernel gets without asking
     const int most = 200 * 1024;
-    cudaError_t ae = cudaFuncSetAttribute(stream_kernel_t<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaError_t ae = cudaFuncSetAttribute(stream_kernel_t<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
@@ -449,7 +465,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (e == cudaSuccess) e = cudaMemset(*p, 0, bytes);
   };
   for (int k = 0; k < 2; ++k) {
-    for (int j = 0; j < 2; ++j) alloc((void **)&h->ema[k][j], h->N * sizeof(float));   // m_0 = 0
+    for (int j = 0; j < 2; ++j) alloc(&h->ema[k][j], h->ema_bytes);   // m_0 = 0 (all-zero bits in either format)
     alloc((void **)&h->hist[k], ring_doubles(h) * sizeof(double));
     alloc((void **)&h->sorted[k], hist_doubles(h) * sizeof(double));
     alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
@@ -588,7 +604,7 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   a.x_row_stride = d;
   a.n_metrics = 3;
   a.mode = kModeDistance;
-  stream_kernel_t<false><<<G + 1, kThreads, 0, s>>>(a);
+  stream_kernel_t<false, false><<<G + 1, kThreads, 0, s>>>(a);
   cudaError_t le = cudaGetLastError();
   cudaError_t fe = cudaFreeAsync(scratch, s);
   SENTINEL_CUDA(nullptr, le);
@@ -661,7 +677,7 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigne
   const long long need = (n_chunks + kReplaceThreads - 1) / kReplaceThreads;
   if (grid > need) grid = need;
   ema_mean_kernel<<<(unsigned)grid, kReplaceThreads, 0, s>>>(
-      h->hs, kind, wp, h->ema[kind][0], h->ema[kind][1], n_chunks, h->R, (int)rows, (float)h->cfg.beta[kind],
+      h->hs, kind, wp, static_cast<float *>(h->ema[kind][0]), static_cast<float *>(h->ema[kind][1]), n_chunks, h->R, (int)rows, (float)h->cfg.beta[kind],
       (float)(1.0 - h->cfg.beta[kind]), warmup ? 1 : 0, flags);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
@@ -713,7 +729,7 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
   const long long need = (n_chunks + kReplaceThreads - 1) / kReplaceThreads;
   if (grid > need) grid = need;
   replace_kernel<<<(unsigned)grid, kReplaceThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], static_cast<uint16_t *>(dev_x_inout), n_chunks, fill,
+      h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], h->bf16 ? 1 : 0, static_cast<uint16_t *>(dev_x_inout), n_chunks, fill,
       dev_replaced_out);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
@@ -723,6 +739,7 @@ int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L,
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (!dev_u_bf16) return fail(h, SENTINEL_ERR_INVALID_ARG, "u is NULL");
   if (h->started) return fail(h, SENTINEL_ERR_INVALID_ARG, "the metric set is fixed once a step was taken or a state imported");
+  if (h->bf16) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads an fp32 reference: not available with ema_bf16");
   if (h->cfg.d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", h->cfg.d);
   int rc = check_swd_shape(h, L, h->cfg.T, h->cfg.d);
   if (rc) return rc;
@@ -925,8 +942,18 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
       }
     }
     out = reinterpret_cast<unsigned char *>(dst);
-    SENTINEL_CUDA(h, cudaMemcpyAsync(out, h->ema[k][ks.active], h->N * sizeof(float), cudaMemcpyDeviceToHost, s));
-    SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+    if (h->bf16) {                                  // the blob always carries fp32: widen (exact)
+      std::vector<uint16_t> half(h->N);
+      SENTINEL_CUDA(h, cudaMemcpyAsync(half.data(), h->ema[k][ks.active], h->ema_bytes, cudaMemcpyDeviceToHost, s));
+      SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+      for (size_t e = 0; e < h->N; ++e) {
+        const unsigned bits = (unsigned)half[e] << 16;
+        memcpy(out + e * sizeof(float), &bits, sizeof bits);
+      }
+    } else {
+      SENTINEL_CUDA(h, cudaMemcpyAsync(out, h->ema[k][ks.active], h->N * sizeof(float), cudaMemcpyDeviceToHost, s));
+      SENTINEL_CUDA(h, cudaStreamSynchronize(s));
+    }
     out += h->N * sizeof(float);
   }
   return SENTINEL_OK;
@@ -1000,7 +1027,19 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
       SENTINEL_CUDA(h, cudaStreamSynchronize(s));     // the staging vectors go out of scope
     }
     p += hist_doubles(h) * sizeof(double);
-    SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], p, h->N * sizeof(float), cudaMemcpyHostToDevice, s));
+    if (h->bf16) {                                  // narrow, to nearest even (exact for a bf16 verifier's own blob)
+      std::vector<uint16_t> half(h->N);
+      for (size_t e = 0; e < h->N; ++e) {
+        unsigned bits;
+        memcpy(&bits, p + e * sizeof(float), sizeof bits);
+        if ((bits & 0x7F800000u) != 0x7F800000u) bits += 0x7FFFu + ((bits >> 16) & 1u);
+        half[e] = (uint16_t)(bits >> 16);
+      }
+      SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], half.data(), h->ema_bytes, cudaMemcpyHostToDevice, s));
+      SENTINEL_CUDA(h, cudaStreamSynchronize(s));     // the staging vector goes out of scope
+    } else {
+      SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], p, h->N * sizeof(float), cudaMemcpyHostToDevice, s));
+    }
     p += h->N * sizeof(float);
   }
   SENTINEL_CUDA(h, cudaMemcpyAsync(h->hs, &st, sizeof st, cudaMemcpyHostToDevice, s));
@@ -1082,7 +1121,7 @@ int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int 
   a.x_row_stride = d;
   a.n_metrics = 3;
   a.mode = kModeDistance;
-  stream_kernel_t<false><<<G + 1, kThreads, 0, s>>>(a);
+  stream_kernel_t<false, false><<<G + 1, kThreads, 0, s>>>(a);
   SENTINEL_CUDA(nullptr, cudaGetLastError());
   return SENTINEL_OK;
 }

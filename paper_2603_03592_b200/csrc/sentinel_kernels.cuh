@@ -85,7 +85,7 @@ struct HandleState {
 struct StreamArgs {
   const uint16_t *x;               // bf16 [B,T,d]
   const float *m_ext;              // distance mode: caller's reference; else unused
-  float *ema[2];                   // the two reference buffers of this kind
+  void *ema[2];                    // the two reference buffers of this kind: fp32, or bf16 if ema_bf16
   HandleState *hs;                 // nullptr in distance mode
   double *hist;                    // this kind's rings: level 0 [4][cap0+units0], level 1 [4][cap1+units1]
   double *sorted;                  // the same windows kept ascending: [4][cap0], [4][cap1]
@@ -102,7 +102,8 @@ struct StreamArgs {
   float beta, one_minus_beta;
   int cap0, cap1;
   int units0, units1;              // entries one iteration can append per level: R and R*B
-  int R, pad3;                     // workers of the stage
+  int R;                           // workers of the stage
+  int ema_bf16;                    // the reference is stored as bf16 (single submissions only)
   long long x_row_stride;          // elements from one row of x to the next (d when dense)
   const float *sw;                 // [1+B] sliced Wasserstein distance of every unit, computed by the
                                    // launches before this one; nullptr when n_metrics = 3
@@ -137,6 +138,50 @@ __device__ __forceinline__ void st_m256(float *p, const F8 &r) {
   asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]),
                   "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7]) : "memory");
+}
+
+// The reference as the kernels see it: 8 consecutive elements as floats, whatever the storage.
+// A bf16 reference is widened on load and rounded to nearest even (cvt.rn) on store.
+__device__ __forceinline__ unsigned pack_bf16x2_rn(float lo, float hi) {
+  unsigned r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // upper half <- first operand
+  return r;
+}
+template <bool kBf16>
+__device__ __forceinline__ F8 load_m8(const void *m, size_t idx) {
+  if (kBf16) {
+    const uint4 v = ld_x128(static_cast<const uint16_t *>(m) + idx);
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    F8 r;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      r.v[2 * j] = __uint_as_float(w[j] << 16);
+      r.v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    }
+    return r;
+  }
+  return ld_m256(static_cast<const float *>(m) + idx);
+}
+template <bool kBf16>
+__device__ __forceinline__ void store_m8(void *m, size_t idx, const F8 &r) {
+  if (kBf16) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(static_cast<uint16_t *>(m) + idx), "r"(pack_bf16x2_rn(r.v[0], r.v[1])),
+                    "r"(pack_bf16x2_rn(r.v[2], r.v[3])), "r"(pack_bf16x2_rn(r.v[4], r.v[5])),
+                    "r"(pack_bf16x2_rn(r.v[6], r.v[7])) : "memory");
+  } else {
+    st_m256(static_cast<float *>(m) + idx, r);
+  }
+}
+template <bool kBf16>
+__device__ __forceinline__ float load_m1(const void *m, size_t idx) {
+  if (kBf16) return __uint_as_float((unsigned)static_cast<const uint16_t *>(m)[idx] << 16);
+  return static_cast<const float *>(m)[idx];
+}
+template <bool kBf16>
+__device__ __forceinline__ void store_m1(void *m, size_t idx, float v) {
+  if (kBf16) static_cast<uint16_t *>(m)[idx] = (uint16_t)(pack_bf16x2_rn(v, 0.f) & 0xFFFFu);
+  else static_cast<float *>(m)[idx] = v;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -227,9 +272,9 @@ constexpr int kSegsPerCta = 2;
 // appendix): rows of x are row_stride elements apart and start on any 2-byte boundary, and d
 // need not be a multiple of 8.  Lanes then own interleaved columns (col = tile + q*32 + lane),
 // so that every 2-byte / 4-byte access of a warp is contiguous; the arithmetic is the same.
-template <bool kScalar>
+template <bool kScalar, bool kBf16>
 __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long long rb,
-                               const float *m_in, float *m_out,
+                               const void *m_in, void *m_out,
                                unsigned long long (*s_part)[kSlotWords],
                                unsigned long long *slot) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -243,7 +288,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
 
   const unsigned x0 = a.x[(size_t)b * a.T * (size_t)a.x_row_stride];
   const unsigned x0pair = x0 | (x0 << 16);
-  const unsigned m0bits = __float_as_uint(m_in[sample_off]);
+  const unsigned m0bits = __float_as_uint(load_m1<kBf16>(m_in, sample_off));
 
   ThreadAcc t = {0., 0., 0., 0., 0., 0., 0u, 0u, 0u, 0u};
 
@@ -266,7 +311,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
 #pragma unroll
       for (int q = 0; q < kPerLane; ++q) {
         const int col = col0 + q * 32;
-        if (col < a.d) { xs[q] = a.x[off_x + col]; ms[q] = m_in[off + col]; }
+        if (col < a.d) { xs[q] = a.x[off_x + col]; ms[q] = load_m1<kBf16>(m_in, off + col); }
       }
 #pragma unroll
       for (int q = 0; q < kPerLane; ++q) {
@@ -278,7 +323,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
           t.m_diff |= __float_as_uint(ms[q]) ^ m0bits;
           const float xf = __uint_as_float(xb << 16);
           element(xf, ms[q], x0f, m0f, g);
-          if (write_ema) m_out[off + col] = fmaf(beta, ms[q], omb * xf);
+          if (write_ema) store_m1<kBf16>(m_out, off + col, fmaf(beta, ms[q], omb * xf));
         }
       }
     } else {
@@ -291,14 +336,14 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
         ok[u] = c < chunks;
         if (ok[u]) {
           xv[u] = ld_x128(a.x + off + (size_t)c * 8);
-          mv[u] = ld_m256(m_in + off + (size_t)c * 8);
+          mv[u] = load_m8<kBf16>(m_in, off + (size_t)c * 8);
         }
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         if (ok[u]) {
           chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
-          if (write_ema) st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+          if (write_ema) store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
         }
       }
     }
@@ -379,8 +424,8 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
   }
 }
 
-template <bool kScalar>
-__device__ void stream_cta(const StreamArgs &a, int c, const float *m_in, float *m_out,
+template <bool kScalar, bool kBf16>
+__device__ void stream_cta(const StreamArgs &a, int c, const void *m_in, void *m_out,
                            unsigned long long (*s_part)[kSlotWords]) {
   const long long R = (long long)a.B * a.T;
   const long long R0 = (R * c) / a.G, R1 = (R * (c + 1)) / a.G;
@@ -391,7 +436,7 @@ __device__ void stream_cta(const StreamArgs &a, int c, const float *m_in, float 
       const int b = (int)(ra / a.T);
       const long long sample_end = (long long)(b + 1) * a.T;
       const long long rb = sample_end < R1 ? sample_end : R1;
-      stream_segment<kScalar>(a, b, ra, rb, m_in, m_out, s_part, slot);
+      stream_segment<kScalar, kBf16>(a, b, ra, rb, m_in, m_out, s_part, slot);
       ra = rb;
     } else if (threadIdx.x == 0) {
       slot[7] = 0ull;                   // tag 0: unused
@@ -915,7 +960,7 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
 // thresholds in view, and finalizes.  No CTA ever waits for another.
 // (kScalar = true is the variant for rows of x that are strided or not 16-byte aligned; it is a
 // kernel of its own so that the vector path keeps its registers)
-template <bool kScalar>
+template <bool kScalar, bool kBf16>
 __global__ void __launch_bounds__(kThreads)
 stream_kernel_t(const StreamArgs a) {
   __shared__ unsigned long long s_part[kWarps][kSlotWords];
@@ -928,8 +973,8 @@ stream_kernel_t(const StreamArgs a) {
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  const float *m_in;
-  float *m_out;
+  const void *m_in;
+  void *m_out;
   if (a.mode == kModeDistance) {
     m_in = a.m_ext;
     m_out = nullptr;
@@ -946,7 +991,7 @@ stream_kernel_t(const StreamArgs a) {
         refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
     }
   } else {
-    stream_cta<kScalar>(a, blockIdx.x - 1, m_in, m_out, s_part);
+    stream_cta<kScalar, kBf16>(a, blockIdx.x - 1, m_in, m_out, s_part);
   }
 
   __threadfence();
@@ -1187,7 +1232,8 @@ replica_kernel(const ReplicaArgs ra) {
         const int b = (int)(row / a.T);
         const long long sample_end = (long long)(b + 1) * a.T;
         const long long row_b = sample_end < r1 ? sample_end : r1;
-        replica_segment(ra, b, row, row_b, a.ema[act], a.ema[act ^ 1], streamed, c, sgm, sh);
+        replica_segment(ra, b, row, row_b, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
+                        streamed, c, sgm, sh);
         row = row_b;
       } else if (threadIdx.x < a.R) {
         ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + sgm) * kSlotWords + 7] = 0ull;   // unused
@@ -1253,26 +1299,22 @@ __device__ __forceinline__ void st_x128(uint16_t *p, const uint4 &v) {
   asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-__device__ __forceinline__ unsigned pack_bf16x2_rn(float lo, float hi) {
-  unsigned r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // upper half <- first operand
-  return r;
-}
-
 __global__ void __launch_bounds__(kReplaceThreads)
-replace_kernel(const HandleState *hs, int kind, const float *ema0, const float *ema1, uint16_t *x,
+replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *ema1, int ema_bf16, uint16_t *x,
                long long n_chunks, int zero_fill, unsigned *replaced_out) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const KindState *ks = &hs->kind[kind];
   const int flagged = ks->last_flagged;
   if (blockIdx.x == 0 && threadIdx.x == 0 && replaced_out) *replaced_out = flagged ? 1u : 0u;
   if (!flagged) return;
-  const float *m = ks->active ? ema1 : ema0;
+  const void *m = ks->active ? ema1 : ema0;
   const long long stride = (long long)gridDim.x * kReplaceThreads;
   for (long long c = (long long)blockIdx.x * kReplaceThreads + threadIdx.x; c < n_chunks; c += stride) {
     uint4 out = make_uint4(0u, 0u, 0u, 0u);
-    if (!zero_fill) {
-      const F8 v = ld_m256(m + c * 8);
+    if (!zero_fill && ema_bf16) {                 // the reference already is a bf16 tensor
+      out = ld_x128(static_cast<const uint16_t *>(m) + c * 8);
+    } else if (!zero_fill) {
+      const F8 v = ld_m256(static_cast<const float *>(m) + c * 8);
       out.x = pack_bf16x2_rn(v.v[0], v.v[1]);
       out.y = pack_bf16x2_rn(v.v[2], v.v[3]);
       out.z = pack_bf16x2_rn(v.v[4], v.v[5]);

@@ -615,3 +615,95 @@ def test_argument_errors_never_reach_the_gpu(sb):
     torch.cuda.synchronize()
     assert bytes(v.sentinel_export_state()) == before      # none of the above touched the state
     v.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# the reference stored as bf16 (ema_bf16 = 1)
+
+def reference_bits_equal(gv, ov, params):
+    """With a bf16 reference both sides round the same single-precision value once: the stored
+    references agree bit for bit, not merely to a tolerance."""
+    st = parse_blob(gv.sentinel_export_state(), params.B, params.T, params.d, params.l)
+    for kind in (ACT, GRAD):
+        assert np.array_equal(st["kinds"][kind]["m"].astype(np.float64), ov.ema(kind)), kind
+
+
+@pytest.mark.parametrize("name,shape,steps", [("cfg2", (5, 40, 1024), 50), ("cfg4", (4, 24, 2056), 40),
+                                              ("cfg3", (3, 70, 520), 70)], ids=["cfg2", "cfg4", "cfg3"])
+def test_streams_in_lockstep_with_a_bf16_reference(sb, oracle_mod, name, shape, steps):
+    w = synth.scaled(synth.WORKLOADS[name], name + "_bf16", *shape, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w, ema_bf16=1)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, steps)
+    assert rec["corrupted"] >= 4
+    compare_state(gv, ov, params)
+    reference_bits_equal(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+    assert rec["near"] <= 1 and rec["k_events"] <= 3, rec
+    # Alg. 4 hands out the stored bf16 reference as it is
+    x, _ = synth.microbatch(w, 0, GRAD, 0, "cuda")
+    loud = (x.float() * 64).to(torch.bfloat16)
+    _, gf = gv.verify(loud, GRAD)
+    ov.verify(synth.bits(loud), GRAD)
+    out = loud.clone()
+    gv.sentinel_replace_if_flagged(out, GRAD, 0)
+    want, did = ov.replace_if_flagged(synth.bits(loud), GRAD)
+    torch.cuda.synchronize()
+    assert did and np.array_equal(synth.bits(out), want)
+    gv.close()
+
+
+def test_bf16_reference_with_strided_rows(sb, oracle_mod):
+    B, T, k, stride = 3, 21, 523, 524
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "compressed_bf16", B, T, stride)
+    gv = sb.Verifier(B, T, k, ema_bf16=1)
+    params = oracle_mod.Params(B=B, T=T, d=k, ema_bf16=1)
+    ov = oracle_mod.Verifier(params)
+    for t in range(12):
+        wide = synth.clean(w, 0, ACT, t, "cuda")
+        packed = wide[:, :, :k].contiguous()
+        gs = torch.empty(1 + B, 3, device="cuda")
+        if t < 8:
+            gv.sentinel_update_reference_strided(wide, ACT, gs)
+            os_, _ = ov.update_reference(synth.bits(packed), ACT)
+        else:
+            gf = torch.empty(1 + B, dtype=torch.int32, device="cuda")
+            gv.sentinel_verify_strided(wide, ACT, gs, gf)
+            os_, of, _ = ov.verify(synth.bits(packed), ACT)
+            assert np.array_equal(gf.cpu().numpy().view(np.uint32), of), t
+        assert_scores_close(gs.cpu().numpy(), os_, float(packed.float().abs().mean()), "step %d" % t)
+    reference_bits_equal(gv, ov, params)
+    gv.close()
+
+
+def test_bf16_reference_restrictions_and_state_round_trip(sb):
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(2, 8, 64, ema_bf16=1, n_workers=2)
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(2, 8, 64, ema_bf16=2)
+    assert e.value.code == sb.ERR_INVALID_ARG
+    gv = sb.Verifier(2, 8, 64, ema_bf16=1)
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_set_directions(synth.directions(4, 64, 1, "cuda"))
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "bf16_rt", 2, 8, 64)
+    for t in range(5):
+        gv.update_reference(synth.clean(w, 0, ACT, t, "cuda"), ACT)
+    blob = bytes(gv.sentinel_export_state())
+    other = sb.Verifier(2, 8, 64, ema_bf16=1)
+    other.sentinel_import_state(blob)
+    assert bytes(other.sentinel_export_state()) == blob
+    x = synth.clean(w, 0, ACT, 5, "cuda")
+    a, b = gv.verify(x, ACT), other.verify(x, ACT)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    # a state written by an fp32 verifier goes in rounded to nearest even
+    f32 = sb.Verifier(2, 8, 64)
+    for t in range(5):
+        f32.update_reference(synth.clean(w, 0, ACT, t, "cuda"), ACT)
+    st = parse_blob(f32.sentinel_export_state(), 2, 8, 64, 100)
+    other.sentinel_import_state(f32.sentinel_export_state())
+    got = parse_blob(other.sentinel_export_state(), 2, 8, 64, 100)["kinds"][ACT]["m"]
+    want = torch.from_numpy(st["kinds"][ACT]["m"]).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(got, want)
+    gv.close(); other.close(); f32.close()
