@@ -97,3 +97,59 @@ def test_cfg2_small_lm_stream_prefix(sb, oracle_mod):
             if name is not None:
                 assert np.any(of & UNIT_BITS), "additive noise of the tensor's own std is caught"
     gv.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# the variants at full size, through properties that hold at any size
+
+def test_cfg4_identical_workers_reduce_to_one_submission(sb):
+    """Four workers handing in the same 4 x 8192 x 8192 tensor: every worker's scores are those of
+    the single-submission call (other summation order: 1e-5), and the mean over four equal
+    tensors is that tensor, so the reference moves exactly (bit for bit) as it does for one
+    submission -- through the one-launch kernel and its speculative mean."""
+    w = synth.WORKLOADS["cfg4"]
+    R = 4
+    one = sb.Verifier(w.B, w.T, w.d)
+    many = sb.Verifier(w.B, w.T, w.d, n_workers=R, window_steps=50)
+    n = 4 * w.B * w.T * w.d
+
+    def act_reference(verifier):        # the reference is the tail of the first kind block of the blob
+        blob = verifier.sentinel_export_state()
+        per_kind = (verifier.sentinel_state_bytes() - 64 - 192) // 2
+        return np.frombuffer(blob, dtype=np.uint8, count=n, offset=64 + 192 + per_kind - n)
+
+    for t in range(5):
+        x = synth.clean(w, 0, ACT, t, "cuda")
+        warm = t < 4
+        if warm:
+            s1, committed = one.update_reference(x, ACT), True
+        else:
+            s1, f1 = one.verify(x, ACT)
+            committed = bool(int(f1[0]) & sb.FLAG_COMMITTED)
+        sr, fr = many.step_replicas([x] * R, ACT, warmup=warm)
+        torch.cuda.synchronize()
+        for r in range(R):
+            assert torch.allclose(sr[r], s1, rtol=1e-5, atol=1e-7), (t, r)
+        if committed:                   # (a flagged step: four of four is a majority, another rule applies)
+            assert all(int(fr[r, 0]) & sb.FLAG_COMMITTED for r in range(R))
+            assert np.array_equal(act_reference(one), act_reference(many)), t
+    one.close(); many.close()
+
+
+def test_cfg4_bf16_reference_first_update(sb):
+    """From m_0 = 0 one update leaves bf16((1-beta) x) in single precision, here checked on the
+    whole 4 x 8192 x 8192 tensor against torch's multiply and conversion."""
+    w = synth.WORKLOADS["cfg4"]
+    gv = sb.Verifier(w.B, w.T, w.d, ema_bf16=1)
+    x = synth.clean(w, 0, ACT, 0, "cuda")
+    gs = gv.update_reference(x, ACT)
+    blob = gv.sentinel_export_state()
+    per_kind = (gv.sentinel_state_bytes() - 64 - 192) // 2
+    n = w.B * w.T * w.d
+    m = torch.from_numpy(np.frombuffer(blob, dtype=np.float32, count=n, offset=64 + 192 + per_kind - 4 * n).copy())
+    want = (x.float() * float(np.float32(1.0 - 0.9))).to(torch.bfloat16).float().cpu().reshape(-1)
+    assert torch.equal(m, want)
+    # the first warm-up step runs against m = 0: L1 = mean |x|, sign flips = share of non-zero x
+    assert float(gs[0, 0]) == pytest.approx(float(x.float().abs().mean()), rel=1e-5)
+    assert float(gs[0, 2]) == pytest.approx(float((x != 0).float().mean()), rel=1e-6)
+    gv.close()
