@@ -284,6 +284,7 @@ cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m
   cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
   int occ = 0;
+  constexpr int kSwdThreads = swd_project_threads(L);
   e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, swd_project_kernel<L>, kSwdThreads, smem);
   if (e != cudaSuccess) return e;
   if (occ < 1) return cudaErrorInvalidConfiguration;
@@ -323,11 +324,12 @@ cudaError_t run_swd(const uint16_t *x, const float *m0, const float *m1, const i
   if (e != cudaSuccess) return e;
   int npad = 1;
   while (npad < T) npad <<= 1;
-  const size_t smem = (size_t)2 * npad * sizeof(float);
+  const size_t smem = (size_t)npad * sizeof(float);
   e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           2 * kSwdMaxTokensPerSample * (int)sizeof(float));
+                           kSwdMaxTokensPerSample * (int)sizeof(float));
   if (e != cudaSuccess) return e;
-  swd_sort_samples_kernel<<<B * L, kSwdSortThreads, smem, s>>>(proj, buf_a, w1_sample, B, T, L, rows, skip);
+  swd_sort_samples_kernel<<<2 * L * B, kSwdSortThreads, smem, s>>>(proj, buf_a, B, T, L, rows, skip);
+  swd_sample_w1_kernel<<<B * L, 256, 0, s>>>(buf_a, w1_sample, B, T, L, rows, skip);
   e = cudaGetLastError();
   float *cur = buf_a, *nxt = buf_b;
   for (int run = 1; run < B && e == cudaSuccess; run *= 2) {     // merge the samples' sorted lists

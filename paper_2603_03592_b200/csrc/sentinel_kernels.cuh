@@ -29,8 +29,8 @@ constexpr int kUnroll = 2;                // 8-element chunks per lane per loop 
 
 constexpr int kMaxWorkers = 16;           // workers (replicas of a stage) one handle can follow
 
-// single submission: verify / warm-up / stateless distance; one worker of a multi-worker
-// iteration: verify / warm-up (no EMA write: the mean over the clean workers follows)
+// single submission (stream_kernel_t): verify / warm-up / stateless distance; all workers of a
+// stage in one launch (replica_kernel): verify / warm-up, passed to each worker's finalize pass
 enum Mode : int { kModeVerify = 0, kModeWarmup = 1, kModeDistance = 2,
                   kModeReplicaVerify = 3, kModeReplicaWarmup = 4 };
 
@@ -959,7 +959,8 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
 // draws the last one has, by the fence/atomic order, everybody's partial sums and the fresh
 // thresholds in view, and finalizes.  No CTA ever waits for another.
 // (kScalar = true is the variant for rows of x that are strided or not 16-byte aligned; it is a
-// kernel of its own so that the vector path keeps its registers)
+// kernel of its own so that the vector path keeps its registers.  kBf16 = true: the reference
+// buffers hold bf16 instead of fp32.)
 template <bool kScalar, bool kBf16>
 __global__ void __launch_bounds__(kThreads)
 stream_kernel_t(const StreamArgs a) {

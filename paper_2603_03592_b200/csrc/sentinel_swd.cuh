@@ -9,7 +9,9 @@
 
 namespace sentinel {
 
-constexpr int kSwdThreads = 512;
+// threads of a projection CTA: as many as the registers allow (the directions fill most of the
+// shared memory, so one CTA per SM is the rule and its threads are all the loads in flight)
+__host__ __device__ constexpr int swd_project_threads(int L) { return L <= 8 ? 768 : 512; }
 constexpr int kSwdSortThreads = 1024;
 constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are sorted in shared memory
 
@@ -21,13 +23,14 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 // between them on the device); every kernel of the chain returns at once if *skip is non-zero
 // (a banned worker's tensor is not read).  Both pointers may be nullptr.
 template <int L>
-__global__ void __launch_bounds__(kSwdThreads)
+__global__ void __launch_bounds__(swd_project_threads(L))
 swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                    const uint16_t *u, float *proj, long long rows, int d) {
   extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
   if (skip && __ldcg(skip)) return;
   const float *m = (active && __ldcg(active)) ? m1 : m0;
   const int chunks = d >> 3;
+  constexpr int kSwdThreads = swd_project_threads(L);
   for (int i = threadIdx.x; i < L * chunks; i += kSwdThreads)
     s_u[i] = reinterpret_cast<const uint4 *>(u)[i];
   __syncthreads();
@@ -40,27 +43,43 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
 #pragma unroll
     for (int l = 0; l < L; ++l) { ax[l] = 0.f; am[l] = 0.f; }
     const size_t off = (size_t)row * d;
-    for (int c = lane; c < chunks; c += 32) {
-      const uint4 xv = ld_x128(x + off + (size_t)c * 8);
-      const F8 mv = ld_m256(m + off + (size_t)c * 8);
-      const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
-      float xf[8];
+    // two chunks per trip, their four loads issued before any arithmetic (more bytes in flight)
+    for (int c0 = lane; c0 < chunks; c0 += 64) {
+      uint4 xv[2];
+      F8 mv[2];
+      bool ok[2];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        xf[2 * j] = __uint_as_float(xw[j] << 16);
-        xf[2 * j + 1] = __uint_as_float(xw[j] & 0xFFFF0000u);
+      for (int h = 0; h < 2; ++h) {
+        const int c = c0 + 32 * h;
+        ok[h] = c < chunks;
+        if (ok[h]) {
+          xv[h] = ld_x128(x + off + (size_t)c * 8);
+          mv[h] = ld_m256(m + off + (size_t)c * 8);
+        }
       }
 #pragma unroll
-      for (int l = 0; l < L; ++l) {
-        const uint4 uv = s_u[l * chunks + c];
-        const unsigned uw[4] = {uv.x, uv.y, uv.z, uv.w};
+      for (int h = 0; h < 2; ++h) {
+        if (!ok[h]) continue;
+        const int c = c0 + 32 * h;
+        const unsigned xw[4] = {xv[h].x, xv[h].y, xv[h].z, xv[h].w};
+        float xf[8];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const float u_lo = __uint_as_float(uw[j] << 16), u_hi = __uint_as_float(uw[j] & 0xFFFF0000u);
-          ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
-          ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
-          am[l] = fmaf(mv.v[2 * j], u_lo, am[l]);
-          am[l] = fmaf(mv.v[2 * j + 1], u_hi, am[l]);
+          xf[2 * j] = __uint_as_float(xw[j] << 16);
+          xf[2 * j + 1] = __uint_as_float(xw[j] & 0xFFFF0000u);
+        }
+#pragma unroll
+        for (int l = 0; l < L; ++l) {
+          const uint4 uv = s_u[l * chunks + c];
+          const unsigned uw[4] = {uv.x, uv.y, uv.z, uv.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float u_lo = __uint_as_float(uw[j] << 16), u_hi = __uint_as_float(uw[j] & 0xFFFF0000u);
+            ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
+            ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
+            am[l] = fmaf(mv[h].v[2 * j], u_lo, am[l]);
+            am[l] = fmaf(mv[h].v[2 * j + 1], u_hi, am[l]);
+          }
         }
       }
     }
@@ -76,7 +95,7 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
 }
 
 // ---------------------------------------------------------------------------------------------
-// per sample and direction: sort the T projections of x and of m, W1 = mean |a_(i) - b_(i)|
+// helpers of the sort / W1 kernels
 __device__ __forceinline__ double block_sum_ordered(double v, double *s_red) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   v = warp_sum(v);
@@ -89,46 +108,45 @@ __device__ __forceinline__ double block_sum_ordered(double v, double *s_red) {
   return total;                                   // valid in thread 0
 }
 
+// one CTA per (sample, direction, cloud): bitonic sort of that list of T projections in shared
+// memory; the sorted list goes back to global memory
 __global__ void __launch_bounds__(kSwdSortThreads)
-swd_sort_samples_kernel(const float *proj, float *sorted, float *w1_sample, int B, int T, int L, long long rows,
-                        const int *skip) {
-  extern __shared__ float s_val[];                // [2][npad]
-  __shared__ double s_red[kSwdSortThreads / 32];
+swd_sort_samples_kernel(const float *proj, float *sorted, int B, int T, int L, long long rows, const int *skip) {
+  extern __shared__ float s_val[];                // [npad]
   if (skip && __ldcg(skip)) return;
-  const int b = blockIdx.x / L, l = blockIdx.x - b * L;
+  const int list = blockIdx.x / B, b = blockIdx.x - list * B;     // list = cloud * L + direction
   int npad = 1;
   while (npad < T) npad <<= 1;
-  float *sa = s_val, *sb = s_val + npad;
-  const float *px = proj + (size_t)l * rows + (size_t)b * T;
-  const float *pm = proj + ((size_t)L + l) * rows + (size_t)b * T;
-  for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) {
-    sa[i] = i < T ? px[i] : CUDART_INF_F;
-    sb[i] = i < T ? pm[i] : CUDART_INF_F;
-  }
+  const float *src = proj + (size_t)list * rows + (size_t)b * T;
+  for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) s_val[i] = i < T ? src[i] : CUDART_INF_F;
   __syncthreads();
-  for (int k2 = 2; k2 <= npad; k2 <<= 1) {        // bitonic sort of both lists, ascending
+  for (int k2 = 2; k2 <= npad; k2 <<= 1) {        // bitonic sort, ascending
     for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
       for (int t = threadIdx.x; t < npad; t += kSwdSortThreads) {
         const int partner = t ^ j2;
         if (partner > t) {
           const bool up = ((t & k2) == 0);
-          const float a0 = sa[t], a1 = sa[partner];
-          if ((a0 > a1) == up) { sa[t] = a1; sa[partner] = a0; }
-          const float b0 = sb[t], b1 = sb[partner];
-          if ((b0 > b1) == up) { sb[t] = b1; sb[partner] = b0; }
+          const float a0 = s_val[t], a1 = s_val[partner];
+          if ((a0 > a1) == up) { s_val[t] = a1; s_val[partner] = a0; }
         }
       }
       __syncthreads();
     }
   }
+  float *dst = sorted + (size_t)list * rows + (size_t)b * T;
+  for (int i = threadIdx.x; i < T; i += kSwdSortThreads) dst[i] = s_val[i];
+}
+
+// per sample and direction: W1 = mean |a_(i) - b_(i)| of the two sorted lists
+__global__ void __launch_bounds__(256)
+swd_sample_w1_kernel(const float *sorted, float *w1_sample, int B, int T, int L, long long rows, const int *skip) {
+  __shared__ double s_red[256 / 32];
+  if (skip && __ldcg(skip)) return;
+  const int b = blockIdx.x / L, l = blockIdx.x - b * L;
+  const float *sa = sorted + (size_t)l * rows + (size_t)b * T;
+  const float *sb = sorted + ((size_t)L + l) * rows + (size_t)b * T;
   double acc = 0.;
-  float *ox = sorted + (size_t)l * rows + (size_t)b * T;
-  float *om = sorted + ((size_t)L + l) * rows + (size_t)b * T;
-  for (int i = threadIdx.x; i < T; i += kSwdSortThreads) {
-    acc += (double)fabsf(sa[i] - sb[i]);
-    ox[i] = sa[i];
-    om[i] = sb[i];
-  }
+  for (int i = threadIdx.x; i < T; i += 256) acc += (double)fabsf(sa[i] - sb[i]);
   const double total = block_sum_ordered(acc, s_red);
   if (threadIdx.x == 0) w1_sample[b * L + l] = (float)(total / (double)T);
 }
