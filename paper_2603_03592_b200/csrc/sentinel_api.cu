@@ -277,21 +277,30 @@ struct DeviceGuard {   // restores the caller's current device
 // sliced Wasserstein distance: the chain of launches, shared by the stateless entry point and
 // by verifiers that carry it as their fourth metric
 
+template <int L, int kT>
+cudaError_t projection_occupancy(size_t smem, int *occ) {
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT>, kT, smem);
+}
+
 template <int L>
 cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                               const uint16_t *u, float *proj, long long rows, int d, int sms, cudaStream_t s) {
   const size_t smem = (size_t)L * d * sizeof(uint16_t);
-  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  int occ_small = 0, occ_large = 0;
+  cudaError_t e = projection_occupancy<L, 512>(smem, &occ_small);
   if (e != cudaSuccess) return e;
-  int occ = 0;
-  constexpr int kSwdThreads = swd_project_threads(L);
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, swd_project_kernel<L>, kSwdThreads, smem);
+  e = projection_occupancy<L, 768>(smem, &occ_large);
   if (e != cudaSuccess) return e;
+  const bool large = occ_large * 768 > occ_small * 512;
+  const int threads = large ? 768 : 512, occ = large ? occ_large : occ_small;
   if (occ < 1) return cudaErrorInvalidConfiguration;
   long long grid = (long long)sms * occ;
-  const long long need = (rows + kSwdThreads / 32 - 1) / (kSwdThreads / 32);
+  const long long need = (rows + threads / 32 - 1) / (threads / 32);
   if (grid > need) grid = need;
-  swd_project_kernel<L><<<(unsigned)grid, kSwdThreads, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d);
+  if (large) swd_project_kernel<L, 768><<<(unsigned)grid, 768, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d);
+  else swd_project_kernel<L, 512><<<(unsigned)grid, 512, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d);
   return cudaGetLastError();
 }
 

@@ -9,9 +9,8 @@
 
 namespace sentinel {
 
-// threads of a projection CTA: as many as the registers allow (the directions fill most of the
-// shared memory, so one CTA per SM is the rule and its threads are all the loads in flight)
-__host__ __device__ constexpr int swd_project_threads(int L) { return L <= 8 ? 768 : 512; }
+// A projection CTA has 512 or 768 threads; the host takes whichever keeps more threads resident
+// per SM (the directions can fill most of the shared memory: then one large CTA is all there is).
 constexpr int kSwdSortThreads = 1024;
 constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are sorted in shared memory
 
@@ -22,15 +21,14 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 // The reference is m1 if *active is non-zero, else m0 (a verifier keeps two buffers and flips
 // between them on the device); every kernel of the chain returns at once if *skip is non-zero
 // (a banned worker's tensor is not read).  Both pointers may be nullptr.
-template <int L>
-__global__ void __launch_bounds__(swd_project_threads(L))
+template <int L, int kSwdThreads>
+__global__ void __launch_bounds__(kSwdThreads, kSwdThreads == 512 ? 2 : 1)
 swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                    const uint16_t *u, float *proj, long long rows, int d) {
   extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
   if (skip && __ldcg(skip)) return;
   const float *m = (active && __ldcg(active)) ? m1 : m0;
   const int chunks = d >> 3;
-  constexpr int kSwdThreads = swd_project_threads(L);
   for (int i = threadIdx.x; i < L * chunks; i += kSwdThreads)
     s_u[i] = reinterpret_cast<const uint4 *>(u)[i];
   __syncthreads();
