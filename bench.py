@@ -368,6 +368,7 @@ def run_ours(args, rank, world, local_rank):
         "microbatches_per_s": round(world * args.steps * nb / (elapsed_ms * 1e-3), 1),
         "tensor_gbs": round(world * args.steps * nb * 2 * N * 2 / (elapsed_ms * 1e-3) / 1e9, 1),
         "ms_per_step_median": round(step_ms[len(step_ms) // 2], 4),
+        "ms_per_step_best": round(step_ms[0], 4),
         "frac_of_8000_nominal": round(gbs / world / 8000.0, 4),
         "gpu_launches": launches,
         "violations_seen": violations,
