@@ -707,3 +707,40 @@ def test_bf16_reference_restrictions_and_state_round_trip(sb):
     want = torch.from_numpy(st["kinds"][ACT]["m"]).to(torch.bfloat16).float().numpy()
     assert np.array_equal(got, want)
     gv.close(); other.close(); f32.close()
+
+
+def test_verify_calls_replay_from_a_cuda_graph(sb):
+    """A verified step is one kernel launch with no allocation and no host decision, so a sequence
+    of calls can be captured once and replayed: every replay is the next step on whatever the
+    input buffers hold, and leaves the same scores, flags and state as the same calls made one
+    by one."""
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "graph", 8, 128, 512)
+    eager, graphed = sb.Verifier(w.B, w.T, w.d), sb.Verifier(w.B, w.T, w.d)
+    for t in range(8):
+        for kind in (ACT, GRAD):
+            x = synth.clean(w, 0, kind, t, "cuda")
+            eager.update_reference(x, kind)
+            graphed.update_reference(x, kind)
+    buf = [torch.empty(w.B, w.T, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    scores = torch.zeros(2, 1 + w.B, 3, device="cuda")
+    flags = torch.zeros(2, 1 + w.B, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for kind in (ACT, GRAD):
+            graphed.sentinel_verify(buf[kind], kind, scores[kind], flags[kind])
+    for t in range(8, 14):
+        xs = [synth.clean(w, 0, kind, t, "cuda") for kind in (ACT, GRAD)]
+        if t == 11:
+            xs[ACT] = synth.corrupt(w, xs[ACT], "scale_sample3", 0, ACT, t)
+        for kind in (ACT, GRAD):
+            buf[kind].copy_(xs[kind])
+        graph.replay()
+        torch.cuda.synchronize()
+        for kind in (ACT, GRAD):
+            es, ef = eager.verify(xs[kind], kind)
+            assert torch.equal(es, scores[kind]) and torch.equal(ef, flags[kind]), (t, kind)
+        if t == 11:
+            assert int(flags[ACT, 4]) & sb.FLAG_L1 and not int(flags[ACT, 0]) & sb.FLAG_COMMITTED
+    assert bytes(eager.sentinel_export_state()) == bytes(graphed.sentinel_export_state())
+    eager.close(); graphed.close()
