@@ -63,6 +63,7 @@ void so_default_params(so_params *p) {
   p->B = 1; p->T = 1; p->d = 8;
   p->R = 1;
   p->ema_bf16 = 0;
+  p->ref_over_batch = 0;
 }
 
 /* ------------------------------------------------------------------------------------ */
@@ -260,7 +261,7 @@ typedef struct so_kind_state {
 
 struct so_verifier {
   so_params p;
-  size_t N, Ns;
+  size_t N, Ns, Nm;
   so_kind_state ks[2];
   int violations[SO_MAX_WORKERS], clean_streak[SO_MAX_WORKERS], banned[SO_MAX_WORKERS];
   uint16_t *u;   /* directions of the sliced Wasserstein metric, bf16 [n_dir][d]; NULL = metric off */
@@ -279,14 +280,16 @@ static void window_push(so_window *w, double val) {
 so_verifier *so_create(const so_params *p) {
   if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1 || p->R < 1 || p->R > SO_MAX_WORKERS) return NULL;
   if (p->ema_bf16 && p->R != 1) return NULL;   /* the bf16 reference exists for one submission per update */
+  if (p->ref_over_batch && (p->R != 1 || p->ema_bf16)) return NULL;   /* likewise the [T,d] reference */
   so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
   v->p = *p;
   v->Ns = (size_t)p->T * (size_t)p->d;
   v->N = v->Ns * (size_t)p->B;
+  v->Nm = p->ref_over_batch ? v->Ns : v->N;   /* elements of the reference */
   v->u = NULL; v->n_dir = 0; v->nm = 3;
   for (int kind = 0; kind < 2; ++kind) {
     so_kind_state *ks = &v->ks[kind];
-    ks->m = (double *)calloc(v->N, sizeof(double));
+    ks->m = (double *)calloc(v->Nm, sizeof(double));
     ks->stats = (double *)calloc((size_t)(1 + p->B) * SO_NSTAT, sizeof(double));
     for (int L = 0; L < 2; ++L)
       for (int i = 0; i < SO_NMETRIC; ++i) {
@@ -303,7 +306,7 @@ so_verifier *so_create(const so_params *p) {
 }
 
 int so_set_directions(so_verifier *v, const uint16_t *u, int n_dir) {
-  if (n_dir < 1 || !u || v->p.ema_bf16) return -1;
+  if (n_dir < 1 || !u || v->p.ema_bf16 || v->p.ref_over_batch) return -1;
   if (v->ks[0].steps || v->ks[1].steps) return -1;   /* the metric set is fixed before the first step */
   free(v->u);
   v->u = (uint16_t *)malloc((size_t)n_dir * (size_t)v->p.d * sizeof(uint16_t));
@@ -330,15 +333,23 @@ void so_destroy(so_verifier *v) {
 static void all_units(so_verifier *v, const uint16_t *x, int kind, double *gam, int *nonfinite) {
   so_kind_state *ks = &v->ks[kind];
   const size_t d = (size_t)v->p.d;
+  /* a [T,d] reference stands for the same tensor in every sample: write the broadcast out */
+  double *wide = NULL;
+  if (v->p.ref_over_batch) {
+    wide = (double *)malloc(v->N * sizeof(double));
+    for (int b = 0; b < v->p.B; ++b) memcpy(wide + (size_t)b * v->Ns, ks->m, v->Ns * sizeof(double));
+  }
+  const double *m = wide ? wide : ks->m;
   for (int r = 0; r <= v->p.B; ++r) {
     /* unit r: the whole tensor (B*T tokens) or sample r-1 (T tokens) */
     const size_t off = (r == 0) ? 0 : (size_t)(r - 1) * v->Ns;
     const size_t n = (r == 0) ? v->N : v->Ns;
     double *g = gam + (size_t)r * SO_NMETRIC;
-    nonfinite[r] = so_distance(x + off, ks->m + off, n, g, ks->stats + (size_t)r * SO_NSTAT);
-    g[SO_SW] = v->u ? so_sliced_wasserstein(x + off, ks->m + off, n / d, d, v->u, (size_t)v->n_dir, NULL)
+    nonfinite[r] = so_distance(x + off, m + off, n, g, ks->stats + (size_t)r * SO_NSTAT);
+    g[SO_SW] = v->u ? so_sliced_wasserstein(x + off, m + off, n / d, d, v->u, (size_t)v->n_dir, NULL)
                     : NAN;
   }
+  free(wide);
 }
 
 static void refresh_thresholds(so_verifier *v, int kind) {
@@ -365,6 +376,14 @@ static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
     const float bf = (float)beta, of = (float)(1.0 - beta);
     for (size_t e = 0; e < v->N; ++e)
       m[e] = so_bf16(so_bf16_round((double)fmaf(bf, (float)m[e], of * (float)so_bf16(x[e]))));
+    return;
+  }
+  if (v->p.ref_over_batch) {   /* Eq. 1 with the mean over the B samples as the submission */
+    for (size_t e = 0; e < v->Ns; ++e) {
+      double sum = 0.0;
+      for (int b = 0; b < v->p.B; ++b) sum += so_bf16(x[(size_t)b * v->Ns + e]);
+      m[e] = beta * m[e] + (1.0 - beta) * (sum / (double)v->p.B);
+    }
     return;
   }
   for (size_t e = 0; e < v->N; ++e) m[e] = beta * m[e] + (1.0 - beta) * so_bf16(x[e]);
@@ -578,7 +597,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
 int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill) {
   if (!v->ks[kind].last_flagged) return 0;
   const double *m = v->ks[kind].m;                 /* a flagged step left m at m_{t-1} */
-  for (size_t e = 0; e < v->N; ++e) x[e] = fill ? 0 : so_bf16_round(m[e]);
+  for (size_t e = 0; e < v->N; ++e) x[e] = fill ? 0 : so_bf16_round(m[e % v->Nm]);
   return 1;
 }
 
@@ -597,7 +616,7 @@ void so_reset_worker(so_verifier *v) {
 const double *so_ema(const so_verifier *v, int kind) { return v->ks[kind].m; }
 
 void so_set_ema(so_verifier *v, int kind, const double *m) {
-  memcpy(v->ks[kind].m, m, v->N * sizeof(double));
+  memcpy(v->ks[kind].m, m, v->Nm * sizeof(double));
   if (v->p.ema_bf16)
     for (size_t e = 0; e < v->N; ++e) v->ks[kind].m[e] = so_bf16(so_bf16_round(m[e]));
 }

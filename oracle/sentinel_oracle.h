@@ -64,6 +64,7 @@ typedef struct so_params {
   int    B, T, d;          /* submission shape                                      */
   int    R;                /* workers (replicas) feeding this boundary, d_s >= 1    */
   int    ema_bf16;         /* != 0: the reference is stored as bf16 (R = 1 only)    */
+  int    ref_over_batch;   /* != 0: one [T,d] reference for all B samples (R = 1)   */
 } so_params;
 
 typedef struct so_verifier so_verifier;
@@ -162,7 +163,7 @@ void so_worker_counters(const so_verifier *v, int r, int out[3]);   /* v_r, stre
 void so_reset_worker(so_verifier *v);
 
 /* State access for tests. */
-const double *so_ema(const so_verifier *v, int kind);                 /* B*T*d values      */
+const double *so_ema(const so_verifier *v, int kind);                 /* B*T*d values (T*d with ref_over_batch) */
 void   so_set_ema(so_verifier *v, int kind, const double *m);
 size_t so_history(const so_verifier *v, int kind, int level, int metric,
                   double *out, size_t cap);                            /* oldest first      */

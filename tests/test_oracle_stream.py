@@ -638,3 +638,62 @@ def test_bf16_reference_is_for_single_submissions_without_directions(oracle_mod)
     m = rs.normal(0, 1, (2, 4, 8))
     v.set_ema(ACT, m)
     assert np.array_equal(v.ema(ACT), from_bits(to_bits(m)))  # stored rounded
+
+
+# ---------------------------------------------------------------------------------------------
+# one [T,d] reference shared by the B samples
+
+def test_shared_reference_is_the_full_reference_of_the_batch_mean(oracle_mod):
+    """Eq. 1 with the mean over the samples as the submission: the [T,d] reference follows the
+    batch mean exactly as a full reference of a one-sample verifier fed that mean would, and the
+    closed form from m_0 = 0 holds."""
+    rs = np.random.default_rng(41)
+    B, T, d = 4, 5, 8
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_batch=1)
+    want = np.zeros((T, d))
+    for t in range(6):
+        xb = to_bits(rs.normal(0.5, 1, (B, T, d)))
+        v.update_reference(xb, ACT)
+        want = 0.9 * want + 0.1 * from_bits(xb).mean(axis=0)
+        assert v.ema(ACT).shape == (T, d)
+        assert v.ema(ACT) == pytest.approx(want, rel=1e-13, abs=1e-16)
+
+
+def test_shared_reference_scores_are_those_against_the_tiled_reference(oracle_mod):
+    """Every unit is compared with the same [T,d] tensor: sample b against m, the whole tensor
+    against B copies of m -- the stateless distances say the same."""
+    rs = np.random.default_rng(42)
+    B, T, d = 3, 4, 8
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_batch=1)
+    for t in range(5):
+        v.update_reference(to_bits(rs.normal(0, 1, (B, T, d)) + np.arange(d)), GRAD)
+    m = v.ema(GRAD)
+    xb = to_bits(rs.normal(0, 1, (B, T, d)) + np.arange(d))
+    scores, flags, _ = v.verify(xb, GRAD)
+    g0, s0, _ = oracle_mod.distance(xb, np.tile(m, (B, 1, 1)))
+    assert np.array_equal(scores[0], g0) and np.array_equal(v.last_stats(GRAD)[0], s0)
+    for b in range(B):
+        gb, _, _ = oracle_mod.distance(xb[b], m)
+        assert np.array_equal(scores[1 + b], gb)
+
+
+def test_shared_reference_flags_commit_and_replacement(oracle_mod, small):
+    v = oracle_mod.Verifier(oracle_mod.Params(B=small.B, T=small.T, d=small.d, ref_over_batch=1))
+    for t in range(14):
+        v.update_reference(synth.bits(synth.clean(small, 0, GRAD, t)), GRAD)
+    g = synth.clean(small, 0, GRAD, 14)
+    _, flags, commit = v.verify(synth.bits(g), GRAD)
+    assert commit and not (flags & 0xFFFF).any()
+    m0 = v.ema(GRAD)
+    loud = (g.float() * 50).to(torch.bfloat16)
+    _, flags, commit = v.verify(synth.bits(loud), GRAD)
+    assert not commit and (flags[0] & 0xFFFF) and np.array_equal(v.ema(GRAD), m0)
+    out, did = v.replace_if_flagged(synth.bits(loud), GRAD)
+    assert did
+    got = from_bits(out)
+    for b in range(small.B):                                 # every sample receives the one reference
+        assert np.all(np.abs(got[b] - m0) <= 2.0 ** -8 * np.abs(m0) + 1e-45)
+    with pytest.raises(ValueError):
+        oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_batch=1, R=2))
+    with pytest.raises(ValueError):
+        oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_batch=1, ema_bf16=1))
