@@ -96,6 +96,7 @@ typedef struct sentinel_config {
   int    device;           /* CUDA device ordinal                                           */
   int    n_workers;        /* workers d_s feeding this boundary (multi-worker calls)   1    */
   int    ema_bf16;         /* 1: the reference is stored as bf16 (see below)           0    */
+  int    ref_over_batch;   /* 1: one [T,d] reference for all B samples (see below)     0    */
 } sentinel_config;
 
 typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundary */
@@ -110,6 +111,15 @@ typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundar
  * flags are computed exactly as with fp32, against the rounded reference.  Restrictions:
  * n_workers = 1, no sentinel_set_directions.  State blobs carry the reference as fp32 either
  * way (widened exactly on export, rounded to nearest even on import). */
+/* ref_over_batch = 1 keeps ONE reference of shape [T,d] for all B samples of a tensor instead of
+ * a [B,T,d] one (the paper states the reference only as "the EMA of the signal"; this reading
+ * treats the samples of a microbatch as draws of the same [T,d] signal): every sample is compared
+ * with it, the whole-tensor unit with B copies of it, and Eq. 1 moves it with the mean over the
+ * samples, m_t = beta m_{t-1} + (1-beta)/B sum_b x[b].  A verified tensor then moves 2 + 8/B bytes
+ * per element and the state shrinks B-fold.  Restrictions: n_workers = 1, fp32 reference,
+ * B <= 16, d a multiple of 8; no strided tensors, no sentinel_set_directions, no per-token buffer.
+ * Gradient replacement writes the one reference into every sample.  State blobs carry T*d
+ * reference values per kind and record the shape in the header. */
 int sentinel_default_config(sentinel_config *cfg);
 
 /* Allocates the state of one boundary on cfg->device: two fp32 [B,T,d] buffers per kind (the
@@ -313,10 +323,11 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
 int sentinel_reset_worker(sentinel_verifier *h, int worker, void *cuda_stream);
 
 /* Checkpointing.  The state is one self-describing blob: a 64-byte header
- * {u64 magic, u32 version = 3, i32 B, T, d, window_steps, n_workers, n_metrics}, then
+ * {u64 magic, u32 version = 3, i32 B, T, d, window_steps, n_workers, n_metrics, ref_over_batch}, then
  * i32 violations[16], clean_streak[16], banned[16], then per kind {i64 steps; i32 count[2];
  * i32 valid[2][4]; f64 thr[2][4][6]; f64 history[level 0: 4][window_steps*n_workers],
- * [level 1: 4][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d]}.  The
+ * [level 1: 4][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d] (m[T*d] with
+ * ref_over_batch)}.  The
  * layout always has room for four metrics; with n_metrics = 3 the fourth slots are unused.
  * A blob goes back only into a verifier with the same n_metrics (the directions themselves
  * are not part of the state: set them before importing).  Export and import wait for the

@@ -26,7 +26,7 @@ constexpr size_t kHeaderBytes = 64;
 struct BlobHeader {
   unsigned long long magic;
   unsigned version;
-  int B, T, d, window_steps, n_workers, n_metrics;
+  int B, T, d, window_steps, n_workers, n_metrics, ref_over_batch;
 };
 
 struct BlobWorkers {      // follows the header
@@ -59,6 +59,8 @@ struct sentinel_verifier {
   float *sw_out = nullptr;          // [1+B] distances of the submission being checked
   void *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // fp32, or bf16 if bf16
   bool bf16 = false;                // the reference is stored as bf16
+  bool shared_ref = false;          // one [T,d] reference for all B samples
+  size_t ema_elems = 0;             // elements of one reference buffer: B*T*d, or T*d if shared_ref
   size_t ema_bytes = 0;             // bytes of one reference buffer
   HandleState *hs = nullptr;
   double *hist[2] = {nullptr, nullptr};      // rings, device layout (ring_offset)
@@ -105,7 +107,7 @@ size_t ring_doubles(const sentinel_verifier *h) {
 }
 
 size_t kind_blob_bytes(const sentinel_verifier *h) {
-  return sizeof(BlobKindHead) + hist_doubles(h) * sizeof(double) + h->N * sizeof(float);
+  return sizeof(BlobKindHead) + hist_doubles(h) * sizeof(double) + h->ema_elems * sizeof(float);
 }
 
 Alg5Params alg5_of(const sentinel_config &c, int kind) {
@@ -190,6 +192,7 @@ int check_call_strided(sentinel_verifier *h, const void *x, int kind, int B, int
   if (row_stride < d) return fail(h, SENTINEL_ERR_INVALID_ARG, "row_stride = %lld is smaller than d = %d", row_stride, d);
   if (reinterpret_cast<uintptr_t>(x) & 1u) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 2-byte aligned");
   if (h->sw_u) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein metric reads dense rows: a verifier with directions takes no strided tensor");
+  if (h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "a verifier with a [T,d] reference takes no strided tensor");
   h->started = true;
   return SENTINEL_OK;
 }
@@ -245,6 +248,15 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
   attr.val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = &attr;
   lc.numAttrs = 1;
+  if (h->shared_ref) {                             // the samples in the workers' place (vector rows only)
+    ReplicaArgs ra;
+    memset(&ra, 0, sizeof ra);
+    ra.s = a;
+    for (int b = 0; b < h->cfg.B; ++b) ra.xs[b] = a.x + (size_t)b * h->Ns;
+    ra.partials = h->partials;
+    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, shared_ref_kernel, ra));
+    return SENTINEL_OK;
+  }
   if (h->bf16) {
     if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, true>, a));
     else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, true>, a));
@@ -428,6 +440,9 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   if (cfg->ema_bf16 != 0 && cfg->ema_bf16 != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ema_bf16 must be 0 or 1, got %d", cfg->ema_bf16);
   if (cfg->ema_bf16 && cfg->n_workers != 1)
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "the bf16 reference is kept for single submissions only (n_workers = 1)");
+  if (cfg->ref_over_batch != 0 && cfg->ref_over_batch != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ref_over_batch must be 0 or 1, got %d", cfg->ref_over_batch);
+  if (cfg->ref_over_batch && (cfg->n_workers != 1 || cfg->ema_bf16 || cfg->B > kMaxWorkers || cfg->d % 8 != 0))
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a [T,d] reference needs n_workers = 1, an fp32 reference, B <= %d and d a multiple of 8", kMaxWorkers);
   if ((long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*n_workers*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d",
                 (long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1), SENTINEL_MAX_WINDOW);
@@ -445,7 +460,9 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->N = h->Ns * cfg->B;
   h->R = cfg->n_workers;
   h->bf16 = cfg->ema_bf16 != 0;
-  h->ema_bytes = h->N * (h->bf16 ? sizeof(uint16_t) : sizeof(float));
+  h->shared_ref = cfg->ref_over_batch != 0;
+  h->ema_elems = h->shared_ref ? h->Ns : h->N;
+  h->ema_bytes = h->ema_elems * (h->bf16 ? sizeof(uint16_t) : sizeof(float));
   h->units0 = h->R;                       // the window spans window_steps iterations of all workers
   h->units1 = h->R * cfg->B;
   h->cap0 = cfg->window_steps * h->units0;
@@ -464,10 +481,12 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
   }
   std::string oerr;
-  h->G = streaming_ctas(cfg->device, cfg->B, cfg->T, &oerr);
+  // (with a [T,d] reference the CTAs share out the T token rows, each with every sample's slice)
+  h->G = h->shared_ref ? streaming_ctas(cfg->device, 1, cfg->T, &oerr) : streaming_ctas(cfg->device, cfg->B, cfg->T, &oerr);
   if (h->G < 1) { delete h; return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str()); }
 
   cudaError_t e = cudaSuccess;
@@ -481,7 +500,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     alloc((void **)&h->sorted[k], hist_doubles(h) * sizeof(double));
     alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
   }
-  alloc((void **)&h->partials, (size_t)h->R * h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));   // per worker
+  alloc((void **)&h->partials, (size_t)(h->shared_ref ? cfg->B : h->R) * h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));   // per worker / per sample
   alloc((void **)&h->hs, sizeof(HandleState));
   if (e == cudaSuccess) {
     HandleState init;
@@ -740,7 +759,8 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
   const long long need = (n_chunks + kReplaceThreads - 1) / kReplaceThreads;
   if (grid > need) grid = need;
   replace_kernel<<<(unsigned)grid, kReplaceThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], h->bf16 ? 1 : 0, static_cast<uint16_t *>(dev_x_inout), n_chunks, fill,
+      h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], h->bf16 ? 1 : 0, static_cast<uint16_t *>(dev_x_inout), n_chunks,
+      h->shared_ref ? (long long)(h->ema_elems / 8) : 0ll, fill,
       dev_replaced_out);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
@@ -751,6 +771,7 @@ int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L,
   if (!dev_u_bf16) return fail(h, SENTINEL_ERR_INVALID_ARG, "u is NULL");
   if (h->started) return fail(h, SENTINEL_ERR_INVALID_ARG, "the metric set is fixed once a step was taken or a state imported");
   if (h->bf16) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads an fp32 reference: not available with ema_bf16");
+  if (h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads a [B,T,d] reference: not available with ref_over_batch");
   if (h->cfg.d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", h->cfg.d);
   int rc = check_swd_shape(h, L, h->cfg.T, h->cfg.d);
   if (rc) return rc;
@@ -864,6 +885,7 @@ int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_
 int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (dev_buf && !aligned16(dev_buf)) return fail(h, SENTINEL_ERR_UNALIGNED, "token buffer is not 16-byte aligned");
+  if (dev_buf && h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "per-token sums are not written with a [T,d] reference");
   const int tpr = tiles_per_row(h->cfg.d);
   if (dev_buf && tpr > 1 && !h->token_part) {      // rows of several tiles need a place for the shares
     DeviceGuard guard(h->cfg.device);
@@ -920,7 +942,7 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
 
   unsigned char *out = static_cast<unsigned char *>(host_buf);
   memset(out, 0, kHeaderBytes);
-  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics};
+  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics, h->shared_ref ? 1 : 0};
   memcpy(out, &hd, sizeof hd);
   out += kHeaderBytes;
   BlobWorkers bw;
@@ -954,18 +976,18 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
     }
     out = reinterpret_cast<unsigned char *>(dst);
     if (h->bf16) {                                  // the blob always carries fp32: widen (exact)
-      std::vector<uint16_t> half(h->N);
+      std::vector<uint16_t> half(h->ema_elems);
       SENTINEL_CUDA(h, cudaMemcpyAsync(half.data(), h->ema[k][ks.active], h->ema_bytes, cudaMemcpyDeviceToHost, s));
       SENTINEL_CUDA(h, cudaStreamSynchronize(s));
-      for (size_t e = 0; e < h->N; ++e) {
+      for (size_t e = 0; e < h->ema_elems; ++e) {
         const unsigned bits = (unsigned)half[e] << 16;
         memcpy(out + e * sizeof(float), &bits, sizeof bits);
       }
     } else {
-      SENTINEL_CUDA(h, cudaMemcpyAsync(out, h->ema[k][ks.active], h->N * sizeof(float), cudaMemcpyDeviceToHost, s));
+      SENTINEL_CUDA(h, cudaMemcpyAsync(out, h->ema[k][ks.active], h->ema_elems * sizeof(float), cudaMemcpyDeviceToHost, s));
       SENTINEL_CUDA(h, cudaStreamSynchronize(s));
     }
-    out += h->N * sizeof(float);
+    out += h->ema_elems * sizeof(float);
   }
   return SENTINEL_OK;
 }
@@ -981,6 +1003,8 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
     return fail(h, SENTINEL_ERR_STATE_SIZE, "not a sentinel state blob of version %u", kVersion);
   if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps || hd.n_workers != h->R)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d, %d workers", hd.B, hd.T, hd.d, hd.window_steps, hd.n_workers);
+  if ((hd.ref_over_batch != 0) != h->shared_ref)
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob and verifier differ in the shape of the reference ([T,d] against [B,T,d])");
   if (hd.n_metrics != h->n_metrics)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob holds %d metrics, this verifier uses %d (set the directions before importing)", hd.n_metrics, h->n_metrics);
   // validate both kinds before touching the device
@@ -1039,8 +1063,8 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
     }
     p += hist_doubles(h) * sizeof(double);
     if (h->bf16) {                                  // narrow, to nearest even (exact for a bf16 verifier's own blob)
-      std::vector<uint16_t> half(h->N);
-      for (size_t e = 0; e < h->N; ++e) {
+      std::vector<uint16_t> half(h->ema_elems);
+      for (size_t e = 0; e < h->ema_elems; ++e) {
         unsigned bits;
         memcpy(&bits, p + e * sizeof(float), sizeof bits);
         if ((bits & 0x7F800000u) != 0x7F800000u) bits += 0x7FFFu + ((bits >> 16) & 1u);
@@ -1049,9 +1073,9 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
       SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], half.data(), h->ema_bytes, cudaMemcpyHostToDevice, s));
       SENTINEL_CUDA(h, cudaStreamSynchronize(s));     // the staging vector goes out of scope
     } else {
-      SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], p, h->N * sizeof(float), cudaMemcpyHostToDevice, s));
+      SENTINEL_CUDA(h, cudaMemcpyAsync(h->ema[k][0], p, h->ema_elems * sizeof(float), cudaMemcpyHostToDevice, s));
     }
-    p += h->N * sizeof(float);
+    p += h->ema_elems * sizeof(float);
   }
   SENTINEL_CUDA(h, cudaMemcpyAsync(h->hs, &st, sizeof st, cudaMemcpyHostToDevice, s));
   SENTINEL_CUDA(h, cudaStreamSynchronize(s));

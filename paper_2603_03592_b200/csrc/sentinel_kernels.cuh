@@ -661,6 +661,8 @@ struct FinalizeTarget {
   const float *sw;                       // [1+B] sliced Wasserstein distances, or nullptr
   int elsewhere;                         // the worker was tainted at another stage: not collected
   int last;                              // the launch ends with this pass: the ticket is re-armed
+  int per_sample_blocks;                 // slots laid out [sample][CTA][segment] (every CTA has rows of every
+                                         // sample) instead of [CTA][segment] tagged with the sample
 };
 
 __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
@@ -695,13 +697,20 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
     long long c_lo = ((long long)b * a.T * a.G) / R - 1, c_hi = ((long long)(b + 1) * a.T * a.G + R - 1) / R;
     if (c_lo < 0) c_lo = 0;
     if (c_hi > a.G - 1) c_hi = a.G - 1;
+    const unsigned long long *block = ft.partials;
+    if (ft.per_sample_blocks) {              // sample b's own block: a slot pair from every CTA
+      c_lo = 0;
+      c_hi = a.G - 1;
+      block += (size_t)b * a.G * kSegsPerCta * kSlotWords;
+    }
     const long long n_slots = (c_hi - c_lo + 1) * kSegsPerCta;
     for (long long q = lane; q < n_slots; q += 32) {
-      const unsigned long long *slot = ft.partials + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
+      const unsigned long long *slot = block + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
       unsigned long long w[kSlotWords];
 #pragma unroll
       for (int j = 0; j < kSlotWords; ++j) w[j] = __ldcg(slot + j);   // one round trip, then the tag
-      if (((w[7] >> kTagShift) & 0xFFull) != (unsigned long long)(b + 1)) continue;
+      const unsigned long long tag = (w[7] >> kTagShift) & 0xFFull;
+      if (ft.per_sample_blocks ? (tag == 0ull) : (tag != (unsigned long long)(b + 1))) continue;
 #pragma unroll
       for (int j = 0; j < 6; ++j) v[j] += __longlong_as_double((long long)w[j]);
       fl += w[6];
@@ -1004,7 +1013,7 @@ stream_kernel_t(const StreamArgs a) {
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const FinalizeTarget ft = {0, a.partials, a.scores_out, a.flags_out, a.sw, 0, 1};
+  const FinalizeTarget ft = {0, a.partials, a.scores_out, a.flags_out, a.sw, 0, 1, 0};
   finalize(a, ft);
 }
 
@@ -1043,8 +1052,11 @@ struct ReplicaShared {
   unsigned x0[kMaxWorkers];                       // the sample's first element, per worker
 };
 
-__device__ void replica_segment(const ReplicaArgs &ra, int b, long long row_a, long long row_b, const float *m_in,
-                                float *m_out, unsigned streamed, int c, int sgm, ReplicaShared &sh) {
+// (n_sets tensors share the tile of m: the R workers of a stage, or the B samples of one tensor
+// when the reference is a single [T,d] tensor for all of them)
+__device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long long row_a, long long row_b,
+                                const float *m_in, float *m_out, unsigned streamed, int c, int sgm,
+                                ReplicaShared &sh) {
   const StreamArgs &a = ra.s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunks = a.d >> 3;                               // d is a multiple of 8 here
@@ -1061,7 +1073,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int b, long long row_a, l
     sh.bits[w][r] = 0u;
   }
   if (threadIdx.x < kWarps) { sh.m_acc[threadIdx.x][0] = sh.m_acc[threadIdx.x][1] = 0.; sh.m_varies[threadIdx.x] = 0u; }
-  if (threadIdx.x < a.R && ((streamed >> threadIdx.x) & 1u)) sh.x0[threadIdx.x] = ra.xs[threadIdx.x][sample_off];
+  if (threadIdx.x < n_sets && ((streamed >> threadIdx.x) & 1u)) sh.x0[threadIdx.x] = ra.xs[threadIdx.x][sample_off];
   const unsigned m0bits = __float_as_uint(m_in[sample_off]);
   const float m0 = __uint_as_float(m0bits);
   __syncthreads();
@@ -1177,7 +1189,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int b, long long row_a, l
 
   __syncthreads();
   // warps -> CTA in a fixed order, one thread per (worker, slot word)
-  if (threadIdx.x < a.R * kSlotWords) {
+  if (threadIdx.x < n_sets * kSlotWords) {
     const int r = threadIdx.x / kSlotWords, w8 = threadIdx.x - r * kSlotWords;
     if ((streamed >> r) & 1u) {
       unsigned long long out;
@@ -1233,7 +1245,7 @@ replica_kernel(const ReplicaArgs ra) {
         const int b = (int)(row / a.T);
         const long long sample_end = (long long)(b + 1) * a.T;
         const long long row_b = sample_end < r1 ? sample_end : r1;
-        replica_segment(ra, b, row, row_b, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
+        replica_segment(ra, a.R, b, row, row_b, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
                         streamed, c, sgm, sh);
         row = row_b;
       } else if (threadIdx.x < a.R) {
@@ -1259,7 +1271,7 @@ replica_kernel(const ReplicaArgs ra) {
                                ra.scores_all + (size_t)r * rows * a.n_metrics,
                                ra.flags_all ? ra.flags_all + (size_t)r * rows : nullptr,
                                ra.sw_all ? ra.sw_all + (size_t)r * rows : nullptr,
-                               (!warmup && ((ra.tainted_in >> r) & 1u)) ? 1 : 0, r == a.R - 1};
+                               (!warmup && ((ra.tainted_in >> r) & 1u)) ? 1 : 0, r == a.R - 1, 0};
     finalize(a, ft);
     __threadfence();                           // the next pass reads the state this one wrote
     __syncthreads();
@@ -1273,6 +1285,49 @@ replica_kernel(const ReplicaArgs ra) {
       ks->mean_done_step = __ldcg(&ks->steps);
     }
   }
+}
+
+// One [T,d] reference for all B samples of a tensor (a variant the paper does not state: the
+// reference of Eq. 1 follows the mean over the samples).  The streaming side is the multi-worker
+// one with the samples in the workers' place -- a tile of m against the B samples' tiles, the
+// candidate m' = beta m + (1-beta)/B sum_b x[b] into the spare buffer -- over the T token rows;
+// the last CTA then finalizes as for any single submission (every sample a unit, all or nothing
+// commit).  2 + 8/B bytes per element of x.
+__global__ void __launch_bounds__(kThreads)
+shared_ref_kernel(const ReplicaArgs ra) {
+  __shared__ ReplicaShared sh;
+  __shared__ int s_last;
+  extern __shared__ double s_dyn[];
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  const StreamArgs &a = ra.s;
+  const int act = __ldcg(&a.hs->kind[a.kind].active);
+  const unsigned all = (a.B >= 32) ? 0xffffffffu : ((1u << a.B) - 1u);
+  if (blockIdx.x == 0) {
+    KindState *ks = &a.hs->kind[a.kind];
+    if (ks->refresh_pending)
+      refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
+  } else {
+    const int c = blockIdx.x - 1;
+    const long long r0 = ((long long)a.T * c) / a.G, r1 = ((long long)a.T * (c + 1)) / a.G;   // token rows
+    replica_segment(ra, a.B, 0, r0, r1, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
+                    all, c, 0, sh);
+    if (threadIdx.x < a.B)                       // the second slot of every pair stays unused
+      ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + 1) * kSlotWords + 7] = 0ull;
+  }
+
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(a.ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const FinalizeTarget ft = {0, ra.partials, a.scores_out, a.flags_out, nullptr, 0, 1, 1};
+  finalize(a, ft);
 }
 
 // Brings both kinds' thresholds up to date outside a streaming launch (queries, export).
@@ -1302,7 +1357,7 @@ __device__ __forceinline__ void st_x128(uint16_t *p, const uint4 &v) {
 
 __global__ void __launch_bounds__(kReplaceThreads)
 replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *ema1, int ema_bf16, uint16_t *x,
-               long long n_chunks, int zero_fill, unsigned *replaced_out) {
+               long long n_chunks, long long ref_chunks, int zero_fill, unsigned *replaced_out) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const KindState *ks = &hs->kind[kind];
   const int flagged = ks->last_flagged;
@@ -1312,10 +1367,11 @@ replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *em
   const long long stride = (long long)gridDim.x * kReplaceThreads;
   for (long long c = (long long)blockIdx.x * kReplaceThreads + threadIdx.x; c < n_chunks; c += stride) {
     uint4 out = make_uint4(0u, 0u, 0u, 0u);
+    const long long cm = ref_chunks ? c % ref_chunks : c;   // a [T,d] reference repeats for every sample
     if (!zero_fill && ema_bf16) {                 // the reference already is a bf16 tensor
-      out = ld_x128(static_cast<const uint16_t *>(m) + c * 8);
+      out = ld_x128(static_cast<const uint16_t *>(m) + cm * 8);
     } else if (!zero_fill) {
-      const F8 v = ld_m256(static_cast<const float *>(m) + c * 8);
+      const F8 v = ld_m256(static_cast<const float *>(m) + cm * 8);
       out.x = pack_bf16x2_rn(v.v[0], v.v[1]);
       out.y = pack_bf16x2_rn(v.v[2], v.v[3]);
       out.z = pack_bf16x2_rn(v.v[4], v.v[5]);

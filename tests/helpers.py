@@ -60,7 +60,8 @@ def oracle_to_blob(v, params) -> bytes:
     """Serialise an oracle verifier into the library's checkpoint format."""
     B, T, d, l, R = params.B, params.T, params.d, params.l, params.R
     M = v.nm                                   # metrics in use; the layout has room for four
-    out = bytearray(struct.pack("<QI6i", MAGIC, 3, B, T, d, l, R, M))
+    shared = int(getattr(params, "ref_over_batch", 0))
+    out = bytearray(struct.pack("<QI7i", MAGIC, 3, B, T, d, l, R, M, shared))
     out += b"\0" * (64 - len(out))
     workers = np.zeros((3, 16), dtype="<i4")
     for r in range(R):
@@ -89,13 +90,13 @@ def oracle_to_blob(v, params) -> bytes:
 def parse_blob(blob, B, T, d, l, R=1) -> dict:
     """Decode a checkpoint blob into plain numpy pieces."""
     buf = memoryview(bytes(blob))
-    magic, version, b, t, dd, ll, rr, M = struct.unpack_from("<QI6i", buf, 0)
+    magic, version, b, t, dd, ll, rr, M, shared = struct.unpack_from("<QI7i", buf, 0)
     assert magic == MAGIC and version == 3 and (b, t, dd, ll, rr) == (B, T, d, l, R) and M in (3, 4)
     workers = np.frombuffer(buf, dtype="<i4", count=48, offset=64).reshape(3, 16)
     off = 64 + 192
     out = {"violations": int(workers[0, 0]), "clean_streak": int(workers[1, 0]), "banned": int(workers[2, 0]),
-           "workers": workers.copy(), "n_metrics": M, "kinds": []}
-    N = B * T * d
+           "workers": workers.copy(), "n_metrics": M, "ref_over_batch": shared, "kinds": []}
+    N = T * d if shared else B * T * d
     for _ in range(2):
         steps, c0, c1 = struct.unpack_from("<q2i", buf, off)
         valid = np.array(struct.unpack_from("<8i", buf, off + 16)).reshape(2, 4).astype(bool)[:, :M]
@@ -108,7 +109,7 @@ def parse_blob(blob, B, T, d, l, R=1) -> dict:
                 if i < M:
                     hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
                 off += 8 * cap
-        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape(B, T, d).copy()
+        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape((T, d) if shared else (B, T, d)).copy()
         off += 4 * N
         out["kinds"].append({"steps": steps, "count": (c0, c1), "valid": valid, "thr": thr,
                              "hist": hist, "m": m})

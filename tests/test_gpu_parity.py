@@ -744,3 +744,71 @@ def test_verify_calls_replay_from_a_cuda_graph(sb):
             assert int(flags[ACT, 4]) & sb.FLAG_L1 and not int(flags[ACT, 0]) & sb.FLAG_COMMITTED
     assert bytes(eager.sentinel_export_state()) == bytes(graphed.sentinel_export_state())
     eager.close(); graphed.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# one [T,d] reference shared by the B samples (ref_over_batch = 1)
+
+@pytest.mark.parametrize("name,shape,steps", [("cfg2", (6, 40, 1024), 50), ("cfg4", (4, 24, 2056), 40),
+                                              ("cfg3", (16, 30, 520), 60), ("cfg2", (1, 37, 264), 40)],
+                         ids=["cfg2_B6", "cfg4_B4", "cfg3_B16", "cfg2_B1"])
+def test_streams_in_lockstep_with_a_shared_reference(sb, oracle_mod, name, shape, steps):
+    w = synth.scaled(synth.WORKLOADS[name], name + "_shared", *shape, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w, ref_over_batch=1)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, steps)
+    assert rec["corrupted"] >= 3
+    compare_state(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+        st = gv.sentinel_get_stats(kind).cpu().numpy()
+        x, _ = synth.microbatch(w, 0, kind, steps - 1, "cuda")
+        assert_stats_close(st, ov.last_stats(kind), max(float(x.float().std()), 1e-30),
+                           max(float(np.abs(ov.last_stats(kind)[0, 4])) ** 0.5, 1e-30), "stats kind %d" % kind)
+    assert rec["near"] <= 2 and rec["k_events"] <= 4, rec
+    # Alg. 4: every sample receives the one reference
+    x, _ = synth.microbatch(w, 0, GRAD, 0, "cuda")
+    loud = (x.float() * 64).to(torch.bfloat16)
+    gv.verify(loud, GRAD)
+    ov.verify(synth.bits(loud), GRAD)
+    out = loud.clone()
+    gv.sentinel_replace_if_flagged(out, GRAD, 0)
+    want, did = ov.replace_if_flagged(synth.bits(loud), GRAD)
+    torch.cuda.synchronize()
+    assert did
+    got = synth.bits(out)
+    gv_, rv_ = oracle_mod.bf16_to_f64(got), oracle_mod.bf16_to_f64(want)
+    assert np.mean(got != want) <= 1e-3 and np.all(np.abs(gv_ - rv_) <= 2.0 ** -7 * np.abs(rv_) + 1e-6 * float(np.std(rv_)))
+    gv.close()
+
+
+def test_shared_reference_restrictions_and_state_round_trip(sb):
+    for kw in ({"n_workers": 2}, {"ema_bf16": 1}):
+        with pytest.raises(sb.SentinelError) as e:
+            sb.Verifier(2, 8, 64, ref_over_batch=1, **kw)
+        assert e.value.code == sb.ERR_UNSUPPORTED
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(17, 8, 64, ref_over_batch=1)
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    gv = sb.Verifier(3, 8, 64, ref_over_batch=1)
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_set_directions(synth.directions(4, 64, 1, "cuda"))
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    s, f = torch.zeros(4, 3, device="cuda"), torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_verify_strided(torch.zeros(3, 8, 65, dtype=torch.bfloat16, device="cuda"), ACT, s, f)
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "shared_rt", 3, 8, 64)
+    for t in range(5):
+        gv.update_reference(synth.clean(w, 0, ACT, t, "cuda"), ACT)
+    blob = bytes(gv.sentinel_export_state())
+    assert len(blob) < len(bytes(sb.Verifier(3, 8, 64).sentinel_export_state()))   # T*d reference values per kind
+    other = sb.Verifier(3, 8, 64, ref_over_batch=1)
+    other.sentinel_import_state(blob)
+    assert bytes(other.sentinel_export_state()) == blob
+    x = synth.clean(w, 0, ACT, 5, "cuda")
+    a, b = gv.verify(x, ACT), other.verify(x, ACT)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(3, 8, 64).sentinel_import_state(blob)                          # another reference shape
+    assert e.value.code == sb.ERR_STATE_SIZE
+    gv.close(); other.close()
