@@ -306,6 +306,28 @@ def run_ours(args, rank, world, local_rank):
                 "tensors_per_s": round(1e3 / hms, 1), "kernel": "stream_kernel_t<false, true>"}
         vh.sentinel_destroy()
 
+    # extra figure, outside the timed region: one [T,d] reference for all samples (2 + 8/B B/element)
+    shared = None
+    if extras and w.B <= 16:
+        vsr = binding.Verifier(w.B, w.T, w.d, device=local_rank, ref_over_batch=1)
+        ss_, sf_ = torch.empty(1 + w.B, 3, dtype=torch.float32, device=device), torch.zeros(1 + w.B, dtype=torch.int32, device=device)
+        for i in range(6):
+            vsr.sentinel_update_reference(xs[0][ACT][i % nd], ACT, ss_, main)
+        vsr.sentinel_verify(xs[0][ACT][6 % nd], ACT, ss_, sf_, main)
+        z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        z0.record(main)
+        for i in range(20):
+            vsr.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, ss_, sf_, main)
+        z1.record(main)
+        torch.cuda.synchronize()
+        zms = z0.elapsed_time(z1) / 20
+        per_el = 2 + 8.0 / w.B
+        shared = {"bytes_per_element": per_el, "ms_per_launch": round(zms, 4),
+                  "achieved_gbs": round(per_el * N / (zms * 1e-3) / 1e9, 1),
+                  "tensors_per_s": round(1e3 / zms, 1), "kernel": "shared_ref_kernel"}
+        vsr.sentinel_destroy()
+
     # extra figure, outside the timed region: the strided (compressed-signal) layout, rows d+1 apart
     strided = None
     if extras:
@@ -398,6 +420,8 @@ def run_ours(args, rank, world, local_rank):
         out["compressed_layout"] = strided
     if half is not None:
         out["bf16_reference"] = half
+    if shared is not None:
+        out["shared_reference"] = shared
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
     return out

@@ -153,3 +153,27 @@ def test_cfg4_bf16_reference_first_update(sb):
     assert float(gs[0, 0]) == pytest.approx(float(x.float().abs().mean()), rel=1e-5)
     assert float(gs[0, 2]) == pytest.approx(float((x != 0).float().mean()), rel=1e-6)
     gv.close()
+
+
+def test_cfg4_shared_reference_of_identical_samples(sb):
+    """4 x 8192 x 8192 with one [T,d] reference: when all samples of every tensor are the same
+    [T,d] slice, the mean over the samples is that slice, so the reference and every sample's
+    scores are those of a one-sample verifier fed the slice (the reference bit for bit)."""
+    w = synth.WORKLOADS["cfg4"]
+    one = sb.Verifier(1, w.T, w.d)
+    shared = sb.Verifier(w.B, w.T, w.d, ref_over_batch=1)
+    for t in range(4):
+        sl = synth.clean(w, 0, ACT, t, "cuda")[:1].contiguous()
+        x = sl.expand(w.B, w.T, w.d).contiguous()
+        s1 = one.update_reference(sl, ACT)
+        ss = shared.update_reference(x, ACT)
+        torch.cuda.synchronize()
+        for r in range(1 + w.B):                 # the whole tensor is B copies of the slice: same scores again
+            assert torch.allclose(ss[r], s1[1], rtol=1e-5, atol=1e-7), (t, r)
+    n = 4 * w.T * w.d
+    def act_reference(v):
+        blob = v.sentinel_export_state()
+        per_kind = (v.sentinel_state_bytes() - 64 - 192) // 2
+        return np.frombuffer(blob, dtype=np.uint8, count=n, offset=64 + 192 + per_kind - n)
+    assert np.array_equal(act_reference(one), act_reference(shared))
+    one.close(); shared.close()
