@@ -19,9 +19,17 @@
  *                                         constant vector z-scores to zero)
  *                                2  SFR   fraction of elements with sign(x) != sign(m),
  *                                         sign in {-1,0,+1}
+ *                                3  SW    sliced Wasserstein distance of the token clouds; only
+ *                                         after sentinel_set_directions (else three metrics)
  *
- * Conventions.  All tensors are dense, row-major [B,T,d] with d fastest.  x is bf16; the
- * reference m is fp32 and owned by the library.  Pointers named dev_* are device pointers on
+ * Variants of a handle (sentinel_config): n_workers > 1 follows all workers of a stage and takes
+ * their tensors together (the fixed-mesh form of Eq. 1, worker loop of Alg. 2 / Alg. 3);
+ * ema_bf16 stores the reference as bf16; ref_over_batch keeps one [T,d] reference for all
+ * samples.
+ *
+ * Conventions.  All tensors are dense, row-major [B,T,d] with d fastest (the _strided entry
+ * points take padded rows).  x is bf16; the reference m is fp32 unless ema_bf16 is set, and is
+ * owned by the library.  Pointers named dev_* are device pointers on
  * the handle's device, host_* are host pointers.  `cuda_stream` is a cudaStream_t passed as
  * void* (NULL = the legacy default stream).  Calls only enqueue work unless stated otherwise;
  * outputs are valid once the stream reaches that point.  A handle is not thread-safe and its

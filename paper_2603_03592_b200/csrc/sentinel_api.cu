@@ -193,7 +193,6 @@ int check_call_strided(sentinel_verifier *h, const void *x, int kind, int B, int
   if (reinterpret_cast<uintptr_t>(x) & 1u) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 2-byte aligned");
   if (h->sw_u) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein metric reads dense rows: a verifier with directions takes no strided tensor");
   if (h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "a verifier with a [T,d] reference takes no strided tensor");
-  h->started = true;
   return SENTINEL_OK;
 }
 
@@ -554,6 +553,7 @@ int sentinel_verify_strided(sentinel_verifier *h, const void *dev_x, sentinel_ki
   if (!dev_scores_out || !dev_flags_out) return fail(h, SENTINEL_ERR_INVALID_ARG, "scores_out or flags_out is NULL");
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
+  h->started = true;
   StreamArgs a = make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out);
   a.x_row_stride = row_stride;
   return launch(h, a, h->G + 1, static_cast<cudaStream_t>(cuda_stream), true);
@@ -565,6 +565,7 @@ int sentinel_update_reference_strided(sentinel_verifier *h, const void *dev_x, s
   if (rc) return rc;
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
+  h->started = true;
   StreamArgs a = make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr);
   a.x_row_stride = row_stride;
   return launch(h, a, h->G + 1, static_cast<cudaStream_t>(cuda_stream), true);
