@@ -45,7 +45,8 @@ def oracle_distance_all(oracle_mod, xb, m64):
 
 
 SHAPES = [(1, 1, 8), (2, 3, 8), (1, 7, 16), (3, 5, 520), (4, 33, 1024), (8, 128, 512),
-          (2, 19, 4104), (5, 64, 2048), (64, 2, 64), (3, 1, 8192), (2, 300, 136)]
+          (2, 19, 4104), (5, 64, 2048), (64, 2, 64), (3, 1, 8192), (2, 300, 136),
+          (1, 2, 65536), (2, 5000, 8), (64, 1, 8)]
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
@@ -292,6 +293,24 @@ def test_long_streams_with_small_windows(sb, oracle_mod, shape, l):
     for kind in (ACT, GRAD):
         compare_thresholds(gv, ov, kind)
     assert rec["near"] + rec["k_events"] <= 6, rec
+    gv.close()
+
+
+def test_stream_at_the_largest_batch_and_window(sb, oracle_mod):
+    """B = 64 samples (the compiled maximum) with the longest window that fits: 63 * 65 = 4095
+    entries per kind across the two levels."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "max_b", 64, 6, 72, corrupt_rate=0.2, warmup=8)
+    gv, ov, params = make_pair(sb, oracle_mod, w, l=63)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, 75, kinds=(ACT,))
+    compare_state(gv, ov, params)
+    compare_thresholds(gv, ov, ACT)
+    assert rec["near"] <= 2 and rec["k_events"] <= 4, rec
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(64, 6, 72, window_steps=64)             # 64 * 65 = 4160 > 4096
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(65, 6, 72, window_steps=10)
+    assert e.value.code == sb.ERR_UNSUPPORTED
     gv.close()
 
 
