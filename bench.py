@@ -193,7 +193,7 @@ def run_ours(args, rank, world, local_rank):
     violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
 
     # extra figure, outside the timed region: gradient replacement (Alg. 4) after a flagged step
-    extras = nb == 1 and args.extras
+    extras = nb == 1 and args.extras and world == 1     # the extra figures are single-GPU figures
     replace = None
     if extras:
         v0 = vs[0]
