@@ -106,12 +106,13 @@ class ClockSampler:
 
 def build_stream(w, boundary, device, count, distinct):
     """`count` microbatches per kind after the warm-up, following the workload's recipe."""
-    xs = {ACT: [], GRAD: []}
+    xs = {ACT: [], GRAD: [], "corrupted": {ACT: [], GRAD: []}}
     n = min(count, distinct)
     for kind in (ACT, GRAD):
         for i in range(n):
-            x, _ = synth.microbatch(w, boundary, kind, w.warmup + i, device)
+            x, name = synth.microbatch(w, boundary, kind, w.warmup + i, device)
             xs[kind].append(x)
+            xs["corrupted"][kind].append(name is not None)
     return xs
 
 
@@ -140,12 +141,13 @@ def run_ours(args, rank, world, local_rank):
     nd = len(xs[0][ACT])
     scores = torch.empty(nb, 2, 1 + w.B, 3, dtype=torch.float32, device=device)
     flags = torch.empty(nb, 2, 1 + w.B, dtype=torch.int32, device=device)
+    flag_log = torch.zeros(total, nb, 2, 1 + w.B, dtype=torch.int32, device=device)   # every step's flags
     torch.cuda.synchronize()
 
     def step(i):
         for b, (v, s) in enumerate(zip(vs, streams)):
-            v.sentinel_verify(xs[b][ACT][i % nd], ACT, scores[b, 0], flags[b, 0], s)
-            v.sentinel_verify(xs[b][GRAD][i % nd], GRAD, scores[b, 1], flags[b, 1], s)
+            v.sentinel_verify(xs[b][ACT][i % nd], ACT, scores[b, 0], flag_log[i, b, 0], s)
+            v.sentinel_verify(xs[b][GRAD][i % nd], GRAD, scores[b, 1], flag_log[i, b, 1], s)
 
     def fork():                                      # side streams start after `main` gets here
         if nb > 1:
@@ -191,6 +193,23 @@ def run_ours(args, rank, world, local_rank):
     elapsed_ms = replicas.max_over_ranks(elapsed_ms)
     launches = 2 * args.steps * nb
     violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
+    # what the detector said on the timed steps (reported, not a target: some of the recipe's
+    # corruptions are statistically invisible to these metrics, and a flagged tensor that comes
+    # round again is flagged again)
+    raised = ((flag_log[args.warmup:] & 0xFFFF) != 0).any(dim=-1).cpu()              # [steps, nb, 2]
+    n_corrupted = n_flagged = n_both = 0
+    for i in range(args.steps):
+        for b in range(nb):
+            for kind in (ACT, GRAD):
+                c = xs[b]["corrupted"][kind][(args.warmup + i) % nd]
+                f = bool(raised[i, b, kind])
+                n_corrupted += c
+                n_flagged += f
+                n_both += c and f
+    detection = {"tensors": args.steps * nb * 2, "corrupted": n_corrupted, "flagged": n_flagged,
+                 "corrupted_and_flagged": n_both, "distinct_tensors_per_kind": nd,
+                 "note": "the stream cycles through the distinct tensors; one that comes round again soon "
+                         "correlates with the reference that absorbed it and is flagged as a replay"}
 
     # extra figure, outside the timed region: gradient replacement (Alg. 4) after a flagged step
     extras = nb == 1 and args.extras and world == 1     # the extra figures are single-GPU figures
@@ -393,7 +412,7 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step_best": round(step_ms[0], 4),
         "frac_of_8000_nominal": round(gbs / world / 8000.0, 4),
         "gpu_launches": launches,
-        "violations_seen": violations,
+        "violations_seen": violations, "detection": detection,
         "clocks": clocks.summary(),
         "e2e": {"value": round(e2e_gbs, 2), "unit": "GB/s", "steps": e2e_steps,
                 "h2d_bytes_per_step": 2 * N * 2 * nb,
