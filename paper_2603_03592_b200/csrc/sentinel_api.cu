@@ -236,8 +236,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
 int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, bool scalar = false) {
   // launched with programmatic stream serialization: the grid may be set up while the previous
   // kernel on the stream drains; every CTA waits for that kernel before it reads anything
-  cudaLaunchConfig_t lc;
-  memset(&lc, 0, sizeof lc);
+  cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)grid);
   lc.blockDim = dim3(kThreads);
   lc.dynamicSmemBytes = h->refresh_smem;
@@ -688,8 +687,7 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigne
     if (rc) return rc;
   }
   {   // every worker against the same m_{t-1}, in one launch
-    cudaLaunchConfig_t lc;
-    memset(&lc, 0, sizeof lc);
+    cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)(h->G + 1));
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = h->refresh_smem;
