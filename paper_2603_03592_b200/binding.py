@@ -134,7 +134,10 @@ def _ptr(t) -> int:
 def sentinel_default_config(**overrides) -> sentinel_config:
     cfg = sentinel_config()
     _check(lib().sentinel_default_config(C.byref(cfg)))
+    known = {name for name, _ in sentinel_config._fields_}
     for k, v in overrides.items():
+        if k not in known:
+            raise TypeError("sentinel_config has no field %r" % k)
         cur = getattr(cfg, k)
         if hasattr(cur, "__len__"):
             cur[0], cur[1] = v
