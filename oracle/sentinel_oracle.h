@@ -18,6 +18,13 @@
  *   - the "x100 above the threshold" severe-deviation rule of Sec. 3.1,
  *   - the forgiveness bookkeeping ("decrements after T_forgiveness consecutive clean steps"),
  *   - the percentile convention (linear interpolation at p*(n-1)).
+ *   - how a worker tainted at another stage enters this stage's bookkeeping (Alg. 2 leaves it
+ *     out of its loop, Alg. 3 adds it to the stage's tainted set: read literally, per kind; a
+ *     worker that was not collected never enters the mean of Eq. 1),
+ *   - the number and the draw of the sliced Wasserstein directions (the caller supplies them),
+ *   - the two storage variants the paper does not mention: a reference stored as bf16 (its
+ *     rounding is pinned to an independent single-precision computation, the choice of the
+ *     variant itself is not the paper's) and one [T,d] reference for all samples of a tensor.
  */
 #ifndef SENTINEL_ORACLE_H
 #define SENTINEL_ORACLE_H

@@ -79,6 +79,26 @@ def test_host_side_argument_checks_need_no_gpu(built):
     assert not h.value
     cfg = binding.sentinel_default_config(B=2, T=0, d=16)
     assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_INVALID_ARG
+    # calls that take a handle refuse NULL before anything else
+    assert L.sentinel_num_metrics(None) == 0
+    assert L.sentinel_set_directions(None, None, 8, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_skip_tainted(None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_verify(None, None, 0, 1, 1, 8, None, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_verify_replicas(None, None, 0, 1, 1, 8, None, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_verify_replicas_tainted(None, None, 0, 1, 1, 1, 8, None, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_verify_strided(None, None, 0, 1, 1, 8, 9, None, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_replace_if_flagged(None, None, 0, 1, 1, 8, 0, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_import_state(None, None, 0, None) == binding.ERR_INVALID_ARG
+    # stateless calls check their pointers and shapes on the host
+    assert L.sentinel_distance(None, None, 1, 1, 8, 0, None, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_sliced_wasserstein(None, None, None, 8, 1, 1, 8, 0, None, None) == binding.ERR_INVALID_ARG
+    assert L.sentinel_distance_noalloc(None, None, 1, 1, 8, 0, None, None, None) == binding.ERR_INVALID_ARG
+    # configuration ranges
+    for bad in (dict(n_workers=17), dict(ema_bf16=2), dict(ref_over_batch=3), dict(window_steps=0)):
+        cfg = binding.sentinel_default_config(B=2, T=4, d=16, **bad)
+        assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_INVALID_ARG, bad
+    with pytest.raises(TypeError):
+        binding.sentinel_default_config(B=2, T=4, d=16, no_such_field=1)
 
 
 def test_product_path_does_not_touch_the_oracle():
