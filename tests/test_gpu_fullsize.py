@@ -177,3 +177,31 @@ def test_cfg4_shared_reference_of_identical_samples(sb):
         return np.frombuffer(blob, dtype=np.uint8, count=n, offset=64 + 192 + per_kind - n)
     assert np.array_equal(act_reference(one), act_reference(shared))
     one.close(); shared.close()
+
+
+def test_cfg4_sliced_wasserstein_units(sb, oracle_mod):
+    """4 x 8192 x 8192, 8 directions.  Two samples against the float64 oracle (projections of
+    8192 tokens in R^8192 each); and the whole-tensor unit through a property: a tensor made of
+    four copies of one sample, against a reference made of four copies of one slice, has the
+    same empirical distributions along every direction as the single sample, hence the same
+    distance."""
+    w = synth.WORKLOADS["cfg4"]
+    u = synth.directions(8, w.d, 5, "cuda")
+    x = synth.clean(w, 0, ACT, 0, "cuda")
+    m = (0.7 * synth.clean(w, 0, ACT, 1, "cuda").float() + 0.05).contiguous()
+    out = torch.empty(1 + w.B, device="cuda")
+    sb.sentinel_sliced_wasserstein(x, m, u, out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    ub = synth.bits(u)
+    for b in (0, 3):
+        want = oracle_mod.sliced_wasserstein(synth.bits(x[b]), m[b].double().cpu().numpy(), ub)[0]
+        assert abs(got[1 + b] - want) <= 1e-3 * want, (b, got[1 + b], want)
+    assert np.all(np.isfinite(got)) and got[0] > 0
+    xs = x[:1].expand(w.B, w.T, w.d).contiguous()
+    ms = m[:1].expand(w.B, w.T, w.d).contiguous()
+    sb.sentinel_sliced_wasserstein(xs, ms, u, out)
+    torch.cuda.synchronize()
+    tiled = out.cpu().numpy().astype(np.float64)
+    assert np.allclose(tiled[1:], got[1], rtol=1e-6)
+    assert tiled[0] == pytest.approx(got[1], rel=1e-5)
