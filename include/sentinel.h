@@ -156,9 +156,11 @@ int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
  * dev_u_bf16: bf16 [L, d] unit directions chosen by the caller (the paper fixes neither
  * their number nor their draw), 16-byte aligned; copied on cuda_stream, and the call waits
  * for it.  L must be 4, 8 or 16; L*d*2 bytes <= 200 KiB; T <= 16384; d a multiple of 8.
- * Every later step first runs the projection / sort launches on the caller's stream (they
- * read x and the reference once more: 6 B/element on top of the streaming pass), then the
- * streaming launch, which picks the distances up.  The projections are fp32: inputs whose
+ * Every later step first runs the projection / sort launches on the caller's stream, then the
+ * streaming launch, which picks the distances up.  With one submission per update the
+ * projections of the reference are carried along from step to step (Eq. 1 is linear), so the
+ * chain reads x once more (2 B/element) and not the reference; with n_workers > 1, and on the
+ * first step after sentinel_import_state, it reads the reference too (6 B/element).  The projections are fp32: inputs whose
  * projections leave the fp32 range give a score that is not a number, which counts as a
  * flag.  Allowed only before the first step and before sentinel_import_state
  * (SENTINEL_ERR_INVALID_ARG afterwards); the four windows' working copies must fit the

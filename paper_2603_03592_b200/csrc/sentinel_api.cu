@@ -57,6 +57,8 @@ struct sentinel_verifier {
   uint16_t *sw_u = nullptr;         // directions, bf16 [sw_L][d]
   float *sw_scratch = nullptr;      // projections and sorted lists
   float *sw_out = nullptr;          // [1+B] distances of the submission being checked
+  double *sw_pm[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // per kind: projections of the reference, [B*T][L], current and spare
+  bool sw_pm_valid[2] = {false, false};   // they match the reference (not so right after a state import)
   void *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // fp32, or bf16 if bf16
   bool bf16 = false;                // the reference is stored as bf16
   bool shared_ref = false;          // one [T,d] reference for all B samples
@@ -287,21 +289,30 @@ struct DeviceGuard {   // restores the caller's current device
 // sliced Wasserstein distance: the chain of launches, shared by the stateless entry point and
 // by verifiers that carry it as their fourth metric
 
-template <int L, int kT>
+// What a verifier adds to the projection launch: its own projections of the reference (kept up
+// to date through the linearity of Eq. 1) and the coefficients of that update.
+struct ProjectionState {
+  double *pm0 = nullptr, *pm1 = nullptr;   // [rows][L] each; nullptr: stateless
+  bool incremental = false;                // take P(m) from the buffers instead of reading m
+  float beta = 0.f, one_minus_beta = 0.f;
+};
+
+template <int L, int kT, bool kIncr>
 cudaError_t projection_occupancy(size_t smem, int *occ) {
-  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT, kIncr>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT>, kT, smem);
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT, kIncr>, kT, smem);
 }
 
-template <int L>
+template <int L, bool kIncr>
 cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
-                              const uint16_t *u, float *proj, long long rows, int d, int sms, cudaStream_t s) {
+                              const uint16_t *u, float *proj, long long rows, int d, int sms, const ProjectionState &ps,
+                              cudaStream_t s) {
   const size_t smem = (size_t)L * d * sizeof(uint16_t);
   int occ_small = 0, occ_large = 0;
-  cudaError_t e = projection_occupancy<L, 512>(smem, &occ_small);
+  cudaError_t e = projection_occupancy<L, 512, kIncr>(smem, &occ_small);
   if (e != cudaSuccess) return e;
-  e = projection_occupancy<L, 768>(smem, &occ_large);
+  e = projection_occupancy<L, 768, kIncr>(smem, &occ_large);
   if (e != cudaSuccess) return e;
   const bool large = occ_large * 768 > occ_small * 512;
   const int threads = large ? 768 : 512, occ = large ? occ_large : occ_small;
@@ -309,8 +320,12 @@ cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m
   long long grid = (long long)sms * occ;
   const long long need = (rows + threads / 32 - 1) / (threads / 32);
   if (grid > need) grid = need;
-  if (large) swd_project_kernel<L, 768><<<(unsigned)grid, 768, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d);
-  else swd_project_kernel<L, 512><<<(unsigned)grid, 512, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d);
+  if (large)
+    swd_project_kernel<L, 768, kIncr><<<(unsigned)grid, 768, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d, ps.pm0,
+                                                                        ps.pm1, ps.beta, ps.one_minus_beta);
+  else
+    swd_project_kernel<L, 512, kIncr><<<(unsigned)grid, 512, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d, ps.pm0,
+                                                                        ps.pm1, ps.beta, ps.one_minus_beta);
   return cudaGetLastError();
 }
 
@@ -331,15 +346,21 @@ int check_swd_shape(sentinel_verifier *h, int L, int T, int d) {
 // nothing runs if *skip != 0 (both read on the device; either may be nullptr).
 cudaError_t run_swd(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                     const uint16_t *u, int L, int B, int T, int d, int sms, float *scratch, float *out,
-                    cudaStream_t s) {
+                    const ProjectionState &ps, cudaStream_t s) {
   const long long rows = (long long)B * T;
   const size_t list_floats = (size_t)2 * L * rows;        // L lists for x, L for m
   float *proj = scratch, *buf_a = proj + list_floats, *buf_b = buf_a + list_floats, *w1_sample = buf_b + list_floats;
   float *w1_tensor = w1_sample + (size_t)B * L;
   cudaError_t e;
-  if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, s);
-  else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, s);
-  else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, s);
+  if (ps.incremental) {
+    if (L == 4) e = launch_projection<4, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    else if (L == 8) e = launch_projection<8, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    else e = launch_projection<16, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+  } else {
+    if (L == 4) e = launch_projection<4, false>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    else if (L == 8) e = launch_projection<8, false>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    else e = launch_projection<16, false>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+  }
   if (e != cudaSuccess) return e;
   int npad = 1;
   while (npad < T) npad <<= 1;
@@ -369,10 +390,19 @@ int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bo
   if (!h->sw_u) return SENTINEL_OK;
   int sms = 0;
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
+  ProjectionState ps;
+  if (h->R == 1) {       // one submission per update: the reference's projections follow it (Eq. 1 is linear)
+    ps.pm0 = h->sw_pm[kind][0];
+    ps.pm1 = h->sw_pm[kind][1];
+    ps.incremental = h->sw_pm_valid[kind];
+    ps.beta = (float)h->cfg.beta[kind];
+    ps.one_minus_beta = (float)(1.0 - h->cfg.beta[kind]);
+  }
   SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), static_cast<const float *>(h->ema[kind][0]),
                            static_cast<const float *>(h->ema[kind][1]), &h->hs->kind[kind].active,
                            may_skip ? &h->hs->banned[worker] : nullptr, h->sw_u, h->sw_L, h->cfg.B, h->cfg.T,
-                           h->cfg.d, sms, h->sw_scratch, h->sw_out + (size_t)worker * (1 + h->cfg.B), s));
+                           h->cfg.d, sms, h->sw_scratch, h->sw_out + (size_t)worker * (1 + h->cfg.B), ps, s));
+  if (h->R == 1) h->sw_pm_valid[kind] = true;      // that launch (re)computed them from m if they were stale
   return SENTINEL_OK;
 }
 
@@ -393,6 +423,8 @@ void free_all(sentinel_verifier *h) {
   cudaFree(h->sw_u);
   cudaFree(h->sw_scratch);
   cudaFree(h->sw_out);
+  for (int k = 0; k < 2; ++k)
+    for (int j = 0; j < 2; ++j) cudaFree(h->sw_pm[k][j]);
 }
 
 }  // namespace
@@ -787,14 +819,30 @@ int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L,
   if (e == cudaSuccess) e = cudaMalloc((void **)&scratch, swd_scratch_floats(L, h->cfg.B, h->cfg.T) * sizeof(float));
   const size_t out_floats = (size_t)h->R * (1 + h->cfg.B);      // a block of 1+B per worker
   if (e == cudaSuccess) e = cudaMalloc((void **)&out, out_floats * sizeof(float));
+  // the reference's own projections, per kind, current and spare: m_0 = 0 projects to 0
+  const size_t pm_bytes = (size_t)h->cfg.B * h->cfg.T * L * sizeof(double);
+  double *pm[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
+  for (int k = 0; k < 2; ++k)
+    for (int j = 0; j < 2; ++j) {
+      if (e == cudaSuccess) e = cudaMalloc((void **)&pm[k][j], pm_bytes);
+      if (e == cudaSuccess) e = cudaMemsetAsync(pm[k][j], 0, pm_bytes, s);
+    }
   if (e == cudaSuccess) e = cudaMemcpyAsync(u, dev_u_bf16, u_bytes, cudaMemcpyDeviceToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(out, 0, out_floats * sizeof(float), s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
     cudaFree(u); cudaFree(scratch); cudaFree(out);
+    for (int k = 0; k < 2; ++k)
+      for (int j = 0; j < 2; ++j) cudaFree(pm[k][j]);
     return fail(h, SENTINEL_ERR_CUDA, "setting the directions failed: %s", cudaGetErrorString(e));
   }
   cudaFree(h->sw_u); cudaFree(h->sw_scratch); cudaFree(h->sw_out);   // directions set twice before the first step
+  for (int k = 0; k < 2; ++k)
+    for (int j = 0; j < 2; ++j) {
+      cudaFree(h->sw_pm[k][j]);
+      h->sw_pm[k][j] = pm[k][j];
+    }
+  h->sw_pm_valid[0] = h->sw_pm_valid[1] = true;
   h->sw_u = u; h->sw_scratch = scratch; h->sw_out = out;
   h->sw_L = L;
   h->n_metrics = kNumMetrics;
@@ -825,7 +873,8 @@ int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const voi
   keep_pool_warm(device);
   SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, swd_scratch_floats(L, B, T) * sizeof(float), s));
   cudaError_t e = run_swd(static_cast<const uint16_t *>(dev_x), dev_m, nullptr, nullptr, nullptr,
-                          static_cast<const uint16_t *>(dev_u_bf16), L, B, T, d, sms, scratch, dev_sw_out, s);
+                          static_cast<const uint16_t *>(dev_u_bf16), L, B, T, d, sms, scratch, dev_sw_out,
+                          ProjectionState(), s);
   cudaError_t fe = cudaFreeAsync(scratch, s);
   SENTINEL_CUDA(nullptr, e);
   SENTINEL_CUDA(nullptr, fe);
@@ -1020,6 +1069,7 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
 
   h->started = true;
+  h->sw_pm_valid[0] = h->sw_pm_valid[1] = false;   // the next step recomputes the reference's projections from m
   HandleState st;
   memset(&st, 0, sizeof st);
   BlobWorkers bw;

@@ -21,29 +21,51 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 // The reference is m1 if *active is non-zero, else m0 (a verifier keeps two buffers and flips
 // between them on the device); every kernel of the chain returns at once if *skip is non-zero
 // (a banned worker's tensor is not read).  Both pointers may be nullptr.
-template <int L, int kSwdThreads>
+//
+// Projection is linear and so is Eq. 1: the projections of the reference obey
+//   P(m_t) = beta P(m_{t-1}) + (1-beta) P(x_t)
+// whenever the reference moves.  A verifier therefore keeps P(m) itself ([rows][L] doubles, two
+// buffers pm0 / pm1 selected by the same `active` word as the reference, so a step that does not
+// commit leaves them alone): this kernel always writes the candidate P(m_t) into the spare one,
+// and with kIncr = true it takes P(m_{t-1}) from the current one instead of reading m at all --
+// 2 B/element of traffic instead of 6.  kIncr = false computes it from m (and stores it, if
+// the buffers are given): the stateless call, and the first step after a state import.
+template <int L, int kSwdThreads, bool kIncr>
 __global__ void __launch_bounds__(kSwdThreads, kSwdThreads == 512 ? 2 : 1)
 swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
-                   const uint16_t *u, float *proj, long long rows, int d) {
+                   const uint16_t *u, float *proj, long long rows, int d, double *pm0, double *pm1, float beta,
+                   float one_minus_beta) {
   extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
   if (skip && __ldcg(skip)) return;
-  const float *m = (active && __ldcg(active)) ? m1 : m0;
+  const bool second = active && __ldcg(active);
+  const float *m = second ? m1 : m0;
+  double *pm_cur = second ? pm1 : pm0, *pm_next = second ? pm0 : pm1;
   const int chunks = d >> 3;
   for (int i = threadIdx.x; i < L * chunks; i += kSwdThreads)
     s_u[i] = reinterpret_cast<const uint4 *>(u)[i];
   __syncthreads();
 
+  // A warp owns kRows whole rows at a time; with two rows every direction word fetched from shared
+  // memory serves both (without the reference to read, shared memory is the busier path).
+  constexpr int kRows = (kIncr && L <= 8) ? 2 : 1;     // (16 directions leave no registers for a second row)
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (kSwdThreads / 32) + (threadIdx.x >> 5);
   const long long n_warps = (long long)gridDim.x * (kSwdThreads / 32);
-  for (long long row = warp; row < rows; row += n_warps) {
-    float ax[L], am[L];
+  for (long long row0 = warp * kRows; row0 < rows; row0 += n_warps * kRows) {
+    float ax[kRows][L], am[L];
 #pragma unroll
-    for (int l = 0; l < L; ++l) { ax[l] = 0.f; am[l] = 0.f; }
-    const size_t off = (size_t)row * d;
-    // two chunks per trip, their four loads issued before any arithmetic (more bytes in flight)
+    for (int l = 0; l < L; ++l) {
+      am[l] = 0.f;
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) ax[r][l] = 0.f;
+    }
+    bool live[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) live[r] = row0 + r < rows;
+    const size_t off = (size_t)row0 * d;
+    // two chunks per trip, their loads issued before any arithmetic (more bytes in flight)
     for (int c0 = lane; c0 < chunks; c0 += 64) {
-      uint4 xv[2];
+      uint4 xv[kRows][2];
       F8 mv[2];
       bool ok[2];
 #pragma unroll
@@ -51,20 +73,25 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
         const int c = c0 + 32 * h;
         ok[h] = c < chunks;
         if (ok[h]) {
-          xv[h] = ld_x128(x + off + (size_t)c * 8);
-          mv[h] = ld_m256(m + off + (size_t)c * 8);
+#pragma unroll
+          for (int r = 0; r < kRows; ++r)
+            if (live[r]) xv[r][h] = ld_x128(x + off + (size_t)r * d + (size_t)c * 8);
+          if (!kIncr) mv[h] = ld_m256(m + off + (size_t)c * 8);
         }
       }
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (!ok[h]) continue;
         const int c = c0 + 32 * h;
-        const unsigned xw[4] = {xv[h].x, xv[h].y, xv[h].z, xv[h].w};
-        float xf[8];
+        float xf[kRows][8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          xf[2 * j] = __uint_as_float(xw[j] << 16);
-          xf[2 * j + 1] = __uint_as_float(xw[j] & 0xFFFF0000u);
+        for (int r = 0; r < kRows; ++r) {
+          const unsigned xw[4] = {xv[r][h].x, xv[r][h].y, xv[r][h].z, xv[r][h].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            xf[r][2 * j] = live[r] ? __uint_as_float(xw[j] << 16) : 0.f;
+            xf[r][2 * j + 1] = live[r] ? __uint_as_float(xw[j] & 0xFFFF0000u) : 0.f;
+          }
         }
 #pragma unroll
         for (int l = 0; l < L; ++l) {
@@ -73,20 +100,36 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float u_lo = __uint_as_float(uw[j] << 16), u_hi = __uint_as_float(uw[j] & 0xFFFF0000u);
-            ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
-            ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
-            am[l] = fmaf(mv[h].v[2 * j], u_lo, am[l]);
-            am[l] = fmaf(mv[h].v[2 * j + 1], u_hi, am[l]);
+#pragma unroll
+            for (int r = 0; r < kRows; ++r) {
+              ax[r][l] = fmaf(xf[r][2 * j], u_lo, ax[r][l]);
+              ax[r][l] = fmaf(xf[r][2 * j + 1], u_hi, ax[r][l]);
+            }
+            if (!kIncr) {
+              am[l] = fmaf(mv[h].v[2 * j], u_lo, am[l]);
+              am[l] = fmaf(mv[h].v[2 * j + 1], u_hi, am[l]);
+            }
           }
         }
       }
     }
 #pragma unroll
-    for (int l = 0; l < L; ++l) {
-      const float sx = warp_sum(ax[l]), sm = warp_sum(am[l]);
-      if (lane == l) {
-        proj[(size_t)l * rows + row] = sx;
-        proj[((size_t)L + l) * rows + row] = sm;
+    for (int r = 0; r < kRows; ++r) {
+      const long long row = row0 + r;
+#pragma unroll
+      for (int l = 0; l < L; ++l) {
+        const float sx = warp_sum(ax[r][l]);
+        const float sm = kIncr ? 0.f : warp_sum(am[l]);
+        if (lane == l && live[r]) {
+          const size_t at = (size_t)row * L + l;
+          const double p_cur = kIncr ? pm_cur[at] : (double)sm;
+          proj[(size_t)l * rows + row] = sx;
+          proj[((size_t)L + l) * rows + row] = (float)p_cur;
+          if (pm_cur) {
+            if (!kIncr) pm_cur[at] = p_cur;
+            pm_next[at] = (double)beta * p_cur + (double)one_minus_beta * (double)sx;
+          }
+        }
       }
     }
   }

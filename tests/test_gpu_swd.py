@@ -155,7 +155,10 @@ def test_streams_in_lockstep_with_four_metrics(sb, oracle_mod, name, shape, L, s
 
 def test_fourth_column_equals_the_stateless_distance(sb, oracle_mod):
     """Column 3 of a verified step is sentinel_sliced_wasserstein of the same tensor against the
-    reference the step was tested with (exported just before), bit for bit."""
+    reference the step was tested with (exported just before).  Not bit for bit: the verifier
+    carries the reference's projections along (float64 recursion of Eq. 1 on the projections)
+    where the stateless call projects the fp32 reference afresh.  Right after a state import the
+    verifier projects the reference afresh too, and the two agree exactly."""
     w = synth.scaled(synth.WORKLOADS["cfg2"], "sw_col", 3, 50, 512)
     gv, ov, params = make_pair(sb, oracle_mod, w)
     u = with_directions(gv, ov, 8, w.d)
@@ -168,7 +171,23 @@ def test_fourth_column_equals_the_stateless_distance(sb, oracle_mod):
     want = torch.empty(1 + w.B, device="cuda")
     sb.sentinel_sliced_wasserstein(x, m, u, want)
     torch.cuda.synchronize()
-    assert torch.equal(gs[:, 3], want)
+    assert torch.allclose(gs[:, 3], want, rtol=2e-5, atol=0)
+    # a state import invalidates the carried projections: the next step recomputes them from m
+    blob = gv.sentinel_export_state()
+    m2 = torch.from_numpy(parse_blob(blob, w.B, w.T, w.d, params.l)["kinds"][ACT]["m"]).cuda()
+    gv.sentinel_import_state(blob)
+    x2 = synth.clean(w, 0, ACT, 6, "cuda")
+    gs2, _ = gv.verify(x2, ACT)
+    sb.sentinel_sliced_wasserstein(x2, m2, u, want)
+    torch.cuda.synchronize()
+    assert torch.equal(gs2[:, 3], want)
+    # ... and the steps after that carry them along again
+    m3 = torch.from_numpy(parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, params.l)["kinds"][ACT]["m"]).cuda()
+    x3 = synth.clean(w, 0, ACT, 7, "cuda")
+    gs3, _ = gv.verify(x3, ACT)
+    sb.sentinel_sliced_wasserstein(x3, m3, u, want)
+    torch.cuda.synchronize()
+    assert torch.allclose(gs3[:, 3], want, rtol=2e-5, atol=0)
     gv.close()
 
 
