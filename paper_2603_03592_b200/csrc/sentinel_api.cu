@@ -297,22 +297,38 @@ struct ProjectionState {
   float beta = 0.f, one_minus_beta = 0.f;
 };
 
-template <int L, int kT, bool kIncr>
-cudaError_t projection_occupancy(size_t smem, int *occ) {
-  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT, kIncr>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT, kIncr>, kT, smem);
+// One launch of the chain, with programmatic stream serialization (see chain_entry()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(grid);
+  lc.blockDim = dim3(block);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
 }
 
-template <int L, bool kIncr>
+template <int L, int kT>
+cudaError_t projection_occupancy(size_t smem, int *occ) {
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT>, kT, smem);
+}
+
+template <int L>
 cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                               const uint16_t *u, float *proj, long long rows, int d, int sms, const ProjectionState &ps,
                               cudaStream_t s) {
   const size_t smem = (size_t)L * d * sizeof(uint16_t);
   int occ_small = 0, occ_large = 0;
-  cudaError_t e = projection_occupancy<L, 512, kIncr>(smem, &occ_small);
+  cudaError_t e = projection_occupancy<L, 512>(smem, &occ_small);
   if (e != cudaSuccess) return e;
-  e = projection_occupancy<L, 768, kIncr>(smem, &occ_large);
+  e = projection_occupancy<L, 768>(smem, &occ_large);
   if (e != cudaSuccess) return e;
   const bool large = occ_large * 768 > occ_small * 512;
   const int threads = large ? 768 : 512, occ = large ? occ_large : occ_small;
@@ -321,12 +337,30 @@ cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m
   const long long need = (rows + threads / 32 - 1) / (threads / 32);
   if (grid > need) grid = need;
   if (large)
-    swd_project_kernel<L, 768, kIncr><<<(unsigned)grid, 768, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d, ps.pm0,
-                                                                        ps.pm1, ps.beta, ps.one_minus_beta);
-  else
-    swd_project_kernel<L, 512, kIncr><<<(unsigned)grid, 512, smem, s>>>(x, m0, m1, active, skip, u, proj, rows, d, ps.pm0,
-                                                                        ps.pm1, ps.beta, ps.one_minus_beta);
-  return cudaGetLastError();
+    return launch_chained(swd_project_kernel<L, 768>, (unsigned)grid, 768, smem, s, x, m0, m1, active, skip, u, proj, rows, d,
+                          ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+  return launch_chained(swd_project_kernel<L, 512>, (unsigned)grid, 512, smem, s, x, m0, m1, active, skip, u, proj, rows, d,
+                        ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+}
+
+// x alone, on the tensor cores: the reference's projections come from the verifier's own buffers
+cudaError_t launch_projection_mma(const uint16_t *x, const int *active, const int *skip, const uint16_t *u, float *proj,
+                                  long long rows, int d, int L, int sms, const ProjectionState &ps, cudaStream_t s) {
+  const size_t smem = (size_t)L * swd_mma_stride(d >> 3) * sizeof(uint4);
+  const long long n_tasks = (rows + 15) / 16;
+  const unsigned grid = (unsigned)(n_tasks < sms ? n_tasks : sms);
+  cudaError_t e;
+  if (L == 16) {
+    e = cudaFuncSetAttribute(swd_project_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
+    if (e != cudaSuccess) return e;
+    return launch_chained(swd_project_mma_kernel<2>, grid, kSwdMmaThreads, smem, s, x, active, skip, u, proj, rows, d, L,
+                          ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+  } else {
+    e = cudaFuncSetAttribute(swd_project_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
+    if (e != cudaSuccess) return e;
+    return launch_chained(swd_project_mma_kernel<1>, grid, kSwdMmaThreads, smem, s, x, active, skip, u, proj, rows, d, L,
+                          ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+  }
 }
 
 // floats of scratch: the projections and two buffers of sorted lists (2L lists of B*T each),
@@ -353,35 +387,32 @@ cudaError_t run_swd(const uint16_t *x, const float *m0, const float *m1, const i
   float *w1_tensor = w1_sample + (size_t)B * L;
   cudaError_t e;
   if (ps.incremental) {
-    if (L == 4) e = launch_projection<4, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    else if (L == 8) e = launch_projection<8, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    else e = launch_projection<16, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    e = launch_projection_mma(x, active, skip, u, proj, rows, d, L, sms, ps, s);
   } else {
-    if (L == 4) e = launch_projection<4, false>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    else if (L == 8) e = launch_projection<8, false>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    else e = launch_projection<16, false>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
   }
   if (e != cudaSuccess) return e;
-  int npad = 1;
+  int npad = 8;
   while (npad < T) npad <<= 1;
   const size_t smem = (size_t)npad * sizeof(float);
   e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSwdMaxTokensPerSample * (int)sizeof(float));
   if (e != cudaSuccess) return e;
-  swd_sort_samples_kernel<<<2 * L * B, kSwdSortThreads, smem, s>>>(proj, buf_a, B, T, L, rows, skip);
-  swd_sample_w1_kernel<<<B * L, 256, 0, s>>>(buf_a, w1_sample, B, T, L, rows, skip);
-  e = cudaGetLastError();
+  e = launch_chained(swd_sort_samples_kernel, 2u * L * B, kSwdSortThreads, smem, s, proj, buf_a, B, T, L, rows, skip);
+  if (e != cudaSuccess) return e;
+  e = launch_chained(swd_sample_w1_kernel, (unsigned)(B * L), 256, 0, s, buf_a, w1_sample, B, T, L, rows, skip);
   float *cur = buf_a, *nxt = buf_b;
   for (int run = 1; run < B && e == cudaSuccess; run *= 2) {     // merge the samples' sorted lists
     const long long total = rows * 2 * L;
-    swd_merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(cur, nxt, rows, T, run, 2 * L, skip);
-    e = cudaGetLastError();
+    e = launch_chained(swd_merge_kernel, (unsigned)((total + 255) / 256), 256, 0, s, cur, nxt, rows, T, run, 2 * L, skip);
     float *t = cur; cur = nxt; nxt = t;
   }
   if (e != cudaSuccess) return e;
-  swd_tensor_w1_kernel<<<L, kSwdSortThreads, 0, s>>>(cur, w1_tensor, rows, L, skip);
-  swd_finish_kernel<<<1, 128, 0, s>>>(w1_tensor, w1_sample, out, B, L, skip);
-  return cudaGetLastError();
+  e = launch_chained(swd_tensor_w1_kernel, (unsigned)L, kSwdSortThreads, 0, s, cur, w1_tensor, rows, L, skip);
+  if (e != cudaSuccess) return e;
+  return launch_chained(swd_finish_kernel, 1, 128, 0, s, w1_tensor, w1_sample, out, B, L, skip);
 }
 
 // A verifier with directions: the distances of this submission against the reference in force,

@@ -12,12 +12,21 @@ namespace sentinel {
 // A projection CTA has 512 or 768 threads; the host takes whichever keeps more threads resident
 // per SM (the directions can fill most of the shared memory: then one large CTA is all there is).
 constexpr int kSwdSortThreads = 1024;
+
+// Every kernel of the chain is launched with programmatic stream serialization and starts with
+// this: the next launch may be set up while this one runs, and nothing is read before the
+// previous launch on the stream has completed and flushed (with a plain launch both do nothing).
+__device__ __forceinline__ void chain_entry() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are sorted in shared memory
 
 // ---------------------------------------------------------------------------------------------
 // projections: proj[(t*L + l)*rows + row] = sum_c v[row][c] * u[l][c], t = 0 for x, 1 for m.
 // A warp owns whole rows; the directions sit in shared memory as bf16 (they are given as bf16).
-// Traffic: x and m are read once, 6 B/element; per element L multiply-adds for each of x and m.
+// Traffic: x and m are read once, 6 B/element; per element L multiply-adds for each of x and m
+// (m is fp32: its half of the work stays on the CUDA cores).
 // The reference is m1 if *active is non-zero, else m0 (a verifier keeps two buffers and flips
 // between them on the device); every kernel of the chain returns at once if *skip is non-zero
 // (a banned worker's tensor is not read).  Both pointers may be nullptr.
@@ -26,16 +35,17 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 //   P(m_t) = beta P(m_{t-1}) + (1-beta) P(x_t)
 // whenever the reference moves.  A verifier therefore keeps P(m) itself ([rows][L] doubles, two
 // buffers pm0 / pm1 selected by the same `active` word as the reference, so a step that does not
-// commit leaves them alone): this kernel always writes the candidate P(m_t) into the spare one,
-// and with kIncr = true it takes P(m_{t-1}) from the current one instead of reading m at all --
-// 2 B/element of traffic instead of 6.  kIncr = false computes it from m (and stores it, if
-// the buffers are given): the stateless call, and the first step after a state import.
-template <int L, int kSwdThreads, bool kIncr>
+// commit leaves them alone).  This kernel computes P(m) from m -- the stateless call, and a
+// verifier's first step or its first step after a state import -- and, if the buffers are given,
+// stores it in the current one and the candidate P(m_t) in the spare one; from then on
+// swd_project_mma_kernel carries the buffers along and reads x only, 2 B/element instead of 6.
+template <int L, int kSwdThreads>
 __global__ void __launch_bounds__(kSwdThreads, kSwdThreads == 512 ? 2 : 1)
 swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                    const uint16_t *u, float *proj, long long rows, int d, double *pm0, double *pm1, float beta,
                    float one_minus_beta) {
   extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
+  chain_entry();
   if (skip && __ldcg(skip)) return;
   const bool second = active && __ldcg(active);
   const float *m = second ? m1 : m0;
@@ -45,27 +55,17 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
     s_u[i] = reinterpret_cast<const uint4 *>(u)[i];
   __syncthreads();
 
-  // A warp owns kRows whole rows at a time; with two rows every direction word fetched from shared
-  // memory serves both (without the reference to read, shared memory is the busier path).
-  constexpr int kRows = (kIncr && L <= 8) ? 2 : 1;     // (16 directions leave no registers for a second row)
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (kSwdThreads / 32) + (threadIdx.x >> 5);
   const long long n_warps = (long long)gridDim.x * (kSwdThreads / 32);
-  for (long long row0 = warp * kRows; row0 < rows; row0 += n_warps * kRows) {
-    float ax[kRows][L], am[L];
+  for (long long row = warp; row < rows; row += n_warps) {
+    float ax[L], am[L];
 #pragma unroll
-    for (int l = 0; l < L; ++l) {
-      am[l] = 0.f;
-#pragma unroll
-      for (int r = 0; r < kRows; ++r) ax[r][l] = 0.f;
-    }
-    bool live[kRows];
-#pragma unroll
-    for (int r = 0; r < kRows; ++r) live[r] = row0 + r < rows;
-    const size_t off = (size_t)row0 * d;
+    for (int l = 0; l < L; ++l) ax[l] = am[l] = 0.f;
+    const size_t off = (size_t)row * d;
     // two chunks per trip, their loads issued before any arithmetic (more bytes in flight)
     for (int c0 = lane; c0 < chunks; c0 += 64) {
-      uint4 xv[kRows][2];
+      uint4 xv[2];
       F8 mv[2];
       bool ok[2];
 #pragma unroll
@@ -73,25 +73,20 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
         const int c = c0 + 32 * h;
         ok[h] = c < chunks;
         if (ok[h]) {
-#pragma unroll
-          for (int r = 0; r < kRows; ++r)
-            if (live[r]) xv[r][h] = ld_x128(x + off + (size_t)r * d + (size_t)c * 8);
-          if (!kIncr) mv[h] = ld_m256(m + off + (size_t)c * 8);
+          xv[h] = ld_x128(x + off + (size_t)c * 8);
+          mv[h] = ld_m256(m + off + (size_t)c * 8);
         }
       }
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (!ok[h]) continue;
         const int c = c0 + 32 * h;
-        float xf[kRows][8];
+        const unsigned xw[4] = {xv[h].x, xv[h].y, xv[h].z, xv[h].w};
+        float xf[8];
 #pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-          const unsigned xw[4] = {xv[r][h].x, xv[r][h].y, xv[r][h].z, xv[r][h].w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            xf[r][2 * j] = live[r] ? __uint_as_float(xw[j] << 16) : 0.f;
-            xf[r][2 * j + 1] = live[r] ? __uint_as_float(xw[j] & 0xFFFF0000u) : 0.f;
-          }
+        for (int j = 0; j < 4; ++j) {
+          xf[2 * j] = __uint_as_float(xw[j] << 16);
+          xf[2 * j + 1] = __uint_as_float(xw[j] & 0xFFFF0000u);
         }
 #pragma unroll
         for (int l = 0; l < L; ++l) {
@@ -100,35 +95,133 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float u_lo = __uint_as_float(uw[j] << 16), u_hi = __uint_as_float(uw[j] & 0xFFFF0000u);
-#pragma unroll
-            for (int r = 0; r < kRows; ++r) {
-              ax[r][l] = fmaf(xf[r][2 * j], u_lo, ax[r][l]);
-              ax[r][l] = fmaf(xf[r][2 * j + 1], u_hi, ax[r][l]);
-            }
-            if (!kIncr) {
-              am[l] = fmaf(mv[h].v[2 * j], u_lo, am[l]);
-              am[l] = fmaf(mv[h].v[2 * j + 1], u_hi, am[l]);
-            }
+            ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
+            ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
+            am[l] = fmaf(mv[h].v[2 * j], u_lo, am[l]);
+            am[l] = fmaf(mv[h].v[2 * j + 1], u_hi, am[l]);
           }
         }
       }
     }
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) {
-      const long long row = row0 + r;
+    for (int l = 0; l < L; ++l) {
+      const float sx = warp_sum(ax[l]), sm = warp_sum(am[l]);
+      if (lane == l) {
+        const size_t at = (size_t)row * L + l;
+        proj[(size_t)l * rows + row] = sx;
+        proj[((size_t)L + l) * rows + row] = sm;
+        if (pm_cur) {
+          pm_cur[at] = (double)sm;
+          pm_next[at] = (double)beta * (double)sm + (double)one_minus_beta * (double)sx;
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The incremental projection (x only) on the tensor cores.  [rows, d] x [d, L] with bf16 operands
+// is a dense contraction, but a skinny one (L <= 16): it is bound by the one read of x, so what
+// matters is that the operands reach the multiplier without a detour.  A warp owns 16 token rows
+// and walks along d; lane (g, q) = (lane / 4, lane % 4) fetches with one 128-bit load the 8
+// consecutive elements [32*cb + 8*q, +8) of row g and of row g + 8.  Those four words are the A
+// fragments of two m16n8k16 multiplies as they stand: a dot product does not care in which order
+// its terms are taken, so the multiply's k-slots (2q, 2q+1 | 2q+8, 2q+9) may stand for columns
+// (8q, 8q+1 | 8q+2, 8q+3) in the first and (8q+4, 8q+5 | 8q+6, 8q+7) in the second, as long as
+// the B fragment -- direction g, same eight columns, one 128-bit load from shared memory --
+// pairs them the same way.  Products of bf16 are exact in fp32; the sums are fp32.
+// The loads of the next 128 columns are issued before the multiplies of the current ones.
+constexpr int kSwdMmaThreads = 512;
+constexpr int kSwdMmaWarps = kSwdMmaThreads / 32;
+
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
+                                                 unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__host__ __device__ inline int swd_mma_stride(int chunks) {     // uint4 per direction in shared memory, = 4 mod 8:
+  return ((chunks + 7) & ~7) + 4;                               // the 8 lanes of a quarter-warp hit 8 different 16-byte banks
+}
+
+template <int NB>            // blocks of 8 directions: 1 for L = 4 or 8, 2 for L = 16
+__global__ void __launch_bounds__(kSwdMmaThreads, 1)
+swd_project_mma_kernel(const uint16_t *x, const int *active, const int *skip, const uint16_t *u, float *proj,
+                       long long rows, int d, int L, double *pm0, double *pm1, float beta, float one_minus_beta) {
+  extern __shared__ uint4 s_u[];                 // [L][stride], 8 bf16 each
+  chain_entry();
+  if (skip && __ldcg(skip)) return;
+  const bool second = active && __ldcg(active);
+  const double *pm_cur = second ? pm1 : pm0;
+  double *pm_next = second ? pm0 : pm1;
+  const int chunks = d >> 3, stride = swd_mma_stride(chunks);
+  for (int i = threadIdx.x; i < L * chunks; i += kSwdMmaThreads) {
+    const int l = i / chunks, c = i - l * chunks;
+    s_u[l * stride + c] = reinterpret_cast<const uint4 *>(u)[i];
+  }
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
+  const long long n_tasks = (rows + 15) >> 4;
+  const int n_groups = (chunks + 15) >> 4;       // 16 chunks = 128 columns = 4 blocks of 32 per trip
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+  // tasks are dealt CTA-first, so that a short list still spreads over all SMs
+  for (long long task = blockIdx.x + (long long)gridDim.x * warp; task < n_tasks;
+       task += (long long)gridDim.x * kSwdMmaWarps) {
+    const long long row_a = task * 16 + g, row_b = row_a + 8;
+    // a row past the end is read as the last row and its result dropped (row i of the product
+    // depends on row i of x alone)
+    const uint16_t *pa = x + (size_t)(row_a < rows ? row_a : rows - 1) * d;
+    const uint16_t *pb = x + (size_t)(row_b < rows ? row_b : rows - 1) * d;
+    float acc[NB][4];
 #pragma unroll
-      for (int l = 0; l < L; ++l) {
-        const float sx = warp_sum(ax[r][l]);
-        const float sm = kIncr ? 0.f : warp_sum(am[l]);
-        if (lane == l && live[r]) {
+    for (int nb = 0; nb < NB; ++nb) acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
+
+    uint4 cur[4][2], nxt[4][2];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = k * 4 + q;
+      cur[k][0] = c < chunks ? ld_x128(pa + (size_t)c * 8) : zero4;
+      cur[k][1] = c < chunks ? ld_x128(pb + (size_t)c * 8) : zero4;
+    }
+    for (int gi = 0; gi < n_groups; ++gi) {
+      if (gi + 1 < n_groups) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int c = (gi + 1) * 16 + k * 4 + q;
+          nxt[k][0] = c < chunks ? ld_x128(pa + (size_t)c * 8) : zero4;
+          nxt[k][1] = c < chunks ? ld_x128(pb + (size_t)c * 8) : zero4;
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = gi * 16 + k * 4 + q;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          const int l = nb * 8 + g;
+          const uint4 uv = (l < L && c < chunks) ? s_u[l * stride + c] : zero4;
+          mma_bf16_16x8x16(acc[nb], cur[k][0].x, cur[k][1].x, cur[k][0].y, cur[k][1].y, uv.x, uv.y);
+          mma_bf16_16x8x16(acc[nb], cur[k][0].z, cur[k][1].z, cur[k][0].w, cur[k][1].w, uv.z, uv.w);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { cur[k][0] = nxt[k][0]; cur[k][1] = nxt[k][1]; }
+    }
+    // accumulator layout: [0], [1] = (row g, directions 2q, 2q+1), [2], [3] = (row g + 8, same)
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const long long row = (e < 2) ? row_a : row_b;
+        const int l = nb * 8 + 2 * q + (e & 1);
+        if (row < rows && l < L) {
           const size_t at = (size_t)row * L + l;
-          const double p_cur = kIncr ? pm_cur[at] : (double)sm;
+          const double p_cur = pm_cur[at];
+          const float sx = acc[nb][e];
           proj[(size_t)l * rows + row] = sx;
           proj[((size_t)L + l) * rows + row] = (float)p_cur;
-          if (pm_cur) {
-            if (!kIncr) pm_cur[at] = p_cur;
-            pm_next[at] = (double)beta * p_cur + (double)one_minus_beta * (double)sx;
-          }
+          pm_next[at] = (double)beta * p_cur + (double)one_minus_beta * (double)sx;
         }
       }
     }
@@ -149,30 +242,91 @@ __device__ __forceinline__ double block_sum_ordered(double v, double *s_red) {
   return total;                                   // valid in thread 0
 }
 
+// One round of the bitonic network on a list in shared memory: every thread takes the 8 entries
+// whose indices differ in the three bits sh+2, sh+1, sh, and runs the first `steps` of the
+// compare-exchange steps on those bits (highest first) in registers -- three steps of the network
+// for one trip through shared memory and one barrier.  k2 is the length of the runs being
+// merged: a pair is put in ascending order iff bit k2 of its index is clear.
+__device__ __forceinline__ void bitonic_round(float *s_val, int npad, int k2, int sh, int steps) {
+  for (int t = threadIdx.x; t < (npad >> 3); t += kSwdSortThreads) {
+    const int low = t & ((1 << sh) - 1), base = ((t >> sh) << (sh + 3)) | low;
+    float v[8];
+    if (sh == 0) {
+      const float4 p0 = reinterpret_cast<const float4 *>(s_val + base)[0];
+      const float4 p1 = reinterpret_cast<const float4 *>(s_val + base)[1];
+      v[0] = p0.x; v[1] = p0.y; v[2] = p0.z; v[3] = p0.w; v[4] = p1.x; v[5] = p1.y; v[6] = p1.z; v[7] = p1.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = s_val[base | (e << sh)];
+    }
+    const bool up = (base & k2) == 0;
+#pragma unroll
+    for (int st = 0; st < 3; ++st) {
+      if (st < steps) {
+        const int bit = 4 >> st;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (!(e & bit)) {
+            const float lo = v[e], hi = v[e | bit];
+            if ((lo > hi) == up) { v[e] = hi; v[e | bit] = lo; }
+          }
+        }
+      }
+    }
+    if (sh == 0) {
+      reinterpret_cast<float4 *>(s_val + base)[0] = make_float4(v[0], v[1], v[2], v[3]);
+      reinterpret_cast<float4 *>(s_val + base)[1] = make_float4(v[4], v[5], v[6], v[7]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s_val[base | (e << sh)] = v[e];
+    }
+  }
+  __syncthreads();
+}
+
 // one CTA per (sample, direction, cloud): bitonic sort of that list of T projections in shared
-// memory; the sorted list goes back to global memory
+// memory (padded with +inf to a power of two, at least 8); the sorted list goes back to global
+// memory
 __global__ void __launch_bounds__(kSwdSortThreads)
 swd_sort_samples_kernel(const float *proj, float *sorted, int B, int T, int L, long long rows, const int *skip) {
   extern __shared__ float s_val[];                // [npad]
+  chain_entry();
   if (skip && __ldcg(skip)) return;
   const int list = blockIdx.x / B, b = blockIdx.x - list * B;     // list = cloud * L + direction
-  int npad = 1;
+  int npad = 8;
   while (npad < T) npad <<= 1;
   const float *src = proj + (size_t)list * rows + (size_t)b * T;
   for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) s_val[i] = i < T ? src[i] : CUDART_INF_F;
   __syncthreads();
-  for (int k2 = 2; k2 <= npad; k2 <<= 1) {        // bitonic sort, ascending
-    for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
-      for (int t = threadIdx.x; t < npad; t += kSwdSortThreads) {
-        const int partner = t ^ j2;
-        if (partner > t) {
-          const bool up = ((t & k2) == 0);
-          const float a0 = s_val[t], a1 = s_val[partner];
-          if ((a0 > a1) == up) { s_val[t] = a1; s_val[partner] = a0; }
+  // runs of 2, 4 and 8: all inside a thread's 8 consecutive entries, the direction per pair
+  for (int t = threadIdx.x; t < (npad >> 3); t += kSwdSortThreads) {
+    float v[8];
+    const float4 p0 = reinterpret_cast<const float4 *>(s_val + t * 8)[0];
+    const float4 p1 = reinterpret_cast<const float4 *>(s_val + t * 8)[1];
+    v[0] = p0.x; v[1] = p0.y; v[2] = p0.z; v[3] = p0.w; v[4] = p1.x; v[5] = p1.y; v[6] = p1.z; v[7] = p1.w;
+#pragma unroll
+    for (int k2 = 2; k2 <= 8; k2 <<= 1) {
+#pragma unroll
+      for (int bit = k2 >> 1; bit > 0; bit >>= 1) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (!(e & bit)) {
+            const bool up = (((t * 8 + e) & k2) == 0);
+            const float lo = v[e], hi = v[e | bit];
+            if ((lo > hi) == up) { v[e] = hi; v[e | bit] = lo; }
+          }
         }
       }
-      __syncthreads();
     }
+    reinterpret_cast<float4 *>(s_val + t * 8)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4 *>(s_val + t * 8)[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+  __syncthreads();
+  for (int k2 = 16, k = 4; k2 <= npad; k2 <<= 1, ++k) {   // merge runs of k2/2 into runs of k2: steps on bits k-1 .. 0
+    int j = k - 1;
+    const int head = (j + 1) % 3;                 // a short round first, so that the rest are full ones ending at bit 0
+    if (head) { bitonic_round(s_val, npad, k2, j - 2, head); j -= head; }
+    for (; j >= 2; j -= 3) bitonic_round(s_val, npad, k2, j - 2, 3);
   }
   float *dst = sorted + (size_t)list * rows + (size_t)b * T;
   for (int i = threadIdx.x; i < T; i += kSwdSortThreads) dst[i] = s_val[i];
@@ -182,6 +336,7 @@ swd_sort_samples_kernel(const float *proj, float *sorted, int B, int T, int L, l
 __global__ void __launch_bounds__(256)
 swd_sample_w1_kernel(const float *sorted, float *w1_sample, int B, int T, int L, long long rows, const int *skip) {
   __shared__ double s_red[256 / 32];
+  chain_entry();
   if (skip && __ldcg(skip)) return;
   const int b = blockIdx.x / L, l = blockIdx.x - b * L;
   const float *sa = sorted + (size_t)l * rows + (size_t)b * T;
@@ -198,6 +353,7 @@ swd_sample_w1_kernel(const float *sorted, float *w1_sample, int B, int T, int L,
 // run plus its rank in the partner run (left run first on ties)
 __global__ void swd_merge_kernel(const float *in, float *out, long long rows, int T, int run, int lists,
                                  const int *skip) {
+  chain_entry();
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= rows * lists || (skip && __ldcg(skip))) return;
   const long long list = e / rows, i = e - list * rows;
@@ -226,6 +382,7 @@ __global__ void swd_merge_kernel(const float *in, float *out, long long rows, in
 __global__ void __launch_bounds__(kSwdSortThreads)
 swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int L, const int *skip) {
   __shared__ double s_red[kSwdSortThreads / 32];
+  chain_entry();
   if (skip && __ldcg(skip)) return;
   const int l = blockIdx.x;
   const float *a = merged + (size_t)l * rows, *b = merged + ((size_t)L + l) * rows;
@@ -238,6 +395,7 @@ swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int 
 // the means over the directions for every unit: out[0] = tensor, out[1+b] = sample b
 __global__ void swd_finish_kernel(const float *w1_tensor, const float *w1_sample, float *out, int B, int L,
                                   const int *skip) {
+  chain_entry();
   if (skip && __ldcg(skip)) return;
   for (int r = threadIdx.x; r <= B; r += blockDim.x) {
     const float *w = r ? w1_sample + (size_t)(r - 1) * L : w1_tensor;
