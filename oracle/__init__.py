@@ -57,7 +57,7 @@ class _Params(C.Structure):
         ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
         ("l", C.c_int), ("c", C.c_int), ("t_forgiveness", C.c_int),
         ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
-        ("R", C.c_int), ("ema_bf16", C.c_int), ("ref_over_batch", C.c_int),
+        ("R", C.c_int), ("ema_bf16", C.c_int), ("ref_over_batch", C.c_int), ("ref_over_tokens", C.c_int),
     ]
 
 
@@ -170,6 +170,7 @@ class Params:
     R: int = 1
     ema_bf16: int = 0
     ref_over_batch: int = 0
+    ref_over_tokens: int = 0
 
     def to_c(self) -> _Params:
         p = _Params()
@@ -184,6 +185,7 @@ class Params:
         p.R = self.R
         p.ema_bf16 = self.ema_bf16
         p.ref_over_batch = self.ref_over_batch
+        p.ref_over_tokens = self.ref_over_tokens
         return p
 
 
@@ -331,13 +333,16 @@ class Verifier:
 
     def ema(self, kind: int) -> np.ndarray:
         p = lib().so_ema(self._h, kind)
+        if self.params.ref_over_tokens:           # one [d] reference for all tokens
+            return np.ctypeslib.as_array(p, shape=(self.d,)).copy()
         if self.params.ref_over_batch:            # one [T,d] reference for all samples
             return np.ctypeslib.as_array(p, shape=(self.T * self.d,)).copy().reshape(self.T, self.d)
         return np.ctypeslib.as_array(p, shape=(self.N,)).copy().reshape(self.B, self.T, self.d)
 
     def set_ema(self, kind: int, m):
         mm = np.ascontiguousarray(m, dtype=np.float64).reshape(-1)
-        assert mm.size == (self.T * self.d if self.params.ref_over_batch else self.N)
+        assert mm.size == (self.d if self.params.ref_over_tokens else
+                           self.T * self.d if self.params.ref_over_batch else self.N)
         lib().so_set_ema(self._h, kind, _dptr(mm))
 
     def history(self, kind: int, level: int, metric: int) -> np.ndarray:

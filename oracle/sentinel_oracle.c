@@ -64,6 +64,7 @@ void so_default_params(so_params *p) {
   p->R = 1;
   p->ema_bf16 = 0;
   p->ref_over_batch = 0;
+  p->ref_over_tokens = 0;
 }
 
 /* ------------------------------------------------------------------------------------ */
@@ -281,11 +282,12 @@ so_verifier *so_create(const so_params *p) {
   if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1 || p->R < 1 || p->R > SO_MAX_WORKERS) return NULL;
   if (p->ema_bf16 && p->R != 1) return NULL;   /* the bf16 reference exists for one submission per update */
   if (p->ref_over_batch && (p->R != 1 || p->ema_bf16)) return NULL;   /* likewise the [T,d] reference */
+  if (p->ref_over_tokens && !p->ref_over_batch) return NULL;          /* [d] = over samples and tokens */
   so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
   v->p = *p;
   v->Ns = (size_t)p->T * (size_t)p->d;
   v->N = v->Ns * (size_t)p->B;
-  v->Nm = p->ref_over_batch ? v->Ns : v->N;   /* elements of the reference */
+  v->Nm = p->ref_over_tokens ? (size_t)p->d : p->ref_over_batch ? v->Ns : v->N;   /* elements of the reference */
   v->u = NULL; v->n_dir = 0; v->nm = 3;
   for (int kind = 0; kind < 2; ++kind) {
     so_kind_state *ks = &v->ks[kind];
@@ -333,11 +335,12 @@ void so_destroy(so_verifier *v) {
 static void all_units(so_verifier *v, const uint16_t *x, int kind, double *gam, int *nonfinite) {
   so_kind_state *ks = &v->ks[kind];
   const size_t d = (size_t)v->p.d;
-  /* a [T,d] reference stands for the same tensor in every sample: write the broadcast out */
+  /* a [T,d] reference stands for the same tensor in every sample, a [d] reference for the same
+   * vector in every token: write the broadcast out */
   double *wide = NULL;
-  if (v->p.ref_over_batch) {
+  if (v->Nm != v->N) {
     wide = (double *)malloc(v->N * sizeof(double));
-    for (int b = 0; b < v->p.B; ++b) memcpy(wide + (size_t)b * v->Ns, ks->m, v->Ns * sizeof(double));
+    for (size_t k = 0; k < v->N / v->Nm; ++k) memcpy(wide + k * v->Nm, ks->m, v->Nm * sizeof(double));
   }
   const double *m = wide ? wide : ks->m;
   for (int r = 0; r <= v->p.B; ++r) {
@@ -378,11 +381,12 @@ static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
       m[e] = so_bf16(so_bf16_round((double)fmaf(bf, (float)m[e], of * (float)so_bf16(x[e]))));
     return;
   }
-  if (v->p.ref_over_batch) {   /* Eq. 1 with the mean over the B samples as the submission */
-    for (size_t e = 0; e < v->Ns; ++e) {
+  if (v->Nm != v->N) {   /* Eq. 1 with the mean over the B samples (the B*T tokens) as the submission */
+    const size_t copies = v->N / v->Nm;
+    for (size_t e = 0; e < v->Nm; ++e) {
       double sum = 0.0;
-      for (int b = 0; b < v->p.B; ++b) sum += so_bf16(x[(size_t)b * v->Ns + e]);
-      m[e] = beta * m[e] + (1.0 - beta) * (sum / (double)v->p.B);
+      for (size_t k = 0; k < copies; ++k) sum += so_bf16(x[k * v->Nm + e]);
+      m[e] = beta * m[e] + (1.0 - beta) * (sum / (double)copies);
     }
     return;
   }

@@ -60,7 +60,8 @@ def oracle_to_blob(v, params) -> bytes:
     """Serialise an oracle verifier into the library's checkpoint format."""
     B, T, d, l, R = params.B, params.T, params.d, params.l, params.R
     M = v.nm                                   # metrics in use; the layout has room for four
-    shared = int(getattr(params, "ref_over_batch", 0))
+    # 0: [B,T,d] reference, 1: one [T,d] reference for all samples, 2: one [d] reference for all tokens
+    shared = 2 if getattr(params, "ref_over_tokens", 0) else int(getattr(params, "ref_over_batch", 0))
     out = bytearray(struct.pack("<QI7i", MAGIC, 3, B, T, d, l, R, M, shared))
     out += b"\0" * (64 - len(out))
     workers = np.zeros((3, 16), dtype="<i4")
@@ -96,7 +97,7 @@ def parse_blob(blob, B, T, d, l, R=1) -> dict:
     off = 64 + 192
     out = {"violations": int(workers[0, 0]), "clean_streak": int(workers[1, 0]), "banned": int(workers[2, 0]),
            "workers": workers.copy(), "n_metrics": M, "ref_over_batch": shared, "kinds": []}
-    N = T * d if shared else B * T * d
+    N = d if shared == 2 else T * d if shared else B * T * d
     for _ in range(2):
         steps, c0, c1 = struct.unpack_from("<q2i", buf, off)
         valid = np.array(struct.unpack_from("<8i", buf, off + 16)).reshape(2, 4).astype(bool)[:, :M]

@@ -697,3 +697,68 @@ def test_shared_reference_flags_commit_and_replacement(oracle_mod, small):
         oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_batch=1, R=2))
     with pytest.raises(ValueError):
         oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_batch=1, ema_bf16=1))
+
+
+# ---------------------------------------------------------------------------------------------
+# one [d] reference shared by all B*T tokens
+
+def test_channel_reference_is_the_full_reference_of_the_token_mean(oracle_mod):
+    """Eq. 1 with the mean over all B*T token rows as the submission: closed form from m_0 = 0,
+    and rows that all equal one vector r give m_t = (1 - beta^t) r."""
+    rs = np.random.default_rng(51)
+    B, T, d = 3, 5, 8
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_batch=1, ref_over_tokens=1)
+    want = np.zeros(d)
+    for t in range(6):
+        xb = to_bits(rs.normal(0.5, 1, (B, T, d)))
+        v.update_reference(xb, ACT)
+        want = 0.9 * want + 0.1 * from_bits(xb).reshape(B * T, d).mean(axis=0)
+        assert v.ema(ACT).shape == (d,)
+        assert v.ema(ACT) == pytest.approx(want, rel=1e-13, abs=1e-16)
+    r = from_bits(to_bits(rs.normal(0, 1, d)))
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_batch=1, ref_over_tokens=1)
+    for t in range(1, 5):
+        v.update_reference(to_bits(np.tile(r, (B, T, 1))), GRAD)
+        assert v.ema(GRAD) == pytest.approx((1 - 0.8 ** t) * r, rel=1e-13, abs=1e-16)
+
+
+def test_channel_reference_scores_are_those_against_the_tiled_reference(oracle_mod):
+    """Every token is compared with the same vector: sample b against T copies of m, the whole
+    tensor against B*T copies -- the stateless distances say the same."""
+    rs = np.random.default_rng(52)
+    B, T, d = 3, 4, 8
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_batch=1, ref_over_tokens=1)
+    for t in range(5):
+        v.update_reference(to_bits(rs.normal(0, 1, (B, T, d)) + np.arange(d)), GRAD)
+    m = v.ema(GRAD)
+    xb = to_bits(rs.normal(0, 1, (B, T, d)) + np.arange(d))
+    scores, flags, _ = v.verify(xb, GRAD)
+    g0, s0, _ = oracle_mod.distance(xb, np.tile(m, (B, T, 1)))
+    assert np.array_equal(scores[0], g0) and np.array_equal(v.last_stats(GRAD)[0], s0)
+    for b in range(B):
+        gb, _, _ = oracle_mod.distance(xb[b], np.tile(m, (T, 1)))
+        assert np.array_equal(scores[1 + b], gb)
+    # a unit's statistics of the reference are those of the vector itself
+    st = v.last_stats(GRAD)
+    assert st[:, 3] == pytest.approx(m.mean(), rel=1e-12) and st[:, 4] == pytest.approx(m.var(), rel=1e-12)
+
+
+def test_channel_reference_flags_commit_and_replacement(oracle_mod, small):
+    v = oracle_mod.Verifier(oracle_mod.Params(B=small.B, T=small.T, d=small.d, ref_over_batch=1, ref_over_tokens=1))
+    for t in range(14):
+        v.update_reference(synth.bits(synth.clean(small, 0, ACT, t)), ACT)
+    h = synth.clean(small, 0, ACT, 14)
+    _, flags, commit = v.verify(synth.bits(h), ACT)
+    assert commit and not (flags & 0xFFFF).any()
+    m0 = v.ema(ACT)
+    loud = (h.float() * 50).to(torch.bfloat16)
+    _, flags, commit = v.verify(synth.bits(loud), ACT)
+    assert not commit and (flags[0] & 0xFFFF) and np.array_equal(v.ema(ACT), m0)
+    out, did = v.replace_if_flagged(synth.bits(loud), ACT)
+    assert did
+    got = from_bits(out)
+    assert np.all(np.abs(got - m0) <= 2.0 ** -8 * np.abs(m0) + 1e-45)      # every token receives the one vector
+    with pytest.raises(ValueError):
+        oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_tokens=1))           # [d] means over samples too
+    with pytest.raises(ValueError):
+        oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_batch=1, ref_over_tokens=1, R=2))
