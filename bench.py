@@ -348,6 +348,27 @@ def run_ours(args, rank, world, local_rank):
                   "tensors_per_s": round(1e3 / zms, 1), "kernel": "shared_ref_kernel"}
         vsr.sentinel_destroy()
 
+    # extra figure, outside the timed region: one [d] reference for all tokens (x alone streams, 2 B/element)
+    channel = None
+    if extras:
+        vcr = binding.Verifier(w.B, w.T, w.d, device=local_rank, ref_over_batch=1, ref_over_tokens=1)
+        cs_, cf_ = torch.empty(1 + w.B, 3, dtype=torch.float32, device=device), torch.zeros(1 + w.B, dtype=torch.int32, device=device)
+        for i in range(6):
+            vcr.sentinel_update_reference(xs[0][ACT][i % nd], ACT, cs_, main)
+        vcr.sentinel_verify(xs[0][ACT][6 % nd], ACT, cs_, cf_, main)
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        q0.record(main)
+        for i in range(20):
+            vcr.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, cs_, cf_, main)
+        q1.record(main)
+        torch.cuda.synchronize()
+        qms = q0.elapsed_time(q1) / 20
+        channel = {"bytes_per_element": 2, "ms_per_step": round(qms, 4),
+                   "achieved_gbs": round(2 * N / (qms * 1e-3) / 1e9, 1),
+                   "tensors_per_s": round(1e3 / qms, 1), "kernels": "channel_ref_kernel + channel_mean_kernel"}
+        vcr.sentinel_destroy()
+
     # extra figure, outside the timed region: the strided (compressed-signal) layout, rows d+1 apart
     strided = None
     if extras:
@@ -449,6 +470,8 @@ def run_ours(args, rank, world, local_rank):
         out["bf16_reference"] = half
     if shared is not None:
         out["shared_reference"] = shared
+    if channel is not None:
+        out["channel_reference"] = channel
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
     return out

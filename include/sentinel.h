@@ -105,6 +105,8 @@ typedef struct sentinel_config {
   int    n_workers;        /* workers d_s feeding this boundary (multi-worker calls)   1    */
   int    ema_bf16;         /* 1: the reference is stored as bf16 (see below)           0    */
   int    ref_over_batch;   /* 1: one [T,d] reference for all B samples (see below)     0    */
+  int    ref_over_tokens;  /* 1 (with ref_over_batch = 1): one [d] reference for all
+                              B*T tokens (see below)                                   0    */
 } sentinel_config;
 
 typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundary */
@@ -128,6 +130,17 @@ typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundar
  * B <= 16, d a multiple of 8; no strided tensors, no sentinel_set_directions, no per-token buffer.
  * Gradient replacement writes the one reference into every sample.  State blobs carry T*d
  * reference values per kind and record the shape in the header. */
+/* ref_over_batch = 1 together with ref_over_tokens = 1 reduces the reference over the tokens as
+ * well: ONE vector of d channels for all B*T token rows of a tensor (the same reading taken one
+ * step further: every token is a draw of one d-dimensional signal).  Every token row is compared
+ * with it -- sample b against T copies, the whole tensor against B*T copies -- and Eq. 1 moves it
+ * with the mean over the token rows, m_t = beta m_{t-1} + (1-beta)/(B*T) sum_{b,t} x[b,t,:].  Only
+ * x is read, 2 bytes per element, and the state of a kind is two vectors.  A step is two launches
+ * (the streaming pass, then a small one that writes the candidate from the column sums and, if
+ * the step committed, makes it the reference); both are enqueued by the same call.  Restrictions:
+ * n_workers = 1, fp32 reference, d a multiple of 8; no strided tensors, no
+ * sentinel_set_directions, no per-token buffer.  Gradient replacement writes the vector into
+ * every token.  State blobs carry d reference values per kind; the header's shape field is 2. */
 int sentinel_default_config(sentinel_config *cfg);
 
 /* Allocates the state of one boundary on cfg->device: two fp32 [B,T,d] buffers per kind (the
@@ -337,7 +350,7 @@ int sentinel_reset_worker(sentinel_verifier *h, int worker, void *cuda_stream);
  * i32 violations[16], clean_streak[16], banned[16], then per kind {i64 steps; i32 count[2];
  * i32 valid[2][4]; f64 thr[2][4][6]; f64 history[level 0: 4][window_steps*n_workers],
  * [level 1: 4][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d] (m[T*d] with
- * ref_over_batch)}.  The
+ * ref_over_batch, header field 1; m[d] with ref_over_tokens as well, header field 2)}.  The
  * layout always has room for four metrics; with n_metrics = 3 the fourth slots are unused.
  * A blob goes back only into a verifier with the same n_metrics (the directions themselves
  * are not part of the state: set them before importing).  Export and import wait for the

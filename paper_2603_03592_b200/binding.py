@@ -50,7 +50,7 @@ class sentinel_config(C.Structure):
         ("shrink_ratio", C.c_double), ("severe_mult", C.c_double),
         ("window_steps", C.c_int), ("ban_violations", C.c_int), ("forgiveness_steps", C.c_int),
         ("metric_mask", C.c_uint), ("B", C.c_int), ("T", C.c_int), ("d", C.c_int),
-        ("device", C.c_int), ("n_workers", C.c_int), ("ema_bf16", C.c_int), ("ref_over_batch", C.c_int),
+        ("device", C.c_int), ("n_workers", C.c_int), ("ema_bf16", C.c_int), ("ref_over_batch", C.c_int), ("ref_over_tokens", C.c_int),
     ]
 
 

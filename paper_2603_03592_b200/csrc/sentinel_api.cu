@@ -62,7 +62,9 @@ struct sentinel_verifier {
   void *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // fp32, or bf16 if bf16
   bool bf16 = false;                // the reference is stored as bf16
   bool shared_ref = false;          // one [T,d] reference for all B samples
-  size_t ema_elems = 0;             // elements of one reference buffer: B*T*d, or T*d if shared_ref
+  bool chan_ref = false;            // one [d] reference for all B*T tokens
+  float *col_part = nullptr;        // chan_ref: column sums of x per streaming CTA and slot
+  size_t ema_elems = 0;             // elements of one reference buffer: B*T*d, T*d if shared_ref, d if chan_ref
   size_t ema_bytes = 0;             // bytes of one reference buffer
   HandleState *hs = nullptr;
   double *hist[2] = {nullptr, nullptr};      // rings, device layout (ring_offset)
@@ -194,7 +196,7 @@ int check_call_strided(sentinel_verifier *h, const void *x, int kind, int B, int
   if (row_stride < d) return fail(h, SENTINEL_ERR_INVALID_ARG, "row_stride = %lld is smaller than d = %d", row_stride, d);
   if (reinterpret_cast<uintptr_t>(x) & 1u) return fail(h, SENTINEL_ERR_UNALIGNED, "x is not 2-byte aligned");
   if (h->sw_u) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein metric reads dense rows: a verifier with directions takes no strided tensor");
-  if (h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "a verifier with a [T,d] reference takes no strided tensor");
+  if (h->shared_ref || h->chan_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "a verifier with a [T,d] or [d] reference takes no strided tensor");
   return SENTINEL_OK;
 }
 
@@ -232,6 +234,8 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.ema_bf16 = h->bf16 ? 1 : 0;
   a.n_metrics = h->n_metrics;
   a.sw = h->sw_out;                 // nullptr until directions are set
+  a.defer_commit = h->chan_ref ? 1 : 0;
+  a.col_part = h->col_part;
   return a;
 }
 
@@ -248,6 +252,19 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
   attr.val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = &attr;
   lc.numAttrs = 1;
+  if (h->chan_ref) {                               // x alone streams; the reference moves in a second launch
+    const size_t col_smem = (size_t)kWarps * kStripe * sizeof(float);      // the warps' column sums
+    if (lc.dynamicSmemBytes < col_smem) lc.dynamicSmemBytes = col_smem;
+    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel, a));
+    cudaLaunchConfig_t lm = lc;
+    lm.gridDim = dim3((unsigned)((h->cfg.d + kChannelMeanCols - 1) / kChannelMeanCols));
+    lm.blockDim = dim3(kChannelMeanCols * kChannelMeanGroups);
+    lm.dynamicSmemBytes = 0;
+    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lm, channel_mean_kernel, h->hs, a.kind, static_cast<float *>(a.ema[0]),
+                                        static_cast<float *>(a.ema[1]), static_cast<const float *>(h->col_part), a.x,
+                                        h->G, h->cfg.B, h->cfg.T, h->cfg.d, a.beta, a.one_minus_beta));
+    return SENTINEL_OK;
+  }
   if (h->shared_ref) {                             // the samples in the workers' place (vector rows only)
     ReplicaArgs ra;
     memset(&ra, 0, sizeof ra);
@@ -448,6 +465,7 @@ void free_all(sentinel_verifier *h) {
   cudaFree(h->hs);
   cudaFree(h->partials);
   cudaFree(h->token_part);
+  cudaFree(h->col_part);
   cudaFree(h->stage_x);
   cudaFree(h->stage_scores);
   cudaFree(h->stage_flags);
@@ -502,8 +520,11 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   if (cfg->ema_bf16 && cfg->n_workers != 1)
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "the bf16 reference is kept for single submissions only (n_workers = 1)");
   if (cfg->ref_over_batch != 0 && cfg->ref_over_batch != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ref_over_batch must be 0 or 1, got %d", cfg->ref_over_batch);
-  if (cfg->ref_over_batch && (cfg->n_workers != 1 || cfg->ema_bf16 || cfg->B > kMaxWorkers || cfg->d % 8 != 0))
+  if (cfg->ref_over_batch && (cfg->n_workers != 1 || cfg->ema_bf16 || (cfg->B > kMaxWorkers && !cfg->ref_over_tokens) || cfg->d % 8 != 0))
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a [T,d] reference needs n_workers = 1, an fp32 reference, B <= %d and d a multiple of 8", kMaxWorkers);
+  if (cfg->ref_over_tokens != 0 && cfg->ref_over_tokens != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ref_over_tokens must be 0 or 1, got %d", cfg->ref_over_tokens);
+  if (cfg->ref_over_tokens && !cfg->ref_over_batch)
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a [d] reference is one for all samples and tokens: set ref_over_batch = 1 as well");
   if ((long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*n_workers*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d",
                 (long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1), SENTINEL_MAX_WINDOW);
@@ -521,8 +542,9 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->N = h->Ns * cfg->B;
   h->R = cfg->n_workers;
   h->bf16 = cfg->ema_bf16 != 0;
-  h->shared_ref = cfg->ref_over_batch != 0;
-  h->ema_elems = h->shared_ref ? h->Ns : h->N;
+  h->chan_ref = cfg->ref_over_tokens != 0;
+  h->shared_ref = cfg->ref_over_batch != 0 && !h->chan_ref;
+  h->ema_elems = h->chan_ref ? (size_t)cfg->d : h->shared_ref ? h->Ns : h->N;
   h->ema_bytes = h->ema_elems * (h->bf16 ? sizeof(uint16_t) : sizeof(float));
   h->units0 = h->R;                       // the window spans window_steps iterations of all workers
   h->units1 = h->R * cfg->B;
@@ -543,6 +565,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
   }
   std::string oerr;
@@ -562,6 +585,7 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     alloc((void **)&h->stats[k], (size_t)(1 + cfg->B) * kNumStats * sizeof(float));
   }
   alloc((void **)&h->partials, (size_t)(h->shared_ref ? cfg->B : h->R) * h->G * kSegsPerCta * kSlotWords * sizeof(unsigned long long));   // per worker / per sample
+  if (h->chan_ref) alloc((void **)&h->col_part, (size_t)h->G * kSegsPerCta * channel_slots(cfg->d) * kStripe * sizeof(float));
   alloc((void **)&h->hs, sizeof(HandleState));
   if (e == cudaSuccess) {
     HandleState init;
@@ -822,7 +846,7 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
   if (grid > need) grid = need;
   replace_kernel<<<(unsigned)grid, kReplaceThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], h->bf16 ? 1 : 0, static_cast<uint16_t *>(dev_x_inout), n_chunks,
-      h->shared_ref ? (long long)(h->ema_elems / 8) : 0ll, fill,
+      (h->shared_ref || h->chan_ref) ? (long long)(h->ema_elems / 8) : 0ll, fill,
       dev_replaced_out);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
@@ -833,7 +857,7 @@ int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L,
   if (!dev_u_bf16) return fail(h, SENTINEL_ERR_INVALID_ARG, "u is NULL");
   if (h->started) return fail(h, SENTINEL_ERR_INVALID_ARG, "the metric set is fixed once a step was taken or a state imported");
   if (h->bf16) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads an fp32 reference: not available with ema_bf16");
-  if (h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads a [B,T,d] reference: not available with ref_over_batch");
+  if (h->shared_ref || h->chan_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads a [B,T,d] reference: not available with ref_over_batch");
   if (h->cfg.d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", h->cfg.d);
   int rc = check_swd_shape(h, L, h->cfg.T, h->cfg.d);
   if (rc) return rc;
@@ -964,7 +988,7 @@ int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_
 int sentinel_set_token_stats_buffer(sentinel_verifier *h, float *dev_buf) {
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (dev_buf && !aligned16(dev_buf)) return fail(h, SENTINEL_ERR_UNALIGNED, "token buffer is not 16-byte aligned");
-  if (dev_buf && h->shared_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "per-token sums are not written with a [T,d] reference");
+  if (dev_buf && (h->shared_ref || h->chan_ref)) return fail(h, SENTINEL_ERR_UNSUPPORTED, "per-token sums are not written with a [T,d] or [d] reference");
   const int tpr = tiles_per_row(h->cfg.d);
   if (dev_buf && tpr > 1 && !h->token_part) {      // rows of several tiles need a place for the shares
     DeviceGuard guard(h->cfg.device);
@@ -1021,7 +1045,7 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
 
   unsigned char *out = static_cast<unsigned char *>(host_buf);
   memset(out, 0, kHeaderBytes);
-  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics, h->shared_ref ? 1 : 0};
+  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics, h->chan_ref ? 2 : h->shared_ref ? 1 : 0};
   memcpy(out, &hd, sizeof hd);
   out += kHeaderBytes;
   BlobWorkers bw;
@@ -1082,8 +1106,8 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
     return fail(h, SENTINEL_ERR_STATE_SIZE, "not a sentinel state blob of version %u", kVersion);
   if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps || hd.n_workers != h->R)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d, %d workers", hd.B, hd.T, hd.d, hd.window_steps, hd.n_workers);
-  if ((hd.ref_over_batch != 0) != h->shared_ref)
-    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob and verifier differ in the shape of the reference ([T,d] against [B,T,d])");
+  if (hd.ref_over_batch != (h->chan_ref ? 2 : h->shared_ref ? 1 : 0))
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob and verifier differ in the shape of the reference ([B,T,d], [T,d] or [d])");
   if (hd.n_metrics != h->n_metrics)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob holds %d metrics, this verifier uses %d (set the directions before importing)", hd.n_metrics, h->n_metrics);
   // validate both kinds before touching the device

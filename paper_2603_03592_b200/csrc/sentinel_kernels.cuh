@@ -68,7 +68,7 @@ struct KindState {
   unsigned step_tainted;    //   workers that raised a flag,
   unsigned step_nonfinite;  //   workers whose tensor held a NaN or an infinity,
   unsigned step_elsewhere;  //   workers tainted at another stage (not collected)
-  int pad;
+  int commit_pending;     // [d] reference: the step committed; channel_mean_kernel writes the candidate and flips `active`
   long long mean_done_step; // the iteration whose mean over the workers is already in place
   int has_thr[2][kNumMetrics];
   double thr[2][kNumMetrics][kNumThr];   // q1 q2 q3 k tau_lower tau_upper
@@ -77,7 +77,8 @@ struct KindState {
 struct HandleState {
   int error;
   unsigned ticket;
-  int pad[2];
+  unsigned ticket2;       // the ticket of channel_mean_kernel
+  int pad;
   int violations[kMaxWorkers], clean_streak[kMaxWorkers], banned[kMaxWorkers];   // per worker
   KindState kind[2];
 };
@@ -113,7 +114,8 @@ struct StreamArgs {
   double severe_mult;
   int ban_violations, forgiveness_steps;
   unsigned metric_mask;
-  int pad;
+  int defer_commit;                // [d] reference: the commit is carried out by channel_mean_kernel
+  float *col_part;                 // [d] reference: column sums of x, [G][2][channel_slots(d)][512]
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -256,6 +258,45 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
   return v;
 }
 
+// A segment's sums, thread -> warp -> CTA in a fixed order (two runs give bit-identical sums),
+// written to the segment's slot with the sample's tag and the shift the sums were taken about.
+__device__ __forceinline__ void reduce_to_slot(const ThreadAcc &t, int b, unsigned x0, unsigned m0bits,
+                                               unsigned long long (*s_part)[kSlotWords], unsigned long long *slot) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const double ws[6] = {warp_sum(t.sx), warp_sum(t.sxx), warp_sum(t.sm),
+                        warp_sum(t.smm), warp_sum(t.sxm), warp_sum(t.ab)};
+  const unsigned long long wf = warp_sum((unsigned long long)t.flips);
+  unsigned long long bits = (t.nf_bits ? kBitNonfinite : 0ull) | (t.x_diff ? kBitXVaries : 0ull) |
+                            (t.m_diff ? kBitMVaries : 0ull);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+  __syncthreads();                      // s_part may still be read from the previous segment
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < 6; ++j) s_part[warp][j] = (unsigned long long)__double_as_longlong(ws[j]);
+    s_part[warp][6] = wf;
+    s_part[warp][7] = bits;
+  }
+  __syncthreads();
+  if (threadIdx.x < kSlotWords) {
+    const int j = threadIdx.x;
+    unsigned long long out;
+    if (j < 6) {
+      double sum = 0.;
+      for (int w = 0; w < kWarps; ++w) sum += __longlong_as_double((long long)s_part[w][j]);
+      out = (unsigned long long)__double_as_longlong(sum);
+    } else if (j == 6) {
+      out = 0ull;
+      for (int w = 0; w < kWarps; ++w) out += s_part[w][6];
+    } else {
+      out = ((unsigned long long)(b + 1) << kTagShift) | ((unsigned long long)x0 << kX0Shift) |
+            ((unsigned long long)m0bits << kM0Shift);       // sample tag and the shift of the sums
+      for (int w = 0; w < kWarps; ++w) out |= s_part[w][7];
+    }
+    slot[j] = out;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // streaming phase
 //
@@ -389,39 +430,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
     }
   }
 
-  // warp -> CTA, in a fixed order so that two runs give bit-identical sums
-  const double ws[6] = {warp_sum(t.sx), warp_sum(t.sxx), warp_sum(t.sm),
-                        warp_sum(t.smm), warp_sum(t.sxm), warp_sum(t.ab)};
-  const unsigned long long wf = warp_sum((unsigned long long)t.flips);
-  unsigned long long bits = (t.nf_bits ? kBitNonfinite : 0ull) | (t.x_diff ? kBitXVaries : 0ull) |
-                            (t.m_diff ? kBitMVaries : 0ull);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
-  __syncthreads();                      // s_part may still be read from the previous segment
-  if (lane == 0) {
-#pragma unroll
-    for (int j = 0; j < 6; ++j) s_part[warp][j] = (unsigned long long)__double_as_longlong(ws[j]);
-    s_part[warp][6] = wf;
-    s_part[warp][7] = bits;
-  }
-  __syncthreads();
-  if (threadIdx.x < kSlotWords) {
-    const int j = threadIdx.x;
-    unsigned long long out;
-    if (j < 6) {
-      double sum = 0.;
-      for (int w = 0; w < kWarps; ++w) sum += __longlong_as_double((long long)s_part[w][j]);
-      out = (unsigned long long)__double_as_longlong(sum);
-    } else if (j == 6) {
-      out = 0ull;
-      for (int w = 0; w < kWarps; ++w) out += s_part[w][6];
-    } else {
-      out = ((unsigned long long)(b + 1) << kTagShift) | ((unsigned long long)x0 << kX0Shift) |
-            ((unsigned long long)m0bits << kM0Shift);       // sample tag and the shift of the sums
-      for (int w = 0; w < kWarps; ++w) out |= s_part[w][7];
-    }
-    slot[j] = out;
-  }
+  reduce_to_slot(t, b, x0, m0bits, s_part, slot);
 }
 
 template <bool kScalar, bool kBf16>
@@ -921,7 +930,10 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
       ks->refresh_pending = 1;
       if (!replica) {
         ks->last_flagged = any_flag ? 1 : 0;
-        if (!any_flag) { ks->active ^= 1; status |= kFlagCommitted; }   // m_t := candidate
+        if (!any_flag) {                         // m_t := candidate
+          if (a.defer_commit) ks->commit_pending = 1; else ks->active ^= 1;
+          status |= kFlagCommitted;
+        }
       }
       if (s_severe) status |= kFlagSevere;
       if (hs->banned[w]) status |= kFlagBanned;
@@ -930,7 +942,7 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
       joined[0] = 1;
       joined[1] = B;
       ks->refresh_pending = 1;
-      if (!replica) ks->active ^= 1;
+      if (!replica) { if (a.defer_commit) ks->commit_pending = 1; else ks->active ^= 1; }
     }
     if (replica) {                               // what the mean over the clean workers needs
       ks->step_collected |= 1u << w;
@@ -1015,6 +1027,288 @@ stream_kernel_t(const StreamArgs a) {
   __threadfence();
   const FinalizeTarget ft = {0, a.partials, a.scores_out, a.flags_out, a.sw, 0, 1, 0};
   finalize(a, ft);
+}
+
+// ---------------------------------------------------------------------------------------------
+// One [d] reference for all B*T tokens of a tensor (a reference reduced over samples and
+// tokens): every token row is compared with the same vector m, and Eq. 1 moves m with the mean
+// over the token rows, m' = beta m + (1-beta)/(B*T) sum_rows x[row, :].  Only x streams (2
+// B/element); the work per element is what bounds the kernel.
+//
+// A CTA owns a block of rows as in the streaming kernel.  Inside, the columns are cut into
+// stripes of 512 (a warp tile) and a warp keeps ONE stripe for all its rows: its tile of m stays
+// in registers, and so do the column sums of x that Eq. 1 needs.  With fewer stripes than warps
+// several warps share a stripe and take every wps-th row (`phases`); with more, a warp does
+// several stripes one after the other.  Each (stripe, phase) pair is a slot: its column sums go
+// to the CTA's block of `col_part`, and channel_mean_kernel adds the blocks up in a fixed order.
+constexpr int kStripe = 8 * 32 * kUnroll;        // columns per stripe
+
+__host__ __device__ inline int channel_stripes(int d) { return (d + kStripe - 1) / kStripe; }
+__host__ __device__ inline int channel_phases(int d) {
+  const int stripes = channel_stripes(d);
+  return stripes < kWarps ? kWarps / stripes : 1;
+}
+__host__ __device__ inline int channel_slots(int d) { return channel_stripes(d) * channel_phases(d); }
+
+// One slot (a warp's stripe of columns, every `phases`-th row from `first` on) of a segment.
+// Per element only what is not linear in x is done: (x - x0)^2, |x - m|, the sign test, the
+// non-finite / constancy bits, and the column sum of x - x0.  The linear sums follow from the
+// column sums when the slot is done: sum (x - x0) = sum_c col_c and sum (x - x0)(m - m0) =
+// sum_c (m_c - m0) col_c, since m is the same in every row.
+// kZeroInM = false is the usual case, no exact zero among this warp's columns of m: then
+// sign(x) != sign(m) iff x, with its sign bit flipped where m is negative, is <= +0 as an integer
+// (a negative number, -0, or +0: x and m differ in sign, or x is zero against a non-zero m).
+template <bool kZeroInM>
+__device__ __forceinline__ void channel_slot(const StreamArgs &a, long long first, long long rb, int phases,
+                                             size_t lane_off, const bool (&ok)[kUnroll],
+                                             const float4 *const (&mp)[kUnroll], float4 *col, unsigned x0pair,
+                                             float x0f, ThreadAcc &t, long long &n_rows) {
+  // Two rows per trip; the next trip's rows are requested before this trip's arithmetic.  The
+  // reference (2 KB per warp, the same for every row) is fetched again each trip through L1
+  // rather than held in registers, which the second set of x would not leave room for.
+  uint4 cur[2][kUnroll], nxt[2][kUnroll];
+  auto fetch = [&](uint4 (&dst)[2][kUnroll], long long row) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const long long r = row + (long long)h * phases;
+      if (r < rb) {
+        const uint16_t *xr = a.x + (size_t)r * a.d + lane_off;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          if (ok[u]) dst[h][u] = ld_x128(xr + (size_t)u * 256);
+      }
+    }
+  };
+  if (first < rb) fetch(cur, first);
+  for (long long row = first; row < rb; row += 2 * phases) {
+    if (row + 2 * phases < rb) fetch(nxt, row + 2 * phases);
+    const bool second = row + phases < rb;
+    float g_sxx = 0.f, g_ab = 0.f;
+    unsigned g_flips = 0u;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (!ok[u]) continue;
+      const float4 lo = __ldg(mp[u]), hi = __ldg(mp[u] + 1);
+      const float mv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+      const float4 c_lo = col[u * 64], c_hi = col[u * 64 + 1];
+      float cs[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !second) continue;
+        const unsigned w4[4] = {cur[h][u].x, cur[h][u].y, cur[h][u].z, cur[h][u].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          t.nf_bits |= ((w4[q] & 0x7F807F80u) + 0x00800080u) & 0x80008000u;
+          t.x_diff |= w4[q] ^ x0pair;
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
+            const float mf = mv[2 * q + hlf];
+            const float xs = xf - x0f;
+            g_sxx = fmaf(xs, xs, g_sxx);
+            g_ab += fabsf(xf - mf);
+            const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
+            if (kZeroInM) g_flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
+            else g_flips += ((int)xt <= 0) ? 1u : 0u;
+            cs[2 * q + hlf] += xs;
+          }
+        }
+      }
+      col[u * 64] = make_float4(cs[0], cs[1], cs[2], cs[3]);
+      col[u * 64 + 1] = make_float4(cs[4], cs[5], cs[6], cs[7]);
+    }
+    t.sxx += (double)g_sxx;
+    t.ab += (double)g_ab;
+    t.flips += g_flips;
+    n_rows += second ? 2 : 1;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) cur[h][u] = nxt[h][u];
+  }
+}
+
+__device__ void channel_segment(const StreamArgs &a, int b, long long ra, long long rb, const float *m_in,
+                                float *col_seg, float *s_col, unsigned long long (*s_part)[kSlotWords],
+                                unsigned long long *slot) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunks = a.d >> 3;                   // d is a multiple of 8 here
+  const int stripes = channel_stripes(a.d), phases = channel_phases(a.d), n_slots = stripes * phases;
+  const unsigned x0 = a.x[(size_t)b * a.T * (size_t)a.d];
+  const unsigned x0pair = x0 | (x0 << 16);
+  const float x0f = __uint_as_float(x0 << 16);
+  const unsigned m0bits = __float_as_uint(__ldg(m_in));
+  const float m0 = __uint_as_float(m0bits);
+
+  ThreadAcc t = {0., 0., 0., 0., 0., 0., 0u, 0u, 0u, 0u};
+  for (int sl = warp; sl < n_slots; sl += kWarps) {
+    const int stripe = sl % stripes, phase = sl / stripes;
+    bool ok[kUnroll];
+    const float4 *mp[kUnroll];                   // this lane's 8 + 8 columns of the reference
+    // the slot's column sums of x - x0 live in the warp's 2 KB of shared memory: a lane only ever
+    // touches its own 8 + 8 words there, so no barrier is needed
+    float4 *col = reinterpret_cast<float4 *>(s_col + warp * kStripe) + lane * 2;
+    float lm = 0.f, lmm = 0.f;                   // this lane's sums of (m - m0), (m - m0)^2 over its columns
+    unsigned m_diff = 0u;
+    bool zero_in_m = false;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int c = stripe * 32 * kUnroll + u * 32 + lane;
+      ok[u] = c < chunks;
+      mp[u] = reinterpret_cast<const float4 *>(m_in) + (size_t)(ok[u] ? c : 0) * 2;
+      col[u * 64] = col[u * 64 + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ok[u]) {
+        const float4 lo = __ldg(mp[u]), hi = __ldg(mp[u] + 1);
+        const float mv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float ms = mv[e] - m0;
+          lm += ms;
+          lmm = fmaf(ms, ms, lmm);
+          m_diff |= __float_as_uint(mv[e]) ^ m0bits;
+          zero_in_m |= (mv[e] == 0.f);
+        }
+      }
+    }
+    long long n_rows = 0;
+    const size_t lane_off = (size_t)(stripe * 32 * kUnroll + lane) * 8;
+    if (__any_sync(0xffffffffu, zero_in_m))
+      channel_slot<true>(a, ra + phase, rb, phases, lane_off, ok, mp, col, x0pair, x0f, t, n_rows);
+    else
+      channel_slot<false>(a, ra + phase, rb, phases, lane_off, ok, mp, col, x0pair, x0f, t, n_rows);
+
+    // what is linear in x, from the column sums; the reference's own sums: its columns once per row
+    float4 *dst = reinterpret_cast<float4 *>(col_seg + (size_t)sl * kStripe) + lane * 2;
+    double s_x = 0., s_xm = 0.;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const float4 c_lo = col[u * 64], c_hi = col[u * 64 + 1];
+      dst[u * 64] = c_lo;
+      dst[u * 64 + 1] = c_hi;
+      if (ok[u]) {
+        const float4 lo = __ldg(mp[u]), hi = __ldg(mp[u] + 1);
+        const float mv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+        const float cs[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          s_x += (double)cs[e];
+          s_xm += (double)(mv[e] - m0) * (double)cs[e];
+        }
+      }
+    }
+    t.sx += s_x;
+    t.sxm += s_xm;
+    t.sm += (double)n_rows * (double)lm;
+    t.smm += (double)n_rows * (double)lmm;
+    if (n_rows) t.m_diff |= m_diff;
+  }
+  reduce_to_slot(t, b, x0, m0bits, s_part, slot);
+}
+
+__global__ void __launch_bounds__(kThreads)
+channel_ref_kernel(const StreamArgs a) {
+  __shared__ unsigned long long s_part[kWarps][kSlotWords];
+  __shared__ int s_last;
+  extern __shared__ double s_dyn[];            // CTA 0: the refresh's working copies; the others: kWarps * kStripe floats
+
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  const int act = __ldcg(&a.hs->kind[a.kind].active);     // written by an earlier launch only
+  const float *m_in = static_cast<const float *>(a.ema[act]);
+
+  if (blockIdx.x == 0) {
+    KindState *ks = &a.hs->kind[a.kind];
+    if (ks->refresh_pending)
+      refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
+  } else {
+    const int c = blockIdx.x - 1;
+    const long long R = (long long)a.B * a.T;
+    const long long R0 = (R * c) / a.G, R1 = (R * (c + 1)) / a.G;
+    const size_t seg_floats = (size_t)channel_slots(a.d) * kStripe;
+    long long ra = R0;
+    for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
+      unsigned long long *slot = a.partials + ((size_t)c * kSegsPerCta + sgm) * kSlotWords;
+      float *col_seg = a.col_part + ((size_t)c * kSegsPerCta + sgm) * seg_floats;
+      if (ra < R1) {
+        const int b = (int)(ra / a.T);
+        const long long sample_end = (long long)(b + 1) * a.T;
+        const long long rb = sample_end < R1 ? sample_end : R1;
+        channel_segment(a, b, ra, rb, m_in, col_seg, reinterpret_cast<float *>(s_dyn), s_part, slot);
+        ra = rb;
+      } else {                                    // no rows: nothing to add
+        for (size_t i = threadIdx.x; i < seg_floats; i += kThreads) col_seg[i] = 0.f;
+        if (threadIdx.x == 0) slot[7] = 0ull;
+      }
+    }
+  }
+
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(a.ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const FinalizeTarget ft = {0, a.partials, a.scores_out, a.flags_out, nullptr, 0, 1, 0};
+  finalize(a, ft);
+}
+
+// Second half of a step with a [d] reference: if the step committed, Eq. 1 with the mean over
+// the token rows into the spare buffer; the last CTA then makes that buffer the reference.  The
+// streaming CTAs left column sums of x - x0 per (CTA, segment, slot), x0 the first element of the
+// segment's sample; they are added in a fixed order, in double precision -- a CTA takes 32
+// columns, its 8 groups of threads every 8th block of partial sums -- and the shifts come back as
+// the one constant T * sum_b x[b,0,0].
+constexpr int kChannelMeanCols = 32, kChannelMeanGroups = 8;
+
+__global__ void __launch_bounds__(kChannelMeanCols * kChannelMeanGroups)
+channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const float *col_part, const uint16_t *x,
+                    int G, int B, int T, int d, float beta, float one_minus_beta) {
+  __shared__ double s_sum[kChannelMeanGroups][kChannelMeanCols];
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  KindState *ks = &hs->kind[kind];
+  // (cleared only by the CTA that draws the last ticket, i.e. after every CTA has read it)
+  if (!__ldcg(&ks->commit_pending)) return;
+  const int act = __ldcg(&ks->active);
+  const float *m_in = act ? ema1 : ema0;
+  float *m_out = act ? ema0 : ema1;
+  const int lane_c = threadIdx.x % kChannelMeanCols, group = threadIdx.x / kChannelMeanCols;
+  const int c = blockIdx.x * kChannelMeanCols + lane_c;
+  const int stripes = channel_stripes(d), phases = channel_phases(d), n_slots = stripes * phases;
+  const int n_blocks = G * kSegsPerCta * phases;           // blocks of partial sums that hold column c
+  double sum = 0.;
+  if (c < d) {
+    const int stripe = c / kStripe, within = c - stripe * kStripe;
+#pragma unroll 4
+    for (int i = group; i < n_blocks; i += kChannelMeanGroups) {
+      const int cs = i / phases, p = i - cs * phases;
+      sum += (double)__ldcg(col_part + ((size_t)cs * n_slots + (size_t)p * stripes + stripe) * kStripe + within);
+    }
+  }
+  s_sum[group][lane_c] = sum;
+  __syncthreads();
+  if (group == 0 && c < d) {
+    double total = 0., shift = 0.;
+    for (int g = 0; g < kChannelMeanGroups; ++g) total += s_sum[g][lane_c];
+    for (int b = 0; b < B; ++b) shift += (double)__uint_as_float((unsigned)x[(size_t)b * T * (size_t)d] << 16);
+    const double rows = (double)B * (double)T;
+    m_out[c] = (float)((double)beta * (double)m_in[c] + (double)one_minus_beta * ((total + (double)T * shift) / rows));
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned tk = atomicAdd(&hs->ticket2, 1u);
+    if (tk == gridDim.x - 1) {
+      __threadfence();
+      ks->active = act ^ 1;
+      ks->commit_pending = 0;
+      hs->ticket2 = 0u;
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

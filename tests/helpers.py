@@ -110,7 +110,7 @@ def parse_blob(blob, B, T, d, l, R=1) -> dict:
                 if i < M:
                     hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
                 off += 8 * cap
-        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape((T, d) if shared else (B, T, d)).copy()
+        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape((d,) if shared == 2 else (T, d) if shared else (B, T, d)).copy()
         off += 4 * N
         out["kinds"].append({"steps": steps, "count": (c0, c1), "valid": valid, "thr": thr,
                              "hist": hist, "m": m})

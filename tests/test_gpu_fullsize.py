@@ -21,9 +21,9 @@ def sb():
     return binding
 
 
-def run_steps(sb, oracle_mod, w, kind, n_warm, corruption):
-    gv = sb.Verifier(w.B, w.T, w.d)
-    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d))
+def run_steps(sb, oracle_mod, w, kind, n_warm, corruption, **variant):
+    gv = sb.Verifier(w.B, w.T, w.d, **variant)
+    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, **variant))
     for t in range(n_warm):
         x = synth.clean(w, 0, kind, t, "cuda")
         gs = gv.update_reference(x, kind)
@@ -177,6 +177,12 @@ def test_cfg4_shared_reference_of_identical_samples(sb):
         return np.frombuffer(blob, dtype=np.uint8, count=n, offset=64 + 192 + per_kind - n)
     assert np.array_equal(act_reference(one), act_reference(shared))
     one.close(); shared.close()
+
+
+def test_cfg4_channel_reference_against_the_oracle(sb, oracle_mod):
+    """4 x 8192 x 8192 with one [d] reference for all tokens: two warm-up steps, a clean and a
+    corrupted verified step, every score, statistic, flag and counter against the oracle."""
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], ACT, 2, "add_uniform_sample", ref_over_batch=1, ref_over_tokens=1)
 
 
 def test_cfg4_sliced_wasserstein_units(sb, oracle_mod):

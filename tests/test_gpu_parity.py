@@ -831,3 +831,95 @@ def test_shared_reference_restrictions_and_state_round_trip(sb):
         sb.Verifier(3, 8, 64).sentinel_import_state(blob)                          # another reference shape
     assert e.value.code == sb.ERR_STATE_SIZE
     gv.close(); other.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# one [d] reference shared by all B*T tokens (ref_over_batch = 1 and ref_over_tokens = 1)
+
+@pytest.mark.parametrize("name,shape,steps", [("cfg2", (6, 40, 1024), 50), ("cfg4", (4, 24, 2056), 40),
+                                              ("cfg3", (16, 30, 520), 60), ("cfg2", (1, 37, 264), 40),
+                                              ("cfg2", (3, 5, 11000), 30), ("cfg4", (39, 3, 512), 30)],
+                         ids=["cfg2_B6", "cfg4_B4", "cfg3_B16", "cfg2_B1", "cfg2_wide", "cfg4_B39"])
+def test_streams_in_lockstep_with_a_channel_reference(sb, oracle_mod, name, shape, steps):
+    w = synth.scaled(synth.WORKLOADS[name], name + "_channel", *shape, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w, ref_over_batch=1, ref_over_tokens=1)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, steps)
+    assert rec["corrupted"] >= 3
+    compare_state(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+        st = gv.sentinel_get_stats(kind).cpu().numpy()
+        x, _ = synth.microbatch(w, 0, kind, steps - 1, "cuda")
+        assert_stats_close(st, ov.last_stats(kind), max(float(x.float().std()), 1e-30),
+                           max(float(np.abs(ov.last_stats(kind)[0, 4])) ** 0.5, 1e-30), "stats kind %d" % kind)
+    assert rec["near"] <= 2 and rec["k_events"] <= 4, rec
+    # Alg. 4: every token receives the one vector
+    x, _ = synth.microbatch(w, 0, GRAD, 0, "cuda")
+    loud = (x.float() * 64).to(torch.bfloat16)
+    gv.verify(loud, GRAD)
+    ov.verify(synth.bits(loud), GRAD)
+    out = loud.clone()
+    gv.sentinel_replace_if_flagged(out, GRAD, 0)
+    want, did = ov.replace_if_flagged(synth.bits(loud), GRAD)
+    torch.cuda.synchronize()
+    assert did
+    got = synth.bits(out)
+    gv_, rv_ = oracle_mod.bf16_to_f64(got), oracle_mod.bf16_to_f64(want)
+    assert np.mean(got != want) <= 1e-3 and np.all(np.abs(gv_ - rv_) <= 2.0 ** -7 * np.abs(rv_) + 1e-6 * float(np.std(rv_)))
+    gv.close()
+
+
+def test_channel_reference_restrictions_and_state_round_trip(sb):
+    with pytest.raises(sb.SentinelError) as e:
+        sb.Verifier(2, 8, 64, ref_over_tokens=1)                                  # [d] means over the samples too
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    for kw in ({"n_workers": 2}, {"ema_bf16": 1}):
+        with pytest.raises(sb.SentinelError) as e:
+            sb.Verifier(2, 8, 64, ref_over_batch=1, ref_over_tokens=1, **kw)
+        assert e.value.code == sb.ERR_UNSUPPORTED
+    gv = sb.Verifier(3, 8, 64, ref_over_batch=1, ref_over_tokens=1)
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_set_directions(synth.directions(4, 64, 1, "cuda"))
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    s, f = torch.zeros(4, 3, device="cuda"), torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(sb.SentinelError) as e:
+        gv.sentinel_verify_strided(torch.zeros(3, 8, 65, dtype=torch.bfloat16, device="cuda"), ACT, s, f)
+    assert e.value.code == sb.ERR_UNSUPPORTED
+    w = synth.scaled(synth.WORKLOADS["cfg1"], "channel_rt", 3, 8, 64)
+    for t in range(5):
+        gv.update_reference(synth.clean(w, 0, ACT, t, "cuda"), ACT)
+    blob = bytes(gv.sentinel_export_state())
+    assert len(blob) < len(bytes(sb.Verifier(3, 8, 64, ref_over_batch=1).sentinel_export_state()))   # d values per kind
+    other = sb.Verifier(3, 8, 64, ref_over_batch=1, ref_over_tokens=1)
+    other.sentinel_import_state(blob)
+    assert bytes(other.sentinel_export_state()) == blob
+    x = synth.clean(w, 0, ACT, 5, "cuda")
+    a, b = gv.verify(x, ACT), other.verify(x, ACT)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    for kw in ({}, {"ref_over_batch": 1}):
+        with pytest.raises(sb.SentinelError) as e:
+            sb.Verifier(3, 8, 64, **kw).sentinel_import_state(blob)               # another reference shape
+        assert e.value.code == sb.ERR_STATE_SIZE
+    gv.close(); other.close()
+
+
+def test_channel_reference_runs_are_bit_reproducible_and_non_finite_input_changes_nothing(sb):
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "channel_rep", 5, 33, 1544)
+    blobs = []
+    for rep in range(2):
+        gv = sb.Verifier(w.B, w.T, w.d, ref_over_batch=1, ref_over_tokens=1)
+        for t in range(8):
+            gv.update_reference(synth.clean(w, 0, GRAD, t, "cuda"), GRAD)
+        before = bytes(gv.sentinel_export_state())
+        bad = synth.clean(w, 0, GRAD, 8, "cuda").clone()
+        bad[2, 7, 100] = float("inf")
+        s, f = gv.verify(bad, GRAD)
+        torch.cuda.synchronize()
+        f = f.cpu().numpy().view(np.uint32)
+        assert f[0] & sb.FLAG_NONFINITE and f[3] & sb.FLAG_NONFINITE and not (f[0] & sb.FLAG_COMMITTED)
+        st = parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, 100)
+        st0 = parse_blob(before, w.B, w.T, w.d, 100)
+        assert np.array_equal(st["kinds"][GRAD]["m"], st0["kinds"][GRAD]["m"])     # the reference did not move
+        blobs.append(bytes(gv.sentinel_export_state()))
+        gv.close()
+    assert blobs[0] == blobs[1]
