@@ -1346,6 +1346,41 @@ struct ReplicaShared {
   unsigned x0[kMaxWorkers];                       // the sample's first element, per worker
 };
 
+// One tensor's tile against the tile of m.  kZeroInM = false is the usual case, no exact zero in
+// the warp's tile of m (found out once per tile, for all tensors that share it): then
+// sign(x) != sign(m) iff x, with its sign bit flipped where m is negative, is <= +0 as an integer
+// (a negative number, -0, or +0: x and m differ in sign, or x is zero against a non-zero m).
+template <bool kZeroInM>
+__device__ __forceinline__ void replica_tile(const uint4 (&cur)[kUnroll], const F8 (&mv)[kUnroll], const bool (&ok)[kUnroll],
+                                             float x0f, float m0, unsigned x0pair, float (&sum)[kUnroll][8], float &sx,
+                                             float &sxx, float &sxm, float &ab, unsigned &flips, unsigned &nf,
+                                             unsigned &x_diff) {
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    if (!ok[u]) continue;
+    const unsigned w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      nf |= ((w4[q] & 0x7F807F80u) + 0x00800080u) & 0x80008000u;
+      x_diff |= w4[q] ^ x0pair;
+#pragma unroll
+      for (int hlf = 0; hlf < 2; ++hlf) {
+        const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
+        const float mf = mv[u].v[2 * q + hlf];
+        const float xs = xf - x0f, ms = mf - m0;
+        sx += xs;
+        sxx = fmaf(xs, xs, sxx);
+        sxm = fmaf(xs, ms, sxm);
+        ab += fabsf(xf - mf);
+        const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
+        if (kZeroInM) flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
+        else flips += ((int)xt <= 0) ? 1u : 0u;
+        sum[u][2 * q + hlf] += xf;
+      }
+    }
+  }
+}
+
 // (n_sets tensors share the tile of m: the R workers of a stage, or the B samples of one tensor
 // when the reference is a single [T,d] tensor for all of them)
 __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long long row_a, long long row_b,
@@ -1393,6 +1428,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
     // the reference's own sums, once per tile
     float g_sm = 0.f, g_smm = 0.f;
     unsigned m_diff = 0u;
+    bool zero_in_m = false;
     float sum[kUnroll][8];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
@@ -1404,9 +1440,11 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
           g_sm += ms;
           g_smm = fmaf(ms, ms, g_smm);
           m_diff |= __float_as_uint(mv[u].v[e]) ^ m0bits;
+          zero_in_m |= (mv[u].v[e] == 0.f);
         }
       }
     }
+    const bool any_zero = __any_sync(0xffffffffu, zero_in_m);
 
     for (unsigned rem = streamed; rem != 0u;) {              // the workers, in order
       const int r = __ffs(rem) - 1;
@@ -1424,29 +1462,8 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
       const float x0f = __uint_as_float(x0 << 16);
       float sx = 0.f, sxx = 0.f, sxm = 0.f, ab = 0.f;
       unsigned flips = 0u, nf = 0u, x_diff = 0u;
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        if (!ok[u]) continue;
-        const unsigned w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          nf |= ((w4[q] & 0x7F807F80u) + 0x00800080u) & 0x80008000u;
-          x_diff |= w4[q] ^ x0pair;
-#pragma unroll
-          for (int hlf = 0; hlf < 2; ++hlf) {
-            const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
-            const float mf = mv[u].v[2 * q + hlf];
-            const float xs = xf - x0f, ms = mf - m0;
-            sx += xs;
-            sxx = fmaf(xs, xs, sxx);
-            sxm = fmaf(xs, ms, sxm);
-            ab += fabsf(xf - mf);
-            const float xt = __uint_as_float(__float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u));
-            flips += (((xf == 0.f) != (mf == 0.f)) || (xt < 0.f)) ? 1u : 0u;
-            sum[u][2 * q + hlf] += xf;
-          }
-        }
-      }
+      if (any_zero) replica_tile<true>(cur, mv, ok, x0f, m0, x0pair, sum, sx, sxx, sxm, ab, flips, nf, x_diff);
+      else replica_tile<false>(cur, mv, ok, x0f, m0, x0pair, sum, sx, sxx, sxm, ab, flips, nf, x_diff);
       sx = warp_sum(sx); sxx = warp_sum(sxx); sxm = warp_sum(sxm); ab = warp_sum(ab);
       flips = __reduce_add_sync(0xffffffffu, flips);
       nf = __reduce_or_sync(0xffffffffu, nf);
