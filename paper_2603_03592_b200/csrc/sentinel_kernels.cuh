@@ -1260,9 +1260,9 @@ channel_ref_kernel(const StreamArgs a) {
 // the token rows into the spare buffer; the last CTA then makes that buffer the reference.  The
 // streaming CTAs left column sums of x - x0 per (CTA, segment, slot), x0 the first element of the
 // segment's sample; they are added in a fixed order, in double precision -- a CTA takes 32
-// columns, its 8 groups of threads every 8th block of partial sums -- and the shifts come back as
+// columns, its 16 groups of threads every 16th block of partial sums -- and the shifts come back as
 // the one constant T * sum_b x[b,0,0].
-constexpr int kChannelMeanCols = 32, kChannelMeanGroups = 8;
+constexpr int kChannelMeanCols = 32, kChannelMeanGroups = 16;
 
 __global__ void __launch_bounds__(kChannelMeanCols * kChannelMeanGroups)
 channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const float *col_part, const uint16_t *x,
@@ -1283,7 +1283,7 @@ channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const f
   double sum = 0.;
   if (c < d) {
     const int stripe = c / kStripe, within = c - stripe * kStripe;
-#pragma unroll 4
+#pragma unroll 8
     for (int i = group; i < n_blocks; i += kChannelMeanGroups) {
       const int cs = i / phases, p = i - cs * phases;
       sum += (double)__ldcg(col_part + ((size_t)cs * n_slots + (size_t)p * stripes + stripe) * kStripe + within);
