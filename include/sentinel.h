@@ -25,7 +25,7 @@
  * Variants of a handle (sentinel_config): n_workers > 1 follows all workers of a stage and takes
  * their tensors together (the fixed-mesh form of Eq. 1, worker loop of Alg. 2 / Alg. 3);
  * ema_bf16 stores the reference as bf16; ref_over_batch keeps one [T,d] reference for all
- * samples.
+ * samples, and with ref_over_tokens one [d] reference for all tokens.
  *
  * Conventions.  All tensors are dense, row-major [B,T,d] with d fastest (the _strided entry
  * points take padded rows).  x is bf16; the reference m is fp32 unless ema_bf16 is set, and is
