@@ -26,6 +26,7 @@ constexpr int kThreads = 640;             // threads per CTA: with kUnroll = 2 a
 constexpr int kWarps = kThreads / 32;
 constexpr int kSlotWords = 8;             // 64-bit words per partial slot
 constexpr int kUnroll = 2;                // 8-element chunks per lane per loop trip
+constexpr int kUnrollBf16 = 4;            // the same with a bf16 reference (vector rows)
 
 constexpr int kMaxWorkers = 16;           // workers (replicas of a stage) one handle can follow
 
@@ -149,19 +150,19 @@ __device__ __forceinline__ unsigned pack_bf16x2_rn(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // upper half <- first operand
   return r;
 }
+__device__ __forceinline__ F8 widen_bf16x8(const uint4 &v) {
+  const unsigned w[4] = {v.x, v.y, v.z, v.w};
+  F8 r;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    r.v[2 * j] = __uint_as_float(w[j] << 16);
+    r.v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+  }
+  return r;
+}
 template <bool kBf16>
 __device__ __forceinline__ F8 load_m8(const void *m, size_t idx) {
-  if (kBf16) {
-    const uint4 v = ld_x128(static_cast<const uint16_t *>(m) + idx);
-    const unsigned w[4] = {v.x, v.y, v.z, v.w};
-    F8 r;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      r.v[2 * j] = __uint_as_float(w[j] << 16);
-      r.v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-    }
-    return r;
-  }
+  if (kBf16) return widen_bf16x8(ld_x128(static_cast<const uint16_t *>(m) + idx));
   return ld_m256(static_cast<const float *>(m) + idx);
 }
 template <bool kBf16>
@@ -318,9 +319,12 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
                                const void *m_in, void *m_out,
                                unsigned long long (*s_part)[kSlotWords],
                                unsigned long long *slot) {
+  // chunks per lane and trip: with a bf16 reference a chunk brings 32 bytes instead of 48, so
+  // a trip takes more of them to keep as many bytes in flight
+  constexpr int kU = (kBf16 && !kScalar) ? kUnrollBf16 : kUnroll;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunks = (a.d + 7) >> 3;
-  const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
+  const int tiles_per_row = (chunks + 32 * kU - 1) / (32 * kU);
   const int n_tiles = (int)(rb - ra) * tiles_per_row;       // < 2^31: rows/G * d/1024
   const size_t sample_off = (size_t)b * a.T * a.d;
   const bool write_ema = (m_out != nullptr);
@@ -339,7 +343,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
   for (int j = warp; j < n_tiles; j += kWarps) {
     const long long row = ra + rr;
     const size_t off = (size_t)row * a.d;
-    const int base = seg * 32 * kUnroll;
+    const int base = seg * 32 * kU;
     GroupAcc g = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0u};
 
     if (kScalar) {
@@ -368,23 +372,27 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
         }
       }
     } else {
-      uint4 xv[kUnroll];
-      F8 mv[kUnroll];
-      bool ok[kUnroll];
+      uint4 xv[kU];
+      F8 mv[kBf16 ? 1 : kU];
+      uint4 mraw[kBf16 ? kU : 1];          // a bf16 reference stays packed until its chunk is worked on
+      bool ok[kU];
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
+      for (int u = 0; u < kU; ++u) {
         const int c = base + u * 32 + lane;
         ok[u] = c < chunks;
         if (ok[u]) {
           xv[u] = ld_x128(a.x + off + (size_t)c * 8);
-          mv[u] = load_m8<kBf16>(m_in, off + (size_t)c * 8);
+          if (kBf16) mraw[u] = ld_x128(static_cast<const uint16_t *>(m_in) + off + (size_t)c * 8);
+          else mv[u] = ld_m256(static_cast<const float *>(m_in) + off + (size_t)c * 8);
         }
       }
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
+      for (int u = 0; u < kU; ++u) {
         if (ok[u]) {
-          chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
-          if (write_ema) store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+          F8 &m8 = mv[kBf16 ? 0 : u];
+          if (kBf16) m8 = widen_bf16x8(mraw[u]);
+          chunk(xv[u], m8, g, t, x0pair, m0bits, beta, omb, write_ema);
+          if (write_ema) store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, m8);
         }
       }
     }
