@@ -384,7 +384,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         cms = c0.elapsed_time(c1) / 9
         strided = {"row_stride": w.d + 1, "bytes_per_element": 10, "ms_per_launch": round(cms, 4),
-                   "achieved_gbs": round(10 * N / (cms * 1e-3) / 1e9, 1), "kernel": "stream_kernel_t<true, false>"}
+                   "achieved_gbs": round(10 * N / (cms * 1e-3) / 1e9, 1), "kernel": "stream_kernel_t<false, false, true> (funnel-shifted rows)"}
         del wide
 
     # end to end through the host-buffer entry point

@@ -274,11 +274,15 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
     SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, shared_ref_kernel, ra));
     return SENTINEL_OK;
   }
+  // strided rows: the funnel-shift variant of the vector path when the width allows it, else scalar
+  const bool shifted = scalar && h->cfg.d % 8 == 0;
   if (h->bf16) {
-    if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, true>, a));
+    if (shifted) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, true, true>, a));
+    else if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, true>, a));
     else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, true>, a));
   } else {
-    if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, false>, a));
+    if (shifted) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, false, true>, a));
+    else if (scalar) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<true, false>, a));
     else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, stream_kernel_t<false, false>, a));
   }
   return SENTINEL_OK;
@@ -562,6 +566,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);

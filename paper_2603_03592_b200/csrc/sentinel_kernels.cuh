@@ -298,6 +298,82 @@ __device__ __forceinline__ void reduce_to_slot(const ThreadAcc &t, int b, unsign
   }
 }
 
+// Rows of x that start on any 2-byte boundary (the compressed-signal layout with a row width that
+// is a multiple of 8): a lane's 8 elements straddle two aligned 16-byte words.  The misalignment
+// `s` (bytes, even) is the same for every chunk of a row.  A lane loads the aligned word below its
+// chunk; the word above it is its neighbour's, fetched by a shuffle -- or by a load of its own
+// for lane 31 and for the last chunk of the row, where no neighbour holds it -- and a funnel
+// shift by s puts the 8 elements in place.  Past the end of the tensor (last chunk of the last row)
+// the upper word is put together from 2-byte loads of the elements that exist.
+__device__ __forceinline__ uint4 shifted_chunk(const uint4 &w0, const uint4 &w1, unsigned s) {
+  const unsigned in[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+  const unsigned bs = (s & 3u) * 8u;
+  uint4 out;
+  switch (s >> 2) {                     // the same for the whole warp
+    case 0:
+      out.x = __funnelshift_r(in[0], in[1], bs); out.y = __funnelshift_r(in[1], in[2], bs);
+      out.z = __funnelshift_r(in[2], in[3], bs); out.w = __funnelshift_r(in[3], in[4], bs);
+      break;
+    case 1:
+      out.x = __funnelshift_r(in[1], in[2], bs); out.y = __funnelshift_r(in[2], in[3], bs);
+      out.z = __funnelshift_r(in[3], in[4], bs); out.w = __funnelshift_r(in[4], in[5], bs);
+      break;
+    case 2:
+      out.x = __funnelshift_r(in[2], in[3], bs); out.y = __funnelshift_r(in[3], in[4], bs);
+      out.z = __funnelshift_r(in[4], in[5], bs); out.w = __funnelshift_r(in[5], in[6], bs);
+      break;
+    default:
+      out.x = __funnelshift_r(in[3], in[4], bs); out.y = __funnelshift_r(in[4], in[5], bs);
+      out.z = __funnelshift_r(in[5], in[6], bs); out.w = __funnelshift_r(in[6], in[7], bs);
+      break;
+  }
+  return out;
+}
+
+template <int kU>
+__device__ __forceinline__ void load_x_shifted(const uint16_t *row_ptr, int base, int chunks, bool last_row,
+                                               const bool (&ok)[kU], uint4 (&xv)[kU]) {
+  const int lane = threadIdx.x & 31;
+  const unsigned s = (unsigned)(reinterpret_cast<uintptr_t>(row_ptr) & 15u);
+  if (s == 0u) {
+#pragma unroll
+    for (int u = 0; u < kU; ++u)
+      if (ok[u]) xv[u] = ld_x128(row_ptr + (size_t)(base + u * 32 + lane) * 8);
+    return;
+  }
+  const uint16_t *al = row_ptr - (s >> 1);                 // 16-byte aligned
+  // all loads first (the few lanes that fetch their own upper word included), then the shuffles
+  uint4 w0[kU], own[kU];
+  bool direct[kU];
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+    const int c = base + u * 32 + lane;
+    w0[u] = own[u] = make_uint4(0u, 0u, 0u, 0u);
+    direct[u] = ok[u] && (lane == 31 || c + 1 >= chunks);  // nobody holds the word above this chunk
+    if (ok[u]) w0[u] = ld_x128(al + (size_t)c * 8);
+    if (direct[u]) {
+      const uint16_t *up = al + (size_t)(c + 1) * 8;
+      if (last_row && c + 1 >= chunks) {                   // only its first s bytes exist for sure
+        unsigned e[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        for (unsigned k = 0; k < (s >> 1); ++k) e[k] = up[k];
+        own[u] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+      } else {
+        own[u] = ld_x128(up);
+      }
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+    uint4 w1;
+    w1.x = __shfl_down_sync(0xffffffffu, w0[u].x, 1);
+    w1.y = __shfl_down_sync(0xffffffffu, w0[u].y, 1);
+    w1.z = __shfl_down_sync(0xffffffffu, w0[u].z, 1);
+    w1.w = __shfl_down_sync(0xffffffffu, w0[u].w, 1);
+    if (direct[u]) w1 = own[u];
+    if (ok[u]) xv[u] = shifted_chunk(w0[u], w1, s);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // streaming phase
 //
@@ -314,7 +390,7 @@ constexpr int kSegsPerCta = 2;
 // appendix): rows of x are row_stride elements apart and start on any 2-byte boundary, and d
 // need not be a multiple of 8.  Lanes then own interleaved columns (col = tile + q*32 + lane),
 // so that every 2-byte / 4-byte access of a warp is contiguous; the arithmetic is the same.
-template <bool kScalar, bool kBf16>
+template <bool kScalar, bool kBf16, bool kShifted>
 __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long long rb,
                                const void *m_in, void *m_out,
                                unsigned long long (*s_part)[kSlotWords],
@@ -381,11 +457,14 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
         const int c = base + u * 32 + lane;
         ok[u] = c < chunks;
         if (ok[u]) {
-          xv[u] = ld_x128(a.x + off + (size_t)c * 8);
+          if (!kShifted) xv[u] = ld_x128(a.x + off + (size_t)c * 8);
           if (kBf16) mraw[u] = ld_x128(static_cast<const uint16_t *>(m_in) + off + (size_t)c * 8);
           else mv[u] = ld_m256(static_cast<const float *>(m_in) + off + (size_t)c * 8);
         }
       }
+      if (kShifted)
+        load_x_shifted<kU>(a.x + (size_t)row * (size_t)a.x_row_stride, base, chunks,
+                           row == (long long)a.B * a.T - 1, ok, xv);
 #pragma unroll
       for (int u = 0; u < kU; ++u) {
         if (ok[u]) {
@@ -441,7 +520,7 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
   reduce_to_slot(t, b, x0, m0bits, s_part, slot);
 }
 
-template <bool kScalar, bool kBf16>
+template <bool kScalar, bool kBf16, bool kShifted>
 __device__ void stream_cta(const StreamArgs &a, int c, const void *m_in, void *m_out,
                            unsigned long long (*s_part)[kSlotWords]) {
   const long long R = (long long)a.B * a.T;
@@ -453,7 +532,7 @@ __device__ void stream_cta(const StreamArgs &a, int c, const void *m_in, void *m
       const int b = (int)(ra / a.T);
       const long long sample_end = (long long)(b + 1) * a.T;
       const long long rb = sample_end < R1 ? sample_end : R1;
-      stream_segment<kScalar, kBf16>(a, b, ra, rb, m_in, m_out, s_part, slot);
+      stream_segment<kScalar, kBf16, kShifted>(a, b, ra, rb, m_in, m_out, s_part, slot);
       ra = rb;
     } else if (threadIdx.x == 0) {
       slot[7] = 0ull;                   // tag 0: unused
@@ -987,10 +1066,11 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
 // step left that pending) while the others stream.  Every CTA then takes a ticket; whoever
 // draws the last one has, by the fence/atomic order, everybody's partial sums and the fresh
 // thresholds in view, and finalizes.  No CTA ever waits for another.
-// (kScalar = true is the variant for rows of x that are strided or not 16-byte aligned; it is a
-// kernel of its own so that the vector path keeps its registers.  kBf16 = true: the reference
-// buffers hold bf16 instead of fp32.)
-template <bool kScalar, bool kBf16>
+// (kScalar = true is the variant for rows of x that are strided or not 16-byte aligned, of any
+// width; kShifted = true the one for such rows when the width is a multiple of 8: the vector
+// path with x put in place by a funnel shift.  They are kernels of their own so that the vector
+// path keeps its registers.  kBf16 = true: the reference buffers hold bf16 instead of fp32.)
+template <bool kScalar, bool kBf16, bool kShifted = false>
 __global__ void __launch_bounds__(kThreads)
 stream_kernel_t(const StreamArgs a) {
   __shared__ unsigned long long s_part[kWarps][kSlotWords];
@@ -1021,7 +1101,7 @@ stream_kernel_t(const StreamArgs a) {
         refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
     }
   } else {
-    stream_cta<kScalar, kBf16>(a, blockIdx.x - 1, m_in, m_out, s_part);
+    stream_cta<kScalar, kBf16, kShifted>(a, blockIdx.x - 1, m_in, m_out, s_part);
   }
 
   __threadfence();

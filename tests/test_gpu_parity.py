@@ -541,6 +541,50 @@ def test_compressed_signal_layout(sb, oracle_mod, k, stride):
     gv.close()
 
 
+@pytest.mark.parametrize("k,stride,offset", [(1024, 1025, 0), (512, 515, 3), (2056, 2057, 5), (264, 272, 7),
+                                             (8, 9, 1), (1528, 1536, 2)],
+                         ids=["k1024_s1025", "k512_s515_o3", "k2056_s2057_o5", "k264_s272_o7", "k8_s9_o1", "k1528_s1536_o2"])
+def test_compressed_signal_layout_with_rows_on_any_2_byte_boundary(sb, oracle_mod, k, stride, offset):
+    """The same layout with k a multiple of 8, where the library puts x in place with a funnel
+    shift and keeps the 128/256-bit path: every misalignment of a row start (strides and base
+    offsets that walk through all residues mod 16 bytes), a last row that ends with the
+    allocation, both reference formats."""
+    B, T = 3, 29
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "compressed_shift", B, T, stride)
+    n = B * T * stride
+    for bf16 in (0, 1):
+        gv = sb.Verifier(B, T, k, ema_bf16=bf16)
+        params = oracle_mod.Params(B=B, T=T, d=k, ema_bf16=bf16)
+        ov = oracle_mod.Verifier(params)
+        for t in range(12):
+            src = synth.clean(w, 0, GRAD, t, "cuda")
+            if t == 10:
+                src = (src.float() * 5).to(torch.bfloat16)
+            # the tensor ends exactly where its allocation ends; its base is `offset` elements in
+            flat = torch.empty(offset + n, dtype=torch.bfloat16, device="cuda")
+            wide = flat[offset:].view(B, T, stride)
+            wide.copy_(src)
+            wide[:, :, k:] = 1000.0                            # never looked at
+            packed = wide[:, :, :k].contiguous()
+            scale = float(packed.float().abs().mean())
+            gs = torch.empty(1 + B, 3, device="cuda")
+            if t < 7:
+                gv.sentinel_update_reference_strided(wide, GRAD, gs)
+                os_, _ = ov.update_reference(synth.bits(packed), GRAD)
+            else:
+                gf = torch.empty(1 + B, dtype=torch.int32, device="cuda")
+                gv.sentinel_verify_strided(wide, GRAD, gs, gf)
+                os_, of, _ = ov.verify(synth.bits(packed), GRAD)
+                assert np.array_equal(gf.cpu().numpy().view(np.uint32), of), t
+            assert_scores_close(gs.cpu().numpy(), os_, scale, "shifted step %d" % t)
+        if bf16:
+            st = parse_blob(gv.sentinel_export_state(), B, T, k, 100)
+            assert np.array_equal(st["kinds"][GRAD]["m"].astype(np.float64), ov.ema(GRAD))   # bit for bit
+        else:
+            compare_state(gv, ov, params)
+        gv.close()
+
+
 def test_runs_are_bit_reproducible(sb):
     w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_rep", 4, 50, 1024)
     blobs, outs = [], []
