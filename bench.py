@@ -38,7 +38,7 @@ MAX_DISTINCT = 24               # distinct input tensors per kind kept resident
 # ncu capture summarised in profiles/stream_kernel_cfg3_ncu_full.md (B=8 x 4096 x 4096; traffic
 # grows in proportion to the element count, so a launch of N elements moves this times N).
 # Set to None whenever the kernel changes until the capture is retaken.
-NCU_DRAM_BYTES_PER_ELEMENT = 9.673
+NCU_DRAM_BYTES_PER_ELEMENT = 9.679
 
 
 def measured_peak_gbs():

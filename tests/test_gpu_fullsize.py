@@ -179,6 +179,33 @@ def test_cfg4_shared_reference_of_identical_samples(sb):
     one.close(); shared.close()
 
 
+def test_cfg4_compressed_layout_equals_the_dense_call_bit_for_bit(sb):
+    """4 x 8192 x 8192 inside a [4, 8192, 8193] tensor (rows on every 2-byte boundary): the
+    funnel-shifted loads hand the arithmetic the same words as the dense call gets, so scores,
+    flags and the whole exported state are the same bits."""
+    w = synth.WORKLOADS["cfg4"]
+    dense, wide_v = sb.Verifier(w.B, w.T, w.d), sb.Verifier(w.B, w.T, w.d)
+    for t in range(4):
+        x = synth.clean(w, 0, GRAD, t, "cuda")
+        if t == 3:
+            x = synth.corrupt(w, x, "add_uniform_sample", 0, GRAD, t)
+        wide = torch.nn.functional.pad(x, (0, 1), value=77.0).contiguous()
+        s2 = torch.empty(1 + w.B, 3, device="cuda")
+        if t < 2:
+            s1 = dense.update_reference(x, GRAD)
+            wide_v.sentinel_update_reference_strided(wide, GRAD, s2)
+        else:
+            s1, f1 = dense.verify(x, GRAD)
+            f2 = torch.empty(1 + w.B, dtype=torch.int32, device="cuda")
+            wide_v.sentinel_verify_strided(wide, GRAD, s2, f2)
+            assert torch.equal(f1, f2), t
+        torch.cuda.synchronize()
+        assert torch.equal(s1, s2), t
+        del wide
+    assert bytes(dense.sentinel_export_state()) == bytes(wide_v.sentinel_export_state())
+    dense.close(); wide_v.close()
+
+
 def test_cfg4_channel_reference_against_the_oracle(sb, oracle_mod):
     """4 x 8192 x 8192 with one [d] reference for all tokens: two warm-up steps, a clean and a
     corrupted verified step, every score, statistic, flag and counter against the oracle."""
