@@ -334,22 +334,22 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned blo
   return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
 }
 
-template <int L, int kT>
+template <int L, int kT, bool kRefOnly>
 cudaError_t projection_occupancy(size_t smem, int *occ) {
-  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT, kRefOnly>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT>, kT, smem);
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT, kRefOnly>, kT, smem);
 }
 
-template <int L>
+template <int L, bool kRefOnly = false>
 cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                               const uint16_t *u, float *proj, long long rows, int d, int sms, const ProjectionState &ps,
                               cudaStream_t s) {
   const size_t smem = (size_t)L * d * sizeof(uint16_t);
   int occ_small = 0, occ_large = 0;
-  cudaError_t e = projection_occupancy<L, 512>(smem, &occ_small);
+  cudaError_t e = projection_occupancy<L, 512, kRefOnly>(smem, &occ_small);
   if (e != cudaSuccess) return e;
-  e = projection_occupancy<L, 768>(smem, &occ_large);
+  e = projection_occupancy<L, 768, kRefOnly>(smem, &occ_large);
   if (e != cudaSuccess) return e;
   const bool large = occ_large * 768 > occ_small * 512;
   const int threads = large ? 768 : 512, occ = large ? occ_large : occ_small;
@@ -358,10 +358,10 @@ cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m
   const long long need = (rows + threads / 32 - 1) / (threads / 32);
   if (grid > need) grid = need;
   if (large)
-    return launch_chained(swd_project_kernel<L, 768>, (unsigned)grid, 768, smem, s, x, m0, m1, active, skip, u, proj, rows, d,
-                          ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
-  return launch_chained(swd_project_kernel<L, 512>, (unsigned)grid, 512, smem, s, x, m0, m1, active, skip, u, proj, rows, d,
-                        ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+    return launch_chained(swd_project_kernel<L, 768, kRefOnly>, (unsigned)grid, 768, smem, s, x, m0, m1, active, skip, u, proj,
+                          rows, d, ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+  return launch_chained(swd_project_kernel<L, 512, kRefOnly>, (unsigned)grid, 512, smem, s, x, m0, m1, active, skip, u, proj,
+                        rows, d, ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
 }
 
 // x alone, on the tensor cores: the reference's projections come from the verifier's own buffers
@@ -443,13 +443,14 @@ int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bo
   int sms = 0;
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
   ProjectionState ps;
-  if (h->R == 1) {       // one submission per update: the reference's projections follow it (Eq. 1 is linear)
-    ps.pm0 = h->sw_pm[kind][0];
-    ps.pm1 = h->sw_pm[kind][1];
-    ps.incremental = h->sw_pm_valid[kind];
-    ps.beta = (float)h->cfg.beta[kind];
-    ps.one_minus_beta = (float)(1.0 - h->cfg.beta[kind]);
-  }
+  ps.pm0 = h->sw_pm[kind][0];
+  ps.pm1 = h->sw_pm[kind][1];
+  ps.beta = (float)h->cfg.beta[kind];
+  ps.one_minus_beta = (float)(1.0 - h->cfg.beta[kind]);
+  // One submission per update: the reference's projections follow it (Eq. 1 is linear).  Several
+  // workers: run_reference_projection has just put P(m) into the current buffer; what the x-only
+  // launch writes into the spare one is never adopted.
+  ps.incremental = h->R == 1 ? h->sw_pm_valid[kind] : true;
   SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), static_cast<const float *>(h->ema[kind][0]),
                            static_cast<const float *>(h->ema[kind][1]), &h->hs->kind[kind].active,
                            may_skip ? &h->hs->banned[worker] : nullptr, h->sw_u, h->sw_L, h->cfg.B, h->cfg.T,
@@ -458,6 +459,32 @@ int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bo
   return SENTINEL_OK;
 }
 
+// A verifier with directions that follows several workers: the reference's projections, once per
+// iteration, for all workers' chains to read.
+int run_reference_projection(sentinel_verifier *h, int kind, cudaStream_t s) {
+  if (!h->sw_u || h->R == 1) return SENTINEL_OK;
+  int sms = 0;
+  SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
+  ProjectionState ps;
+  ps.pm0 = h->sw_pm[kind][0];
+  ps.pm1 = h->sw_pm[kind][1];
+  const float *m0 = static_cast<const float *>(h->ema[kind][0]), *m1 = static_cast<const float *>(h->ema[kind][1]);
+  const int *active = &h->hs->kind[kind].active;
+  const long long rows = (long long)h->cfg.B * h->cfg.T;
+  cudaError_t e;
+  if (h->sw_L == 4) e = launch_projection<4, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  else if (h->sw_L == 8) e = launch_projection<8, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  else e = launch_projection<16, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  SENTINEL_CUDA(h, e);
+  return SENTINEL_OK;
+}
+
+// a single submission (worker slot 0), whatever the number of workers the handle follows
+int run_single_swd(sentinel_verifier *h, const void *x, int kind, cudaStream_t s) {
+  int rc = run_reference_projection(h, kind, s);
+  if (rc) return rc;
+  return run_handle_swd(h, x, kind, 0, false, s);
+}
 
 void free_all(sentinel_verifier *h) {
   for (int k = 0; k < 2; ++k) {
@@ -619,7 +646,7 @@ int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
   h->started = true;
-  rc = run_handle_swd(h, dev_x, kind, 0, false, static_cast<cudaStream_t>(cuda_stream));
+  rc = run_single_swd(h, dev_x, kind, static_cast<cudaStream_t>(cuda_stream));
   if (rc) return rc;
   return launch(h, make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out), h->G + 1,
                 static_cast<cudaStream_t>(cuda_stream));
@@ -632,7 +659,7 @@ int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_
   DeviceGuard guard(h->cfg.device);
   SENTINEL_CUDA(h, guard.status);
   h->started = true;
-  rc = run_handle_swd(h, dev_x, kind, 0, false, static_cast<cudaStream_t>(cuda_stream));
+  rc = run_single_swd(h, dev_x, kind, static_cast<cudaStream_t>(cuda_stream));
   if (rc) return rc;
   return launch(h, make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr), h->G + 1,
                 static_cast<cudaStream_t>(cuda_stream));
@@ -682,7 +709,7 @@ int sentinel_verify_host(sentinel_verifier *h, const void *host_x, sentinel_kind
   }
   SENTINEL_CUDA(h, cudaMemcpyAsync(h->stage_x, host_x, h->N * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
   h->started = true;
-  int rc = run_handle_swd(h, h->stage_x, kind, 0, false, s);
+  int rc = run_single_swd(h, h->stage_x, kind, s);
   if (rc) return rc;
   rc = launch(h, make_args(h, h->stage_x, kind, kModeVerify, h->stage_scores, h->stage_flags), h->G + 1, s);
   if (rc) return rc;
@@ -772,6 +799,10 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigne
   ra.tainted_in = tainted_in;
   WorkerPointers wp;
   memset(&wp, 0, sizeof wp);
+  {
+    int rc = run_reference_projection(h, kind, s);
+    if (rc) return rc;
+  }
   for (int r = 0; r < h->R; ++r) {
     if ((tainted_in >> r) & 1u) continue;
     ra.xs[r] = wp.x[r] = static_cast<const uint16_t *>(xs[r]);

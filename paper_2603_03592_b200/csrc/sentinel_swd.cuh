@@ -39,7 +39,11 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 // verifier's first step or its first step after a state import -- and, if the buffers are given,
 // stores it in the current one and the candidate P(m_t) in the spare one; from then on
 // swd_project_mma_kernel carries the buffers along and reads x only, 2 B/element instead of 6.
-template <int L, int kSwdThreads>
+// kRefOnly = true projects the reference alone into the current buffer (x is not read, nothing
+// else is written): once per iteration of a verifier that follows several workers, whose
+// reference moves with the mean over the clean workers rather than by that recursion; its
+// workers then all take the x-only launch against the same P(m).
+template <int L, int kSwdThreads, bool kRefOnly = false>
 __global__ void __launch_bounds__(kSwdThreads, kSwdThreads == 512 ? 2 : 1)
 swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
                    const uint16_t *u, float *proj, long long rows, int d, double *pm0, double *pm1, float beta,
@@ -73,7 +77,7 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
         const int c = c0 + 32 * h;
         ok[h] = c < chunks;
         if (ok[h]) {
-          xv[h] = ld_x128(x + off + (size_t)c * 8);
+          if (!kRefOnly) xv[h] = ld_x128(x + off + (size_t)c * 8);
           mv[h] = ld_m256(m + off + (size_t)c * 8);
         }
       }
@@ -81,12 +85,12 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
       for (int h = 0; h < 2; ++h) {
         if (!ok[h]) continue;
         const int c = c0 + 32 * h;
-        const unsigned xw[4] = {xv[h].x, xv[h].y, xv[h].z, xv[h].w};
         float xf[8];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          xf[2 * j] = __uint_as_float(xw[j] << 16);
-          xf[2 * j + 1] = __uint_as_float(xw[j] & 0xFFFF0000u);
+          const unsigned xw = kRefOnly ? 0u : (j == 0 ? xv[h].x : j == 1 ? xv[h].y : j == 2 ? xv[h].z : xv[h].w);
+          xf[2 * j] = __uint_as_float(xw << 16);
+          xf[2 * j + 1] = __uint_as_float(xw & 0xFFFF0000u);
         }
 #pragma unroll
         for (int l = 0; l < L; ++l) {
@@ -95,8 +99,10 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float u_lo = __uint_as_float(uw[j] << 16), u_hi = __uint_as_float(uw[j] & 0xFFFF0000u);
-            ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
-            ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
+            if (!kRefOnly) {
+              ax[l] = fmaf(xf[2 * j], u_lo, ax[l]);
+              ax[l] = fmaf(xf[2 * j + 1], u_hi, ax[l]);
+            }
             am[l] = fmaf(mv[h].v[2 * j], u_lo, am[l]);
             am[l] = fmaf(mv[h].v[2 * j + 1], u_hi, am[l]);
           }
@@ -105,9 +111,13 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
     }
 #pragma unroll
     for (int l = 0; l < L; ++l) {
-      const float sx = warp_sum(ax[l]), sm = warp_sum(am[l]);
+      const float sx = kRefOnly ? 0.f : warp_sum(ax[l]), sm = warp_sum(am[l]);
       if (lane == l) {
         const size_t at = (size_t)row * L + l;
+        if (kRefOnly) {
+          pm_cur[at] = (double)sm;
+          continue;
+        }
         proj[(size_t)l * rows + row] = sx;
         proj[((size_t)L + l) * rows + row] = sm;
         if (pm_cur) {
