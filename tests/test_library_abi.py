@@ -94,9 +94,15 @@ def test_host_side_argument_checks_need_no_gpu(built):
     assert L.sentinel_sliced_wasserstein(None, None, None, 8, 1, 1, 8, 0, None, None) == binding.ERR_INVALID_ARG
     assert L.sentinel_distance_noalloc(None, None, 1, 1, 8, 0, None, None, None) == binding.ERR_INVALID_ARG
     # configuration ranges
-    for bad in (dict(n_workers=17), dict(ema_bf16=2), dict(ref_over_batch=3), dict(window_steps=0)):
+    for bad in (dict(n_workers=17), dict(ema_bf16=2), dict(ref_over_batch=3), dict(window_steps=0),
+                dict(ref_over_batch=1, ref_over_tokens=2)):
         cfg = binding.sentinel_default_config(B=2, T=4, d=16, **bad)
         assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_INVALID_ARG, bad
+    # combinations of variants that are not built
+    for bad in (dict(ref_over_tokens=1), dict(ref_over_batch=1, n_workers=2), dict(ema_bf16=1, n_workers=2),
+                dict(ref_over_batch=1, ref_over_tokens=1, ema_bf16=1)):
+        cfg = binding.sentinel_default_config(B=2, T=4, d=16, **bad)
+        assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_UNSUPPORTED, bad
     with pytest.raises(TypeError):
         binding.sentinel_default_config(B=2, T=4, d=16, no_such_field=1)
 
