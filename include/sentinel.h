@@ -196,9 +196,13 @@ int sentinel_update_reference(sentinel_verifier *h, const void *dev_x, sentinel_
  * 2-byte alignment only; d may be any positive number.  This is the layout of a
  * subspace-compressed signal, of which the verifier checks x[:, :, :-1] (SWARM appendix,
  * "compatibility with subspace compression"): pass the [B,T,k+1] tensor with d = k and
- * row_stride = k+1.  The reference stays dense [B,T,d].  Same arithmetic, scalar instead of
- * 128/256-bit memory accesses.  A handle created with d % 8 != 0 can only be used through
- * these two calls (and the queries / checkpointing). */
+ * row_stride = k+1.  The reference stays dense [B,T,d].  Same arithmetic.  With d a multiple
+ * of 8 the 128/256-bit accesses are kept and x is read in aligned 16-byte words that are shifted
+ * into place: bytes of such a word that lie outside the verified elements (up to 14 before the
+ * first element of a row or after its last one) are read and ignored, and no word is read that
+ * holds no verified element.  With any other d the accesses are scalar (slower).  A handle
+ * created with d % 8 != 0 can only be used through these two calls (and the queries /
+ * checkpointing). */
 int sentinel_verify_strided(sentinel_verifier *h, const void *dev_x, sentinel_kind kind, int B, int T,
                             int d, long long row_stride, void *cuda_stream, float *dev_scores_out,
                             unsigned *dev_flags_out);
