@@ -136,6 +136,43 @@ def test_cfg4_identical_workers_reduce_to_one_submission(sb):
     one.close(); many.close()
 
 
+def test_cfg3_two_workers_against_the_oracle(sb, oracle_mod):
+    """8 x 4096 x 4096, two workers per iteration: two warm-up iterations, a clean verified one and
+    one in which worker 1 submits a tensor five times too large -- every worker's scores, flags
+    and counters, and a sample of the reference after the mean over the clean workers."""
+    w = synth.WORKLOADS["cfg3"]
+    R = 2
+    gv = sb.Verifier(w.B, w.T, w.d, n_workers=R)
+    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, R=R))
+    for t in range(4):
+        xs = [synth.clean(w, r, GRAD, t, "cuda") for r in range(R)]
+        if t == 3:
+            xs[1] = (xs[1].float() * 5).to(torch.bfloat16)
+        thr, valid = ov.thresholds(GRAD)
+        gs, gf = gv.step_replicas(xs, GRAD, t < 2)
+        os_, of, n_clean = ov.step_replicas([synth.bits(x) for x in xs], GRAD, t < 2)
+        torch.cuda.synchronize()
+        gs, gf = gs.cpu().numpy(), gf.cpu().numpy().view(np.uint32)
+        for r in range(R):
+            assert_scores_close(gs[r], os_[r], float(xs[r].float().abs().mean()), "iteration %d worker %d" % (t, r))
+        if t >= 2 and not np.array_equal(gf, of):
+            for r in range(R):
+                near = near_threshold(os_[r], thr, valid, w.B)
+                assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+        if t == 3:
+            assert of[1, 0] & UNIT_BITS and not (of[0, 0] & UNIT_BITS) and n_clean == 1
+    for r in range(R):
+        assert gv.sentinel_get_worker_counters(r) == ov.worker_counters(r)
+    blob = gv.sentinel_export_state()
+    per_kind = (gv.sentinel_state_bytes() - 64 - 192) // 2
+    n = w.B * w.T * w.d
+    m_gpu = np.frombuffer(blob, dtype="<f4", count=n, offset=64 + 192 + 2 * per_kind - 4 * n)   # the gradients' reference
+    m_ref = ov.ema(GRAD).reshape(-1)
+    idx = np.random.default_rng(0).integers(0, n, 200000)
+    assert np.max(np.abs(m_gpu[idx] - m_ref[idx])) <= 1e-5 * float(np.abs(m_ref[idx]).max())
+    gv.close()
+
+
 def test_cfg4_bf16_reference_first_update(sb):
     """From m_0 = 0 one update leaves bf16((1-beta) x) in single precision, here checked on the
     whole 4 x 8192 x 8192 tensor against torch's multiply and conversion."""
