@@ -333,16 +333,17 @@ class Verifier:
 
     def ema(self, kind: int) -> np.ndarray:
         p = lib().so_ema(self._h, kind)
-        if self.params.ref_over_tokens:           # one [d] reference for all tokens
-            return np.ctypeslib.as_array(p, shape=(self.d,)).copy()
-        if self.params.ref_over_batch:            # one [T,d] reference for all samples
-            return np.ctypeslib.as_array(p, shape=(self.T * self.d,)).copy().reshape(self.T, self.d)
-        return np.ctypeslib.as_array(p, shape=(self.N,)).copy().reshape(self.B, self.T, self.d)
+        shape = self.ref_shape()
+        return np.ctypeslib.as_array(p, shape=(int(np.prod(shape)),)).copy().reshape(shape)
+
+    def ref_shape(self) -> tuple:
+        """[B,T,d], or with the reference reduced over the samples / the tokens: [T,d], [B,d], [d]."""
+        over_b, over_t = self.params.ref_over_batch, self.params.ref_over_tokens
+        return tuple(([] if over_b else [self.B]) + ([] if over_t else [self.T]) + [self.d])
 
     def set_ema(self, kind: int, m):
         mm = np.ascontiguousarray(m, dtype=np.float64).reshape(-1)
-        assert mm.size == (self.d if self.params.ref_over_tokens else
-                           self.T * self.d if self.params.ref_over_batch else self.N)
+        assert mm.size == int(np.prod(self.ref_shape()))
         lib().so_set_ema(self._h, kind, _dptr(mm))
 
     def history(self, kind: int, level: int, metric: int) -> np.ndarray:

@@ -278,16 +278,25 @@ static void window_push(so_window *w, double val) {
   w->v[w->n++] = val;
 }
 
+/* which element of the reference stands for element e of a [B,T,d] tensor */
+static size_t ref_index(const so_verifier *v, size_t e) {
+  const size_t d = (size_t)v->p.d, c = e % d, t = (e / d) % (size_t)v->p.T, b = e / v->Ns;
+  const size_t tt = v->p.ref_over_tokens ? 0 : t, bb = v->p.ref_over_batch ? 0 : b;
+  const size_t rows_per_sample = v->p.ref_over_tokens ? 1 : (size_t)v->p.T;
+  return (bb * rows_per_sample + tt) * d + c;
+}
+
 so_verifier *so_create(const so_params *p) {
   if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1 || p->R < 1 || p->R > SO_MAX_WORKERS) return NULL;
   if (p->ema_bf16 && p->R != 1) return NULL;   /* the bf16 reference exists for one submission per update */
   if (p->ref_over_batch && (p->R != 1 || p->ema_bf16)) return NULL;   /* likewise the [T,d] reference */
-  if (p->ref_over_tokens && !p->ref_over_batch) return NULL;          /* [d] = over samples and tokens */
+  if (p->ref_over_tokens && (p->R != 1 || p->ema_bf16)) return NULL;  /* and the [B,d] / [d] references */
   so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
   v->p = *p;
   v->Ns = (size_t)p->T * (size_t)p->d;
   v->N = v->Ns * (size_t)p->B;
-  v->Nm = p->ref_over_tokens ? (size_t)p->d : p->ref_over_batch ? v->Ns : v->N;   /* elements of the reference */
+  /* elements of the reference: [B,T,d], [T,d] (over the samples), [B,d] (over the tokens), [d] (over both) */
+  v->Nm = (p->ref_over_batch ? 1u : (size_t)p->B) * (p->ref_over_tokens ? 1u : (size_t)p->T) * (size_t)p->d;
   v->u = NULL; v->n_dir = 0; v->nm = 3;
   for (int kind = 0; kind < 2; ++kind) {
     so_kind_state *ks = &v->ks[kind];
@@ -340,7 +349,7 @@ static void all_units(so_verifier *v, const uint16_t *x, int kind, double *gam, 
   double *wide = NULL;
   if (v->Nm != v->N) {
     wide = (double *)malloc(v->N * sizeof(double));
-    for (size_t k = 0; k < v->N / v->Nm; ++k) memcpy(wide + k * v->Nm, ks->m, v->Nm * sizeof(double));
+    for (size_t e = 0; e < v->N; ++e) wide[e] = ks->m[ref_index(v, e)];
   }
   const double *m = wide ? wide : ks->m;
   for (int r = 0; r <= v->p.B; ++r) {
@@ -381,13 +390,12 @@ static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
       m[e] = so_bf16(so_bf16_round((double)fmaf(bf, (float)m[e], of * (float)so_bf16(x[e]))));
     return;
   }
-  if (v->Nm != v->N) {   /* Eq. 1 with the mean over the B samples (the B*T tokens) as the submission */
+  if (v->Nm != v->N) {   /* Eq. 1 with the mean over the samples and / or tokens as the submission */
     const size_t copies = v->N / v->Nm;
-    for (size_t e = 0; e < v->Nm; ++e) {
-      double sum = 0.0;
-      for (size_t k = 0; k < copies; ++k) sum += so_bf16(x[k * v->Nm + e]);
-      m[e] = beta * m[e] + (1.0 - beta) * (sum / (double)copies);
-    }
+    double *sum = (double *)calloc(v->Nm, sizeof(double));
+    for (size_t e = 0; e < v->N; ++e) sum[ref_index(v, e)] += so_bf16(x[e]);
+    for (size_t i = 0; i < v->Nm; ++i) m[i] = beta * m[i] + (1.0 - beta) * (sum[i] / (double)copies);
+    free(sum);
     return;
   }
   for (size_t e = 0; e < v->N; ++e) m[e] = beta * m[e] + (1.0 - beta) * so_bf16(x[e]);
@@ -601,7 +609,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
 int so_replace_if_flagged(const so_verifier *v, uint16_t *x, int kind, int fill) {
   if (!v->ks[kind].last_flagged) return 0;
   const double *m = v->ks[kind].m;                 /* a flagged step left m at m_{t-1} */
-  for (size_t e = 0; e < v->N; ++e) x[e] = fill ? 0 : so_bf16_round(m[e % v->Nm]);
+  for (size_t e = 0; e < v->N; ++e) x[e] = fill ? 0 : so_bf16_round(m[ref_index(v, e)]);
   return 1;
 }
 

@@ -24,8 +24,8 @@
  *   - the number and the draw of the sliced Wasserstein directions (the caller supplies them),
  *   - the two storage variants the paper does not mention: a reference stored as bf16 (its
  *     rounding is pinned to an independent single-precision computation, the choice of the
- *     variant itself is not the paper's), one [T,d] reference for all samples of a tensor and
- *     one [d] reference for all its tokens (Eq. 1 with the mean over the samples / tokens).
+ *     variant itself is not the paper's), and the references reduced over the samples ([T,d]),
+ *     over the tokens ([B,d]) or over both ([d]) (Eq. 1 with the mean over what is reduced).
  */
 #ifndef SENTINEL_ORACLE_H
 #define SENTINEL_ORACLE_H
@@ -73,7 +73,8 @@ typedef struct so_params {
   int    R;                /* workers (replicas) feeding this boundary, d_s >= 1    */
   int    ema_bf16;         /* != 0: the reference is stored as bf16 (R = 1 only)    */
   int    ref_over_batch;   /* != 0: one [T,d] reference for all B samples (R = 1)   */
-  int    ref_over_tokens;  /* != 0 (with ref_over_batch): one [d] reference for all B*T tokens */
+  int    ref_over_tokens;  /* != 0: one reference row for all T tokens of a sample: [B,d], or
+                              [d] together with ref_over_batch (R = 1)               */
 } so_params;
 
 typedef struct so_verifier so_verifier;
@@ -172,7 +173,7 @@ void so_worker_counters(const so_verifier *v, int r, int out[3]);   /* v_r, stre
 void so_reset_worker(so_verifier *v);
 
 /* State access for tests. */
-const double *so_ema(const so_verifier *v, int kind);                 /* B*T*d values (T*d with ref_over_batch, d with ref_over_tokens too) */
+const double *so_ema(const so_verifier *v, int kind);                 /* B*T*d values; T*d with ref_over_batch, B*d with ref_over_tokens, d with both */
 void   so_set_ema(so_verifier *v, int kind, const double *m);
 size_t so_history(const so_verifier *v, int kind, int level, int metric,
                   double *out, size_t cap);                            /* oldest first      */

@@ -60,8 +60,10 @@ def oracle_to_blob(v, params) -> bytes:
     """Serialise an oracle verifier into the library's checkpoint format."""
     B, T, d, l, R = params.B, params.T, params.d, params.l, params.R
     M = v.nm                                   # metrics in use; the layout has room for four
-    # 0: [B,T,d] reference, 1: one [T,d] reference for all samples, 2: one [d] reference for all tokens
-    shared = 2 if getattr(params, "ref_over_tokens", 0) else int(getattr(params, "ref_over_batch", 0))
+    # 0: [B,T,d] reference, 1: one [T,d] reference for all samples, 2: one [d] reference for all
+    # tokens, 3: a [B,d] reference, one vector per sample
+    over_b, over_t = int(getattr(params, "ref_over_batch", 0)), int(getattr(params, "ref_over_tokens", 0))
+    shared = {(0, 0): 0, (1, 0): 1, (1, 1): 2, (0, 1): 3}[(over_b, over_t)]
     out = bytearray(struct.pack("<QI7i", MAGIC, 3, B, T, d, l, R, M, shared))
     out += b"\0" * (64 - len(out))
     workers = np.zeros((3, 16), dtype="<i4")
@@ -97,7 +99,8 @@ def parse_blob(blob, B, T, d, l, R=1) -> dict:
     off = 64 + 192
     out = {"violations": int(workers[0, 0]), "clean_streak": int(workers[1, 0]), "banned": int(workers[2, 0]),
            "workers": workers.copy(), "n_metrics": M, "ref_over_batch": shared, "kinds": []}
-    N = d if shared == 2 else T * d if shared else B * T * d
+    ref_shape = {0: (B, T, d), 1: (T, d), 2: (d,), 3: (B, d)}[shared]
+    N = int(np.prod(ref_shape))
     for _ in range(2):
         steps, c0, c1 = struct.unpack_from("<q2i", buf, off)
         valid = np.array(struct.unpack_from("<8i", buf, off + 16)).reshape(2, 4).astype(bool)[:, :M]
@@ -110,7 +113,7 @@ def parse_blob(blob, B, T, d, l, R=1) -> dict:
                 if i < M:
                     hist[L][i] = np.frombuffer(buf, dtype="<f8", count=cap, offset=off)[:cnt].copy()
                 off += 8 * cap
-        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape((d,) if shared == 2 else (T, d) if shared else (B, T, d)).copy()
+        m = np.frombuffer(buf, dtype="<f4", count=N, offset=off).reshape(ref_shape).copy()
         off += 4 * N
         out["kinds"].append({"steps": steps, "count": (c0, c1), "valid": valid, "thr": thr,
                              "hist": hist, "m": m})

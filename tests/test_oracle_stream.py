@@ -759,6 +759,64 @@ def test_channel_reference_flags_commit_and_replacement(oracle_mod, small):
     got = from_bits(out)
     assert np.all(np.abs(got - m0) <= 2.0 ** -8 * np.abs(m0) + 1e-45)      # every token receives the one vector
     with pytest.raises(ValueError):
-        oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_tokens=1))           # [d] means over samples too
-    with pytest.raises(ValueError):
         oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_batch=1, ref_over_tokens=1, R=2))
+
+
+# ---------------------------------------------------------------------------------------------
+# one [B,d] reference: a vector per sample, shared by the sample's T tokens
+
+def test_per_sample_channel_reference_follows_each_samples_token_mean(oracle_mod):
+    """Eq. 1 with the mean over the T token rows of every sample: closed form from m_0 = 0, and
+    the samples do not mix (changing sample 1 leaves the reference of sample 0 alone)."""
+    rs = np.random.default_rng(61)
+    B, T, d = 3, 5, 8
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_tokens=1)
+    u = make(oracle_mod, B=B, T=T, d=d, ref_over_tokens=1)
+    want = np.zeros((B, d))
+    for t in range(6):
+        x = rs.normal(0.5, 1, (B, T, d))
+        xb = to_bits(x)
+        v.update_reference(xb, ACT)
+        y = x.copy(); y[1] += 3.0
+        u.update_reference(to_bits(y), ACT)
+        want = 0.9 * want + 0.1 * from_bits(xb).mean(axis=1)
+        assert v.ema(ACT).shape == (B, d)
+        assert v.ema(ACT) == pytest.approx(want, rel=1e-13, abs=1e-16)
+        assert np.array_equal(u.ema(ACT)[[0, 2]], v.ema(ACT)[[0, 2]]) and not np.allclose(u.ema(ACT)[1], v.ema(ACT)[1])
+
+
+def test_per_sample_channel_reference_scores_are_those_against_the_tiled_reference(oracle_mod):
+    rs = np.random.default_rng(62)
+    B, T, d = 3, 4, 8
+    v = make(oracle_mod, B=B, T=T, d=d, ref_over_tokens=1)
+    for t in range(5):
+        v.update_reference(to_bits(rs.normal(0, 1, (B, T, d)) + np.arange(d) + np.arange(B)[:, None, None]), GRAD)
+    m = v.ema(GRAD)                                                      # [B, d]
+    xb = to_bits(rs.normal(0, 1, (B, T, d)) + np.arange(d))
+    scores, flags, _ = v.verify(xb, GRAD)
+    tiled = np.repeat(m[:, None, :], T, axis=1)                          # [B, T, d]
+    g0, s0, _ = oracle_mod.distance(xb, tiled)
+    assert np.array_equal(scores[0], g0) and np.array_equal(v.last_stats(GRAD)[0], s0)
+    for b in range(B):
+        gb, _, _ = oracle_mod.distance(xb[b], tiled[b])
+        assert np.array_equal(scores[1 + b], gb)
+
+
+def test_per_sample_channel_reference_commit_and_replacement(oracle_mod, small):
+    v = oracle_mod.Verifier(oracle_mod.Params(B=small.B, T=small.T, d=small.d, ref_over_tokens=1))
+    for t in range(14):
+        v.update_reference(synth.bits(synth.clean(small, 0, ACT, t)), ACT)
+    h = synth.clean(small, 0, ACT, 14)
+    _, flags, commit = v.verify(synth.bits(h), ACT)
+    assert commit and not (flags & 0xFFFF).any()
+    m0 = v.ema(ACT)
+    loud = (h.float() * 50).to(torch.bfloat16)
+    _, flags, commit = v.verify(synth.bits(loud), ACT)
+    assert not commit and (flags[0] & 0xFFFF) and np.array_equal(v.ema(ACT), m0)
+    out, did = v.replace_if_flagged(synth.bits(loud), ACT)
+    assert did
+    got = from_bits(out)
+    for b in range(small.B):                                 # every token of sample b receives that sample's vector
+        assert np.all(np.abs(got[b] - m0[b]) <= 2.0 ** -8 * np.abs(m0[b]) + 1e-45)
+    with pytest.raises(ValueError):
+        oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_tokens=1, ema_bf16=1))
