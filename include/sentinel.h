@@ -25,7 +25,8 @@
  * Variants of a handle (sentinel_config): n_workers > 1 follows all workers of a stage and takes
  * their tensors together (the fixed-mesh form of Eq. 1, worker loop of Alg. 2 / Alg. 3);
  * ema_bf16 stores the reference as bf16; ref_over_batch keeps one [T,d] reference for all
- * samples, and with ref_over_tokens one [d] reference for all tokens.
+ * samples, ref_over_tokens one vector per sample for all its tokens ([B,d]; with both: one [d]
+ * vector).
  *
  * Conventions.  All tensors are dense, row-major [B,T,d] with d fastest (the _strided entry
  * points take padded rows).  x is bf16; the reference m is fp32 unless ema_bf16 is set, and is
@@ -105,8 +106,8 @@ typedef struct sentinel_config {
   int    n_workers;        /* workers d_s feeding this boundary (multi-worker calls)   1    */
   int    ema_bf16;         /* 1: the reference is stored as bf16 (see below)           0    */
   int    ref_over_batch;   /* 1: one [T,d] reference for all B samples (see below)     0    */
-  int    ref_over_tokens;  /* 1 (with ref_over_batch = 1): one [d] reference for all
-                              B*T tokens (see below)                                   0    */
+  int    ref_over_tokens;  /* 1: one reference row for all T tokens of a sample: [B,d],
+                              or [d] together with ref_over_batch (see below)          0    */
 } sentinel_config;
 
 typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundary */
@@ -140,7 +141,10 @@ typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundar
  * the step committed, makes it the reference); both are enqueued by the same call.  Restrictions:
  * n_workers = 1, fp32 reference, d a multiple of 8; no strided tensors, no
  * sentinel_set_directions, no per-token buffer.  Gradient replacement writes the vector into
- * every token.  State blobs carry d reference values per kind; the header's shape field is 2. */
+ * every token.  State blobs carry d reference values per kind; the header's shape field is 2.
+ * ref_over_tokens = 1 alone keeps one such vector PER SAMPLE, a [B,d] reference: the tokens of
+ * sample b are compared with vector b, which Eq. 1 moves with the mean over that sample's T token
+ * rows; everything else as above.  State blobs then carry B*d values per kind, shape field 3. */
 int sentinel_default_config(sentinel_config *cfg);
 
 /* Allocates the state of one boundary on cfg->device: two fp32 [B,T,d] buffers per kind (the
@@ -354,7 +358,8 @@ int sentinel_reset_worker(sentinel_verifier *h, int worker, void *cuda_stream);
  * i32 violations[16], clean_streak[16], banned[16], then per kind {i64 steps; i32 count[2];
  * i32 valid[2][4]; f64 thr[2][4][6]; f64 history[level 0: 4][window_steps*n_workers],
  * [level 1: 4][window_steps*n_workers*B] (oldest first, zero-padded); f32 m[B*T*d] (m[T*d] with
- * ref_over_batch, header field 1; m[d] with ref_over_tokens as well, header field 2)}.  The
+ * ref_over_batch, header field 1; m[d] with ref_over_tokens as well, field 2; m[B*d] with
+ * ref_over_tokens alone, field 3)}.  The
  * layout always has room for four metrics; with n_metrics = 3 the fourth slots are unused.
  * A blob goes back only into a verifier with the same n_metrics (the directions themselves
  * are not part of the state: set them before importing).  Export and import wait for the

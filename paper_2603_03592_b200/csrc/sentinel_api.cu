@@ -62,7 +62,8 @@ struct sentinel_verifier {
   void *ema[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // fp32, or bf16 if bf16
   bool bf16 = false;                // the reference is stored as bf16
   bool shared_ref = false;          // one [T,d] reference for all B samples
-  bool chan_ref = false;            // one [d] reference for all B*T tokens
+  bool chan_ref = false;            // the reference is reduced over the tokens: one [d] vector, or
+  bool chan_per_sample = false;     //   one per sample ([B,d])
   float *col_part = nullptr;        // chan_ref: column sums of x per streaming CTA and slot
   size_t ema_elems = 0;             // elements of one reference buffer: B*T*d, T*d if shared_ref, d if chan_ref
   size_t ema_bytes = 0;             // bytes of one reference buffer
@@ -235,6 +236,7 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.n_metrics = h->n_metrics;
   a.sw = h->sw_out;                 // nullptr until directions are set
   a.defer_commit = h->chan_ref ? 1 : 0;
+  a.ref_per_sample = h->chan_per_sample ? 1 : 0;
   a.col_part = h->col_part;
   return a;
 }
@@ -257,12 +259,12 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
     if (lc.dynamicSmemBytes < col_smem) lc.dynamicSmemBytes = col_smem;
     SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel, a));
     cudaLaunchConfig_t lm = lc;
-    lm.gridDim = dim3((unsigned)((h->cfg.d + kChannelMeanCols - 1) / kChannelMeanCols));
+    lm.gridDim = dim3((unsigned)((h->cfg.d + kChannelMeanCols - 1) / kChannelMeanCols), h->chan_per_sample ? (unsigned)h->cfg.B : 1u);
     lm.blockDim = dim3(kChannelMeanCols * kChannelMeanGroups);
     lm.dynamicSmemBytes = 0;
     SENTINEL_CUDA(h, cudaLaunchKernelEx(&lm, channel_mean_kernel, h->hs, a.kind, static_cast<float *>(a.ema[0]),
                                         static_cast<float *>(a.ema[1]), static_cast<const float *>(h->col_part), a.x,
-                                        h->G, h->cfg.B, h->cfg.T, h->cfg.d, a.beta, a.one_minus_beta));
+                                        h->G, h->cfg.B, h->cfg.T, h->cfg.d, h->chan_per_sample ? 1 : 0, a.beta, a.one_minus_beta));
     return SENTINEL_OK;
   }
   if (h->shared_ref) {                             // the samples in the workers' place (vector rows only)
@@ -554,8 +556,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   if (cfg->ref_over_batch && (cfg->n_workers != 1 || cfg->ema_bf16 || (cfg->B > kMaxWorkers && !cfg->ref_over_tokens) || cfg->d % 8 != 0))
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a [T,d] reference needs n_workers = 1, an fp32 reference, B <= %d and d a multiple of 8", kMaxWorkers);
   if (cfg->ref_over_tokens != 0 && cfg->ref_over_tokens != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ref_over_tokens must be 0 or 1, got %d", cfg->ref_over_tokens);
-  if (cfg->ref_over_tokens && !cfg->ref_over_batch)
-    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a [d] reference is one for all samples and tokens: set ref_over_batch = 1 as well");
+  if (cfg->ref_over_tokens && (cfg->n_workers != 1 || cfg->ema_bf16 || cfg->d % 8 != 0))
+    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a reference reduced over the tokens needs n_workers = 1, an fp32 reference and d a multiple of 8");
   if ((long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1) > SENTINEL_MAX_WINDOW)
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "window_steps*n_workers*(B+1) = %lld exceeds SENTINEL_MAX_WINDOW = %d",
                 (long long)cfg->window_steps * cfg->n_workers * (cfg->B + 1), SENTINEL_MAX_WINDOW);
@@ -575,7 +577,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   h->bf16 = cfg->ema_bf16 != 0;
   h->chan_ref = cfg->ref_over_tokens != 0;
   h->shared_ref = cfg->ref_over_batch != 0 && !h->chan_ref;
-  h->ema_elems = h->chan_ref ? (size_t)cfg->d : h->shared_ref ? h->Ns : h->N;
+  h->chan_per_sample = h->chan_ref && cfg->ref_over_batch == 0;
+  h->ema_elems = h->chan_ref ? (size_t)cfg->d * (h->chan_per_sample ? (size_t)cfg->B : 1u) : h->shared_ref ? h->Ns : h->N;
   h->ema_bytes = h->ema_elems * (h->bf16 ? sizeof(uint16_t) : sizeof(float));
   h->units0 = h->R;                       // the window spans window_steps iterations of all workers
   h->units1 = h->R * cfg->B;
@@ -883,7 +886,8 @@ int sentinel_replace_if_flagged(sentinel_verifier *h, void *dev_x_inout, sentine
   if (grid > need) grid = need;
   replace_kernel<<<(unsigned)grid, kReplaceThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       h->hs, (int)kind, h->ema[kind][0], h->ema[kind][1], h->bf16 ? 1 : 0, static_cast<uint16_t *>(dev_x_inout), n_chunks,
-      (h->shared_ref || h->chan_ref) ? (long long)(h->ema_elems / 8) : 0ll, fill,
+      h->chan_ref ? (long long)(h->cfg.d / 8) : h->shared_ref ? (long long)(h->ema_elems / 8) : 0ll,
+      h->chan_per_sample ? (long long)(h->Ns / 8) : 0ll, fill,
       dev_replaced_out);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
@@ -1082,7 +1086,7 @@ int sentinel_export_state(sentinel_verifier *h, void *host_buf, size_t n, void *
 
   unsigned char *out = static_cast<unsigned char *>(host_buf);
   memset(out, 0, kHeaderBytes);
-  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics, h->chan_ref ? 2 : h->shared_ref ? 1 : 0};
+  BlobHeader hd = {kMagic, kVersion, h->cfg.B, h->cfg.T, h->cfg.d, h->cfg.window_steps, h->R, h->n_metrics, h->chan_per_sample ? 3 : h->chan_ref ? 2 : h->shared_ref ? 1 : 0};
   memcpy(out, &hd, sizeof hd);
   out += kHeaderBytes;
   BlobWorkers bw;
@@ -1143,8 +1147,8 @@ int sentinel_import_state(sentinel_verifier *h, const void *host_buf, size_t n, 
     return fail(h, SENTINEL_ERR_STATE_SIZE, "not a sentinel state blob of version %u", kVersion);
   if (hd.B != h->cfg.B || hd.T != h->cfg.T || hd.d != h->cfg.d || hd.window_steps != h->cfg.window_steps || hd.n_workers != h->R)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob is for shape [%d,%d,%d], window %d, %d workers", hd.B, hd.T, hd.d, hd.window_steps, hd.n_workers);
-  if (hd.ref_over_batch != (h->chan_ref ? 2 : h->shared_ref ? 1 : 0))
-    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob and verifier differ in the shape of the reference ([B,T,d], [T,d] or [d])");
+  if (hd.ref_over_batch != (h->chan_per_sample ? 3 : h->chan_ref ? 2 : h->shared_ref ? 1 : 0))
+    return fail(h, SENTINEL_ERR_STATE_SIZE, "blob and verifier differ in the shape of the reference ([B,T,d], [T,d], [d] or [B,d])");
   if (hd.n_metrics != h->n_metrics)
     return fail(h, SENTINEL_ERR_STATE_SIZE, "blob holds %d metrics, this verifier uses %d (set the directions before importing)", hd.n_metrics, h->n_metrics);
   // validate both kinds before touching the device

@@ -110,7 +110,7 @@ struct StreamArgs {
   const float *sw;                 // [1+B] sliced Wasserstein distance of every unit, computed by the
                                    // launches before this one; nullptr when n_metrics = 3
   int n_metrics;                   // metrics in use: 3, or 4 with the sliced Wasserstein distance
-  int pad2;
+  int ref_per_sample;              // reduced reference with a vector per sample ([B,d]) instead of one ([d])
   Alg5Params a5;
   double severe_mult;
   int ban_violations, forgiveness_steps;
@@ -1225,6 +1225,7 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
   const unsigned x0 = a.x[(size_t)b * a.T * (size_t)a.d];
   const unsigned x0pair = x0 | (x0 << 16);
   const float x0f = __uint_as_float(x0 << 16);
+  if (a.ref_per_sample) m_in += (size_t)b * a.d;           // sample b's own vector
   const unsigned m0bits = __float_as_uint(__ldg(m_in));
   const float m0 = __uint_as_float(m0bits);
 
@@ -1354,7 +1355,7 @@ constexpr int kChannelMeanCols = 32, kChannelMeanGroups = 16;
 
 __global__ void __launch_bounds__(kChannelMeanCols * kChannelMeanGroups)
 channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const float *col_part, const uint16_t *x,
-                    int G, int B, int T, int d, float beta, float one_minus_beta) {
+                    int G, int B, int T, int d, int per_sample, float beta, float one_minus_beta) {
   __shared__ double s_sum[kChannelMeanGroups][kChannelMeanCols];
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -1362,18 +1363,25 @@ channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const f
   // (cleared only by the CTA that draws the last ticket, i.e. after every CTA has read it)
   if (!__ldcg(&ks->commit_pending)) return;
   const int act = __ldcg(&ks->active);
-  const float *m_in = act ? ema1 : ema0;
-  float *m_out = act ? ema0 : ema1;
+  // blockIdx.y: with a vector per sample, the sample whose vector this CTA moves
+  const int sample = per_sample ? (int)blockIdx.y : -1;
+  const size_t ref_off = per_sample ? (size_t)sample * d : 0;
+  const float *m_in = (act ? ema1 : ema0) + ref_off;
+  float *m_out = (act ? ema0 : ema1) + ref_off;
   const int lane_c = threadIdx.x % kChannelMeanCols, group = threadIdx.x / kChannelMeanCols;
   const int c = blockIdx.x * kChannelMeanCols + lane_c;
   const int stripes = channel_stripes(d), phases = channel_phases(d), n_slots = stripes * phases;
   const int n_blocks = G * kSegsPerCta * phases;           // blocks of partial sums that hold column c
+  const long long R = (long long)B * T;
   double sum = 0.;
   if (c < d) {
     const int stripe = c / kStripe, within = c - stripe * kStripe;
 #pragma unroll 8
     for (int i = group; i < n_blocks; i += kChannelMeanGroups) {
-      const int cs = i / phases, p = i - cs * phases;
+      const int cs = i / phases, p = i - cs * phases;      // (CTA, segment) pair and row phase
+      // CTA cs/2 owns rows [R*cta/G, R*(cta+1)/G): its first segment lies in the sample of its first
+      // row, its second (if any: else blocks of zeros) in the next one
+      if (per_sample && (int)(((R * (cs >> 1)) / G) / T) + (cs & 1) != sample) continue;
       sum += (double)__ldcg(col_part + ((size_t)cs * n_slots + (size_t)p * stripes + stripe) * kStripe + within);
     }
   }
@@ -1382,15 +1390,16 @@ channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const f
   if (group == 0 && c < d) {
     double total = 0., shift = 0.;
     for (int g = 0; g < kChannelMeanGroups; ++g) total += s_sum[g][lane_c];
-    for (int b = 0; b < B; ++b) shift += (double)__uint_as_float((unsigned)x[(size_t)b * T * (size_t)d] << 16);
-    const double rows = (double)B * (double)T;
+    for (int b = per_sample ? sample : 0; b < (per_sample ? sample + 1 : B); ++b)
+      shift += (double)__uint_as_float((unsigned)x[(size_t)b * T * (size_t)d] << 16);
+    const double rows = per_sample ? (double)T : (double)B * (double)T;
     m_out[c] = (float)((double)beta * (double)m_in[c] + (double)one_minus_beta * ((total + (double)T * shift) / rows));
   }
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
     const unsigned tk = atomicAdd(&hs->ticket2, 1u);
-    if (tk == gridDim.x - 1) {
+    if (tk == gridDim.x * gridDim.y - 1) {
       __threadfence();
       ks->active = act ^ 1;
       ks->commit_pending = 0;
@@ -1756,7 +1765,8 @@ __device__ __forceinline__ void st_x128(uint16_t *p, const uint4 &v) {
 
 __global__ void __launch_bounds__(kReplaceThreads)
 replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *ema1, int ema_bf16, uint16_t *x,
-               long long n_chunks, long long ref_chunks, int zero_fill, unsigned *replaced_out) {
+               long long n_chunks, long long ref_chunks, long long sample_chunks, int zero_fill,
+               unsigned *replaced_out) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const KindState *ks = &hs->kind[kind];
   const int flagged = ks->last_flagged;
@@ -1766,7 +1776,9 @@ replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *em
   const long long stride = (long long)gridDim.x * kReplaceThreads;
   for (long long c = (long long)blockIdx.x * kReplaceThreads + threadIdx.x; c < n_chunks; c += stride) {
     uint4 out = make_uint4(0u, 0u, 0u, 0u);
-    const long long cm = ref_chunks ? c % ref_chunks : c;   // a [T,d] reference repeats for every sample
+    // a [T,d] or [d] reference repeats every ref_chunks; a [B,d] one holds a row of ref_chunks per sample
+    const long long cm = sample_chunks ? (c / sample_chunks) * ref_chunks + c % ref_chunks
+                                       : ref_chunks ? c % ref_chunks : c;
     if (!zero_fill && ema_bf16) {                 // the reference already is a bf16 tensor
       out = ld_x128(static_cast<const uint16_t *>(m) + cm * 8);
     } else if (!zero_fill) {

@@ -249,6 +249,11 @@ def test_cfg4_channel_reference_against_the_oracle(sb, oracle_mod):
     run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], ACT, 2, "add_uniform_sample", ref_over_batch=1, ref_over_tokens=1)
 
 
+def test_cfg4_channel_reference_per_sample_against_the_oracle(sb, oracle_mod):
+    """The same with a vector per sample ([B,d])."""
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], GRAD, 2, "add_uniform_sample", ref_over_tokens=1)
+
+
 def test_cfg4_sliced_wasserstein_units(sb, oracle_mod):
     """4 x 8192 x 8192, 8 directions.  Two samples against the float64 oracle (projections of
     8192 tokens in R^8192 each); and the whole-tensor unit through a property: a tensor made of

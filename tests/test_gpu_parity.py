@@ -913,10 +913,54 @@ def test_streams_in_lockstep_with_a_channel_reference(sb, oracle_mod, name, shap
     gv.close()
 
 
-def test_channel_reference_restrictions_and_state_round_trip(sb):
+@pytest.mark.parametrize("name,shape,steps", [("cfg2", (6, 40, 1024), 50), ("cfg4", (4, 24, 2056), 40),
+                                              ("cfg3", (16, 30, 520), 60), ("cfg2", (1, 37, 264), 40),
+                                              ("cfg4", (39, 8, 512), 30), ("cfg2", (5, 200, 264), 30)],
+                         ids=["cfg2_B6", "cfg4_B4", "cfg3_B16", "cfg2_B1", "cfg4_B39", "cfg2_T200"])
+def test_streams_in_lockstep_with_a_channel_reference_per_sample(sb, oracle_mod, name, shape, steps):
+    """[B,d]: one vector per sample (ref_over_tokens = 1 alone).  B = 39 with T = 8 gives CTAs two
+    or three rows each and samples that several CTAs share; T = 200 gives CTAs that straddle two
+    samples.  (Samples are kept at 4096 elements or more: with fewer, a single sign decided by
+    rounding where the reference is all but zero moves the sign-flip ratio by more than 1e-3.)"""
+    w = synth.scaled(synth.WORKLOADS[name], name + "_channel_ps", *shape, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w, ref_over_tokens=1)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, steps)
+    assert rec["corrupted"] >= 3
+    compare_state(gv, ov, params)
+    for kind in (ACT, GRAD):
+        compare_thresholds(gv, ov, kind)
+        st = gv.sentinel_get_stats(kind).cpu().numpy()
+        x, _ = synth.microbatch(w, 0, kind, steps - 1, "cuda")
+        assert_stats_close(st, ov.last_stats(kind), max(float(x.float().std()), 1e-30),
+                           max(float(np.abs(ov.last_stats(kind)[0, 4])) ** 0.5, 1e-30), "stats kind %d" % kind)
+    assert rec["near"] <= 2 and rec["k_events"] <= 4, rec
+    x, _ = synth.microbatch(w, 0, GRAD, 0, "cuda")
+    loud = (x.float() * 64).to(torch.bfloat16)
+    gv.verify(loud, GRAD)
+    ov.verify(synth.bits(loud), GRAD)
+    out = loud.clone()
+    gv.sentinel_replace_if_flagged(out, GRAD, 0)
+    want, did = ov.replace_if_flagged(synth.bits(loud), GRAD)
+    torch.cuda.synchronize()
+    assert did
+    got = synth.bits(out)
+    gv_, rv_ = oracle_mod.bf16_to_f64(got), oracle_mod.bf16_to_f64(want)
+    assert np.mean(got != want) <= 1e-3 and np.all(np.abs(gv_ - rv_) <= 2.0 ** -7 * np.abs(rv_) + 1e-6 * float(np.std(rv_)))
+    blob = bytes(gv.sentinel_export_state())                                       # round trip, another shape refused
+    other = sb.Verifier(w.B, w.T, w.d, ref_over_tokens=1)
+    other.sentinel_import_state(blob)
+    assert bytes(other.sentinel_export_state()) == blob
     with pytest.raises(sb.SentinelError) as e:
-        sb.Verifier(2, 8, 64, ref_over_tokens=1)                                  # [d] means over the samples too
-    assert e.value.code == sb.ERR_UNSUPPORTED
+        sb.Verifier(w.B, w.T, w.d, ref_over_batch=1, ref_over_tokens=1).sentinel_import_state(blob)
+    assert e.value.code == sb.ERR_STATE_SIZE
+    gv.close(); other.close()
+
+
+def test_channel_reference_restrictions_and_state_round_trip(sb):
+    for kw in ({"n_workers": 2}, {"ema_bf16": 1}):
+        with pytest.raises(sb.SentinelError) as e:
+            sb.Verifier(2, 8, 64, ref_over_tokens=1, **kw)
+        assert e.value.code == sb.ERR_UNSUPPORTED
     for kw in ({"n_workers": 2}, {"ema_bf16": 1}):
         with pytest.raises(sb.SentinelError) as e:
             sb.Verifier(2, 8, 64, ref_over_batch=1, ref_over_tokens=1, **kw)
