@@ -257,7 +257,8 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
   if (h->chan_ref) {                               // x alone streams; the reference moves in a second launch
     const size_t col_smem = (size_t)kWarps * kStripe * sizeof(float);      // the warps' column sums
     if (lc.dynamicSmemBytes < col_smem) lc.dynamicSmemBytes = col_smem;
-    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel, a));
+    if (h->chan_per_sample) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel<true>, a));
+    else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel<false>, a));
     cudaLaunchConfig_t lm = lc;
     lm.gridDim = dim3((unsigned)((h->cfg.d + kChannelMeanCols - 1) / kChannelMeanCols), h->chan_per_sample ? (unsigned)h->cfg.B : 1u);
     lm.blockDim = dim3(kChannelMeanCols * kChannelMeanGroups);
@@ -601,7 +602,8 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
   }
   std::string oerr;

@@ -1147,20 +1147,21 @@ __host__ __device__ inline int channel_slots(int d) { return channel_stripes(d) 
 // sign(x) != sign(m) iff x, with its sign bit flipped where m is negative, is <= +0 as an integer
 // (a negative number, -0, or +0: x and m differ in sign, or x is zero against a non-zero m).
 template <bool kZeroInM>
-__device__ __forceinline__ void channel_slot(const StreamArgs &a, long long first, long long rb, int phases,
-                                             size_t lane_off, const bool (&ok)[kUnroll],
+__device__ __forceinline__ void channel_slot(const uint16_t *xseg, int d, int first, int rb, int phases,
+                                             const bool (&ok)[kUnroll],
                                              const float4 *const (&mp)[kUnroll], float4 *col, unsigned x0pair,
-                                             float x0f, ThreadAcc &t, long long &n_rows) {
+                                             float x0f, ThreadAcc &t, int &n_rows) {
+  // (xseg: this lane's first chunk in the first row of the segment; rows are counted from there)
   // Two rows per trip; the next trip's rows are requested before this trip's arithmetic.  The
   // reference (2 KB per warp, the same for every row) is fetched again each trip through L1
   // rather than held in registers, which the second set of x would not leave room for.
   uint4 cur[2][kUnroll], nxt[2][kUnroll];
-  auto fetch = [&](uint4 (&dst)[2][kUnroll], long long row) {
+  auto fetch = [&](uint4 (&dst)[2][kUnroll], int row) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const long long r = row + (long long)h * phases;
+      const int r = row + h * phases;
       if (r < rb) {
-        const uint16_t *xr = a.x + (size_t)r * a.d + lane_off;
+        const uint16_t *xr = xseg + (size_t)r * d;
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u)
           if (ok[u]) dst[h][u] = ld_x128(xr + (size_t)u * 256);
@@ -1168,7 +1169,7 @@ __device__ __forceinline__ void channel_slot(const StreamArgs &a, long long firs
     }
   };
   if (first < rb) fetch(cur, first);
-  for (long long row = first; row < rb; row += 2 * phases) {
+  for (int row = first; row < rb; row += 2 * phases) {
     if (row + 2 * phases < rb) fetch(nxt, row + 2 * phases);
     const bool second = row + phases < rb;
     float g_sxx = 0.f, g_ab = 0.f;
@@ -1225,7 +1226,6 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
   const unsigned x0 = a.x[(size_t)b * a.T * (size_t)a.d];
   const unsigned x0pair = x0 | (x0 << 16);
   const float x0f = __uint_as_float(x0 << 16);
-  if (a.ref_per_sample) m_in += (size_t)b * a.d;           // sample b's own vector
   const unsigned m0bits = __float_as_uint(__ldg(m_in));
   const float m0 = __uint_as_float(m0bits);
 
@@ -1259,12 +1259,12 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
         }
       }
     }
-    long long n_rows = 0;
-    const size_t lane_off = (size_t)(stripe * 32 * kUnroll + lane) * 8;
+    int n_rows = 0;
+    const uint16_t *xseg = a.x + (size_t)ra * a.d + (size_t)(stripe * 32 * kUnroll + lane) * 8;
     if (__any_sync(0xffffffffu, zero_in_m))
-      channel_slot<true>(a, ra + phase, rb, phases, lane_off, ok, mp, col, x0pair, x0f, t, n_rows);
+      channel_slot<true>(xseg, a.d, phase, (int)(rb - ra), phases, ok, mp, col, x0pair, x0f, t, n_rows);
     else
-      channel_slot<false>(a, ra + phase, rb, phases, lane_off, ok, mp, col, x0pair, x0f, t, n_rows);
+      channel_slot<false>(xseg, a.d, phase, (int)(rb - ra), phases, ok, mp, col, x0pair, x0f, t, n_rows);
 
     // what is linear in x, from the column sums; the reference's own sums: its columns once per row
     float4 *dst = reinterpret_cast<float4 *>(col_seg + (size_t)sl * kStripe) + lane * 2;
@@ -1294,6 +1294,9 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
   reduce_to_slot(t, b, x0, m0bits, s_part, slot);
 }
 
+// (kPerSample: a vector per sample, [B,d], instead of one, [d]; a kernel of its own so that the
+// code of either form does not depend on the other's addressing)
+template <bool kPerSample>
 __global__ void __launch_bounds__(kThreads)
 channel_ref_kernel(const StreamArgs a) {
   __shared__ unsigned long long s_part[kWarps][kSlotWords];
@@ -1323,7 +1326,8 @@ channel_ref_kernel(const StreamArgs a) {
         const int b = (int)(ra / a.T);
         const long long sample_end = (long long)(b + 1) * a.T;
         const long long rb = sample_end < R1 ? sample_end : R1;
-        channel_segment(a, b, ra, rb, m_in, col_seg, reinterpret_cast<float *>(s_dyn), s_part, slot);
+        channel_segment(a, b, ra, rb, kPerSample ? m_in + (size_t)b * a.d : m_in, col_seg,
+                        reinterpret_cast<float *>(s_dyn), s_part, slot);
         ra = rb;
       } else {                                    // no rows: nothing to add
         for (size_t i = threadIdx.x; i < seg_floats; i += kThreads) col_seg[i] = 0.f;
@@ -1371,18 +1375,36 @@ channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const f
   const int lane_c = threadIdx.x % kChannelMeanCols, group = threadIdx.x / kChannelMeanCols;
   const int c = blockIdx.x * kChannelMeanCols + lane_c;
   const int stripes = channel_stripes(d), phases = channel_phases(d), n_slots = stripes * phases;
-  const int n_blocks = G * kSegsPerCta * phases;           // blocks of partial sums that hold column c
   const long long R = (long long)B * T;
+  // (CTA, segment) pairs whose blocks of partial sums can belong to this vector: all of them, or
+  // with a vector per sample the CTAs whose rows [R*cta/G, R*(cta+1)/G) can touch the sample's
+  // (a superset; the test in the loop decides)
+  int cs_lo = 0, cs_hi = G * kSegsPerCta;
+  if (per_sample) {
+    long long lo = ((long long)sample * T * G) / R - 1, hi = ((long long)(sample + 1) * T * G + R - 1) / R + 1;
+    if (lo < 0) lo = 0;
+    if (hi > G) hi = G;
+    cs_lo = (int)lo * kSegsPerCta;
+    cs_hi = (int)hi * kSegsPerCta;
+  }
   double sum = 0.;
   if (c < d) {
     const int stripe = c / kStripe, within = c - stripe * kStripe;
+    const float *src = col_part + (size_t)stripe * kStripe + within;
+    if (!per_sample) {
 #pragma unroll 8
-    for (int i = group; i < n_blocks; i += kChannelMeanGroups) {
-      const int cs = i / phases, p = i - cs * phases;      // (CTA, segment) pair and row phase
-      // CTA cs/2 owns rows [R*cta/G, R*(cta+1)/G): its first segment lies in the sample of its first
-      // row, its second (if any: else blocks of zeros) in the next one
-      if (per_sample && (int)(((R * (cs >> 1)) / G) / T) + (cs & 1) != sample) continue;
-      sum += (double)__ldcg(col_part + ((size_t)cs * n_slots + (size_t)p * stripes + stripe) * kStripe + within);
+      for (int i = group; i < cs_hi * phases; i += kChannelMeanGroups) {
+        const int cs = i / phases, p = i - cs * phases;    // (CTA, segment) pair and row phase
+        sum += (double)__ldcg(src + ((size_t)cs * n_slots + (size_t)p * stripes) * kStripe);
+      }
+    } else {
+      for (int i = cs_lo * phases + group; i < cs_hi * phases; i += kChannelMeanGroups) {
+        const int cs = i / phases, p = i - cs * phases;
+        // a CTA's first segment lies in the sample of its first row, its second (if any: else blocks
+        // of zeros) in the next one
+        if ((int)(((R * (cs >> 1)) / G) / T) + (cs & 1) != sample) continue;
+        sum += (double)__ldcg(src + ((size_t)cs * n_slots + (size_t)p * stripes) * kStripe);
+      }
     }
   }
   s_sum[group][lane_c] = sum;
