@@ -368,6 +368,19 @@ def run_ours(args, rank, world, local_rank):
                    "achieved_gbs": round(2 * N / (qms * 1e-3) / 1e9, 1),
                    "tensors_per_s": round(1e3 / qms, 1), "kernels": "channel_ref_kernel + channel_mean_kernel"}
         vcr.sentinel_destroy()
+        # the same with a vector per sample ([B,d])
+        vps = binding.Verifier(w.B, w.T, w.d, device=local_rank, ref_over_tokens=1)
+        for i in range(6):
+            vps.sentinel_update_reference(xs[0][ACT][i % nd], ACT, cs_, main)
+        vps.sentinel_verify(xs[0][ACT][6 % nd], ACT, cs_, cf_, main)
+        torch.cuda.synchronize()
+        q0.record(main)
+        for i in range(20):
+            vps.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, cs_, cf_, main)
+        q1.record(main)
+        torch.cuda.synchronize()
+        channel["ms_per_step_vector_per_sample"] = round(q0.elapsed_time(q1) / 20, 4)
+        vps.sentinel_destroy()
 
     # extra figure, outside the timed region: the strided (compressed-signal) layout, rows d+1 apart
     strided = None
