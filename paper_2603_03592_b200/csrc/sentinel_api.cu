@@ -129,12 +129,12 @@ Alg5Params alg5_of(const sentinel_config &c, int kind) {
 }
 
 // How many CTAs stream: every resident slot but the one of CTA 0, never more than there are
-// rows.  A CTA's rows may straddle one sample boundary at most, which needs G >= B.
-int streaming_ctas(int device, int B, int T, std::string *err) {
-  int sms = 0, occ = 0;
+// rows.  A CTA's rows may straddle one sample boundary at most, which needs G >= B.  `occ` is the
+// number of CTAs of the kernel(s) to be launched that an SM keeps resident, as resident_ctas()
+// found it for their CTA size and shared memory.
+int streaming_ctas(int device, int occ, int B, int T, std::string *err) {
+  int sms = 0;
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-  if (e == cudaSuccess)
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, stream_kernel_t<false, false>, kThreads, 0);
   if (e != cudaSuccess || sms < 1 || occ < 1) {
     if (err) *err = std::string("occupancy query failed: ") + cudaGetErrorString(e);
     return -1;
@@ -147,6 +147,29 @@ int streaming_ctas(int device, int B, int T, std::string *err) {
     return -1;
   }
   return (int)G;
+}
+
+// Resident CTAs per SM of one kernel as it will be launched (its CTA size, its dynamic shared
+// memory); -1 on failure.  `lowest` carries the minimum over several kernels.
+template <typename K>
+void resident_ctas(K kernel, int threads, size_t smem, int *lowest, cudaError_t *status) {
+  int occ = 0;
+  if (*status == cudaSuccess && smem > 48u * 1024u)
+    *status = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (*status == cudaSuccess) *status = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, threads, smem);
+  if (*status == cudaSuccess && (*lowest < 0 || occ < *lowest)) *lowest = occ;
+}
+
+// the stateless distance: stream_kernel_t<false, false> with no dynamic shared memory
+int distance_ctas(int device, int B, int T, std::string *err) {
+  int occ = -1;
+  cudaError_t e = cudaSuccess;
+  resident_ctas(stream_kernel_t<false, false>, kThreads, 0, &occ, &e);
+  if (e != cudaSuccess) {
+    if (err) *err = std::string("occupancy query failed: ") + cudaGetErrorString(e);
+    return -1;
+  }
+  return streaming_ctas(device, occ, B, T, err);
 }
 
 // The stateless entry points take their scratch from the device's default memory pool.  By
@@ -274,7 +297,13 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
     ra.s = a;
     for (int b = 0; b < h->cfg.B; ++b) ra.xs[b] = a.x + (size_t)b * h->Ns;
     ra.partials = h->partials;
-    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, shared_ref_kernel, ra));
+    if (h->cfg.B <= kFewSets) {
+      lc.blockDim = dim3(kFewThreads);
+      lc.dynamicSmemBytes = std::max(lc.dynamicSmemBytes, few_smem_bytes());   // the threads' fp64 sums
+      SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, shared_ref_kernel<true>, ra));
+    } else {
+      SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, shared_ref_kernel<false>, ra));
+    }
     return SENTINEL_OK;
   }
   // strided rows: the funnel-shift variant of the vector path when the width allows it, else scalar
@@ -600,15 +629,48 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(ae)); }
   }
   std::string oerr;
-  // (with a [T,d] reference the CTAs share out the T token rows, each with every sample's slice)
-  h->G = h->shared_ref ? streaming_ctas(cfg->device, 1, cfg->T, &oerr) : streaming_ctas(cfg->device, cfg->B, cfg->T, &oerr);
+  {
+    // Every kernel this handle can launch, with the CTA size and the most dynamic shared memory it
+    // can be launched with (the windows' working copies for four metrics, if directions may still
+    // be set): G follows the one that keeps the fewest CTAs resident.
+    size_t smem = h->refresh_smem;
+    const size_t smem4 = refresh_smem_doubles(h->cap0, h->cap1, h->units0, h->units1, kNumMetrics) * sizeof(double);
+    if (smem4 <= 200u * 1024u) smem = smem4;
+    int occ = -1;
+    cudaError_t oe = cudaSuccess;
+    if (h->chan_ref) {
+      const size_t sm = std::max(smem, (size_t)kWarps * kStripe * sizeof(float));
+      if (h->chan_per_sample) resident_ctas(channel_ref_kernel<true>, kThreads, sm, &occ, &oe);
+      else resident_ctas(channel_ref_kernel<false>, kThreads, sm, &occ, &oe);
+    } else if (h->shared_ref) {
+      if (cfg->B <= kFewSets) resident_ctas(shared_ref_kernel<true>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
+      else resident_ctas(shared_ref_kernel<false>, kThreads, smem, &occ, &oe);
+    } else {
+      if (h->R > 1 && h->R <= kFewSets) resident_ctas(replica_kernel<true>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
+      else if (h->R > 1) resident_ctas(replica_kernel<false>, kThreads, smem, &occ, &oe);
+      if (h->bf16) {
+        resident_ctas(stream_kernel_t<false, true>, kThreads, smem, &occ, &oe);
+        resident_ctas(stream_kernel_t<true, true>, kThreads, smem, &occ, &oe);
+        resident_ctas(stream_kernel_t<false, true, true>, kThreads, smem, &occ, &oe);
+      } else {
+        resident_ctas(stream_kernel_t<false, false>, kThreads, smem, &occ, &oe);
+        resident_ctas(stream_kernel_t<true, false>, kThreads, smem, &occ, &oe);
+        resident_ctas(stream_kernel_t<false, false, true>, kThreads, smem, &occ, &oe);
+      }
+    }
+    if (oe != cudaSuccess) { delete h; return fail(nullptr, SENTINEL_ERR_CUDA, "occupancy query failed: %s", cudaGetErrorString(oe)); }
+    // (with a [T,d] reference the CTAs share out the T token rows, each with every sample's slice)
+    h->G = h->shared_ref ? streaming_ctas(cfg->device, occ, 1, cfg->T, &oerr) : streaming_ctas(cfg->device, occ, cfg->B, cfg->T, &oerr);
+  }
   if (h->G < 1) { delete h; return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str()); }
 
   cudaError_t e = cudaSuccess;
@@ -738,7 +800,7 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
 
   std::string oerr;
-  const int G = streaming_ctas(device, B, T, &oerr);
+  const int G = distance_ctas(device, B, T, &oerr);
   if (G < 1) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str());
   // scratch: two partial slots per streaming CTA, then the ticket word
   const size_t slot_bytes = (size_t)G * kSegsPerCta * kSlotWords * sizeof(unsigned long long);
@@ -818,15 +880,17 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigne
   {   // every worker against the same m_{t-1}, in one launch
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)(h->G + 1));
-    lc.blockDim = dim3(kThreads);
-    lc.dynamicSmemBytes = h->refresh_smem;
+    const bool few = h->R <= kFewSets;              // every worker's sums in registers
+    lc.blockDim = dim3(few ? kFewThreads : kThreads);
+    lc.dynamicSmemBytes = few ? std::max(h->refresh_smem, few_smem_bytes()) : h->refresh_smem;
     lc.stream = s;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = &attr;
     lc.numAttrs = 1;
-    SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel, ra));
+    if (few) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<true>, ra));
+    else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<false>, ra));
   }
   int sms = 0;
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
@@ -1277,7 +1341,7 @@ int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
 
   std::string oerr;
-  const int G = streaming_ctas(device, B, T, &oerr);
+  const int G = distance_ctas(device, B, T, &oerr);
   if (G < 1) return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "%s", oerr.c_str());
   const size_t slot_bytes = (size_t)G * kSegsPerCta * kSlotWords * sizeof(unsigned long long);
   if (slot_bytes + kNoAllocTicketBytes > (size_t)SENTINEL_NOALLOC_SCRATCH_BYTES)

@@ -13,6 +13,8 @@
 #include <math_constants.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace sentinel {
 
 constexpr int kNumMetrics = 4;          // room for L1, z-scored L2, sign flips and the sliced Wasserstein
@@ -567,8 +569,11 @@ __host__ __device__ inline size_t sorted_offset(int L, int i, int cap0, int cap1
 
 // One thread group per (level, metric) window: three warps each with three metrics in use, two
 // with four.
-__host__ __device__ inline int refresh_group_threads(int n_metrics) { return (kThreads / (2 * n_metrics)) & ~31; }
-static_assert(2 * kNumMetrics * 64 <= kThreads, "one thread group per window");
+__host__ __device__ inline int refresh_group_threads(int n_metrics, int cta_threads) {
+  return (cta_threads / (2 * n_metrics)) & ~31;
+}
+constexpr int kMinThreads = 2 * kNumMetrics * 64;   // one thread group of two warps per window at least
+static_assert(kMinThreads <= kThreads, "one thread group per window");
 
 __device__ __forceinline__ void group_barrier(int group, int group_threads) {   // named barrier 1 + group
   asm volatile("bar.sync %0, %1;" :: "r"(group + 1), "r"(group_threads) : "memory");
@@ -623,7 +628,7 @@ __device__ __forceinline__ int warp_count_outside(const double *s, int n, double
 // the windows are handled side by side, each by a group of warps with its own named barrier.
 __device__ void refresh_thresholds(KindState *ks, const double *hist, double *sorted, int cap0, int cap1,
                                    int units0, int units1, int n_metrics, const Alg5Params &a5, double *s_dyn) {
-  const int group_threads = refresh_group_threads(n_metrics);
+  const int group_threads = refresh_group_threads(n_metrics, (int)blockDim.x);   // any CTA of kMinThreads or more
   const int group = threadIdx.x / group_threads;
   const int gt = threadIdx.x - group * group_threads;
   if (group < 2 * n_metrics) {
@@ -771,21 +776,23 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
   __shared__ __align__(8) HandleState s_hs;
   static_assert(sizeof(HandleState) % 8 == 0, "copied as 64-bit words");
   constexpr int kStateWords = (int)(sizeof(HandleState) / 8);
-  constexpr int kDecider = kThreads - 1;         // the thread that keeps the counters
+  static_assert(kStateWords <= kMinThreads, "one thread per word of the state");
+  const int n_threads = (int)blockDim.x, n_warps = n_threads >> 5;   // (kernels of several CTA sizes end here)
+  const int kDecider = n_threads - 1;            // the thread that keeps the counters
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = a.B, rows = B + 1;
   const size_t Ns = (size_t)a.T * a.d;
 
   if (tid == 0) { s_severe = 0; s_no_thr = 0; s_status = 0u; }
-  if (a.hs && tid >= kThreads - kStateWords) {      // the last warps: the first ones gather sums
-    const int w = tid - (kThreads - kStateWords);
+  if (a.hs && tid >= n_threads - kStateWords) {     // the last warps: the first ones gather sums
+    const int w = tid - (n_threads - kStateWords);
     reinterpret_cast<unsigned long long *>(&s_hs)[w] =
         __ldcg(reinterpret_cast<const unsigned long long *>(a.hs) + w);
   }
 
   // per-sample sums over the slots tagged with that sample, in CTA order
-  for (int b = warp; b < B; b += kWarps) {
+  for (int b = warp; b < B; b += n_warps) {
     double v[6] = {0., 0., 0., 0., 0., 0.};
     unsigned long long fl = 0ull, bits = 0ull, first = 0ull;
     // streaming CTAs whose rows can touch sample b (a superset; the tag decides)
@@ -1500,6 +1507,271 @@ __device__ __forceinline__ void replica_tile(const uint4 (&cur)[kUnroll], const 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Up to kFewSets tensors against the tile of m with every sum carried in registers.
+//
+// The general path below reduces each tile's sums across the warp and folds them into shared
+// fp64 accumulators, once per tensor and tile: a third of its instructions.  With few tensors a
+// thread can keep its own fp32 sums per tensor over kFoldTiles tiles (64 elements per tensor: the
+// rounding of so short a run stays near 1e-7 of the sum) and then adds them to its own fp64
+// accumulators, which live in shared memory, one column per thread; threads are added up once,
+// when the segment is done, in a fixed order.  Non-finite elements are found through the sum of
+// |x - m|: it is not a finite number as soon as one x is not, so the exact test of the exponent
+// bits runs only for a tile after which that sum is not finite.
+constexpr int kFewSets = 4;
+constexpr int kFoldTiles = 4;
+constexpr int kFewThreads = 512;                  // threads per CTA of the kernels that take this path
+constexpr int kFewWarps = kFewThreads / 32;
+
+// A CTA's rows lie in one sample or straddle one boundary: two segments, each with its own shift
+// values, sums and slot.  A warp's tiles come in ascending row order, so it crosses over once.
+struct FewShared {
+  const uint16_t *ptr[kFewSets];                  // the tensors that stream, in order
+  int widx[kFewSets];                             // which worker / sample each of them is (its slot block)
+  unsigned x0[kSegsPerCta][kFewSets];             // the sample's first element, per segment and tensor
+  unsigned m0bits[kSegsPerCta];                   // the sample's first element of the reference
+  double red[kSegsPerCta][kFewSets * 4 + 2];      // the CTA's sums
+  unsigned flips[kSegsPerCta][kFewWarps][kFewSets];
+  unsigned bits[kSegsPerCta][kFewWarps][kFewSets];   // kBitNonfinite | kBitXVaries
+  unsigned m_varies[kSegsPerCta][kFewWarps];
+};
+// dynamic shared memory of such a CTA: per segment and thread a column of fp64 sums
+__host__ __device__ inline size_t few_smem_bytes() {
+  return (size_t)kSegsPerCta * (kFewSets * 4 + 2) * kFewThreads * sizeof(double);
+}
+
+template <bool kZeroInM>
+__device__ __forceinline__ void few_tile(const uint4 (&cur)[kUnroll], const F8 (&mv)[kUnroll], const bool (&ok)[kUnroll],
+                                         float x0f, float m0, unsigned x0pair, float (&sum)[kUnroll][8], float &sx,
+                                         float &sxx, float &sxm, float &ab, unsigned &flips, unsigned &x_diff) {
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    if (!ok[u]) continue;
+    const unsigned w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      x_diff |= w4[q] ^ x0pair;
+#pragma unroll
+      for (int hlf = 0; hlf < 2; ++hlf) {
+        const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
+        const float mf = mv[u].v[2 * q + hlf];
+        const float xs = xf - x0f, ms = mf - m0;
+        sx += xs;
+        sxx = fmaf(xs, xs, sxx);
+        sxm = fmaf(xs, ms, sxm);
+        ab += fabsf(xf - mf);
+        const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
+        if (kZeroInM) flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
+        else flips += ((int)xt <= 0) ? 1u : 0u;
+        sum[u][2 * q + hlf] += xf;
+      }
+    }
+  }
+}
+
+// Rows [r0, r1) of the flat [rows, d] view, of which [r0, cut) lie in sample b0 and [cut, r1) in
+// sample b0 + 1 (cut = r1: one segment).
+template <int NR>
+__device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int b0, long long r0, long long cut,
+                         long long r1, const float *m_in, float *m_out, int c, FewShared &fs, double *s_acc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunks = a.d >> 3;                               // d is a multiple of 8 here
+  const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
+  const int n_tiles = (int)(r1 - r0) * tiles_per_row;
+  const int cut_rr = (int)(cut - r0);                        // first row (from r0) of the second segment
+  const float beta = a.beta, wgt = a.one_minus_beta / (float)NR;
+  constexpr int kSums = NR * 4 + 2;                          // per tensor 4 sums, then the reference's 2
+
+  for (int q = tid; q < kSegsPerCta * kSums * kFewThreads; q += kFewThreads) s_acc[q] = 0.;
+  for (int q = tid; q < kSegsPerCta * kFewWarps * kFewSets; q += kFewThreads) {
+    (&fs.flips[0][0][0])[q] = 0u;
+    (&fs.bits[0][0][0])[q] = 0u;
+  }
+  if (tid < kSegsPerCta * kFewWarps) (&fs.m_varies[0][0])[tid] = 0u;
+  __syncthreads();                                           // fs.ptr is in place
+  if (tid < kSegsPerCta * NR) {
+    const int sg = tid / NR, r = tid - sg * NR;
+    const size_t sample_off = (size_t)(b0 + sg) * a.T * a.d;
+    if (sg == 0 || cut < r1) fs.x0[sg][r] = fs.ptr[r][sample_off];
+  } else if (tid >= 32 && tid < 32 + kSegsPerCta) {
+    const int sg = tid - 32;
+    if (sg == 0 || cut < r1) fs.m0bits[sg] = __float_as_uint(m_in[(size_t)(b0 + sg) * a.T * a.d]);
+  }
+  __syncthreads();
+
+  float sx[NR], sxx[NR], sxm[NR], ab[NR];
+  unsigned fl[NR], xd[NR];
+  unsigned nf_mask = 0u, m_diff = 0u;
+  float g_sm = 0.f, g_smm = 0.f;
+#pragma unroll
+  for (int r = 0; r < NR; ++r) { sx[r] = sxx[r] = sxm[r] = ab[r] = 0.f; fl[r] = xd[r] = 0u; }
+  int sg = 0;                                                // the segment this warp is in
+  double *acc = s_acc + tid;                                 // this thread's column of segment sg
+  auto fold = [&]() {                                        // the short fp32 runs into this thread's fp64 sums
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      acc[(r * 4 + 0) * kFewThreads] += (double)sx[r];
+      acc[(r * 4 + 1) * kFewThreads] += (double)sxx[r];
+      acc[(r * 4 + 2) * kFewThreads] += (double)sxm[r];
+      acc[(r * 4 + 3) * kFewThreads] += (double)ab[r];
+      sx[r] = sxx[r] = sxm[r] = ab[r] = 0.f;
+    }
+    acc[(NR * 4 + 0) * kFewThreads] += (double)g_sm;
+    acc[(NR * 4 + 1) * kFewThreads] += (double)g_smm;
+    g_sm = g_smm = 0.f;
+  };
+  auto leave_segment = [&]() {                               // counts and bits of segment sg, per warp
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      const unsigned wf = __reduce_add_sync(0xffffffffu, fl[r]);
+      const unsigned wx = __reduce_or_sync(0xffffffffu, xd[r]);
+      const unsigned wn = __reduce_or_sync(0xffffffffu, (nf_mask >> r) & 1u);
+      if (lane == 0) {
+        fs.flips[sg][warp][r] = wf;
+        fs.bits[sg][warp][r] = (wn ? (unsigned)kBitNonfinite : 0u) | (wx ? (unsigned)kBitXVaries : 0u);
+      }
+      fl[r] = xd[r] = 0u;
+    }
+    const unsigned wm = __reduce_or_sync(0xffffffffu, m_diff);
+    if (lane == 0) fs.m_varies[sg][warp] = wm;
+    nf_mask = m_diff = 0u;
+  };
+
+  const int step_rr = kFewWarps / tiles_per_row, step_seg = kFewWarps % tiles_per_row;
+  int rr = warp / tiles_per_row, seg = warp % tiles_per_row;
+  int since_fold = 0;
+  unsigned m0bits = fs.m0bits[0];
+  float m0 = __uint_as_float(m0bits);
+  for (int j = warp; j < n_tiles; j += kFewWarps) {
+    if (sg == 0 && rr >= cut_rr) {                           // this warp enters the second segment
+      fold();
+      leave_segment();
+      since_fold = 0;
+      sg = 1;
+      acc += kSums * kFewThreads;
+      m0bits = fs.m0bits[1];
+      m0 = __uint_as_float(m0bits);
+    }
+    const size_t off = (size_t)(r0 + rr) * a.d;
+    const int base = seg * 32 * kUnroll;
+    F8 mv[kUnroll];
+    uint4 xv[kUnroll];
+    bool ok[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int ch = base + u * 32 + lane;
+      ok[u] = ch < chunks;
+      if (ok[u]) {
+        mv[u] = ld_m256(m_in + off + (size_t)ch * 8);
+        xv[u] = ld_x128(fs.ptr[0] + off + (size_t)ch * 8);
+      }
+    }
+    // the reference's own sums, once per tile
+    bool zero_in_m = false;
+    float sum[kUnroll][8];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        sum[u][e] = 0.f;
+        if (ok[u]) {
+          const float ms = mv[u].v[e] - m0;
+          g_sm += ms;
+          g_smm = fmaf(ms, ms, g_smm);
+          m_diff |= __float_as_uint(mv[u].v[e]) ^ m0bits;
+          zero_in_m |= (mv[u].v[e] == 0.f);
+        }
+      }
+    }
+    const bool any_zero = __any_sync(0xffffffffu, zero_in_m);
+
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {                           // the tensors, in order
+      uint4 cur[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) cur[u] = xv[u];
+      if (r + 1 < NR) {                                      // the next tensor's tile, ahead of the arithmetic
+        const uint16_t *xn = fs.ptr[r + 1] + off;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          if (ok[u]) xv[u] = ld_x128(xn + (size_t)(base + u * 32 + lane) * 8);
+      }
+      const unsigned x0 = fs.x0[sg][r], x0pair = x0 | (x0 << 16);
+      const float x0f = __uint_as_float(x0 << 16);
+      if (any_zero) few_tile<true>(cur, mv, ok, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
+      else few_tile<false>(cur, mv, ok, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
+      if (__any_sync(0xffffffffu, !(ab[r] <= 3.4028234664e38f))) {   // not a finite sum: look at the bits
+        unsigned nf = 0u;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          if (ok[u]) nf |= (((cur[u].x & 0x7F807F80u) + 0x00800080u) | ((cur[u].y & 0x7F807F80u) + 0x00800080u) |
+                            ((cur[u].z & 0x7F807F80u) + 0x00800080u) | ((cur[u].w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
+        if (nf) nf_mask |= 1u << r;
+      }
+    }
+    // Eq. 1 with the mean over the tensors
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (!ok[u]) continue;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mv[u].v[e] = fmaf(beta, mv[u].v[e], wgt * sum[u][e]);
+      st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+    }
+    if (++since_fold == kFoldTiles) { fold(); since_fold = 0; }
+    rr += step_rr;
+    seg += step_seg;
+    if (seg >= tiles_per_row) { seg -= tiles_per_row; ++rr; }
+  }
+  fold();
+  leave_segment();
+
+  // threads -> CTA in a fixed order: the fp64 columns one quantity per warp in turn
+  __syncthreads();
+  for (int q = warp; q < kSegsPerCta * kSums; q += kFewWarps) {
+    const int qs = q / kSums, qq = q - qs * kSums;
+    const double *col = s_acc + (size_t)q * kFewThreads;
+    double v = 0.;
+    for (int t = lane; t < kFewThreads; t += 32) v += col[t];
+    v = warp_sum(v);
+    if (lane == 0) fs.red[qs][qq] = v;
+  }
+  __syncthreads();
+  if (tid < kSegsPerCta * NR * kSlotWords) {
+    const int sgm = tid / (NR * kSlotWords), r = (tid / kSlotWords) % NR, w8 = tid % kSlotWords;
+    unsigned long long *slot = partials + (((size_t)fs.widx[r] * a.G + c) * kSegsPerCta + sgm) * kSlotWords;
+    if (sgm == 1 && cut >= r1) {
+      if (w8 == 7) slot[7] = 0ull;                           // no second segment: tag 0, unused
+    } else {
+      const double *red = fs.red[sgm];
+      unsigned long long out;
+      if (w8 < 6) {
+        const double t = (w8 == 0) ? red[r * 4 + 0] : (w8 == 1) ? red[r * 4 + 1] : (w8 == 2) ? red[NR * 4 + 0]
+                       : (w8 == 3) ? red[NR * 4 + 1] : (w8 == 4) ? red[r * 4 + 2] : red[r * 4 + 3];
+        out = (unsigned long long)__double_as_longlong(t);
+      } else if (w8 == 6) {
+        out = 0ull;
+        for (int w = 0; w < kFewWarps; ++w) out += fs.flips[sgm][w][r];
+      } else {
+        out = ((unsigned long long)(b0 + sgm + 1) << kTagShift) | ((unsigned long long)fs.x0[sgm][r] << kX0Shift) |
+              ((unsigned long long)fs.m0bits[sgm] << kM0Shift);
+        for (int w = 0; w < kFewWarps; ++w) out |= fs.bits[sgm][w][r] | (fs.m_varies[sgm][w] ? kBitMVaries : 0ull);
+      }
+      slot[w8] = out;
+    }
+  }
+}
+
+__device__ __forceinline__ void few_dispatch(int n, const StreamArgs &a, unsigned long long *partials, int b0,
+                                             long long r0, long long cut, long long r1, const float *m_in, float *m_out,
+                                             int c, FewShared &fs, double *s_acc) {
+  switch (n) {
+    case 1: few_rows<1>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
+    case 2: few_rows<2>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
+    case 3: few_rows<3>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
+    default: few_rows<4>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
+  }
+}
+
 // (n_sets tensors share the tile of m: the R workers of a stage, or the B samples of one tensor
 // when the reference is a single [T,d] tensor for all of them)
 __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long long row_a, long long row_b,
@@ -1642,11 +1914,14 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
   }
 }
 
-__global__ void __launch_bounds__(kThreads)
+// (kFew: a handle that follows at most kFewSets workers -- their sums stay in registers; a kernel
+// of its own, with its own CTA size, so that neither form pays for the other's registers)
+template <bool kFew>
+__global__ void __launch_bounds__(kFew ? kFewThreads : kThreads)
 replica_kernel(const ReplicaArgs ra) {
-  __shared__ ReplicaShared sh;
+  __shared__ typename std::conditional<kFew, FewShared, ReplicaShared>::type sh;
   __shared__ int s_last;
-  extern __shared__ double s_dyn[];            // the refresh's working copies (CTA 0)
+  extern __shared__ double s_dyn[];            // CTA 0: the refresh's working copies; the others: the threads' fp64 sums
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -1669,17 +1944,29 @@ replica_kernel(const ReplicaArgs ra) {
     const int c = blockIdx.x - 1;
     const long long rows = (long long)a.B * a.T;
     const long long r0 = (rows * c) / a.G, r1 = (rows * (c + 1)) / a.G;
-    long long row = r0;
-    for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
-      if (row < r1) {
-        const int b = (int)(row / a.T);
-        const long long sample_end = (long long)(b + 1) * a.T;
-        const long long row_b = sample_end < r1 ? sample_end : r1;
-        replica_segment(ra, a.R, b, row, row_b, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
-                        streamed, c, sgm, sh);
-        row = row_b;
-      } else if (threadIdx.x < a.R) {
-        ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + sgm) * kSlotWords + 7] = 0ull;   // unused
+    const int n_streamed = __popc(streamed);
+    if constexpr (kFew) {
+      if (threadIdx.x == 0) {                                // the tensors that stream, in worker order
+        int n = 0;
+        for (int r = 0; r < a.R; ++r)
+          if ((streamed >> r) & 1u) { sh.ptr[n] = ra.xs[r]; sh.widx[n] = r; ++n; }
+      }
+    }
+    // segment 0: the CTA's rows up to the end of the sample its first row lies in; segment 1: the
+    // rest, if any
+    const int b0 = (int)(r0 / a.T);
+    const long long cut = ((long long)(b0 + 1) * a.T < r1) ? (long long)(b0 + 1) * a.T : r1;
+    if constexpr (kFew) {
+      few_dispatch(n_streamed, a, ra.partials, b0, r0, cut, r1, static_cast<const float *>(a.ema[act]),
+                   static_cast<float *>(a.ema[act ^ 1]), c, sh, s_dyn);
+    } else {
+      for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
+        const long long row = sgm ? cut : r0, row_b = sgm ? r1 : cut;
+        if (row < row_b)
+          replica_segment(ra, a.R, b0 + sgm, row, row_b, static_cast<const float *>(a.ema[act]),
+                          static_cast<float *>(a.ema[act ^ 1]), streamed, c, sgm, sh);
+        else if (threadIdx.x < a.R)
+          ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + sgm) * kSlotWords + 7] = 0ull;   // unused
       }
     }
   }
@@ -1723,9 +2010,11 @@ replica_kernel(const ReplicaArgs ra) {
 // candidate m' = beta m + (1-beta)/B sum_b x[b] into the spare buffer -- over the T token rows;
 // the last CTA then finalizes as for any single submission (every sample a unit, all or nothing
 // commit).  2 + 8/B bytes per element of x.
-__global__ void __launch_bounds__(kThreads)
+// (kFew: at most kFewSets samples, as for the workers above)
+template <bool kFew>
+__global__ void __launch_bounds__(kFew ? kFewThreads : kThreads)
 shared_ref_kernel(const ReplicaArgs ra) {
-  __shared__ ReplicaShared sh;
+  __shared__ typename std::conditional<kFew, FewShared, ReplicaShared>::type sh;
   __shared__ int s_last;
   extern __shared__ double s_dyn[];
   asm volatile("griddepcontrol.launch_dependents;");
@@ -1741,9 +2030,15 @@ shared_ref_kernel(const ReplicaArgs ra) {
   } else {
     const int c = blockIdx.x - 1;
     const long long r0 = ((long long)a.T * c) / a.G, r1 = ((long long)a.T * (c + 1)) / a.G;   // token rows
-    replica_segment(ra, a.B, 0, r0, r1, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
-                    all, c, 0, sh);
-    if (threadIdx.x < a.B)                       // the second slot of every pair stays unused
+    if constexpr (kFew) {
+      if (threadIdx.x < a.B) { sh.ptr[threadIdx.x] = ra.xs[threadIdx.x]; sh.widx[threadIdx.x] = threadIdx.x; }
+      few_dispatch(a.B, a, ra.partials, 0, r0, r1, r1, static_cast<const float *>(a.ema[act]),
+                   static_cast<float *>(a.ema[act ^ 1]), c, sh, s_dyn);
+    } else {
+      replica_segment(ra, a.B, 0, r0, r1, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
+                      all, c, 0, sh);
+    }
+    if (!kFew && threadIdx.x < a.B)              // the second slot of every pair stays unused
       ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + 1) * kSlotWords + 7] = 0ull;
   }
 
