@@ -1508,20 +1508,34 @@ __device__ __forceinline__ void replica_tile(const uint4 (&cur)[kUnroll], const 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Up to kFewSets tensors against the tile of m with every sum carried in registers.
+// Up to kFewSets tensors against the tile of m: sums in registers, tiles staged by bulk copies.
 //
 // The general path below reduces each tile's sums across the warp and folds them into shared
 // fp64 accumulators, once per tensor and tile: a third of its instructions.  With few tensors a
-// thread can keep its own fp32 sums per tensor over kFoldTiles tiles (64 elements per tensor: the
-// rounding of so short a run stays near 1e-7 of the sum) and then adds them to its own fp64
-// accumulators, which live in shared memory, one column per thread; threads are added up once,
-// when the segment is done, in a fixed order.  Non-finite elements are found through the sum of
-// |x - m|: it is not a finite number as soon as one x is not, so the exact test of the exponent
-// bits runs only for a tile after which that sum is not finite.
+// thread keeps its own fp32 sums per tensor over kFoldTiles tiles (128 elements per tensor: the
+// rounding of so short a run stays below 1e-6 of the sum, and the runs are many), after which
+// the warp adds them up and folds them into its fp64 accumulators in shared memory; the warps are
+// added up once, when the CTA's rows are done, in a fixed order.  Non-finite elements are found
+// through the sum of |x - m|: it is not a finite number as soon as one x is not, so the exact
+// test of the exponent bits runs only for a tile after which that sum is not finite.
+//
+// Each warp owns a two-stage ring in shared memory.  A stage holds one warp tile of the
+// reference (2 KB) and the same tile of every tensor (1 KB each); one lane fills it with bulk
+// asynchronous copies (cp.async.bulk, completion counted in bytes on the stage's mbarrier) two
+// tiles ahead of the arithmetic, so that a tile's worth of bytes per warp is in flight the
+// whole time without a register being held for it.  The warp that waits on a stage is the one
+// that filled it; a wait that does not end (it always should) gives up after kStageWaitNs,
+// records kErrStagingTimeout in the handle and skips the warp's remaining tiles.
 constexpr int kFewSets = 4;
-constexpr int kFoldTiles = 4;
+constexpr int kFoldTiles = 8;
 constexpr int kFewThreads = 512;                  // threads per CTA of the kernels that take this path
 constexpr int kFewWarps = kFewThreads / 32;
+constexpr int kStageDepth = 2;
+constexpr int kTileBytesM = 32 * kUnroll * 8 * 4; // a warp tile of the reference: 2048 bytes
+constexpr int kTileBytesX = 32 * kUnroll * 8 * 2; // and of a bf16 tensor: 1024 bytes
+constexpr int kStageBytes = kTileBytesM + kFewSets * kTileBytesX;
+constexpr unsigned long long kStageWaitNs = 2000000000ull;
+constexpr int kErrStagingTimeout = 1;             // HandleState.error: a staged copy did not arrive
 
 // A CTA's rows lie in one sample or straddle one boundary: two segments, each with its own shift
 // values, sums and slot.  A warp's tiles come in ascending row order, so it crosses over once.
@@ -1530,65 +1544,106 @@ struct FewShared {
   int widx[kFewSets];                             // which worker / sample each of them is (its slot block)
   unsigned x0[kSegsPerCta][kFewSets];             // the sample's first element, per segment and tensor
   unsigned m0bits[kSegsPerCta];                   // the sample's first element of the reference
-  double red[kSegsPerCta][kFewSets * 4 + 2];      // the CTA's sums
   unsigned flips[kSegsPerCta][kFewWarps][kFewSets];
   unsigned bits[kSegsPerCta][kFewWarps][kFewSets];   // kBitNonfinite | kBitXVaries
   unsigned m_varies[kSegsPerCta][kFewWarps];
+  int timed_out;
 };
-// dynamic shared memory of such a CTA: per segment and thread a column of fp64 sums
-__host__ __device__ inline size_t few_smem_bytes() {
-  return (size_t)kSegsPerCta * (kFewSets * 4 + 2) * kFewThreads * sizeof(double);
+struct __align__(128) FewWarp {                   // a warp's part of the dynamic shared memory
+  unsigned char stage[kStageDepth][kStageBytes];
+  double acc[kSegsPerCta][kFewSets * 4 + 2];      // per tensor sums of (x-x0), (x-x0)^2, (x-x0)(m-m0), |x-m|; then of (m-m0), (m-m0)^2
+  unsigned long long bar[kStageDepth];
+};
+__host__ __device__ inline size_t few_smem_bytes() { return (size_t)kFewWarps * sizeof(FewWarp); }
+
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned arrivals) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+// global -> this CTA's shared memory, 16-byte aligned on both sides, a multiple of 16 bytes
+__device__ __forceinline__ void bulk_copy_in(unsigned dst, const void *src, unsigned bytes, unsigned bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned done;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done != 0u;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase `parity` of a stage's barrier; false if it did not complete in kStageWaitNs.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > kStageWaitNs) return false;
+  }
 }
 
+// one tensor's 8-element chunk against the chunk of m (kZeroInM = false: no exact zero in the
+// warp's tile of m, see replica_tile)
 template <bool kZeroInM>
-__device__ __forceinline__ void few_tile(const uint4 (&cur)[kUnroll], const F8 (&mv)[kUnroll], const bool (&ok)[kUnroll],
-                                         float x0f, float m0, unsigned x0pair, float (&sum)[kUnroll][8], float &sx,
-                                         float &sxx, float &sxm, float &ab, unsigned &flips, unsigned &x_diff) {
+__device__ __forceinline__ void few_chunk(const uint4 &cur, const F8 &mv, float x0f, float m0, unsigned x0pair,
+                                          float (&sum)[8], float &sx, float &sxx, float &sxm, float &ab,
+                                          unsigned &flips, unsigned &x_diff) {
+  const unsigned w4[4] = {cur.x, cur.y, cur.z, cur.w};
 #pragma unroll
-  for (int u = 0; u < kUnroll; ++u) {
-    if (!ok[u]) continue;
-    const unsigned w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
+  for (int q = 0; q < 4; ++q) {
+    x_diff |= w4[q] ^ x0pair;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      x_diff |= w4[q] ^ x0pair;
-#pragma unroll
-      for (int hlf = 0; hlf < 2; ++hlf) {
-        const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
-        const float mf = mv[u].v[2 * q + hlf];
-        const float xs = xf - x0f, ms = mf - m0;
-        sx += xs;
-        sxx = fmaf(xs, xs, sxx);
-        sxm = fmaf(xs, ms, sxm);
-        ab += fabsf(xf - mf);
-        const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
-        if (kZeroInM) flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
-        else flips += ((int)xt <= 0) ? 1u : 0u;
-        sum[u][2 * q + hlf] += xf;
-      }
+    for (int hlf = 0; hlf < 2; ++hlf) {
+      const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
+      const float mf = mv.v[2 * q + hlf];
+      const float xs = xf - x0f, ms = mf - m0;
+      sx += xs;
+      sxx = fmaf(xs, xs, sxx);
+      sxm = fmaf(xs, ms, sxm);
+      ab += fabsf(xf - mf);
+      const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
+      if (kZeroInM) flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
+      else flips += ((int)xt <= 0) ? 1u : 0u;
+      sum[2 * q + hlf] += xf;
     }
   }
 }
 
 // Rows [r0, r1) of the flat [rows, d] view, of which [r0, cut) lie in sample b0 and [cut, r1) in
-// sample b0 + 1 (cut = r1: one segment).
-template <int NR>
+// sample b0 + 1 (cut = r1: one segment).  kFull: d is a multiple of the warp tile, no ragged tile.
+template <int NR, bool kFull>
 __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int b0, long long r0, long long cut,
-                         long long r1, const float *m_in, float *m_out, int c, FewShared &fs, double *s_acc) {
+                         long long r1, const float *m_in, float *m_out, int c, FewShared &fs, FewWarp *fw_all) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunks = a.d >> 3;                               // d is a multiple of 8 here
   const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
   const int n_tiles = (int)(r1 - r0) * tiles_per_row;
   const int cut_rr = (int)(cut - r0);                        // first row (from r0) of the second segment
   const float beta = a.beta, wgt = a.one_minus_beta / (float)NR;
-  constexpr int kSums = NR * 4 + 2;                          // per tensor 4 sums, then the reference's 2
+  FewWarp &fw = fw_all[warp];
 
-  for (int q = tid; q < kSegsPerCta * kSums * kFewThreads; q += kFewThreads) s_acc[q] = 0.;
   for (int q = tid; q < kSegsPerCta * kFewWarps * kFewSets; q += kFewThreads) {
     (&fs.flips[0][0][0])[q] = 0u;
     (&fs.bits[0][0][0])[q] = 0u;
   }
   if (tid < kSegsPerCta * kFewWarps) (&fs.m_varies[0][0])[tid] = 0u;
-  __syncthreads();                                           // fs.ptr is in place
+  if (tid == 0) fs.timed_out = 0;
+  for (int q = lane; q < kSegsPerCta * (kFewSets * 4 + 2); q += 32) (&fw.acc[0][0])[q] = 0.;
+  if (lane == 0) {
+#pragma unroll
+    for (int st = 0; st < kStageDepth; ++st) mbar_init(smem_addr(&fw.bar[st]), 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();                                           // fs.ptr is in place, the barriers are ready
   if (tid < kSegsPerCta * NR) {
     const int sg = tid / NR, r = tid - sg * NR;
     const size_t sample_off = (size_t)(b0 + sg) * a.T * a.d;
@@ -1597,7 +1652,34 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     const int sg = tid - 32;
     if (sg == 0 || cut < r1) fs.m0bits[sg] = __float_as_uint(m_in[(size_t)(b0 + sg) * a.T * a.d]);
   }
-  __syncthreads();
+
+  // the warp's tiles: tile t is row r0 + rr, 512 columns from seg * 512 on; the producer's cursor
+  // runs kStageDepth tiles ahead of the consumer's
+  const int step_rr = kFewWarps / tiles_per_row, step_seg = kFewWarps % tiles_per_row;
+  int rr = warp / tiles_per_row, seg = warp % tiles_per_row;
+  int p_rr = rr, p_seg = seg, p_j = warp, p_t = 0;
+  auto issue = [&]() {                                       // fills stage p_t % kStageDepth with the producer's tile
+    if (p_j < n_tiles && lane == 0) {
+      const int st = p_t % kStageDepth;
+      const size_t off = (size_t)(r0 + p_rr) * a.d + (size_t)p_seg * (32 * kUnroll * 8);
+      int vc = 32 * kUnroll;                                 // chunks of this tile that exist
+      if (!kFull && chunks - p_seg * 32 * kUnroll < vc) vc = chunks - p_seg * 32 * kUnroll;
+      const unsigned bar = smem_addr(&fw.bar[st]), dst = smem_addr(&fw.stage[st][0]);
+      mbar_arrive_expect(bar, (unsigned)vc * (32u + 16u * NR));
+      bulk_copy_in(dst, m_in + off, (unsigned)vc * 32u, bar);
+#pragma unroll
+      for (int r = 0; r < NR; ++r)
+        bulk_copy_in(dst + kTileBytesM + r * kTileBytesX, fs.ptr[r] + off, (unsigned)vc * 16u, bar);
+    }
+    p_j += kFewWarps;
+    ++p_t;
+    p_rr += step_rr;
+    p_seg += step_seg;
+    if (p_seg >= tiles_per_row) { p_seg -= tiles_per_row; ++p_rr; }
+  };
+#pragma unroll
+  for (int st = 0; st < kStageDepth; ++st) issue();
+  __syncthreads();                                           // fs.x0, fs.m0bits
 
   float sx[NR], sxx[NR], sxm[NR], ab[NR];
   unsigned fl[NR], xd[NR];
@@ -1606,18 +1688,23 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
 #pragma unroll
   for (int r = 0; r < NR; ++r) { sx[r] = sxx[r] = sxm[r] = ab[r] = 0.f; fl[r] = xd[r] = 0u; }
   int sg = 0;                                                // the segment this warp is in
-  double *acc = s_acc + tid;                                 // this thread's column of segment sg
-  auto fold = [&]() {                                        // the short fp32 runs into this thread's fp64 sums
+  auto fold = [&]() {                                        // the short fp32 runs: lanes added up, into the warp's fp64 sums
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
-      acc[(r * 4 + 0) * kFewThreads] += (double)sx[r];
-      acc[(r * 4 + 1) * kFewThreads] += (double)sxx[r];
-      acc[(r * 4 + 2) * kFewThreads] += (double)sxm[r];
-      acc[(r * 4 + 3) * kFewThreads] += (double)ab[r];
+      const float v0 = warp_sum(sx[r]), v1 = warp_sum(sxx[r]), v2 = warp_sum(sxm[r]), v3 = warp_sum(ab[r]);
+      if (lane == 0) {
+        fw.acc[sg][r * 4 + 0] += (double)v0;
+        fw.acc[sg][r * 4 + 1] += (double)v1;
+        fw.acc[sg][r * 4 + 2] += (double)v2;
+        fw.acc[sg][r * 4 + 3] += (double)v3;
+      }
       sx[r] = sxx[r] = sxm[r] = ab[r] = 0.f;
     }
-    acc[(NR * 4 + 0) * kFewThreads] += (double)g_sm;
-    acc[(NR * 4 + 1) * kFewThreads] += (double)g_smm;
+    const float v4 = warp_sum(g_sm), v5 = warp_sum(g_smm);
+    if (lane == 0) {
+      fw.acc[sg][NR * 4 + 0] += (double)v4;
+      fw.acc[sg][NR * 4 + 1] += (double)v5;
+    }
     g_sm = g_smm = 0.f;
   };
   auto leave_segment = [&]() {                               // counts and bits of segment sg, per warp
@@ -1637,117 +1724,126 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     nf_mask = m_diff = 0u;
   };
 
-  const int step_rr = kFewWarps / tiles_per_row, step_seg = kFewWarps % tiles_per_row;
-  int rr = warp / tiles_per_row, seg = warp % tiles_per_row;
-  int since_fold = 0;
+  int since_fold = 0, t = 0;
   unsigned m0bits = fs.m0bits[0];
   float m0 = __uint_as_float(m0bits);
-  for (int j = warp; j < n_tiles; j += kFewWarps) {
+  bool alive = true;
+  for (int j = warp; j < n_tiles; j += kFewWarps, ++t) {
     if (sg == 0 && rr >= cut_rr) {                           // this warp enters the second segment
       fold();
       leave_segment();
       since_fold = 0;
       sg = 1;
-      acc += kSums * kFewThreads;
       m0bits = fs.m0bits[1];
       m0 = __uint_as_float(m0bits);
     }
+    const int st = t % kStageDepth;
+    if (!__all_sync(0xffffffffu, mbar_wait(smem_addr(&fw.bar[st]), (unsigned)(t / kStageDepth) & 1u))) {
+      alive = false;                                         // the tile never arrived: give up on this warp's rows
+      break;
+    }
     const size_t off = (size_t)(r0 + rr) * a.d;
     const int base = seg * 32 * kUnroll;
-    F8 mv[kUnroll];
-    uint4 xv[kUnroll];
-    bool ok[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int ch = base + u * 32 + lane;
-      ok[u] = ch < chunks;
-      if (ok[u]) {
-        mv[u] = ld_m256(m_in + off + (size_t)ch * 8);
-        xv[u] = ld_x128(fs.ptr[0] + off + (size_t)ch * 8);
-      }
-    }
-    // the reference's own sums, once per tile
+    const unsigned char *stage = fw.stage[st];
+    // does the warp's tile of m hold an exact zero?  (decides which sign test serves: one look at
+    // the staged tile before the arithmetic)
     bool zero_in_m = false;
-    float sum[kUnroll][8];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        sum[u][e] = 0.f;
-        if (ok[u]) {
-          const float ms = mv[u].v[e] - m0;
-          g_sm += ms;
-          g_smm = fmaf(ms, ms, g_smm);
-          m_diff |= __float_as_uint(mv[u].v[e]) ^ m0bits;
-          zero_in_m |= (mv[u].v[e] == 0.f);
-        }
+      if (kFull || base + u * 32 + lane < chunks) {
+        const float4 *src = reinterpret_cast<const float4 *>(stage + (size_t)(u * 32 + lane) * 32);
+        const float4 lo = src[0], hi = src[1];
+        zero_in_m |= (lo.x == 0.f) | (lo.y == 0.f) | (lo.z == 0.f) | (lo.w == 0.f) |
+                     (hi.x == 0.f) | (hi.y == 0.f) | (hi.z == 0.f) | (hi.w == 0.f);
       }
     }
     const bool any_zero = __any_sync(0xffffffffu, zero_in_m);
 
+    // chunk by chunk: the chunk of m, every tensor's chunk against it, the candidate's chunk out
 #pragma unroll
-    for (int r = 0; r < NR; ++r) {                           // the tensors, in order
-      uint4 cur[kUnroll];
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) cur[u] = xv[u];
-      if (r + 1 < NR) {                                      // the next tensor's tile, ahead of the arithmetic
-        const uint16_t *xn = fs.ptr[r + 1] + off;
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-          if (ok[u]) xv[u] = ld_x128(xn + (size_t)(base + u * 32 + lane) * 8);
+    for (int u = 0; u < kUnroll; ++u) {
+      const bool ok = kFull || (base + u * 32 + lane < chunks);
+      if (!ok) continue;
+      F8 mv;
+      {
+        const float4 *src = reinterpret_cast<const float4 *>(stage + (size_t)(u * 32 + lane) * 32);
+        const float4 lo = src[0], hi = src[1];
+        mv.v[0] = lo.x; mv.v[1] = lo.y; mv.v[2] = lo.z; mv.v[3] = lo.w;
+        mv.v[4] = hi.x; mv.v[5] = hi.y; mv.v[6] = hi.z; mv.v[7] = hi.w;
       }
-      const unsigned x0 = fs.x0[sg][r], x0pair = x0 | (x0 << 16);
-      const float x0f = __uint_as_float(x0 << 16);
-      if (any_zero) few_tile<true>(cur, mv, ok, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
-      else few_tile<false>(cur, mv, ok, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
-      if (__any_sync(0xffffffffu, !(ab[r] <= 3.4028234664e38f))) {   // not a finite sum: look at the bits
+      float sum[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {                          // the reference's own sums, once per tile
+        sum[e] = 0.f;
+        const float ms = mv.v[e] - m0;
+        g_sm += ms;
+        g_smm = fmaf(ms, ms, g_smm);
+        m_diff |= __float_as_uint(mv.v[e]) ^ m0bits;
+      }
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {                         // the tensors, in order
+        const uint4 cur = *reinterpret_cast<const uint4 *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+        const unsigned x0 = fs.x0[sg][r], x0pair = x0 | (x0 << 16);
+        const float x0f = __uint_as_float(x0 << 16);
+        if (any_zero) few_chunk<true>(cur, mv, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
+        else few_chunk<false>(cur, mv, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
+      }
+      // Eq. 1 with the mean over the tensors
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mv.v[e] = fmaf(beta, mv.v[e], wgt * sum[e]);
+      st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv);
+    }
+    // a sum of |x - m| that is not a finite number: look at the exponent bits of that tensor's tile
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      if (__any_sync(0xffffffffu, !(ab[r] <= 3.4028234664e38f))) {
         unsigned nf = 0u;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-          if (ok[u]) nf |= (((cur[u].x & 0x7F807F80u) + 0x00800080u) | ((cur[u].y & 0x7F807F80u) + 0x00800080u) |
-                            ((cur[u].z & 0x7F807F80u) + 0x00800080u) | ((cur[u].w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
+        for (int u = 0; u < kUnroll; ++u) {
+          if (kFull || base + u * 32 + lane < chunks) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+            nf |= (((w.x & 0x7F807F80u) + 0x00800080u) | ((w.y & 0x7F807F80u) + 0x00800080u) |
+                   ((w.z & 0x7F807F80u) + 0x00800080u) | ((w.w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
+          }
+        }
         if (nf) nf_mask |= 1u << r;
       }
     }
-    // Eq. 1 with the mean over the tensors
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      if (!ok[u]) continue;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mv[u].v[e] = fmaf(beta, mv[u].v[e], wgt * sum[u][e]);
-      st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
-    }
+    // every lane has used what it read from the stage (the sums above depend on it): refill it
+    __syncwarp();
+    issue();
     if (++since_fold == kFoldTiles) { fold(); since_fold = 0; }
     rr += step_rr;
     seg += step_seg;
     if (seg >= tiles_per_row) { seg -= tiles_per_row; ++rr; }
   }
+  if (!alive) {
+    // the copies still in flight target this CTA's shared memory: give them the same time to land
+    for (int k = 1; k < kStageDepth; ++k) {
+      const int tt = t + k;
+      if (warp + tt * kFewWarps < n_tiles) mbar_wait(smem_addr(&fw.bar[tt % kStageDepth]), (unsigned)(tt / kStageDepth) & 1u);
+    }
+    if (lane == 0) fs.timed_out = 1;
+  }
   fold();
   leave_segment();
 
-  // threads -> CTA in a fixed order: the fp64 columns one quantity per warp in turn
+  // warps -> CTA in a fixed order
   __syncthreads();
-  for (int q = warp; q < kSegsPerCta * kSums; q += kFewWarps) {
-    const int qs = q / kSums, qq = q - qs * kSums;
-    const double *col = s_acc + (size_t)q * kFewThreads;
-    double v = 0.;
-    for (int t = lane; t < kFewThreads; t += 32) v += col[t];
-    v = warp_sum(v);
-    if (lane == 0) fs.red[qs][qq] = v;
-  }
-  __syncthreads();
+  if (tid == 0 && fs.timed_out) atomicExch(&a.hs->error, kErrStagingTimeout);
   if (tid < kSegsPerCta * NR * kSlotWords) {
     const int sgm = tid / (NR * kSlotWords), r = (tid / kSlotWords) % NR, w8 = tid % kSlotWords;
     unsigned long long *slot = partials + (((size_t)fs.widx[r] * a.G + c) * kSegsPerCta + sgm) * kSlotWords;
     if (sgm == 1 && cut >= r1) {
       if (w8 == 7) slot[7] = 0ull;                           // no second segment: tag 0, unused
     } else {
-      const double *red = fs.red[sgm];
       unsigned long long out;
       if (w8 < 6) {
-        const double t = (w8 == 0) ? red[r * 4 + 0] : (w8 == 1) ? red[r * 4 + 1] : (w8 == 2) ? red[NR * 4 + 0]
-                       : (w8 == 3) ? red[NR * 4 + 1] : (w8 == 4) ? red[r * 4 + 2] : red[r * 4 + 3];
-        out = (unsigned long long)__double_as_longlong(t);
+        const int q = (w8 == 0) ? r * 4 + 0 : (w8 == 1) ? r * 4 + 1 : (w8 == 2) ? NR * 4 + 0
+                    : (w8 == 3) ? NR * 4 + 1 : (w8 == 4) ? r * 4 + 2 : r * 4 + 3;
+        double v = 0.;
+        for (int w = 0; w < kFewWarps; ++w) v += fw_all[w].acc[sgm][q];
+        out = (unsigned long long)__double_as_longlong(v);
       } else if (w8 == 6) {
         out = 0ull;
         for (int w = 0; w < kFewWarps; ++w) out += fs.flips[sgm][w][r];
@@ -1763,12 +1859,22 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
 
 __device__ __forceinline__ void few_dispatch(int n, const StreamArgs &a, unsigned long long *partials, int b0,
                                              long long r0, long long cut, long long r1, const float *m_in, float *m_out,
-                                             int c, FewShared &fs, double *s_acc) {
-  switch (n) {
-    case 1: few_rows<1>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
-    case 2: few_rows<2>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
-    case 3: few_rows<3>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
-    default: few_rows<4>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, s_acc); break;
+                                             int c, FewShared &fs, double *s_dyn) {
+  FewWarp *fw = reinterpret_cast<FewWarp *>(s_dyn);
+  if (a.d % (32 * kUnroll * 8) == 0) {
+    switch (n) {
+      case 1: few_rows<1, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 2: few_rows<2, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 3: few_rows<3, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      default: few_rows<4, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+    }
+  } else {
+    switch (n) {
+      case 1: few_rows<1, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 2: few_rows<2, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 3: few_rows<3, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      default: few_rows<4, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+    }
   }
 }
 
@@ -1921,7 +2027,7 @@ __global__ void __launch_bounds__(kFew ? kFewThreads : kThreads)
 replica_kernel(const ReplicaArgs ra) {
   __shared__ typename std::conditional<kFew, FewShared, ReplicaShared>::type sh;
   __shared__ int s_last;
-  extern __shared__ double s_dyn[];            // CTA 0: the refresh's working copies; the others: the threads' fp64 sums
+  extern __shared__ __align__(128) double s_dyn[];   // CTA 0: the refresh's working copies; the others: the warps' staging rings
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -2016,7 +2122,7 @@ __global__ void __launch_bounds__(kFew ? kFewThreads : kThreads)
 shared_ref_kernel(const ReplicaArgs ra) {
   __shared__ typename std::conditional<kFew, FewShared, ReplicaShared>::type sh;
   __shared__ int s_last;
-  extern __shared__ double s_dyn[];
+  extern __shared__ __align__(128) double s_dyn[];
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
