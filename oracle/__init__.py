@@ -75,6 +75,12 @@ def lib():
         L.so_bf16.restype = C.c_double
         L.so_distance.argtypes = [u16p, dp, C.c_size_t, dp, dp]
         L.so_distance.restype = C.c_int
+        L.so_token_sums.argtypes = [u16p, dp, C.c_size_t, dp]
+        L.so_token_sums.restype = None
+        L.so_out_of_bounds.argtypes = [C.c_double, C.c_double, C.c_double]
+        L.so_out_of_bounds.restype = C.c_int
+        L.so_severe.argtypes = [C.c_int, C.c_double, C.c_double, C.c_double, C.c_double]
+        L.so_severe.restype = C.c_int
         L.so_percentile.argtypes = [dp, C.c_size_t, C.c_double]
         L.so_percentile.restype = C.c_double
         L.so_adaptive_iqr.argtypes = [dp, C.c_size_t, C.c_double, C.c_int, C.c_double,
@@ -208,6 +214,29 @@ def distance(x_bits, m) -> tuple[np.ndarray, np.ndarray, bool]:
     s = np.empty(NSTAT)
     nf = lib().so_distance(_u16ptr(xb), _dptr(mm), xb.size, _dptr(g), _dptr(s))
     return g, s, bool(nf)
+
+
+def token_sums(x_bits, m) -> np.ndarray:
+    """Per token row: sum_c x, sum_c x^2, sum_c |x - m|, sign mismatches.  x_bits [..., d] against
+    m of the same shape; returns [..., 4]."""
+    xb = np.ascontiguousarray(_bits(x_bits))
+    mm = np.ascontiguousarray(np.broadcast_to(np.asarray(m, dtype=np.float64), xb.shape))
+    d = xb.shape[-1]
+    rows = xb.reshape(-1, d)
+    mrows = mm.reshape(-1, d)
+    out = np.empty((rows.shape[0], 4))
+    for i in range(rows.shape[0]):
+        xr, mr = np.ascontiguousarray(rows[i]), np.ascontiguousarray(mrows[i])
+        lib().so_token_sums(_u16ptr(xr), _dptr(mr), d, _dptr(out[i]))
+    return out.reshape(xb.shape[:-1] + (4,))
+
+
+def out_of_bounds(gamma: float, tau_lower: float, tau_upper: float) -> bool:
+    return bool(lib().so_out_of_bounds(gamma, tau_lower, tau_upper))
+
+
+def severe(flagged: bool, gamma: float, q2: float, tau_upper: float, severe_mult: float) -> bool:
+    return bool(lib().so_severe(int(flagged), gamma, q2, tau_upper, severe_mult))
 
 
 def sliced_wasserstein(x_bits, m, u_bits):

@@ -401,6 +401,33 @@ static void ema_update(so_verifier *v, const uint16_t *x, int kind) {
   for (size_t e = 0; e < v->N; ++e) m[e] = beta * m[e] + (1.0 - beta) * so_bf16(x[e]);
 }
 
+/* Eq. 3 / Alg. 5: a deviation is out of bounds when it does not lie in the closed interval
+ * [tau_lower, tau_upper].  Written as the negation of "lies inside", so that a deviation that is
+ * not a number counts as outside (and, being flagged, never joins the history). */
+int so_out_of_bounds(double gamma, double tau_lower, double tau_upper) {
+  return !(gamma >= tau_lower && gamma <= tau_upper);
+}
+
+/* Sec. 3.1: a worker is banned at once when its deviation lies "x100 above the threshold".  The
+ * rule speaks of a deviation that broke the threshold, so it is looked at only for a metric
+ * that flagged: |gamma - q2| >= severe_mult * (tau_upper - q2). */
+int so_severe(int flagged, double gamma, double q2, double tau_upper, double severe_mult) {
+  return flagged && fabs(gamma - q2) >= severe_mult * (tau_upper - q2);
+}
+
+/* The first level of the reduction, for one token row: sum_c x, sum_c x^2, sum_c |x - m| and the
+ * number of channels with sign(x) != sign(m) (Sec. 3.1 measures before the mean over tokens). */
+void so_token_sums(const uint16_t *x, const double *m, size_t d, double out[4]) {
+  out[0] = out[1] = out[2] = out[3] = 0.0;
+  for (size_t c = 0; c < d; ++c) {
+    const double xv = so_bf16(x[c]);
+    out[0] += xv;
+    out[1] += xv * xv;
+    out[2] += fabs(xv - m[c]);
+    out[3] += (sign3(xv) != sign3(m[c])) ? 1.0 : 0.0;
+  }
+}
+
 /* Sec. 3.1, violation counter with forgiveness, kept per worker */
 static void count_violation(so_verifier *v, int r, int flagged, int severe) {
   const so_params *p = &v->p;
@@ -464,9 +491,10 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
         if (!((p->metric_mask >> i) & 1u)) continue;
         const double *t = ks->thr[L][i];
         const double g = gam[(size_t)r * SO_NMETRIC + i];
-        if (g < t[4] || g > t[5]) f |= (1u << i);
+        const int out = so_out_of_bounds(g, t[4], t[5]);
+        if (out) f |= (1u << i);
         /* 3. severe deviation, tested on the whole-tensor unit */
-        if (r == 0 && fabs(g - t[1]) >= p->severe_mult * (t[5] - t[1])) severe = 1;
+        if (r == 0 && so_severe(out, g, t[1], t[5], p->severe_mult)) severe = 1;
       }
     }
     flags[r] = f;
@@ -546,8 +574,9 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
           if (!((p->metric_mask >> i) & 1u)) continue;
           const double *t = ks->thr[L][i];
           const double g = gam[(size_t)u * SO_NMETRIC + i];
-          if (g < t[4] || g > t[5]) f |= (1u << i);
-          if (u == 0 && fabs(g - t[1]) >= p->severe_mult * (t[5] - t[1])) severe_w[r] = 1;
+          const int out = so_out_of_bounds(g, t[4], t[5]);
+          if (out) f |= (1u << i);
+          if (u == 0 && so_severe(out, g, t[1], t[5], p->severe_mult)) severe_w[r] = 1;
         }
       }
       fl[u] = f;

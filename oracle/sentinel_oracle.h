@@ -22,9 +22,12 @@
  *     out of its loop, Alg. 3 adds it to the stage's tainted set: read literally, per kind; a
  *     worker that was not collected never enters the mean of Eq. 1),
  *   - the number and the draw of the sliced Wasserstein directions (the caller supplies them),
- *   - the two storage variants the paper does not mention: a reference stored as bf16 (its
- *     rounding is pinned to an independent single-precision computation, the choice of the
- *     variant itself is not the paper's), and the references reduced over the samples ([T,d]),
+ *   - the two storage variants the paper does not mention: a reference stored as bf16 (the one
+ *     place where this oracle leaves float64: which of two neighbouring bf16 values an element
+ *     takes is a decision of the arithmetic, so the update m = bf16(fma(beta, m, (1-beta) x)) is
+ *     taken in single precision, the precision the stored format implies, and agrees with a
+ *     single-precision implementation bit for bit; it is pinned to an independent float64
+ *     emulation of that fused update, the choice of the variant itself is not the paper's), and the references reduced over the samples ([T,d]),
  *     over the tokens ([B,d]) or over both ([d]) (Eq. 1 with the mean over what is reduced).
  */
 #ifndef SENTINEL_ORACLE_H
@@ -90,6 +93,18 @@ double so_bf16(uint16_t bits);
  * values m.  gamma[3] = {L1, normalised L2, SFR}; stat[8] as listed above.  Returns 1 when x
  * holds a NaN or an infinity (then every output is NaN), else 0. */
 int so_distance(const uint16_t *x, const double *m, size_t n, double gamma[3], double stat[8]);
+
+/* The first reduction level for one token row of d channels: out = {sum_c x, sum_c x^2,
+ * sum_c |x - m|, #{c : sign(x) != sign(m)}} (the per-token terms of the Sec. 3.1 measures). */
+void so_token_sums(const uint16_t *x, const double *m, size_t d, double out[4]);
+
+/* Eq. 3 / Alg. 5: 1 when gamma does not lie in [tau_lower, tau_upper]; a gamma that is not a
+ * number is outside. */
+int so_out_of_bounds(double gamma, double tau_lower, double tau_upper);
+
+/* Sec. 3.1, immediate ban: 1 when the metric flagged and |gamma - q2| >= severe_mult *
+ * (tau_upper - q2).  (Parity unpinned: the paper only says "x100 above the threshold".) */
+int so_severe(int flagged, double gamma, double q2, double tau_upper, double severe_mult);
 
 /* Percentile of an ascending array by linear interpolation at position p*(n-1), p in [0,1]. */
 double so_percentile(const double *sorted, size_t n, double p);

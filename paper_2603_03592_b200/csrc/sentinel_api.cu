@@ -807,7 +807,13 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   unsigned char *scratch = nullptr;
   keep_pool_warm(device);
   SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, slot_bytes + 256, s));
-  SENTINEL_CUDA(nullptr, cudaMemsetAsync(scratch + slot_bytes, 0, 256, s));
+  {
+    const cudaError_t me = cudaMemsetAsync(scratch + slot_bytes, 0, 256, s);
+    if (me != cudaSuccess) {
+      cudaFreeAsync(scratch, s);                       // nothing was launched on it
+      return fail(nullptr, SENTINEL_ERR_CUDA, "clearing the scratch failed: %s", cudaGetErrorString(me));
+    }
+  }
 
   StreamArgs a;
   memset(&a, 0, sizeof a);

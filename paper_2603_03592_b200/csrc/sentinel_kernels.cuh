@@ -954,8 +954,11 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
         const double tau_lower = ks->thr[L][i][4], tau_upper = ks->thr[L][i][5];
         // (written so that a score that is not a number -- projections beyond the fp32 range --
         // counts as outside and never joins the history)
-        if (!(g[i] >= tau_lower && g[i] <= tau_upper)) my_flag |= (1u << i);
-        if (tid == 0 && fabs(g[i] - q2) >= a.severe_mult * (tau_upper - q2)) s_severe = 1;
+        const bool outside = !(g[i] >= tau_lower && g[i] <= tau_upper);
+        if (outside) my_flag |= (1u << i);
+        // ("x100 above the threshold", Sec. 3.1, is said of a deviation that broke the threshold: a
+        // clean step never counts as severe, not even when the window is a single point)
+        if (tid == 0 && outside && fabs(g[i] - q2) >= a.severe_mult * (tau_upper - q2)) s_severe = 1;
       }
     }
     s_flag[tid] = my_flag;

@@ -339,3 +339,47 @@ def test_sliced_wasserstein_against_scipy_and_closed_forms(oracle_mod, rng):
     bad = x.copy()
     bad[3, 4] = np.inf
     assert np.isnan(oracle_mod.sliced_wasserstein(to_bits(bad), m, ub)[0])
+
+
+# ---------------------------------------------------------------- decision rules, token sums
+
+def test_out_of_bounds_is_the_negated_closed_interval(oracle_mod):
+    """Eq. 3 / Alg. 5: flagged iff outside [tau_lower, tau_upper]; the bounds themselves are inside,
+    and a deviation that is not a number is outside."""
+    ob = oracle_mod.out_of_bounds
+    assert not ob(1.0, 1.0, 2.0) and not ob(2.0, 1.0, 2.0) and not ob(1.5, 1.0, 2.0)
+    assert ob(np.nextafter(1.0, 0.0), 1.0, 2.0) and ob(np.nextafter(2.0, 3.0), 1.0, 2.0)
+    assert ob(float("nan"), 1.0, 2.0) and ob(float("inf"), 1.0, 2.0) and ob(-float("inf"), 1.0, 2.0)
+    assert not ob(0.0, 0.0, 0.0)                      # a degenerate interval still holds its point
+
+
+def test_severe_rule_needs_a_flag(oracle_mod):
+    """Sec. 3.1: 'x100 above the threshold' is said of a deviation that broke the threshold."""
+    sv = oracle_mod.severe
+    assert sv(True, 1.0 + 100 * 0.5, 1.0, 1.5, 100.0)            # exactly 100 allowed deviations
+    assert not sv(True, 1.0 + 99.9 * 0.5, 1.0, 1.5, 100.0)
+    assert sv(True, 1.0 - 100 * 0.5, 1.0, 1.5, 100.0)            # two-sided
+    assert not sv(False, 1e9, 1.0, 1.5, 100.0)                   # not flagged: never severe
+    assert not sv(False, 1.0, 1.0, 1.0, 100.0)                   # tau_upper == q2, clean step on the median
+    assert sv(True, 2.0, 1.0, 1.0, 100.0)                        # zero allowed deviation, flagged
+    assert not sv(True, float("nan"), 1.0, 1.5, 100.0)           # not a number: flagged, but no distance
+
+
+def test_token_sums_by_hand_and_against_the_unit_measures(oracle_mod, rng):
+    """Hand-written rows (small integers and halves are exact in bf16), then the identity that ties
+    the token sums to the pinned unit measures: summed over the rows of a unit and divided by its
+    size they are the L1 distance and the sign-flip ratio of so_distance."""
+    x = np.array([[1.0, -2.0, 0.0, 3.0, -0.0, 0.5, -4.0, 8.0]])
+    m = np.array([[1.0, 2.0, 0.0, -1.0, 1.0, 0.25, -4.0, 0.0]])
+    got = oracle_mod.token_sums(to_bits(x), m)
+    #  sum x = 6.5; sum x^2 = 1+4+0+9+0+0.25+16+64 = 94.25; |x-m| = 0+4+0+4+1+0.25+0+8 = 17.25
+    #  sign mismatches: (-2,2) (3,-1) (-0,1) (8,0) -> 4
+    assert got.tolist() == [[6.5, 94.25, 17.25, 4.0]]
+    xb = to_bits(rng.normal(0.2, 1.3, (5, 24)))
+    mm = rng.normal(0.0, 1.0, (5, 24))
+    ts = oracle_mod.token_sums(xb, mm)
+    gam, stat, _ = oracle_mod.distance(xb, mm)
+    assert ts[:, 2].sum() / xb.size == pytest.approx(gam[0], rel=1e-13)
+    assert ts[:, 3].sum() / xb.size == pytest.approx(gam[2], rel=1e-13)
+    assert ts[:, 0].sum() / xb.size == pytest.approx(stat[0], rel=1e-12, abs=1e-15)
+    assert np.sqrt(ts[:, 1].sum()) == pytest.approx(stat[2], rel=1e-13)

@@ -820,3 +820,25 @@ def test_per_sample_channel_reference_commit_and_replacement(oracle_mod, small):
         assert np.all(np.abs(got[b] - m0[b]) <= 2.0 ** -8 * np.abs(m0[b]) + 1e-45)
     with pytest.raises(ValueError):
         oracle_mod.Verifier(oracle_mod.Params(B=2, T=4, d=8, ref_over_tokens=1, ema_bf16=1))
+
+
+def test_a_constant_history_does_not_make_clean_steps_severe(oracle_mod):
+    """With iqr_eps = 0 and lambda = 0 a window of identical deviations gives tau_upper = q2.  A
+    clean step on the median then has |gamma - q2| = 0 >= 100 * 0: the severe rule must not fire
+    for it (it speaks of a deviation that broke the threshold), while a flagged step at any
+    distance from such a window does."""
+    v = make(oracle_mod, B=1, T=2, d=8, eps=(0.0, 0.0), lam=(0.0, 0.0))
+    xb = to_bits(np.tile(np.array([1.0, -2.0, 3.0, 0.5, -1.5, 2.5, -0.25, 4.0]), (1, 2, 1)))
+    v.set_ema(ACT, np.zeros((1, 2, 8)))
+    for _ in range(6):                                   # beta irrelevant: keep the reference at 0
+        v.update_reference(xb, ACT)
+        v.set_ema(ACT, np.zeros((1, 2, 8)))
+    thr, valid = v.thresholds(ACT)
+    assert valid.all() and np.all(thr[:, :, 5] == thr[:, :, 1])          # tau_upper == q2 everywhere
+    scores, flags, commit = v.verify(xb, ACT)
+    assert commit and not (flags[0] & oracle_mod.FLAG_SEVERE) and not (flags[0] & 0xFFFF)
+    assert v.counters() == (0, 1, 0)
+    v.set_ema(ACT, np.zeros((1, 2, 8)))
+    scores, flags, commit = v.verify(to_bits(2.0 * from_bits(xb)), ACT)  # L1 doubles: off the single point
+    assert not commit and (flags[0] & oracle_mod.FLAG_L1) and (flags[0] & oracle_mod.FLAG_SEVERE)
+    assert v.counters() == (1, 0, 1)
