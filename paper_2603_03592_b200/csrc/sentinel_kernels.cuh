@@ -1593,16 +1593,34 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
   }
 }
 
-// one tensor's 8-element chunk against the chunk of m (kZeroInM = false: no exact zero in the
-// warp's tile of m, see replica_tile)
+// One tensor's 8-element chunk against the chunk of m.  Sign mismatches are counted in units of
+// kFlipUnit.  kZeroInM = true: the general three-valued sign test, element by element.
+// kZeroInM = false (no exact zero in this chunk of m, the usual case): on the packed pairs --
+// msp holds the sign bits of the two m's of a pair at bits 15 and 31, so (w ^ msp) & 0x80008000
+// has a bit set per element whose sign bit differs from m's, and a byte-wise dot product with
+// ones adds them up (0x80 each).  That is the mismatch count unless x holds an exact zero (a
+// zero counts as a mismatch whatever its sign bit): zmin follows the smallest magnitude of the
+// tensor's tile, and the caller corrects the count of a tile in which it reached zero.
+constexpr unsigned kFlipUnit = 128u;
+
+__device__ __forceinline__ unsigned min_abs_bf16x2(unsigned a, unsigned b) {   // per half: min(|a|, |b|), sign bit unspecified
+  unsigned r;
+  asm("min.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
 template <bool kZeroInM>
-__device__ __forceinline__ void few_chunk(const uint4 &cur, const F8 &mv, float x0f, float m0, unsigned x0pair,
-                                          float (&sum)[8], float &sx, float &sxx, float &sxm, float &ab,
-                                          unsigned &flips, unsigned &x_diff) {
+__device__ __forceinline__ void few_chunk(const uint4 &cur, const F8 &mv, const unsigned (&msp)[4], float x0f, float m0,
+                                          unsigned x0pair, float (&sum)[8], float &sx, float &sxx, float &sxm,
+                                          float &ab, unsigned &flips, unsigned &x_diff, unsigned &zmin) {
   const unsigned w4[4] = {cur.x, cur.y, cur.z, cur.w};
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     x_diff |= w4[q] ^ x0pair;
+    if (!kZeroInM) {
+      flips = __dp4a((w4[q] ^ msp[q]) & 0x80008000u, 0x01010101u, flips);
+      zmin = min_abs_bf16x2(zmin, w4[q]);
+    }
 #pragma unroll
     for (int hlf = 0; hlf < 2; ++hlf) {
       const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
@@ -1612,12 +1630,42 @@ __device__ __forceinline__ void few_chunk(const uint4 &cur, const F8 &mv, float 
       sxx = fmaf(xs, xs, sxx);
       sxm = fmaf(xs, ms, sxm);
       ab += fabsf(xf - mf);
-      const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
-      if (kZeroInM) flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
-      else flips += ((int)xt <= 0) ? 1u : 0u;
+      if (kZeroInM) {
+        const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
+        flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? kFlipUnit : 0u;
+      }
       sum[2 * q + hlf] += xf;
     }
   }
+}
+
+// The two rare corrections of a tile, kept out of line so that they cost the streaming loop no
+// registers.  `valid` = this lane's chunks (bit u) that exist.
+// Exponent bits of all ones (NaN or infinity) among this lane's elements of tensor r's tile?
+__device__ __noinline__ unsigned few_nonfinite_in_tile(const unsigned char *stage, int r, int lane, unsigned valid) {
+  unsigned nf = 0u;
+  for (int u = 0; u < kUnroll; ++u) {
+    if (!((valid >> u) & 1u)) continue;
+    const uint4 w = *reinterpret_cast<const uint4 *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+    nf |= (((w.x & 0x7F807F80u) + 0x00800080u) | ((w.y & 0x7F807F80u) + 0x00800080u) |
+           ((w.z & 0x7F807F80u) + 0x00800080u) | ((w.w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
+  }
+  return nf;
+}
+// Exact zeros of tensor r whose sign bit equals that of m, in the chunks where the packed sign
+// test ran (it did not count them): each is a mismatch all the same.  Returns their number.
+__device__ __noinline__ unsigned few_uncounted_zeros(const unsigned char *stage, int r, int lane, unsigned valid) {
+  unsigned n = 0u;
+  for (int u = 0; u < kUnroll; ++u) {
+    if (!((valid >> u) & 1u)) continue;
+    const uint16_t *xw = reinterpret_cast<const uint16_t *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+    const unsigned *mw = reinterpret_cast<const unsigned *>(stage + (size_t)(u * 32 + lane) * 32);
+    for (int e = 0; e < 8; ++e) {
+      const unsigned xb = xw[e];
+      if ((xb & 0x7FFFu) == 0u && (xb >> 15) == (mw[e] >> 31)) ++n;
+    }
+  }
+  return n;
 }
 
 // Rows [r0, r1) of the flat [rows, d] view, of which [r0, cut) lie in sample b0 and [cut, r1) in
@@ -1656,14 +1704,15 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     if (sg == 0 || cut < r1) fs.m0bits[sg] = __float_as_uint(m_in[(size_t)(b0 + sg) * a.T * a.d]);
   }
 
-  // the warp's tiles: tile t is row r0 + rr, 512 columns from seg * 512 on; the producer's cursor
-  // runs kStageDepth tiles ahead of the consumer's
-  const int step_rr = kFewWarps / tiles_per_row, step_seg = kFewWarps % tiles_per_row;
-  int rr = warp / tiles_per_row, seg = warp % tiles_per_row;
-  int p_rr = rr, p_seg = seg, p_j = warp, p_t = 0;
-  auto issue = [&]() {                                       // fills stage p_t % kStageDepth with the producer's tile
-    if (p_j < n_tiles && lane == 0) {
-      const int st = p_t % kStageDepth;
+  // the warp's tiles: tile number j = warp + t * kFewWarps is row r0 + j / tiles_per_row, 512
+  // columns from (j % tiles_per_row) * 512 on; stage t % kStageDepth holds it.  The producer runs
+  // kStageDepth tiles ahead of the consumer.  (Row and column are worked out from j each time:
+  // a division per tile costs less than the registers a running cursor would hold.)
+  auto issue = [&](int pt) {                                 // fills stage pt % kStageDepth with the warp's tile pt
+    const int pj = warp + pt * kFewWarps;
+    if (pj < n_tiles && lane == 0) {
+      const int p_rr = pj / tiles_per_row, p_seg = pj - p_rr * tiles_per_row;
+      const int st = pt % kStageDepth;
       const size_t off = (size_t)(r0 + p_rr) * a.d + (size_t)p_seg * (32 * kUnroll * 8);
       int vc = 32 * kUnroll;                                 // chunks of this tile that exist
       if (!kFull && chunks - p_seg * 32 * kUnroll < vc) vc = chunks - p_seg * 32 * kUnroll;
@@ -1674,23 +1723,25 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
       for (int r = 0; r < NR; ++r)
         bulk_copy_in(dst + kTileBytesM + r * kTileBytesX, fs.ptr[r] + off, (unsigned)vc * 16u, bar);
     }
-    p_j += kFewWarps;
-    ++p_t;
-    p_rr += step_rr;
-    p_seg += step_seg;
-    if (p_seg >= tiles_per_row) { p_seg -= tiles_per_row; ++p_rr; }
   };
 #pragma unroll
-  for (int st = 0; st < kStageDepth; ++st) issue();
+  for (int st = 0; st < kStageDepth; ++st) issue(st);
   __syncthreads();                                           // fs.x0, fs.m0bits
 
-  float sx[NR], sxx[NR], sxm[NR], ab[NR];
+  float sx[NR], sxx[NR], sxm[NR], ab[NR], x0f[NR];
   unsigned fl[NR], xd[NR];
-  unsigned nf_mask = 0u, m_diff = 0u;
+  unsigned m_diff = 0u;
   float g_sm = 0.f, g_smm = 0.f;
 #pragma unroll
   for (int r = 0; r < NR; ++r) { sx[r] = sxx[r] = sxm[r] = ab[r] = 0.f; fl[r] = xd[r] = 0u; }
   int sg = 0;                                                // the segment this warp is in
+  auto enter_segment = [&]() {                               // the shift values of segment sg
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      x0f[r] = __uint_as_float(fs.x0[sg][r] << 16);
+    }
+  };
+  enter_segment();
   auto fold = [&]() {                                        // the short fp32 runs: lanes added up, into the warp's fp64 sums
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
@@ -1715,30 +1766,30 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     for (int r = 0; r < NR; ++r) {
       const unsigned wf = __reduce_add_sync(0xffffffffu, fl[r]);
       const unsigned wx = __reduce_or_sync(0xffffffffu, xd[r]);
-      const unsigned wn = __reduce_or_sync(0xffffffffu, (nf_mask >> r) & 1u);
       if (lane == 0) {
-        fs.flips[sg][warp][r] = wf;
-        fs.bits[sg][warp][r] = (wn ? (unsigned)kBitNonfinite : 0u) | (wx ? (unsigned)kBitXVaries : 0u);
+        fs.flips[sg][warp][r] = wf / kFlipUnit;
+        if (wx) atomicOr(&fs.bits[sg][warp][r], (unsigned)kBitXVaries);   // (the non-finite bit may be there already)
       }
       fl[r] = xd[r] = 0u;
     }
     const unsigned wm = __reduce_or_sync(0xffffffffu, m_diff);
     if (lane == 0) fs.m_varies[sg][warp] = wm;
-    nf_mask = m_diff = 0u;
+    m_diff = 0u;
   };
 
-  int since_fold = 0, t = 0;
+  int t = 0;
   unsigned m0bits = fs.m0bits[0];
   float m0 = __uint_as_float(m0bits);
   bool alive = true;
   for (int j = warp; j < n_tiles; j += kFewWarps, ++t) {
+    const int rr = j / tiles_per_row, seg = j - rr * tiles_per_row;
     if (sg == 0 && rr >= cut_rr) {                           // this warp enters the second segment
       fold();
       leave_segment();
-      since_fold = 0;
       sg = 1;
       m0bits = fs.m0bits[1];
       m0 = __uint_as_float(m0bits);
+      enter_segment();
     }
     const int st = t % kStageDepth;
     if (!__all_sync(0xffffffffu, mbar_wait(smem_addr(&fw.bar[st]), (unsigned)(t / kStageDepth) & 1u))) {
@@ -1748,77 +1799,73 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     const size_t off = (size_t)(r0 + rr) * a.d;
     const int base = seg * 32 * kUnroll;
     const unsigned char *stage = fw.stage[st];
-    // does the warp's tile of m hold an exact zero?  (decides which sign test serves: one look at
-    // the staged tile before the arithmetic)
-    bool zero_in_m = false;
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      if (kFull || base + u * 32 + lane < chunks) {
-        const float4 *src = reinterpret_cast<const float4 *>(stage + (size_t)(u * 32 + lane) * 32);
-        const float4 lo = src[0], hi = src[1];
-        zero_in_m |= (lo.x == 0.f) | (lo.y == 0.f) | (lo.z == 0.f) | (lo.w == 0.f) |
-                     (hi.x == 0.f) | (hi.y == 0.f) | (hi.z == 0.f) | (hi.w == 0.f);
-      }
-    }
-    const bool any_zero = __any_sync(0xffffffffu, zero_in_m);
-
     // chunk by chunk: the chunk of m, every tensor's chunk against it, the candidate's chunk out
+    unsigned zmin = 0x7F7F7F7Fu;                             // smallest magnitudes met in the tensors' tiles
+    unsigned fast_chunks = 0u;                               // chunks that took the packed sign test
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const bool ok = kFull || (base + u * 32 + lane < chunks);
-      if (!ok) continue;
       F8 mv;
-      {
+      unsigned msp[4];
+      float sum[8];
+      float mmin = 1.f;
+      if (ok) {
         const float4 *src = reinterpret_cast<const float4 *>(stage + (size_t)(u * 32 + lane) * 32);
         const float4 lo = src[0], hi = src[1];
         mv.v[0] = lo.x; mv.v[1] = lo.y; mv.v[2] = lo.z; mv.v[3] = lo.w;
         mv.v[4] = hi.x; mv.v[5] = hi.y; mv.v[6] = hi.z; mv.v[7] = hi.w;
-      }
-      float sum[8];
+        mmin = fminf(fminf(fminf(fabsf(lo.x), fabsf(lo.y)), fminf(fabsf(lo.z), fabsf(lo.w))),
+                     fminf(fminf(fabsf(hi.x), fabsf(hi.y)), fminf(fabsf(hi.z), fabsf(hi.w))));
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {                          // the reference's own sums, once per tile
-        sum[e] = 0.f;
-        const float ms = mv.v[e] - m0;
-        g_sm += ms;
-        g_smm = fmaf(ms, ms, g_smm);
-        m_diff |= __float_as_uint(mv.v[e]) ^ m0bits;
-      }
+        for (int e = 0; e < 8; ++e) {                        // the reference's own sums, once per tile
+          sum[e] = 0.f;
+          const float ms = mv.v[e] - m0;
+          g_sm += ms;
+          g_smm = fmaf(ms, ms, g_smm);
+          m_diff |= __float_as_uint(mv.v[e]) ^ m0bits;
+        }
 #pragma unroll
-      for (int r = 0; r < NR; ++r) {                         // the tensors, in order
-        const uint4 cur = *reinterpret_cast<const uint4 *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
-        const unsigned x0 = fs.x0[sg][r], x0pair = x0 | (x0 << 16);
-        const float x0f = __uint_as_float(x0 << 16);
-        if (any_zero) few_chunk<true>(cur, mv, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
-        else few_chunk<false>(cur, mv, x0f, m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r]);
+        for (int q = 0; q < 4; ++q)                          // byte 3 of each m of a pair into bytes 1 and 3
+          msp[q] = __byte_perm(__float_as_uint(mv.v[2 * q]), __float_as_uint(mv.v[2 * q + 1]), 0x7733);
       }
-      // Eq. 1 with the mean over the tensors
+      // an exact zero in this chunk of m (for any lane): the general sign test serves
+      const bool any_zero = __any_sync(0xffffffffu, !(mmin > 0.f));
+      if (!any_zero) fast_chunks |= 1u << u;
+      if (ok) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) mv.v[e] = fmaf(beta, mv.v[e], wgt * sum[e]);
-      st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv);
+        for (int r = 0; r < NR; ++r) {                       // the tensors, in order
+          const uint4 cur = *reinterpret_cast<const uint4 *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+          const unsigned x0pair = __byte_perm(__float_as_uint(x0f[r]), 0u, 0x3232);   // the bf16 pattern in both halves
+          if (any_zero) few_chunk<true>(cur, mv, msp, x0f[r], m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r], zmin);
+          else few_chunk<false>(cur, mv, msp, x0f[r], m0, x0pair, sum, sx[r], sxx[r], sxm[r], ab[r], fl[r], xd[r], zmin);
+        }
+        // Eq. 1 with the mean over the tensors
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mv.v[e] = fmaf(beta, mv.v[e], wgt * sum[e]);
+        st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv);
+      }
+    }
+    unsigned valid = 0u;                                     // this lane's chunks of the tile
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (kFull || base + u * 32 + lane < chunks) valid |= 1u << u;
+    // a tile with an exact zero in some tensor: where the packed test ran, a zero whose sign bit
+    // equals that of m was not counted
+    if (__any_sync(0xffffffffu, ((zmin & 0x7FFFu) == 0u) || ((zmin & 0x7FFF0000u) == 0u))) {
+#pragma unroll
+      for (int r = 0; r < NR; ++r) fl[r] += kFlipUnit * few_uncounted_zeros(stage, r, lane, valid & fast_chunks);
     }
     // a sum of |x - m| that is not a finite number: look at the exponent bits of that tensor's tile
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
       if (__any_sync(0xffffffffu, !(ab[r] <= 3.4028234664e38f))) {
-        unsigned nf = 0u;
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          if (kFull || base + u * 32 + lane < chunks) {
-            const uint4 w = *reinterpret_cast<const uint4 *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
-            nf |= (((w.x & 0x7F807F80u) + 0x00800080u) | ((w.y & 0x7F807F80u) + 0x00800080u) |
-                   ((w.z & 0x7F807F80u) + 0x00800080u) | ((w.w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
-          }
-        }
-        if (nf) nf_mask |= 1u << r;
+        if (few_nonfinite_in_tile(stage, r, lane, valid)) atomicOr(&fs.bits[sg][warp][r], (unsigned)kBitNonfinite);
       }
     }
     // every lane has used what it read from the stage (the sums above depend on it): refill it
     __syncwarp();
-    issue();
-    if (++since_fold == kFoldTiles) { fold(); since_fold = 0; }
-    rr += step_rr;
-    seg += step_seg;
-    if (seg >= tiles_per_row) { seg -= tiles_per_row; ++rr; }
+    issue(t + kStageDepth);
+    if ((t & (kFoldTiles - 1)) == kFoldTiles - 1) fold();
   }
   if (!alive) {
     // the copies still in flight target this CTA's shared memory: give them the same time to land
