@@ -34,6 +34,7 @@ from paper_2603_03592_b200 import replicas, synth  # noqa: E402
 ACT, GRAD = 0, 1
 BYTES_PER_ELEMENT = 10          # 2 (x, bf16 read) + 4 (m read) + 4 (EMA candidate write)
 MAX_DISTINCT = 24               # distinct input tensors per kind kept resident
+FOUR_METRIC_BYTES = 12          # a verified tensor with the sliced Wasserstein distance: x twice, the reference read and written
 # dram__bytes_read.sum + dram__bytes_write.sum per element of the current stream_kernel, from the
 # ncu capture summarised in profiles/stream_kernel_cfg3_ncu_full.md (B=8 x 4096 x 4096; traffic
 # grows in proportion to the element count, so a launch of N elements moves this times N).
@@ -51,10 +52,12 @@ def measured_peak_gbs():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+    """Samples SM clocks and throttle reasons with nvidia-smi while the benchmark runs; a summary
+    is taken over the samples that fall inside a wall-clock window (the timed region)."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    BAD = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
 
     def __init__(self, index: int):
         self.index, self.lines, self.proc = index, [], None
@@ -73,35 +76,46 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
     def __exit__(self, *exc):
         if self.proc:
-            time.sleep(0.15)
             self.proc.terminate()          # the exact process started above
             try:
                 self.proc.wait(timeout=5)
             except subprocess.TimeoutExpired:
                 self.proc.kill()
 
-    def summary(self) -> dict:
-        sm, smax, reasons = [], [], set()
+    @staticmethod
+    def _when(stamp: str, fallback: float) -> float:
+        try:                               # "2026/01/31 12:00:00.123", the sampler's own clock
+            head, _, ms = stamp.partition(".")
+            return time.mktime(time.strptime(head, "%Y/%m/%d %H:%M:%S")) + (float("0." + ms) if ms else 0.0)
+        except ValueError:
+            return fallback
+
+    def summary(self, t0: float | None = None, t1: float | None = None) -> dict:
+        """Median SM clock and the throttle reasons seen between wall-clock times t0 and t1 (all
+        samples if no window is given or none fell inside it)."""
+        rows = []
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        for seen, line in list(self.lines):
             tok = [t.strip() for t in line.split(",")]
-            if len(tok) < 6:
+            if len(tok) < 7:
                 continue
             try:
-                sm.append(float(tok[0]))
-                smax.append(float(tok[1]))
+                rows.append((self._when(tok[0], seen), float(tok[1]), float(tok[2]),
+                             [n for n, v in zip(names, tok[3:7]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, val in zip(names, tok[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        inside = [r for r in rows if t0 is not None and t0 - 0.02 <= r[0] <= t1 + 0.02]
+        used, window = (inside, "timed region") if inside else (rows, "whole run")
+        sm = sorted(r[1] for r in used)
+        reasons = sorted({n for r in used for n in r[3]})
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None,
+                "sm_max_mhz": max((r[2] for r in used), default=None),
+                "samples": len(sm), "window": window, "reasons": reasons,
+                "rejected": any(n in self.BAD for n in reasons)}
 
 
 def build_stream(w, boundary, device, count, distinct):
@@ -116,12 +130,38 @@ def build_stream(w, boundary, device, count, distinct):
     return xs
 
 
-def run_ours(args, rank, world, local_rank):
-    from paper_2603_03592_b200 import binding
-    binding.lib()                                   # no library, no benchmark: there is no fallback
-    torch.cuda.set_device(local_rank)
+MIN_TIMED_MS = 200.0            # device time the timed region covers at least, whatever --steps is
+
+
+def timed_calls(fn, stream, min_ms=60.0, min_calls=6, max_calls=400):
+    """Median and best duration (ms) of fn(i), one CUDA-event pair per call on `stream`, over at
+    least min_calls calls and min_ms of device time."""
+    durations = []
+    i = 0
+    while True:
+        batch = min_calls if not durations else max(2, min(64, int(min_calls * 1.5)))
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(batch + 1)]
+        marks[0].record(stream)
+        for k in range(batch):
+            fn(i)
+            i += 1
+            marks[k + 1].record(stream)
+        torch.cuda.synchronize()
+        durations += [marks[k].elapsed_time(marks[k + 1]) for k in range(batch)]
+        if (sum(durations) >= min_ms and len(durations) >= min_calls) or len(durations) >= max_calls:
+            break
+    durations.sort()
+    return durations[len(durations) // 2], durations[0], len(durations)
+
+
+class Measured:
+    """What measure_workload leaves behind for the figures taken after the timed region."""
+
+
+def measure_workload(binding, w, args, rank, world, local_rank, sampler, steps, warmup, min_ms, distinct):
+    """The timed region of one workload: `steps` verified microbatches per boundary (h and g each),
+    repeated until at least min_ms of device time have passed.  Returns (figures, Measured)."""
     device = torch.device("cuda", local_rank)
-    w = synth.WORKLOADS[args.workload]
     N = w.B * w.T * w.d
     nb = w.boundaries                               # independent stage boundaries, one stream each
     main = torch.cuda.current_stream()
@@ -135,19 +175,18 @@ def run_ours(args, rank, world, local_rank):
                 v.sentinel_update_reference(synth.clean(w, b, kind, t, device), kind)
     torch.cuda.synchronize()
 
-    total = args.warmup + args.steps
-    distinct = args.distinct if nb == 1 else min(args.distinct, 12)   # 8 boundaries: bound the footprint
-    xs = [build_stream(w, b, device, total, distinct) for b in range(nb)]
+    distinct = distinct if nb == 1 else min(distinct, 12)   # 8 boundaries: bound the footprint
+    xs = [build_stream(w, b, device, warmup + steps, distinct) for b in range(nb)]
     nd = len(xs[0][ACT])
     scores = torch.empty(nb, 2, 1 + w.B, 3, dtype=torch.float32, device=device)
     flags = torch.empty(nb, 2, 1 + w.B, dtype=torch.int32, device=device)
-    flag_log = torch.zeros(total, nb, 2, 1 + w.B, dtype=torch.int32, device=device)   # every step's flags
+    flag_log = torch.zeros(nd, nb, 2, 1 + w.B, dtype=torch.int32, device=device)   # flags of the last pass over each input
     torch.cuda.synchronize()
 
     def step(i):
         for b, (v, s) in enumerate(zip(vs, streams)):
-            v.sentinel_verify(xs[b][ACT][i % nd], ACT, scores[b, 0], flag_log[i, b, 0], s)
-            v.sentinel_verify(xs[b][GRAD][i % nd], GRAD, scores[b, 1], flag_log[i, b, 1], s)
+            v.sentinel_verify(xs[b][ACT][i % nd], ACT, scores[b, 0], flag_log[i % nd, b, 0], s)
+            v.sentinel_verify(xs[b][GRAD][i % nd], GRAD, scores[b, 1], flag_log[i % nd, b, 1], s)
 
     def fork():                                      # side streams start after `main` gets here
         if nb > 1:
@@ -164,78 +203,161 @@ def run_ours(args, rank, world, local_rank):
                 main.wait_event(ev)
 
     fork()
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(i)
     join()
     torch.cuda.synchronize()
-    replicas.barrier()
-    torch.cuda.synchronize()
 
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    with ClockSampler(local_rank) as clocks:
-        marks[0].record(main)
-        fork()
-        for i in range(args.steps):
-            step(args.warmup + i)
-            if nb == 1:
-                marks[i + 1].record(main)
-        join()
-        if nb > 1:
-            marks[-1].record(main)
-        torch.cuda.synchronize()
+    # how often the list of `steps` steps is gone through: an estimate from a short untimed pass
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(main)
+    fork()
+    for i in range(min(steps, 4)):
+        step(warmup + i)
+    join()
+    e1.record(main)
+    torch.cuda.synchronize()
+    est_ms = e0.elapsed_time(e1) / min(steps, 4)
+    repeats = max(1, int(-(-min_ms // max(est_ms * steps, 1e-3))))
+    repeats = int(replicas.max_over_ranks(repeats))      # every rank times the same number of steps
+    timed = steps * repeats
+
     replicas.barrier()
     torch.cuda.synchronize()
-    local_ms = elapsed_ms = marks[0].elapsed_time(marks[-1])
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(timed + 1)]
+    t_wall0 = time.time()
+    marks[0].record(main)
+    fork()
+    for i in range(timed):
+        step(warmup + (i % steps))
+        if nb == 1:
+            marks[i + 1].record(main)
+    join()
+    if nb > 1:
+        marks[-1].record(main)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    replicas.barrier()
+    torch.cuda.synchronize()
+    local_ms = marks[0].elapsed_time(marks[-1])
     if nb == 1:
-        step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+        step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(timed))
     else:
-        step_ms = [local_ms / args.steps]
-    elapsed_ms = replicas.max_over_ranks(elapsed_ms)
-    launches = 2 * args.steps * nb
-    violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
-    # what the detector said on the timed steps (reported, not a target: some of the recipe's
-    # corruptions are statistically invisible to these metrics, and a flagged tensor that comes
-    # round again is flagged again)
-    raised = ((flag_log[args.warmup:] & 0xFFFF) != 0).any(dim=-1).cpu()              # [steps, nb, 2]
+        step_ms = [local_ms / timed]
+    elapsed_ms = replicas.max_over_ranks(local_ms)
+    launches = 2 * timed * nb
+    time.sleep(0.05)                                 # let the sampler's last lines arrive
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    # what the detector said on the last pass over the inputs (reported, not a target: some of the
+    # recipe's corruptions are statistically invisible to these metrics, and a flagged tensor that
+    # comes round again is flagged again)
+    raised = ((flag_log & 0xFFFF) != 0).any(dim=-1).cpu()                       # [nd, nb, 2]
     n_corrupted = n_flagged = n_both = 0
-    for i in range(args.steps):
+    seen = min(nd, steps)
+    for i in range(seen):
         for b in range(nb):
             for kind in (ACT, GRAD):
-                c = xs[b]["corrupted"][kind][(args.warmup + i) % nd]
-                f = bool(raised[i, b, kind])
+                c = xs[b]["corrupted"][kind][(warmup + i) % nd]
+                f = bool(raised[(warmup + i) % nd, b, kind])
                 n_corrupted += c
                 n_flagged += f
                 n_both += c and f
-    detection = {"tensors": args.steps * nb * 2, "corrupted": n_corrupted, "flagged": n_flagged,
+    detection = {"tensors": seen * nb * 2, "corrupted": n_corrupted, "flagged": n_flagged,
                  "corrupted_and_flagged": n_both, "distinct_tensors_per_kind": nd,
-                 "note": "the stream cycles through the distinct tensors; one that comes round again soon "
-                         "correlates with the reference that absorbed it and is flagged as a replay"}
+                 "note": "verdicts of the last pass over the distinct tensors; the stream cycles through them, and "
+                         "one that comes round again soon correlates with the reference that absorbed it and is "
+                         "flagged as a replay"}
 
-    # extra figure, outside the timed region: gradient replacement (Alg. 4) after a flagged step
+    bytes_step = 2 * N * BYTES_PER_ELEMENT * nb             # two tensors per boundary per step
+    cycle_bytes = nb * nd * 2 * N * BYTES_PER_ELEMENT       # one pass over the cycled inputs, against the 126 MB L2
+    if cycle_bytes > 4 * 126e6:
+        l2_note = "inputs larger than L2: %d MiB read+written per launch, %d distinct tensors per kind" % (
+            N * BYTES_PER_ELEMENT >> 20, nd)
+    else:
+        l2_note = ("inputs and state of a whole cycle (%d MiB) stay near the 126 MB L2: a launch-latency figure, "
+                   "not a bandwidth figure" % (cycle_bytes >> 20))
+    gbs = world * timed * bytes_step / (elapsed_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak_gbs()
+    kernel_ms = local_ms / launches                         # the timed region holds these launches only
+    achieved = N * BYTES_PER_ELEMENT / (kernel_ms * 1e-3) / 1e9
+    fig = {
+        "value": round(gbs, 1), "ms_per_step": round(elapsed_ms / timed, 4),
+        "ms_per_step_median": round(step_ms[len(step_ms) // 2], 4), "ms_per_step_best": round(step_ms[0], 4),
+        "timed_steps": timed, "repeats": repeats, "timed_ms": round(elapsed_ms, 2),
+        "microbatches_per_s": round(world * timed * nb / (elapsed_ms * 1e-3), 1),
+        "tensor_gbs": round(world * timed * nb * 2 * N * 2 / (elapsed_ms * 1e-3) / 1e9, 1),
+        "frac_of_8000_nominal": round(gbs / world / 8000.0, 4),
+        "gpu_launches": launches, "detection": detection, "clocks": clocks, "l2": l2_note,
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "peak_source": "%s copy bandwidth" % peak_kind,
+                     "kernel": "stream_kernel", "avg_launch_ms": round(kernel_ms, 4),
+                     "note": ("launches of different boundaries overlap: time per launch is the "
+                              "timed region divided by the launches" if nb > 1 else
+                              "timed region / launches; the region holds these launches only"),
+                     "traffic": (args.traffic if args.traffic is not None else
+                                 (round(NCU_DRAM_BYTES_PER_ELEMENT * N) if NCU_DRAM_BYTES_PER_ELEMENT else None)),
+                     "traffic_source": "ncu on B=8x4096x4096, scaled by element count"},
+    }
+    m = Measured()
+    m.vs, m.xs, m.nd, m.N, m.nb, m.scores, m.flags, m.main, m.device = vs, xs, nd, N, nb, scores, flags, main, device
+    m.bytes_step = bytes_step
+    return fig, m
+
+
+def workload_text(w):
+    nb = w.boundaries
+    return "%s: B=%d x T=%d x d=%d bf16, activations %s, gradients N(0,%g), %g%% corrupted%s" % (
+        w.name, w.B, w.T, w.d, w.act, w.grad_std, 100 * w.corrupt_rate,
+        ", %d boundaries on %d CUDA streams" % (nb, nb) if nb > 1 else "")
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2603_03592_b200 import binding
+    binding.lib()                                   # no library, no benchmark: there is no fallback
+    torch.cuda.set_device(local_rank)
+    w = synth.WORKLOADS[args.workload]
+    with ClockSampler(local_rank) as sampler:
+        fig, m = measure_workload(binding, w, args, rank, world, local_rank, sampler, args.steps, args.warmup,
+                                  args.min_ms, args.distinct)
+        if fig["clocks"]["rejected"]:               # a thermal or hardware slowdown: measured again, once
+            for v in m.vs:
+                v.sentinel_destroy()
+            del m
+            torch.cuda.empty_cache()
+            first = fig["clocks"]
+            fig, m = measure_workload(binding, w, args, rank, world, local_rank, sampler, args.steps, args.warmup,
+                                      args.min_ms, args.distinct)
+            fig["clocks"]["first_attempt"] = first
+        out = run_after_timed_region(binding, w, args, rank, world, local_rank, fig, m, sampler)
+    return out
+
+
+def run_after_timed_region(binding, w, args, rank, world, local_rank, fig, m, sampler):
+    vs, xs, nd, N, nb, scores, flags, main, device = m.vs, m.xs, m.nd, m.N, m.nb, m.scores, m.flags, m.main, m.device
+    violations = sum(int(v.sentinel_get_counters()["violations"]) for v in vs)
+
+    # The figures below are taken outside the timed region, each over at least 60 ms of device
+    # time: the median of per-call CUDA-event durations on the launching stream.
     extras = nb == 1 and args.extras and world == 1     # the extra figures are single-GPU figures
-    replace = None
-    if extras:
+    extra_keys = {}
+    pick1 = lambda i: xs[0][ACT][i % nd]
+
+    if extras:   # gradient replacement (Alg. 4) after a flagged step
         v0 = vs[0]
         loud = (xs[0][GRAD][0].float() * 64.0).to(torch.bfloat16)
         v0.sentinel_verify(loud, GRAD, scores[0, 1], flags[0, 1], main)       # flagged: no commit
         outs = [torch.empty_like(loud) for _ in range(4)]
         for o in outs:
             v0.sentinel_replace_if_flagged(o, GRAD, 0, None, main)
-        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        r0.record(main)
-        for i in range(12):
-            v0.sentinel_replace_if_flagged(outs[i % 4], GRAD, 0, None, main)
-        r1.record(main)
-        torch.cuda.synchronize()
-        rms = r0.elapsed_time(r1) / 12
-        replace = {"kernel": "replace_kernel", "bytes_per_element": 6, "ms_per_launch": round(rms, 4),
-                   "achieved_gbs": round(6 * N / (rms * 1e-3) / 1e9, 1),
-                   "flagged": bool(int(flags[0, 1, 0]) & 0xFFFF)}
+        rms, rbest, rn = timed_calls(lambda i: v0.sentinel_replace_if_flagged(outs[i % 4], GRAD, 0, None, main), main)
+        extra_keys["gradient_replacement"] = {
+            "kernel": "replace_kernel", "bytes_per_element": 6, "ms_per_launch": round(rms, 4),
+            "ms_best": round(rbest, 4), "calls": rn, "achieved_gbs": round(6 * N / (rms * 1e-3) / 1e9, 1),
+            "flagged": bool(int(flags[0, 1, 0]) & 0xFFFF)}
+        del outs, loud
 
-    # extra figure, outside the timed region: sliced Wasserstein distance along 8 directions
-    swd = None
-    if extras and 8 * w.d * 2 <= 200 * 1024 and w.T <= 16384:
+    if extras and 8 * w.d * 2 <= 200 * 1024 and w.T <= 16384:   # sliced Wasserstein distance along 8 directions
         g = torch.Generator(device=device).manual_seed(11)
         u = torch.randn(8, w.d, generator=g, device=device)
         u = (u / u.norm(dim=1, keepdim=True)).to(torch.bfloat16).contiguous()
@@ -243,43 +365,27 @@ def run_ours(args, rank, world, local_rank):
         sw = torch.empty(1 + w.B, dtype=torch.float32, device=device)
         for _ in range(2):
             binding.sentinel_sliced_wasserstein(xs[0][ACT][0], ref, u, sw, main)
-        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        s0.record(main)
-        for i in range(8):
-            binding.sentinel_sliced_wasserstein(xs[0][ACT][i % nd], ref, u, sw, main)
-        s1.record(main)
-        torch.cuda.synchronize()
-        sms = s0.elapsed_time(s1) / 8
-        swd = {"directions": 8, "bytes_per_element": 6, "ms_per_call": round(sms, 4),
-               "achieved_gbs": round(6 * N / (sms * 1e-3) / 1e9, 1),
+        sms, sbest, sn = timed_calls(lambda i: binding.sentinel_sliced_wasserstein(pick1(i), ref, u, sw, main), main)
+        swd = {"directions": 8, "bytes_per_element": 6, "ms_per_call": round(sms, 4), "ms_best": round(sbest, 4),
+               "calls": sn, "achieved_gbs": round(6 * N / (sms * 1e-3) / 1e9, 1),
                "kernels": "swd_project_kernel + sort, merge, finish", "value_row0": float(sw[0])}
         del ref
-        # the same distance as the verifier's fourth metric: one verified tensor per call, the
-        # projection / sort chain (x only: the reference's projections are carried along) followed by
-        # the streaming launch: 2 + 6 B/element read, 4 written
+        # the same distance as the verifier's fourth metric: one verified tensor per call
         v4 = binding.Verifier(w.B, w.T, w.d, device=local_rank)
         v4.sentinel_set_directions(u, main)
         s4 = torch.empty(1 + w.B, 4, dtype=torch.float32, device=device)
         f4 = torch.zeros(1 + w.B, dtype=torch.int32, device=device)
         for i in range(4):
-            v4.sentinel_update_reference(xs[0][ACT][i % nd], ACT, s4, main)
-        v4.sentinel_verify(xs[0][ACT][4 % nd], ACT, s4, f4, main)
-        torch.cuda.synchronize()
-        s0.record(main)
-        for i in range(8):
-            v4.sentinel_verify(xs[0][ACT][(5 + i) % nd], ACT, s4, f4, main)
-        s1.record(main)
-        torch.cuda.synchronize()
-        vms = s0.elapsed_time(s1) / 8
-        swd["verify_with_four_metrics"] = {"ms_per_tensor": round(vms, 4), "bytes_per_element": 12,
-                                           "achieved_gbs": round(12 * N / (vms * 1e-3) / 1e9, 1)}
+            v4.sentinel_update_reference(pick1(i), ACT, s4, main)
+        v4.sentinel_verify(pick1(4), ACT, s4, f4, main)
+        vms, vbest, vn = timed_calls(lambda i: v4.sentinel_verify(pick1(5 + i), ACT, s4, f4, main), main)
+        swd["verify_with_four_metrics"] = {"ms_per_tensor": round(vms, 4), "ms_best": round(vbest, 4), "calls": vn,
+                                           "bytes_per_element": FOUR_METRIC_BYTES,
+                                           "achieved_gbs": round(FOUR_METRIC_BYTES * N / (vms * 1e-3) / 1e9, 1)}
         v4.close()
+        extra_keys["sliced_wasserstein"] = swd
 
-    # extra figure, outside the timed region: one iteration with R workers of the stage
-    # (one launch: 2R B/element of tensors + 4 B read and 4 B written of the reference)
-    replicas_fig = None
-    if extras:
+    if extras:   # one iteration with R workers of the stage (2R B/element of tensors + the reference read and written)
         R = 4 if 100 * 4 * (w.B + 1) <= 4096 else 2
         vr = binding.Verifier(w.B, w.T, w.d, device=local_rank, n_workers=R)
         rs = torch.empty(R, 1 + w.B, 3, dtype=torch.float32, device=device)
@@ -288,116 +394,49 @@ def run_ours(args, rank, world, local_rank):
         for i in range(4):
             vr.sentinel_update_reference_replicas(pick(i), ACT, rs, rf, main)
         vr.sentinel_verify_replicas(pick(4), ACT, rs, rf, main)
-        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        q0.record(main)
-        for i in range(6):
-            vr.sentinel_verify_replicas(pick(5 + i), ACT, rs, rf, main)
-        q1.record(main)
-        torch.cuda.synchronize()
-        qms = q0.elapsed_time(q1) / 6
-        per_el = 2 * R + 8                      # every tensor once, the reference read and written once
-        flagged_workers = int(((rf[:, 0] & 0xFFFF) != 0).sum())
-        replicas_fig = {"workers": R, "bytes_per_element": per_el, "ms_per_iteration": round(qms, 4),
-                        "achieved_gbs": round(per_el * N / (qms * 1e-3) / 1e9, 1),
-                        "submissions_per_s": round(R / (qms * 1e-3), 1),
-                        "flagged_workers_last_iteration": flagged_workers,
-                        "kernels": "replica_kernel (all workers, speculative mean) + ema_mean_kernel (report bits)"}
+        qms, qbest, qn = timed_calls(lambda i: vr.sentinel_verify_replicas(pick(5 + i), ACT, rs, rf, main), main)
+        per_el = 2 * R + 8
+        extra_keys["multi_worker_iteration"] = {
+            "workers": R, "bytes_per_element": per_el, "ms_per_iteration": round(qms, 4), "ms_best": round(qbest, 4),
+            "calls": qn, "achieved_gbs": round(per_el * N / (qms * 1e-3) / 1e9, 1),
+            "submissions_per_s": round(R / (qms * 1e-3), 1),
+            "flagged_workers_last_iteration": int(((rf[:, 0] & 0xFFFF) != 0).sum()),
+            "error_word": int(vr.sentinel_get_counters()["error"]),
+            "kernels": "replica_kernel (all workers, speculative mean) + ema_mean_kernel (report bits)"}
         vr.sentinel_destroy()
 
-    # extra figure, outside the timed region: the reference kept as bf16 (6 B/element per tensor)
-    half = None
-    if extras:
-        vh = binding.Verifier(w.B, w.T, w.d, device=local_rank, ema_bf16=1)
-        hs_, hf_ = torch.empty(1 + w.B, 3, dtype=torch.float32, device=device), torch.zeros(1 + w.B, dtype=torch.int32, device=device)
+    def single_variant(name, per_el, kernel, **kw):   # a verifier option, one verified tensor per call
+        v = binding.Verifier(w.B, w.T, w.d, device=local_rank, **kw)
+        s_, f_ = (torch.empty(1 + w.B, 3, dtype=torch.float32, device=device),
+                  torch.zeros(1 + w.B, dtype=torch.int32, device=device))
         for i in range(6):
-            vh.sentinel_update_reference(xs[0][ACT][i % nd], ACT, hs_, main)
-        vh.sentinel_verify(xs[0][ACT][6 % nd], ACT, hs_, hf_, main)
-        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        h0.record(main)
-        for i in range(20):
-            vh.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, hs_, hf_, main)
-        h1.record(main)
-        torch.cuda.synchronize()
-        hms = h0.elapsed_time(h1) / 20
-        half = {"bytes_per_element": 6, "ms_per_launch": round(hms, 4),
-                "achieved_gbs": round(6 * N / (hms * 1e-3) / 1e9, 1),
-                "tensors_per_s": round(1e3 / hms, 1), "kernel": "stream_kernel_t<false, true>"}
-        vh.sentinel_destroy()
+            v.sentinel_update_reference(pick1(i), ACT, s_, main)
+        v.sentinel_verify(pick1(6), ACT, s_, f_, main)
+        ms, best, n = timed_calls(lambda i: v.sentinel_verify(pick1(7 + i), ACT, s_, f_, main), main)
+        err = int(v.sentinel_get_counters()["error"])
+        v.sentinel_destroy()
+        return {"bytes_per_element": per_el, "ms_per_launch": round(ms, 4), "ms_best": round(best, 4), "calls": n,
+                "achieved_gbs": round(per_el * N / (ms * 1e-3) / 1e9, 1), "tensors_per_s": round(1e3 / ms, 1),
+                "error_word": err, "kernel": kernel}
 
-    # extra figure, outside the timed region: one [T,d] reference for all samples (2 + 8/B B/element)
-    shared = None
-    if extras and w.B <= 16:
-        vsr = binding.Verifier(w.B, w.T, w.d, device=local_rank, ref_over_batch=1)
-        ss_, sf_ = torch.empty(1 + w.B, 3, dtype=torch.float32, device=device), torch.zeros(1 + w.B, dtype=torch.int32, device=device)
-        for i in range(6):
-            vsr.sentinel_update_reference(xs[0][ACT][i % nd], ACT, ss_, main)
-        vsr.sentinel_verify(xs[0][ACT][6 % nd], ACT, ss_, sf_, main)
-        z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        z0.record(main)
-        for i in range(20):
-            vsr.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, ss_, sf_, main)
-        z1.record(main)
-        torch.cuda.synchronize()
-        zms = z0.elapsed_time(z1) / 20
-        per_el = 2 + 8.0 / w.B
-        shared = {"bytes_per_element": per_el, "ms_per_launch": round(zms, 4),
-                  "achieved_gbs": round(per_el * N / (zms * 1e-3) / 1e9, 1),
-                  "tensors_per_s": round(1e3 / zms, 1), "kernel": "shared_ref_kernel"}
-        vsr.sentinel_destroy()
-
-    # extra figure, outside the timed region: one [d] reference for all tokens (x alone streams, 2 B/element)
-    channel = None
     if extras:
-        vcr = binding.Verifier(w.B, w.T, w.d, device=local_rank, ref_over_batch=1, ref_over_tokens=1)
-        cs_, cf_ = torch.empty(1 + w.B, 3, dtype=torch.float32, device=device), torch.zeros(1 + w.B, dtype=torch.int32, device=device)
-        for i in range(6):
-            vcr.sentinel_update_reference(xs[0][ACT][i % nd], ACT, cs_, main)
-        vcr.sentinel_verify(xs[0][ACT][6 % nd], ACT, cs_, cf_, main)
-        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        q0.record(main)
-        for i in range(20):
-            vcr.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, cs_, cf_, main)
-        q1.record(main)
-        torch.cuda.synchronize()
-        qms = q0.elapsed_time(q1) / 20
-        channel = {"bytes_per_element": 2, "ms_per_step": round(qms, 4),
-                   "achieved_gbs": round(2 * N / (qms * 1e-3) / 1e9, 1),
-                   "tensors_per_s": round(1e3 / qms, 1), "kernels": "channel_ref_kernel + channel_mean_kernel"}
-        vcr.sentinel_destroy()
-        # the same with a vector per sample ([B,d])
-        vps = binding.Verifier(w.B, w.T, w.d, device=local_rank, ref_over_tokens=1)
-        for i in range(6):
-            vps.sentinel_update_reference(xs[0][ACT][i % nd], ACT, cs_, main)
-        vps.sentinel_verify(xs[0][ACT][6 % nd], ACT, cs_, cf_, main)
-        torch.cuda.synchronize()
-        q0.record(main)
-        for i in range(20):
-            vps.sentinel_verify(xs[0][ACT][(7 + i) % nd], ACT, cs_, cf_, main)
-        q1.record(main)
-        torch.cuda.synchronize()
-        channel["ms_per_step_vector_per_sample"] = round(q0.elapsed_time(q1) / 20, 4)
-        vps.sentinel_destroy()
+        extra_keys["bf16_reference"] = single_variant("bf16", 6, "stream_kernel_t<false, true>", ema_bf16=1)
+        if w.B <= 16:
+            extra_keys["shared_reference"] = single_variant("shared", 2 + 8.0 / w.B, "shared_ref_kernel", ref_over_batch=1)
+        ch = single_variant("channel", 2, "channel_ref_kernel + channel_mean_kernel", ref_over_batch=1, ref_over_tokens=1)
+        ch["ms_per_step"] = ch.pop("ms_per_launch")
+        ch["ms_per_step_vector_per_sample"] = single_variant("channel_b", 2, "", ref_over_tokens=1)["ms_per_launch"]
+        extra_keys["channel_reference"] = ch
 
-    # extra figure, outside the timed region: the strided (compressed-signal) layout, rows d+1 apart
-    strided = None
-    if extras:
+    if extras:   # the strided (compressed-signal) layout, rows d+1 apart
         wide = [torch.nn.functional.pad(xs[0][ACT][i % nd], (0, 1)).contiguous() for i in range(3)]
         for i in range(2):
             vs[0].sentinel_update_reference_strided(wide[i], ACT, scores[0, 0], main)
-        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        c0.record(main)
-        for i in range(9):
-            vs[0].sentinel_update_reference_strided(wide[i % 3], ACT, scores[0, 0], main)
-        c1.record(main)
-        torch.cuda.synchronize()
-        cms = c0.elapsed_time(c1) / 9
-        strided = {"row_stride": w.d + 1, "bytes_per_element": 10, "ms_per_launch": round(cms, 4),
-                   "achieved_gbs": round(10 * N / (cms * 1e-3) / 1e9, 1), "kernel": "stream_kernel_t<false, false, true> (funnel-shifted rows)"}
+        cms, cbest, cn = timed_calls(lambda i: vs[0].sentinel_update_reference_strided(wide[i % 3], ACT, scores[0, 0], main), main)
+        extra_keys["compressed_layout"] = {
+            "row_stride": w.d + 1, "bytes_per_element": 10, "ms_per_launch": round(cms, 4), "ms_best": round(cbest, 4),
+            "calls": cn, "achieved_gbs": round(10 * N / (cms * 1e-3) / 1e9, 1),
+            "kernel": "stream_kernel_t<false, false, true> (funnel-shifted rows)"}
         del wide
 
     # end to end through the host-buffer entry point
@@ -419,74 +458,59 @@ def run_ours(args, rank, world, local_rank):
     e1.record(main)
     torch.cuda.synchronize()
     e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1))
+    error_word = max(int(v.sentinel_get_counters()["error"]) for v in vs)
     for v in vs:
         v.sentinel_destroy()
+    del hx
+    h2d_step = 2 * N * 2 * nb
+    e2e_gbs = world * e2e_steps * m.bytes_step / (e2e_ms * 1e-3) / 1e9
 
-    bytes_step = 2 * N * BYTES_PER_ELEMENT * nb             # two tensors per boundary per step
-    # what one pass over the cycled inputs touches, against the 126 MB L2
-    cycle_bytes = nb * nd * 2 * N * BYTES_PER_ELEMENT
-    if cycle_bytes > 4 * 126e6:
-        l2_note = "inputs larger than L2: %d MiB read+written per launch, %d distinct tensors per kind" % (
-            N * BYTES_PER_ELEMENT >> 20, nd)
-    else:
-        l2_note = ("inputs and state of a whole cycle (%d MiB) stay near the 126 MB L2: a launch-latency figure, "
-                   "not a bandwidth figure" % (cycle_bytes >> 20))
-    gbs = world * args.steps * bytes_step / (elapsed_ms * 1e-3) / 1e9
-    e2e_gbs = world * e2e_steps * bytes_step / (e2e_ms * 1e-3) / 1e9
-    peak, peak_kind = measured_peak_gbs()
-    kernel_ms = local_ms / launches              # the timed region holds these launches only
-    achieved = N * BYTES_PER_ELEMENT / (kernel_ms * 1e-3) / 1e9
     out = {
         "metric": "verified GB/s (x bf16 read + reference fp32 read + EMA fp32 write = 10 B/element)",
-        "value": round(gbs, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": round(elapsed_ms / args.steps, 4),
+        "value": fig["value"], "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": fig["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "impl": "sentinel_b200",
-        "config": {"workload": "%s: B=%d x T=%d x d=%d bf16, activations %s, gradients N(0,%g), "
-                               "%g%% corrupted%s" % (w.name, w.B, w.T, w.d, w.act, w.grad_std, 100 * w.corrupt_rate,
-                                                     ", %d boundaries on %d CUDA streams" % (nb, nb) if nb > 1 else ""),
+        "config": {"workload": workload_text(w),
                    "step": "sentinel_verify(h, ACT) + sentinel_verify(g, GRAD)" + (" on each boundary" if nb > 1 else ""),
-                   "l2": l2_note,
-                   "replicas": world},
-        "microbatches_per_s": round(world * args.steps * nb / (elapsed_ms * 1e-3), 1),
-        "tensor_gbs": round(world * args.steps * nb * 2 * N * 2 / (elapsed_ms * 1e-3) / 1e9, 1),
-        "ms_per_step_median": round(step_ms[len(step_ms) // 2], 4),
-        "ms_per_step_best": round(step_ms[0], 4),
-        "frac_of_8000_nominal": round(gbs / world / 8000.0, 4),
-        "gpu_launches": launches,
-        "violations_seen": violations, "detection": detection,
-        "clocks": clocks.summary(),
+                   "timed": "the %d steps gone through %d times (%d steps, %.0f ms of device time): at least %.0f ms "
+                            "whatever --steps is" % (args.steps, fig["repeats"], fig["timed_steps"], fig["timed_ms"], args.min_ms),
+                   "l2": fig["l2"], "replicas": world},
+        "timed_steps": fig["timed_steps"], "microbatches_per_s": fig["microbatches_per_s"],
+        "tensor_gbs": fig["tensor_gbs"], "ms_per_step_median": fig["ms_per_step_median"],
+        "ms_per_step_best": fig["ms_per_step_best"], "frac_of_8000_nominal": fig["frac_of_8000_nominal"],
+        "gpu_launches": fig["gpu_launches"], "violations_seen": violations, "error_word": error_word,
+        "detection": fig["detection"], "clocks": fig["clocks"],
         "e2e": {"value": round(e2e_gbs, 2), "unit": "GB/s", "steps": e2e_steps,
-                "h2d_bytes_per_step": 2 * N * 2 * nb,
-                "d2h_bytes_per_step": 2 * (1 + w.B) * (3 * 4 + 4) * nb,
+                "h2d_bytes_per_step": h2d_step, "d2h_bytes_per_step": 2 * (1 + w.B) * (3 * 4 + 4) * nb,
+                "bound": "pcie", "h2d_gbs": round(world * e2e_steps * h2d_step / (e2e_ms * 1e-3) / 1e9, 2),
+                "note": "one staging buffer: copy in, launch, copy out, in stream order; the host-to-device copy is "
+                        "what the time is spent on",
                 "api": "sentinel_verify_host"},
-        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                     "frac": round(achieved / peak, 4), "peak_source": "%s copy bandwidth" % peak_kind,
-                     "kernel": "stream_kernel",
-                     "avg_launch_ms": round(kernel_ms, 4),
-                     "note": ("launches of different boundaries overlap: time per launch is the "
-                              "timed region divided by the launches" if nb > 1 else
-                              "timed region / launches; the region holds these launches only"),
-                     "traffic": (args.traffic if args.traffic is not None else
-                                 (round(NCU_DRAM_BYTES_PER_ELEMENT * N) if NCU_DRAM_BYTES_PER_ELEMENT else None)),
-                     "traffic_source": "ncu on B=8x4096x4096, scaled by element count"},
+        "roofline": fig["roofline"],
     }
-    if replace is not None:
-        out["gradient_replacement"] = replace
-    if swd is not None:
-        out["sliced_wasserstein"] = swd
-    if replicas_fig is not None:
-        out["multi_worker_iteration"] = replicas_fig
-    if strided is not None:
-        out["compressed_layout"] = strided
-    if half is not None:
-        out["bf16_reference"] = half
-    if shared is not None:
-        out["shared_reference"] = shared
-    if channel is not None:
-        out["channel_reference"] = channel
+    out.update(extra_keys)
+
+    # the other stream configurations, after this one's buffers are gone: same measurement, shorter
+    if extras and args.workload == "cfg4" and args.also:
+        del xs, vs, m.xs, m.vs, scores, flags
+        torch.cuda.empty_cache()
+        for name in args.also.split(","):
+            wo = synth.WORKLOADS[name]
+            f2, m2 = measure_workload(binding, wo, args, rank, world, local_rank, sampler, min(args.steps, 24),
+                                      args.warmup, args.min_ms / 2, 12)
+            for v in m2.vs:
+                v.sentinel_destroy()
+            del m2
+            torch.cuda.empty_cache()
+            out[name] = {"workload": workload_text(wo), "value": f2["value"], "unit": "GB/s",
+                         "ms_per_launch": f2["roofline"]["avg_launch_ms"], "frac": f2["roofline"]["frac"],
+                         "frac_of_8000_nominal": f2["frac_of_8000_nominal"],
+                         "microbatches_per_s": f2["microbatches_per_s"], "ms_per_step_median": f2["ms_per_step_median"],
+                         "timed_steps": f2["timed_steps"], "gpu_launches": f2["gpu_launches"], "clocks": f2["clocks"]}
     if rank == 0 and args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
+        out["cpu_baseline"]["all_cores"] = cpu_baseline_all_cores(w, args.cpu_seconds)
     return out
 
 
@@ -519,6 +543,60 @@ def cpu_baseline(w, budget_s):
             "sample": "%d steps (h and g) of one sample [1,%d,%d] of the workload, float64, single thread"
                       % (done, ws.T, ws.d),
             "ms_per_step": round(1e3 * t_total / done, 1)}
+
+
+def _oracle_process(name, rows, index, budget_s, gate, results):
+    """One of the processes of cpu_baseline_all_cores: its own slice of the workload, its own oracle
+    verifier (unchanged, single-threaded), timed between a common start and its own end."""
+    torch.set_num_threads(1)
+    import oracle
+    ws = oracle_sample_shape(synth.WORKLOADS[name], rows)
+    v = oracle.Verifier(oracle.Params(B=ws.B, T=ws.T, d=ws.d))
+    for kind in (ACT, GRAD):
+        v.update_reference(synth.bits(synth.clean(ws, index, kind, 0)), kind)
+    xs = [(synth.bits(synth.clean(ws, index, ACT, 1 + i)), synth.bits(synth.clean(ws, index, GRAD, 1 + i)))
+          for i in range(2)]
+    gate.wait()                                      # every process starts its steps together
+    t0 = time.perf_counter()
+    done = 0
+    while time.perf_counter() - t0 < budget_s:
+        v.verify(xs[done % 2][0], ACT)
+        v.verify(xs[done % 2][1], GRAD)
+        done += 1
+    results.put((done, time.perf_counter() - t0, ws.B * ws.T * ws.d))
+    v.close()
+
+
+def cpu_baseline_all_cores(w, budget_s):
+    """The same oracle on every core this process may use: one process per core (started with
+    `spawn`: a fork after the first CUDA call would hang), each verifying its own slice."""
+    import multiprocessing as mp
+    cores = len(os.sched_getaffinity(0))
+    rows = 1024
+    ctx = mp.get_context("spawn")
+    gate, results = ctx.Barrier(cores), ctx.Queue()
+    procs = [ctx.Process(target=_oracle_process, args=(w.name, rows, i, min(budget_s, 10.0), gate, results))
+             for i in range(cores)]
+    for p in procs:
+        p.start()
+    got = []
+    try:
+        for _ in procs:
+            got.append(results.get(timeout=180 + budget_s))
+    except Exception as e:                            # a process died: report what there is
+        for p in procs:
+            p.terminate()
+        return {"unavailable": "all-cores run failed: %r" % (e,), "cores": cores}
+    for p in procs:
+        p.join()
+    steps = sum(g[0] for g in got)
+    wall = max(g[1] for g in got)
+    n = got[0][2]
+    return {"value": round(steps * 2 * n * BYTES_PER_ELEMENT / wall / 1e9, 4), "unit": "GB/s", "cores": cores,
+            "kind": "oracle",
+            "sample": "%d processes, one per core, each %d..%d steps (h and g) of its own slice [1,%d,%d] of the "
+                      "workload, float64, for %.0f s" % (cores, min(g[0] for g in got), max(g[0] for g in got),
+                                                         min(rows, w.T), w.d, wall)}
 
 
 def run_reference(args, rank, world):
@@ -574,6 +652,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-extras", dest="extras", action="store_false",
                     help="skip the extra figures measured after the timed region")
+    ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
+                    help="device time the timed region covers at least (the steps are gone through again)")
+    ap.add_argument("--also", default="cfg3,cfg5",
+                    help="workloads measured after the default one (cfg4) in the same run; '' for none")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the current kernel, if known")
     args = ap.parse_args()
