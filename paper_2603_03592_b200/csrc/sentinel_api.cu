@@ -278,8 +278,8 @@ int launch(sentinel_verifier *h, const StreamArgs &a, int grid, cudaStream_t s, 
   lc.attrs = &attr;
   lc.numAttrs = 1;
   if (h->chan_ref) {                               // x alone streams; the reference moves in a second launch
-    const size_t col_smem = (size_t)kWarps * kStripe * sizeof(float);      // the warps' column sums
-    if (lc.dynamicSmemBytes < col_smem) lc.dynamicSmemBytes = col_smem;
+    lc.blockDim = dim3(kChanThreads);
+    lc.dynamicSmemBytes = std::max(lc.dynamicSmemBytes, channel_smem_bytes());      // the warps' staging rings
     if (h->chan_per_sample) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel<true>, a));
     else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, channel_ref_kernel<false>, a));
     cudaLaunchConfig_t lm = lc;
@@ -648,9 +648,9 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     int occ = -1;
     cudaError_t oe = cudaSuccess;
     if (h->chan_ref) {
-      const size_t sm = std::max(smem, (size_t)kWarps * kStripe * sizeof(float));
-      if (h->chan_per_sample) resident_ctas(channel_ref_kernel<true>, kThreads, sm, &occ, &oe);
-      else resident_ctas(channel_ref_kernel<false>, kThreads, sm, &occ, &oe);
+      const size_t sm = std::max(smem, channel_smem_bytes());
+      if (h->chan_per_sample) resident_ctas(channel_ref_kernel<true>, kChanThreads, sm, &occ, &oe);
+      else resident_ctas(channel_ref_kernel<false>, kChanThreads, sm, &occ, &oe);
     } else if (h->shared_ref) {
       if (cfg->B <= kFewSets) resident_ctas(shared_ref_kernel<true>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
       else resident_ctas(shared_ref_kernel<false>, kThreads, smem, &occ, &oe);

@@ -190,6 +190,68 @@ __device__ __forceinline__ void store_m1(void *m, size_t idx, float v) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// staging through shared memory: bulk asynchronous copies that complete on an mbarrier
+//
+// A warp fills its own stages (one lane issues the copies) and is the only one to wait on them.
+// A wait that does not end -- it always should -- gives up after kStageWaitNs; the kernel then
+// records kErrStagingTimeout in HandleState.error and leaves the affected rows out.
+constexpr int kTileBytesM = 32 * kUnroll * 8 * 4; // a warp tile (512 elements) of an fp32 reference: 2048 bytes
+constexpr int kTileBytesX = 32 * kUnroll * 8 * 2; // and of a bf16 tensor: 1024 bytes
+constexpr unsigned long long kStageWaitNs = 2000000000ull;
+constexpr int kErrStagingTimeout = 1;             // HandleState.error: a staged copy did not arrive
+
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned arrivals) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+// global -> this CTA's shared memory, 16-byte aligned on both sides, a multiple of 16 bytes
+__device__ __forceinline__ void bulk_copy_in(unsigned dst, const void *src, unsigned bytes, unsigned bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned done;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done != 0u;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase `parity` of a stage's barrier; false if it did not complete in kStageWaitNs.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > kStageWaitNs) return false;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// sign mismatches on packed bf16 pairs
+//
+// With the sign bits of the two m's of a pair at bits 15 and 31 of `msp`, (w ^ msp) & 0x80008000
+// has a bit set per element of the pair whose sign bit differs from m's, and a byte-wise dot
+// product with ones adds them up, 0x80 = kFlipUnit each.  That is the count of sign(x) != sign(m)
+// as long as neither side holds an exact zero (a zero differs from any non-zero whatever its sign
+// bit): the caller makes sure of m beforehand and follows the smallest magnitude of x with
+// min_abs_bf16x2 to correct the count of a tile in which it reached zero.
+constexpr unsigned kFlipUnit = 128u;
+
+__device__ __forceinline__ unsigned min_abs_bf16x2(unsigned a, unsigned b) {   // per half: min(|a|, |b|), sign bit unspecified
+  unsigned r;
+  asm("min.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// ---------------------------------------------------------------------------------------------
 // per-element work
 
 struct GroupAcc {            // fp32 partial sums over one loop trip (<= 8*kUnroll elements)
@@ -265,7 +327,7 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
 // written to the segment's slot with the sample's tag and the shift the sums were taken about.
 __device__ __forceinline__ void reduce_to_slot(const ThreadAcc &t, int b, unsigned x0, unsigned m0bits,
                                                unsigned long long (*s_part)[kSlotWords], unsigned long long *slot) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = (int)blockDim.x >> 5;   // (<= kWarps)
   const double ws[6] = {warp_sum(t.sx), warp_sum(t.sxx), warp_sum(t.sm),
                         warp_sum(t.smm), warp_sum(t.sxm), warp_sum(t.ab)};
   const unsigned long long wf = warp_sum((unsigned long long)t.flips);
@@ -286,15 +348,15 @@ __device__ __forceinline__ void reduce_to_slot(const ThreadAcc &t, int b, unsign
     unsigned long long out;
     if (j < 6) {
       double sum = 0.;
-      for (int w = 0; w < kWarps; ++w) sum += __longlong_as_double((long long)s_part[w][j]);
+      for (int w = 0; w < n_warps; ++w) sum += __longlong_as_double((long long)s_part[w][j]);
       out = (unsigned long long)__double_as_longlong(sum);
     } else if (j == 6) {
       out = 0ull;
-      for (int w = 0; w < kWarps; ++w) out += s_part[w][6];
+      for (int w = 0; w < n_warps; ++w) out += s_part[w][6];
     } else {
       out = ((unsigned long long)(b + 1) << kTagShift) | ((unsigned long long)x0 << kX0Shift) |
             ((unsigned long long)m0bits << kM0Shift);       // sample tag and the shift of the sums
-      for (int w = 0; w < kWarps; ++w) out |= s_part[w][7];
+      for (int w = 0; w < n_warps; ++w) out |= s_part[w][7];
     }
     slot[j] = out;
   }
@@ -1140,95 +1202,155 @@ stream_kernel_t(const StreamArgs a) {
 // several stripes one after the other.  Each (stripe, phase) pair is a slot: its column sums go
 // to the CTA's block of `col_part`, and channel_mean_kernel adds the blocks up in a fixed order.
 constexpr int kStripe = 8 * 32 * kUnroll;        // columns per stripe
+constexpr int kChanThreads = 512;                 // threads per CTA of channel_ref_kernel: 16 warps, a stripe each at d = 8192
+constexpr int kChanWarps = kChanThreads / 32;
+constexpr int kChanRows = 4;                      // rows of a stripe that one stage holds
+constexpr int kChanDepth = 2;                     // stages per warp
 
 __host__ __device__ inline int channel_stripes(int d) { return (d + kStripe - 1) / kStripe; }
 __host__ __device__ inline int channel_phases(int d) {
   const int stripes = channel_stripes(d);
-  return stripes < kWarps ? kWarps / stripes : 1;
+  return stripes < kChanWarps ? kChanWarps / stripes : 1;
 }
 __host__ __device__ inline int channel_slots(int d) { return channel_stripes(d) * channel_phases(d); }
 
-// One slot (a warp's stripe of columns, every `phases`-th row from `first` on) of a segment.
-// Per element only what is not linear in x is done: (x - x0)^2, |x - m|, the sign test, the
-// non-finite / constancy bits, and the column sum of x - x0.  The linear sums follow from the
-// column sums when the slot is done: sum (x - x0) = sum_c col_c and sum (x - x0)(m - m0) =
-// sum_c (m_c - m0) col_c, since m is the same in every row.
-// kZeroInM = false is the usual case, no exact zero among this warp's columns of m: then
-// sign(x) != sign(m) iff x, with its sign bit flipped where m is negative, is <= +0 as an integer
-// (a negative number, -0, or +0: x and m differ in sign, or x is zero against a non-zero m).
-template <bool kZeroInM>
-__device__ __forceinline__ void channel_slot(const uint16_t *xseg, int d, int first, int rb, int phases,
-                                             const bool (&ok)[kUnroll],
-                                             const float4 *const (&mp)[kUnroll], float4 *col, unsigned x0pair,
-                                             float x0f, ThreadAcc &t, int &n_rows) {
-  // (xseg: this lane's first chunk in the first row of the segment; rows are counted from there)
-  // Two rows per trip; the next trip's rows are requested before this trip's arithmetic.  The
-  // reference (2 KB per warp, the same for every row) is fetched again each trip through L1
-  // rather than held in registers, which the second set of x would not leave room for.
-  uint4 cur[2][kUnroll], nxt[2][kUnroll];
-  auto fetch = [&](uint4 (&dst)[2][kUnroll], int row) {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int r = row + h * phases;
-      if (r < rb) {
-        const uint16_t *xr = xseg + (size_t)r * d;
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-          if (ok[u]) dst[h][u] = ld_x128(xr + (size_t)u * 256);
+// a warp's part of the dynamic shared memory: its ring of stages (kChanRows rows of its stripe,
+// 1 KB each, filled by bulk copies two stages ahead of the arithmetic) and their barriers
+struct __align__(128) ChanWarp {
+  unsigned char stage[kChanDepth][kChanRows * kTileBytesX];
+  unsigned long long bar[kChanDepth];
+};
+__host__ __device__ inline size_t channel_smem_bytes() { return (size_t)kChanWarps * sizeof(ChanWarp); }
+
+// what a warp carries from slot to slot
+struct ChanState {
+  unsigned stages_done;      // stages this warp has consumed since the launch: stage index and barrier phase follow from it
+  bool alive;                // false once a wait gave up
+};
+
+// Exact zeros of the staged rows whose sign bit equals that of m (the packed sign test did not
+// count them), and non-finite elements: the two rare looks at a stage, kept out of line.
+__device__ __noinline__ unsigned channel_uncounted_zeros(const unsigned char *stage, int rows, int lane, unsigned valid,
+                                                         const float *m_stripe) {
+  unsigned n = 0u;
+  for (int i = 0; i < rows; ++i)
+    for (int u = 0; u < kUnroll; ++u) {
+      if (!((valid >> u) & 1u)) continue;
+      const uint16_t *xw = reinterpret_cast<const uint16_t *>(stage + i * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+      const float *mw = m_stripe + (size_t)(u * 32 + lane) * 8;
+      for (int e = 0; e < 8; ++e) {
+        const unsigned xb = xw[e];
+        if ((xb & 0x7FFFu) == 0u && (xb >> 15) == (__float_as_uint(__ldg(mw + e)) >> 31)) ++n;
       }
     }
-  };
-  if (first < rb) fetch(cur, first);
-  for (int row = first; row < rb; row += 2 * phases) {
-    if (row + 2 * phases < rb) fetch(nxt, row + 2 * phases);
-    const bool second = row + phases < rb;
-    float g_sxx = 0.f, g_ab = 0.f;
-    unsigned g_flips = 0u;
-#pragma unroll
+  return n;
+}
+__device__ __noinline__ unsigned channel_nonfinite_in_stage(const unsigned char *stage, int rows, int lane, unsigned valid) {
+  unsigned nf = 0u;
+  for (int i = 0; i < rows; ++i)
     for (int u = 0; u < kUnroll; ++u) {
-      if (!ok[u]) continue;
-      const float4 lo = __ldg(mp[u]), hi = __ldg(mp[u] + 1);
-      const float mv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-      const float4 c_lo = col[u * 64], c_hi = col[u * 64 + 1];
-      float cs[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+      if (!((valid >> u) & 1u)) continue;
+      const uint4 w = *reinterpret_cast<const uint4 *>(stage + i * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+      nf |= (((w.x & 0x7F807F80u) + 0x00800080u) | ((w.y & 0x7F807F80u) + 0x00800080u) |
+             ((w.z & 0x7F807F80u) + 0x00800080u) | ((w.w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
+    }
+  return nf;
+}
+
+// One slot (a warp's stripe of columns, every `phases`-th row from `first` on) of a segment.
+// Per element only what is not linear in x is done: (x - x0)^2, |x - m|, the sign test on the
+// packed pairs, the constancy bits, and the column sum of x - x0.  The linear sums follow from
+// the column sums when the slot is done: sum (x - x0) = sum_c col_c and sum (x - x0)(m - m0) =
+// sum_c (m_c - m0) col_c, since m is the same in every row.  Non-finite elements show in the sum
+// of |x - m| (not a finite number then), exact zeros of x in the packed minimum: either is looked
+// at once per stage, and the stage is gone through again only if it shows.
+// kZeroInM = true (an exact zero among this warp's columns of m): the general sign test.
+template <bool kZeroInM>
+__device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_pitch, int n_rows, int vc,
+                                             const bool (&ok)[kUnroll], const F8 (&mv)[kUnroll],
+                                             const unsigned (&msp)[kUnroll][4], const float *m_stripe,
+                                             float (&cs)[kUnroll][8], unsigned x0pair, float x0f, ThreadAcc &t,
+                                             ChanWarp &cw, ChanState &st) {
+  // (xslot: the first element of the stripe in the slot's first row; rows are row_pitch elements apart)
+  const int lane = threadIdx.x & 31;
+  const int n_stages = (n_rows + kChanRows - 1) / kChanRows;
+  const unsigned valid = (ok[0] ? 1u : 0u) | (ok[1] ? 2u : 0u);
+  static_assert(kUnroll == 2, "two chunks per lane and row");
+  // the ring is addressed by the warp's running stage count, so that barrier phases carry on
+  // from slot to slot; `head` = count at which this slot's stage 0 is consumed
+  const unsigned head = st.stages_done;
+  auto fill = [&](int s) {
+    if (s < n_stages && lane == 0) {
+      const int rows = (n_rows - s * kChanRows < kChanRows) ? n_rows - s * kChanRows : kChanRows;
+      const unsigned k = head + (unsigned)s, slot = k % kChanDepth;
+      const unsigned bar = smem_addr(&cw.bar[slot]), dst = smem_addr(&cw.stage[slot][0]);
+      mbar_arrive_expect(bar, (unsigned)(rows * vc) * 16u);
+      for (int i = 0; i < rows; ++i)
+        bulk_copy_in(dst + i * kTileBytesX, xslot + (size_t)(s * kChanRows + i) * row_pitch, (unsigned)vc * 16u, bar);
+    }
+  };
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (h == 1 && !second) continue;
-        const unsigned w4[4] = {cur[h][u].x, cur[h][u].y, cur[h][u].z, cur[h][u].w};
+  for (int s = 0; s < kChanDepth; ++s) fill(s);
+
+  for (int s = 0; s < n_stages; ++s) {
+    const unsigned k = head + (unsigned)s, slot = k % kChanDepth;
+    if (!__all_sync(0xffffffffu, mbar_wait(smem_addr(&cw.bar[slot]), (k / kChanDepth) & 1u))) {
+      // the stage never arrived: wait out what else is in flight, then give up on the warp's rows
+      for (int q = 1; q < kChanDepth; ++q)
+        if (s + q < n_stages) mbar_wait(smem_addr(&cw.bar[(k + q) % kChanDepth]), ((k + q) / kChanDepth) & 1u);
+      st.alive = false;
+      st.stages_done = k;                                    // (nothing is issued any more)
+      return;
+    }
+    const unsigned char *stage = cw.stage[slot];
+    const int rows = (n_rows - s * kChanRows < kChanRows) ? n_rows - s * kChanRows : kChanRows;
+    float g_sxx = 0.f, g_ab = 0.f;
+    unsigned flips = 0u, zmin = 0x7F7F7F7Fu;
+    for (int i = 0; i < rows; ++i) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (!ok[u]) continue;
+        const uint4 w = *reinterpret_cast<const uint4 *>(stage + i * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+        const unsigned w4[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          t.nf_bits |= ((w4[q] & 0x7F807F80u) + 0x00800080u) & 0x80008000u;
           t.x_diff |= w4[q] ^ x0pair;
+          if (!kZeroInM) {
+            flips = __dp4a((w4[q] ^ msp[u][q]) & 0x80008000u, 0x01010101u, flips);
+            zmin = min_abs_bf16x2(zmin, w4[q]);
+          }
 #pragma unroll
           for (int hlf = 0; hlf < 2; ++hlf) {
             const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
-            const float mf = mv[2 * q + hlf];
+            const float mf = mv[u].v[2 * q + hlf];
             const float xs = xf - x0f;
             g_sxx = fmaf(xs, xs, g_sxx);
             g_ab += fabsf(xf - mf);
-            const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
-            if (kZeroInM) g_flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? 1u : 0u;
-            else g_flips += ((int)xt <= 0) ? 1u : 0u;
-            cs[2 * q + hlf] += xs;
+            if (kZeroInM) {
+              const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
+              flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? kFlipUnit : 0u;
+            }
+            cs[u][2 * q + hlf] += xs;
           }
         }
       }
-      col[u * 64] = make_float4(cs[0], cs[1], cs[2], cs[3]);
-      col[u * 64 + 1] = make_float4(cs[4], cs[5], cs[6], cs[7]);
     }
-    t.sxx += (double)g_sxx;
+    if (!kZeroInM && __any_sync(0xffffffffu, ((zmin & 0x7FFFu) == 0u) || ((zmin & 0x7FFF0000u) == 0u)))
+      flips += kFlipUnit * channel_uncounted_zeros(stage, rows, lane, valid, m_stripe);
+    if (__any_sync(0xffffffffu, !(g_ab <= 3.4028234664e38f)))
+      t.nf_bits |= channel_nonfinite_in_stage(stage, rows, lane, valid);
+    t.sxx += (double)g_sxx;                                  // the short fp32 runs into the fp64 sums
     t.ab += (double)g_ab;
-    t.flips += g_flips;
-    n_rows += second ? 2 : 1;
-#pragma unroll
-    for (int h = 0; h < 2; ++h)
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) cur[h][u] = nxt[h][u];
+    t.flips += flips / kFlipUnit;
+    // every lane has used what it read from the stage (the sums above depend on it): refill it
+    __syncwarp();
+    fill(s + kChanDepth);
   }
+  st.stages_done = head + (unsigned)n_stages;
 }
 
 __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long long rb, const float *m_in,
-                                float *col_seg, float *s_col, unsigned long long (*s_part)[kSlotWords],
+                                float *col_seg, ChanWarp &cw, ChanState &st, unsigned long long (*s_part)[kSlotWords],
                                 unsigned long long *slot) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunks = a.d >> 3;                   // d is a multiple of 8 here
@@ -1238,68 +1360,75 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
   const float x0f = __uint_as_float(x0 << 16);
   const unsigned m0bits = __float_as_uint(__ldg(m_in));
   const float m0 = __uint_as_float(m0bits);
+  const int seg_rows = (int)(rb - ra);
 
   ThreadAcc t = {0., 0., 0., 0., 0., 0., 0u, 0u, 0u, 0u};
-  for (int sl = warp; sl < n_slots; sl += kWarps) {
+  for (int sl = warp; sl < n_slots; sl += kChanWarps) {
     const int stripe = sl % stripes, phase = sl / stripes;
     bool ok[kUnroll];
-    const float4 *mp[kUnroll];                   // this lane's 8 + 8 columns of the reference
-    // the slot's column sums of x - x0 live in the warp's 2 KB of shared memory: a lane only ever
-    // touches its own 8 + 8 words there, so no barrier is needed
-    float4 *col = reinterpret_cast<float4 *>(s_col + warp * kStripe) + lane * 2;
+    F8 mv[kUnroll];                              // this lane's 8 + 8 columns of the reference
+    unsigned msp[kUnroll][4];                    // their sign bits, per pair at bits 15 and 31
+    float cs[kUnroll][8];                        // column sums of x - x0 over the slot's rows
     float lm = 0.f, lmm = 0.f;                   // this lane's sums of (m - m0), (m - m0)^2 over its columns
     unsigned m_diff = 0u;
     bool zero_in_m = false;
+    int vc = chunks - stripe * 32 * kUnroll;     // chunks of this stripe that exist
+    if (vc > 32 * kUnroll) vc = 32 * kUnroll;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int c = stripe * 32 * kUnroll + u * 32 + lane;
       ok[u] = c < chunks;
-      mp[u] = reinterpret_cast<const float4 *>(m_in) + (size_t)(ok[u] ? c : 0) * 2;
-      col[u * 64] = col[u * 64 + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { cs[u][e] = 0.f; mv[u].v[e] = 1.f; }
       if (ok[u]) {
-        const float4 lo = __ldg(mp[u]), hi = __ldg(mp[u] + 1);
-        const float mv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+        const float4 *mp = reinterpret_cast<const float4 *>(m_in) + (size_t)c * 2;
+        const float4 lo = __ldg(mp), hi = __ldg(mp + 1);
+        mv[u].v[0] = lo.x; mv[u].v[1] = lo.y; mv[u].v[2] = lo.z; mv[u].v[3] = lo.w;
+        mv[u].v[4] = hi.x; mv[u].v[5] = hi.y; mv[u].v[6] = hi.z; mv[u].v[7] = hi.w;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const float ms = mv[e] - m0;
+          const float ms = mv[u].v[e] - m0;
           lm += ms;
           lmm = fmaf(ms, ms, lmm);
-          m_diff |= __float_as_uint(mv[e]) ^ m0bits;
-          zero_in_m |= (mv[e] == 0.f);
+          m_diff |= __float_as_uint(mv[u].v[e]) ^ m0bits;
+          zero_in_m |= (mv[u].v[e] == 0.f);
         }
       }
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        msp[u][q] = __byte_perm(__float_as_uint(mv[u].v[2 * q]), __float_as_uint(mv[u].v[2 * q + 1]), 0x7733);
     }
-    int n_rows = 0;
-    const uint16_t *xseg = a.x + (size_t)ra * a.d + (size_t)(stripe * 32 * kUnroll + lane) * 8;
-    if (__any_sync(0xffffffffu, zero_in_m))
-      channel_slot<true>(xseg, a.d, phase, (int)(rb - ra), phases, ok, mp, col, x0pair, x0f, t, n_rows);
-    else
-      channel_slot<false>(xseg, a.d, phase, (int)(rb - ra), phases, ok, mp, col, x0pair, x0f, t, n_rows);
+    const int n_rows = (seg_rows - phase + phases - 1) / phases;      // rows phase, phase + phases, ... of the segment
+    const uint16_t *xslot = a.x + (size_t)(ra + phase) * a.d + (size_t)stripe * kStripe;
+    const float *m_stripe = m_in + (size_t)stripe * kStripe;
+    if (st.alive && n_rows > 0) {
+      if (__any_sync(0xffffffffu, zero_in_m))
+        channel_slot<true>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+      else
+        channel_slot<false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+    }
 
     // what is linear in x, from the column sums; the reference's own sums: its columns once per row
     float4 *dst = reinterpret_cast<float4 *>(col_seg + (size_t)sl * kStripe) + lane * 2;
     double s_x = 0., s_xm = 0.;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      const float4 c_lo = col[u * 64], c_hi = col[u * 64 + 1];
-      dst[u * 64] = c_lo;
-      dst[u * 64 + 1] = c_hi;
+      dst[u * 64] = make_float4(cs[u][0], cs[u][1], cs[u][2], cs[u][3]);
+      dst[u * 64 + 1] = make_float4(cs[u][4], cs[u][5], cs[u][6], cs[u][7]);
       if (ok[u]) {
-        const float4 lo = __ldg(mp[u]), hi = __ldg(mp[u] + 1);
-        const float mv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-        const float cs[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          s_x += (double)cs[e];
-          s_xm += (double)(mv[e] - m0) * (double)cs[e];
+          s_x += (double)cs[u][e];
+          s_xm += (double)(mv[u].v[e] - m0) * (double)cs[u][e];
         }
       }
     }
     t.sx += s_x;
     t.sxm += s_xm;
-    t.sm += (double)n_rows * (double)lm;
-    t.smm += (double)n_rows * (double)lmm;
-    if (n_rows) t.m_diff |= m_diff;
+    const int rows_done = (n_rows > 0) ? n_rows : 0;
+    t.sm += (double)rows_done * (double)lm;
+    t.smm += (double)rows_done * (double)lmm;
+    if (rows_done) t.m_diff |= m_diff;
   }
   reduce_to_slot(t, b, x0, m0bits, s_part, slot);
 }
@@ -1307,11 +1436,11 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
 // (kPerSample: a vector per sample, [B,d], instead of one, [d]; a kernel of its own so that the
 // code of either form does not depend on the other's addressing)
 template <bool kPerSample>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kChanThreads)
 channel_ref_kernel(const StreamArgs a) {
   __shared__ unsigned long long s_part[kWarps][kSlotWords];
   __shared__ int s_last;
-  extern __shared__ double s_dyn[];            // CTA 0: the refresh's working copies; the others: kWarps * kStripe floats
+  extern __shared__ __align__(128) double s_dyn[];   // CTA 0: the refresh's working copies; the others: the warps' staging rings
 
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -1325,6 +1454,16 @@ channel_ref_kernel(const StreamArgs a) {
       refresh_thresholds(ks, a.hist, a.sorted, a.cap0, a.cap1, a.units0, a.units1, a.n_metrics, a.a5, s_dyn);
   } else {
     const int c = blockIdx.x - 1;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    ChanWarp &cw = reinterpret_cast<ChanWarp *>(s_dyn)[warp];
+    if (lane == 0) {
+#pragma unroll
+      for (int k = 0; k < kChanDepth; ++k) mbar_init(smem_addr(&cw.bar[k]), 1u);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    ChanState st = {0u, true};
     const long long R = (long long)a.B * a.T;
     const long long R0 = (R * c) / a.G, R1 = (R * (c + 1)) / a.G;
     const size_t seg_floats = (size_t)channel_slots(a.d) * kStripe;
@@ -1336,14 +1475,14 @@ channel_ref_kernel(const StreamArgs a) {
         const int b = (int)(ra / a.T);
         const long long sample_end = (long long)(b + 1) * a.T;
         const long long rb = sample_end < R1 ? sample_end : R1;
-        channel_segment(a, b, ra, rb, kPerSample ? m_in + (size_t)b * a.d : m_in, col_seg,
-                        reinterpret_cast<float *>(s_dyn), s_part, slot);
+        channel_segment(a, b, ra, rb, kPerSample ? m_in + (size_t)b * a.d : m_in, col_seg, cw, st, s_part, slot);
         ra = rb;
       } else {                                    // no rows: nothing to add
-        for (size_t i = threadIdx.x; i < seg_floats; i += kThreads) col_seg[i] = 0.f;
+        for (size_t i = threadIdx.x; i < seg_floats; i += kChanThreads) col_seg[i] = 0.f;
         if (threadIdx.x == 0) slot[7] = 0ull;
       }
     }
+    if (!st.alive && lane == 0) atomicExch(&a.hs->error, kErrStagingTimeout);
   }
 
   __threadfence();
@@ -1534,11 +1673,7 @@ constexpr int kFoldTiles = 8;
 constexpr int kFewThreads = 512;                  // threads per CTA of the kernels that take this path
 constexpr int kFewWarps = kFewThreads / 32;
 constexpr int kStageDepth = 2;
-constexpr int kTileBytesM = 32 * kUnroll * 8 * 4; // a warp tile of the reference: 2048 bytes
-constexpr int kTileBytesX = 32 * kUnroll * 8 * 2; // and of a bf16 tensor: 1024 bytes
 constexpr int kStageBytes = kTileBytesM + kFewSets * kTileBytesX;
-constexpr unsigned long long kStageWaitNs = 2000000000ull;
-constexpr int kErrStagingTimeout = 1;             // HandleState.error: a staged copy did not arrive
 
 // A CTA's rows lie in one sample or straddle one boundary: two segments, each with its own shift
 // values, sums and slot.  A warp's tiles come in ascending row order, so it crosses over once.
@@ -1559,40 +1694,6 @@ struct __align__(128) FewWarp {                   // a warp's part of the dynami
 };
 __host__ __device__ inline size_t few_smem_bytes() { return (size_t)kFewWarps * sizeof(FewWarp); }
 
-__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned arrivals) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(arrivals) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect(unsigned bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
-}
-// global -> this CTA's shared memory, 16-byte aligned on both sides, a multiple of 16 bytes
-__device__ __forceinline__ void bulk_copy_in(unsigned dst, const void *src, unsigned bytes, unsigned bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
-  unsigned done;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-  return done != 0u;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Waits for the phase `parity` of a stage's barrier; false if it did not complete in kStageWaitNs.
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (;;) {
-    for (int i = 0; i < 64; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > kStageWaitNs) return false;
-  }
-}
-
 // One tensor's 8-element chunk against the chunk of m.  Sign mismatches are counted in units of
 // kFlipUnit.  kZeroInM = true: the general three-valued sign test, element by element.
 // kZeroInM = false (no exact zero in this chunk of m, the usual case): on the packed pairs --
@@ -1601,14 +1702,6 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
 // ones adds them up (0x80 each).  That is the mismatch count unless x holds an exact zero (a
 // zero counts as a mismatch whatever its sign bit): zmin follows the smallest magnitude of the
 // tensor's tile, and the caller corrects the count of a tile in which it reached zero.
-constexpr unsigned kFlipUnit = 128u;
-
-__device__ __forceinline__ unsigned min_abs_bf16x2(unsigned a, unsigned b) {   // per half: min(|a|, |b|), sign bit unspecified
-  unsigned r;
-  asm("min.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-  return r;
-}
-
 template <bool kZeroInM>
 __device__ __forceinline__ void few_chunk(const uint4 &cur, const F8 &mv, const unsigned (&msp)[4], float x0f, float m0,
                                           unsigned x0pair, float (&sum)[8], float &sx, float &sxx, float &sxm,
