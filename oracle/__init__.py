@@ -107,6 +107,8 @@ def lib():
         L.so_skip_tainted.argtypes = [C.c_void_p, C.c_int]
         L.so_skip_tainted.restype = None
         L.so_step_replicas.restype = C.c_int
+        L.so_count_violation.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
+        L.so_count_violation.restype = None
         L.so_worker_counters.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int)]
         L.so_worker_counters.restype = None
         L.so_reset_worker.argtypes = [C.c_void_p]
@@ -351,6 +353,10 @@ class Verifier:
     def skip_tainted(self, kind: int) -> None:
         """The worker this verifier follows was tainted at another stage in this step."""
         lib().so_skip_tainted(self._h, kind)
+
+    def count_violation(self, flagged: bool, severe: bool, r: int = 0) -> None:
+        """One step of worker r's violation counter (Sec. 3.1) without a submission."""
+        lib().so_count_violation(self._h, r, int(bool(flagged)), int(bool(severe)))
 
     def worker_counters(self, r: int) -> tuple[int, int, int]:
         out = (C.c_int * 3)()

@@ -429,7 +429,7 @@ void so_token_sums(const uint16_t *x, const double *m, size_t d, double out[4]) 
 }
 
 /* Sec. 3.1, violation counter with forgiveness, kept per worker */
-static void count_violation(so_verifier *v, int r, int flagged, int severe) {
+void so_count_violation(so_verifier *v, int r, int flagged, int severe) {
   const so_params *p = &v->p;
   if (flagged) {
     v->violations[r] += 1;
@@ -502,7 +502,7 @@ int so_verify(so_verifier *v, const uint16_t *x, int kind, double *scores, uint3
   }
 
   /* 4. violation counter with forgiveness */
-  count_violation(v, 0, any_flag, severe);
+  so_count_violation(v, 0, any_flag, severe);
 
   /* 5. clean units join the history; thresholds are refreshed for the next step */
   for (int r = 0; r < rows; ++r) {
@@ -583,7 +583,7 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
       if (f) any_flag = 1;
     }
     tainted[r] = any_flag;
-    if (!warmup) count_violation(v, r, any_flag, severe_w[r]);
+    if (!warmup) so_count_violation(v, r, any_flag, severe_w[r]);
     /* deviations of unflagged units join the pooled history (warm-up: of every unit, unless
      * the submission is non-finite) */
     if (!(warmup && any_flag))

@@ -183,6 +183,11 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
  * and it is marked flagged so that so_replace_if_flagged replaces the outgoing tensor. */
 void so_skip_tainted(so_verifier *v, int kind);
 void so_worker_counters(const so_verifier *v, int r, int out[3]);   /* v_r, streak, banned */
+/* Sec. 3.1, "Violation Counter with Forgiveness", one step of worker r's counter: a violation
+ * adds one and bans at c violations or on a severe deviation; T_forgiveness clean steps in a row
+ * take one off.  (so_verify and so_step_replicas call this; it is exported so that a caller who
+ * verifies the two kinds of a boundary in two oracle instances can keep their common counter.) */
+void so_count_violation(so_verifier *v, int r, int flagged, int severe);
 
 /* A new worker now feeds this boundary: clear its violation counter, streak and ban. */
 void so_reset_worker(so_verifier *v);

@@ -1204,7 +1204,7 @@ stream_kernel_t(const StreamArgs a) {
 constexpr int kStripe = 8 * 32 * kUnroll;        // columns per stripe
 constexpr int kChanThreads = 512;                 // threads per CTA of channel_ref_kernel: 16 warps, a stripe each at d = 8192
 constexpr int kChanWarps = kChanThreads / 32;
-constexpr int kChanRows = 4;                      // rows of a stripe that one stage holds
+constexpr int kChanRows = 6;                      // rows of a stripe that one stage holds
 constexpr int kChanDepth = 2;                     // stages per warp
 
 __host__ __device__ inline int channel_stripes(int d) { return (d + kStripe - 1) / kStripe; }
@@ -1257,6 +1257,18 @@ __device__ __noinline__ unsigned channel_nonfinite_in_stage(const unsigned char 
   return nf;
 }
 
+__device__ __noinline__ unsigned channel_differs_in_stage(const unsigned char *stage, int rows, int lane, unsigned valid,
+                                                          unsigned x0pair) {
+  unsigned diff = 0u;
+  for (int i = 0; i < rows; ++i)
+    for (int u = 0; u < kUnroll; ++u) {
+      if (!((valid >> u) & 1u)) continue;
+      const uint4 w = *reinterpret_cast<const uint4 *>(stage + i * kTileBytesX + (size_t)(u * 32 + lane) * 16);
+      diff |= (w.x ^ x0pair) | (w.y ^ x0pair) | (w.z ^ x0pair) | (w.w ^ x0pair);
+    }
+  return diff;
+}
+
 // One slot (a warp's stripe of columns, every `phases`-th row from `first` on) of a segment.
 // Per element only what is not linear in x is done: (x - x0)^2, |x - m|, the sign test on the
 // packed pairs, the constancy bits, and the column sum of x - x0.  The linear sums follow from
@@ -1265,7 +1277,7 @@ __device__ __noinline__ unsigned channel_nonfinite_in_stage(const unsigned char 
 // of |x - m| (not a finite number then), exact zeros of x in the packed minimum: either is looked
 // at once per stage, and the stage is gone through again only if it shows.
 // kZeroInM = true (an exact zero among this warp's columns of m): the general sign test.
-template <bool kZeroInM>
+template <bool kZeroInM, bool kFull>
 __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_pitch, int n_rows, int vc,
                                              const bool (&ok)[kUnroll], const F8 (&mv)[kUnroll],
                                              const unsigned (&msp)[kUnroll][4], const float *m_stripe,
@@ -1304,17 +1316,18 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
     }
     const unsigned char *stage = cw.stage[slot];
     const int rows = (n_rows - s * kChanRows < kChanRows) ? n_rows - s * kChanRows : kChanRows;
-    float g_sxx = 0.f, g_ab = 0.f;
+    float g_sxx[kUnroll] = {0.f, 0.f}, g_ab[kUnroll] = {0.f, 0.f};   // (two chains each: the adds of a row do not wait for one another)
     unsigned flips = 0u, zmin = 0x7F7F7F7Fu;
-    for (int i = 0; i < rows; ++i) {
+#pragma unroll
+    for (int i = 0; i < kChanRows; ++i) {
+      if (i >= rows) break;
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        if (!ok[u]) continue;
+        if (!kFull && !ok[u]) continue;
         const uint4 w = *reinterpret_cast<const uint4 *>(stage + i * kTileBytesX + (size_t)(u * 32 + lane) * 16);
         const unsigned w4[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          t.x_diff |= w4[q] ^ x0pair;
           if (!kZeroInM) {
             flips = __dp4a((w4[q] ^ msp[u][q]) & 0x80008000u, 0x01010101u, flips);
             zmin = min_abs_bf16x2(zmin, w4[q]);
@@ -1324,8 +1337,8 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
             const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
             const float mf = mv[u].v[2 * q + hlf];
             const float xs = xf - x0f;
-            g_sxx = fmaf(xs, xs, g_sxx);
-            g_ab += fabsf(xf - mf);
+            g_sxx[u] = fmaf(xs, xs, g_sxx[u]);
+            g_ab[u] += fabsf(xf - mf);
             if (kZeroInM) {
               const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
               flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? kFlipUnit : 0u;
@@ -1337,10 +1350,15 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
     }
     if (!kZeroInM && __any_sync(0xffffffffu, ((zmin & 0x7FFFu) == 0u) || ((zmin & 0x7FFF0000u) == 0u)))
       flips += kFlipUnit * channel_uncounted_zeros(stage, rows, lane, valid, m_stripe);
-    if (__any_sync(0xffffffffu, !(g_ab <= 3.4028234664e38f)))
+    if (__any_sync(0xffffffffu, !(g_ab[0] + g_ab[1] <= 3.4028234664e38f)))
       t.nf_bits |= channel_nonfinite_in_stage(stage, rows, lane, valid);
-    t.sxx += (double)g_sxx;                                  // the short fp32 runs into the fp64 sums
-    t.ab += (double)g_ab;
+    // does x vary?  A non-zero sum of (x - x0)^2 says so; a lane whose sum is zero (all its elements
+    // equal to x0, or differences too small to square) has its bit patterns compared
+    if (g_sxx[0] + g_sxx[1] > 0.f) t.x_diff |= 1u;
+    if (__any_sync(0xffffffffu, !(g_sxx[0] + g_sxx[1] > 0.f)))
+      t.x_diff |= channel_differs_in_stage(stage, rows, lane, valid, x0pair);
+    t.sxx += (double)g_sxx[0] + (double)g_sxx[1];            // the short fp32 runs into the fp64 sums
+    t.ab += (double)g_ab[0] + (double)g_ab[1];
     t.flips += flips / kFlipUnit;
     // every lane has used what it read from the stage (the sums above depend on it): refill it
     __syncwarp();
@@ -1349,9 +1367,11 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
   st.stages_done = head + (unsigned)n_stages;
 }
 
+// (merge: the column sums are added to what the CTA's first segment left in col_seg instead of
+// replacing it -- one vector for all samples needs no separation by sample)
 __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long long rb, const float *m_in,
-                                float *col_seg, ChanWarp &cw, ChanState &st, unsigned long long (*s_part)[kSlotWords],
-                                unsigned long long *slot) {
+                                float *col_seg, bool merge, ChanWarp &cw, ChanState &st,
+                                unsigned long long (*s_part)[kSlotWords], unsigned long long *slot) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunks = a.d >> 3;                   // d is a multiple of 8 here
   const int stripes = channel_stripes(a.d), phases = channel_phases(a.d), n_slots = stripes * phases;
@@ -1402,10 +1422,13 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
     const uint16_t *xslot = a.x + (size_t)(ra + phase) * a.d + (size_t)stripe * kStripe;
     const float *m_stripe = m_in + (size_t)stripe * kStripe;
     if (st.alive && n_rows > 0) {
-      if (__any_sync(0xffffffffu, zero_in_m))
-        channel_slot<true>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+      const bool full = vc == 32 * kUnroll;              // every lane has both its chunks
+      if (__any_sync(0xffffffffu, zero_in_m))              // (rare: the reference starts out as all zeros)
+        channel_slot<true, false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+      else if (full)
+        channel_slot<false, true>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
       else
-        channel_slot<false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+        channel_slot<false, false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
     }
 
     // what is linear in x, from the column sums; the reference's own sums: its columns once per row
@@ -1413,8 +1436,15 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
     double s_x = 0., s_xm = 0.;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      dst[u * 64] = make_float4(cs[u][0], cs[u][1], cs[u][2], cs[u][3]);
-      dst[u * 64 + 1] = make_float4(cs[u][4], cs[u][5], cs[u][6], cs[u][7]);
+      float4 lo = make_float4(cs[u][0], cs[u][1], cs[u][2], cs[u][3]);
+      float4 hi = make_float4(cs[u][4], cs[u][5], cs[u][6], cs[u][7]);
+      if (merge) {                               // (written by this very lane while it did the first segment)
+        const float4 plo = dst[u * 64], phi = dst[u * 64 + 1];
+        lo.x += plo.x; lo.y += plo.y; lo.z += plo.z; lo.w += plo.w;
+        hi.x += phi.x; hi.y += phi.y; hi.z += phi.z; hi.w += phi.w;
+      }
+      dst[u * 64] = lo;
+      dst[u * 64 + 1] = hi;
       if (ok[u]) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -1470,15 +1500,19 @@ channel_ref_kernel(const StreamArgs a) {
     long long ra = R0;
     for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
       unsigned long long *slot = a.partials + ((size_t)c * kSegsPerCta + sgm) * kSlotWords;
-      float *col_seg = a.col_part + ((size_t)c * kSegsPerCta + sgm) * seg_floats;
+      // column sums: a block per (CTA, segment) with a vector per sample, one block per CTA (both
+      // segments added) with one vector for all
+      const bool merge = !kPerSample && sgm > 0;
+      float *col_seg = a.col_part + ((size_t)c * kSegsPerCta + (kPerSample ? sgm : 0)) * seg_floats;
       if (ra < R1) {
         const int b = (int)(ra / a.T);
         const long long sample_end = (long long)(b + 1) * a.T;
         const long long rb = sample_end < R1 ? sample_end : R1;
-        channel_segment(a, b, ra, rb, kPerSample ? m_in + (size_t)b * a.d : m_in, col_seg, cw, st, s_part, slot);
+        channel_segment(a, b, ra, rb, kPerSample ? m_in + (size_t)b * a.d : m_in, col_seg, merge, cw, st, s_part, slot);
         ra = rb;
       } else {                                    // no rows: nothing to add
-        for (size_t i = threadIdx.x; i < seg_floats; i += kChanThreads) col_seg[i] = 0.f;
+        if (kPerSample)
+          for (size_t i = threadIdx.x; i < seg_floats; i += kChanThreads) col_seg[i] = 0.f;
         if (threadIdx.x == 0) slot[7] = 0ull;
       }
     }
@@ -1540,11 +1574,11 @@ channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const f
   if (c < d) {
     const int stripe = c / kStripe, within = c - stripe * kStripe;
     const float *src = col_part + (size_t)stripe * kStripe + within;
-    if (!per_sample) {
+    if (!per_sample) {                         // one block per CTA: its first, with both segments added
 #pragma unroll 8
-      for (int i = group; i < cs_hi * phases; i += kChannelMeanGroups) {
-        const int cs = i / phases, p = i - cs * phases;    // (CTA, segment) pair and row phase
-        sum += (double)__ldcg(src + ((size_t)cs * n_slots + (size_t)p * stripes) * kStripe);
+      for (int i = group; i < G * phases; i += kChannelMeanGroups) {
+        const int cta = i / phases, p = i - cta * phases;  // CTA and row phase
+        sum += (double)__ldcg(src + ((size_t)cta * kSegsPerCta * n_slots + (size_t)p * stripes) * kStripe);
       }
     } else {
       for (int i = cs_lo * phases + group; i < cs_hi * phases; i += kChannelMeanGroups) {
