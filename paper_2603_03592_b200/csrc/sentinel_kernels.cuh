@@ -252,6 +252,30 @@ __device__ __forceinline__ unsigned min_abs_bf16x2(unsigned a, unsigned b) {   /
 }
 
 // ---------------------------------------------------------------------------------------------
+// two single-precision operations per instruction (add/sub/fma.f32x2, new on sm_100): the
+// arithmetic-bound kernels below issue half as many floating-point instructions with them; each
+// half is rounded as the scalar instruction would round it
+struct F2 { float lo, hi; };
+__device__ __forceinline__ F2 add2(F2 a, F2 b) {
+  F2 r;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tadd.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.lo), "=f"(r.hi) : "f"(a.lo), "f"(a.hi), "f"(b.lo), "f"(b.hi));
+  return r;
+}
+__device__ __forceinline__ F2 sub2(F2 a, F2 b) {
+  F2 r;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tsub.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.lo), "=f"(r.hi) : "f"(a.lo), "f"(a.hi), "f"(b.lo), "f"(b.hi));
+  return r;
+}
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) {
+  F2 r;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\tfma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.lo), "=f"(r.hi) : "f"(a.lo), "f"(a.hi), "f"(b.lo), "f"(b.hi), "f"(c.lo), "f"(c.hi));
+  return r;
+}
+
+// ---------------------------------------------------------------------------------------------
 // per-element work
 
 struct GroupAcc {            // fp32 partial sums over one loop trip (<= 8*kUnroll elements)
@@ -1316,11 +1340,11 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
     }
     const unsigned char *stage = cw.stage[slot];
     const int rows = (n_rows - s * kChanRows < kChanRows) ? n_rows - s * kChanRows : kChanRows;
-    float g_sxx[kUnroll] = {0.f, 0.f}, g_ab[kUnroll] = {0.f, 0.f};   // (two chains each: the adds of a row do not wait for one another)
+    F2 g_sxx2[kUnroll] = {{0.f, 0.f}, {0.f, 0.f}};             // (several chains: the adds of a row do not wait for one another)
+    float g_ab[kUnroll] = {0.f, 0.f};
     unsigned flips = 0u, zmin = 0x7F7F7F7Fu;
-#pragma unroll
-    for (int i = 0; i < kChanRows; ++i) {
-      if (i >= rows) break;
+#pragma unroll 2
+    for (int i = 0; i < rows; ++i) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         if (!kFull && !ok[u]) continue;
@@ -1332,18 +1356,21 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
             flips = __dp4a((w4[q] ^ msp[u][q]) & 0x80008000u, 0x01010101u, flips);
             zmin = min_abs_bf16x2(zmin, w4[q]);
           }
-#pragma unroll
-          for (int hlf = 0; hlf < 2; ++hlf) {
-            const float xf = __uint_as_float(hlf ? (w4[q] & 0xFFFF0000u) : (w4[q] << 16));
-            const float mf = mv[u].v[2 * q + hlf];
-            const float xs = xf - x0f;
-            g_sxx[u] = fmaf(xs, xs, g_sxx[u]);
-            g_ab[u] += fabsf(xf - mf);
-            if (kZeroInM) {
-              const unsigned xt = __float_as_uint(xf) ^ (__float_as_uint(mf) & 0x80000000u);
-              flips += (((xf == 0.f) != (mf == 0.f)) || (__uint_as_float(xt) < 0.f)) ? kFlipUnit : 0u;
-            }
-            cs[u][2 * q + hlf] += xs;
+          const F2 xf = {__uint_as_float(w4[q] << 16), __uint_as_float(w4[q] & 0xFFFF0000u)};
+          const F2 mf = {mv[u].v[2 * q], mv[u].v[2 * q + 1]};
+          const F2 xs = sub2(xf, F2{x0f, x0f});
+          const F2 df = sub2(xf, mf);
+          g_sxx2[u] = fma2(xs, xs, g_sxx2[u]);
+          g_ab[u] += fabsf(df.lo);
+          g_ab[u] += fabsf(df.hi);
+          const F2 c2 = add2(F2{cs[u][2 * q], cs[u][2 * q + 1]}, xs);
+          cs[u][2 * q] = c2.lo;
+          cs[u][2 * q + 1] = c2.hi;
+          if (kZeroInM) {
+            const unsigned xl = __float_as_uint(xf.lo) ^ (__float_as_uint(mf.lo) & 0x80000000u);
+            const unsigned xh = __float_as_uint(xf.hi) ^ (__float_as_uint(mf.hi) & 0x80000000u);
+            flips += (((xf.lo == 0.f) != (mf.lo == 0.f)) || (__uint_as_float(xl) < 0.f)) ? kFlipUnit : 0u;
+            flips += (((xf.hi == 0.f) != (mf.hi == 0.f)) || (__uint_as_float(xh) < 0.f)) ? kFlipUnit : 0u;
           }
         }
       }
@@ -1354,6 +1381,7 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
       t.nf_bits |= channel_nonfinite_in_stage(stage, rows, lane, valid);
     // does x vary?  A non-zero sum of (x - x0)^2 says so; a lane whose sum is zero (all its elements
     // equal to x0, or differences too small to square) has its bit patterns compared
+    const float g_sxx[kUnroll] = {g_sxx2[0].lo + g_sxx2[0].hi, g_sxx2[1].lo + g_sxx2[1].hi};
     if (g_sxx[0] + g_sxx[1] > 0.f) t.x_diff |= 1u;
     if (__any_sync(0xffffffffu, !(g_sxx[0] + g_sxx[1] > 0.f)))
       t.x_diff |= channel_differs_in_stage(stage, rows, lane, valid, x0pair);
