@@ -279,8 +279,24 @@ int sentinel_get_thresholds(sentinel_verifier *h, sentinel_kind kind, double *ho
                             int *host_valid, void *cuda_stream);
 
 /* host_out int64 [6]: violations v, clean streak, banned (of worker 0), steps(ACT),
- * steps(GRAD), the error word written by device code (0 = none).  Waits for the stream. */
+ * steps(GRAD), the error word written by device code: 0 = none, SENTINEL_DEVICE_STAGING_TIMEOUT =
+ * a staged copy of the multi-worker, [T,d]- or [d]-reference kernels did not arrive within two
+ * seconds (the warp's remaining rows were left out: the step's results are not to be used),
+ * SENTINEL_DEVICE_OUT_OF_BOUNDS = the checked build skipped an access that would have left its
+ * buffer (see sentinel_bounds_violations).  Waits for the stream. */
+#define SENTINEL_DEVICE_STAGING_TIMEOUT 1
+#define SENTINEL_DEVICE_OUT_OF_BOUNDS 2
 int sentinel_get_counters(sentinel_verifier *h, long long *host_out, void *cuda_stream);
+
+/* The checked build of the library (libsentinel_checked.so: the same sources compiled with
+ * -DSENTINEL_CHECK_BOUNDS; the paper has no counterpart) compares every global-memory index that
+ * its kernels derive from the shape -- B, T, d, the row stride, the number of CTAs, the window
+ * sizes -- with the extent of the buffer before the access; an access that would leave the buffer
+ * is skipped and counted, nothing traps.  host_count receives the number of skipped accesses on
+ * `device` since the library was loaded, host_first_site (may be NULL) a code for where the first
+ * one happened (0 = none).  Synchronises the device.  The normal build does no such checks:
+ * there the call sets both to 0 and returns SENTINEL_ERR_UNSUPPORTED. */
+int sentinel_bounds_violations(int device, unsigned long long *host_count, int *host_first_site);
 
 /* host_out int64 [3]: violations, clean streak, banned of worker `worker`.  Waits. */
 int sentinel_get_worker_counters(sentinel_verifier *h, int worker, long long *host_out, void *cuda_stream);

@@ -27,20 +27,34 @@ def _inputs():
     return files
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library; returns its path."""
+LIB_CHECKED = os.path.join(_HERE, "libsentinel_checked.so")     # the same sources with -DSENTINEL_CHECK_BOUNDS
+
+
+def _compile(target: str, extra: list, force: bool, verbose: bool) -> str:
     newest = max(os.path.getmtime(f) for f in _inputs())
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
-        return LIB
+    if not force and os.path.exists(target) and os.path.getmtime(target) >= newest:
+        return target
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", tmp, *_sources()]
+    tmp = target + ".tmp%d" % os.getpid()
+    cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", INCLUDE, "-I", CSRC, "-o", tmp, *_sources()]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, target)
+    return target
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile every .cu under csrc/ into one shared library; returns its path."""
+    return _compile(LIB, [], force, verbose)
+
+
+def build_checked(force: bool = False, verbose: bool = False) -> str:
+    """The checked build: every index derived from the shape is compared with its buffer's extent
+    before the access (a debugging aid; the kernels are slower)."""
+    return _compile(LIB_CHECKED, ["-DSENTINEL_CHECK_BOUNDS"], force, verbose)
 
 
 if __name__ == "__main__":
     print(build(force=True, verbose=True))
+    print(build_checked(force=True))

@@ -39,6 +39,7 @@ EXPORTS = (
     "sentinel_get_stats", "sentinel_get_thresholds", "sentinel_get_counters",
     "sentinel_set_token_stats_buffer", "sentinel_reset_worker", "sentinel_state_bytes",
     "sentinel_export_state", "sentinel_import_state", "sentinel_last_error", "sentinel_destroy",
+    "sentinel_bounds_violations",
 )
 
 
@@ -61,10 +62,25 @@ class SentinelError(RuntimeError):
 
 
 _lib = None
+_lib_file = None          # None: the normal build; else the path of the library to load
 
 
 def lib_path() -> str:
-    return _build.LIB
+    return _lib_file or _build.LIB
+
+
+def use_library(path: str | None) -> None:
+    """Switch the binding to another build of the library (the checked build, for one) or, with
+    None, back to the normal one.  Handles made with one build must be closed before the switch."""
+    global _lib, _lib_file
+    _lib, _lib_file = None, path
+
+
+def sentinel_bounds_violations(device: int = 0) -> tuple[int, int]:
+    """(skipped accesses, site of the first) of the checked build; raises on the normal one."""
+    count, site = C.c_ulonglong(0), C.c_int(0)
+    _check(lib().sentinel_bounds_violations(device, C.byref(count), C.byref(site)))
+    return int(count.value), int(site.value)
 
 
 def lib():
@@ -108,6 +124,7 @@ def lib():
         L.sentinel_last_error.argtypes = [vp]
         L.sentinel_last_error.restype = C.c_char_p
         L.sentinel_destroy.argtypes = [vp]
+        L.sentinel_bounds_violations.argtypes = [ip, vp, vp]
         for name in EXPORTS:
             if name not in ("sentinel_state_bytes", "sentinel_last_error"):
                 getattr(L, name).restype = C.c_int

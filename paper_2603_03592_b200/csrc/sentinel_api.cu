@@ -261,6 +261,13 @@ StreamArgs make_args(sentinel_verifier *h, const void *x, int kind, int mode, fl
   a.defer_commit = h->chan_ref ? 1 : 0;
   a.ref_per_sample = h->chan_per_sample ? 1 : 0;
   a.col_part = h->col_part;
+  // what the checked build compares indices with
+  a.x_extent = h->shared_ref ? (long long)h->Ns : (long long)h->N;    // (a [T,d] reference: per sample slice)
+  a.ref_extent = (long long)h->ema_elems;
+  a.partials_words = (long long)(h->shared_ref ? h->cfg.B : h->R) * h->G * kSegsPerCta * kSlotWords;
+  a.ring_doubles = (long long)ring_doubles(h);
+  a.sorted_doubles = (long long)hist_doubles(h);
+  a.col_floats = h->chan_ref ? (long long)h->G * kSegsPerCta * channel_slots(h->cfg.d) * kStripe : 0;
   return a;
 }
 
@@ -742,6 +749,7 @@ int sentinel_verify_strided(sentinel_verifier *h, const void *dev_x, sentinel_ki
   h->started = true;
   StreamArgs a = make_args(h, dev_x, kind, kModeVerify, dev_scores_out, dev_flags_out);
   a.x_row_stride = row_stride;
+  a.x_extent = ((long long)B * T - 1) * row_stride + d;
   return launch(h, a, h->G + 1, static_cast<cudaStream_t>(cuda_stream), true);
 }
 
@@ -754,6 +762,7 @@ int sentinel_update_reference_strided(sentinel_verifier *h, const void *dev_x, s
   h->started = true;
   StreamArgs a = make_args(h, dev_x, kind, kModeWarmup, dev_scores_out, nullptr);
   a.x_row_stride = row_stride;
+  a.x_extent = ((long long)B * T - 1) * row_stride + d;
   return launch(h, a, h->G + 1, static_cast<cudaStream_t>(cuda_stream), true);
 }
 
@@ -825,6 +834,8 @@ int sentinel_distance(const void *dev_x, const float *dev_m, int B, int T, int d
   a.stats_out = dev_stats_out;
   a.B = B; a.T = T; a.d = d; a.G = G;
   a.x_row_stride = d;
+  a.x_extent = a.ref_extent = (long long)B * T * d;
+  a.partials_words = (long long)G * kSegsPerCta * kSlotWords;
   a.n_metrics = 3;
   a.mode = kModeDistance;
   stream_kernel_t<false, false><<<G + 1, kThreads, 0, s>>>(a);
@@ -1371,11 +1382,35 @@ int sentinel_distance_noalloc(const void *dev_x, const float *dev_m, int B, int 
   a.stats_out = dev_stats_out;
   a.B = B; a.T = T; a.d = d; a.G = G;
   a.x_row_stride = d;
+  a.x_extent = a.ref_extent = (long long)B * T * d;
+  a.partials_words = (long long)G * kSegsPerCta * kSlotWords;
   a.n_metrics = 3;
   a.mode = kModeDistance;
   stream_kernel_t<false, false><<<G + 1, kThreads, 0, s>>>(a);
   SENTINEL_CUDA(nullptr, cudaGetLastError());
   return SENTINEL_OK;
+}
+
+int sentinel_bounds_violations(int device, unsigned long long *host_count, int *host_first_site) {
+  if (!host_count) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "host_count is NULL");
+#ifdef SENTINEL_CHECK_BOUNDS
+  int ndev = 0;
+  SENTINEL_CUDA(nullptr, cudaGetDeviceCount(&ndev));
+  if (device < 0 || device >= ndev) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "device %d does not exist", device);
+  DeviceGuard guard(device);
+  SENTINEL_CUDA(nullptr, guard.status);
+  SENTINEL_CUDA(nullptr, cudaDeviceSynchronize());
+  int site = 0;
+  SENTINEL_CUDA(nullptr, cudaMemcpyFromSymbol(host_count, g_bounds_violations, sizeof *host_count));
+  SENTINEL_CUDA(nullptr, cudaMemcpyFromSymbol(&site, g_bounds_first_site, sizeof site));
+  if (host_first_site) *host_first_site = site;
+  return SENTINEL_OK;
+#else
+  (void)device;
+  *host_count = 0ull;
+  if (host_first_site) *host_first_site = 0;
+  return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "this library was built without bounds checks (-DSENTINEL_CHECK_BOUNDS)");
+#endif
 }
 
 const char *sentinel_last_error(const sentinel_verifier *h) { return h ? h->err.c_str() : g_error.c_str(); }

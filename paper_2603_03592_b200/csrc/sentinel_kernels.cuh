@@ -119,7 +119,38 @@ struct StreamArgs {
   unsigned metric_mask;
   int defer_commit;                // [d] reference: the commit is carried out by channel_mean_kernel
   float *col_part;                 // [d] reference: column sums of x, [G][2][channel_slots(d)][512]
+  // extents, in elements, of what the indices below are checked against in the checked build
+  long long x_extent;              // of x from its first element: (B*T - 1) * row stride + d
+  long long ref_extent;            // of one reference buffer
+  long long partials_words;        // of the partial slots
+  long long ring_doubles, sorted_doubles;   // of this kind's rings and ascending copies
+  long long col_floats;            // of col_part
 };
+
+// ---------------------------------------------------------------------------------------------
+// The checked build (-DSENTINEL_CHECK_BOUNDS, a second library target): before a kernel touches
+// global memory through an index that was worked out from the shape (B, T, d, the row stride, the
+// number of CTAs, the ring sizes), the range is compared with the extent of the buffer.  An access
+// that would leave it is skipped and counted; nothing traps.  The count and the site of the first
+// violation are read with sentinel_bounds_violations(), and the last CTA of a launch writes
+// kErrBounds into HandleState.error.  In the normal build the checks compile to nothing.
+constexpr int kErrBounds = 2;                     // HandleState.error: an index left its buffer (checked build)
+enum Site : int { kSiteX = 1, kSiteRefIn, kSiteRefOut, kSiteToken, kSiteSlot, kSiteRing, kSiteSorted, kSiteOut,
+                  kSiteStageX, kSiteStageRef, kSiteColumns, kSiteReplace };
+#ifdef SENTINEL_CHECK_BOUNDS
+__device__ unsigned long long g_bounds_violations = 0ull;
+__device__ int g_bounds_first_site = 0;
+__device__ __forceinline__ bool in_bounds(int site, long long first, long long count, long long extent) {
+  if (first >= 0 && count >= 0 && first + count <= extent) return true;
+  atomicAdd(&g_bounds_violations, 1ull);
+  atomicCAS(&g_bounds_first_site, 0, site);
+  return false;
+}
+#define SENTINEL_BOUNDS(site, first, count, extent) \
+  ::sentinel::in_bounds((site), (long long)(first), (long long)(count), (long long)(extent))
+#else
+#define SENTINEL_BOUNDS(site, first, count, extent) true
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // memory access helpers
@@ -268,6 +299,12 @@ __device__ __forceinline__ F2 sub2(F2 a, F2 b) {
       : "=f"(r.lo), "=f"(r.hi) : "f"(a.lo), "f"(a.hi), "f"(b.lo), "f"(b.hi));
   return r;
 }
+__device__ __forceinline__ F2 mul2(F2 a, F2 b) {
+  F2 r;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(r.lo), "=f"(r.hi) : "f"(a.lo), "f"(a.hi), "f"(b.lo), "f"(b.hi));
+  return r;
+}
 __device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) {
   F2 r;
   asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\tfma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
@@ -329,6 +366,73 @@ __device__ __forceinline__ void chunk(const uint4 &xv, F8 &mv, GroupAcc &g, Thre
       mv.v[2 * j + 1] = fmaf(beta, m_hi, omb * x_hi);
     }
   }
+}
+
+// The same chunk with a bf16 reference, which leaves the arithmetic as the bound (6 bytes per
+// element move instead of 10): x and m stay packed pairs as long as they can.  The sums run on
+// two-wide instructions (even elements in one half, odd ones in the other; the halves are added
+// when the trip is folded), sign mismatches are counted on the packed words (the sign bits of a
+// bf16 pair sit where the test wants them), the smallest magnitudes of x and of m are followed so
+// that a trip with an exact zero in it can be counted again element by element, and non-finite
+// elements show in the sum of |x - m|.  The candidate is fma(beta, m, (1-beta) x) per element,
+// each half rounded as the scalar instructions round, then to bf16 (nearest even): bit for bit
+// the value of the scalar path.
+struct PairAcc {             // one loop trip: two-wide fp32 sums, packed counters
+  F2 sx, sxx, sm, smm, sxm;
+  float ab[2];
+  unsigned flips;            // in units of kFlipUnit
+  unsigned zmin;             // per half: smallest magnitude met in x or in m
+};
+
+__device__ __forceinline__ void chunk_packed(const uint4 &xv, const uint4 &mraw, uint4 &out, PairAcc &g, ThreadAcc &t,
+                                             unsigned x0pair, unsigned m0pair, float x0, float m0, float beta, float omb,
+                                             bool write_ema) {
+  const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w}, mw[4] = {mraw.x, mraw.y, mraw.z, mraw.w};
+  unsigned ow[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    t.x_diff |= xw[j] ^ x0pair;
+    t.m_diff |= mw[j] ^ m0pair;
+    g.flips = __dp4a((xw[j] ^ mw[j]) & 0x80008000u, 0x01010101u, g.flips);
+    g.zmin = min_abs_bf16x2(min_abs_bf16x2(g.zmin, xw[j]), mw[j]);
+    const F2 xf = {__uint_as_float(xw[j] << 16), __uint_as_float(xw[j] & 0xFFFF0000u)};
+    const F2 mf = {__uint_as_float(mw[j] << 16), __uint_as_float(mw[j] & 0xFFFF0000u)};
+    const F2 xs = sub2(xf, F2{x0, x0}), ms = sub2(mf, F2{m0, m0});
+    g.sx = add2(g.sx, xs);
+    g.sm = add2(g.sm, ms);
+    g.sxx = fma2(xs, xs, g.sxx);
+    g.smm = fma2(ms, ms, g.smm);
+    g.sxm = fma2(xs, ms, g.sxm);
+    const F2 df = sub2(xf, mf);
+    g.ab[0] += fabsf(df.lo);
+    g.ab[1] += fabsf(df.hi);
+    if (write_ema) {
+      const F2 cand = fma2(F2{beta, beta}, mf, mul2(F2{omb, omb}, xf));
+      ow[j] = pack_bf16x2_rn(cand.lo, cand.hi);
+    }
+  }
+  out = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+}
+
+// sign(x) != sign(m), three-valued, element by element on a packed chunk (the trips in which the
+// packed count does not hold: an exact zero on either side)
+__device__ __forceinline__ unsigned flips_exact(const uint4 &xv, const uint4 &mraw) {
+  const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w}, mw[4] = {mraw.x, mraw.y, mraw.z, mraw.w};
+  unsigned n = 0u;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const unsigned xb = h ? (xw[j] >> 16) : (xw[j] & 0xFFFFu), mb = h ? (mw[j] >> 16) : (mw[j] & 0xFFFFu);
+      const bool xz = (xb & 0x7FFFu) == 0u, mz = (mb & 0x7FFFu) == 0u;
+      n += ((xz != mz) || (!xz && !mz && ((xb ^ mb) & 0x8000u))) ? 1u : 0u;
+    }
+  }
+  return n;
+}
+__device__ __forceinline__ unsigned nonfinite_bits(const uint4 &xv) {
+  return (((xv.x & 0x7F807F80u) + 0x00800080u) | ((xv.y & 0x7F807F80u) + 0x00800080u) |
+          ((xv.z & 0x7F807F80u) + 0x00800080u) | ((xv.w & 0x7F807F80u) + 0x00800080u)) & 0x80008000u;
 }
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -418,15 +522,21 @@ __device__ __forceinline__ uint4 shifted_chunk(const uint4 &w0, const uint4 &w1,
   return out;
 }
 
+// (row_first, x_extent: where the row starts in x and how many elements x has, for the checked
+// build: an aligned word may begin up to 7 elements below the row and end as many above it, inside
+// the 16-byte granule the row's first or last element lies in -- except past the last row, which
+// is why that row's upper word is put together from the elements that exist)
 template <int kU>
 __device__ __forceinline__ void load_x_shifted(const uint16_t *row_ptr, int base, int chunks, bool last_row,
-                                               const bool (&ok)[kU], uint4 (&xv)[kU]) {
+                                               const bool (&ok)[kU], uint4 (&xv)[kU], long long row_first,
+                                               long long x_extent) {
   const int lane = threadIdx.x & 31;
   const unsigned s = (unsigned)(reinterpret_cast<uintptr_t>(row_ptr) & 15u);
   if (s == 0u) {
 #pragma unroll
     for (int u = 0; u < kU; ++u)
-      if (ok[u]) xv[u] = ld_x128(row_ptr + (size_t)(base + u * 32 + lane) * 8);
+      if (ok[u] && SENTINEL_BOUNDS(kSiteX, row_first + (long long)(base + u * 32 + lane) * 8, 8, x_extent))
+        xv[u] = ld_x128(row_ptr + (size_t)(base + u * 32 + lane) * 8);
     return;
   }
   const uint16_t *al = row_ptr - (s >> 1);                 // 16-byte aligned
@@ -438,14 +548,17 @@ __device__ __forceinline__ void load_x_shifted(const uint16_t *row_ptr, int base
     const int c = base + u * 32 + lane;
     w0[u] = own[u] = make_uint4(0u, 0u, 0u, 0u);
     direct[u] = ok[u] && (lane == 31 || c + 1 >= chunks);  // nobody holds the word above this chunk
-    if (ok[u]) w0[u] = ld_x128(al + (size_t)c * 8);
+    // (in elements of x: the aligned word below chunk c begins at row_first - s/2 + 8c)
+    [[maybe_unused]] const long long lower = row_first - (long long)(s >> 1) + (long long)c * 8;
+    if (ok[u] && SENTINEL_BOUNDS(kSiteX, lower + 7, 1, x_extent + 7)) w0[u] = ld_x128(al + (size_t)c * 8);
     if (direct[u]) {
       const uint16_t *up = al + (size_t)(c + 1) * 8;
       if (last_row && c + 1 >= chunks) {                   // only its first s bytes exist for sure
         unsigned e[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-        for (unsigned k = 0; k < (s >> 1); ++k) e[k] = up[k];
+        if (SENTINEL_BOUNDS(kSiteX, lower + 8, (long long)(s >> 1), x_extent))
+          for (unsigned k = 0; k < (s >> 1); ++k) e[k] = up[k];
         own[u] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
-      } else {
+      } else if (SENTINEL_BOUNDS(kSiteX, lower + 8, 1, x_extent)) {   // (the word above a row that is not the last begins inside x)
         own[u] = ld_x128(up);
       }
     }
@@ -495,9 +608,11 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
   const bool tokens = (a.token_out != nullptr);
   const float beta = a.beta, omb = a.one_minus_beta;
 
-  const unsigned x0 = a.x[(size_t)b * a.T * (size_t)a.x_row_stride];
+  const unsigned x0 = SENTINEL_BOUNDS(kSiteX, (long long)b * a.T * a.x_row_stride, 1, a.x_extent)
+                          ? a.x[(size_t)b * a.T * (size_t)a.x_row_stride] : 0u;
   const unsigned x0pair = x0 | (x0 << 16);
-  const unsigned m0bits = __float_as_uint(load_m1<kBf16>(m_in, sample_off));
+  const unsigned m0bits = SENTINEL_BOUNDS(kSiteRefIn, sample_off, 1, a.ref_extent)
+                              ? __float_as_uint(load_m1<kBf16>(m_in, sample_off)) : 0u;
 
   ThreadAcc t = {0., 0., 0., 0., 0., 0., 0u, 0u, 0u, 0u};
 
@@ -520,7 +635,11 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
 #pragma unroll
       for (int q = 0; q < kPerLane; ++q) {
         const int col = col0 + q * 32;
-        if (col < a.d) { xs[q] = a.x[off_x + col]; ms[q] = load_m1<kBf16>(m_in, off + col); }
+        if (col < a.d && SENTINEL_BOUNDS(kSiteX, off_x + col, 1, a.x_extent) &&
+            SENTINEL_BOUNDS(kSiteRefIn, off + col, 1, a.ref_extent)) {
+          xs[q] = a.x[off_x + col];
+          ms[q] = load_m1<kBf16>(m_in, off + col);
+        }
       }
 #pragma unroll
       for (int q = 0; q < kPerLane; ++q) {
@@ -532,7 +651,8 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
           t.m_diff |= __float_as_uint(ms[q]) ^ m0bits;
           const float xf = __uint_as_float(xb << 16);
           element(xf, ms[q], x0f, m0f, g);
-          if (write_ema) store_m1<kBf16>(m_out, off + col, fmaf(beta, ms[q], omb * xf));
+          if (write_ema && SENTINEL_BOUNDS(kSiteRefOut, off + col, 1, a.ref_extent))
+            store_m1<kBf16>(m_out, off + col, fmaf(beta, ms[q], omb * xf));
         }
       }
     } else {
@@ -543,7 +663,8 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
 #pragma unroll
       for (int u = 0; u < kU; ++u) {
         const int c = base + u * 32 + lane;
-        ok[u] = c < chunks;
+        ok[u] = c < chunks && SENTINEL_BOUNDS(kSiteRefIn, off + (size_t)c * 8, 8, a.ref_extent) &&
+                (kShifted || SENTINEL_BOUNDS(kSiteX, off + (size_t)c * 8, 8, a.x_extent));
         if (ok[u]) {
           if (!kShifted) xv[u] = ld_x128(a.x + off + (size_t)c * 8);
           if (kBf16) mraw[u] = ld_x128(static_cast<const uint16_t *>(m_in) + off + (size_t)c * 8);
@@ -552,14 +673,48 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
       }
       if (kShifted)
         load_x_shifted<kU>(a.x + (size_t)row * (size_t)a.x_row_stride, base, chunks,
-                           row == (long long)a.B * a.T - 1, ok, xv);
+                           row == (long long)a.B * a.T - 1, ok, xv, row * a.x_row_stride, a.x_extent);
+      if (kBf16) {
+        // the packed path (see chunk_packed): m0 is a bf16 value here, m0bits >> 16 its pattern
+        PairAcc p = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, 0u, 0x7F7F7F7Fu};
+        const unsigned m0pair = (m0bits >> 16) | (m0bits & 0xFFFF0000u);
+        const float x0f = __uint_as_float(x0 << 16), m0f = __uint_as_float(m0bits);
 #pragma unroll
-      for (int u = 0; u < kU; ++u) {
-        if (ok[u]) {
-          F8 &m8 = mv[kBf16 ? 0 : u];
-          if (kBf16) m8 = widen_bf16x8(mraw[u]);
-          chunk(xv[u], m8, g, t, x0pair, m0bits, beta, omb, write_ema);
-          if (write_ema) store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, m8);
+        for (int u = 0; u < kU; ++u) {
+          if (ok[u]) {
+            uint4 cand;
+            chunk_packed(xv[u], mraw[u], cand, p, t, x0pair, m0pair, x0f, m0f, beta, omb, write_ema);
+            if (write_ema)
+              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                           :: "l"(static_cast<uint16_t *>(m_out) + off + (size_t)(base + u * 32 + lane) * 8),
+                              "r"(cand.x), "r"(cand.y), "r"(cand.z), "r"(cand.w) : "memory");
+          }
+        }
+        unsigned flips = p.flips / kFlipUnit;
+        // an exact zero in x or m somewhere in this trip: count again, element by element
+        if (__any_sync(0xffffffffu, ((p.zmin & 0x7FFFu) == 0u) || ((p.zmin & 0x7FFF0000u) == 0u))) {
+          flips = 0u;
+#pragma unroll
+          for (int u = 0; u < kU; ++u)
+            if (ok[u]) flips += flips_exact(xv[u], mraw[u]);
+        }
+        const float ab = p.ab[0] + p.ab[1];
+        if (__any_sync(0xffffffffu, !(ab <= 3.4028234664e38f))) {   // not a finite sum: look at the bits
+#pragma unroll
+          for (int u = 0; u < kU; ++u)
+            if (ok[u]) t.nf_bits |= nonfinite_bits(xv[u]);
+        }
+        g.sx = p.sx.lo + p.sx.hi;     g.sxx = p.sxx.lo + p.sxx.hi;
+        g.sm = p.sm.lo + p.sm.hi;     g.smm = p.smm.lo + p.smm.hi;
+        g.sxm = p.sxm.lo + p.sxm.hi;  g.ab = ab;
+        g.flips = flips;
+      } else {
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+          if (ok[u]) {
+            chunk(xv[u], mv[u], g, t, x0pair, m0bits, beta, omb, write_ema);
+            if (write_ema) store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+          }
         }
       }
     }
@@ -572,7 +727,8 @@ __device__ void stream_segment(const StreamArgs &a, int b, long long ra, long lo
     if (tokens) {                       // this tile's share of the token's sums
       const float sx = warp_sum(g.sx), sxx = warp_sum(g.sxx), ab = warp_sum(g.ab);
       const float fl = warp_sum((float)g.flips);
-      if (lane == 0) {
+      if (lane == 0 && SENTINEL_BOUNDS(kSiteToken, row, 1, (long long)a.B * a.T) &&
+          SENTINEL_BOUNDS(kSiteToken, seg, 1, tiles_per_row)) {
         float4 *dst = (tiles_per_row == 1) ? reinterpret_cast<float4 *>(a.token_out) + row
                                            : reinterpret_cast<float4 *>(a.token_part) + row * tiles_per_row + seg;
         float4 v = make_float4(sx, sxx, ab, fl);
@@ -616,6 +772,7 @@ __device__ void stream_cta(const StreamArgs &a, int c, const void *m_in, void *m
   long long ra = R0;
   for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
     unsigned long long *slot = a.partials + ((size_t)c * kSegsPerCta + sgm) * kSlotWords;
+    if (!SENTINEL_BOUNDS(kSiteSlot, ((size_t)c * kSegsPerCta + sgm) * kSlotWords, kSlotWords, a.partials_words)) continue;
     if (ra < R1) {
       const int b = (int)(ra / a.T);
       const long long sample_end = (long long)(b + 1) * a.T;
@@ -732,6 +889,13 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, double *so
                                  : (size_t)i * window_smem_doubles(cap0, units0));
       double *s_new = s_old + cap, *s_stage = s_new + cap, *s_out = s_stage + 2 * units, *s_in = s_out + units;
 
+#ifdef SENTINEL_CHECK_BOUNDS
+      const bool window_ok = SENTINEL_BOUNDS(kSiteSorted, n_old, 0, cap) && SENTINEL_BOUNDS(kSiteSorted, n, 0, cap) &&
+                             SENTINEL_BOUNDS(kSiteRing, evicted, 0, units) && SENTINEL_BOUNDS(kSiteRing, joined, 0, units) &&
+                             SENTINEL_BOUNDS(kSiteRing, head, 1, size);
+      if (!window_ok) { group_barrier(group, group_threads); group_barrier(group, group_threads); group_barrier(group, group_threads); }
+      if (window_ok) {
+#endif
       for (int p = gt; p < n_old; p += group_threads) s_old[p] = srt[p];
       // the entries pushed out sit just before the head, the ones that joined at the tail;
       // stage them, then rank-sort them (they are few) into s_out / s_in
@@ -818,6 +982,9 @@ __device__ void refresh_thresholds(KindState *ks, const double *hist, double *so
           ks->has_thr[L][i] = 1;
         }
       }
+#ifdef SENTINEL_CHECK_BOUNDS
+      }
+#endif
     }
   }
   __syncthreads();
@@ -895,6 +1062,7 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
     const long long n_slots = (c_hi - c_lo + 1) * kSegsPerCta;
     for (long long q = lane; q < n_slots; q += 32) {
       const unsigned long long *slot = block + ((size_t)c_lo * kSegsPerCta + q) * kSlotWords;
+      if (!SENTINEL_BOUNDS(kSiteSlot, c_lo * kSegsPerCta + q, 1, (long long)a.G * kSegsPerCta)) continue;
       unsigned long long w[kSlotWords];
 #pragma unroll
       for (int j = 0; j < kSlotWords; ++j) w[j] = __ldcg(slot + j);   // one round trip, then the tag
@@ -1069,7 +1237,8 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
       const int idx = (int)(((long long)ring_head + ring_count + k) % size);
 #pragma unroll
       for (int i = 0; i < kNumMetrics; ++i)
-        if (i < a.n_metrics) a.hist[ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx] = g[i];
+        if (i < a.n_metrics && SENTINEL_BOUNDS(kSiteRing, ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx, 1, a.ring_doubles))
+          a.hist[ring_offset(L, i, a.cap0, a.cap1, a.units0, a.units1) + idx] = g[i];
     }
     if (ft.scores_out) {
 #pragma unroll
@@ -1142,6 +1311,9 @@ __device__ void finalize(const StreamArgs &a, const FinalizeTarget &ft) {
       if (ks->refresh_pending) { ks->last_joined[L] += joined[L]; ks->last_evicted[L] += evicted; }
     }
     if (ft.last) s_hs.ticket = 0u;               // ready for the next launch
+#ifdef SENTINEL_CHECK_BOUNDS
+    if (*reinterpret_cast<volatile unsigned long long *>(&g_bounds_violations)) hs->error = kErrBounds;
+#endif
     s_status = status;
   }
   __syncthreads();
@@ -1306,7 +1478,7 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
                                              const bool (&ok)[kUnroll], const F8 (&mv)[kUnroll],
                                              const unsigned (&msp)[kUnroll][4], const float *m_stripe,
                                              float (&cs)[kUnroll][8], unsigned x0pair, float x0f, ThreadAcc &t,
-                                             ChanWarp &cw, ChanState &st) {
+                                             ChanWarp &cw, ChanState &st, long long x_first, long long x_extent) {
   // (xslot: the first element of the stripe in the slot's first row; rows are row_pitch elements apart)
   const int lane = threadIdx.x & 31;
   const int n_stages = (n_rows + kChanRows - 1) / kChanRows;
@@ -1320,9 +1492,15 @@ __device__ __forceinline__ void channel_slot(const uint16_t *xslot, size_t row_p
       const int rows = (n_rows - s * kChanRows < kChanRows) ? n_rows - s * kChanRows : kChanRows;
       const unsigned k = head + (unsigned)s, slot = k % kChanDepth;
       const unsigned bar = smem_addr(&cw.bar[slot]), dst = smem_addr(&cw.stage[slot][0]);
-      mbar_arrive_expect(bar, (unsigned)(rows * vc) * 16u);
-      for (int i = 0; i < rows; ++i)
-        bulk_copy_in(dst + i * kTileBytesX, xslot + (size_t)(s * kChanRows + i) * row_pitch, (unsigned)vc * 16u, bar);
+      // (checked build: the last element of the stage's last row must lie in x)
+      if (SENTINEL_BOUNDS(kSiteStageX, x_first + (long long)(s * kChanRows + rows - 1) * (long long)row_pitch, (long long)vc * 8, x_extent) &&
+          SENTINEL_BOUNDS(kSiteStageX, x_first + (long long)(s * kChanRows) * (long long)row_pitch, (long long)vc * 8, x_extent)) {
+        mbar_arrive_expect(bar, (unsigned)(rows * vc) * 16u);
+        for (int i = 0; i < rows; ++i)
+          bulk_copy_in(dst + i * kTileBytesX, xslot + (size_t)(s * kChanRows + i) * row_pitch, (unsigned)vc * 16u, bar);
+      } else {
+        mbar_arrive_expect(bar, 0u);
+      }
     }
   };
 #pragma unroll
@@ -1425,7 +1603,7 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int c = stripe * 32 * kUnroll + u * 32 + lane;
-      ok[u] = c < chunks;
+      ok[u] = c < chunks && SENTINEL_BOUNDS(kSiteRefIn, (long long)c * 8, 8, a.d);
 #pragma unroll
       for (int e = 0; e < 8; ++e) { cs[u][e] = 0.f; mv[u].v[e] = 1.f; }
       if (ok[u]) {
@@ -1452,27 +1630,30 @@ __device__ void channel_segment(const StreamArgs &a, int b, long long ra, long l
     if (st.alive && n_rows > 0) {
       const bool full = vc == 32 * kUnroll;              // every lane has both its chunks
       if (__any_sync(0xffffffffu, zero_in_m))              // (rare: the reference starts out as all zeros)
-        channel_slot<true, false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+        channel_slot<true, false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st, (long long)(xslot - a.x), a.x_extent);
       else if (full)
-        channel_slot<false, true>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+        channel_slot<false, true>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st, (long long)(xslot - a.x), a.x_extent);
       else
-        channel_slot<false, false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st);
+        channel_slot<false, false>(xslot, (size_t)phases * a.d, n_rows, vc, ok, mv, msp, m_stripe, cs, x0pair, x0f, t, cw, st, (long long)(xslot - a.x), a.x_extent);
     }
 
     // what is linear in x, from the column sums; the reference's own sums: its columns once per row
     float4 *dst = reinterpret_cast<float4 *>(col_seg + (size_t)sl * kStripe) + lane * 2;
+    const bool col_ok = SENTINEL_BOUNDS(kSiteColumns, (col_seg - a.col_part) + (long long)(sl + 1) * kStripe, 0, a.col_floats);
     double s_x = 0., s_xm = 0.;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       float4 lo = make_float4(cs[u][0], cs[u][1], cs[u][2], cs[u][3]);
       float4 hi = make_float4(cs[u][4], cs[u][5], cs[u][6], cs[u][7]);
-      if (merge) {                               // (written by this very lane while it did the first segment)
+      if (merge && col_ok) {                     // (written by this very lane while it did the first segment)
         const float4 plo = dst[u * 64], phi = dst[u * 64 + 1];
         lo.x += plo.x; lo.y += plo.y; lo.z += plo.z; lo.w += plo.w;
         hi.x += phi.x; hi.y += phi.y; hi.z += phi.z; hi.w += phi.w;
       }
-      dst[u * 64] = lo;
-      dst[u * 64 + 1] = hi;
+      if (col_ok) {
+        dst[u * 64] = lo;
+        dst[u * 64 + 1] = hi;
+      }
       if (ok[u]) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -1872,11 +2053,16 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
       int vc = 32 * kUnroll;                                 // chunks of this tile that exist
       if (!kFull && chunks - p_seg * 32 * kUnroll < vc) vc = chunks - p_seg * 32 * kUnroll;
       const unsigned bar = smem_addr(&fw.bar[st]), dst = smem_addr(&fw.stage[st][0]);
-      mbar_arrive_expect(bar, (unsigned)vc * (32u + 16u * NR));
-      bulk_copy_in(dst, m_in + off, (unsigned)vc * 32u, bar);
+      if (SENTINEL_BOUNDS(kSiteStageRef, off, (long long)vc * 8, a.ref_extent) &&
+          SENTINEL_BOUNDS(kSiteStageX, off, (long long)vc * 8, a.x_extent)) {
+        mbar_arrive_expect(bar, (unsigned)vc * (32u + 16u * NR));
+        bulk_copy_in(dst, m_in + off, (unsigned)vc * 32u, bar);
 #pragma unroll
-      for (int r = 0; r < NR; ++r)
-        bulk_copy_in(dst + kTileBytesM + r * kTileBytesX, fs.ptr[r] + off, (unsigned)vc * 16u, bar);
+        for (int r = 0; r < NR; ++r)
+          bulk_copy_in(dst + kTileBytesM + r * kTileBytesX, fs.ptr[r] + off, (unsigned)vc * 16u, bar);
+      } else {
+        mbar_arrive_expect(bar, 0u);                         // (checked build: nothing is copied, the wait still ends)
+      }
     }
   };
 #pragma unroll
@@ -1997,7 +2183,8 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
         // Eq. 1 with the mean over the tensors
 #pragma unroll
         for (int e = 0; e < 8; ++e) mv.v[e] = fmaf(beta, mv.v[e], wgt * sum[e]);
-        st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv);
+        if (SENTINEL_BOUNDS(kSiteRefOut, off + (size_t)(base + u * 32 + lane) * 8, 8, a.ref_extent))
+          st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv);
       }
     }
     unsigned valid = 0u;                                     // this lane's chunks of the tile
@@ -2039,7 +2226,9 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
   if (tid < kSegsPerCta * NR * kSlotWords) {
     const int sgm = tid / (NR * kSlotWords), r = (tid / kSlotWords) % NR, w8 = tid % kSlotWords;
     unsigned long long *slot = partials + (((size_t)fs.widx[r] * a.G + c) * kSegsPerCta + sgm) * kSlotWords;
-    if (sgm == 1 && cut >= r1) {
+    if (!SENTINEL_BOUNDS(kSiteSlot, (((size_t)fs.widx[r] * a.G + c) * kSegsPerCta + sgm) * kSlotWords, kSlotWords, a.partials_words)) {
+      // (checked build: the slot lies outside the buffer; nothing is written)
+    } else if (sgm == 1 && cut >= r1) {
       if (w8 == 7) slot[7] = 0ull;                           // no second segment: tag 0, unused
     } else {
       unsigned long long out;
@@ -2407,6 +2596,9 @@ replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *em
     // a [T,d] or [d] reference repeats every ref_chunks; a [B,d] one holds a row of ref_chunks per sample
     const long long cm = sample_chunks ? (c / sample_chunks) * ref_chunks + c % ref_chunks
                                        : ref_chunks ? c % ref_chunks : c;
+    if (!SENTINEL_BOUNDS(kSiteReplace, c, 1, n_chunks) ||
+        !SENTINEL_BOUNDS(kSiteReplace, cm, 1, sample_chunks ? (n_chunks / sample_chunks) * ref_chunks : ref_chunks ? ref_chunks : n_chunks))
+      continue;
     if (!zero_fill && ema_bf16) {                 // the reference already is a bf16 tensor
       out = ld_x128(static_cast<const uint16_t *>(m) + cm * 8);
     } else if (!zero_fill) {

@@ -139,3 +139,24 @@ def whole_step_k_events(gt, gvalid, ot, ovalid, params, kind) -> int:
             assert whole, "k differs by no whole number of steps: %r vs %r" % (gt[L, i, 3], ot[L, i, 3])
             events += 1
     return events
+
+
+def assert_thresholds_close(gt, ot, valid, params, kind, what=""):
+    """Bounds of Alg. 5, library against oracle.  The quartiles are functions of scores that agree
+    to 1e-3, so they are compared at 1e-3 on the scale of the median.  tau = q2 -+ k*IQR amplifies
+    a difference of the quartiles k-fold (k reaches the hundreds where a window is narrow), so the
+    bounds are checked for what they must be: Alg. 5's last lines applied to the library's own
+    quartiles and multiplier, to rounding."""
+    lam, eps = params.lam[kind], params.eps[kind]
+    for L in range(2):
+        for i in range(valid.shape[1]):
+            if not valid[L, i]:
+                continue
+            q1, q2, q3, k, lo, hi = gt[L, i]
+            tol = REL * np.maximum(np.abs(ot[L, i, :3]), abs(ot[L, i, 1]))
+            assert np.all(np.abs(gt[L, i, :3] - ot[L, i, :3]) <= tol), (what, L, i, gt[L, i], ot[L, i])
+            iqr = max(q3 - q1, eps)
+            want_lo = min(q2 - k * iqr, q2 - lam * abs(q2))
+            want_hi = max(q2 + k * iqr, q2 + lam * abs(q2))
+            scale = max(abs(q2), k * iqr, 1e-300)
+            assert abs(lo - want_lo) <= 1e-12 * scale and abs(hi - want_hi) <= 1e-12 * scale, (what, L, i, gt[L, i])

@@ -84,8 +84,13 @@ class OracleStream:
         self.proc.start()
 
     def step(self, bits, t, warm):
-        """Hands the worker the tensor of step t (uint16 bit patterns of the stream's shape)."""
-        np.copyto(self.x, bits)
+        """Hands the worker the tensor of step t: uint16 bit patterns of the stream's shape, or a
+        bf16 torch tensor (copied from the device straight into the mapped file)."""
+        if hasattr(bits, "data_ptr"):
+            import torch
+            torch.from_numpy(self.x.view(np.int16)).copy_(bits.detach().contiguous().view(torch.int16))
+        else:
+            np.copyto(self.x, bits)
         self.cmd.put(("step", t, warm))
 
     def ready(self):

@@ -1,6 +1,7 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration ``bench.py`` times
 (same entry points, same shapes): every score of every unit and every flag against the float64
-oracle run on the same tensors.  A few steps per shape keep the oracle within about a minute."""
+oracle run on the same tensors.  Here: the variants (several workers, the storage forms of the
+reference, the sliced Wasserstein distance), a few steps each."""
 import numpy as np
 import pytest
 import torch
@@ -51,52 +52,8 @@ def run_steps(sb, oracle_mod, w, kind, n_warm, corruption, **variant):
     gv.close()
 
 
-def test_cfg4_wide_model_activations(sb, oracle_mod):
-    """B=4 x T=8192 x d=8192 (512 MiB per tensor), Student-t activations, uniform noise on one sample."""
-    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], ACT, 2, "add_uniform_sample")
-
-
-def test_cfg4_wide_model_gradients(sb, oracle_mod):
-    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], GRAD, 1, "add_uniform_sample")
-
-
-def test_cfg3_1b_class_zeroed_tokens(sb, oracle_mod):
-    """B=8 x T=4096 x d=4096, lognormal channel scales; 10% of the token rows zeroed."""
-    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg3"], ACT, 2, "zero_tokens")
-
-
-def test_cfg5_boundary_shape_gradients(sb, oracle_mod):
-    """B=16 x T=2048 x d=4096 (the many-boundary sweep's shape), additive Gaussian noise."""
-    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg5"], GRAD, 2, "add_gauss")
-
-
-def test_cfg2_small_lm_stream_prefix(sb, oracle_mod):
-    """B=16 x T=1024 x d=2048: the full 16-step warm-up and the first verified steps of the
-    stream, corruptions as the recipe draws them."""
-    w = synth.WORKLOADS["cfg2"]
-    gv = sb.Verifier(w.B, w.T, w.d)
-    ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d))
-    for t in range(w.warmup + 6):
-        x, name = synth.microbatch(w, 0, ACT, t, "cuda")
-        if t == w.warmup + 3 and name is None:
-            x, name = synth.corrupt(w, x, "add_gauss", 0, ACT, t), "add_gauss"
-        scale = float(x.float().abs().mean())
-        if t < w.warmup:
-            gs = gv.update_reference(x, ACT)
-            os_, _ = ov.update_reference(synth.bits(x), ACT)
-            assert_scores_close(gs.cpu().numpy(), os_, scale, "cfg2 warm-up %d" % t)
-        else:
-            thr, valid = ov.thresholds(ACT)
-            gs, gf = gv.verify(x, ACT)
-            os_, of, _ = ov.verify(synth.bits(x), ACT)
-            gf = gf.cpu().numpy().view(np.uint32)
-            assert_scores_close(gs.cpu().numpy(), os_, scale, "cfg2 verify %d" % t)
-            if not np.array_equal(gf, of):
-                near = near_threshold(os_, thr, valid, w.B)
-                assert np.all(near[((gf ^ of) & UNIT_BITS) != 0]), (t, gf, of)
-            if name is not None:
-                assert np.any(of & UNIT_BITS), "additive noise of the tensor's own std is caught"
-    gv.close()
+# (The plain verifier at the full shapes of configurations 2 to 5 -- whole streams, both kinds, in
+# lockstep with oracle processes -- is test_gpu_streams_as_stated.py.)
 
 
 # ---------------------------------------------------------------------------------------------

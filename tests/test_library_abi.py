@@ -33,13 +33,21 @@ def test_library_exports_every_declared_symbol(built):
         assert hasattr(lib, name), name
 
 
+def test_checked_build_exports_the_same_symbols():
+    """The second target (the same sources with bounds checks compiled in) builds and loads too."""
+    from paper_2603_03592_b200 import _build
+    lib = ctypes.CDLL(_build.build_checked())
+    for name in declared_entry_points():
+        assert hasattr(lib, name), name
+
+
 def test_binding_mirrors_the_header(built):
     from paper_2603_03592_b200 import binding
     assert sorted(binding.EXPORTS) == declared_entry_points()
     binding.lib()
     for name in binding.EXPORTS:
         if name in ("sentinel_default_config", "sentinel_distance", "sentinel_distance_noalloc",
-                    "sentinel_sliced_wasserstein"):
+                    "sentinel_sliced_wasserstein", "sentinel_bounds_violations"):
             assert hasattr(binding, name)
         elif name not in ("sentinel_verifier_create", "sentinel_last_error"):
             assert hasattr(binding.Verifier, name), name

@@ -78,3 +78,31 @@ def test_invalid_arguments_are_rejected_before_any_launch(sb):
     assert L.sentinel_distance_noalloc(x.data_ptr(), m.data_ptr(), 65, 4, 16, 0, st, s.data_ptr(), None) == sb.ERR_UNSUPPORTED
     assert L.sentinel_distance_noalloc(x.data_ptr(), m.data_ptr(), 2, 4, 16, 99, st, s.data_ptr(), None) == sb.ERR_INVALID_ARG
     assert b"device" in L.sentinel_last_error(None)
+
+
+def test_calls_after_the_first_take_no_device_memory(sb):
+    """What the entry point is for: once its first call on the device has looked up the built-in
+    array, further calls leave the device's free memory exactly where it was (cudaMemGetInfo
+    before and after, with every tensor of the test created beforehand)."""
+    g = torch.Generator(device="cuda").manual_seed(7)
+    B, T, d = 6, 96, 1024
+    xs = [(torch.randn(B, T, d, generator=g, device="cuda")).to(torch.bfloat16) for _ in range(4)]
+    m = torch.randn(B, T, d, generator=g, device="cuda")
+    outs = [torch.empty(1 + B, 3, device="cuda") for _ in xs]
+    stats = [torch.empty(1 + B, 8, device="cuda") for _ in xs]
+    sb.sentinel_distance_noalloc(xs[0], m, outs[0], stats[0])      # the priming call
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(5):
+        for x, s, st in zip(xs, outs, stats):
+            sb.sentinel_distance_noalloc(x, m, s, st)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, (free_before, free_after)
+    # (the arithmetic of the refusal: 256 bytes of ticket and two 64-byte slots per streaming CTA
+    # must fit the array; this device's launch does, with room)
+    import re, os
+    header = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "sentinel.h")).read()
+    size = int(re.search(r"#define\s+SENTINEL_NOALLOC_SCRATCH_BYTES\s+\(?(\d+)", header).group(1))
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert 256 + 2 * 64 * sms <= size
