@@ -288,7 +288,6 @@ static size_t ref_index(const so_verifier *v, size_t e) {
 
 so_verifier *so_create(const so_params *p) {
   if (p->B < 1 || p->T < 1 || p->d < 1 || p->l < 1 || p->R < 1 || p->R > SO_MAX_WORKERS) return NULL;
-  if (p->ema_bf16 && p->R != 1) return NULL;   /* the bf16 reference exists for one submission per update */
   if (p->ref_over_batch && (p->R != 1 || p->ema_bf16)) return NULL;   /* likewise the [T,d] reference */
   if (p->ref_over_tokens && (p->R != 1 || p->ema_bf16)) return NULL;  /* and the [B,d] / [d] references */
   so_verifier *v = (so_verifier *)calloc(1, sizeof *v);
@@ -317,7 +316,7 @@ so_verifier *so_create(const so_params *p) {
 }
 
 int so_set_directions(so_verifier *v, const uint16_t *u, int n_dir) {
-  if (n_dir < 1 || !u || v->p.ema_bf16 || v->p.ref_over_batch) return -1;
+  if (n_dir < 1 || !u || v->p.ref_over_batch) return -1;
   if (v->ks[0].steps || v->ks[1].steps) return -1;   /* the metric set is fixed before the first step */
   free(v->u);
   v->u = (uint16_t *)malloc((size_t)n_dir * (size_t)v->p.d * sizeof(uint16_t));
@@ -614,6 +613,19 @@ int so_step_replicas(so_verifier *v, const uint16_t *const *xs, int kind, int wa
   if (n_clean > 0) {
     double *m = ks->m;
     const double beta = p->beta[kind];
+    if (p->ema_bf16) {
+      /* The reference is stored as bf16: as for one submission per update, which of two
+       * neighbouring bf16 values an element takes is decided in single precision -- the clean
+       * submissions added up in worker order, weighted by (1-beta)/|clean|, one fused
+       * multiply-add with beta m, one rounding to nearest even. */
+      const float bf = (float)beta, wf = (float)(1.0 - beta) / (float)n_clean;
+      for (size_t e = 0; e < v->N; ++e) {
+        float sum = 0.0f;
+        for (int r = 0; r < R; ++r)
+          if (collected[r] && !tainted[r]) sum += (float)so_bf16(xs[r][e]);
+        m[e] = so_bf16(so_bf16_round((double)fmaf(bf, (float)m[e], wf * sum)));
+      }
+    } else
     for (size_t e = 0; e < v->N; ++e) {
       double sum = 0.0;
       for (int r = 0; r < R; ++r)

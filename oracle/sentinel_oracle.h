@@ -74,7 +74,7 @@ typedef struct so_params {
   unsigned metric_mask;    /* which metrics may raise a flag (bit i = metric i)     */
   int    B, T, d;          /* submission shape                                      */
   int    R;                /* workers (replicas) feeding this boundary, d_s >= 1    */
-  int    ema_bf16;         /* != 0: the reference is stored as bf16 (R = 1 only)    */
+  int    ema_bf16;         /* != 0: the reference is stored as bf16                 */
   int    ref_over_batch;   /* != 0: one [T,d] reference for all B samples (R = 1)   */
   int    ref_over_tokens;  /* != 0: one reference row for all T tokens of a sample: [B,d], or
                               [d] together with ref_over_batch (R = 1)               */

@@ -628,16 +628,53 @@ def test_bf16_reference_settles_within_a_few_ulps_of_a_constant_input(oracle_mod
     assert np.any(m1 != x)                                   # and it is not x itself everywhere
 
 
-def test_bf16_reference_is_for_single_submissions_without_directions(oracle_mod):
-    with pytest.raises(ValueError):
-        make(oracle_mod, ema_bf16=1, R=2)
+def test_bf16_reference_stores_rounded_values(oracle_mod):
     v = make(oracle_mod, ema_bf16=1)
-    with pytest.raises(RuntimeError):
-        v.set_directions(_directions(np.random.default_rng(1), 4, 8))
     rs = np.random.default_rng(34)
     m = rs.normal(0, 1, (2, 4, 8))
     v.set_ema(ACT, m)
     assert np.array_equal(v.ema(ACT), from_bits(to_bits(m)))  # stored rounded
+
+
+def test_bf16_reference_with_several_workers_is_the_single_precision_mean_rounded_once(oracle_mod):
+    """m_t = bf16(fma(beta, m_{t-1}, (1-beta)/n * sum_r x^(r))) in float32, the sum in worker
+    order.  Expected values: every float32 step formed exactly in float64 (operands of 24 bits or
+    fewer) and rounded to float32, then torch's float32 -> bfloat16 conversion."""
+    rs = np.random.default_rng(35)
+    R = 3
+    v = make(oracle_mod, B=2, T=5, d=16, ema_bf16=1, R=R)
+    beta32 = np.float32(0.8)
+    w32 = np.float32(np.float32(1.0 - 0.8) / np.float32(R))
+    m = np.zeros((2, 5, 16), dtype=np.float32)
+    for t in range(8):
+        xbs = [to_bits(rs.normal(-0.3, 1.2, (2, 5, 16))) for _ in range(R)]
+        v.step_replicas(xbs, GRAD, True)
+        total = np.zeros_like(m)
+        for xb in xbs:                                           # float32 adds, in worker order
+            total = (total.astype(np.float64) + from_bits(xb)).astype(np.float32)
+        prod = (np.float64(w32) * total.astype(np.float64)).astype(np.float32)
+        fused = (np.float64(beta32) * m.astype(np.float64) + prod.astype(np.float64)).astype(np.float32)
+        m = _as_bf16_f32(fused)
+        assert np.array_equal(v.ema(GRAD), m.astype(np.float64)), t
+    assert np.all(v.ema(ACT) == 0.0)
+
+
+def test_bf16_reference_takes_directions(oracle_mod):
+    """The sliced Wasserstein column of a bf16-reference verifier is the stateless distance against
+    the stored (rounded) reference."""
+    rs = np.random.default_rng(36)
+    B, T, d = 2, 6, 16
+    v = make(oracle_mod, B=B, T=T, d=d, ema_bf16=1)
+    u = _directions(rs, 4, d)
+    v.set_directions(u)
+    for t in range(4):
+        v.update_reference(to_bits(rs.normal(0, 1, (B, T, d))), ACT)
+    m = v.ema(ACT).copy()
+    xb = to_bits(rs.normal(0, 1, (B, T, d)))
+    scores, _, _ = v.verify(xb, ACT)
+    assert scores.shape[1] == 4
+    assert scores[0, 3] == pytest.approx(oracle_mod.sliced_wasserstein(xb.reshape(B * T, d), m.reshape(B * T, d), u)[0], rel=1e-13)
+    assert scores[2, 3] == pytest.approx(oracle_mod.sliced_wasserstein(xb[1], m[1], u)[0], rel=1e-13)
 
 
 # ---------------------------------------------------------------------------------------------
