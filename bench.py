@@ -383,6 +383,17 @@ def run_after_timed_region(binding, w, args, rank, world, local_rank, fig, m, sa
                                            "bytes_per_element": FOUR_METRIC_BYTES,
                                            "achieved_gbs": round(FOUR_METRIC_BYTES * N / (vms * 1e-3) / 1e9, 1)}
         v4.close()
+        # ... and with the reference stored as bf16: x twice, the reference twice (projected afresh) and written once
+        v4b = binding.Verifier(w.B, w.T, w.d, device=local_rank, ema_bf16=1)
+        v4b.sentinel_set_directions(u, main)
+        for i in range(4):
+            v4b.sentinel_update_reference(pick1(i), ACT, s4, main)
+        v4b.sentinel_verify(pick1(4), ACT, s4, f4, main)
+        wms, wbest, wn = timed_calls(lambda i: v4b.sentinel_verify(pick1(5 + i), ACT, s4, f4, main), main)
+        swd["verify_with_four_metrics_bf16_reference"] = {"ms_per_tensor": round(wms, 4), "ms_best": round(wbest, 4),
+                                                          "calls": wn, "bytes_per_element": 10,
+                                                          "achieved_gbs": round(10 * N / (wms * 1e-3) / 1e9, 1)}
+        v4b.close()
         extra_keys["sliced_wasserstein"] = swd
 
     if extras:   # one iteration with R workers of the stage (2R B/element of tensors + the reference read and written)
@@ -404,6 +415,16 @@ def run_after_timed_region(binding, w, args, rank, world, local_rank, fig, m, sa
             "error_word": int(vr.sentinel_get_counters()["error"]),
             "kernels": "replica_kernel (all workers, speculative mean) + ema_mean_kernel (report bits)"}
         vr.sentinel_destroy()
+        # the same iteration with the reference stored as bf16 (2R + 4 B/element)
+        vb = binding.Verifier(w.B, w.T, w.d, device=local_rank, n_workers=R, ema_bf16=1)
+        for i in range(4):
+            vb.sentinel_update_reference_replicas(pick(i), ACT, rs, rf, main)
+        vb.sentinel_verify_replicas(pick(4), ACT, rs, rf, main)
+        bms, bbest, bn = timed_calls(lambda i: vb.sentinel_verify_replicas(pick(5 + i), ACT, rs, rf, main), main)
+        extra_keys["multi_worker_iteration"]["bf16_reference"] = {
+            "bytes_per_element": 2 * R + 4, "ms_per_iteration": round(bms, 4), "ms_best": round(bbest, 4), "calls": bn,
+            "achieved_gbs": round((2 * R + 4) * N / (bms * 1e-3) / 1e9, 1)}
+        vb.sentinel_destroy()
 
     def single_variant(name, per_el, kernel, **kw):   # a verifier option, one verified tensor per call
         v = binding.Verifier(w.B, w.T, w.d, device=local_rank, **kw)

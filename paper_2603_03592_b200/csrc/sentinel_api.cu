@@ -373,22 +373,22 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned blo
   return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
 }
 
-template <int L, int kT, bool kRefOnly>
+template <int L, int kT, bool kRefOnly, bool kBf16>
 cudaError_t projection_occupancy(size_t smem, int *occ) {
-  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT, kRefOnly>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(swd_project_kernel<L, kT, kRefOnly, kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT, kRefOnly>, kT, smem);
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, swd_project_kernel<L, kT, kRefOnly, kBf16>, kT, smem);
 }
 
-template <int L, bool kRefOnly = false>
-cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
+template <int L, bool kRefOnly = false, bool kBf16 = false>
+cudaError_t launch_projection(const uint16_t *x, const void *m0, const void *m1, const int *active, const int *skip,
                               const uint16_t *u, float *proj, long long rows, int d, int sms, const ProjectionState &ps,
                               cudaStream_t s) {
   const size_t smem = (size_t)L * d * sizeof(uint16_t);
   int occ_small = 0, occ_large = 0;
-  cudaError_t e = projection_occupancy<L, 512, kRefOnly>(smem, &occ_small);
+  cudaError_t e = projection_occupancy<L, 512, kRefOnly, kBf16>(smem, &occ_small);
   if (e != cudaSuccess) return e;
-  e = projection_occupancy<L, 768, kRefOnly>(smem, &occ_large);
+  e = projection_occupancy<L, 768, kRefOnly, kBf16>(smem, &occ_large);
   if (e != cudaSuccess) return e;
   const bool large = occ_large * 768 > occ_small * 512;
   const int threads = large ? 768 : 512, occ = large ? occ_large : occ_small;
@@ -397,9 +397,9 @@ cudaError_t launch_projection(const uint16_t *x, const float *m0, const float *m
   const long long need = (rows + threads / 32 - 1) / (threads / 32);
   if (grid > need) grid = need;
   if (large)
-    return launch_chained(swd_project_kernel<L, 768, kRefOnly>, (unsigned)grid, 768, smem, s, x, m0, m1, active, skip, u, proj,
+    return launch_chained(swd_project_kernel<L, 768, kRefOnly, kBf16>, (unsigned)grid, 768, smem, s, x, m0, m1, active, skip, u, proj,
                           rows, d, ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
-  return launch_chained(swd_project_kernel<L, 512, kRefOnly>, (unsigned)grid, 512, smem, s, x, m0, m1, active, skip, u, proj,
+  return launch_chained(swd_project_kernel<L, 512, kRefOnly, kBf16>, (unsigned)grid, 512, smem, s, x, m0, m1, active, skip, u, proj,
                         rows, d, ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
 }
 
@@ -438,7 +438,8 @@ int check_swd_shape(sentinel_verifier *h, int L, int T, int d) {
 
 // out[0] = the whole tensor, out[1+b] = sample b.  The reference is m1 if *active != 0, else m0;
 // nothing runs if *skip != 0 (both read on the device; either may be nullptr).
-cudaError_t run_swd(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
+// (ref_bf16: m0 / m1 hold bf16 instead of fp32)
+cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_bf16, const int *active, const int *skip,
                     const uint16_t *u, int L, int B, int T, int d, int sms, float *scratch, float *out,
                     const ProjectionState &ps, cudaStream_t s) {
   const long long rows = (long long)B * T;
@@ -449,9 +450,15 @@ cudaError_t run_swd(const uint16_t *x, const float *m0, const float *m1, const i
   if (ps.incremental) {
     e = launch_projection_mma(x, active, skip, u, proj, rows, d, L, sms, ps, s);
   } else {
-    if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    if (ref_bf16) {
+      if (L == 4) e = launch_projection<4, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+      else if (L == 8) e = launch_projection<8, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+      else e = launch_projection<16, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    } else {
+      if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+      else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+      else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    }
   }
   if (e != cudaSuccess) return e;
   int npad = 8;
@@ -490,11 +497,14 @@ int run_handle_swd(sentinel_verifier *h, const void *x, int kind, int worker, bo
   // workers: run_reference_projection has just put P(m) into the current buffer; what the x-only
   // launch writes into the spare one is never adopted.
   ps.incremental = h->R == 1 ? h->sw_pm_valid[kind] : true;
-  SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), static_cast<const float *>(h->ema[kind][0]),
-                           static_cast<const float *>(h->ema[kind][1]), &h->hs->kind[kind].active,
+  // A bf16 reference is rounded when it is stored, so its projections do not follow the recursion:
+  // a single-submission verifier projects it afresh every step (2 + 2 B/element read instead of 2).
+  if (h->bf16 && h->R == 1) { ps.incremental = false; ps.pm0 = ps.pm1 = nullptr; }
+  SENTINEL_CUDA(h, run_swd(static_cast<const uint16_t *>(x), h->ema[kind][0], h->ema[kind][1], h->bf16,
+                           &h->hs->kind[kind].active,
                            may_skip ? &h->hs->banned[worker] : nullptr, h->sw_u, h->sw_L, h->cfg.B, h->cfg.T,
                            h->cfg.d, sms, h->sw_scratch, h->sw_out + (size_t)worker * (1 + h->cfg.B), ps, s));
-  if (h->R == 1) h->sw_pm_valid[kind] = true;      // that launch (re)computed them from m if they were stale
+  if (h->R == 1 && !h->bf16) h->sw_pm_valid[kind] = true;      // that launch (re)computed them from m if they were stale
   return SENTINEL_OK;
 }
 
@@ -507,11 +517,15 @@ int run_reference_projection(sentinel_verifier *h, int kind, cudaStream_t s) {
   ProjectionState ps;
   ps.pm0 = h->sw_pm[kind][0];
   ps.pm1 = h->sw_pm[kind][1];
-  const float *m0 = static_cast<const float *>(h->ema[kind][0]), *m1 = static_cast<const float *>(h->ema[kind][1]);
+  const void *m0 = h->ema[kind][0], *m1 = h->ema[kind][1];
   const int *active = &h->hs->kind[kind].active;
   const long long rows = (long long)h->cfg.B * h->cfg.T;
   cudaError_t e;
-  if (h->sw_L == 4) e = launch_projection<4, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  if (h->bf16) {
+    if (h->sw_L == 4) e = launch_projection<4, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+    else if (h->sw_L == 8) e = launch_projection<8, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+    else e = launch_projection<16, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  } else if (h->sw_L == 4) e = launch_projection<4, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
   else if (h->sw_L == 8) e = launch_projection<8, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
   else e = launch_projection<16, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
   SENTINEL_CUDA(h, e);
@@ -587,8 +601,6 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
   if (cfg->n_workers < 1 || cfg->n_workers > SENTINEL_MAX_WORKERS)
     return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "n_workers = %d is outside 1..%d", cfg->n_workers, SENTINEL_MAX_WORKERS);
   if (cfg->ema_bf16 != 0 && cfg->ema_bf16 != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ema_bf16 must be 0 or 1, got %d", cfg->ema_bf16);
-  if (cfg->ema_bf16 && cfg->n_workers != 1)
-    return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "the bf16 reference is kept for single submissions only (n_workers = 1)");
   if (cfg->ref_over_batch != 0 && cfg->ref_over_batch != 1) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "ref_over_batch must be 0 or 1, got %d", cfg->ref_over_batch);
   if (cfg->ref_over_batch && (cfg->n_workers != 1 || cfg->ema_bf16 || (cfg->B > kMaxWorkers && !cfg->ref_over_tokens) || cfg->d % 8 != 0))
     return fail(nullptr, SENTINEL_ERR_UNSUPPORTED, "a [T,d] reference needs n_workers = 1, an fp32 reference, B <= %d and d a multiple of 8", kMaxWorkers);
@@ -636,8 +648,10 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(stream_kernel_t<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(refresh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (ae == cudaSuccess) ae = cudaFuncSetAttribute(replica_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(shared_ref_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     if (ae == cudaSuccess) ae = cudaFuncSetAttribute(channel_ref_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
@@ -662,8 +676,10 @@ int sentinel_verifier_create(const sentinel_config *cfg, sentinel_verifier **out
       if (cfg->B <= kFewSets) resident_ctas(shared_ref_kernel<true>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
       else resident_ctas(shared_ref_kernel<false>, kThreads, smem, &occ, &oe);
     } else {
-      if (h->R > 1 && h->R <= kFewSets) resident_ctas(replica_kernel<true>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
-      else if (h->R > 1) resident_ctas(replica_kernel<false>, kThreads, smem, &occ, &oe);
+      if (h->R > 1 && h->R <= kFewSets && h->bf16) resident_ctas(replica_kernel<true, true>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
+      else if (h->R > 1 && h->R <= kFewSets) resident_ctas(replica_kernel<true, false>, kFewThreads, std::max(smem, few_smem_bytes()), &occ, &oe);
+      else if (h->R > 1 && h->bf16) resident_ctas(replica_kernel<false, true>, kThreads, smem, &occ, &oe);
+      else if (h->R > 1) resident_ctas(replica_kernel<false, false>, kThreads, smem, &occ, &oe);
       if (h->bf16) {
         resident_ctas(stream_kernel_t<false, true>, kThreads, smem, &occ, &oe);
         resident_ctas(stream_kernel_t<true, true>, kThreads, smem, &occ, &oe);
@@ -906,8 +922,10 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigne
     attr.val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = &attr;
     lc.numAttrs = 1;
-    if (few) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<true>, ra));
-    else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<false>, ra));
+    if (few && h->bf16) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<true, true>, ra));
+    else if (few) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<true, false>, ra));
+    else if (h->bf16) SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<false, true>, ra));
+    else SENTINEL_CUDA(h, cudaLaunchKernelEx(&lc, replica_kernel<false, false>, ra));
   }
   int sms = 0;
   SENTINEL_CUDA(h, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device));
@@ -915,9 +933,14 @@ int step_replicas(sentinel_verifier *h, const void *const *xs, int kind, unsigne
   long long grid = (long long)sms * 8;
   const long long need = (n_chunks + kReplaceThreads - 1) / kReplaceThreads;
   if (grid > need) grid = need;
-  ema_mean_kernel<<<(unsigned)grid, kReplaceThreads, 0, s>>>(
-      h->hs, kind, wp, static_cast<float *>(h->ema[kind][0]), static_cast<float *>(h->ema[kind][1]), n_chunks, h->R, (int)rows, (float)h->cfg.beta[kind],
-      (float)(1.0 - h->cfg.beta[kind]), warmup ? 1 : 0, flags);
+  if (h->bf16)
+    ema_mean_kernel<true><<<(unsigned)grid, kReplaceThreads, 0, s>>>(
+        h->hs, kind, wp, h->ema[kind][0], h->ema[kind][1], n_chunks, h->R, (int)rows, (float)h->cfg.beta[kind],
+        (float)(1.0 - h->cfg.beta[kind]), warmup ? 1 : 0, flags);
+  else
+    ema_mean_kernel<false><<<(unsigned)grid, kReplaceThreads, 0, s>>>(
+        h->hs, kind, wp, h->ema[kind][0], h->ema[kind][1], n_chunks, h->R, (int)rows, (float)h->cfg.beta[kind],
+        (float)(1.0 - h->cfg.beta[kind]), warmup ? 1 : 0, flags);
   SENTINEL_CUDA(h, cudaGetLastError());
   return SENTINEL_OK;
 }
@@ -980,7 +1003,6 @@ int sentinel_set_directions(sentinel_verifier *h, const void *dev_u_bf16, int L,
   if (!h) return fail(nullptr, SENTINEL_ERR_INVALID_ARG, "handle is NULL");
   if (!dev_u_bf16) return fail(h, SENTINEL_ERR_INVALID_ARG, "u is NULL");
   if (h->started) return fail(h, SENTINEL_ERR_INVALID_ARG, "the metric set is fixed once a step was taken or a state imported");
-  if (h->bf16) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads an fp32 reference: not available with ema_bf16");
   if (h->shared_ref || h->chan_ref) return fail(h, SENTINEL_ERR_UNSUPPORTED, "the sliced Wasserstein chain reads a [B,T,d] reference: not available with ref_over_batch");
   if (h->cfg.d % 8 != 0) return fail(h, SENTINEL_ERR_UNALIGNED, "d = %d is not a multiple of 8", h->cfg.d);
   int rc = check_swd_shape(h, L, h->cfg.T, h->cfg.d);
@@ -1051,7 +1073,7 @@ int sentinel_sliced_wasserstein(const void *dev_x, const float *dev_m, const voi
   float *scratch = nullptr;
   keep_pool_warm(device);
   SENTINEL_CUDA(nullptr, cudaMallocAsync((void **)&scratch, swd_scratch_floats(L, B, T) * sizeof(float), s));
-  cudaError_t e = run_swd(static_cast<const uint16_t *>(dev_x), dev_m, nullptr, nullptr, nullptr,
+  cudaError_t e = run_swd(static_cast<const uint16_t *>(dev_x), dev_m, nullptr, false, nullptr, nullptr,
                           static_cast<const uint16_t *>(dev_u_bf16), L, B, T, d, sms, scratch, dev_sw_out,
                           ProjectionState(), s);
   cudaError_t fe = cudaFreeAsync(scratch, s);

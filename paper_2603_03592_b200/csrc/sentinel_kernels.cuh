@@ -1990,15 +1990,19 @@ __device__ __noinline__ unsigned few_nonfinite_in_tile(const unsigned char *stag
 }
 // Exact zeros of tensor r whose sign bit equals that of m, in the chunks where the packed sign
 // test ran (it did not count them): each is a mismatch all the same.  Returns their number.
-__device__ __noinline__ unsigned few_uncounted_zeros(const unsigned char *stage, int r, int lane, unsigned valid) {
+// (ref_bf16: the staged tile of the reference holds bf16)
+__device__ __noinline__ unsigned few_uncounted_zeros(const unsigned char *stage, int r, int lane, unsigned valid,
+                                                     int ref_bf16) {
   unsigned n = 0u;
   for (int u = 0; u < kUnroll; ++u) {
     if (!((valid >> u) & 1u)) continue;
     const uint16_t *xw = reinterpret_cast<const uint16_t *>(stage + kTileBytesM + r * kTileBytesX + (size_t)(u * 32 + lane) * 16);
     const unsigned *mw = reinterpret_cast<const unsigned *>(stage + (size_t)(u * 32 + lane) * 32);
+    const uint16_t *mh = reinterpret_cast<const uint16_t *>(stage + (size_t)(u * 32 + lane) * 16);
     for (int e = 0; e < 8; ++e) {
       const unsigned xb = xw[e];
-      if ((xb & 0x7FFFu) == 0u && (xb >> 15) == (mw[e] >> 31)) ++n;
+      const unsigned m_sign = ref_bf16 ? (unsigned)(mh[e] >> 15) : (mw[e] >> 31);
+      if ((xb & 0x7FFFu) == 0u && (xb >> 15) == m_sign) ++n;
     }
   }
   return n;
@@ -2006,9 +2010,12 @@ __device__ __noinline__ unsigned few_uncounted_zeros(const unsigned char *stage,
 
 // Rows [r0, r1) of the flat [rows, d] view, of which [r0, cut) lie in sample b0 and [cut, r1) in
 // sample b0 + 1 (cut = r1: one segment).  kFull: d is a multiple of the warp tile, no ragged tile.
-template <int NR, bool kFull>
+// kBf16: the reference buffers hold bf16 (its tile is staged as 1 KB, widened when read, and the
+// candidate is rounded to nearest even when stored).
+template <int NR, bool kFull, bool kBf16>
 __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int b0, long long r0, long long cut,
-                         long long r1, const float *m_in, float *m_out, int c, FewShared &fs, FewWarp *fw_all) {
+                         long long r1, const void *m_in, void *m_out, int c, FewShared &fs, FewWarp *fw_all) {
+  constexpr unsigned kRefChunkBytes = kBf16 ? 16u : 32u;     // a lane's 8 elements of the reference
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunks = a.d >> 3;                               // d is a multiple of 8 here
   const int tiles_per_row = (chunks + 32 * kUnroll - 1) / (32 * kUnroll);
@@ -2037,7 +2044,7 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     if (sg == 0 || cut < r1) fs.x0[sg][r] = fs.ptr[r][sample_off];
   } else if (tid >= 32 && tid < 32 + kSegsPerCta) {
     const int sg = tid - 32;
-    if (sg == 0 || cut < r1) fs.m0bits[sg] = __float_as_uint(m_in[(size_t)(b0 + sg) * a.T * a.d]);
+    if (sg == 0 || cut < r1) fs.m0bits[sg] = __float_as_uint(load_m1<kBf16>(m_in, (size_t)(b0 + sg) * a.T * a.d));
   }
 
   // the warp's tiles: tile number j = warp + t * kFewWarps is row r0 + j / tiles_per_row, 512
@@ -2055,8 +2062,8 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
       const unsigned bar = smem_addr(&fw.bar[st]), dst = smem_addr(&fw.stage[st][0]);
       if (SENTINEL_BOUNDS(kSiteStageRef, off, (long long)vc * 8, a.ref_extent) &&
           SENTINEL_BOUNDS(kSiteStageX, off, (long long)vc * 8, a.x_extent)) {
-        mbar_arrive_expect(bar, (unsigned)vc * (32u + 16u * NR));
-        bulk_copy_in(dst, m_in + off, (unsigned)vc * 32u, bar);
+        mbar_arrive_expect(bar, (unsigned)vc * (kRefChunkBytes + 16u * NR));
+        bulk_copy_in(dst, static_cast<const unsigned char *>(m_in) + off * (kBf16 ? 2 : 4), (unsigned)vc * kRefChunkBytes, bar);
 #pragma unroll
         for (int r = 0; r < NR; ++r)
           bulk_copy_in(dst + kTileBytesM + r * kTileBytesX, fs.ptr[r] + off, (unsigned)vc * 16u, bar);
@@ -2151,12 +2158,16 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
       float sum[8];
       float mmin = 1.f;
       if (ok) {
-        const float4 *src = reinterpret_cast<const float4 *>(stage + (size_t)(u * 32 + lane) * 32);
-        const float4 lo = src[0], hi = src[1];
-        mv.v[0] = lo.x; mv.v[1] = lo.y; mv.v[2] = lo.z; mv.v[3] = lo.w;
-        mv.v[4] = hi.x; mv.v[5] = hi.y; mv.v[6] = hi.z; mv.v[7] = hi.w;
-        mmin = fminf(fminf(fminf(fabsf(lo.x), fabsf(lo.y)), fminf(fabsf(lo.z), fabsf(lo.w))),
-                     fminf(fminf(fabsf(hi.x), fabsf(hi.y)), fminf(fabsf(hi.z), fabsf(hi.w))));
+        if (kBf16) {
+          mv = widen_bf16x8(*reinterpret_cast<const uint4 *>(stage + (size_t)(u * 32 + lane) * 16));
+        } else {
+          const float4 *src = reinterpret_cast<const float4 *>(stage + (size_t)(u * 32 + lane) * 32);
+          const float4 lo = src[0], hi = src[1];
+          mv.v[0] = lo.x; mv.v[1] = lo.y; mv.v[2] = lo.z; mv.v[3] = lo.w;
+          mv.v[4] = hi.x; mv.v[5] = hi.y; mv.v[6] = hi.z; mv.v[7] = hi.w;
+        }
+        mmin = fminf(fminf(fminf(fabsf(mv.v[0]), fabsf(mv.v[1])), fminf(fabsf(mv.v[2]), fabsf(mv.v[3]))),
+                     fminf(fminf(fabsf(mv.v[4]), fabsf(mv.v[5])), fminf(fabsf(mv.v[6]), fabsf(mv.v[7]))));
 #pragma unroll
         for (int e = 0; e < 8; ++e) {                        // the reference's own sums, once per tile
           sum[e] = 0.f;
@@ -2184,7 +2195,7 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
 #pragma unroll
         for (int e = 0; e < 8; ++e) mv.v[e] = fmaf(beta, mv.v[e], wgt * sum[e]);
         if (SENTINEL_BOUNDS(kSiteRefOut, off + (size_t)(base + u * 32 + lane) * 8, 8, a.ref_extent))
-          st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv);
+          store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, mv);
       }
     }
     unsigned valid = 0u;                                     // this lane's chunks of the tile
@@ -2195,7 +2206,7 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
     // equals that of m was not counted
     if (__any_sync(0xffffffffu, ((zmin & 0x7FFFu) == 0u) || ((zmin & 0x7FFF0000u) == 0u))) {
 #pragma unroll
-      for (int r = 0; r < NR; ++r) fl[r] += kFlipUnit * few_uncounted_zeros(stage, r, lane, valid & fast_chunks);
+      for (int r = 0; r < NR; ++r) fl[r] += kFlipUnit * few_uncounted_zeros(stage, r, lane, valid & fast_chunks, kBf16 ? 1 : 0);
     }
     // a sum of |x - m| that is not a finite number: look at the exponent bits of that tensor's tile
 #pragma unroll
@@ -2251,31 +2262,33 @@ __device__ void few_rows(const StreamArgs &a, unsigned long long *partials, int 
   }
 }
 
+template <bool kBf16>
 __device__ __forceinline__ void few_dispatch(int n, const StreamArgs &a, unsigned long long *partials, int b0,
-                                             long long r0, long long cut, long long r1, const float *m_in, float *m_out,
+                                             long long r0, long long cut, long long r1, const void *m_in, void *m_out,
                                              int c, FewShared &fs, double *s_dyn) {
   FewWarp *fw = reinterpret_cast<FewWarp *>(s_dyn);
   if (a.d % (32 * kUnroll * 8) == 0) {
     switch (n) {
-      case 1: few_rows<1, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
-      case 2: few_rows<2, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
-      case 3: few_rows<3, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
-      default: few_rows<4, true>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 1: few_rows<1, true, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 2: few_rows<2, true, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 3: few_rows<3, true, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      default: few_rows<4, true, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
     }
   } else {
     switch (n) {
-      case 1: few_rows<1, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
-      case 2: few_rows<2, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
-      case 3: few_rows<3, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
-      default: few_rows<4, false>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 1: few_rows<1, false, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 2: few_rows<2, false, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      case 3: few_rows<3, false, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
+      default: few_rows<4, false, kBf16>(a, partials, b0, r0, cut, r1, m_in, m_out, c, fs, fw); break;
     }
   }
 }
 
 // (n_sets tensors share the tile of m: the R workers of a stage, or the B samples of one tensor
 // when the reference is a single [T,d] tensor for all of them)
+template <bool kBf16>
 __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long long row_a, long long row_b,
-                                const float *m_in, float *m_out, unsigned streamed, int c, int sgm,
+                                const void *m_in, void *m_out, unsigned streamed, int c, int sgm,
                                 ReplicaShared &sh) {
   const StreamArgs &a = ra.s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -2294,7 +2307,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
   }
   if (threadIdx.x < kWarps) { sh.m_acc[threadIdx.x][0] = sh.m_acc[threadIdx.x][1] = 0.; sh.m_varies[threadIdx.x] = 0u; }
   if (threadIdx.x < n_sets && ((streamed >> threadIdx.x) & 1u)) sh.x0[threadIdx.x] = ra.xs[threadIdx.x][sample_off];
-  const unsigned m0bits = __float_as_uint(m_in[sample_off]);
+  const unsigned m0bits = __float_as_uint(load_m1<kBf16>(m_in, sample_off));
   const float m0 = __uint_as_float(m0bits);
   __syncthreads();
 
@@ -2312,7 +2325,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
       const int ch = base + u * 32 + lane;
       ok[u] = ch < chunks;
       if (ok[u]) {
-        mv[u] = ld_m256(m_in + off + (size_t)ch * 8);
+        mv[u] = load_m8<kBf16>(m_in, off + (size_t)ch * 8);
         xv[u] = ld_x128(ra.xs[first] + off + (size_t)ch * 8);
       }
     }
@@ -2382,7 +2395,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
       if (!ok[u]) continue;
 #pragma unroll
       for (int e = 0; e < 8; ++e) mv[u].v[e] = fmaf(beta, mv[u].v[e], wgt * sum[u][e]);
-      st_m256(m_out + off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
+      store_m8<kBf16>(m_out, off + (size_t)(base + u * 32 + lane) * 8, mv[u]);
     }
     rr += step_rr;
     seg += step_seg;
@@ -2416,7 +2429,7 @@ __device__ void replica_segment(const ReplicaArgs &ra, int n_sets, int b, long l
 
 // (kFew: a handle that follows at most kFewSets workers -- their sums stay in registers; a kernel
 // of its own, with its own CTA size, so that neither form pays for the other's registers)
-template <bool kFew>
+template <bool kFew, bool kBf16 = false>
 __global__ void __launch_bounds__(kFew ? kFewThreads : kThreads)
 replica_kernel(const ReplicaArgs ra) {
   __shared__ typename std::conditional<kFew, FewShared, ReplicaShared>::type sh;
@@ -2457,14 +2470,12 @@ replica_kernel(const ReplicaArgs ra) {
     const int b0 = (int)(r0 / a.T);
     const long long cut = ((long long)(b0 + 1) * a.T < r1) ? (long long)(b0 + 1) * a.T : r1;
     if constexpr (kFew) {
-      few_dispatch(n_streamed, a, ra.partials, b0, r0, cut, r1, static_cast<const float *>(a.ema[act]),
-                   static_cast<float *>(a.ema[act ^ 1]), c, sh, s_dyn);
+      few_dispatch<kBf16>(n_streamed, a, ra.partials, b0, r0, cut, r1, a.ema[act], a.ema[act ^ 1], c, sh, s_dyn);
     } else {
       for (int sgm = 0; sgm < kSegsPerCta; ++sgm) {
         const long long row = sgm ? cut : r0, row_b = sgm ? r1 : cut;
         if (row < row_b)
-          replica_segment(ra, a.R, b0 + sgm, row, row_b, static_cast<const float *>(a.ema[act]),
-                          static_cast<float *>(a.ema[act ^ 1]), streamed, c, sgm, sh);
+          replica_segment<kBf16>(ra, a.R, b0 + sgm, row, row_b, a.ema[act], a.ema[act ^ 1], streamed, c, sgm, sh);
         else if (threadIdx.x < a.R)
           ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + sgm) * kSlotWords + 7] = 0ull;   // unused
       }
@@ -2532,11 +2543,9 @@ shared_ref_kernel(const ReplicaArgs ra) {
     const long long r0 = ((long long)a.T * c) / a.G, r1 = ((long long)a.T * (c + 1)) / a.G;   // token rows
     if constexpr (kFew) {
       if (threadIdx.x < a.B) { sh.ptr[threadIdx.x] = ra.xs[threadIdx.x]; sh.widx[threadIdx.x] = threadIdx.x; }
-      few_dispatch(a.B, a, ra.partials, 0, r0, r1, r1, static_cast<const float *>(a.ema[act]),
-                   static_cast<float *>(a.ema[act ^ 1]), c, sh, s_dyn);
+      few_dispatch<false>(a.B, a, ra.partials, 0, r0, r1, r1, a.ema[act], a.ema[act ^ 1], c, sh, s_dyn);
     } else {
-      replica_segment(ra, a.B, 0, r0, r1, static_cast<const float *>(a.ema[act]), static_cast<float *>(a.ema[act ^ 1]),
-                      all, c, 0, sh);
+      replica_segment<false>(ra, a.B, 0, r0, r1, a.ema[act], a.ema[act ^ 1], all, c, 0, sh);
     }
     if (!kFew && threadIdx.x < a.B)              // the second slot of every pair stays unused
       ra.partials[(((size_t)threadIdx.x * a.G + c) * kSegsPerCta + 1) * kSlotWords + 7] = 0ull;
@@ -2624,8 +2633,9 @@ replace_kernel(const HandleState *hs, int kind, const void *ema0, const void *em
 // Traffic when it runs: 4 B read + 4 B written of m and 2 B per clean worker, per element.
 struct WorkerPointers { const uint16_t *x[kMaxWorkers]; };
 
+template <bool kBf16>
 __global__ void __launch_bounds__(kReplaceThreads)
-ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, float *ema0, float *ema1, long long n_chunks,
+ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, void *ema0, void *ema1, long long n_chunks,
                 int R, int rows, float beta, float one_minus_beta, int warmup, unsigned *flags_out) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   KindState *ks = &hs->kind[kind];
@@ -2645,11 +2655,11 @@ ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, float *ema0, float
         flags_out[(size_t)r * rows] |= ((clean >> r) & 1u ? kFlagCommitted : 0u) | (natural ? kFlagNaturalShift : 0u);
   }
   if (n_clean == 0 || done) return;
-  float *m = ks->active ? ema1 : ema0;
+  void *m = ks->active ? ema1 : ema0;
   const float wgt = one_minus_beta / (float)n_clean;
   const long long stride = (long long)gridDim.x * kReplaceThreads;
   for (long long c = (long long)blockIdx.x * kReplaceThreads + threadIdx.x; c < n_chunks; c += stride) {
-    F8 mv = ld_m256(m + c * 8);
+    F8 mv = load_m8<kBf16>(m, (size_t)c * 8);
     float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     for (int r = 0; r < R; ++r) {
       if (!((clean >> r) & 1u)) continue;
@@ -2663,7 +2673,7 @@ ema_mean_kernel(HandleState *hs, int kind, WorkerPointers xs, float *ema0, float
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) mv.v[j] = fmaf(beta, mv.v[j], wgt * sum[j]);
-    st_m256(m + c * 8, mv);
+    store_m8<kBf16>(m, (size_t)c * 8, mv);
   }
 }
 

@@ -43,16 +43,18 @@ constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are
 // else is written): once per iteration of a verifier that follows several workers, whose
 // reference moves with the mean over the clean workers rather than by that recursion; its
 // workers then all take the x-only launch against the same P(m).
-template <int L, int kSwdThreads, bool kRefOnly = false>
+// kBf16: the reference buffers hold bf16 (widened on load; such a verifier projects its reference
+// afresh every step, because the rounding of the stored reference does not follow the recursion).
+template <int L, int kSwdThreads, bool kRefOnly = false, bool kBf16 = false>
 __global__ void __launch_bounds__(kSwdThreads, kSwdThreads == 512 ? 2 : 1)
-swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const int *active, const int *skip,
+swd_project_kernel(const uint16_t *x, const void *m0, const void *m1, const int *active, const int *skip,
                    const uint16_t *u, float *proj, long long rows, int d, double *pm0, double *pm1, float beta,
                    float one_minus_beta) {
   extern __shared__ uint4 s_u[];                 // [L][d/8], 8 bf16 each
   chain_entry();
   if (skip && __ldcg(skip)) return;
   const bool second = active && __ldcg(active);
-  const float *m = second ? m1 : m0;
+  const void *m = second ? m1 : m0;
   double *pm_cur = second ? pm1 : pm0, *pm_next = second ? pm0 : pm1;
   const int chunks = d >> 3;
   for (int i = threadIdx.x; i < L * chunks; i += kSwdThreads)
@@ -78,7 +80,7 @@ swd_project_kernel(const uint16_t *x, const float *m0, const float *m1, const in
         ok[h] = c < chunks;
         if (ok[h]) {
           if (!kRefOnly) xv[h] = ld_x128(x + off + (size_t)c * 8);
-          mv[h] = ld_m256(m + off + (size_t)c * 8);
+          mv[h] = load_m8<kBf16>(m, off + (size_t)c * 8);
         }
       }
 #pragma unroll

@@ -740,15 +740,12 @@ def test_bf16_reference_with_strided_rows(sb, oracle_mod):
 
 def test_bf16_reference_restrictions_and_state_round_trip(sb):
     with pytest.raises(sb.SentinelError) as e:
-        sb.Verifier(2, 8, 64, ema_bf16=1, n_workers=2)
-    assert e.value.code == sb.ERR_UNSUPPORTED
-    with pytest.raises(sb.SentinelError) as e:
         sb.Verifier(2, 8, 64, ema_bf16=2)
     assert e.value.code == sb.ERR_INVALID_ARG
-    gv = sb.Verifier(2, 8, 64, ema_bf16=1)
     with pytest.raises(sb.SentinelError) as e:
-        gv.sentinel_set_directions(synth.directions(4, 64, 1, "cuda"))
+        sb.Verifier(2, 8, 64, ema_bf16=1, ref_over_batch=1)
     assert e.value.code == sb.ERR_UNSUPPORTED
+    gv = sb.Verifier(2, 8, 64, ema_bf16=1)
     w = synth.scaled(synth.WORKLOADS["cfg1"], "bf16_rt", 2, 8, 64)
     for t in range(5):
         gv.update_reference(synth.clean(w, 0, ACT, t, "cuda"), ACT)

@@ -241,3 +241,32 @@ def test_skip_tainted_single_submission(sb, oracle_mod):
     torch.cuda.synchronize()
     assert replaced.item() == 0
     gv.close()
+
+
+@pytest.mark.parametrize("shape,R", [((3, 12, 264), 4), ((2, 20, 1024), 2), ((4, 6, 64), 7)],
+                         ids=["3x12x264_R4", "2x20x1024_R2", "4x6x64_R7"])
+def test_iterations_in_lockstep_with_a_bf16_reference(sb, oracle_mod, shape, R):
+    """The fixed-mesh verifier (several workers per iteration) with the reference stored as bf16:
+    warm-up, clean iterations (the mean written by the scoring launch), a tainted worker (the mean
+    over the clean ones taken afterwards), a flagged majority; the stored reference agrees with the
+    oracle's bit for bit after every iteration."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "replicas_bf16", *shape)
+    gv, ov, params = pair(sb, oracle_mod, w, R, l=5, c=3, ema_bf16=1)
+    script = [("warm", {})] * 6 + [("verify", {})] * 2 + [("verify", {1: 6.0})] + [("verify", {})] + \
+             [("verify", {r: 3.0 for r in range(R // 2 + 1)})] + [("verify", {})]
+    for t, (what, scale) in enumerate(script):
+        xs = inputs(w, R, ACT, t, scale)
+        thr, valid = ov.thresholds(ACT)
+        gs, gf, os_, of, n = step_both(gv, ov, xs, ACT, warmup=(what == "warm"))
+        for r in range(R):
+            assert_scores_close(gs[r], os_[r], float(xs[r].float().abs().mean()), "step %d worker %d" % (t, r))
+        if what != "warm" and not np.array_equal(gf, of):
+            for r in range(R):
+                near = near_threshold(os_[r], thr, valid, w.B)
+                assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            gv.sentinel_import_state(oracle_to_blob(ov, params))
+        if whole_step_k_events(*gv.sentinel_get_thresholds(ACT), *ov.thresholds(ACT), params, ACT):
+            gv.sentinel_import_state(oracle_to_blob(ov, params))
+        st = parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, params.l, R)
+        assert np.array_equal(st["kinds"][ACT]["m"].astype(np.float64), ov.ema(ACT)), t
+    gv.close()

@@ -266,3 +266,20 @@ def test_directions_argument_checks(sb):
         big.sentinel_set_directions(u)                                      # four windows' copies do not fit
     assert e.value.code == sb.ERR_UNSUPPORTED
     big.close()
+
+
+def test_streams_in_lockstep_with_four_metrics_and_a_bf16_reference(sb, oracle_mod):
+    """Directions on a verifier whose reference is stored as bf16: the reference is projected
+    afresh every step (its stored values are rounded, so its projections do not follow Eq. 1's
+    recursion); four columns in lockstep, the stored reference bit for bit."""
+    w = synth.scaled(synth.WORKLOADS["cfg2"], "cfg2_sw_bf16", 4, 40, 264, corrupt_rate=0.25)
+    gv, ov, params = make_pair(sb, oracle_mod, w, ema_bf16=1)
+    with_directions(gv, ov, 8, w.d)
+    rec = lockstep(sb, oracle_mod, w, gv, ov, params, 40)
+    assert rec["corrupted"] >= 3
+    st = parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, params.l)
+    for kind in (ACT, GRAD):
+        assert np.array_equal(st["kinds"][kind]["m"].astype(np.float64), ov.ema(kind))
+        compare_thresholds(gv, ov, kind)
+    assert rec["near"] <= 2 and rec["k_events"] <= 4, rec
+    gv.close()

@@ -107,7 +107,7 @@ def test_host_side_argument_checks_need_no_gpu(built):
         cfg = binding.sentinel_default_config(B=2, T=4, d=16, **bad)
         assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_INVALID_ARG, bad
     # combinations of variants that are not built
-    for bad in (dict(ref_over_tokens=1, n_workers=2), dict(ref_over_batch=1, n_workers=2), dict(ema_bf16=1, n_workers=2),
+    for bad in (dict(ref_over_tokens=1, n_workers=2), dict(ref_over_batch=1, n_workers=2), dict(ema_bf16=1, ref_over_batch=1),
                 dict(ref_over_batch=1, ref_over_tokens=1, ema_bf16=1)):
         cfg = binding.sentinel_default_config(B=2, T=4, d=16, **bad)
         assert L.sentinel_verifier_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.ERR_UNSUPPORTED, bad
