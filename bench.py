@@ -133,11 +133,15 @@ def build_stream(w, boundary, device, count, distinct):
 MIN_TIMED_MS = 200.0            # device time the timed region covers at least, whatever --steps is
 
 
-def timed_calls(fn, stream, min_ms=60.0, min_calls=6, max_calls=400):
+EXTRAS_MIN_MS = 60.0            # device time each figure after the timed region covers at least (--extras-ms)
+
+
+def timed_calls(fn, stream, min_ms=None, min_calls=6, max_calls=400):
     """Median and best duration (ms) of fn(i), one CUDA-event pair per call on `stream`, over at
     least min_calls calls and min_ms of device time."""
     durations = []
     i = 0
+    min_ms = EXTRAS_MIN_MS if min_ms is None else min_ms
     while True:
         batch = min_calls if not durations else max(2, min(64, int(min_calls * 1.5)))
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(batch + 1)]
@@ -675,11 +679,15 @@ def main():
                     help="skip the extra figures measured after the timed region")
     ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
                     help="device time the timed region covers at least (the steps are gone through again)")
+    ap.add_argument("--extras-ms", type=float, default=EXTRAS_MIN_MS,
+                    help="device time each figure taken after the timed region covers at least")
     ap.add_argument("--also", default="cfg3,cfg5",
                     help="workloads measured after the default one (cfg4) in the same run; '' for none")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the current kernel, if known")
     args = ap.parse_args()
+    global EXTRAS_MIN_MS
+    EXTRAS_MIN_MS = args.extras_ms
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":        # rank 0 alone works; no process group is needed
