@@ -664,6 +664,7 @@ def run_reference(args, rank, world):
 
 
 def main():
+    global EXTRAS_MIN_MS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
@@ -686,7 +687,6 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the current kernel, if known")
     args = ap.parse_args()
-    global EXTRAS_MIN_MS
     EXTRAS_MIN_MS = args.extras_ms
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
