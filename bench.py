@@ -372,7 +372,7 @@ def run_after_timed_region(binding, w, args, rank, world, local_rank, fig, m, sa
         sms, sbest, sn = timed_calls(lambda i: binding.sentinel_sliced_wasserstein(pick1(i), ref, u, sw, main), main)
         swd = {"directions": 8, "bytes_per_element": 6, "ms_per_call": round(sms, 4), "ms_best": round(sbest, 4),
                "calls": sn, "achieved_gbs": round(6 * N / (sms * 1e-3) / 1e9, 1),
-               "kernels": "swd_project_kernel + sort, merge, finish", "value_row0": float(sw[0])}
+               "kernels": "swd_project_ref_mma_kernel + swd_sort_samples_kernel + swd_merge_kernel (all rounds but the last) + swd_w1_kernel", "value_row0": float(sw[0])}
         del ref
         # the same distance as the verifier's fourth metric: one verified tensor per call
         v4 = binding.Verifier(w.B, w.T, w.d, device=local_rank)

@@ -119,9 +119,12 @@ typedef struct sentinel_verifier sentinel_verifier; /* opaque: one stage boundar
  * the update is m_t = bf16(fma(beta, m_{t-1}, (1-beta) x)) in single precision with one
  * rounding to nearest even, so a reference stops moving once (1-beta)|x - m| falls below half
  * a bf16 ulp of m (it settles within 1/(2(1-beta)) ulps of a steady input).  Scores, bounds and
- * flags are computed exactly as with fp32, against the rounded reference.  Restrictions:
- * n_workers = 1, no sentinel_set_directions.  State blobs carry the reference as fp32 either
- * way (widened exactly on export, rounded to nearest even on import). */
+ * flags are computed exactly as with fp32, against the rounded reference.  With n_workers > 1
+ * the mean over the clean workers is taken in single precision in worker order and enters the
+ * same one-rounding update; with sentinel_set_directions the projections of the reference are
+ * taken from the stored bf16 values every step (a rounded reference does not follow the linear
+ * recursion), so the chain reads 2 + 2 B/element.  State blobs carry the reference as fp32
+ * either way (widened exactly on export, rounded to nearest even on import). */
 /* ref_over_batch = 1 keeps ONE reference of shape [T,d] for all B samples of a tensor instead of
  * a [B,T,d] one (the paper states the reference only as "the EMA of the signal"; this reading
  * treats the samples of a microbatch as draws of the same [T,d] signal): every sample is compared
@@ -176,8 +179,9 @@ int sentinel_verify(sentinel_verifier *h, const void *dev_x, sentinel_kind kind,
  * Every later step first runs the projection / sort launches on the caller's stream, then the
  * streaming launch, which picks the distances up.  With one submission per update the
  * projections of the reference are carried along from step to step (Eq. 1 is linear), so the
- * chain reads x once more (2 B/element) and not the reference; with n_workers > 1, and on the
- * first step after sentinel_import_state, it reads the reference too (6 B/element).  The projections are fp32: inputs whose
+ * chain reads x once more (2 B/element) and not the reference; with n_workers > 1, with a
+ * bf16 reference, and on the first step after sentinel_import_state, it reads the reference
+ * too.  The projections are fp32: inputs whose
  * projections leave the fp32 range give a score that is not a number, which counts as a
  * flag.  Allowed only before the first step and before sentinel_import_state
  * (SENTINEL_ERR_INVALID_ARG afterwards); the four windows' working copies must fit the

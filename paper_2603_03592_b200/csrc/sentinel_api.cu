@@ -423,10 +423,42 @@ cudaError_t launch_projection_mma(const uint16_t *x, const int *active, const in
   }
 }
 
-// floats of scratch: the projections and two buffers of sorted lists (2L lists of B*T each),
-// then W1 per (sample, direction) and per direction
+// x and the stored reference (or the reference alone) on the tensor cores.  *fits = false, and
+// nothing is launched, if the directions and the warps' partial sums do not fit in shared memory
+// together (the caller then takes swd_project_kernel).
+template <int NB, bool kWithX, bool kBf16>
+cudaError_t launch_projection_ref_mma_nb(const uint16_t *x, const void *m0, const void *m1, const int *active, const int *skip,
+                                         const uint16_t *u, float *proj, long long rows, int d, int L, int sms,
+                                         const ProjectionState &ps, cudaStream_t s, bool *fits) {
+  const size_t smem = (size_t)L * swd_mma_stride(d >> 3) * sizeof(uint4) +
+                      (size_t)kSwdRefWarps * (kWithX ? 2 : 1) * NB * 4 * 32 * sizeof(float);
+  *fits = smem <= 227u * 1024u;
+  if (!*fits) return cudaSuccess;
+  const long long n_tasks = (rows + 15) / 16;
+  const unsigned grid = (unsigned)(n_tasks < sms ? n_tasks : sms);
+  cudaError_t e = cudaFuncSetAttribute(swd_project_ref_mma_kernel<NB, kWithX, kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e != cudaSuccess) return e;
+  return launch_chained(swd_project_ref_mma_kernel<NB, kWithX, kBf16>, grid, kSwdRefThreads, smem, s, x, m0, m1, active, skip, u,
+                        proj, rows, d, L, ps.pm0, ps.pm1, ps.beta, ps.one_minus_beta);
+}
+
+template <bool kWithX>
+cudaError_t launch_projection_ref_mma(const uint16_t *x, const void *m0, const void *m1, bool ref_bf16, const int *active,
+                                      const int *skip, const uint16_t *u, float *proj, long long rows, int d, int L, int sms,
+                                      const ProjectionState &ps, cudaStream_t s, bool *fits) {
+  if (L == 16) {
+    if (ref_bf16) return launch_projection_ref_mma_nb<2, kWithX, true>(x, m0, m1, active, skip, u, proj, rows, d, L, sms, ps, s, fits);
+    return launch_projection_ref_mma_nb<2, kWithX, false>(x, m0, m1, active, skip, u, proj, rows, d, L, sms, ps, s, fits);
+  }
+  if (ref_bf16) return launch_projection_ref_mma_nb<1, kWithX, true>(x, m0, m1, active, skip, u, proj, rows, d, L, sms, ps, s, fits);
+  return launch_projection_ref_mma_nb<1, kWithX, false>(x, m0, m1, active, skip, u, proj, rows, d, L, sms, ps, s, fits);
+}
+
+// floats of scratch: the projections, the sorted lists and one more buffer of that size for the
+// merge rounds (2L lists of B*T each; the projections are free again by then and serve as the
+// other buffer), then swd_w1_kernel's per-CTA sums (doubles) and its ticket word
 size_t swd_scratch_floats(int L, int B, int T) {
-  return (size_t)3 * 2 * L * ((size_t)B * T) + (size_t)(B + 1) * L;
+  return (size_t)3 * 2 * L * ((size_t)B * T) + 2 * swd_w1_partials(L, B, T) + 4;
 }
 
 int check_swd_shape(sentinel_verifier *h, int L, int T, int d) {
@@ -444,20 +476,25 @@ cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_
                     const ProjectionState &ps, cudaStream_t s) {
   const long long rows = (long long)B * T;
   const size_t list_floats = (size_t)2 * L * rows;        // L lists for x, L for m
-  float *proj = scratch, *buf_a = proj + list_floats, *buf_b = buf_a + list_floats, *w1_sample = buf_b + list_floats;
-  float *w1_tensor = w1_sample + (size_t)B * L;
+  float *proj = scratch, *sorted = proj + list_floats, *spare = sorted + list_floats;
+  double *partial = reinterpret_cast<double *>(spare + list_floats);      // (list_floats is even: 8-byte aligned)
+  unsigned *ticket = reinterpret_cast<unsigned *>(partial + swd_w1_partials(L, B, T));
   cudaError_t e;
   if (ps.incremental) {
     e = launch_projection_mma(x, active, skip, u, proj, rows, d, L, sms, ps, s);
   } else {
-    if (ref_bf16) {
-      if (L == 4) e = launch_projection<4, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-      else if (L == 8) e = launch_projection<8, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-      else e = launch_projection<16, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-    } else {
-      if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-      else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
-      else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+    bool fits = false;
+    e = launch_projection_ref_mma<true>(x, m0, m1, ref_bf16, active, skip, u, proj, rows, d, L, sms, ps, s, &fits);
+    if (e == cudaSuccess && !fits) {
+      if (ref_bf16) {
+        if (L == 4) e = launch_projection<4, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+        else if (L == 8) e = launch_projection<8, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+        else e = launch_projection<16, false, true>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+      } else {
+        if (L == 4) e = launch_projection<4>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+        else if (L == 8) e = launch_projection<8>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+        else e = launch_projection<16>(x, m0, m1, active, skip, u, proj, rows, d, sms, ps, s);
+      }
     }
   }
   if (e != cudaSuccess) return e;
@@ -467,19 +504,23 @@ cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_
   e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSwdMaxTokensPerSample * (int)sizeof(float));
   if (e != cudaSuccess) return e;
-  e = launch_chained(swd_sort_samples_kernel, 2u * L * B, kSwdSortThreads, smem, s, proj, buf_a, B, T, L, rows, skip);
+  e = launch_chained(swd_sort_samples_kernel, 2u * L * B, kSwdSortThreads, smem, s, proj, sorted, ticket, B, T, L, rows, skip);
   if (e != cudaSuccess) return e;
-  e = launch_chained(swd_sample_w1_kernel, (unsigned)(B * L), 256, 0, s, buf_a, w1_sample, B, T, L, rows, skip);
-  float *cur = buf_a, *nxt = buf_b;
-  for (int run = 1; run < B && e == cudaSuccess; run *= 2) {     // merge the samples' sorted lists
-    const long long total = rows * 2 * L;
-    e = launch_chained(swd_merge_kernel, (unsigned)((total + 255) / 256), 256, 0, s, cur, nxt, rows, T, run, 2 * L, skip);
-    float *t = cur; cur = nxt; nxt = t;
+  // all merge rounds but the last write their output: sorted -> spare -> proj -> spare ...
+  const float *runs = sorted;
+  long long run_len = T;
+  float *dst = spare;
+  while (2 * run_len < rows) {
+    const long long tasks = (rows + kSwdMergeSpan - 1) / kSwdMergeSpan * 2 * L;
+    e = launch_chained(swd_merge_kernel, (unsigned)((tasks + kSwdW1Threads - 1) / kSwdW1Threads), kSwdW1Threads, 0, s, runs, dst,
+                       rows, run_len, 2 * L, skip);
+    if (e != cudaSuccess) return e;
+    runs = dst;
+    dst = dst == spare ? proj : spare;
+    run_len *= 2;
   }
-  if (e != cudaSuccess) return e;
-  e = launch_chained(swd_tensor_w1_kernel, (unsigned)L, kSwdSortThreads, 0, s, cur, w1_tensor, rows, L, skip);
-  if (e != cudaSuccess) return e;
-  return launch_chained(swd_finish_kernel, 1, 128, 0, s, w1_tensor, w1_sample, out, B, L, skip);
+  const unsigned grid = (unsigned)((B > 1 ? L * swd_w1_chunks(rows) : 0) + L * B * swd_w1_chunks(T));
+  return launch_chained(swd_w1_kernel, grid, kSwdW1Threads, 0, s, sorted, runs, run_len, partial, ticket, out, B, T, L, rows, skip);
 }
 
 // A verifier with directions: the distances of this submission against the reference in force,
@@ -520,14 +561,18 @@ int run_reference_projection(sentinel_verifier *h, int kind, cudaStream_t s) {
   const void *m0 = h->ema[kind][0], *m1 = h->ema[kind][1];
   const int *active = &h->hs->kind[kind].active;
   const long long rows = (long long)h->cfg.B * h->cfg.T;
-  cudaError_t e;
-  if (h->bf16) {
-    if (h->sw_L == 4) e = launch_projection<4, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
-    else if (h->sw_L == 8) e = launch_projection<8, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
-    else e = launch_projection<16, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
-  } else if (h->sw_L == 4) e = launch_projection<4, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
-  else if (h->sw_L == 8) e = launch_projection<8, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
-  else e = launch_projection<16, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  bool fits = false;
+  cudaError_t e = launch_projection_ref_mma<false>(nullptr, m0, m1, h->bf16, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d,
+                                                   h->sw_L, sms, ps, s, &fits);
+  if (e == cudaSuccess && !fits) {
+    if (h->bf16) {
+      if (h->sw_L == 4) e = launch_projection<4, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+      else if (h->sw_L == 8) e = launch_projection<8, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+      else e = launch_projection<16, true, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+    } else if (h->sw_L == 4) e = launch_projection<4, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+    else if (h->sw_L == 8) e = launch_projection<8, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+    else e = launch_projection<16, true>(nullptr, m0, m1, active, nullptr, h->sw_u, nullptr, rows, h->cfg.d, sms, ps, s);
+  }
   SENTINEL_CUDA(h, e);
   return SENTINEL_OK;
 }

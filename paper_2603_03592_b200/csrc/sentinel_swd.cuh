@@ -241,6 +241,196 @@ swd_project_mma_kernel(const uint16_t *x, const int *active, const int *skip, co
 }
 
 // ---------------------------------------------------------------------------------------------
+// Both projections on the tensor cores: P(x) as above and P(m) of a stored reference.
+//
+// A bf16 reference is an operand as it stands.  An fp32 one is split, exactly, into three bf16
+// terms: hi = the upper 16 bits of m, mid = the upper 16 bits of m - hi, lo = m - hi - mid (a
+// 24-bit significand in three pieces of 8; both differences are exact in fp32 and lo needs no
+// rounding), so  m . u = hi . u + mid . u + lo . u  with every product exact in fp32 and the three
+// multiplies accumulating into the same fp32 sums.  (A reference value that is not finite makes
+// the differences, hence the projection, not a number.)
+//
+// Work is dealt differently from the x-only kernel: a CTA owns 16 token rows at a time and its
+// twelve warps split the columns of those rows among them, so every task keeps the whole CTA
+// loading (whole-row tasks per warp would leave most warps of an SM without work on the last
+// round); the warps' partial sums meet in shared memory and are added in warp order.
+constexpr int kSwdRefThreads = 384;
+constexpr int kSwdRefWarps = kSwdRefThreads / 32;
+
+template <bool kBf16> struct RefWords;
+template <> struct RefWords<true> { uint4 v; };
+template <> struct RefWords<false> { F8 v; };
+
+template <bool kBf16>
+__device__ __forceinline__ RefWords<kBf16> load_ref8(const void *m, size_t at) {
+  RefWords<kBf16> r;
+  if constexpr (kBf16) r.v = ld_x128(static_cast<const uint16_t *>(m) + at);
+  else r.v = load_m8<false>(m, at);
+  return r;
+}
+
+// the pair (e, o) as two bf16 in one word (e in the low half), each the upper 16 bits of its float
+__device__ __forceinline__ unsigned upper_halves(float e, float o) {
+  return __byte_perm(__float_as_uint(e), __float_as_uint(o), 0x7632);
+}
+__device__ __forceinline__ float upper_part(float v) { return __uint_as_float(__float_as_uint(v) & 0xFFFF0000u); }
+
+// acc += (rows g | g + 8 of the reference, 8 columns) x (direction fragment uv)
+template <bool kBf16>
+__device__ __forceinline__ void mma_ref8(float (&acc)[4], const RefWords<kBf16> &ra, const RefWords<kBf16> &rb, const uint4 &uv) {
+  if constexpr (kBf16) {
+    mma_bf16_16x8x16(acc, ra.v.x, rb.v.x, ra.v.y, rb.v.y, uv.x, uv.y);
+    mma_bf16_16x8x16(acc, ra.v.z, rb.v.z, ra.v.w, rb.v.w, uv.z, uv.w);
+  } else {
+    unsigned a[3][4], b[3][4];                    // [term][pair of columns]
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float e = ra.v.v[2 * j], o = ra.v.v[2 * j + 1];
+      a[0][j] = upper_halves(e, o);
+      e -= upper_part(e); o -= upper_part(o);
+      a[1][j] = upper_halves(e, o);
+      e -= upper_part(e); o -= upper_part(o);
+      a[2][j] = upper_halves(e, o);
+      e = rb.v.v[2 * j]; o = rb.v.v[2 * j + 1];
+      b[0][j] = upper_halves(e, o);
+      e -= upper_part(e); o -= upper_part(o);
+      b[1][j] = upper_halves(e, o);
+      e -= upper_part(e); o -= upper_part(o);
+      b[2][j] = upper_halves(e, o);
+    }
+#pragma unroll
+    for (int t = 2; t >= 0; --t) {                // the small terms first
+      mma_bf16_16x8x16(acc, a[t][0], b[t][0], a[t][1], b[t][1], uv.x, uv.y);
+      mma_bf16_16x8x16(acc, a[t][2], b[t][2], a[t][3], b[t][3], uv.z, uv.w);
+    }
+  }
+}
+
+template <int NB, bool kWithX, bool kBf16>    // NB blocks of 8 directions; kWithX = false: the reference alone
+__global__ void __launch_bounds__(kSwdRefThreads, 1)
+swd_project_ref_mma_kernel(const uint16_t *x, const void *m0, const void *m1, const int *active, const int *skip,
+                           const uint16_t *u, float *proj, long long rows, int d, int L, double *pm0, double *pm1,
+                           float beta, float one_minus_beta) {
+  extern __shared__ uint4 s_u[];                 // [L][stride], 8 bf16 each; then the warps' partial sums
+  chain_entry();
+  if (skip && __ldcg(skip)) return;
+  const bool second = active && __ldcg(active);
+  const void *m = second ? m1 : m0;
+  double *pm_cur = second ? pm1 : pm0, *pm_next = second ? pm0 : pm1;
+  const int chunks = d >> 3, stride = swd_mma_stride(chunks);
+  constexpr int kSets = kWithX ? 2 : 1, kVals = kSets * NB * 4;     // accumulator words of a lane
+  float *s_acc = reinterpret_cast<float *>(s_u + (size_t)L * stride);            // [warp][kVals][32]
+  for (int i = threadIdx.x; i < L * chunks; i += kSwdRefThreads) {
+    const int l = i / chunks, c = i - l * chunks;
+    s_u[l * stride + c] = reinterpret_cast<const uint4 *>(u)[i];
+  }
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
+  const long long n_tasks = (rows + 15) >> 4;
+  const int n_blocks = (chunks + 3) >> 2;        // blocks of 32 columns (4 chunks, one per q)
+  const int blk0 = (int)((long long)n_blocks * warp / kSwdRefWarps), blk1 = (int)((long long)n_blocks * (warp + 1) / kSwdRefWarps);
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+  RefWords<kBf16> zero_ref;
+  if constexpr (kBf16) zero_ref.v = zero4;
+  else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) zero_ref.v.v[j] = 0.f;
+  }
+  for (long long task = blockIdx.x; task < n_tasks; task += gridDim.x) {
+    const long long row_a = task * 16 + g, row_b = row_a + 8;
+    // a row past the end is read as the last row and its result dropped
+    const size_t off_a = (size_t)(row_a < rows ? row_a : rows - 1) * d, off_b = (size_t)(row_b < rows ? row_b : rows - 1) * d;
+    float acc[kSets][NB][4];
+#pragma unroll
+    for (int st = 0; st < kSets; ++st)
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) acc[st][nb][0] = acc[st][nb][1] = acc[st][nb][2] = acc[st][nb][3] = 0.f;
+
+    // two blocks of 32 columns per trip; the loads of the next trip are issued before the multiplies of this one
+    uint4 xc[2][2], xn[2][2];
+    RefWords<kBf16> rc[2][2], rn[2][2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int c = (blk0 + k) * 4 + q;
+      const bool ok = blk0 + k < blk1 && c < chunks;
+      if constexpr (kWithX) {
+        xc[k][0] = ok ? ld_x128(x + off_a + (size_t)c * 8) : zero4;
+        xc[k][1] = ok ? ld_x128(x + off_b + (size_t)c * 8) : zero4;
+      }
+      rc[k][0] = ok ? load_ref8<kBf16>(m, off_a + (size_t)c * 8) : zero_ref;
+      rc[k][1] = ok ? load_ref8<kBf16>(m, off_b + (size_t)c * 8) : zero_ref;
+    }
+    for (int blk = blk0; blk < blk1; blk += 2) {
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int c = (blk + 2 + k) * 4 + q;
+        const bool ok = blk + 2 + k < blk1 && c < chunks;
+        if constexpr (kWithX) {
+          xn[k][0] = ok ? ld_x128(x + off_a + (size_t)c * 8) : zero4;
+          xn[k][1] = ok ? ld_x128(x + off_b + (size_t)c * 8) : zero4;
+        }
+        rn[k][0] = ok ? load_ref8<kBf16>(m, off_a + (size_t)c * 8) : zero_ref;
+        rn[k][1] = ok ? load_ref8<kBf16>(m, off_b + (size_t)c * 8) : zero_ref;
+      }
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int c = (blk + k) * 4 + q;
+        const bool ok = blk + k < blk1 && c < chunks;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          const int l = nb * 8 + g;
+          const uint4 uv = (l < L && ok) ? s_u[l * stride + c] : zero4;
+          if constexpr (kWithX) {
+            mma_bf16_16x8x16(acc[0][nb], xc[k][0].x, xc[k][1].x, xc[k][0].y, xc[k][1].y, uv.x, uv.y);
+            mma_bf16_16x8x16(acc[0][nb], xc[k][0].z, xc[k][1].z, xc[k][0].w, xc[k][1].w, uv.z, uv.w);
+          }
+          mma_ref8<kBf16>(acc[kSets - 1][nb], rc[k][0], rc[k][1], uv);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        if constexpr (kWithX) { xc[k][0] = xn[k][0]; xc[k][1] = xn[k][1]; }
+        rc[k][0] = rn[k][0]; rc[k][1] = rn[k][1];
+      }
+    }
+    // the warps' sums meet in shared memory; the first warps add them in warp order and write
+    __syncthreads();                              // (the previous task's sums have been read)
+#pragma unroll
+    for (int st = 0; st < kSets; ++st)
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s_acc[(warp * kVals + (st * NB + nb) * 4 + e) * 32 + lane] = acc[st][nb][e];
+    __syncthreads();
+    // accumulator layout: [0], [1] = (row g, directions 2q, 2q+1), [2], [3] = (row g + 8, same)
+    for (int item = threadIdx.x; item < NB * 4 * 32; item += kSwdRefThreads) {
+      const int ln = item & 31, e = (item >> 5) & 3, nb = item >> 7;
+      const int gg = ln >> 2, qq = ln & 3;
+      const long long row = task * 16 + gg + ((e < 2) ? 0 : 8);
+      const int l = nb * 8 + 2 * qq + (e & 1);
+      if (row >= rows || l >= L) continue;
+      float sx = 0.f, sm = 0.f;
+      for (int w = 0; w < kSwdRefWarps; ++w) {
+        if constexpr (kWithX) sx += s_acc[(w * kVals + nb * 4 + e) * 32 + ln];
+        sm += s_acc[(w * kVals + ((kSets - 1) * NB + nb) * 4 + e) * 32 + ln];
+      }
+      const size_t at = (size_t)row * L + l;
+      if constexpr (!kWithX) {
+        pm_cur[at] = (double)sm;
+      } else {
+        proj[(size_t)l * rows + row] = sx;
+        proj[((size_t)L + l) * rows + row] = sm;
+        if (pm_cur) {
+          pm_cur[at] = (double)sm;
+          pm_next[at] = (double)beta * (double)sm + (double)one_minus_beta * (double)sx;
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // helpers of the sort / W1 kernels
 __device__ __forceinline__ double block_sum_ordered(double v, double *s_red) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -298,12 +488,14 @@ __device__ __forceinline__ void bitonic_round(float *s_val, int npad, int k2, in
 
 // one CTA per (sample, direction, cloud): bitonic sort of that list of T projections in shared
 // memory (padded with +inf to a power of two, at least 8); the sorted list goes back to global
-// memory
+// memory.  Also clears the ticket word of swd_w1_kernel, a later launch of the chain.
 __global__ void __launch_bounds__(kSwdSortThreads)
-swd_sort_samples_kernel(const float *proj, float *sorted, int B, int T, int L, long long rows, const int *skip) {
+swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int B, int T, int L, long long rows,
+                        const int *skip) {
   extern __shared__ float s_val[];                // [npad]
   chain_entry();
   if (skip && __ldcg(skip)) return;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *ticket = 0u;
   const int list = blockIdx.x / B, b = blockIdx.x - list * B;     // list = cloud * L + direction
   int npad = 8;
   while (npad < T) npad <<= 1;
@@ -344,76 +536,188 @@ swd_sort_samples_kernel(const float *proj, float *sorted, int B, int T, int L, l
   for (int i = threadIdx.x; i < T; i += kSwdSortThreads) dst[i] = s_val[i];
 }
 
-// per sample and direction: W1 = mean |a_(i) - b_(i)| of the two sorted lists
-__global__ void __launch_bounds__(256)
-swd_sample_w1_kernel(const float *sorted, float *w1_sample, int B, int T, int L, long long rows, const int *skip) {
-  __shared__ double s_red[256 / 32];
-  chain_entry();
-  if (skip && __ldcg(skip)) return;
-  const int b = blockIdx.x / L, l = blockIdx.x - b * L;
-  const float *sa = sorted + (size_t)l * rows + (size_t)b * T;
-  const float *sb = sorted + ((size_t)L + l) * rows + (size_t)b * T;
-  double acc = 0.;
-  for (int i = threadIdx.x; i < T; i += 256) acc += (double)fabsf(sa[i] - sb[i]);
-  const double total = block_sum_ordered(acc, s_red);
-  if (threadIdx.x == 0) w1_sample[b * L + l] = (float)(total / (double)T);
-}
-
 // ---------------------------------------------------------------------------------------------
-// one round of merging: in every list (2L of them, each B sorted runs of T) neighbouring pairs
-// of runs of `run` samples become one sorted run; an element's place is its index in its own
-// run plus its rank in the partner run (left run first on ties)
-__global__ void swd_merge_kernel(const float *in, float *out, long long rows, int T, int run, int lists,
-                                 const int *skip) {
-  chain_entry();
-  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= rows * lists || (skip && __ldcg(skip))) return;
-  const long long list = e / rows, i = e - list * rows;
-  const float *src = in + list * rows;
-  const long long run_len = (long long)run * T;
-  const long long r = i / run_len, pair_start = (r & ~1ll) * run_len;
-  const long long own_start = r * run_len;
-  const long long other_start = (r & 1) ? own_start - run_len : own_start + run_len;
-  const float v = src[i];
-  long long pos = i - own_start;
-  if (other_start < rows) {
-    long long lo = 0, hi = run_len;
-    if (other_start + hi > rows) hi = rows - other_start;
-    const float *other = src + other_start;
-    if (r & 1) {                                  // right run: after the left entries <= v
-      while (lo < hi) { const long long mid = (lo + hi) >> 1; if (other[mid] <= v) lo = mid + 1; else hi = mid; }
-    } else {                                      // left run: after the right entries < v
-      while (lo < hi) { const long long mid = (lo + hi) >> 1; if (other[mid] < v) lo = mid + 1; else hi = mid; }
-    }
-    pos += lo;
+// From the sorted sample lists to W1 of every unit.
+//
+// A sample: its two lists have T entries each, so W1 = mean_i |a_(i) - b_(i)|.
+// The whole tensor: the B sorted runs of a list are merged pairwise, ceil(log2 B) rounds, into one
+// sorted list of B*T entries per cloud and direction, and W1 = mean_i |A_(i) - B_(i)| again.
+//
+// A merge is split the way a merge path is: a thread produces kSwdMergeSpan consecutive entries of
+// the output.  One bisection tells it how many entries of the left run come before its first
+// output (ties: left run first); its outputs are then among the next kSwdMergeSpan entries of
+// either run, which it loads in one go and merges in registers (the smaller halves of a bitonic
+// merge network).  Linear work, and one chain of dependent loads per thread instead of one per entry.
+//
+// The last round does not write its output: a thread merges the same span of the x cloud and of
+// the reference cloud and adds up |A_(i) - B_(i)| at once (swd_w1_kernel).  The same launch has
+// CTAs for the samples' W1, and the CTA that draws the last ticket adds the per-CTA sums in a
+// fixed order and writes the means over the directions: out[0] = the whole tensor, out[1+b] =
+// sample b.  The ticket word must be zero at launch (the sort kernel clears it).
+constexpr int kSwdMergeSpan = 8;
+constexpr int kSwdW1Threads = 256;
+constexpr int kSwdW1Span = kSwdW1Threads * kSwdMergeSpan;         // entries a CTA covers
+
+// how many entries of the left run come before merged position d (0 <= d <= la + lb)
+__device__ __forceinline__ int merge_split(const float *left, int la, const float *right, int lb, int d) {
+  int lo = d > lb ? d - lb : 0, hi = d < la ? d : la;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (left[mid] <= right[d - 1 - mid]) lo = mid + 1; else hi = mid;
   }
-  out[list * rows + pair_start + pos] = v;
+  return lo;
 }
 
-// whole-tensor unit: W1 per direction from the fully merged lists, one CTA per direction
-__global__ void __launch_bounds__(kSwdSortThreads)
-swd_tensor_w1_kernel(const float *merged, float *w1_tensor, long long rows, int L, const int *skip) {
-  __shared__ double s_red[kSwdSortThreads / 32];
-  chain_entry();
-  if (skip && __ldcg(skip)) return;
-  const int l = blockIdx.x;
-  const float *a = merged + (size_t)l * rows, *b = merged + ((size_t)L + l) * rows;
-  double acc = 0.;
-  for (long long i = threadIdx.x; i < rows; i += kSwdSortThreads) acc += (double)fabsf(a[i] - b[i]);
-  const double total = block_sum_ordered(acc, s_red);
-  if (threadIdx.x == 0) w1_tensor[l] = (float)(total / (double)rows);
+// merged entries d .. d + 7 of (left, right); +inf past the end
+__device__ __forceinline__ void merge_span(const float *left, int la, const float *right, int lb, int d, float (&out)[kSwdMergeSpan]) {
+  const int a = merge_split(left, la, right, lb, d), b = d - a;
+  float ca[kSwdMergeSpan], cb[kSwdMergeSpan];
+#pragma unroll
+  for (int k = 0; k < kSwdMergeSpan; ++k) {
+    ca[k] = a + k < la ? left[a + k] : CUDART_INF_F;
+    cb[k] = b + k < lb ? right[b + k] : CUDART_INF_F;
+  }
+  // the 8 smallest of two ascending runs of 8: min(ca[k], cb[7-k]) is a bitonic sequence of them
+#pragma unroll
+  for (int k = 0; k < kSwdMergeSpan; ++k) out[k] = fminf(ca[k], cb[kSwdMergeSpan - 1 - k]);
+#pragma unroll
+  for (int dist = kSwdMergeSpan / 2; dist > 0; dist >>= 1) {
+#pragma unroll
+    for (int k = 0; k < kSwdMergeSpan; ++k) {
+      if (!(k & dist)) {
+        const float lo = fminf(out[k], out[k | dist]), hi = fmaxf(out[k], out[k | dist]);
+        out[k] = lo; out[k | dist] = hi;
+      }
+    }
+  }
 }
 
-// the means over the directions for every unit: out[0] = tensor, out[1+b] = sample b
-__global__ void swd_finish_kernel(const float *w1_tensor, const float *w1_sample, float *out, int B, int L,
-                                  const int *skip) {
+// the two runs that meet at merged position `at` of a list whose runs of `run_len` entries are
+// merged pairwise: returns the position inside the pair
+__device__ __forceinline__ int merge_pair(const float *list, long long rows, long long run_len, long long at,
+                                          const float *&left, int &la, const float *&right, int &lb) {
+  const long long start = at / (2 * run_len) * (2 * run_len);
+  const long long left_len = rows - start < run_len ? rows - start : run_len;
+  const long long right_len = rows - start - left_len < run_len ? rows - start - left_len : run_len;
+  left = list + start; la = (int)left_len;
+  right = left + left_len; lb = (int)right_len;
+  return (int)(at - start);
+}
+
+// one round that is not the last: runs of run_len entries become runs of twice that
+__global__ void __launch_bounds__(kSwdW1Threads)
+swd_merge_kernel(const float *in, float *out, long long rows, long long run_len, int lists, const int *skip) {
   chain_entry();
   if (skip && __ldcg(skip)) return;
-  for (int r = threadIdx.x; r <= B; r += blockDim.x) {
-    const float *w = r ? w1_sample + (size_t)(r - 1) * L : w1_tensor;
-    double s = 0.;
-    for (int l = 0; l < L; ++l) s += (double)w[l];
-    out[r] = (float)(s / L);
+  const long long spans = (rows + kSwdMergeSpan - 1) / kSwdMergeSpan;
+  const long long task = (long long)blockIdx.x * kSwdW1Threads + threadIdx.x;
+  if (task >= spans * lists) return;
+  const long long list = task / spans, at = (task - list * spans) * kSwdMergeSpan;
+  const float *left, *right;
+  int la, lb;
+  // (a span may straddle two pairs only if 2 * run_len is not a multiple of the span: run_len is a multiple of T, any T,
+  // so the entries past the end of this pair are produced one by one below)
+  const int d = merge_pair(in + list * rows, rows, run_len, at, left, la, right, lb);
+  float v[kSwdMergeSpan];
+  merge_span(left, la, right, lb, d, v);
+  float *dst = out + list * rows + at;
+  const int n_here = la + lb - d < kSwdMergeSpan ? la + lb - d : kSwdMergeSpan;
+#pragma unroll
+  for (int k = 0; k < kSwdMergeSpan; ++k)
+    if (k < n_here) dst[k] = v[k];
+  if (n_here < kSwdMergeSpan) {                   // the rest of the span lies in the next pair (or past the end)
+    for (int k = n_here; k < kSwdMergeSpan && at + k < rows; ++k) {
+      const float *l2, *r2;
+      int la2, lb2;
+      const int d2 = merge_pair(in + list * rows, rows, run_len, at + k, l2, la2, r2, lb2);
+      float w[kSwdMergeSpan];
+      merge_span(l2, la2, r2, lb2, d2, w);
+      dst[k] = w[0];
+    }
+  }
+}
+
+__host__ __device__ inline int swd_w1_chunks(long long n) { return (int)((n + kSwdW1Span - 1) / kSwdW1Span); }
+// doubles of `partial`: per direction the whole-tensor CTAs' sums, then per (direction, sample) the sample CTAs'
+__host__ __device__ inline size_t swd_w1_partials(int L, int B, int T) {
+  return (size_t)L * swd_w1_chunks((long long)B * T) + (size_t)L * B * swd_w1_chunks(T);
+}
+
+// `sorted`: the samples' sorted lists, [2L][B][T]; `runs`: the lists after all merge rounds but the last
+// (runs of run_len entries; == sorted if there was no earlier round; unused if B == 1)
+__global__ void __launch_bounds__(kSwdW1Threads)
+swd_w1_kernel(const float *sorted, const float *runs, long long run_len, double *partial, unsigned *ticket, float *out, int B,
+              int T, int L, long long rows, const int *skip) {
+  __shared__ double s_red[kSwdW1Threads / 32];
+  __shared__ float s_w1[(kMaxB + 1) * 16];        // W1 per (unit, direction), L <= 16
+  __shared__ bool s_last;
+  chain_entry();
+  if (skip && __ldcg(skip)) return;
+  const int tensor_chunks = B > 1 ? swd_w1_chunks(rows) : 0, sample_chunks = swd_w1_chunks(T);
+  const int n_tensor = L * tensor_chunks;
+  double term = 0.;
+  if ((int)blockIdx.x < n_tensor) {               // a span of the last merge round, both clouds
+    const int l = blockIdx.x / tensor_chunks, chunk = blockIdx.x - l * tensor_chunks;
+    const long long at = ((long long)chunk * kSwdW1Threads + threadIdx.x) * kSwdMergeSpan;
+    if (at < rows) {
+      float va[kSwdMergeSpan], vb[kSwdMergeSpan];
+      const float *left, *right;
+      int la, lb;
+      int d = merge_pair(runs + (size_t)l * rows, rows, run_len, at, left, la, right, lb);
+      merge_span(left, la, right, lb, d, va);
+      d = merge_pair(runs + ((size_t)L + l) * rows, rows, run_len, at, left, la, right, lb);
+      merge_span(left, la, right, lb, d, vb);
+#pragma unroll
+      for (int k = 0; k < kSwdMergeSpan; ++k)
+        if (at + k < rows) term += (double)fabsf(va[k] - vb[k]);
+    }
+  } else {                                        // a span of one sample's two lists
+    const int unit = (blockIdx.x - n_tensor) / sample_chunks, chunk = (blockIdx.x - n_tensor) - unit * sample_chunks;
+    const int l = unit / B, b = unit - l * B;
+    const float *sa = sorted + (size_t)l * rows + (size_t)b * T, *sb = sorted + ((size_t)L + l) * rows + (size_t)b * T;
+    const int at = (chunk * kSwdW1Threads + threadIdx.x) * kSwdMergeSpan;
+#pragma unroll
+    for (int k = 0; k < kSwdMergeSpan; ++k)
+      if (at + k < T) term += (double)fabsf(sa[at + k] - sb[at + k]);
+  }
+  const double sum = block_sum_ordered(term, s_red);
+  if (threadIdx.x == 0) {
+    partial[blockIdx.x] = sum;
+    __threadfence();
+    s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // unit r = 0: the whole tensor, r = 1 + b: sample b.  One warp per (unit, direction): lane j adds
+  // the CTA sums j, j + 32, ... in that order, the lanes are combined by the shuffle tree
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int pair = warp; pair < (B + 1) * L; pair += kSwdW1Threads / 32) {
+    const int r = pair / L, dir = pair - r * L;
+    double w1 = 0., n = (double)T;
+    if (r == 0 && B > 1) {
+      for (int k = lane; k < tensor_chunks; k += 32) w1 += __ldcg(partial + (size_t)dir * tensor_chunks + k);
+      n = (double)rows;
+    } else {
+      const int bb = r == 0 ? 0 : r - 1;
+      for (int k = lane; k < sample_chunks; k += 32) w1 += __ldcg(partial + n_tensor + ((size_t)dir * B + bb) * sample_chunks + k);
+    }
+    w1 = warp_sum(w1);
+    if (lane == 0) s_w1[pair] = (float)(w1 / n);
+  }
+  __syncthreads();
+  // a sample with an entry that is not finite has a W1 that is not finite; the merges above may have
+  // dropped such an entry (min / max of a number and a NaN is the number), so the whole tensor's
+  // W1 is declared not a number along with it
+  for (int r = threadIdx.x; r <= B; r += kSwdW1Threads) {
+    double mean = 0.;
+    for (int dir = 0; dir < L; ++dir) mean += (double)s_w1[r * L + dir];
+    if (r == 0) {
+      bool finite = true;
+      for (int k = L; k < (B + 1) * L; ++k) finite = finite && fabsf(s_w1[k]) < CUDART_INF_F;
+      if (!finite) mean = (double)CUDART_NAN_F;
+    }
+    out[r] = (float)(mean / L);
   }
 }
 

@@ -34,6 +34,7 @@ def run_steps(sb, oracle_mod, w, kind, n_warm, corruption, **variant):
         assert_stats_close(st, ov.last_stats(kind), float(x.float().std()),
                            max(float(np.abs(ov.last_stats(kind)[0, 4])) ** 0.5, 1e-30), "%s stats %d" % (w.name, t))
     # a clean verified step, then a corrupted one
+    near_events = 0
     for t, name in ((n_warm, None), (n_warm + 1, corruption)):
         x = synth.clean(w, 0, kind, t, "cuda")
         if name:
@@ -46,7 +47,9 @@ def run_steps(sb, oracle_mod, w, kind, n_warm, corruption, **variant):
         if not np.array_equal(gf, of):
             near = near_threshold(os_, thr, valid, w.B)
             assert np.all(near[((gf ^ of) & UNIT_BITS) != 0]), (gf, of)
+            near_events += 1
         assert bool(gf[0] & sb.FLAG_COMMITTED) == commit
+    assert near_events <= 1, near_events
     c = gv.sentinel_get_counters()
     assert (c["violations"], c["clean_streak"], c["banned"]) == ov.counters()
     gv.close()
@@ -101,6 +104,7 @@ def test_cfg3_two_workers_against_the_oracle(sb, oracle_mod):
     R = 2
     gv = sb.Verifier(w.B, w.T, w.d, n_workers=R)
     ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, R=R))
+    near_events = 0
     for t in range(4):
         xs = [synth.clean(w, r, GRAD, t, "cuda") for r in range(R)]
         if t == 3:
@@ -116,8 +120,10 @@ def test_cfg3_two_workers_against_the_oracle(sb, oracle_mod):
             for r in range(R):
                 near = near_threshold(os_[r], thr, valid, w.B)
                 assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            near_events += 1
         if t == 3:
             assert of[1, 0] & UNIT_BITS and not (of[0, 0] & UNIT_BITS) and n_clean == 1
+    assert near_events == 0, near_events                    # (the counters below would differ otherwise)
     for r in range(R):
         assert gv.sentinel_get_worker_counters(r) == ov.worker_counters(r)
     blob = gv.sentinel_export_state()

@@ -77,7 +77,7 @@ def test_iterations_in_lockstep(sb, oracle_mod, shape, R):
     gv, ov, params = pair(sb, oracle_mod, w, R, l=5, c=2)
     script = [("warm", {})] * 8 + [("verify", {})] * 3 + [("verify", {1: 6.0})] + [("verify", {})] + \
              [("verify", {r: 3.0 for r in range(R // 2 + 1)})] + [("verify", {1: 6.0})] + [("verify", {})] * 2
-    k_events = 0
+    k_events, near_events = 0, 0
     for kind in (ACT, GRAD):
         for t, (what, scale) in enumerate(script):
             xs = inputs(w, R, kind, t, scale)
@@ -93,6 +93,7 @@ def test_iterations_in_lockstep(sb, oracle_mod, shape, R):
                 for r in range(R):
                     near = near_threshold(os_[r], thr, valid, w.B)
                     assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+                near_events += 1
                 gv.sentinel_import_state(oracle_to_blob(ov, params))
             if scale and len(scale) > 1:
                 assert np.all(of[:, 0] & sb.FLAG_NATURAL_SHIFT)
@@ -102,7 +103,8 @@ def test_iterations_in_lockstep(sb, oracle_mod, shape, R):
                 gv.sentinel_import_state(oracle_to_blob(ov, params))
         check_state(gv, ov, params, kinds=(kind,))
     assert ov.worker_counters(1)[2] == 1                    # worker 1 ended up banned
-    assert k_events <= 4, k_events
+    print("re-alignments: %d near a bound, %d multiplier events" % (near_events, k_events))
+    assert near_events <= 2 and k_events <= 4, (near_events, k_events)
     gv.close()
 
 
@@ -168,6 +170,7 @@ def test_workers_tainted_elsewhere(sb, oracle_mod, kind):
         step_both(gv, ov, inputs(w, R, kind, t), kind, warmup=True)
     plan = [(0b0000, {}), (0b0010, {}), (0b1100, {0: 6.0}), (0b0001, {}), (0b0000, {3: 6.0}), (0b0000, {3: 6.0}),
             (0b1000, {}), (0b1111, {}), (0b0000, {})]
+    near_events, k_events = 0, 0
     for t, (mask, scale) in enumerate(plan, start=10):
         xs = inputs(w, R, kind, t, scale)
         thr, valid = ov.thresholds(kind)
@@ -178,9 +181,11 @@ def test_workers_tainted_elsewhere(sb, oracle_mod, kind):
             for r in range(R):
                 near = near_threshold(os_[r], thr, valid, w.B)
                 assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            near_events += 1
             gv.sentinel_import_state(oracle_to_blob(ov, params))
         ev = whole_step_k_events(*gv.sentinel_get_thresholds(kind), *ov.thresholds(kind), params, kind)
         if ev:
+            k_events += ev
             gv.sentinel_import_state(oracle_to_blob(ov, params))
         # the verdict Alg. 4 acts on
         probe = xs[0].clone()
@@ -190,6 +195,8 @@ def test_workers_tainted_elsewhere(sb, oracle_mod, kind):
         assert bool(replaced.item()) == ov.replace_if_flagged(synth.bits(xs[0]), kind)[1], (t, mask)
         check_state(gv, ov, params, kinds=(kind,))
     assert ov.worker_counters(3)[2] == 1                    # banned on the way; its bit then changes nothing
+    print("re-alignments: %d near a bound, %d multiplier events" % (near_events, k_events))
+    assert near_events <= 2 and k_events <= 4, (near_events, k_events)
     gv.close()
 
 
@@ -254,6 +261,7 @@ def test_iterations_in_lockstep_with_a_bf16_reference(sb, oracle_mod, shape, R):
     gv, ov, params = pair(sb, oracle_mod, w, R, l=5, c=3, ema_bf16=1)
     script = [("warm", {})] * 6 + [("verify", {})] * 2 + [("verify", {1: 6.0})] + [("verify", {})] + \
              [("verify", {r: 3.0 for r in range(R // 2 + 1)})] + [("verify", {})]
+    near_events, k_events = 0, 0
     for t, (what, scale) in enumerate(script):
         xs = inputs(w, R, ACT, t, scale)
         thr, valid = ov.thresholds(ACT)
@@ -264,9 +272,14 @@ def test_iterations_in_lockstep_with_a_bf16_reference(sb, oracle_mod, shape, R):
             for r in range(R):
                 near = near_threshold(os_[r], thr, valid, w.B)
                 assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            near_events += 1
             gv.sentinel_import_state(oracle_to_blob(ov, params))
-        if whole_step_k_events(*gv.sentinel_get_thresholds(ACT), *ov.thresholds(ACT), params, ACT):
+        ev = whole_step_k_events(*gv.sentinel_get_thresholds(ACT), *ov.thresholds(ACT), params, ACT)
+        if ev:
+            k_events += ev
             gv.sentinel_import_state(oracle_to_blob(ov, params))
         st = parse_blob(gv.sentinel_export_state(), w.B, w.T, w.d, params.l, R)
         assert np.array_equal(st["kinds"][ACT]["m"].astype(np.float64), ov.ema(ACT)), t
+    print("re-alignments: %d near a bound, %d multiplier events" % (near_events, k_events))
+    assert near_events <= 2 and k_events <= 4, (near_events, k_events)
     gv.close()

@@ -218,6 +218,7 @@ def test_worker_iterations_with_four_metrics(sb, oracle_mod):
     with_directions(gv, ov, 8, w.d)
     script = [("warm", {})] * 8 + [("verify", {})] * 2 + [("verify", {1: 6.0})] + [("verify", {})] + \
              [("verify", {1: 6.0})] + [("verify", {})] * 2
+    near_events, k_events = 0, 0
     for t, (what, scale) in enumerate(script):
         xs = rep.inputs(w, R, ACT, t, scale)
         thr, valid = ov.thresholds(ACT)
@@ -229,10 +230,14 @@ def test_worker_iterations_with_four_metrics(sb, oracle_mod):
             for r in range(R):
                 near = near_threshold(os_[r], thr, valid, w.B)
                 assert np.all(near[((gf[r] ^ of[r]) & UNIT_BITS) != 0]), (t, r, gf[r], of[r])
+            near_events += 1
             gv.sentinel_import_state(oracle_to_blob(ov, params))
         ev = rep.whole_step_k_events(*gv.sentinel_get_thresholds(ACT), *ov.thresholds(ACT), params, ACT)
         if ev:
+            k_events += ev
             gv.sentinel_import_state(oracle_to_blob(ov, params))
+    print("re-alignments: %d near a bound, %d multiplier events" % (near_events, k_events))
+    assert near_events <= 2 and k_events <= 4, (near_events, k_events)
     assert ov.worker_counters(1)[2] == 1                    # banned, then skipped
     rep.check_state(gv, ov, params, kinds=(ACT,))
     gv.close()
