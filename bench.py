@@ -36,10 +36,10 @@ BYTES_PER_ELEMENT = 10          # 2 (x, bf16 read) + 4 (m read) + 4 (EMA candida
 MAX_DISTINCT = 24               # distinct input tensors per kind kept resident
 FOUR_METRIC_BYTES = 12          # a verified tensor with the sliced Wasserstein distance: x twice, the reference read and written
 # dram__bytes_read.sum + dram__bytes_write.sum per element of the current stream_kernel, from the
-# ncu capture summarised in profiles/stream_kernel_cfg3_ncu_full.md (B=8 x 4096 x 4096; traffic
+# ncu capture summarised in profiles/all_kernels_cfg3_ncu.md (B=8 x 4096 x 4096; traffic
 # grows in proportion to the element count, so a launch of N elements moves this times N).
 # Set to None whenever the kernel changes until the capture is retaken.
-NCU_DRAM_BYTES_PER_ELEMENT = 9.679
+NCU_DRAM_BYTES_PER_ELEMENT = 9.677
 
 
 def measured_peak_gbs():

@@ -498,29 +498,41 @@ cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_
     }
   }
   if (e != cudaSuccess) return e;
+  // few lists: each sample's list is sorted as two halves on twice as many SMs, and a merge round follows
+  const int pieces = (T % 2 == 0 && T >= 1024 && 2 * L * B * 2 <= sms) ? 2 : 1;
   int npad = 8;
-  while (npad < T) npad <<= 1;
+  while (npad < T / pieces) npad <<= 1;
   const size_t smem = (size_t)npad * sizeof(float);
   e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSwdMaxTokensPerSample * (int)sizeof(float));
   if (e != cudaSuccess) return e;
-  e = launch_chained(swd_sort_samples_kernel, 2u * L * B, kSwdSortThreads, smem, s, proj, sorted, ticket, B, T, L, rows, skip);
+  e = launch_chained(swd_sort_samples_kernel, 2u * L * B * pieces, kSwdSortThreads, smem, s, proj, sorted, ticket, B, T, pieces, L,
+                     rows, skip);
   if (e != cudaSuccess) return e;
-  // all merge rounds but the last write their output: sorted -> spare -> proj -> spare ...
-  const float *runs = sorted;
-  long long run_len = T;
-  float *dst = spare;
-  while (2 * run_len < rows) {
-    const long long tasks = (rows + kSwdMergeSpan - 1) / kSwdMergeSpan * 2 * L;
-    e = launch_chained(swd_merge_kernel, (unsigned)((tasks + kSwdW1Threads - 1) / kSwdW1Threads), kSwdW1Threads, 0, s, runs, dst,
-                       rows, run_len, 2 * L, skip);
+  const long long span_tasks = (rows + kSwdMergeSpan - 1) / kSwdMergeSpan * 2 * L;
+  const unsigned merge_grid = (unsigned)((span_tasks + kSwdW1Threads - 1) / kSwdW1Threads);
+  // the three buffers: `samples` holds the samples' sorted lists until swd_w1_kernel has read them,
+  // the merge rounds (all but the last, which swd_w1_kernel does itself) alternate between the other two
+  const float *samples = sorted;
+  float *free_a = spare, *free_b = proj;
+  if (pieces == 2) {
+    e = launch_chained(swd_merge_kernel, merge_grid, kSwdW1Threads, 0, s, sorted, spare, rows, (long long)(T / 2), 2 * L, skip);
     if (e != cudaSuccess) return e;
-    runs = dst;
-    dst = dst == spare ? proj : spare;
+    samples = spare;
+    free_a = proj;
+    free_b = sorted;
+  }
+  const float *runs = samples;
+  long long run_len = T;
+  while (2 * run_len < rows) {
+    e = launch_chained(swd_merge_kernel, merge_grid, kSwdW1Threads, 0, s, runs, free_a, rows, run_len, 2 * L, skip);
+    if (e != cudaSuccess) return e;
+    runs = free_a;
+    float *t = free_a; free_a = free_b; free_b = t;
     run_len *= 2;
   }
   const unsigned grid = (unsigned)((B > 1 ? L * swd_w1_chunks(rows) : 0) + L * B * swd_w1_chunks(T));
-  return launch_chained(swd_w1_kernel, grid, kSwdW1Threads, 0, s, sorted, runs, run_len, partial, ticket, out, B, T, L, rows, skip);
+  return launch_chained(swd_w1_kernel, grid, kSwdW1Threads, 0, s, samples, runs, run_len, partial, ticket, out, B, T, L, rows, skip);
 }
 
 // A verifier with directions: the distances of this submission against the reference in force,

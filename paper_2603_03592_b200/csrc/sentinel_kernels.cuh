@@ -1792,9 +1792,9 @@ channel_mean_kernel(HandleState *hs, int kind, float *ema0, float *ema1, const f
     } else {
       for (int i = cs_lo * phases + group; i < cs_hi * phases; i += kChannelMeanGroups) {
         const int cs = i / phases, p = i - cs * phases;
-        // a CTA's first segment lies in the sample of its first row, its second (if any: else blocks
-        // of zeros) in the next one
-        if ((int)(((R * (cs >> 1)) / G) / T) + (cs & 1) != sample) continue;
+        // a CTA's first segment lies in the sample of its first row, floor(floor(B*T*cta/G) / T) =
+        // floor(B*cta/G), its second (if any: else blocks of zeros) in the next one
+        if ((B * (cs >> 1)) / G + (cs & 1) != sample) continue;
         sum += (double)__ldcg(src + ((size_t)cs * n_slots + (size_t)p * stripes) * kStripe);
       }
     }

@@ -486,20 +486,25 @@ __device__ __forceinline__ void bitonic_round(float *s_val, int npad, int k2, in
   __syncthreads();
 }
 
-// one CTA per (sample, direction, cloud): bitonic sort of that list of T projections in shared
+// one CTA per (sample, direction, cloud) and piece: bitonic sort of a list of projections in shared
 // memory (padded with +inf to a power of two, at least 8); the sorted list goes back to global
-// memory.  Also clears the ticket word of swd_w1_kernel, a later launch of the chain.
+// memory.  pieces = 1: the sample's T projections; pieces = 2 (T even): each half of them on a CTA of
+// its own -- twice the SMs at work where the lists are few -- and a merge round puts the halves
+// together.  Also clears the ticket word of swd_w1_kernel, a later launch of the chain.
 __global__ void __launch_bounds__(kSwdSortThreads)
-swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int B, int T, int L, long long rows,
-                        const int *skip) {
+swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int B, int T_sample, int pieces, int L,
+                        long long rows, const int *skip) {
   extern __shared__ float s_val[];                // [npad]
   chain_entry();
   if (skip && __ldcg(skip)) return;
   if (blockIdx.x == 0 && threadIdx.x == 0) *ticket = 0u;
-  const int list = blockIdx.x / B, b = blockIdx.x - list * B;     // list = cloud * L + direction
+  const int T = T_sample / pieces;                // entries this CTA sorts
+  const int run = blockIdx.x / pieces, piece = blockIdx.x - run * pieces;
+  const int list = run / B, b = run - list * B;   // list = cloud * L + direction
   int npad = 8;
   while (npad < T) npad <<= 1;
-  const float *src = proj + (size_t)list * rows + (size_t)b * T;
+  const size_t first = (size_t)list * rows + (size_t)b * T_sample + (size_t)piece * T;
+  const float *src = proj + first;
   for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) s_val[i] = i < T ? src[i] : CUDART_INF_F;
   __syncthreads();
   // runs of 2, 4 and 8: all inside a thread's 8 consecutive entries, the direction per pair
@@ -532,7 +537,7 @@ swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int 
     if (head) { bitonic_round(s_val, npad, k2, j - 2, head); j -= head; }
     for (; j >= 2; j -= 3) bitonic_round(s_val, npad, k2, j - 2, 3);
   }
-  float *dst = sorted + (size_t)list * rows + (size_t)b * T;
+  float *dst = sorted + first;
   for (int i = threadIdx.x; i < T; i += kSwdSortThreads) dst[i] = s_val[i];
 }
 

@@ -43,7 +43,9 @@ def run(sb, x, m, u):
 
 
 CASES = [((1, 1, 8), 4), ((2, 3, 16), 4), ((3, 37, 520), 8), ((5, 100, 1024), 16), ((4, 128, 2048), 8),
-         ((8, 64, 512), 4), ((7, 33, 264), 16), ((1, 700, 136), 8)]
+         ((8, 64, 512), 4), ((7, 33, 264), 16), ((1, 700, 136), 8),
+         # long lists that are few: each sample's list is sorted as two halves (T even, at least 1024) and merged
+         ((2, 1536, 264), 8), ((1, 2048, 136), 8), ((3, 1024, 72), 4), ((5, 1030, 40), 4), ((2, 1025, 64), 4)]
 
 
 @pytest.mark.parametrize("shape,L", CASES, ids=["%dx%dx%d_L%d" % (*s, l) for s, l in CASES])
@@ -59,6 +61,20 @@ def test_matches_oracle_over_shapes(sb, oracle_mod, shape, L):
     want = oracle_all_units(oracle_mod, x, m, u)
     scale = float(x.float().std())
     assert np.all(np.abs(got - want) <= REL * np.maximum(np.abs(want), 1e-3 * scale)), (got, want)
+
+
+def test_an_entry_that_is_not_finite_spoils_its_sample_and_the_whole_tensor(sb):
+    B, T, d, L = 3, 1200, 64, 8
+    g = torch.Generator(device="cuda").manual_seed(21)
+    x = torch.randn(B, T, d, generator=g, device="cuda").to(torch.bfloat16)
+    m = torch.randn(B, T, d, generator=g, device="cuda")
+    u = directions(L, d, 2)
+    for bad in (float("inf"), float("nan")):
+        y = x.clone()
+        y[1, 700, 5] = bad
+        got = run(sb, y, m, u)
+        assert np.isfinite(got[1]) and np.isfinite(got[3]), got
+        assert not np.isfinite(got[0]) and not np.isfinite(got[2]), got
 
 
 def test_closed_forms_on_gpu(sb):
