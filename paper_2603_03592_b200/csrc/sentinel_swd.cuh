@@ -505,7 +505,12 @@ swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int 
   while (npad < T) npad <<= 1;
   const size_t first = (size_t)list * rows + (size_t)b * T_sample + (size_t)piece * T;
   const float *src = proj + first;
-  for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) s_val[i] = i < T ? src[i] : CUDART_INF_F;
+  // a projection that is not a number is sorted, merged and matched as +inf: the comparisons and
+  // min / max of the later steps then see ordered values only, and the sample's W1 comes out not finite
+  for (int i = threadIdx.x; i < npad; i += kSwdSortThreads) {
+    const float v = i < T ? src[i] : CUDART_INF_F;
+    s_val[i] = v == v ? v : CUDART_INF_F;
+  }
   __syncthreads();
   // runs of 2, 4 and 8: all inside a thread's 8 consecutive entries, the direction per pair
   for (int t = threadIdx.x; t < (npad >> 3); t += kSwdSortThreads) {
@@ -711,9 +716,8 @@ swd_w1_kernel(const float *sorted, const float *runs, long long run_len, double 
     if (lane == 0) s_w1[pair] = (float)(w1 / n);
   }
   __syncthreads();
-  // a sample with an entry that is not finite has a W1 that is not finite; the merges above may have
-  // dropped such an entry (min / max of a number and a NaN is the number), so the whole tensor's
-  // W1 is declared not a number along with it
+  // a sample with an entry that is not finite has a W1 that is not finite (inf, or inf - inf); the
+  // whole tensor's W1 is declared not a number along with it, whatever the merged lists gave
   for (int r = threadIdx.x; r <= B; r += kSwdW1Threads) {
     double mean = 0.;
     for (int dir = 0; dir < L; ++dir) mean += (double)s_w1[r * L + dir];
