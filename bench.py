@@ -39,7 +39,7 @@ FOUR_METRIC_BYTES = 12          # a verified tensor with the sliced Wasserstein 
 # ncu capture summarised in profiles/all_kernels_cfg3_ncu.md (B=8 x 4096 x 4096; traffic
 # grows in proportion to the element count, so a launch of N elements moves this times N).
 # Set to None whenever the kernel changes until the capture is retaken.
-NCU_DRAM_BYTES_PER_ELEMENT = 9.677
+NCU_DRAM_BYTES_PER_ELEMENT = 9.672
 
 
 def measured_peak_gbs():
