@@ -22,9 +22,13 @@ def sb():
     return binding
 
 
-def run_steps(sb, oracle_mod, w, kind, n_warm, corruption, **variant):
+def run_steps(sb, oracle_mod, w, kind, n_warm, corruption, directions=0, **variant):
     gv = sb.Verifier(w.B, w.T, w.d, **variant)
     ov = oracle_mod.Verifier(oracle_mod.Params(B=w.B, T=w.T, d=w.d, **variant))
+    if directions:                                          # the sliced Wasserstein distance as a fourth metric
+        u = synth.directions(directions, w.d, 7, "cuda")
+        gv.sentinel_set_directions(u)
+        ov.set_directions(synth.bits(u))
     for t in range(n_warm):
         x = synth.clean(w, 0, kind, t, "cuda")
         gs = gv.update_reference(x, kind)
@@ -215,6 +219,13 @@ def test_cfg4_channel_reference_against_the_oracle(sb, oracle_mod):
 def test_cfg4_channel_reference_per_sample_against_the_oracle(sb, oracle_mod):
     """The same with a vector per sample ([B,d])."""
     run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], GRAD, 2, "add_uniform_sample", ref_over_tokens=1)
+
+
+def test_cfg4_steps_with_four_metrics_against_the_oracle(sb, oracle_mod):
+    """4 x 8192 x 8192 with 8 directions as the verifier's fourth metric: two warm-up steps (the second
+    one takes the reference's projections from the recursion), a clean verified step and one with
+    uniform noise on a sample -- all four scores of every unit, flags and counters."""
+    run_steps(sb, oracle_mod, synth.WORKLOADS["cfg4"], ACT, 2, "add_uniform_sample", directions=8)
 
 
 def test_cfg4_sliced_wasserstein_units(sb, oracle_mod):
