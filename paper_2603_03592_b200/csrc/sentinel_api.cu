@@ -506,8 +506,11 @@ cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_
   e = cudaFuncSetAttribute(swd_sort_samples_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSwdMaxTokensPerSample * (int)sizeof(float));
   if (e != cudaSuccess) return e;
+  SwdExtents ext;                                  // (from the layout of the scratch, not from the kernels' own arithmetic)
+  ext.list_floats = (long long)(sorted - proj);
+  ext.partial_doubles = (long long)(reinterpret_cast<double *>(ticket) - partial);
   e = launch_chained(swd_sort_samples_kernel, 2u * L * B * pieces, kSwdSortThreads, smem, s, proj, sorted, ticket, B, T, pieces, L,
-                     rows, skip);
+                     rows, skip, ext);
   if (e != cudaSuccess) return e;
   const long long span_tasks = (rows + kSwdMergeSpan - 1) / kSwdMergeSpan * 2 * L;
   const unsigned merge_grid = (unsigned)((span_tasks + kSwdW1Threads - 1) / kSwdW1Threads);
@@ -516,7 +519,7 @@ cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_
   const float *samples = sorted;
   float *free_a = spare, *free_b = proj;
   if (pieces == 2) {
-    e = launch_chained(swd_merge_kernel, merge_grid, kSwdW1Threads, 0, s, sorted, spare, rows, (long long)(T / 2), 2 * L, skip);
+    e = launch_chained(swd_merge_kernel, merge_grid, kSwdW1Threads, 0, s, sorted, spare, rows, (long long)(T / 2), 2 * L, skip, ext);
     if (e != cudaSuccess) return e;
     samples = spare;
     free_a = proj;
@@ -525,14 +528,14 @@ cudaError_t run_swd(const uint16_t *x, const void *m0, const void *m1, bool ref_
   const float *runs = samples;
   long long run_len = T;
   while (2 * run_len < rows) {
-    e = launch_chained(swd_merge_kernel, merge_grid, kSwdW1Threads, 0, s, runs, free_a, rows, run_len, 2 * L, skip);
+    e = launch_chained(swd_merge_kernel, merge_grid, kSwdW1Threads, 0, s, runs, free_a, rows, run_len, 2 * L, skip, ext);
     if (e != cudaSuccess) return e;
     runs = free_a;
     float *t = free_a; free_a = free_b; free_b = t;
     run_len *= 2;
   }
   const unsigned grid = (unsigned)((B > 1 ? L * swd_w1_chunks(rows) : 0) + L * B * swd_w1_chunks(T));
-  return launch_chained(swd_w1_kernel, grid, kSwdW1Threads, 0, s, samples, runs, run_len, partial, ticket, out, B, T, L, rows, skip);
+  return launch_chained(swd_w1_kernel, grid, kSwdW1Threads, 0, s, samples, runs, run_len, partial, ticket, out, B, T, L, rows, skip, ext);
 }
 
 // A verifier with directions: the distances of this submission against the reference in force,

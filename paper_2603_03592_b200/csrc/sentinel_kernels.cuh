@@ -136,7 +136,7 @@ struct StreamArgs {
 // kErrBounds into HandleState.error.  In the normal build the checks compile to nothing.
 constexpr int kErrBounds = 2;                     // HandleState.error: an index left its buffer (checked build)
 enum Site : int { kSiteX = 1, kSiteRefIn, kSiteRefOut, kSiteToken, kSiteSlot, kSiteRing, kSiteSorted, kSiteOut,
-                  kSiteStageX, kSiteStageRef, kSiteColumns, kSiteReplace };
+                  kSiteStageX, kSiteStageRef, kSiteColumns, kSiteReplace, kSiteSwdLists, kSiteSwdPartial };
 #ifdef SENTINEL_CHECK_BOUNDS
 __device__ unsigned long long g_bounds_violations = 0ull;
 __device__ int g_bounds_first_site = 0;

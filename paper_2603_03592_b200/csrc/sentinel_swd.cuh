@@ -22,6 +22,12 @@ __device__ __forceinline__ void chain_entry() {
 }
 constexpr int kSwdMaxTokensPerSample = 16384;    // one sample's projections are sorted in shared memory
 
+// extents, for the checked build, of what the sort / merge / W1 launches index: floats of one buffer
+// of lists (projections, sorted lists, merge buffer: 2L lists of B*T each) and doubles of the per-CTA sums
+struct SwdExtents {
+  long long list_floats, partial_doubles;
+};
+
 // ---------------------------------------------------------------------------------------------
 // projections: proj[(t*L + l)*rows + row] = sum_c v[row][c] * u[l][c], t = 0 for x, 1 for m.
 // A warp owns whole rows; the directions sit in shared memory as bf16 (they are given as bf16).
@@ -493,7 +499,7 @@ __device__ __forceinline__ void bitonic_round(float *s_val, int npad, int k2, in
 // together.  Also clears the ticket word of swd_w1_kernel, a later launch of the chain.
 __global__ void __launch_bounds__(kSwdSortThreads)
 swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int B, int T_sample, int pieces, int L,
-                        long long rows, const int *skip) {
+                        long long rows, const int *skip, const SwdExtents ext) {
   extern __shared__ float s_val[];                // [npad]
   chain_entry();
   if (skip && __ldcg(skip)) return;
@@ -504,6 +510,7 @@ swd_sort_samples_kernel(const float *proj, float *sorted, unsigned *ticket, int 
   int npad = 8;
   while (npad < T) npad <<= 1;
   const size_t first = (size_t)list * rows + (size_t)b * T_sample + (size_t)piece * T;
+  if (!SENTINEL_BOUNDS(kSiteSwdLists, first, T, ext.list_floats)) return;      // (the whole CTA: the list is read and written as one)
   const float *src = proj + first;
   // a projection that is not a number is sorted, merged and matched as +inf: the comparisons and
   // min / max of the later steps then see ordered values only, and the sample's W1 comes out not finite
@@ -616,7 +623,8 @@ __device__ __forceinline__ int merge_pair(const float *list, long long rows, lon
 
 // one round that is not the last: runs of run_len entries become runs of twice that
 __global__ void __launch_bounds__(kSwdW1Threads)
-swd_merge_kernel(const float *in, float *out, long long rows, long long run_len, int lists, const int *skip) {
+swd_merge_kernel(const float *in, float *out, long long rows, long long run_len, int lists, const int *skip,
+                 const SwdExtents ext) {
   chain_entry();
   if (skip && __ldcg(skip)) return;
   const long long spans = (rows + kSwdMergeSpan - 1) / kSwdMergeSpan;
@@ -628,6 +636,10 @@ swd_merge_kernel(const float *in, float *out, long long rows, long long run_len,
   // (a span may straddle two pairs only if 2 * run_len is not a multiple of the span: run_len is a multiple of T, any T,
   // so the entries past the end of this pair are produced one by one below)
   const int d = merge_pair(in + list * rows, rows, run_len, at, left, la, right, lb);
+  // the pair's two runs and this thread's outputs lie inside the list, the list inside the buffer
+  if (!SENTINEL_BOUNDS(kSiteSwdLists, left - in, la + lb, ext.list_floats) ||
+      !SENTINEL_BOUNDS(kSiteSwdLists, list * rows + at, (rows - at < kSwdMergeSpan ? rows - at : kSwdMergeSpan), ext.list_floats))
+    return;
   float v[kSwdMergeSpan];
   merge_span(left, la, right, lb, d, v);
   float *dst = out + list * rows + at;
@@ -657,7 +669,7 @@ __host__ __device__ inline size_t swd_w1_partials(int L, int B, int T) {
 // (runs of run_len entries; == sorted if there was no earlier round; unused if B == 1)
 __global__ void __launch_bounds__(kSwdW1Threads)
 swd_w1_kernel(const float *sorted, const float *runs, long long run_len, double *partial, unsigned *ticket, float *out, int B,
-              int T, int L, long long rows, const int *skip) {
+              int T, int L, long long rows, const int *skip, const SwdExtents ext) {
   __shared__ double s_red[kSwdW1Threads / 32];
   __shared__ float s_w1[(kMaxB + 1) * 16];        // W1 per (unit, direction), L <= 16
   __shared__ bool s_last;
@@ -669,7 +681,7 @@ swd_w1_kernel(const float *sorted, const float *runs, long long run_len, double 
   if ((int)blockIdx.x < n_tensor) {               // a span of the last merge round, both clouds
     const int l = blockIdx.x / tensor_chunks, chunk = blockIdx.x - l * tensor_chunks;
     const long long at = ((long long)chunk * kSwdW1Threads + threadIdx.x) * kSwdMergeSpan;
-    if (at < rows) {
+    if (at < rows && SENTINEL_BOUNDS(kSiteSwdLists, ((size_t)L + l) * rows, rows, ext.list_floats)) {   // (both clouds' lists of direction l)
       float va[kSwdMergeSpan], vb[kSwdMergeSpan];
       const float *left, *right;
       int la, lb;
@@ -686,13 +698,14 @@ swd_w1_kernel(const float *sorted, const float *runs, long long run_len, double 
     const int l = unit / B, b = unit - l * B;
     const float *sa = sorted + (size_t)l * rows + (size_t)b * T, *sb = sorted + ((size_t)L + l) * rows + (size_t)b * T;
     const int at = (chunk * kSwdW1Threads + threadIdx.x) * kSwdMergeSpan;
+    const bool inside = SENTINEL_BOUNDS(kSiteSwdLists, ((size_t)L + l) * rows + (size_t)b * T, T, ext.list_floats);
 #pragma unroll
     for (int k = 0; k < kSwdMergeSpan; ++k)
-      if (at + k < T) term += (double)fabsf(sa[at + k] - sb[at + k]);
+      if (inside && at + k < T) term += (double)fabsf(sa[at + k] - sb[at + k]);
   }
   const double sum = block_sum_ordered(term, s_red);
   if (threadIdx.x == 0) {
-    partial[blockIdx.x] = sum;
+    if (SENTINEL_BOUNDS(kSiteSwdPartial, blockIdx.x, 1, ext.partial_doubles)) partial[blockIdx.x] = sum;
     __threadfence();
     s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
   }

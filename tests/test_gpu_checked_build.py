@@ -161,3 +161,39 @@ def test_iterations_with_several_workers(builds, shape, R):
         return res
 
     same(*on_both(binding, checked, run))
+
+
+SWD_SHAPES = [((1, 1, 8), 4), ((3, 37, 520), 8), ((5, 100, 1024), 16), ((2, 1536, 264), 8), ((1, 2048, 136), 8),
+              ((5, 1030, 40), 4), ((2, 1025, 64), 4)]
+
+
+def test_sliced_wasserstein_sort_merge_and_w1_launches(builds):
+    """The launches that follow the projections (sort per sample, whole and in halves; merge rounds with
+    odd sample counts and token counts that are no multiple of the span; the last round with the
+    W1 sums): stateless calls over ragged shapes, and a verifier with directions over a short stream."""
+    binding, checked = builds
+
+    def run(sb):
+        res = []
+        for (B, T, d), L in SWD_SHAPES:
+            g = torch.Generator(device="cuda").manual_seed(B * 5 + T * 3 + d)
+            x = (torch.randn(B, T, d, generator=g, device="cuda") * 1.1).to(torch.bfloat16)
+            m = torch.randn(B, T, d, generator=g, device="cuda")
+            out = torch.empty(1 + B, device="cuda")
+            sb.sentinel_sliced_wasserstein(x, m, synth.directions(L, d, 3, "cuda"), out)
+            res.append(out.cpu().numpy())
+        w = synth.scaled(synth.WORKLOADS["cfg2"], "checked_swd", 3, 40, 264)
+        gv = sb.Verifier(w.B, w.T, w.d, window_steps=4)
+        gv.sentinel_set_directions(synth.directions(8, w.d, 1, "cuda"))
+        for t in range(9):
+            x = synth.clean(w, 0, ACT, t, "cuda")
+            if t < 4:
+                res.append(gv.update_reference(x, ACT).cpu().numpy())
+            else:
+                gs, gf = gv.verify(x, ACT)
+                res += [gs.cpu().numpy(), gf.cpu().numpy()]
+        assert gv.sentinel_get_counters()["error"] == 0
+        gv.close()
+        return res
+
+    same(*on_both(binding, checked, run))
